@@ -1,0 +1,129 @@
+"""Python face of the CPU checker in ``lr_oracle.c`` (float64, plain loops).
+
+TEST INFRASTRUCTURE ONLY: imported by the tests, the smoke check and the benchmark's CPU-baseline
+leg.  The product (CUDA) path never imports this package and this package never imports the
+product.  The C file's header lists what each routine follows in the paper and how it is pinned.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "lr_oracle.c")
+_SO = os.path.join(_HERE, "liblr_oracle.so")
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile ``lr_oracle.c`` with gcc (-O2, OpenMP, no fast-math) if the shared object is stale."""
+    if force or not os.path.exists(_SO) or os.path.getmtime(_SO) < os.path.getmtime(_SRC):
+        tmp = _SO + f".tmp{os.getpid()}"
+        subprocess.check_call(["gcc", "-O2", "-fopenmp", "-fPIC", "-shared", "-std=c11",
+                               "-fno-fast-math", "-ffp-contract=off", "-o", tmp, _SRC, "-lm"])
+        os.replace(tmp, _SO)
+    return _SO
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        lib = ctypes.CDLL(build())
+        P, I64, I32, D = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int32, ctypes.c_double
+        lib.oracle_threads.restype = ctypes.c_int
+        lib.oracle_set_threads.argtypes = [ctypes.c_int]
+        lib.oracle_loss_grad.argtypes = [P, P, I64, I32, P, D, P, P, P]
+        lib.oracle_fit.argtypes = [P, P, I64, I32, D, I32, P, P, P, P, P, ctypes.c_int]
+        lib.oracle_predict.argtypes = [P, I64, I32, P, D, D, P, P]
+        lib.oracle_f1.argtypes = [P, P, I64, P, P, P, P]
+        _lib = lib
+    return _lib
+
+
+def _f32(a, shape=None):
+    a = np.ascontiguousarray(a, dtype=np.float32)
+    if shape is not None:
+        assert a.shape == shape, (a.shape, shape)
+    return a
+
+
+def _ptr(a):
+    return a.ctypes.data_as(ctypes.c_void_p) if a is not None else None
+
+
+def threads() -> int:
+    return int(_load().oracle_threads())
+
+
+def set_threads(t: int) -> None:
+    _load().oracle_set_threads(int(t))
+
+
+def loss_grad(X, y, w, b):
+    """(loss, grad_w[n], grad_b) in float64 at parameters (w, b); X, y are fp32 arrays."""
+    X = _f32(X)
+    m, n = X.shape
+    y = _f32(y, (m,))
+    w = np.ascontiguousarray(w, dtype=np.float64)
+    assert w.shape == (n,)
+    loss, gb = np.zeros(1), np.zeros(1)
+    gw = np.zeros(n)
+    rc = _load().oracle_loss_grad(_ptr(X), _ptr(y), m, n, _ptr(w), float(b), _ptr(loss), _ptr(gw), _ptr(gb))
+    if rc != 0:
+        raise ValueError("oracle_loss_grad: bad arguments")
+    return float(loss[0]), gw, float(gb[0])
+
+
+def fit(X, y, lr, iters, w0=None, b0=0.0, history=False, round_to_fp32=False):
+    """Run ``iters`` full-batch GD steps from (w0, b0) (zeros by default).
+
+    Returns ``(w, b, loss_hist)``; with ``history=True`` also ``w_hist[(iters+1), n]`` and
+    ``b_hist[iters+1]``.  ``loss_hist[t]`` is the loss before update t.
+    """
+    X = _f32(X)
+    m, n = X.shape
+    y = _f32(y, (m,))
+    w = np.zeros(n) if w0 is None else np.array(w0, dtype=np.float64).copy()
+    assert w.shape == (n,)
+    b = np.array([float(b0)])
+    lh = np.zeros(max(iters, 1))
+    wh = np.zeros((iters + 1, n)) if history else None
+    bh = np.zeros(iters + 1) if history else None
+    rc = _load().oracle_fit(_ptr(X), _ptr(y), m, n, float(lr), int(iters), _ptr(w), _ptr(b), _ptr(lh),
+                            _ptr(wh), _ptr(bh), int(bool(round_to_fp32)))
+    if rc != 0:
+        raise ValueError("oracle_fit: bad arguments")
+    lh = lh[:iters]
+    if history:
+        return w, float(b[0]), lh, wh, bh
+    return w, float(b[0]), lh
+
+
+def predict(X, w, b, thr, return_z=False):
+    """uint8 labels[m]: 1 iff sigmoid(x.w + b) >= thr (decided as z >= logit(thr))."""
+    X = _f32(X)
+    m, n = X.shape
+    w = np.ascontiguousarray(w, dtype=np.float64)
+    assert w.shape == (n,)
+    labels = np.zeros(m, dtype=np.uint8)
+    z = np.zeros(m) if return_z else None
+    rc = _load().oracle_predict(_ptr(X), m, n, _ptr(w), float(b), float(thr), _ptr(labels), _ptr(z))
+    if rc != 0:
+        raise ValueError("oracle_predict: bad arguments")
+    return (labels, z) if return_z else labels
+
+
+def f1_score(labels, y):
+    """(f1, tp, fp, fn) of uint8 labels against fp32 0/1 targets."""
+    labels = np.ascontiguousarray(labels, dtype=np.uint8)
+    y = _f32(y, labels.shape)
+    tp, fp, fn = ctypes.c_int64(), ctypes.c_int64(), ctypes.c_int64()
+    f1 = ctypes.c_double()
+    rc = _load().oracle_f1(_ptr(labels), _ptr(y), labels.shape[0], ctypes.byref(tp), ctypes.byref(fp),
+                           ctypes.byref(fn), ctypes.byref(f1))
+    if rc != 0:
+        raise ValueError("oracle_f1: bad arguments")
+    return f1.value, tp.value, fp.value, fn.value

@@ -1,0 +1,170 @@
+/*
+ * CPU checker ("oracle") for full-batch gradient-descent logistic regression.
+ *
+ * TEST INFRASTRUCTURE ONLY.  This file is the slow, plain float64 statement of what the GPU
+ * library must compute.  It shares no code, header, table or helper with the CUDA path and is
+ * called only from the tests, the smoke check and the benchmark's CPU-baseline leg.
+ *
+ * What it follows (paper: "High Performance Computing Applied to Logistic Regression"):
+ *   - model            p(y=1|x) = 1/(1+exp(-w.x-b))                    Section II-A, model equation
+ *   - sigmoid          1/(1+e^-x)                                      Eq. 1
+ *   - log-likelihood   l(w,b) = sum_i y_i log p_i + (1-y_i) log(1-p_i) Section II-A
+ *   - gradient step    grad = (1/m) err.X ; W = W - alpha*grad         Algorithm 1 (sequential version)
+ *   - error sign       res <- sigmoid(res) - Y, then w <- w - alpha*grad  Algorithm 7 with Algorithm 5
+ *
+ * Readings taken where the paper is silent or inconsistent:
+ *   - "Loss" is never defined; it is taken as the mean negative log-likelihood, loss = -l/m,
+ *     matching the 1/m of Algorithm 1.
+ *   - Algorithm 1 writes error = Y - y_pred and still subtracts alpha*grad (which would ascend);
+ *     Algorithm 7 computes y_pred - Y.  The descent reading err = p - y is used.
+ *   - The model has a bias b but Algorithms 1/7 carry only W; b is kept as an explicit scalar
+ *     with grad_b = (1/m) sum_i err_i and the same learning rate.
+ *   - Algorithm 7 drops the 1/m; it is kept (Algorithm 1).
+ *   - Prediction threshold: the caller's thr; label = 1 iff p >= thr, decided as z >= log(thr/(1-thr)).
+ *   - F1 with no true positives is 0.
+ *
+ * Arithmetic: X and y arrive as fp32 bits and are promoted element by element; everything else is
+ * double.  Per-row loss is evaluated as max(z,0) + log1p(exp(-|z|)) - y*z, which equals
+ * -[y log p + (1-y) log(1-p)] for y in {0,1} and stays finite for large |z|.
+ * Rows are summed in index order inside fixed blocks of ORACLE_BLOCK_ROWS rows and the block sums
+ * are added in block order, so the result does not depend on the thread count.
+ *
+ * Pins (tests, CPU only): ln 2 at w=b=0, X^T(0.5-y)/m at w=b=0, closed-form one- and two-row cases,
+ * central finite differences, label-flip symmetry, row duplication, ones-column/bias equivalence,
+ * saturation at |z|=40, descent-lemma monotonicity, planted-w* recovery, float64 autograd of a
+ * library BCE-with-logits, brute-force predict and hand-counted F1.  No function here is unpinned.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+#define ORACLE_BLOCK_ROWS 1024
+
+int oracle_threads(void) {
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
+
+void oracle_set_threads(int t) {
+#ifdef _OPENMP
+    if (t > 0) omp_set_num_threads(t);
+#else
+    (void)t;
+#endif
+}
+
+/* z_i = b + sum_j X[i][j] w[j]   (Section II-A model equation; Algorithm 1, y_pred = sigmoid(W X^T)) */
+static double row_logit(const float* xi, int32_t n, const double* w, double b) {
+    double z = b;
+    for (int32_t j = 0; j < n; ++j) z += (double)xi[j] * w[j];
+    return z;
+}
+
+/* sums over rows [r0, r1): s[0..n) = sum x_ij e_i ; s[n] = sum e_i ; s[n+1] = sum L_i */
+static void block_sums(const float* X, const float* y, int64_t r0, int64_t r1, int32_t n,
+                       const double* w, double b, double* s) {
+    for (int32_t j = 0; j < n + 2; ++j) s[j] = 0.0;
+    for (int64_t i = r0; i < r1; ++i) {
+        const float* xi = X + i * (int64_t)n;
+        double z = row_logit(xi, n, w, b);
+        double p = 1.0 / (1.0 + exp(-z));                                   /* Eq. 1 */
+        double yi = (double)y[i];
+        double e = p - yi;                                                  /* Algorithm 7 with Algorithm 5 */
+        double L = fmax(z, 0.0) + log1p(exp(-fabs(z))) - yi * z;            /* -log-likelihood term */
+        for (int32_t j = 0; j < n; ++j) s[j] += (double)xi[j] * e;          /* err.X, Algorithm 1 */
+        s[n] += e;
+        s[n + 1] += L;
+    }
+}
+
+/* loss = -l/m ; grad_w = X^T err / m ; grad_b = sum err / m.  Returns 0, or -1 on bad arguments / no memory. */
+int oracle_loss_grad(const float* X, const float* y, int64_t m, int32_t n, const double* w, double b,
+                     double* loss, double* grad_w, double* grad_b) {
+    if (!X || !y || !w || !loss || !grad_w || !grad_b || m < 1 || n < 1) return -1;
+    int64_t nblocks = (m + ORACLE_BLOCK_ROWS - 1) / ORACLE_BLOCK_ROWS;
+    size_t stride = (size_t)n + 2;
+    double* part = (double*)malloc(sizeof(double) * stride * (size_t)nblocks);
+    if (!part) return -1;
+#pragma omp parallel for schedule(static)
+    for (int64_t k = 0; k < nblocks; ++k) {
+        int64_t r0 = k * ORACLE_BLOCK_ROWS;
+        int64_t r1 = r0 + ORACLE_BLOCK_ROWS < m ? r0 + ORACLE_BLOCK_ROWS : m;
+        block_sums(X, y, r0, r1, n, w, b, part + (size_t)k * stride);
+    }
+    double inv_m = 1.0 / (double)m;
+    for (int32_t j = 0; j < n + 2; ++j) {
+        double s = 0.0;
+        for (int64_t k = 0; k < nblocks; ++k) s += part[(size_t)k * stride + j];
+        if (j < n) grad_w[j] = s * inv_m;
+        else if (j == n) *grad_b = s * inv_m;
+        else *loss = s * inv_m;
+    }
+    free(part);
+    return 0;
+}
+
+/*
+ * iters steps of  w <- w - lr*grad_w, b <- b - lr*grad_b  (Algorithm 1 update; Algorithm 7 sign).
+ * w[n], b[1] in/out.  loss_hist[iters] (nullable) receives the loss at the parameters BEFORE each update.
+ * w_hist[(iters+1)*n], b_hist[iters+1] (nullable) receive the whole trajectory including the start.
+ * round_to_fp32 != 0 rounds w and b to fp32 after every update (sensitivity study only).
+ */
+int oracle_fit(const float* X, const float* y, int64_t m, int32_t n, double lr, int32_t iters,
+               double* w, double* b, double* loss_hist, double* w_hist, double* b_hist, int round_to_fp32) {
+    if (!X || !y || !w || !b || m < 1 || n < 1 || iters < 0) return -1;
+    double* g = (double*)malloc(sizeof(double) * (size_t)n);
+    if (!g) return -1;
+    if (w_hist) memcpy(w_hist, w, sizeof(double) * (size_t)n);
+    if (b_hist) b_hist[0] = *b;
+    for (int32_t t = 0; t < iters; ++t) {
+        double loss, gb;
+        if (oracle_loss_grad(X, y, m, n, w, *b, &loss, g, &gb) != 0) { free(g); return -1; }
+        if (loss_hist) loss_hist[t] = loss;
+        for (int32_t j = 0; j < n; ++j) w[j] -= lr * g[j];
+        *b -= lr * gb;
+        if (round_to_fp32) {
+            for (int32_t j = 0; j < n; ++j) w[j] = (double)(float)w[j];
+            *b = (double)(float)*b;
+        }
+        if (w_hist) memcpy(w_hist + (size_t)(t + 1) * n, w, sizeof(double) * (size_t)n);
+        if (b_hist) b_hist[t + 1] = *b;
+    }
+    free(g);
+    return 0;
+}
+
+/* label_i = 1 iff p_i >= thr, decided in logit space: z_i >= log(thr/(1-thr)).  z_out (nullable) gets z. */
+int oracle_predict(const float* X, int64_t m, int32_t n, const double* w, double b, double thr,
+                   uint8_t* labels, double* z_out) {
+    if (!X || !w || !labels || m < 1 || n < 1 || !(thr > 0.0 && thr < 1.0)) return -1;
+    double cut = log(thr / (1.0 - thr));
+#pragma omp parallel for schedule(static)
+    for (int64_t i = 0; i < m; ++i) {
+        double z = row_logit(X + i * (int64_t)n, n, w, b);
+        labels[i] = (uint8_t)(z >= cut ? 1 : 0);
+        if (z_out) z_out[i] = z;
+    }
+    return 0;
+}
+
+/* Confusion counts of labels against y (y > 0.5 is positive) and F1 = 2TP/(2TP+FP+FN), 0 when TP = 0. */
+int oracle_f1(const uint8_t* labels, const float* y, int64_t m, int64_t* tp, int64_t* fp, int64_t* fn, double* f1) {
+    if (!labels || !y || m < 0 || !tp || !fp || !fn || !f1) return -1;
+    int64_t a = 0, c = 0, d = 0;
+    for (int64_t i = 0; i < m; ++i) {
+        int pos = y[i] > 0.5f, pred = labels[i] != 0;
+        a += (pred && pos);
+        c += (pred && !pos);
+        d += (!pred && pos);
+    }
+    *tp = a; *fp = c; *fn = d;
+    *f1 = a > 0 ? (2.0 * (double)a) / (2.0 * (double)a + (double)c + (double)d) : 0.0;
+    return 0;
+}
