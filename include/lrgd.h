@@ -1,0 +1,145 @@
+/*
+ * lrgd -- full-batch gradient-descent logistic regression on one NVIDIA B200 (sm_100a).
+ *
+ * C-ABI boundary.  Plain pointers and sizes only.  Pointers named d_* are DEVICE pointers and
+ * pointers named h_* are HOST pointers; both are owned by the caller.  The library never frees or
+ * reallocates caller memory; it owns only the workspace inside an lr_ctx.
+ *
+ * Data layout: X is fp32, row-major, m rows by n columns with leading dimension n (row i starts at
+ * X + i*n); y is fp32 with values 0.0f or 1.0f; w is fp32[n]; b is one fp32.  All arithmetic on the
+ * m*n stream is fp32; the cross-block reduction is carried in fp64.
+ *
+ * What is computed (paper: "High Performance Computing Applied to Logistic Regression"):
+ *   z_i = x_i.w + b, p_i = 1/(1+exp(-z_i))                 model equation of Section II-A, Eq. 1
+ *   err_i = p_i - y_i                                      Algorithm 7 (sigmoid, then Substract(Y, res))
+ *   loss = -(1/m) sum_i [y_i log p_i + (1-y_i) log(1-p_i)] mean negative log-likelihood, Section II-A
+ *   grad_w = X^T err / m, grad_b = sum err / m             Algorithm 1 (the 1/m err.X line)
+ *   w <- w - lr*grad_w, b <- b - lr*grad_b                 Algorithm 1 update, Algorithm 7 sign
+ *
+ * Streams: every device-pointer call enqueues its kernels on `stream` (a cudaStream_t passed as
+ * void*, NULL = the legacy default stream) and returns without synchronising; outputs are valid once
+ * the caller has synchronised that stream.  One lr_ctx must not be used from two streams at once.
+ *
+ * Errors: every call returns LR_OK (0) or a negative LR_ERR_* code; nothing is launched when
+ * argument validation fails.  A wait inside a kernel that exceeds its bound makes the kernel finish
+ * early and set a device status word, read back with lr_last_device_status.
+ *
+ * There is no CPU fallback: without a usable CUDA device lr_create fails with LR_ERR_CUDA.
+ */
+#ifndef LRGD_H
+#define LRGD_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+    LR_OK = 0,
+    LR_ERR_NULL = -1,       /* a required pointer is NULL */
+    LR_ERR_SHAPE = -2,      /* m < 1, n < 1, n > n_max of the ctx, iters < 0, m too large */
+    LR_ERR_ALIGNMENT = -3,  /* a float pointer is not 4-byte aligned */
+    LR_ERR_VALUE = -4,      /* thr outside (0,1), lr not finite */
+    LR_ERR_CUDA = -5,       /* a CUDA runtime call failed; see lr_last_cuda_error */
+    LR_ERR_TIMEOUT = -6,    /* a bounded device-side wait expired (reported by lr_last_device_status) */
+    LR_ERR_NOMEM = -7       /* host or device allocation failed */
+};
+
+typedef struct lr_ctx lr_ctx;
+
+/* Launch plan for a given shape, as chosen by the host logic (pure host code, no CUDA call). */
+typedef struct lr_plan {
+    int32_t variant;       /* 0 = row-per-lane-group staged kernel, 1 = row-split staged kernel, 2 = unstaged generic kernel */
+    int32_t lanes_per_row; /* staged kernels: lanes that share one row (8, 16, 32; 256 for the row-split kernel) */
+    int32_t vec_per_lane;  /* staged kernels: 16-byte column groups owned by one lane */
+    int32_t rows_per_batch;/* rows one warp (or one CTA for the row-split kernel) holds in registers at a time */
+    int32_t tile_rows;     /* rows per asynchronously staged tile */
+    int32_t stages;        /* tiles in flight per CTA */
+    int32_t grid;          /* CTAs */
+    int32_t threads;       /* threads per CTA */
+    int32_t smem_bytes;    /* dynamic shared memory per CTA */
+} lr_plan;
+
+/*
+ * Host-only: fills *out with the launch plan lr_loss_grad / lr_fit / lr_predict use for an m-by-n
+ * problem whose X pointer is 16-byte aligned (x_aligned16 != 0) or not, on a device with sm_count
+ * multiprocessors.  Makes no CUDA call.  Returns LR_ERR_NULL / LR_ERR_SHAPE on bad arguments.
+ */
+int lr_plan_query(int64_t m, int32_t n, int32_t x_aligned16, int32_t sm_count, lr_plan* out);
+
+/*
+ * Creates a context on CUDA device `device` with workspace for problems of up to n_max columns
+ * (any m).  Allocates the per-CTA partial-sum buffer and the device status word.
+ * Errors: LR_ERR_NULL (out), LR_ERR_SHAPE (n_max < 1), LR_ERR_CUDA, LR_ERR_NOMEM.
+ */
+int lr_create(lr_ctx** out, int32_t device, int32_t n_max);
+
+/* Frees the context's workspace (synchronises the device first).  NULL is accepted. */
+int lr_destroy(lr_ctx* ctx);
+
+/*
+ * One full-batch pass at fixed parameters (Section II-A loss; Algorithm 1 gradient):
+ *   d_loss[0] = loss, d_grad_w[0..n) = X^T err / m, d_grad_b[0] = sum err / m.
+ * Inputs d_X [m*n], d_y [m], d_w [n], d_b [1] are read only.  Two kernels are enqueued: the fused
+ * streaming kernel (reads X once) and the fixed-order cross-CTA reduction.
+ */
+int lr_loss_grad(lr_ctx* ctx, const float* d_X, const float* d_y, int64_t m, int32_t n,
+                 const float* d_w, const float* d_b,
+                 float* d_loss, float* d_grad_w, float* d_grad_b, void* stream);
+
+/*
+ * `iters` gradient-descent steps (Algorithm 1 update with Algorithm 7's sign), fixed count, no
+ * host synchronisation inside the loop.  d_w [n] and d_b [1] hold the start point on entry (the
+ * caller zeroes them for a cold start) and the result on exit.  d_loss_hist is NULL or [iters] and
+ * receives the loss at the parameters BEFORE update t.  iters == 0 is a no-op.
+ * Results are bit-reproducible for a given shape and device, and fit(a) followed by fit(b) equals
+ * fit(a+b) bit for bit.
+ */
+int lr_fit(lr_ctx* ctx, const float* d_X, const float* d_y, int64_t m, int32_t n,
+           float lr, int32_t iters, float* d_w, float* d_b, float* d_loss_hist, void* stream);
+
+/*
+ * d_labels[i] = 1 if sigmoid(x_i.w + b) >= thr else 0, decided in logit space as
+ * z_i >= log(thr/(1-thr)) evaluated in fp32 (the paper reports f1 but states no threshold; the
+ * caller supplies it).  0 < thr < 1.  d_labels is uint8 [m].
+ */
+int lr_predict(lr_ctx* ctx, const float* d_X, int64_t m, int32_t n,
+               const float* d_w, const float* d_b, float thr, uint8_t* d_labels, void* stream);
+
+/*
+ * Host-buffer variants: copy h_X, h_y (and h_w, h_b) to device buffers owned by the context
+ * (allocated or grown on first use), run the same kernels, copy the results back, and synchronise.
+ * h_w / h_b are in-out as for lr_fit; h_loss_hist is NULL or [iters]; h_labels is uint8 [m].
+ * Pinned host memory makes the copies faster but is not required.
+ */
+int lr_fit_host(lr_ctx* ctx, const float* h_X, const float* h_y, int64_t m, int32_t n,
+                float lr, int32_t iters, float* h_w, float* h_b, float* h_loss_hist);
+int lr_predict_host(lr_ctx* ctx, const float* h_X, int64_t m, int32_t n,
+                    const float* h_w, const float* h_b, float thr, uint8_t* h_labels);
+
+/*
+ * Per-kernel timing for measurement.  While enabled, lr_loss_grad / lr_fit / lr_predict bracket every
+ * launch of the streaming kernel with CUDA events on the caller's stream (up to 4096 launches since
+ * the last reset).  lr_profile_read synchronises those events and returns the number of bracketed
+ * launches and the sum of their durations in milliseconds, then clears the record.
+ */
+int lr_profile_enable(lr_ctx* ctx, int32_t on);
+int lr_profile_read(lr_ctx* ctx, int32_t* launches, double* total_ms);
+
+/* Number of kernels this context has launched since it was created. */
+int lr_launch_count(lr_ctx* ctx, int64_t* out);
+
+/* Synchronises the device and returns in *out the device status word: LR_OK or LR_ERR_TIMEOUT.  Clears it. */
+int lr_last_device_status(lr_ctx* ctx, int32_t* out);
+
+/* The cudaError_t value of the most recent failing CUDA call made through this context (0 if none). */
+int lr_last_cuda_error(lr_ctx* ctx);
+
+/* Static description of a status code. */
+const char* lr_status_string(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LRGD_H */

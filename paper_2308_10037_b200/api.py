@@ -1,0 +1,243 @@
+"""Thin ctypes binding over the C-ABI library ``liblrgd.so`` (declared in ``include/lrgd.h``).
+
+Argument marshalling only: every step of the computation runs in the CUDA kernels behind the C
+entry points.  PyTorch supplies device memory and the current stream.  Loading fails loudly when the
+library has not been built; there is no fallback of any kind.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import numpy as np
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "liblrgd.so")
+
+LR_OK = 0
+LR_ERR_NULL, LR_ERR_SHAPE, LR_ERR_ALIGNMENT, LR_ERR_VALUE, LR_ERR_CUDA, LR_ERR_TIMEOUT, LR_ERR_NOMEM = range(-1, -8, -1)
+
+EXPORTS = ["lr_plan_query", "lr_create", "lr_destroy", "lr_loss_grad", "lr_fit", "lr_predict", "lr_fit_host",
+           "lr_predict_host", "lr_profile_enable", "lr_profile_read", "lr_launch_count", "lr_last_device_status",
+           "lr_last_cuda_error", "lr_status_string"]
+
+
+class LrPlan(ctypes.Structure):
+    _fields_ = [(k, ctypes.c_int32) for k in ("variant", "lanes_per_row", "vec_per_lane", "rows_per_batch", "tile_rows",
+                                              "stages", "grid", "threads", "smem_bytes")]
+
+    def as_dict(self):
+        return {k: int(getattr(self, k)) for k, _ in self._fields_}
+
+
+class LrError(RuntimeError):
+    def __init__(self, code: int, where: str, detail: str = ""):
+        self.code = code
+        super().__init__(f"{where}: {status_string(code)} (code {code}){detail}")
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """The loaded C-ABI library.  Raises if it has not been built (run ``python -m paper_2308_10037_b200.build``)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2308_10037_b200.build` "
+                              "(nvcc, sm_100a).  There is no CPU fallback.")
+        L = ctypes.CDLL(LIB_PATH)
+        P, I64, I32, F = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int32, ctypes.c_float
+        L.lr_plan_query.argtypes = [I64, I32, I32, I32, ctypes.POINTER(LrPlan)]
+        L.lr_create.argtypes = [ctypes.POINTER(P), I32, I32]
+        L.lr_destroy.argtypes = [P]
+        L.lr_loss_grad.argtypes = [P, P, P, I64, I32, P, P, P, P, P, P]
+        L.lr_fit.argtypes = [P, P, P, I64, I32, F, I32, P, P, P, P]
+        L.lr_predict.argtypes = [P, P, I64, I32, P, P, F, P, P]
+        L.lr_fit_host.argtypes = [P, P, P, I64, I32, F, I32, P, P, P]
+        L.lr_predict_host.argtypes = [P, P, I64, I32, P, P, F, P]
+        L.lr_profile_enable.argtypes = [P, I32]
+        L.lr_profile_read.argtypes = [P, ctypes.POINTER(I32), ctypes.POINTER(ctypes.c_double)]
+        L.lr_launch_count.argtypes = [P, ctypes.POINTER(I64)]
+        L.lr_last_device_status.argtypes = [P, ctypes.POINTER(I32)]
+        L.lr_last_cuda_error.argtypes = [P]
+        L.lr_status_string.argtypes = [ctypes.c_int]
+        L.lr_status_string.restype = ctypes.c_char_p
+        for name in EXPORTS:
+            if name != "lr_status_string":
+                getattr(L, name).restype = ctypes.c_int
+        _lib = L
+    return _lib
+
+
+def status_string(code: int) -> str:
+    return lib().lr_status_string(int(code)).decode()
+
+
+def plan_query(m: int, n: int, x_aligned16: bool = True, sm_count: int = 148) -> dict:
+    """Host-only view of the launch plan for an m-by-n problem (no CUDA call)."""
+    p = LrPlan()
+    rc = lib().lr_plan_query(int(m), int(n), int(bool(x_aligned16)), int(sm_count), ctypes.byref(p))
+    if rc != LR_OK:
+        raise LrError(rc, "lr_plan_query")
+    return p.as_dict()
+
+
+def _dev_ptr(t: torch.Tensor | None, dtype, name: str):
+    if t is None:
+        return None
+    if not (isinstance(t, torch.Tensor) and t.is_cuda and t.dtype == dtype and t.is_contiguous()):
+        raise TypeError(f"{name}: expected a contiguous CUDA tensor of dtype {dtype}")
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def _host_ptr(a, dtype, name: str):
+    if a is None:
+        return None
+    if isinstance(a, torch.Tensor):
+        if a.is_cuda or not a.is_contiguous() or a.dtype != dtype:
+            raise TypeError(f"{name}: expected a contiguous CPU tensor of dtype {dtype}")
+        return ctypes.c_void_p(a.data_ptr())
+    npdt = {torch.float32: np.float32, torch.uint8: np.uint8}[dtype]
+    if not (isinstance(a, np.ndarray) and a.dtype == npdt and a.flags.c_contiguous):
+        raise TypeError(f"{name}: expected a C-contiguous numpy array of dtype {npdt}")
+    return ctypes.c_void_p(a.ctypes.data)
+
+
+class Context:
+    """Owns one ``lr_ctx``: workspace for problems of up to ``n_max`` columns on one device."""
+
+    def __init__(self, n_max: int = 4096, device: int | None = None):
+        self._h = ctypes.c_void_p()
+        self.device = torch.cuda.current_device() if device is None else int(device)
+        self.n_max = int(n_max)
+        rc = lib().lr_create(ctypes.byref(self._h), self.device, self.n_max)
+        if rc != LR_OK:
+            self._h = ctypes.c_void_p()
+            raise LrError(rc, "lr_create")
+
+    def close(self):
+        if getattr(self, "_h", None) is not None and self._h:
+            lib().lr_destroy(self._h)
+            self._h = ctypes.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def _check(self, rc: int, where: str):
+        if rc != LR_OK:
+            detail = f"; cudaError {lib().lr_last_cuda_error(self._h)}" if rc == LR_ERR_CUDA else ""
+            raise LrError(rc, where, detail)
+
+    def _stream(self):
+        return ctypes.c_void_p(torch.cuda.current_stream(self.device).cuda_stream)
+
+    # ---- device-pointer entry points -------------------------------------------------------------
+    def loss_grad(self, X, y, w, b):
+        m, n = X.shape
+        loss = torch.empty(1, dtype=torch.float32, device=X.device)
+        gw = torch.empty(n, dtype=torch.float32, device=X.device)
+        gb = torch.empty(1, dtype=torch.float32, device=X.device)
+        rc = lib().lr_loss_grad(self._h, _dev_ptr(X, torch.float32, "X"), _dev_ptr(y, torch.float32, "y"), m, n,
+                                _dev_ptr(w, torch.float32, "w"), _dev_ptr(b, torch.float32, "b"),
+                                _dev_ptr(loss, torch.float32, "loss"), _dev_ptr(gw, torch.float32, "grad_w"),
+                                _dev_ptr(gb, torch.float32, "grad_b"), self._stream())
+        self._check(rc, "lr_loss_grad")
+        return loss, gw, gb
+
+    def fit(self, X, y, lr, iters, w, b, loss_hist=None):
+        """In place on ``w`` [n] and ``b`` [1]; ``loss_hist`` is None or a float32 CUDA tensor [iters]."""
+        m, n = X.shape
+        rc = lib().lr_fit(self._h, _dev_ptr(X, torch.float32, "X"), _dev_ptr(y, torch.float32, "y"), m, n, float(lr),
+                          int(iters), _dev_ptr(w, torch.float32, "w"), _dev_ptr(b, torch.float32, "b"),
+                          _dev_ptr(loss_hist, torch.float32, "loss_hist"), self._stream())
+        self._check(rc, "lr_fit")
+
+    def predict(self, X, w, b, thr):
+        m, n = X.shape
+        labels = torch.empty(m, dtype=torch.uint8, device=X.device)
+        rc = lib().lr_predict(self._h, _dev_ptr(X, torch.float32, "X"), m, n, _dev_ptr(w, torch.float32, "w"),
+                              _dev_ptr(b, torch.float32, "b"), float(thr), _dev_ptr(labels, torch.uint8, "labels"),
+                              self._stream())
+        self._check(rc, "lr_predict")
+        return labels
+
+    # ---- host-pointer entry points ---------------------------------------------------------------
+    def fit_host(self, X, y, lr, iters, w, b, loss_hist=None):
+        """X, y, w, b (and loss_hist) are CPU tensors or numpy arrays; w, b are updated in place."""
+        m, n = X.shape
+        rc = lib().lr_fit_host(self._h, _host_ptr(X, torch.float32, "X"), _host_ptr(y, torch.float32, "y"), m, n,
+                               float(lr), int(iters), _host_ptr(w, torch.float32, "w"), _host_ptr(b, torch.float32, "b"),
+                               _host_ptr(loss_hist, torch.float32, "loss_hist"))
+        self._check(rc, "lr_fit_host")
+
+    def predict_host(self, X, w, b, thr, labels):
+        m, n = X.shape
+        rc = lib().lr_predict_host(self._h, _host_ptr(X, torch.float32, "X"), m, n, _host_ptr(w, torch.float32, "w"),
+                                   _host_ptr(b, torch.float32, "b"), float(thr), _host_ptr(labels, torch.uint8, "labels"))
+        self._check(rc, "lr_predict_host")
+
+    # ---- measurement / status --------------------------------------------------------------------
+    def profile_enable(self, on: bool = True):
+        self._check(lib().lr_profile_enable(self._h, int(bool(on))), "lr_profile_enable")
+
+    def profile_read(self):
+        n, ms = ctypes.c_int32(), ctypes.c_double()
+        self._check(lib().lr_profile_read(self._h, ctypes.byref(n), ctypes.byref(ms)), "lr_profile_read")
+        return n.value, ms.value
+
+    def launch_count(self) -> int:
+        v = ctypes.c_int64()
+        self._check(lib().lr_launch_count(self._h, ctypes.byref(v)), "lr_launch_count")
+        return v.value
+
+    def device_status(self) -> int:
+        v = ctypes.c_int32()
+        self._check(lib().lr_last_device_status(self._h, ctypes.byref(v)), "lr_last_device_status")
+        return v.value
+
+
+_default_ctx: dict[int, Context] = {}
+
+
+def _ctx_for(X: torch.Tensor, ctx: Context | None) -> Context:
+    if ctx is not None:
+        return ctx
+    dev = X.device.index if X.device.index is not None else torch.cuda.current_device()
+    n = int(X.shape[1])
+    c = _default_ctx.get(dev)
+    if c is None or c.n_max < n:
+        if c is not None:
+            c.close()
+        c = _default_ctx[dev] = Context(n_max=max(4096, n), device=dev)
+    return c
+
+
+def _as_b(b, device) -> torch.Tensor:
+    if isinstance(b, torch.Tensor):
+        return b.reshape(1)
+    return torch.tensor([float(b)], dtype=torch.float32, device=device)
+
+
+def lr_loss_grad(X, y, w, b, ctx: Context | None = None):
+    """(loss[1], grad_w[n], grad_b[1]) as float32 CUDA tensors at the parameters (w, b)."""
+    return _ctx_for(X, ctx).loss_grad(X, y, w, _as_b(b, X.device))
+
+
+def lr_fit(X, y, lr, iters, w0=None, b0=None, return_history=False, ctx: Context | None = None):
+    """``iters`` full-batch gradient-descent steps from (w0, b0) (zeros by default).  Returns (w, b[, loss_hist])."""
+    n = int(X.shape[1])
+    w = torch.zeros(n, dtype=torch.float32, device=X.device) if w0 is None else w0.detach().clone()
+    b = torch.zeros(1, dtype=torch.float32, device=X.device) if b0 is None else _as_b(b0, X.device).clone()
+    hist = torch.empty(int(iters), dtype=torch.float32, device=X.device) if return_history else None
+    _ctx_for(X, ctx).fit(X, y, lr, iters, w, b, hist)
+    return (w, b, hist) if return_history else (w, b)
+
+
+def lr_predict(X, w, b, thr, ctx: Context | None = None):
+    """uint8 CUDA tensor [m]: 1 where sigmoid(x.w + b) >= thr."""
+    return _ctx_for(X, ctx).predict(X, w, _as_b(b, X.device), thr)

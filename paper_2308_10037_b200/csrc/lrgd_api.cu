@@ -1,0 +1,453 @@
+// C-ABI layer: argument validation, launch planning, workspace, and the iteration loop.
+// The declarations and their contracts are in include/lrgd.h.
+#include "../../include/lrgd.h"
+
+#include <cmath>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "lrgd_generic.cuh"
+#include "lrgd_reduce.cuh"
+#include "lrgd_stream_rows.cuh"
+
+using namespace lrgd;
+
+namespace {
+
+constexpr int kNW = 15;                        // consumer warps of the staged kernel (+1 producer warp = 512 threads)
+constexpr int kStageTargetBytes = 32 * 1024;
+constexpr int kStageBudgetBytes = 200 * 1024;  // shared memory the stage ring may take (227 KB per CTA on sm_100)
+constexpr int kMaxGridPerSm = 8;               // widest launch any variant uses, in CTAs per SM
+constexpr int kMaxProfiled = 4096;
+constexpr int64_t kMaxRows = int64_t(1) << 40;
+
+struct RowShape { int nv, lpr, rb; };
+
+// Which instantiation of the staged kernel covers n4 = n/4 column groups per row.
+bool row_shape_for(int n4, RowShape* s) {
+    if (n4 <= 8) *s = {1, 8, 8};
+    else if (n4 <= 16) *s = {1, 16, 8};
+    else if (n4 <= 32) *s = {1, 32, 8};
+    else if (n4 <= 64) *s = {2, 32, 8};
+    else if (n4 <= 128) *s = {4, 32, 4};
+    else return false;
+    return true;
+}
+
+int make_plan(int64_t m, int32_t n, bool aligned16, int32_t sms, lr_plan* P) {
+    if (!P) return LR_ERR_NULL;
+    if (m < 1 || m > kMaxRows || n < 1 || sms < 1) return LR_ERR_SHAPE;
+    std::memset(P, 0, sizeof(*P));
+    RowShape rs;
+    if (aligned16 && n % 4 == 0 && row_shape_for(n / 4, &rs)) {
+        const int rpb = rs.rb * (32 / rs.lpr);
+        const int64_t row_bytes = int64_t(n) * 4;
+        const int64_t bpt_cap = std::max<int64_t>(1, kStageTargetBytes / (rpb * row_bytes));
+        const int64_t bpt_fill = (m + int64_t(sms) * rpb - 1) / (int64_t(sms) * rpb);   // spread small problems over all SMs
+        const int bpt = int(std::min(bpt_cap, std::max<int64_t>(1, bpt_fill)));
+        const int R = bpt * rpb;
+        const int64_t T = (m + R - 1) / R;
+        const int grid = int(std::min<int64_t>(T, sms));
+        const int64_t tiles_per_cta = (T + grid - 1) / grid;
+        const int64_t tile_stride = (R * row_bytes + 127) & ~int64_t(127);
+        const int64_t per_stage = tile_stride + int64_t(R) * 4;
+        int S = int(std::min<int64_t>(kMaxStages, kStageBudgetBytes / per_stage));
+        S = int(std::min<int64_t>(S, std::max<int64_t>(2, tiles_per_cta)));
+        if (S < 1) S = 1;
+        const int64_t combine = int64_t(kNW) * n * 8 + 2 * kNW * 8;
+        P->variant = 0;
+        P->lanes_per_row = rs.lpr;
+        P->vec_per_lane = rs.nv;
+        P->rows_per_batch = rpb;
+        P->tile_rows = R;
+        P->stages = S;
+        P->grid = grid;
+        P->threads = (kNW + 1) * 32;
+        P->smem_bytes = int(kHeaderBytes + std::max<int64_t>(S * per_stage, combine));
+        if (tiles_per_cta * bpt >= (int64_t(1) << 31)) return LR_ERR_SHAPE;
+        return LR_OK;
+    }
+    const int64_t nchunks = (m + kGenRows - 1) / kGenRows;
+    P->variant = 2;
+    P->lanes_per_row = 32;
+    P->vec_per_lane = 0;
+    P->rows_per_batch = 1;
+    P->tile_rows = kGenRows;
+    P->stages = 0;
+    P->grid = int(std::min<int64_t>(nchunks, int64_t(sms) * kMaxGridPerSm));
+    P->threads = kGenThreads;
+    P->smem_bytes = 0;
+    return LR_OK;
+}
+
+}  // namespace
+
+struct lr_ctx {
+    int device = 0;
+    int sm_count = 0;
+    int n_max = 0;
+    double* d_partial = nullptr;
+    int* d_status = nullptr;
+    // buffers of the host-pointer entry points (grown on demand)
+    void* d_hX = nullptr; size_t hX_bytes = 0;
+    void* d_hy = nullptr; size_t hy_bytes = 0;
+    void* d_hw = nullptr; size_t hw_bytes = 0;      // w[n] | b | loss_hist
+    void* d_hl = nullptr; size_t hl_bytes = 0;      // labels
+    cudaStream_t hstream = nullptr;
+    // profiling
+    bool prof = false;
+    std::vector<cudaEvent_t> ev;                    // pairs: start, stop
+    int prof_used = 0;
+    int64_t launches = 0;
+    int last_cuda = 0;
+};
+
+namespace {
+
+struct DeviceGuard {
+    int prev = -1;
+    bool ok = true;
+    explicit DeviceGuard(lr_ctx* c) {
+        if (cudaGetDevice(&prev) != cudaSuccess) { prev = -1; }
+        cudaError_t e = cudaSetDevice(c->device);
+        if (e != cudaSuccess) { c->last_cuda = int(e); ok = false; }
+    }
+    ~DeviceGuard() { if (prev >= 0) cudaSetDevice(prev); }
+};
+
+#define LR_CK(ctx, call)                                 \
+    do {                                                 \
+        cudaError_t e__ = (call);                        \
+        if (e__ != cudaSuccess) {                        \
+            (ctx)->last_cuda = int(e__);                 \
+            return LR_ERR_CUDA;                          \
+        }                                                \
+    } while (0)
+
+bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
+
+template <int NV, int LPR, int RB, bool PRED>
+cudaError_t launch_rows_t(const lr_plan& P, const StreamParams& sp, cudaStream_t st) {
+    auto kern = k_stream_rows<NV, LPR, RB, kNW, PRED>;
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, P.smem_bytes);
+    if (e != cudaSuccess) return e;
+    kern<<<P.grid, P.threads, P.smem_bytes, st>>>(sp);
+    return cudaGetLastError();
+}
+
+template <bool PRED>
+cudaError_t launch_rows(const lr_plan& P, const StreamParams& sp, cudaStream_t st) {
+    if (P.lanes_per_row == 8) return launch_rows_t<1, 8, 8, PRED>(P, sp, st);
+    if (P.lanes_per_row == 16) return launch_rows_t<1, 16, 8, PRED>(P, sp, st);
+    if (P.vec_per_lane == 1) return launch_rows_t<1, 32, 8, PRED>(P, sp, st);
+    if (P.vec_per_lane == 2) return launch_rows_t<2, 32, 8, PRED>(P, sp, st);
+    return launch_rows_t<4, 32, 4, PRED>(P, sp, st);
+}
+
+struct Pass {
+    const float* X; const float* y; int64_t m; int32_t n; const float* w; const float* b;
+};
+
+// Enqueues the streaming kernel for one pass (loss/grad partials, or labels when `labels` is set).
+int launch_stream_pass(lr_ctx* ctx, const lr_plan& P, const Pass& a, uint8_t* labels, float cut, cudaStream_t st) {
+    const bool predict = labels != nullptr;
+    const bool timed = ctx->prof && ctx->prof_used < kMaxProfiled;
+    if (timed) {
+        while (int(ctx->ev.size()) < 2 * (ctx->prof_used + 1)) {
+            cudaEvent_t e;
+            LR_CK(ctx, cudaEventCreate(&e));
+            ctx->ev.push_back(e);
+        }
+        LR_CK(ctx, cudaEventRecord(ctx->ev[2 * ctx->prof_used], st));
+    }
+    cudaError_t e;
+    if (P.variant == 0) {
+        StreamParams sp;
+        sp.X = a.X; sp.y = a.y; sp.m = a.m; sp.n = a.n; sp.w = a.w; sp.b = a.b;
+        sp.partial = ctx->d_partial; sp.labels = labels; sp.cut = cut; sp.status = ctx->d_status;
+        sp.bpt = P.tile_rows / P.rows_per_batch; sp.stages = P.stages;
+        sp.stage_y = (!predict && aligned(a.y, 16)) ? 1 : 0;
+        sp.num_tiles = (a.m + P.tile_rows - 1) / P.tile_rows;
+        e = predict ? launch_rows<true>(P, sp, st) : launch_rows<false>(P, sp, st);
+    } else {
+        GenericParams gp;
+        gp.X = a.X; gp.y = a.y; gp.m = a.m; gp.n = a.n; gp.w = a.w; gp.b = a.b;
+        gp.partial = ctx->d_partial; gp.labels = labels; gp.cut = cut;
+        if (predict) k_generic<true><<<P.grid, P.threads, 0, st>>>(gp);
+        else k_generic<false><<<P.grid, P.threads, 0, st>>>(gp);
+        e = cudaGetLastError();
+    }
+    LR_CK(ctx, e);
+    ctx->launches += 1;
+    if (timed) {
+        LR_CK(ctx, cudaEventRecord(ctx->ev[2 * ctx->prof_used + 1], st));
+        ctx->prof_used += 1;
+    }
+    return LR_OK;
+}
+
+int launch_reduce(lr_ctx* ctx, const lr_plan& P, int64_t m, int32_t n, double lr, bool update, float* w, float* b,
+                  float* grad_w, float* grad_b, float* loss_out, cudaStream_t st) {
+    ReduceParams rp;
+    rp.partial = ctx->d_partial; rp.G = P.grid; rp.n = n; rp.inv_m = 1.0 / double(m); rp.lr = lr;
+    rp.update = update ? 1 : 0; rp.w = w; rp.b = b; rp.grad_w = grad_w; rp.grad_b = grad_b; rp.loss_out = loss_out;
+    dim3 block(32, kRedSlices);
+    k_reduce_update<<<(n + 2 + 31) / 32, block, 0, st>>>(rp);
+    LR_CK(ctx, cudaGetLastError());
+    ctx->launches += 1;
+    return LR_OK;
+}
+
+int check_common(lr_ctx* ctx, const void* X, int64_t m, int32_t n, const void* w, const void* b) {
+    if (!ctx || !X || !w || !b) return LR_ERR_NULL;
+    if (m < 1 || m > kMaxRows || n < 1 || n > ctx->n_max) return LR_ERR_SHAPE;
+    if (!aligned(X, 4) || !aligned(w, 4) || !aligned(b, 4)) return LR_ERR_ALIGNMENT;
+    return LR_OK;
+}
+
+int grow(lr_ctx* ctx, void** buf, size_t* have, size_t need) {
+    if (*have >= need) return LR_OK;
+    if (*buf) { LR_CK(ctx, cudaFree(*buf)); *buf = nullptr; *have = 0; }
+    cudaError_t e = cudaMalloc(buf, need);
+    if (e != cudaSuccess) { ctx->last_cuda = int(e); *buf = nullptr; return e == cudaErrorMemoryAllocation ? LR_ERR_NOMEM : LR_ERR_CUDA; }
+    *have = need;
+    return LR_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int lr_plan_query(int64_t m, int32_t n, int32_t x_aligned16, int32_t sm_count, lr_plan* out) {
+    if (!out) return LR_ERR_NULL;
+    return make_plan(m, n, x_aligned16 != 0, sm_count, out);
+}
+
+int lr_create(lr_ctx** out, int32_t device, int32_t n_max) {
+    if (!out) return LR_ERR_NULL;
+    *out = nullptr;
+    if (n_max < 1) return LR_ERR_SHAPE;
+    lr_ctx* c = new (std::nothrow) lr_ctx();
+    if (!c) return LR_ERR_NOMEM;
+    c->device = device;
+    c->n_max = n_max;
+    int prev = -1;
+    cudaGetDevice(&prev);
+    int rc = LR_OK;
+    cudaError_t e = cudaSetDevice(device);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, device);
+    if (e == cudaSuccess) {
+        const size_t bytes = size_t(c->sm_count) * kMaxGridPerSm * (size_t(n_max) + 2) * sizeof(double);
+        e = cudaMalloc(reinterpret_cast<void**>(&c->d_partial), bytes);
+        if (e == cudaErrorMemoryAllocation) rc = LR_ERR_NOMEM;
+    }
+    if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&c->d_status), sizeof(int));
+    if (e == cudaSuccess) e = cudaMemset(c->d_status, 0, sizeof(int));
+    if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&c->hstream, cudaStreamNonBlocking);
+    if (prev >= 0) cudaSetDevice(prev);
+    if (e != cudaSuccess) {
+        if (c->d_partial) cudaFree(c->d_partial);
+        if (c->d_status) cudaFree(c->d_status);
+        delete c;
+        return rc != LR_OK ? rc : LR_ERR_CUDA;
+    }
+    *out = c;
+    return LR_OK;
+}
+
+int lr_destroy(lr_ctx* ctx) {
+    if (!ctx) return LR_OK;
+    {
+        DeviceGuard g(ctx);
+        cudaDeviceSynchronize();
+        for (cudaEvent_t e : ctx->ev) cudaEventDestroy(e);
+        if (ctx->hstream) cudaStreamDestroy(ctx->hstream);
+        cudaFree(ctx->d_partial);
+        cudaFree(ctx->d_status);
+        cudaFree(ctx->d_hX);
+        cudaFree(ctx->d_hy);
+        cudaFree(ctx->d_hw);
+        cudaFree(ctx->d_hl);
+    }
+    delete ctx;
+    return LR_OK;
+}
+
+int lr_loss_grad(lr_ctx* ctx, const float* d_X, const float* d_y, int64_t m, int32_t n, const float* d_w,
+                 const float* d_b, float* d_loss, float* d_grad_w, float* d_grad_b, void* stream) {
+    int rc = check_common(ctx, d_X, m, n, d_w, d_b);
+    if (rc != LR_OK) return rc;
+    if (!d_y || !d_loss || !d_grad_w || !d_grad_b) return LR_ERR_NULL;
+    if (!aligned(d_y, 4) || !aligned(d_loss, 4) || !aligned(d_grad_w, 4) || !aligned(d_grad_b, 4)) return LR_ERR_ALIGNMENT;
+    lr_plan P;
+    rc = make_plan(m, n, aligned(d_X, 16), ctx->sm_count, &P);
+    if (rc != LR_OK) return rc;
+    DeviceGuard g(ctx);
+    if (!g.ok) return LR_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    rc = launch_stream_pass(ctx, P, Pass{d_X, d_y, m, n, d_w, d_b}, nullptr, 0.f, st);
+    if (rc != LR_OK) return rc;
+    return launch_reduce(ctx, P, m, n, 0.0, false, nullptr, nullptr, d_grad_w, d_grad_b, d_loss, st);
+}
+
+int lr_fit(lr_ctx* ctx, const float* d_X, const float* d_y, int64_t m, int32_t n, float lr, int32_t iters,
+           float* d_w, float* d_b, float* d_loss_hist, void* stream) {
+    int rc = check_common(ctx, d_X, m, n, d_w, d_b);
+    if (rc != LR_OK) return rc;
+    if (!d_y) return LR_ERR_NULL;
+    if (iters < 0) return LR_ERR_SHAPE;
+    if (!aligned(d_y, 4) || (d_loss_hist && !aligned(d_loss_hist, 4))) return LR_ERR_ALIGNMENT;
+    if (!std::isfinite(lr)) return LR_ERR_VALUE;
+    lr_plan P;
+    rc = make_plan(m, n, aligned(d_X, 16), ctx->sm_count, &P);
+    if (rc != LR_OK) return rc;
+    if (iters == 0) return LR_OK;
+    DeviceGuard g(ctx);
+    if (!g.ok) return LR_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    for (int32_t t = 0; t < iters; ++t) {
+        rc = launch_stream_pass(ctx, P, Pass{d_X, d_y, m, n, d_w, d_b}, nullptr, 0.f, st);
+        if (rc != LR_OK) return rc;
+        rc = launch_reduce(ctx, P, m, n, double(lr), true, d_w, d_b, nullptr, nullptr,
+                           d_loss_hist ? d_loss_hist + t : nullptr, st);
+        if (rc != LR_OK) return rc;
+    }
+    return LR_OK;
+}
+
+int lr_predict(lr_ctx* ctx, const float* d_X, int64_t m, int32_t n, const float* d_w, const float* d_b, float thr,
+               uint8_t* d_labels, void* stream) {
+    int rc = check_common(ctx, d_X, m, n, d_w, d_b);
+    if (rc != LR_OK) return rc;
+    if (!d_labels) return LR_ERR_NULL;
+    if (!(thr > 0.f && thr < 1.f)) return LR_ERR_VALUE;
+    lr_plan P;
+    rc = make_plan(m, n, aligned(d_X, 16), ctx->sm_count, &P);
+    if (rc != LR_OK) return rc;
+    DeviceGuard g(ctx);
+    if (!g.ok) return LR_ERR_CUDA;
+    const float cut = static_cast<float>(std::log(double(thr) / (1.0 - double(thr))));
+    return launch_stream_pass(ctx, P, Pass{d_X, nullptr, m, n, d_w, d_b}, d_labels, cut, static_cast<cudaStream_t>(stream));
+}
+
+int lr_fit_host(lr_ctx* ctx, const float* h_X, const float* h_y, int64_t m, int32_t n, float lr, int32_t iters,
+                float* h_w, float* h_b, float* h_loss_hist) {
+    int rc = check_common(ctx, h_X, m, n, h_w, h_b);
+    if (rc != LR_OK) return rc;
+    if (!h_y) return LR_ERR_NULL;
+    if (iters < 0) return LR_ERR_SHAPE;
+    if (!std::isfinite(lr)) return LR_ERR_VALUE;
+    DeviceGuard g(ctx);
+    if (!g.ok) return LR_ERR_CUDA;
+    const size_t xb = size_t(m) * n * 4, yb = size_t(m) * 4;
+    const size_t wb = (size_t(n) + 1 + size_t(iters)) * 4;
+    if ((rc = grow(ctx, &ctx->d_hX, &ctx->hX_bytes, xb)) != LR_OK) return rc;
+    if ((rc = grow(ctx, &ctx->d_hy, &ctx->hy_bytes, yb)) != LR_OK) return rc;
+    if ((rc = grow(ctx, &ctx->d_hw, &ctx->hw_bytes, wb)) != LR_OK) return rc;
+    float* dX = static_cast<float*>(ctx->d_hX);
+    float* dy = static_cast<float*>(ctx->d_hy);
+    float* dw = static_cast<float*>(ctx->d_hw);
+    float* db = dw + n;
+    float* dh = db + 1;
+    cudaStream_t st = ctx->hstream;
+    LR_CK(ctx, cudaMemcpyAsync(dX, h_X, xb, cudaMemcpyHostToDevice, st));
+    LR_CK(ctx, cudaMemcpyAsync(dy, h_y, yb, cudaMemcpyHostToDevice, st));
+    LR_CK(ctx, cudaMemcpyAsync(dw, h_w, size_t(n) * 4, cudaMemcpyHostToDevice, st));
+    LR_CK(ctx, cudaMemcpyAsync(db, h_b, 4, cudaMemcpyHostToDevice, st));
+    rc = lr_fit(ctx, dX, dy, m, n, lr, iters, dw, db, h_loss_hist ? dh : nullptr, st);
+    if (rc != LR_OK) return rc;
+    LR_CK(ctx, cudaMemcpyAsync(h_w, dw, size_t(n) * 4, cudaMemcpyDeviceToHost, st));
+    LR_CK(ctx, cudaMemcpyAsync(h_b, db, 4, cudaMemcpyDeviceToHost, st));
+    if (h_loss_hist && iters > 0) LR_CK(ctx, cudaMemcpyAsync(h_loss_hist, dh, size_t(iters) * 4, cudaMemcpyDeviceToHost, st));
+    LR_CK(ctx, cudaStreamSynchronize(st));
+    return LR_OK;
+}
+
+int lr_predict_host(lr_ctx* ctx, const float* h_X, int64_t m, int32_t n, const float* h_w, const float* h_b, float thr,
+                    uint8_t* h_labels) {
+    int rc = check_common(ctx, h_X, m, n, h_w, h_b);
+    if (rc != LR_OK) return rc;
+    if (!h_labels) return LR_ERR_NULL;
+    if (!(thr > 0.f && thr < 1.f)) return LR_ERR_VALUE;
+    DeviceGuard g(ctx);
+    if (!g.ok) return LR_ERR_CUDA;
+    const size_t xb = size_t(m) * n * 4;
+    if ((rc = grow(ctx, &ctx->d_hX, &ctx->hX_bytes, xb)) != LR_OK) return rc;
+    if ((rc = grow(ctx, &ctx->d_hw, &ctx->hw_bytes, (size_t(n) + 1) * 4)) != LR_OK) return rc;
+    if ((rc = grow(ctx, &ctx->d_hl, &ctx->hl_bytes, size_t(m))) != LR_OK) return rc;
+    float* dX = static_cast<float*>(ctx->d_hX);
+    float* dw = static_cast<float*>(ctx->d_hw);
+    float* db = dw + n;
+    uint8_t* dl = static_cast<uint8_t*>(ctx->d_hl);
+    cudaStream_t st = ctx->hstream;
+    LR_CK(ctx, cudaMemcpyAsync(dX, h_X, xb, cudaMemcpyHostToDevice, st));
+    LR_CK(ctx, cudaMemcpyAsync(dw, h_w, size_t(n) * 4, cudaMemcpyHostToDevice, st));
+    LR_CK(ctx, cudaMemcpyAsync(db, h_b, 4, cudaMemcpyHostToDevice, st));
+    rc = lr_predict(ctx, dX, m, n, dw, db, thr, dl, st);
+    if (rc != LR_OK) return rc;
+    LR_CK(ctx, cudaMemcpyAsync(h_labels, dl, size_t(m), cudaMemcpyDeviceToHost, st));
+    LR_CK(ctx, cudaStreamSynchronize(st));
+    return LR_OK;
+}
+
+int lr_profile_enable(lr_ctx* ctx, int32_t on) {
+    if (!ctx) return LR_ERR_NULL;
+    ctx->prof = on != 0;
+    ctx->prof_used = 0;
+    return LR_OK;
+}
+
+int lr_profile_read(lr_ctx* ctx, int32_t* launches, double* total_ms) {
+    if (!ctx || !launches || !total_ms) return LR_ERR_NULL;
+    DeviceGuard g(ctx);
+    if (!g.ok) return LR_ERR_CUDA;
+    double sum = 0.0;
+    for (int i = 0; i < ctx->prof_used; ++i) {
+        LR_CK(ctx, cudaEventSynchronize(ctx->ev[2 * i + 1]));
+        float ms = 0.f;
+        LR_CK(ctx, cudaEventElapsedTime(&ms, ctx->ev[2 * i], ctx->ev[2 * i + 1]));
+        sum += ms;
+    }
+    *launches = ctx->prof_used;
+    *total_ms = sum;
+    ctx->prof_used = 0;
+    return LR_OK;
+}
+
+int lr_launch_count(lr_ctx* ctx, int64_t* out) {
+    if (!ctx || !out) return LR_ERR_NULL;
+    *out = ctx->launches;
+    return LR_OK;
+}
+
+int lr_last_device_status(lr_ctx* ctx, int32_t* out) {
+    if (!ctx || !out) return LR_ERR_NULL;
+    DeviceGuard g(ctx);
+    if (!g.ok) return LR_ERR_CUDA;
+    LR_CK(ctx, cudaDeviceSynchronize());
+    int v = 0;
+    LR_CK(ctx, cudaMemcpy(&v, ctx->d_status, sizeof(int), cudaMemcpyDeviceToHost));
+    LR_CK(ctx, cudaMemset(ctx->d_status, 0, sizeof(int)));
+    *out = v;
+    return LR_OK;
+}
+
+int lr_last_cuda_error(lr_ctx* ctx) { return ctx ? ctx->last_cuda : 0; }
+
+const char* lr_status_string(int code) {
+    switch (code) {
+        case LR_OK: return "ok";
+        case LR_ERR_NULL: return "a required pointer is NULL";
+        case LR_ERR_SHAPE: return "shape out of range (m, n, iters) or larger than the context allows";
+        case LR_ERR_ALIGNMENT: return "a float pointer is not 4-byte aligned";
+        case LR_ERR_VALUE: return "value out of range (thr must be in (0,1), lr finite)";
+        case LR_ERR_CUDA: return "a CUDA runtime call failed";
+        case LR_ERR_TIMEOUT: return "a bounded device-side wait expired";
+        case LR_ERR_NOMEM: return "allocation failed";
+        default: return "unknown status";
+    }
+}
+
+}  // extern "C"

@@ -1,0 +1,105 @@
+// Shared device helpers: mbarrier / bulk-async-copy wrappers (sm_90+ PTX, used here on sm_100a),
+// bounded waits, and the per-row logistic terms.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace lrgd {
+
+constexpr int kStatusTimeout = -6;                 // LR_ERR_TIMEOUT
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s per wait, then the kernel gives up
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+
+__device__ __forceinline__ unsigned long long global_timer_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+
+__device__ __forceinline__ void fence_mbar_init() {
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+
+// Waits for the phase with the given parity to complete, for at most kWaitLimitNs.  On expiry (or when
+// another thread of the CTA has already given up) raises *abort_flag and returns false.
+__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const unsigned long long t0 = global_timer_ns();
+    for (;;) {
+#pragma unroll 1
+        for (int i = 0; i < 32; ++i)
+            if (mbar_try_wait(bar, parity)) return true;
+        if (*abort_flag) return false;
+        if (global_timer_ns() - t0 > kWaitLimitNs) {
+            *abort_flag = 1;
+            return false;
+        }
+    }
+}
+
+__device__ __forceinline__ uint64_t l2_policy_evict_first() {
+    uint64_t pol;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
+}
+
+// 1-D bulk asynchronous copy global -> shared; completion is signalled on `bar` as transferred bytes.
+// dst, src 16-byte aligned, bytes a non-zero multiple of 16.
+__device__ __forceinline__ void bulk_copy_g2s(void* dst, const void* src, uint32_t bytes, uint64_t* bar, uint64_t policy) {
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
+        ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)), "l"(policy)
+        : "memory");
+}
+
+// Per-row logistic terms in fp32 from the logit z and the target y:
+//   err  = sigmoid(z) - y            (Eq. 1; Algorithm 7's sigmoid followed by Substract(Y, res))
+//   loss = max(z,0) + log1p(exp(-|z|)) - y*z  ( = -[y log p + (1-y) log(1-p)], finite for any z )
+// For y exactly 1 the error is formed as -sigmoid(-z) so that it keeps full relative precision when p -> 1.
+__device__ __forceinline__ void logistic_terms(float z, float y, float& err, float& loss) {
+    const float t = expf(-fabsf(z));
+    const float r = 1.0f / (1.0f + t);
+    const float tr = t * r;
+    const float p = z >= 0.0f ? r : tr;      // sigmoid(z)
+    const float q = z >= 0.0f ? tr : r;      // sigmoid(-z) = 1 - p
+    err = (y == 1.0f) ? -q : (p - y);
+    loss = fmaxf(z, 0.0f) + log1pf(t) - y * z;
+}
+
+template <int V>
+struct Log2 {
+    static constexpr int value = 1 + Log2<V / 2>::value;
+};
+template <>
+struct Log2<1> {
+    static constexpr int value = 0;
+};
+
+}  // namespace lrgd

@@ -1,0 +1,86 @@
+"""CPU-only checks of the C-ABI library: it loads, exports what the header declares, and its host
+logic (launch planning, argument validation that needs no device) behaves."""
+import ctypes
+import os
+import re
+
+import pytest
+
+from paper_2308_10037_b200 import api
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    from paper_2308_10037_b200 import build
+    build.build()
+
+
+def _declared():
+    text = open(os.path.join(ROOT, "include", "lrgd.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(lr_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported():
+    L = api.lib()
+    names = _declared()
+    assert "lr_loss_grad" in names and "lr_fit" in names and "lr_predict" in names
+    for name in names:
+        assert hasattr(L, name), name
+    assert sorted(api.EXPORTS) == names
+
+
+def test_status_strings():
+    assert api.status_string(0) == "ok"
+    for code in range(-7, 0):
+        assert api.status_string(code) not in ("ok", "unknown status")
+    assert api.status_string(-99) == "unknown status"
+
+
+def test_null_context_is_rejected_before_any_cuda_call():
+    L = api.lib()
+    one = ctypes.c_void_p(16)
+    assert L.lr_loss_grad(None, one, one, 4, 4, one, one, one, one, one, None) == api.LR_ERR_NULL
+    assert L.lr_fit(None, one, one, 4, 4, 0.1, 1, one, one, None, None) == api.LR_ERR_NULL
+    assert L.lr_predict(None, one, 4, 4, one, one, 0.5, one, None) == api.LR_ERR_NULL
+    assert L.lr_create(None, 0, 4) == api.LR_ERR_NULL
+    h = ctypes.c_void_p()
+    assert L.lr_create(ctypes.byref(h), 0, 0) == api.LR_ERR_SHAPE
+    assert L.lr_destroy(None) == api.LR_OK
+
+
+@pytest.mark.parametrize("m,n,lpr,nv", [(10_000, 32, 8, 1), (16_000_000, 64, 16, 1), (1_000_000, 100, 32, 1),
+                                         (4_000_000, 256, 32, 2), (11_000_000, 28, 8, 1), (5000, 512, 32, 4)])
+def test_plan_staged_shapes(m, n, lpr, nv):
+    p = api.plan_query(m, n)
+    assert p["variant"] == 0 and p["lanes_per_row"] == lpr and p["vec_per_lane"] == nv
+    assert p["threads"] == 512 and 1 <= p["grid"] <= 148
+    assert p["tile_rows"] % p["rows_per_batch"] == 0 and p["tile_rows"] % 4 == 0
+    assert p["tile_rows"] * n * 4 <= 32 * 1024 or p["tile_rows"] == p["rows_per_batch"]
+    assert 1 <= p["stages"] <= 8
+    assert p["smem_bytes"] <= 227 * 1024
+    # every row is covered by exactly one tile
+    tiles = -(-m // p["tile_rows"])
+    assert p["grid"] == min(tiles, 148)
+
+
+def test_plan_falls_back_for_unaligned_or_odd_shapes():
+    assert api.plan_query(1000, 30)["variant"] == 2          # n not a multiple of 4
+    assert api.plan_query(1000, 32, x_aligned16=False)["variant"] == 2
+    assert api.plan_query(1000, 8192)["variant"] == 2         # wider than any staged kernel
+    g = api.plan_query(100, 30)
+    assert g["grid"] == 2 and g["threads"] == 256
+
+
+def test_plan_rejects_bad_shapes():
+    for m, n in [(0, 4), (4, 0), (-1, 4), (1 << 41, 4)]:
+        with pytest.raises(api.LrError) as e:
+            api.plan_query(m, n)
+        assert e.value.code == api.LR_ERR_SHAPE
+
+
+def test_small_problems_spread_over_all_sms():
+    p = api.plan_query(10_000, 32, sm_count=148)
+    assert p["grid"] >= 100

@@ -1,0 +1,208 @@
+"""GPU parity: the CUDA path, called through the C-ABI binding, against the float64 CPU checker on the
+same seeded inputs.  Tolerances (fp32 storage and accumulation against float64):
+  gradient (grad_w, grad_b stacked) relative L2 <= 1e-5, loss absolute <= 1e-6,
+  final parameters after a fit relative L2 <= 1e-4, predicted labels agreeing on >= 99.99 % of rows.
+"""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2308_10037_b200 import api, datagen
+
+pytestmark = pytest.mark.gpu
+
+GRAD_TOL, LOSS_TOL, W_TOL, LABEL_AGREE = 1e-5, 1e-6, 1e-4, 0.9999
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    from paper_2308_10037_b200 import build
+    build.build()
+    c = api.Context(n_max=8200, device=0)
+    yield c
+    assert c.device_status() == 0
+    c.close()
+
+
+def dev(a):
+    return torch.from_numpy(np.ascontiguousarray(a)).cuda()
+
+
+def rel_l2(a, b):
+    a, b = np.asarray(a, dtype=np.float64).ravel(), np.asarray(b, dtype=np.float64).ravel()
+    return float(np.linalg.norm(a - b) / max(np.linalg.norm(b), 1e-300))
+
+
+def check_loss_grad(ctx, X, y, w, b, grad_tol=GRAD_TOL, loss_tol=LOSS_TOL):
+    L, g, g0 = oracle.loss_grad(X, y, np.asarray(w, dtype=np.float64), float(b))
+    dl, dg, dg0 = ctx.loss_grad(dev(X), dev(y), dev(np.asarray(w, dtype=np.float32)), dev(np.array([b], dtype=np.float32)))
+    torch.cuda.synchronize()
+    assert abs(dl.item() - L) <= loss_tol, (dl.item(), L)
+    got = np.concatenate([dg.cpu().numpy(), dg0.cpu().numpy()])
+    assert rel_l2(got, np.concatenate([g, [g0]])) <= grad_tol
+    return got
+
+
+# shapes: every staged instantiation (n/4 <= 8, 16, 32, 64, 128), partly filled lane groups (28, 100, 200, 36),
+# the unstaged kernel (n % 4 != 0, n > 512), and row counts that are tiny, ragged, or span many tiles
+SHAPES = [(1, 4), (7, 4), (8, 3), (33, 28), (1000, 32), (4097, 32), (5003, 64), (2500, 36), (3001, 100), (9999, 256),
+          (777, 200), (1500, 512), (2049, 260), (640, 30), (1025, 101), (300, 1), (130, 4096), (50, 8192), (20011, 8)]
+
+
+@pytest.mark.parametrize("m,n", SHAPES)
+def test_loss_grad_matches_oracle(ctx, m, n):
+    X, y, w, b = datagen.random_problem(m, n, seed=1000 + m + n, wscale=1.5)
+    check_loss_grad(ctx, X, y, w, b)
+
+
+@pytest.mark.parametrize("m,n", [(1000, 32), (3001, 100), (9999, 256), (640, 30)])
+def test_zero_parameters_give_ln2(ctx, m, n):
+    X, y, _, _ = datagen.random_problem(m, n, seed=7)
+    dl, dg, dg0 = ctx.loss_grad(dev(X), dev(y), torch.zeros(n, device="cuda"), torch.zeros(1, device="cuda"))
+    assert abs(dl.item() - math.log(2)) <= LOSS_TOL
+    ref = X.astype(np.float64).T @ (0.5 - y.astype(np.float64)) / m
+    assert rel_l2(dg.cpu().numpy(), ref) <= GRAD_TOL
+
+
+def test_saturated_rows_stay_finite(ctx):
+    # |z| up to ~90: p rounds to 0 or 1 in fp32, the loss must stay finite and match
+    # the loss is ~38 here and is returned as one fp32 (spacing 3.8e-6), so its tolerance is one fp32 ulp of the value
+    X, y, w, b = datagen.random_problem(4000, 64, seed=3, wscale=90.0)
+    got = check_loss_grad(ctx, X, y, w, b, loss_tol=38.1 * 2.0 ** -23)
+    assert np.isfinite(got).all()
+
+
+def test_unaligned_views_use_the_unstaged_kernel(ctx):
+    X, y, w, b = datagen.random_problem(1201, 32, seed=11)
+    buf = torch.zeros(X.size + 1, dtype=torch.float32, device="cuda")
+    buf[1:] = dev(X).ravel()
+    Xv = buf[1:].view(1201, 32)                      # 4-byte aligned only
+    assert Xv.data_ptr() % 16 == 4
+    ybuf = torch.zeros(1202, dtype=torch.float32, device="cuda")
+    ybuf[1:] = dev(y)
+    L, g, g0 = oracle.loss_grad(X, y, w, b)
+    dl, dg, dg0 = ctx.loss_grad(Xv, ybuf[1:], dev(w), dev(np.array([b], dtype=np.float32)))
+    assert abs(dl.item() - L) <= LOSS_TOL and rel_l2(dg.cpu().numpy(), g) <= GRAD_TOL
+    # aligned X with an unaligned y: staged X, y read directly
+    dl2, dg2, _ = ctx.loss_grad(dev(X), ybuf[1:], dev(w), dev(np.array([b], dtype=np.float32)))
+    assert abs(dl2.item() - L) <= LOSS_TOL and rel_l2(dg2.cpu().numpy(), g) <= GRAD_TOL
+
+
+SMALL_WORKLOADS = [("cfg1", 10_000), ("cfg2", 40_000), ("cfg3", 30_011), ("cfg4", 3_000), ("cfg5", 100_003),
+                   ("higgs_like", 50_001)]
+
+
+@pytest.mark.parametrize("name,m", SMALL_WORKLOADS)
+def test_teacher_forced_trajectory(ctx, name, m):
+    # feed the checker's own iterates (rounded to fp32) to the GPU pass, so errors cannot compound
+    wl = datagen.scaled(datagen.WORKLOADS[name], m)
+    X, y, _, _ = datagen.generate(wl)
+    iters = min(wl.iters, 40)
+    _, _, lh, wh, bh = oracle.fit(X, y, wl.lr, iters, history=True)
+    dX, dy = dev(X), dev(y)
+    for t in sorted({0, 1, 2, iters // 2, iters - 1}):
+        w32 = wh[t].astype(np.float32)
+        b32 = np.float32(bh[t])
+        L, g, g0 = oracle.loss_grad(X, y, w32.astype(np.float64), float(b32))
+        dl, dg, dg0 = ctx.loss_grad(dX, dy, dev(w32), dev(np.array([b32])))
+        assert abs(dl.item() - L) <= LOSS_TOL, (t, dl.item(), L)
+        got = np.concatenate([dg.cpu().numpy(), dg0.cpu().numpy()])
+        assert rel_l2(got, np.concatenate([g, [g0]])) <= GRAD_TOL, t
+
+
+@pytest.mark.parametrize("name,m", SMALL_WORKLOADS)
+def test_fit_matches_oracle(ctx, name, m):
+    wl = datagen.scaled(datagen.WORKLOADS[name], m)
+    X, y, _, _ = datagen.generate(wl)
+    w_ref, b_ref, lh_ref = oracle.fit(X, y, wl.lr, wl.iters)
+    w, b, lh = api.lr_fit(dev(X), dev(y), wl.lr, wl.iters, return_history=True, ctx=ctx)
+    got = np.concatenate([w.cpu().numpy(), b.cpu().numpy()])
+    ref = np.concatenate([w_ref, [b_ref]])
+    if name == "cfg4":
+        # lr = 0.05 is above 2/L for uncentred U[0,1) features: the iteration is not a contraction, so rounding
+        # differences are amplified; the checker's own fp32-rounded rerun sets the scale of what is attainable
+        w_r, b_r, _ = oracle.fit(X, y, wl.lr, wl.iters, round_to_fp32=True)
+        own = rel_l2(np.concatenate([w_r, [b_r]]), ref)
+        assert rel_l2(got, ref) <= max(W_TOL, 20 * own)
+    else:
+        assert rel_l2(got, ref) <= W_TOL
+        assert np.max(np.abs(lh.cpu().numpy().astype(np.float64) - lh_ref)) <= LOSS_TOL
+
+
+def test_fit_is_deterministic_and_resumable(ctx):
+    wl = datagen.scaled(datagen.WORKLOADS["cfg3"], 20_000)
+    X, y, _, _ = datagen.generate(wl)
+    dX, dy = dev(X), dev(y)
+    w1, b1, h1 = api.lr_fit(dX, dy, wl.lr, 12, return_history=True, ctx=ctx)
+    w2, b2, h2 = api.lr_fit(dX, dy, wl.lr, 12, return_history=True, ctx=ctx)
+    assert torch.equal(w1, w2) and torch.equal(b1, b2) and torch.equal(h1, h2)
+    wa, ba = api.lr_fit(dX, dy, wl.lr, 7, ctx=ctx)
+    wb, bb = api.lr_fit(dX, dy, wl.lr, 5, w0=wa, b0=ba, ctx=ctx)
+    assert torch.equal(wb, w1) and torch.equal(bb, b1)
+    w0, b0 = api.lr_fit(dX, dy, wl.lr, 0, ctx=ctx)
+    assert not w0.any() and not b0.any()
+
+
+@pytest.mark.parametrize("m,n", [(5003, 64), (9999, 256), (3001, 100), (640, 30), (130, 4096), (33, 28)])
+def test_predict_matches_oracle(ctx, m, n):
+    X, y, w, b = datagen.random_problem(m, n, seed=50 + n, wscale=2.0)
+    dX, dw, db = dev(X), dev(w), dev(np.array([b], dtype=np.float32))
+    for thr in (0.5, 0.2, 0.9):
+        ref, z = oracle.predict(X, w, b, thr, return_z=True)
+        got = ctx.predict(dX, dw, db, thr).cpu().numpy()
+        cut = math.log(thr / (1 - thr))
+        clear = np.abs(z - cut) > 1e-4 * (1 + np.abs(z))   # rows whose decision is not within fp32 noise of the cut
+        assert np.array_equal(got[clear], ref[clear])
+        assert (got == ref).mean() >= LABEL_AGREE or m < 10_000 and (got != ref).sum() <= 1
+
+
+def test_predict_after_fit_agrees_and_f1_matches(ctx):
+    wl = datagen.scaled(datagen.WORKLOADS["cfg2"], 60_000)
+    X, y, _, _ = datagen.generate(wl)
+    dX, dy = dev(X), dev(y)
+    w, b = api.lr_fit(dX, dy, wl.lr, 50, ctx=ctx)
+    labels = api.lr_predict(dX, w, b, 0.5, ctx=ctx).cpu().numpy()
+    w_ref, b_ref, _ = oracle.fit(X, y, wl.lr, 50)
+    ref = oracle.predict(X, w_ref, b_ref, 0.5)
+    assert (labels == ref).mean() >= LABEL_AGREE
+    assert abs(oracle.f1_score(labels, y)[0] - oracle.f1_score(ref, y)[0]) < 1e-3
+
+
+def test_host_entry_points_equal_device_entry_points(ctx):
+    wl = datagen.scaled(datagen.WORKLOADS["cfg5"], 30_001)
+    X, y, _, _ = datagen.generate(wl)
+    w = np.zeros(wl.n, dtype=np.float32)
+    b = np.zeros(1, dtype=np.float32)
+    hist = np.zeros(9, dtype=np.float32)
+    ctx.fit_host(X, y, wl.lr, 9, w, b, hist)
+    dw, db, dh = api.lr_fit(dev(X), dev(y), wl.lr, 9, return_history=True, ctx=ctx)
+    assert np.array_equal(w, dw.cpu().numpy()) and np.array_equal(b, db.cpu().numpy())
+    assert np.array_equal(hist, dh.cpu().numpy())
+    labels = np.zeros(wl.m, dtype=np.uint8)
+    ctx.predict_host(X, w, b, 0.02, labels)
+    assert np.array_equal(labels, api.lr_predict(dev(X), dw, db, 0.02, ctx=ctx).cpu().numpy())
+
+
+def test_argument_errors_with_a_live_context(ctx):
+    X, y, w, b = datagen.random_problem(64, 8, seed=1)
+    dX, dy, dw, db = dev(X), dev(y), dev(w), dev(np.array([b], dtype=np.float32))
+    small = api.Context(n_max=4, device=0)
+    with pytest.raises(api.LrError) as e:
+        small.loss_grad(dX, dy, dw, db)
+    assert e.value.code == api.LR_ERR_SHAPE
+    small.close()
+    with pytest.raises(api.LrError) as e:
+        ctx.predict(dX, dw, db, 1.0)
+    assert e.value.code == api.LR_ERR_VALUE
+    with pytest.raises(api.LrError) as e:
+        ctx.fit(dX, dy, float("nan"), 1, dw.clone(), db.clone())
+    assert e.value.code == api.LR_ERR_VALUE
+    with pytest.raises(api.LrError) as e:
+        ctx.fit(dX, dy, 0.1, -1, dw.clone(), db.clone())
+    assert e.value.code == api.LR_ERR_SHAPE
+    n0 = ctx.launch_count()
+    ctx.loss_grad(dX, dy, dw, db)
+    assert ctx.launch_count() == n0 + 2
