@@ -54,8 +54,8 @@ typedef struct lr_plan {
     int32_t lanes_per_row; /* staged kernels: lanes that share one row (8, 16, 32; 256 for the row-split kernel) */
     int32_t vec_per_lane;  /* staged kernels: 16-byte column groups owned by one lane */
     int32_t rows_per_batch;/* rows one warp (or one CTA for the row-split kernel) holds in registers at a time */
-    int32_t tile_rows;     /* rows per asynchronously staged tile */
-    int32_t stages;        /* tiles in flight per CTA */
+    int32_t tile_rows;     /* rows per asynchronously staged shared-memory stage */
+    int32_t stages;        /* stages (copies in flight) per warp; per CTA for the row-split kernel */
     int32_t grid;          /* CTAs */
     int32_t threads;       /* threads per CTA */
     int32_t smem_bytes;    /* dynamic shared memory per CTA */
@@ -106,6 +106,20 @@ int lr_fit(lr_ctx* ctx, const float* d_X, const float* d_y, int64_t m, int32_t n
  */
 int lr_predict(lr_ctx* ctx, const float* d_X, int64_t m, int32_t n,
                const float* d_w, const float* d_b, float thr, uint8_t* d_labels, void* stream);
+
+/*
+ * Row-sharded data parallelism (the natural split of Algorithm 1's sums over rows; the paper itself
+ * runs on one device).  Each shard holds a contiguous block of rows.  lr_shard_sums runs the fused
+ * pass on the local rows and writes the UNNORMALISED fp64 sums d_sums[0..n) = X^T err,
+ * d_sums[n] = sum err, d_sums[n+1] = sum of per-row loss terms.  After the caller has gathered the
+ * `parts` sum vectors into d_sums_all [parts][n+2] (rank order), lr_apply_sums adds them in index
+ * order, scales by 1/m_total and applies  w <- w - lr*grad_w, b <- b - lr*grad_b  (every rank gets
+ * bit-identical parameters); d_loss (nullable) receives the global loss before the update.
+ */
+int lr_shard_sums(lr_ctx* ctx, const float* d_X, const float* d_y, int64_t m_local, int32_t n,
+                  const float* d_w, const float* d_b, double* d_sums, void* stream);
+int lr_apply_sums(lr_ctx* ctx, const double* d_sums_all, int32_t parts, int64_t m_total, int32_t n,
+                  float lr, float* d_w, float* d_b, float* d_loss, void* stream);
 
 /*
  * Host-buffer variants: copy h_X, h_y (and h_w, h_b) to device buffers owned by the context

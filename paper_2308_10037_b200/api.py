@@ -13,12 +13,13 @@ import numpy as np
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "liblrgd.so")
+LIB_PATH = os.environ.get("LRGD_LIB") or os.path.join(_HERE, "liblrgd.so")   # LRGD_LIB: another build of the same library
 
 LR_OK = 0
 LR_ERR_NULL, LR_ERR_SHAPE, LR_ERR_ALIGNMENT, LR_ERR_VALUE, LR_ERR_CUDA, LR_ERR_TIMEOUT, LR_ERR_NOMEM = range(-1, -8, -1)
 
-EXPORTS = ["lr_plan_query", "lr_create", "lr_destroy", "lr_loss_grad", "lr_fit", "lr_predict", "lr_fit_host",
+EXPORTS = ["lr_plan_query", "lr_create", "lr_destroy", "lr_loss_grad", "lr_fit", "lr_predict", "lr_shard_sums",
+           "lr_apply_sums", "lr_fit_host",
            "lr_predict_host", "lr_profile_enable", "lr_profile_read", "lr_launch_count", "lr_last_device_status",
            "lr_last_cuda_error", "lr_status_string"]
 
@@ -55,6 +56,8 @@ def lib() -> ctypes.CDLL:
         L.lr_loss_grad.argtypes = [P, P, P, I64, I32, P, P, P, P, P, P]
         L.lr_fit.argtypes = [P, P, P, I64, I32, F, I32, P, P, P, P]
         L.lr_predict.argtypes = [P, P, I64, I32, P, P, F, P, P]
+        L.lr_shard_sums.argtypes = [P, P, P, I64, I32, P, P, P, P]
+        L.lr_apply_sums.argtypes = [P, P, I32, I64, I32, F, P, P, P, P]
         L.lr_fit_host.argtypes = [P, P, P, I64, I32, F, I32, P, P, P]
         L.lr_predict_host.argtypes = [P, P, I64, I32, P, P, F, P]
         L.lr_profile_enable.argtypes = [P, I32]
@@ -165,6 +168,22 @@ class Context:
                               self._stream())
         self._check(rc, "lr_predict")
         return labels
+
+    def shard_sums(self, X, y, w, b, sums):
+        """Unnormalised fp64 sums [n+2] of the local rows into ``sums`` (float64 CUDA tensor)."""
+        m, n = X.shape
+        rc = lib().lr_shard_sums(self._h, _dev_ptr(X, torch.float32, "X"), _dev_ptr(y, torch.float32, "y"), m, n,
+                                 _dev_ptr(w, torch.float32, "w"), _dev_ptr(b, torch.float32, "b"),
+                                 _dev_ptr(sums, torch.float64, "sums"), self._stream())
+        self._check(rc, "lr_shard_sums")
+
+    def apply_sums(self, sums_all, m_total, lr, w, b, loss=None):
+        """Adds the ``parts`` rows of ``sums_all`` [parts, n+2] in order and applies the update to w, b in place."""
+        parts, n2 = sums_all.shape
+        rc = lib().lr_apply_sums(self._h, _dev_ptr(sums_all, torch.float64, "sums_all"), parts, int(m_total), n2 - 2,
+                                 float(lr), _dev_ptr(w, torch.float32, "w"), _dev_ptr(b, torch.float32, "b"),
+                                 _dev_ptr(loss, torch.float32, "loss"), self._stream())
+        self._check(rc, "lr_apply_sums")
 
     # ---- host-pointer entry points ---------------------------------------------------------------
     def fit_host(self, X, y, lr, iters, w, b, loss_hist=None):

@@ -16,12 +16,14 @@ using namespace lrgd;
 
 namespace {
 
-constexpr int kNW = 15;                        // consumer warps of the staged kernel (+1 producer warp = 512 threads)
-constexpr int kStageTargetBytes = 32 * 1024;
-constexpr int kStageBudgetBytes = 200 * 1024;  // shared memory the stage ring may take (227 KB per CTA on sm_100)
+constexpr int kNW = 16;                        // warps per CTA of the staged kernel (512 threads, one CTA per SM)
+constexpr int kStageBudgetBytes = 208 * 1024;  // shared memory the warps' stages may take (227 KB per CTA on sm_100)
 constexpr int kMaxGridPerSm = 8;               // widest launch any variant uses, in CTAs per SM
 constexpr int kMaxProfiled = 4096;
 constexpr int64_t kMaxRows = int64_t(1) << 40;
+#ifndef LRGD_NV2_RB
+#define LRGD_NV2_RB 4                          // register batch (rows per warp) of the 132..256-column instantiation
+#endif
 
 struct RowShape { int nv, lpr, rb; };
 
@@ -30,8 +32,8 @@ bool row_shape_for(int n4, RowShape* s) {
     if (n4 <= 8) *s = {1, 8, 8};
     else if (n4 <= 16) *s = {1, 16, 8};
     else if (n4 <= 32) *s = {1, 32, 8};
-    else if (n4 <= 64) *s = {2, 32, 8};
-    else if (n4 <= 128) *s = {4, 32, 4};
+    else if (n4 <= 64) *s = {2, 32, LRGD_NV2_RB};
+    else if (n4 <= 128) *s = {4, 32, 2};
     else return false;
     return true;
 }
@@ -42,31 +44,27 @@ int make_plan(int64_t m, int32_t n, bool aligned16, int32_t sms, lr_plan* P) {
     std::memset(P, 0, sizeof(*P));
     RowShape rs;
     if (aligned16 && n % 4 == 0 && row_shape_for(n / 4, &rs)) {
-        const int rpb = rs.rb * (32 / rs.lpr);
-        const int64_t row_bytes = int64_t(n) * 4;
-        const int64_t bpt_cap = std::max<int64_t>(1, kStageTargetBytes / (rpb * row_bytes));
-        const int64_t bpt_fill = (m + int64_t(sms) * rpb - 1) / (int64_t(sms) * rpb);   // spread small problems over all SMs
-        const int bpt = int(std::min(bpt_cap, std::max<int64_t>(1, bpt_fill)));
-        const int R = bpt * rpb;
-        const int64_t T = (m + R - 1) / R;
-        const int grid = int(std::min<int64_t>(T, sms));
-        const int64_t tiles_per_cta = (T + grid - 1) / grid;
-        const int64_t tile_stride = (R * row_bytes + 127) & ~int64_t(127);
-        const int64_t per_stage = tile_stride + int64_t(R) * 4;
-        int S = int(std::min<int64_t>(kMaxStages, kStageBudgetBytes / per_stage));
-        S = int(std::min<int64_t>(S, std::max<int64_t>(2, tiles_per_cta)));
-        if (S < 1) S = 1;
+        const int rpb = rs.rb * (32 / rs.lpr);                                  // rows per batch = rows per stage
+        const int64_t B = (m + rpb - 1) / rpb;                                  // batches
+        const int64_t slots = (B + kNW - 1) / kNW;                              // CTA-level groups of kNW batches
+        const int grid = int(std::min<int64_t>(slots, sms));
+        const int64_t per_warp = (slots + grid - 1) / grid;                     // most batches any warp handles
+        const int64_t x_stride = (int64_t(rpb) * n * 4 + 127) & ~int64_t(127);
+        const int64_t stage_stride = x_stride + ((int64_t(rpb) * 4 + 127) & ~int64_t(127));
+        int D = int(std::min<int64_t>(kMaxDepth, kStageBudgetBytes / (kNW * stage_stride)));
+        D = int(std::min<int64_t>(D, per_warp));
+        if (D < 1) D = 1;
         const int64_t combine = int64_t(kNW) * n * 8 + 2 * kNW * 8;
         P->variant = 0;
         P->lanes_per_row = rs.lpr;
         P->vec_per_lane = rs.nv;
         P->rows_per_batch = rpb;
-        P->tile_rows = R;
-        P->stages = S;
+        P->tile_rows = rpb;
+        P->stages = D;
         P->grid = grid;
-        P->threads = (kNW + 1) * 32;
-        P->smem_bytes = int(kHeaderBytes + std::max<int64_t>(S * per_stage, combine));
-        if (tiles_per_cta * bpt >= (int64_t(1) << 31)) return LR_ERR_SHAPE;
+        P->threads = kNW * 32;
+        P->smem_bytes = int(kHeaderBytes + std::max<int64_t>(int64_t(kNW) * D * stage_stride, combine));
+        if (per_warp >= (int64_t(1) << 31)) return LR_ERR_SHAPE;
         return LR_OK;
     }
     const int64_t nchunks = (m + kGenRows - 1) / kGenRows;
@@ -142,8 +140,8 @@ cudaError_t launch_rows(const lr_plan& P, const StreamParams& sp, cudaStream_t s
     if (P.lanes_per_row == 8) return launch_rows_t<1, 8, 8, PRED>(P, sp, st);
     if (P.lanes_per_row == 16) return launch_rows_t<1, 16, 8, PRED>(P, sp, st);
     if (P.vec_per_lane == 1) return launch_rows_t<1, 32, 8, PRED>(P, sp, st);
-    if (P.vec_per_lane == 2) return launch_rows_t<2, 32, 8, PRED>(P, sp, st);
-    return launch_rows_t<4, 32, 4, PRED>(P, sp, st);
+    if (P.vec_per_lane == 2) return launch_rows_t<2, 32, LRGD_NV2_RB, PRED>(P, sp, st);
+    return launch_rows_t<4, 32, 2, PRED>(P, sp, st);
 }
 
 struct Pass {
@@ -167,9 +165,9 @@ int launch_stream_pass(lr_ctx* ctx, const lr_plan& P, const Pass& a, uint8_t* la
         StreamParams sp;
         sp.X = a.X; sp.y = a.y; sp.m = a.m; sp.n = a.n; sp.w = a.w; sp.b = a.b;
         sp.partial = ctx->d_partial; sp.labels = labels; sp.cut = cut; sp.status = ctx->d_status;
-        sp.bpt = P.tile_rows / P.rows_per_batch; sp.stages = P.stages;
+        sp.depth = P.stages;
         sp.stage_y = (!predict && aligned(a.y, 16)) ? 1 : 0;
-        sp.num_tiles = (a.m + P.tile_rows - 1) / P.tile_rows;
+        sp.num_batches = (a.m + P.rows_per_batch - 1) / P.rows_per_batch;
         e = predict ? launch_rows<true>(P, sp, st) : launch_rows<false>(P, sp, st);
     } else {
         GenericParams gp;
@@ -188,11 +186,12 @@ int launch_stream_pass(lr_ctx* ctx, const lr_plan& P, const Pass& a, uint8_t* la
     return LR_OK;
 }
 
-int launch_reduce(lr_ctx* ctx, const lr_plan& P, int64_t m, int32_t n, double lr, bool update, float* w, float* b,
-                  float* grad_w, float* grad_b, float* loss_out, cudaStream_t st) {
+int launch_reduce(lr_ctx* ctx, const double* partial, int G, int64_t m, int32_t n, double lr, bool update, float* w,
+                  float* b, float* grad_w, float* grad_b, float* loss_out, double* raw_sums, cudaStream_t st) {
     ReduceParams rp;
-    rp.partial = ctx->d_partial; rp.G = P.grid; rp.n = n; rp.inv_m = 1.0 / double(m); rp.lr = lr;
+    rp.partial = partial; rp.G = G; rp.n = n; rp.inv_m = 1.0 / double(m); rp.lr = lr;
     rp.update = update ? 1 : 0; rp.w = w; rp.b = b; rp.grad_w = grad_w; rp.grad_b = grad_b; rp.loss_out = loss_out;
+    rp.raw_sums = raw_sums;
     dim3 block(32, kRedSlices);
     k_reduce_update<<<(n + 2 + 31) / 32, block, 0, st>>>(rp);
     LR_CK(ctx, cudaGetLastError());
@@ -289,7 +288,8 @@ int lr_loss_grad(lr_ctx* ctx, const float* d_X, const float* d_y, int64_t m, int
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     rc = launch_stream_pass(ctx, P, Pass{d_X, d_y, m, n, d_w, d_b}, nullptr, 0.f, st);
     if (rc != LR_OK) return rc;
-    return launch_reduce(ctx, P, m, n, 0.0, false, nullptr, nullptr, d_grad_w, d_grad_b, d_loss, st);
+    return launch_reduce(ctx, ctx->d_partial, P.grid, m, n, 0.0, false, nullptr, nullptr, d_grad_w, d_grad_b, d_loss,
+                         nullptr, st);
 }
 
 int lr_fit(lr_ctx* ctx, const float* d_X, const float* d_y, int64_t m, int32_t n, float lr, int32_t iters,
@@ -310,8 +310,8 @@ int lr_fit(lr_ctx* ctx, const float* d_X, const float* d_y, int64_t m, int32_t n
     for (int32_t t = 0; t < iters; ++t) {
         rc = launch_stream_pass(ctx, P, Pass{d_X, d_y, m, n, d_w, d_b}, nullptr, 0.f, st);
         if (rc != LR_OK) return rc;
-        rc = launch_reduce(ctx, P, m, n, double(lr), true, d_w, d_b, nullptr, nullptr,
-                           d_loss_hist ? d_loss_hist + t : nullptr, st);
+        rc = launch_reduce(ctx, ctx->d_partial, P.grid, m, n, double(lr), true, d_w, d_b, nullptr, nullptr,
+                           d_loss_hist ? d_loss_hist + t : nullptr, nullptr, st);
         if (rc != LR_OK) return rc;
     }
     return LR_OK;
@@ -330,6 +330,36 @@ int lr_predict(lr_ctx* ctx, const float* d_X, int64_t m, int32_t n, const float*
     if (!g.ok) return LR_ERR_CUDA;
     const float cut = static_cast<float>(std::log(double(thr) / (1.0 - double(thr))));
     return launch_stream_pass(ctx, P, Pass{d_X, nullptr, m, n, d_w, d_b}, d_labels, cut, static_cast<cudaStream_t>(stream));
+}
+
+int lr_shard_sums(lr_ctx* ctx, const float* d_X, const float* d_y, int64_t m_local, int32_t n, const float* d_w,
+                  const float* d_b, double* d_sums, void* stream) {
+    int rc = check_common(ctx, d_X, m_local, n, d_w, d_b);
+    if (rc != LR_OK) return rc;
+    if (!d_y || !d_sums) return LR_ERR_NULL;
+    if (!aligned(d_y, 4) || !aligned(d_sums, 8)) return LR_ERR_ALIGNMENT;
+    lr_plan P;
+    rc = make_plan(m_local, n, aligned(d_X, 16), ctx->sm_count, &P);
+    if (rc != LR_OK) return rc;
+    DeviceGuard g(ctx);
+    if (!g.ok) return LR_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    rc = launch_stream_pass(ctx, P, Pass{d_X, d_y, m_local, n, d_w, d_b}, nullptr, 0.f, st);
+    if (rc != LR_OK) return rc;
+    return launch_reduce(ctx, ctx->d_partial, P.grid, m_local, n, 0.0, false, nullptr, nullptr, nullptr, nullptr, nullptr,
+                         d_sums, st);
+}
+
+int lr_apply_sums(lr_ctx* ctx, const double* d_sums_all, int32_t parts, int64_t m_total, int32_t n, float lr, float* d_w,
+                  float* d_b, float* d_loss, void* stream) {
+    if (!ctx || !d_sums_all || !d_w || !d_b) return LR_ERR_NULL;
+    if (parts < 1 || m_total < 1 || n < 1 || n > ctx->n_max) return LR_ERR_SHAPE;
+    if (!aligned(d_sums_all, 8) || !aligned(d_w, 4) || !aligned(d_b, 4) || (d_loss && !aligned(d_loss, 4))) return LR_ERR_ALIGNMENT;
+    if (!std::isfinite(lr)) return LR_ERR_VALUE;
+    DeviceGuard g(ctx);
+    if (!g.ok) return LR_ERR_CUDA;
+    return launch_reduce(ctx, d_sums_all, parts, m_total, n, double(lr), true, d_w, d_b, nullptr, nullptr, d_loss, nullptr,
+                         static_cast<cudaStream_t>(stream));
 }
 
 int lr_fit_host(lr_ctx* ctx, const float* h_X, const float* h_y, int64_t m, int32_t n, float lr, int32_t iters,

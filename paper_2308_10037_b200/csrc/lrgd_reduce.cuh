@@ -23,6 +23,7 @@ struct ReduceParams {
     float* grad_w;
     float* grad_b;
     float* loss_out;          // nullable
+    double* raw_sums;         // non-null: write the unscaled fp64 sums [n+2] here and nothing else
 };
 
 __global__ void __launch_bounds__(32 * kRedSlices) k_reduce_update(const ReduceParams p) {
@@ -44,6 +45,10 @@ __global__ void __launch_bounds__(32 * kRedSlices) k_reduce_update(const ReduceP
     double t = 0.0;
 #pragma unroll
     for (int k = 0; k < kRedSlices; ++k) t += sh[k][threadIdx.x];
+    if (p.raw_sums) {
+        p.raw_sums[col] = t;
+        return;
+    }
     const double v = t * p.inv_m;
     if (col < p.n) {
         if (p.update) p.w[col] = static_cast<float>(static_cast<double>(p.w[col]) - p.lr * v);

@@ -57,13 +57,14 @@ def test_plan_staged_shapes(m, n, lpr, nv):
     p = api.plan_query(m, n)
     assert p["variant"] == 0 and p["lanes_per_row"] == lpr and p["vec_per_lane"] == nv
     assert p["threads"] == 512 and 1 <= p["grid"] <= 148
-    assert p["tile_rows"] % p["rows_per_batch"] == 0 and p["tile_rows"] % 4 == 0
-    assert p["tile_rows"] * n * 4 <= 32 * 1024 or p["tile_rows"] == p["rows_per_batch"]
-    assert 1 <= p["stages"] <= 8
+    assert p["tile_rows"] == p["rows_per_batch"]              # one stage holds one register batch
+    assert 1 <= p["stages"] <= 4
     assert p["smem_bytes"] <= 227 * 1024
-    # every row is covered by exactly one tile
-    tiles = -(-m // p["tile_rows"])
-    assert p["grid"] == min(tiles, 148)
+    stage = -(-p["tile_rows"] * n * 4 // 128) * 128 + 128
+    assert 1024 + 16 * p["stages"] * stage <= p["smem_bytes"]
+    # 16 warps per CTA take one batch each per round; the grid never exceeds the rounds available
+    batches = -(-m // p["rows_per_batch"])
+    assert p["grid"] == min(-(-batches // 16), 148)
 
 
 def test_plan_falls_back_for_unaligned_or_odd_shapes():
@@ -81,6 +82,8 @@ def test_plan_rejects_bad_shapes():
         assert e.value.code == api.LR_ERR_SHAPE
 
 
-def test_small_problems_spread_over_all_sms():
-    p = api.plan_query(10_000, 32, sm_count=148)
-    assert p["grid"] >= 100
+def test_pipeline_depth_follows_the_shared_memory_budget():
+    assert api.plan_query(4_000_000, 256)["stages"] == 3        # 4 KB batches: three per warp fit
+    assert api.plan_query(16_000_000, 64)["stages"] == 3
+    assert api.plan_query(1_000_000, 100)["stages"] == 4        # 3.2 KB batches
+    assert api.plan_query(100, 32)["stages"] == 1               # one batch per warp at most
