@@ -33,6 +33,9 @@ if ROOT not in sys.path:
 METRIC = "GD iterations/sec (full-batch, m x n fp32)"
 UNIT = "iterations/s"
 NOMINAL_HBM_GBS = 8000.0
+# dram__bytes_read.sum + dram__bytes_write.sum of the streaming kernel per row of X, from the ncu capture summarised in
+# profiles/ (taken at m = 500,000 and scaled by rows).  Remove an entry when its kernel changes.
+NCU_TRAFFIC_BYTES_PER_ROW = {"cfg3": (514.026752e6 + 3.22944e6) / 500_000}
 FALLBACK_HBM_GBS = 6650.0
 
 
@@ -266,7 +269,8 @@ def main():
     achieved = bytes_per_launch / (k1_ms * 1e-3) / 1e9
     peak, peak_kind = measured_hbm_peak()
     roofline = {"bound": "hbm", "kernel": "k_stream_rows (fused loss/gradient pass)", "achieved": achieved, "peak": peak,
-                "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "traffic": None,
+                "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
+                "traffic": (NCU_TRAFFIC_BYTES_PER_ROW[args.workload] * wl.m if args.workload in NCU_TRAFFIC_BYTES_PER_ROW else None),
                 "bytes_per_launch": bytes_per_launch, "avg_launch_ms": k1_ms, "launches_timed": n_l,
                 "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS}
 
