@@ -150,6 +150,36 @@ int lr_last_device_status(lr_ctx* ctx, int32_t* out);
 /* The cudaError_t value of the most recent failing CUDA call made through this context (0 if none). */
 int lr_last_cuda_error(lr_ctx* ctx);
 
+/*
+ * lr_loss_grad without any allocation.  (The paper has no counterpart; this exists for callers that
+ * must not allocate.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits -- a latency-critical loop that cannot
+ * afford the allocator's lock or the device-wide synchronisation a cudaFree brings; a process whose
+ * device memory has been handed in full to another allocator (a framework's caching pool), where a
+ * late cudaMalloc can fail; a plug-in whose host forbids allocation after start-up.  lr_create
+ * allocates a workspace, so those callers cannot use a context.
+ *
+ * Same computation and outputs as lr_loss_grad (d_loss[1], d_grad_w[n], d_grad_b[1]; inputs read only),
+ * but no lr_ctx: the per-CTA partial sums go to a fixed array that is part of the library's device
+ * image (about 2 MiB on every GPU that loads the library, until the process exits).  The call makes no
+ * cudaMalloc / cudaFree and calls no allocating routine.
+ *
+ * Limits: n <= LR_NOALLOC_MAX_N (else LR_ERR_SHAPE, nothing launched); device index < 64.
+ * d_status is NULL or a device int32 that the call zeroes and the kernel sets to LR_ERR_TIMEOUT if a
+ * bounded device-side wait expires (read it after synchronising the stream).
+ * First call on a device: resolves the array's device address and reads the SM count; make that first
+ * call outside any stream capture.
+ * Sharing: every call on a device uses the same array and finds the previous call's contents in it;
+ * the call clears what has to start from zero itself.  Two calls that overlap on the GPU (different
+ * streams, or different host threads without ordering) race on the array -- order them on one stream
+ * or with events.
+ */
+#define LR_NOALLOC_MAX_N 1022
+int lr_loss_grad_noalloc(int32_t device, const float* d_X, const float* d_y, int64_t m, int32_t n,
+                         const float* d_w, const float* d_b,
+                         float* d_loss, float* d_grad_w, float* d_grad_b, int32_t* d_status, void* stream);
+
 /* Static description of a status code. */
 const char* lr_status_string(int code);
 

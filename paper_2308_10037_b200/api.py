@@ -21,7 +21,7 @@ LR_ERR_NULL, LR_ERR_SHAPE, LR_ERR_ALIGNMENT, LR_ERR_VALUE, LR_ERR_CUDA, LR_ERR_T
 EXPORTS = ["lr_plan_query", "lr_create", "lr_destroy", "lr_loss_grad", "lr_fit", "lr_predict", "lr_shard_sums",
            "lr_apply_sums", "lr_fit_host",
            "lr_predict_host", "lr_profile_enable", "lr_profile_read", "lr_launch_count", "lr_last_device_status",
-           "lr_last_cuda_error", "lr_status_string"]
+           "lr_last_cuda_error", "lr_status_string", "lr_loss_grad_noalloc"]
 
 
 class LrPlan(ctypes.Structure):
@@ -58,6 +58,7 @@ def lib() -> ctypes.CDLL:
         L.lr_predict.argtypes = [P, P, I64, I32, P, P, F, P, P]
         L.lr_shard_sums.argtypes = [P, P, P, I64, I32, P, P, P, P]
         L.lr_apply_sums.argtypes = [P, P, I32, I64, I32, F, P, P, P, P]
+        L.lr_loss_grad_noalloc.argtypes = [I32, P, P, I64, I32, P, P, P, P, P, P, P]
         L.lr_fit_host.argtypes = [P, P, P, I64, I32, F, I32, P, P, P]
         L.lr_predict_host.argtypes = [P, P, I64, I32, P, P, F, P]
         L.lr_profile_enable.argtypes = [P, I32]
@@ -260,3 +261,26 @@ def lr_fit(X, y, lr, iters, w0=None, b0=None, return_history=False, ctx: Context
 def lr_predict(X, w, b, thr, ctx: Context | None = None):
     """uint8 CUDA tensor [m]: 1 where sigmoid(x.w + b) >= thr."""
     return _ctx_for(X, ctx).predict(X, w, _as_b(b, X.device), thr)
+
+
+LR_NOALLOC_MAX_N = 1022
+
+
+def lr_loss_grad_noalloc(X, y, w, b, loss, grad_w, grad_b, status=None):
+    """Allocation-free ``lr_loss_grad``: no context, no workspace allocation inside the library.
+
+    For callers that cannot allocate device memory when they call (latency-critical loops, processes whose
+    device memory is fully owned by another allocator, hosts with a no-allocation-after-start rule).  The
+    caller passes every buffer, outputs included: ``loss`` [1], ``grad_w`` [n], ``grad_b`` [1] float32 and
+    optionally ``status`` [1] int32, all CUDA tensors that already exist.  Scratch lives in a fixed array
+    inside the library (n <= LR_NOALLOC_MAX_N); calls that overlap on the GPU race on it.
+    """
+    m, n = X.shape
+    dev = X.device.index if X.device.index is not None else torch.cuda.current_device()
+    rc = lib().lr_loss_grad_noalloc(int(dev), _dev_ptr(X, torch.float32, "X"), _dev_ptr(y, torch.float32, "y"), m, n,
+                                    _dev_ptr(w, torch.float32, "w"), _dev_ptr(b, torch.float32, "b"),
+                                    _dev_ptr(loss, torch.float32, "loss"), _dev_ptr(grad_w, torch.float32, "grad_w"),
+                                    _dev_ptr(grad_b, torch.float32, "grad_b"), _dev_ptr(status, torch.int32, "status"),
+                                    ctypes.c_void_p(torch.cuda.current_stream(dev).cuda_stream))
+    if rc != LR_OK:
+        raise LrError(rc, "lr_loss_grad_noalloc")

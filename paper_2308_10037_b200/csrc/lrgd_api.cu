@@ -5,6 +5,7 @@
 #include <cmath>
 #include <cstdlib>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <vector>
 
@@ -481,3 +482,95 @@ const char* lr_status_string(int code) {
 }
 
 }  // extern "C"
+
+// ------------------------------------------------------------------------------------------------------
+// Allocation-free loss/gradient pass.  The per-CTA partial sums that lr_loss_grad keeps in a context's
+// cudaMalloc'ed workspace live here in a fixed array inside the library's device image instead.
+// ------------------------------------------------------------------------------------------------------
+namespace {
+
+constexpr int kNoAllocMaxGrid = 256;                                    // CTAs
+constexpr int kNoAllocRowDoubles = LR_NOALLOC_MAX_N + 2;                // one partial row: n columns, sum err, sum loss
+constexpr size_t kNoAllocScratchDoubles = size_t(kNoAllocMaxGrid) * kNoAllocRowDoubles + 2;   // + status word slot
+
+// 2 MiB + 16 B on every GPU that loads the library, for the life of the process.
+static __device__ __align__(256) double g_noalloc_scratch[kNoAllocScratchDoubles];
+
+constexpr int kNoAllocMaxDevices = 64;
+struct NoAllocDevice {
+    double* scratch = nullptr;      // device address of g_noalloc_scratch on this device (NOT the host-side symbol)
+    int sm_count = 0;
+};
+NoAllocDevice g_noalloc_dev[kNoAllocMaxDevices];
+std::mutex g_noalloc_mutex;
+
+// First use on `device` (which must be current): resolve the symbol to its device address and cache it.
+int noalloc_setup(int device, NoAllocDevice** out) {
+    if (device < 0 || device >= kNoAllocMaxDevices) return LR_ERR_SHAPE;
+    std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+    NoAllocDevice& d = g_noalloc_dev[device];
+    if (!d.scratch) {
+        double* ptr = nullptr;
+        if (cudaGetSymbolAddress(reinterpret_cast<void**>(&ptr), g_noalloc_scratch) != cudaSuccess || !ptr) return LR_ERR_CUDA;
+        int sms = 0;
+        if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device) != cudaSuccess || sms < 1) return LR_ERR_CUDA;
+        d.sm_count = sms;
+        d.scratch = ptr;
+    }
+    *out = &d;
+    return LR_OK;
+}
+
+}  // namespace
+
+extern "C" int lr_loss_grad_noalloc(int32_t device, const float* d_X, const float* d_y, int64_t m, int32_t n,
+                                    const float* d_w, const float* d_b, float* d_loss, float* d_grad_w, float* d_grad_b,
+                                    int32_t* d_status, void* stream) {
+    if (!d_X || !d_y || !d_w || !d_b || !d_loss || !d_grad_w || !d_grad_b) return LR_ERR_NULL;
+    if (m < 1 || m > kMaxRows || n < 1) return LR_ERR_SHAPE;
+    if (n > LR_NOALLOC_MAX_N) return LR_ERR_SHAPE;                      // the fixed scratch holds rows of at most this many columns
+    if (!aligned(d_X, 4) || !aligned(d_y, 4) || !aligned(d_w, 4) || !aligned(d_b, 4) || !aligned(d_loss, 4) ||
+        !aligned(d_grad_w, 4) || !aligned(d_grad_b, 4) || (d_status && !aligned(d_status, 4)))
+        return LR_ERR_ALIGNMENT;
+    int prev = -1;
+    cudaGetDevice(&prev);
+    if (cudaSetDevice(device) != cudaSuccess) return LR_ERR_CUDA;
+    struct Restore { int p; ~Restore() { if (p >= 0) cudaSetDevice(p); } } restore{prev};
+
+    NoAllocDevice* dev = nullptr;
+    int rc = noalloc_setup(device, &dev);
+    if (rc != LR_OK) return rc;
+    lr_plan P;
+    rc = make_plan(m, n, aligned(d_X, 16), dev->sm_count, &P);
+    if (rc != LR_OK) return rc;
+    if (P.grid > kNoAllocMaxGrid) P.grid = kNoAllocMaxGrid;            // only the unstaged kernel asks for more; it strides over its chunks
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    double* partial = dev->scratch;
+    int* status = d_status ? d_status : reinterpret_cast<int*>(dev->scratch + size_t(kNoAllocMaxGrid) * kNoAllocRowDoubles);
+    // the array keeps whatever the previous call left: the status word must start at zero (the partial rows are
+    // fully rewritten by the CTAs that the reduction reads)
+    if (cudaMemsetAsync(status, 0, sizeof(int), st) != cudaSuccess) return LR_ERR_CUDA;
+    cudaError_t e;
+    if (P.variant == 0) {
+        StreamParams sp;
+        sp.X = d_X; sp.y = d_y; sp.m = m; sp.n = n; sp.w = d_w; sp.b = d_b;
+        sp.partial = partial; sp.labels = nullptr; sp.cut = 0.f; sp.status = status;
+        sp.depth = P.stages;
+        sp.stage_y = aligned(d_y, 16) ? 1 : 0;
+        sp.num_batches = (m + P.rows_per_batch - 1) / P.rows_per_batch;
+        e = launch_rows<false>(P, sp, st);
+    } else {
+        GenericParams gp;
+        gp.X = d_X; gp.y = d_y; gp.m = m; gp.n = n; gp.w = d_w; gp.b = d_b;
+        gp.partial = partial; gp.labels = nullptr; gp.cut = 0.f;
+        k_generic<false><<<P.grid, P.threads, 0, st>>>(gp);
+        e = cudaGetLastError();
+    }
+    if (e != cudaSuccess) return LR_ERR_CUDA;
+    ReduceParams rp;
+    rp.partial = partial; rp.G = P.grid; rp.n = n; rp.inv_m = 1.0 / double(m); rp.lr = 0.0; rp.update = 0;
+    rp.w = nullptr; rp.b = nullptr; rp.grad_w = d_grad_w; rp.grad_b = d_grad_b; rp.loss_out = d_loss; rp.raw_sums = nullptr;
+    k_reduce_update<<<(n + 2 + 31) / 32, dim3(32, kRedSlices), 0, st>>>(rp);
+    if (cudaGetLastError() != cudaSuccess) return LR_ERR_CUDA;
+    return LR_OK;
+}
