@@ -14,7 +14,7 @@ from paper_2308_10037_b200 import api, datagen
 
 pytestmark = pytest.mark.gpu
 
-GRAD_TOL, LOSS_TOL, W_TOL, LABEL_AGREE = 1e-5, 1e-6, 1e-4, 0.9999
+from _parity import GRAD_TOL, LABEL_AGREE, LOSS_TOL, W_TOL, assert_grad_close, grad_noise_floor, rel_l2
 
 
 @pytest.fixture(scope="module")
@@ -29,11 +29,6 @@ def ctx():
 
 def dev(a):
     return torch.from_numpy(np.ascontiguousarray(a)).cuda()
-
-
-def rel_l2(a, b):
-    a, b = np.asarray(a, dtype=np.float64).ravel(), np.asarray(b, dtype=np.float64).ravel()
-    return float(np.linalg.norm(a - b) / max(np.linalg.norm(b), 1e-300))
 
 
 def check_loss_grad(ctx, X, y, w, b, grad_tol=GRAD_TOL, loss_tol=LOSS_TOL):
@@ -105,6 +100,7 @@ def test_teacher_forced_trajectory(ctx, name, m):
     iters = min(wl.iters, 40)
     _, _, lh, wh, bh = oracle.fit(X, y, wl.lr, iters, history=True)
     dX, dy = dev(X), dev(y)
+    floor = grad_noise_floor(X)
     for t in sorted({0, 1, 2, iters // 2, iters - 1}):
         w32 = wh[t].astype(np.float32)
         b32 = np.float32(bh[t])
@@ -112,7 +108,7 @@ def test_teacher_forced_trajectory(ctx, name, m):
         dl, dg, dg0 = ctx.loss_grad(dX, dy, dev(w32), dev(np.array([b32])))
         assert abs(dl.item() - L) <= LOSS_TOL, (t, dl.item(), L)
         got = np.concatenate([dg.cpu().numpy(), dg0.cpu().numpy()])
-        assert rel_l2(got, np.concatenate([g, [g0]])) <= GRAD_TOL, t
+        assert_grad_close(got, np.concatenate([g, [g0]]), floor, (name, t))
 
 
 @pytest.mark.parametrize("name,m", SMALL_WORKLOADS)
