@@ -51,7 +51,7 @@ typedef struct lr_ctx lr_ctx;
 /* Launch plan for a given shape, as chosen by the host logic (pure host code, no CUDA call). */
 typedef struct lr_plan {
     int32_t variant;       /* 0 = row-per-lane-group staged kernel, 1 = row-split staged kernel, 2 = unstaged generic kernel */
-    int32_t lanes_per_row; /* staged kernels: lanes that share one row (8, 16, 32; 256 for the row-split kernel) */
+    int32_t lanes_per_row; /* staged kernels: lanes that share one row (8, 16, 32; 512 for the row-split kernel) */
     int32_t vec_per_lane;  /* staged kernels: 16-byte column groups owned by one lane */
     int32_t rows_per_batch;/* rows one warp (or one CTA for the row-split kernel) holds in registers at a time */
     int32_t tile_rows;     /* rows per asynchronously staged shared-memory stage */

@@ -12,6 +12,7 @@
 #include "lrgd_generic.cuh"
 #include "lrgd_reduce.cuh"
 #include "lrgd_stream_rows.cuh"
+#include "lrgd_stream_split.cuh"
 
 using namespace lrgd;
 
@@ -66,6 +67,31 @@ int make_plan(int64_t m, int32_t n, bool aligned16, int32_t sms, lr_plan* P) {
         P->threads = kNW * 32;
         P->smem_bytes = int(kHeaderBytes + std::max<int64_t>(int64_t(kNW) * D * stage_stride, combine));
         if (per_warp >= (int64_t(1) << 31)) return LR_ERR_SHAPE;
+        return LR_OK;
+    }
+    if (aligned16 && n % 4 == 0 && n / 4 <= kNW * 64) {
+        // wide rows: the warps of a CTA split each row by columns
+        const int cw = (n / 4 + kNW - 1) / kNW;                                 // 16-byte column groups per warp slice
+        const int nv = cw > 32 ? 2 : 1;
+        const int rb = nv == 2 ? 4 : 8;
+        const int64_t B = (m + rb - 1) / rb;
+        const int grid = int(std::min<int64_t>(B, sms));
+        const int64_t per_cta = (B + grid - 1) / grid;
+        const int64_t row_stride = (int64_t(cw) * 16 + 127) & ~int64_t(127);
+        const int64_t stage_stride = rb * row_stride;
+        int D = int(std::min<int64_t>(kMaxDepth, kStageBudgetBytes / (kNW * stage_stride)));
+        D = int(std::min<int64_t>(D, per_cta));
+        if (D < 1) D = 1;
+        P->variant = 1;
+        P->lanes_per_row = kNW * 32;
+        P->vec_per_lane = nv;
+        P->rows_per_batch = rb;
+        P->tile_rows = rb;
+        P->stages = D;
+        P->grid = grid;
+        P->threads = kNW * 32;
+        P->smem_bytes = int(kSplitHeaderBytes + int64_t(kNW) * D * stage_stride);
+        if (per_cta >= (int64_t(1) << 31)) return LR_ERR_SHAPE;
         return LR_OK;
     }
     const int64_t nchunks = (m + kGenRows - 1) / kGenRows;
@@ -145,6 +171,21 @@ cudaError_t launch_rows(const lr_plan& P, const StreamParams& sp, cudaStream_t s
     return launch_rows_t<4, 32, 2, PRED>(P, sp, st);
 }
 
+template <int NV, int RB, bool PRED>
+cudaError_t launch_split_t(const lr_plan& P, const SplitParams& sp, cudaStream_t st) {
+    auto kern = k_stream_split<NV, RB, kNW, PRED>;
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, P.smem_bytes);
+    if (e != cudaSuccess) return e;
+    kern<<<P.grid, P.threads, P.smem_bytes, st>>>(sp);
+    return cudaGetLastError();
+}
+
+template <bool PRED>
+cudaError_t launch_split(const lr_plan& P, const SplitParams& sp, cudaStream_t st) {
+    if (P.vec_per_lane == 2) return launch_split_t<2, 4, PRED>(P, sp, st);
+    return launch_split_t<1, 8, PRED>(P, sp, st);
+}
+
 struct Pass {
     const float* X; const float* y; int64_t m; int32_t n; const float* w; const float* b;
 };
@@ -170,6 +211,14 @@ int launch_stream_pass(lr_ctx* ctx, const lr_plan& P, const Pass& a, uint8_t* la
         sp.stage_y = (!predict && aligned(a.y, 16)) ? 1 : 0;
         sp.num_batches = (a.m + P.rows_per_batch - 1) / P.rows_per_batch;
         e = predict ? launch_rows<true>(P, sp, st) : launch_rows<false>(P, sp, st);
+    } else if (P.variant == 1) {
+        SplitParams sp;
+        sp.X = a.X; sp.y = a.y; sp.m = a.m; sp.n = a.n; sp.w = a.w; sp.b = a.b;
+        sp.partial = ctx->d_partial; sp.labels = labels; sp.cut = cut; sp.status = ctx->d_status;
+        sp.depth = P.stages;
+        sp.cw = (a.n / 4 + kNW - 1) / kNW;
+        sp.num_batches = (a.m + P.rows_per_batch - 1) / P.rows_per_batch;
+        e = predict ? launch_split<true>(P, sp, st) : launch_split<false>(P, sp, st);
     } else {
         GenericParams gp;
         gp.X = a.X; gp.y = a.y; gp.m = a.m; gp.n = a.n; gp.w = a.w; gp.b = a.b;
@@ -559,6 +608,14 @@ extern "C" int lr_loss_grad_noalloc(int32_t device, const float* d_X, const floa
         sp.stage_y = aligned(d_y, 16) ? 1 : 0;
         sp.num_batches = (m + P.rows_per_batch - 1) / P.rows_per_batch;
         e = launch_rows<false>(P, sp, st);
+    } else if (P.variant == 1) {
+        SplitParams sp;
+        sp.X = d_X; sp.y = d_y; sp.m = m; sp.n = n; sp.w = d_w; sp.b = d_b;
+        sp.partial = partial; sp.labels = nullptr; sp.cut = 0.f; sp.status = status;
+        sp.depth = P.stages;
+        sp.cw = (n / 4 + kNW - 1) / kNW;
+        sp.num_batches = (m + P.rows_per_batch - 1) / P.rows_per_batch;
+        e = launch_split<false>(P, sp, st);
     } else {
         GenericParams gp;
         gp.X = d_X; gp.y = d_y; gp.m = m; gp.n = n; gp.w = d_w; gp.b = d_b;

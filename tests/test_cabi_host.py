@@ -75,6 +75,16 @@ def test_plan_falls_back_for_unaligned_or_odd_shapes():
     assert g["grid"] == 2 and g["threads"] == 256
 
 
+@pytest.mark.parametrize("m,n,nv,rb", [(100_000, 4096, 2, 4), (5000, 1024, 1, 8), (5000, 516, 1, 8), (5000, 2052, 2, 4)])
+def test_plan_wide_rows_are_split_across_warps(m, n, nv, rb):
+    p = api.plan_query(m, n)
+    assert p["variant"] == 1 and p["vec_per_lane"] == nv and p["rows_per_batch"] == rb
+    assert p["threads"] == 512 and p["grid"] == min(-(-m // rb), 148)
+    cw = -(-(n // 4) // 16)
+    stage = rb * (-(-cw * 16 // 128) * 128)
+    assert 1 <= p["stages"] <= 4 and p["smem_bytes"] == 2048 + 16 * p["stages"] * stage <= 227 * 1024
+
+
 def test_plan_rejects_bad_shapes():
     for m, n in [(0, 4), (4, 0), (-1, 4), (1 << 41, 4)]:
         with pytest.raises(api.LrError) as e:

@@ -1,6 +1,7 @@
 """GPU parity: the CUDA path, called through the C-ABI binding, against the float64 CPU checker on the
 same seeded inputs.  Tolerances (fp32 storage and accumulation against float64):
-  gradient (grad_w, grad_b stacked) relative L2 <= 1e-5, loss absolute <= 1e-6,
+  gradient (grad_w, grad_b stacked) relative L2 <= 1e-5 (with the fp32 noise floor of ``_parity`` at converged
+  iterates), loss absolute <= 1e-6,
   final parameters after a fit relative L2 <= 1e-4, predicted labels agreeing on >= 99.99 % of rows.
 """
 import math
@@ -46,7 +47,9 @@ def check_loss_grad(ctx, X, y, w, b, grad_tol=GRAD_TOL, loss_tol=LOSS_TOL):
 SHAPES = [(1, 4), (7, 4), (8, 3), (33, 28), (1000, 32), (4097, 32), (5003, 64), (2500, 36), (3001, 100), (9999, 256),
           (777, 200), (1500, 512), (2049, 260), (640, 30), (1025, 101), (300, 1), (130, 4096), (50, 8192), (20011, 8),
           # enough rows that every warp refills its shared-memory stages many times, with a ragged last batch
-          (200_003, 256), (400_001, 32), (200_002, 64), (120_007, 100), (150_001, 28), (60_001, 512), (90_001, 200)]
+          (200_003, 256), (400_001, 32), (200_002, 64), (120_007, 100), (150_001, 28), (60_001, 512), (90_001, 200),
+          # wide rows split across the warps of a CTA: full and partly idle warp slices, ragged last batch, stage reuse
+          (5_001, 4096), (20_003, 1024), (2_500, 516), (1_203, 2052), (701, 4092), (9_000, 2048), (3, 4096)]
 
 
 @pytest.mark.parametrize("m,n", SHAPES)
@@ -144,7 +147,8 @@ def test_fit_is_deterministic_and_resumable(ctx):
     assert not w0.any() and not b0.any()
 
 
-@pytest.mark.parametrize("m,n", [(5003, 64), (9999, 256), (3001, 100), (640, 30), (130, 4096), (33, 28)])
+@pytest.mark.parametrize("m,n", [(5003, 64), (9999, 256), (3001, 100), (640, 30), (130, 4096), (33, 28), (4001, 1028),
+                                 (50, 8192)])
 def test_predict_matches_oracle(ctx, m, n):
     X, y, w, b = datagen.random_problem(m, n, seed=50 + n, wscale=2.0)
     dX, dw, db = dev(X), dev(w), dev(np.array([b], dtype=np.float32))

@@ -58,7 +58,8 @@ def test_two_calls_in_a_row_match_the_context_entry_point():
         # shapes served by the other kernel variants, again back to back
         _run_pair(ctx, 70_003, 32, seed=903)
         _run_pair(ctx, 20_000, 30, seed=904)        # n % 4 != 0: unstaged kernel, its grid is capped by the array size
-        _run_pair(ctx, 900, 1020, seed=905)
+        _run_pair(ctx, 900, 1020, seed=905)         # wide rows: the row-split kernel
+        _run_pair(ctx, 800, 1022, seed=906)
         assert ctx.device_status() == 0
     finally:
         ctx.close()
