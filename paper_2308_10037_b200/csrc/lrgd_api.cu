@@ -18,7 +18,10 @@ using namespace lrgd;
 
 namespace {
 
-constexpr int kNW = 16;                        // warps per CTA of the staged kernel (512 threads, one CTA per SM)
+#ifndef LRGD_NW
+#define LRGD_NW 16
+#endif
+constexpr int kNW = LRGD_NW;                   // warps per CTA of the staged kernels (512 threads, one CTA per SM)
 constexpr int kStageBudgetBytes = 208 * 1024;  // shared memory the warps' stages may take (227 KB per CTA on sm_100)
 constexpr int kMaxGridPerSm = 8;               // widest launch any variant uses, in CTAs per SM
 constexpr int kMaxProfiled = 4096;
@@ -51,8 +54,7 @@ int make_plan(int64_t m, int32_t n, bool aligned16, int32_t sms, lr_plan* P) {
         const int64_t slots = (B + kNW - 1) / kNW;                              // CTA-level groups of kNW batches
         const int grid = int(std::min<int64_t>(slots, sms));
         const int64_t per_warp = (slots + grid - 1) / grid;                     // most batches any warp handles
-        const int64_t x_stride = (int64_t(rpb) * n * 4 + 127) & ~int64_t(127);
-        const int64_t stage_stride = x_stride + ((int64_t(rpb) * 4 + 127) & ~int64_t(127));
+        const int64_t stage_stride = (int64_t(rpb) * n * 4 + 127) & ~int64_t(127);
         int D = int(std::min<int64_t>(kMaxDepth, kStageBudgetBytes / (kNW * stage_stride)));
         D = int(std::min<int64_t>(D, per_warp));
         if (D < 1) D = 1;
@@ -208,7 +210,6 @@ int launch_stream_pass(lr_ctx* ctx, const lr_plan& P, const Pass& a, uint8_t* la
         sp.X = a.X; sp.y = a.y; sp.m = a.m; sp.n = a.n; sp.w = a.w; sp.b = a.b;
         sp.partial = ctx->d_partial; sp.labels = labels; sp.cut = cut; sp.status = ctx->d_status;
         sp.depth = P.stages;
-        sp.stage_y = (!predict && aligned(a.y, 16)) ? 1 : 0;
         sp.num_batches = (a.m + P.rows_per_batch - 1) / P.rows_per_batch;
         e = predict ? launch_rows<true>(P, sp, st) : launch_rows<false>(P, sp, st);
     } else if (P.variant == 1) {
@@ -605,7 +606,6 @@ extern "C" int lr_loss_grad_noalloc(int32_t device, const float* d_X, const floa
         sp.X = d_X; sp.y = d_y; sp.m = m; sp.n = n; sp.w = d_w; sp.b = d_b;
         sp.partial = partial; sp.labels = nullptr; sp.cut = 0.f; sp.status = status;
         sp.depth = P.stages;
-        sp.stage_y = aligned(d_y, 16) ? 1 : 0;
         sp.num_batches = (m + P.rows_per_batch - 1) / P.rows_per_batch;
         e = launch_rows<false>(P, sp, st);
     } else if (P.variant == 1) {

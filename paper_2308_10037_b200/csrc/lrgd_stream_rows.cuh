@@ -2,7 +2,8 @@
 //
 // Every warp runs its own small asynchronous pipeline: it owns `depth` shared-memory stages, each the
 // size of one batch of rows, and its elected lane keeps them filled with 1-D bulk asynchronous copies
-// (contiguous row ranges of X plus the matching slice of y) that complete on the warp's own mbarriers.
+// (contiguous row ranges of X) that complete on the warp's own mbarriers.  The few y values of a batch are
+// read with a plain load issued one batch ahead (a second, tiny bulk copy per batch measurably slows the stream).
 // Stages are never shared between warps, so a barrier only ever sees consecutive fills from one
 // waiter and its one-bit phase parity is unambiguous; there is no producer warp and no release barrier.
 // Per batch the warp
@@ -39,7 +40,6 @@ struct StreamParams {
     float cut;                // predict: logit(thr)
     int* status;              // device status word
     int depth;                // stages per warp (1..kMaxDepth)
-    int stage_y;              // 1: y slices are staged with the batch (y 16-byte aligned)
     long long num_batches;    // ceil(m / rows per batch)
 };
 
@@ -74,7 +74,6 @@ __global__ void __launch_bounds__(NW * 32, 1) k_stream_rows(const StreamParams p
     constexpr int LOG_RB = Log2<RB>::value;
     constexpr int SHIFT = LOG_LPR - LOG_RB;        // duplicate lanes per row after the reduction = 2^SHIFT
     static_assert(SHIFT >= 0, "rows per batch slot must not exceed lanes per row");
-    constexpr bool kCanStageY = RPB % 4 == 0;      // a staged y slice must be a multiple of 16 bytes
     static_assert(NW * kMaxDepth * 8 + 16 <= kHeaderBytes, "header too small");
     constexpr unsigned FULL = 0xffffffffu;
 
@@ -86,8 +85,7 @@ __global__ void __launch_bounds__(NW * 32, 1) k_stream_rows(const StreamParams p
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int D = p.depth;
     const int n = p.n, n4 = n >> 2;
-    const uint32_t x_stride = (static_cast<uint32_t>(RPB) * n * 4u + 127u) & ~127u;
-    const uint32_t stage_stride = x_stride + ((RPB * 4u + 127u) & ~127u);
+    const uint32_t stage_stride = (static_cast<uint32_t>(RPB) * n * 4u + 127u) & ~127u;
     unsigned char* my_stages = data + static_cast<size_t>(warp) * D * stage_stride;
     uint64_t* my_bars = bars + warp * kMaxDepth;
 
@@ -104,17 +102,15 @@ __global__ void __launch_bounds__(NW * 32, 1) k_stream_rows(const StreamParams p
     __syncthreads();
 
     const uint64_t pol = l2_policy_evict_first();
-    // (re)fills stage d with this warp's i-th batch; called by lane 0 only
-    auto issue = [&](int i, int d) {
-        const long long row0 = ((static_cast<long long>(i) * gridDim.x + blockIdx.x) * NW + warp) * RPB;
-        const long long left = p.m - row0;
-        const int rows = left < RPB ? static_cast<int>(left) : RPB;
-        const uint32_t xbytes = static_cast<uint32_t>(rows) * n * 4u;
-        const bool with_y = !PREDICT && kCanStageY && p.stage_y && rows == RPB;
-        unsigned char* dst = my_stages + static_cast<size_t>(d) * stage_stride;
-        mbar_arrive_expect_tx(&my_bars[d], xbytes + (with_y ? RPB * 4u : 0u));
-        bulk_copy_g2s(dst, p.X + row0 * n, xbytes, &my_bars[d], pol);
-        if (with_y) bulk_copy_g2s(dst + x_stride, p.y + row0, RPB * 4u, &my_bars[d], pol);
+    const long long stride_rows = static_cast<long long>(gridDim.x) * NW * RPB;       // rows between this warp's batches
+    long long row0 = (static_cast<long long>(blockIdx.x) * NW + warp) * RPB;          // first row of the current batch
+    // (re)fills stage d with the batch that starts at row r0; called by lane 0 only
+    auto issue = [&](long long r0, int d) {
+        const long long left = p.m - r0;
+        const uint32_t rows = left < RPB ? static_cast<uint32_t>(left) : RPB;
+        const uint32_t xbytes = rows * n * 4u;
+        mbar_arrive_expect_tx(&my_bars[d], xbytes);
+        bulk_copy_g2s(my_stages + static_cast<size_t>(d) * stage_stride, p.X + r0 * n, xbytes, &my_bars[d], pol);
     };
 
     float4 acc[NV];
@@ -142,8 +138,13 @@ __global__ void __launch_bounds__(NW * 32, 1) k_stream_rows(const StreamParams p
 
     if (lane == 0) {
         const int pre = cnt < D ? cnt : D;
-        for (int d = 0; d < pre; ++d) issue(d, d);
+        for (int d = 0; d < pre; ++d) issue(row0 + d * stride_rows, d);
     }
+    float y_next = 0.f;                            // y of this lane's row in the next batch, loaded one batch ahead
+    if constexpr (!PREDICT) {
+        if (cnt > 0 && row0 + myr < p.m) y_next = __ldg(p.y + row0 + myr);
+    }
+    const bool full_cols = n4 == NV * LPR;         // every lane's column groups exist
     int issued = cnt < D ? cnt : D;                // warp-uniform count of batches whose copies were issued
     int done = 0;                                  // batches whose stage wait has succeeded
     int since_flush = 0;
@@ -156,33 +157,38 @@ __global__ void __launch_bounds__(NW * 32, 1) k_stream_rows(const StreamParams p
         if (!ok) break;
         done = i + 1;
 
-        const long long row0 = ((static_cast<long long>(i) * gridDim.x + blockIdx.x) * NW + warp) * RPB;
         const long long left = p.m - row0;
         const int rows = left < RPB ? static_cast<int>(left) : RPB;
-        const unsigned char* stage = my_stages + static_cast<size_t>(d) * stage_stride;
-        const float4* t4 = reinterpret_cast<const float4*>(stage);
+        const float4* t4 = reinterpret_cast<const float4*>(my_stages + static_cast<size_t>(d) * stage_stride);
         float4 x[RB][NV];
+        if (full_cols && rows == RPB) {
 #pragma unroll
-        for (int r8 = 0; r8 < RB; ++r8) {
-            const int r = r8 * RPW + slot;
+            for (int r8 = 0; r8 < RB; ++r8)
 #pragma unroll
-            for (int k2 = 0; k2 < NV; ++k2) {
-                const int idx = sub + k2 * LPR;
-                x[r8][k2] = (r < rows && idx < n4) ? t4[r * n4 + idx] : make_float4(0.f, 0.f, 0.f, 0.f);
+                for (int k2 = 0; k2 < NV; ++k2) x[r8][k2] = t4[(r8 * RPW + slot) * (NV * LPR) + sub + k2 * LPR];
+        } else {
+#pragma unroll
+            for (int r8 = 0; r8 < RB; ++r8) {
+                const int r = r8 * RPW + slot;
+#pragma unroll
+                for (int k2 = 0; k2 < NV; ++k2) {
+                    const int idx = sub + k2 * LPR;
+                    x[r8][k2] = (r < rows && idx < n4) ? t4[r * n4 + idx] : make_float4(0.f, 0.f, 0.f, 0.f);
+                }
             }
         }
         const bool myvalid = myr < rows;
-        float yv = 0.f;
+        const float yv = y_next;
         if constexpr (!PREDICT) {
-            if (myvalid)
-                yv = (kCanStageY && p.stage_y && rows == RPB) ? reinterpret_cast<const float*>(stage + x_stride)[myr] : __ldg(p.y + row0 + myr);
+            const long long rn = row0 + stride_rows + myr;
+            y_next = (i + 1 < cnt && rn < p.m) ? __ldg(p.y + rn) : 0.f;
         }
         // the batch now lives in registers: re-arm this stage with the batch `depth` steps ahead
         __syncwarp();
         if (i + D < cnt) {
             if (lane == 0) {
                 fence_proxy_async_smem();
-                issue(i + D, d);
+                issue(row0 + D * stride_rows, d);
             }
             issued = i + D + 1;
         }
@@ -233,6 +239,7 @@ __global__ void __launch_bounds__(NW * 32, 1) k_stream_rows(const StreamParams p
                 dse += se; dsl += sl; se = 0.f; sl = 0.f;
             }
         }
+        row0 += stride_rows;
     }
 
     if (done < cnt) {

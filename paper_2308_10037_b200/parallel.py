@@ -35,9 +35,10 @@ def fit_sharded(local_sums: Callable[[torch.Tensor], None], apply_sums: Callable
     """
     world = dist.get_world_size(group)
     gathered = torch.empty((world, sums.numel()), dtype=sums.dtype, device=sums.device)
+    rows = [gathered[r] for r in range(world)]          # views: the collective writes straight into `gathered`
     for t in range(int(iters)):
         local_sums(sums)
-        dist.all_gather_into_tensor(gathered, sums, group=group)
+        dist.all_gather(rows, sums, group=group)        # supported by both NCCL and gloo
         apply_sums(gathered, t)
 
 

@@ -60,7 +60,7 @@ def test_plan_staged_shapes(m, n, lpr, nv):
     assert p["tile_rows"] == p["rows_per_batch"]              # one stage holds one register batch
     assert 1 <= p["stages"] <= 4
     assert p["smem_bytes"] <= 227 * 1024
-    stage = -(-p["tile_rows"] * n * 4 // 128) * 128 + 128
+    stage = -(-p["tile_rows"] * n * 4 // 128) * 128
     assert 1024 + 16 * p["stages"] * stage <= p["smem_bytes"]
     # 16 warps per CTA take one batch each per round; the grid never exceeds the rounds available
     batches = -(-m // p["rows_per_batch"])
