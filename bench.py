@@ -35,7 +35,7 @@ UNIT = "iterations/s"
 NOMINAL_HBM_GBS = 8000.0
 # dram__bytes_read.sum + dram__bytes_write.sum of the streaming kernel per row of X, from the ncu capture summarised in
 # profiles/ (taken at m = 500,000 and scaled by rows).  Remove an entry when its kernel changes.
-NCU_TRAFFIC_BYTES_PER_ROW = {"cfg3": (514.026752e6 + 3.22944e6) / 500_000}
+NCU_TRAFFIC_BYTES_PER_ROW = {"cfg3": (514.024192e6 + 3.515648e6) / 500_000}
 FALLBACK_HBM_GBS = 6650.0
 
 
