@@ -159,6 +159,53 @@ def workload_config(wl, n_gpus):
             "parallelism": "single GPU" if n_gpus == 1 else f"dp{n_gpus} row-sharded, all-gather of n+2 fp64 sums per iteration"}
 
 
+def run_tol(args, wl):
+    """Time to tolerance with the paper's stopping rule (Algorithm 7) on one GPU: `--tol ALPHA,EPS`.
+
+    Trains on the first 90 % of the rows until ||grad||_2 <= EPS (at most --steps updates), scores F1 at threshold 0.5 on
+    the held-out 10 %, and times the CPU checker on the same training rows for a bounded number of iterations.
+    """
+    import numpy as np
+    import torch
+    import oracle
+    from paper_2308_10037_b200 import api, build, datagen
+    alpha, eps = (float(v) for v in args.tol.split(","))
+    build.build()
+    X, y, _, _ = datagen.generate(wl)
+    m_tr = int(0.9 * wl.m)
+    dX, dy = torch.from_numpy(X).cuda(), torch.from_numpy(y).cuda()
+    ctx = api.Context(n_max=wl.n, device=0)
+    w = torch.zeros(wl.n, device="cuda")
+    b = torch.zeros(1, device="cuda")
+    ctx.fit(dX[:m_tr], dy[:m_tr], alpha, args.warmup, w, b)          # warm-up launches, result discarded
+    torch.cuda.synchronize()
+    w.zero_(); b.zero_()
+    launches0 = ctx.launch_count()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record()
+    iters, nrm = ctx.fit_tol(dX[:m_tr], dy[:m_tr], alpha, eps, args.steps, w, b, check_every=64)
+    ev1.record()
+    torch.cuda.synchronize()
+    secs = ev0.elapsed_time(ev1) / 1e3
+    labels = ctx.predict(dX[m_tr:], w, b, 0.5).cpu().numpy()
+    f1 = oracle.f1_score(labels, y[m_tr:])[0]
+    k = max(2, min(iters, 40))
+    t0 = time.perf_counter()
+    oracle.fit(X[:m_tr], y[:m_tr], alpha, k)
+    cpu_it_s = k / (time.perf_counter() - t0)
+    line = {"metric": "seconds to ||grad||_2 <= eps (Algorithm 7 stopping rule)", "value": secs, "unit": "s", "n_gpus": 1,
+            "steps": iters, "warmup": args.warmup, "ms_per_step": 1e3 * secs / max(iters, 1), "higher_is_better": False,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": f"{wl.name}: m={wl.m} x n={wl.n}, first 90 % train / last 10 % test, alpha={alpha}, eps={eps}",
+                       "max_updates": args.steps},
+            "updates": iters, "grad_norm": nrm, "converged": bool(nrm <= eps), "f1_test": f1,
+            "cpu_baseline": {"value": iters / cpu_it_s, "unit": "s", "cores": oracle.threads(), "kind": "oracle",
+                             "sample": f"{k} iterations of oracle.fit on the training rows, extrapolated to {iters} updates"},
+            "gpu_launches": ctx.launch_count() - launches0}
+    print(json.dumps(line))
+    ctx.close()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -167,6 +214,7 @@ def main():
     ap.add_argument("--workload", default="cfg3")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--rows", type=int, default=0, help="override the workload's row count (profiling on a smaller case)")
+    ap.add_argument("--tol", default="", help="ALPHA,EPS: time-to-tolerance mode (Algorithm 7 stopping rule); --steps caps the updates")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
@@ -183,6 +231,10 @@ def main():
     if args.impl == "reference":
         if rank == 0:
             run_reference(args, wl)
+        return
+    if args.tol:
+        if rank == 0:
+            run_tol(args, wl)
         return
 
     import numpy as np

@@ -100,6 +100,25 @@ int lr_fit(lr_ctx* ctx, const float* d_X, const float* d_y, int64_t m, int32_t n
            float lr, int32_t iters, float* d_w, float* d_b, float* d_loss_hist, void* stream);
 
 /*
+ * Gradient descent with the paper's stopping rule (Algorithm 7's loop; the norm is Algorithm 4's):
+ *   repeat { grad at the current (w, b);  w <- w - lr*grad_w, b <- b - lr*grad_b;
+ *            if ||(grad_w, grad_b)||_2 <= eps: stop }   -- the update is applied before the test, as in
+ * Algorithm 7 -- for at most max_iters updates.  The norm is formed on the device in fp64 from the same
+ * sums the update uses; once it is met a device flag turns every later launch of this call into a
+ * no-op, so the result does not depend on check_every.  The host enqueues check_every iterations at a
+ * time and then synchronises `stream` to read the flag (this call blocks, unlike lr_fit).
+ * d_w, d_b in/out as for lr_fit; d_loss_hist / d_gnorm_hist are NULL or [max_iters] (entries past the
+ * stopping iteration are left untouched); *iters_done receives the number of updates applied and
+ * *grad_norm the norm of the last applied gradient (-1 if max_iters == 0).  The caller tells
+ * "converged" from "ran out of iterations" by comparing *grad_norm with eps.
+ * Errors as lr_fit, plus LR_ERR_SHAPE for check_every < 1 and LR_ERR_VALUE for eps < 0 or not finite.
+ */
+int lr_fit_tol(lr_ctx* ctx, const float* d_X, const float* d_y, int64_t m, int32_t n,
+               float lr, float eps, int32_t max_iters, int32_t check_every,
+               float* d_w, float* d_b, float* d_loss_hist, float* d_gnorm_hist,
+               int32_t* iters_done, float* grad_norm, void* stream);
+
+/*
  * d_labels[i] = 1 if sigmoid(x_i.w + b) >= thr else 0, decided in logit space as
  * z_i >= log(thr/(1-thr)) evaluated in fp32 (the paper reports f1 but states no threshold; the
  * caller supplies it).  0 < thr < 1.  d_labels is uint8 [m].

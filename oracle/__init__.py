@@ -38,6 +38,7 @@ def _load():
         lib.oracle_loss_grad.argtypes = [P, P, I64, I32, P, D, P, P, P]
         lib.oracle_fit.argtypes = [P, P, I64, I32, D, I32, P, P, P, P, P, ctypes.c_int]
         lib.oracle_predict.argtypes = [P, I64, I32, P, D, D, P, P]
+        lib.oracle_fit_tol.argtypes = [P, P, I64, I32, D, D, I32, P, P, P, P, P, P]
         lib.oracle_f1.argtypes = [P, P, I64, P, P, P, P]
         _lib = lib
     return _lib
@@ -100,6 +101,27 @@ def fit(X, y, lr, iters, w0=None, b0=0.0, history=False, round_to_fp32=False):
     if history:
         return w, float(b[0]), lh, wh, bh
     return w, float(b[0]), lh
+
+
+def fit_tol(X, y, lr, eps, max_iters, w0=None, b0=0.0):
+    """GD with the stopping rule ||grad||_2 <= eps tested after each update (at most ``max_iters`` updates).
+
+    Returns ``(w, b, iters_done, grad_norm, loss_hist[:iters_done], gnorm_hist[:iters_done])``.
+    """
+    X = _f32(X)
+    m, n = X.shape
+    y = _f32(y, (m,))
+    w = np.zeros(n) if w0 is None else np.array(w0, dtype=np.float64).copy()
+    b = np.array([float(b0)])
+    lh, gh = np.zeros(max(max_iters, 1)), np.zeros(max(max_iters, 1))
+    done = ctypes.c_int32()
+    nrm = ctypes.c_double()
+    rc = _load().oracle_fit_tol(_ptr(X), _ptr(y), m, n, float(lr), float(eps), int(max_iters), _ptr(w), _ptr(b), _ptr(lh),
+                                _ptr(gh), ctypes.byref(done), ctypes.byref(nrm))
+    if rc != 0:
+        raise ValueError("oracle_fit_tol: bad arguments")
+    k = done.value
+    return w, float(b[0]), k, nrm.value, lh[:k], gh[:k]
 
 
 def predict(X, w, b, thr, return_z=False):

@@ -140,6 +140,39 @@ int oracle_fit(const float* X, const float* y, int64_t m, int32_t n, double lr, 
     return 0;
 }
 
+/*
+ * Algorithm 7's loop: form the gradient at the current point, apply the update, then stop if the 2-norm of the
+ * gradient just applied is <= eps (Algorithm 4 gives the squared norm; Algorithm 7 compares its square root).
+ * Reading: the bias is part of the model, so the norm is taken over (grad_w, grad_b) stacked.
+ * At most max_iters updates.  *iters_done = updates applied, *grad_norm = norm of the last applied gradient
+ * (-1 when max_iters == 0).  loss_hist / gnorm_hist (nullable, [max_iters]) are filled up to the stopping iteration.
+ */
+int oracle_fit_tol(const float* X, const float* y, int64_t m, int32_t n, double lr, double eps, int32_t max_iters,
+                   double* w, double* b, double* loss_hist, double* gnorm_hist, int32_t* iters_done, double* grad_norm) {
+    if (!X || !y || !w || !b || !iters_done || !grad_norm || m < 1 || n < 1 || max_iters < 0 || !(eps >= 0.0)) return -1;
+    double* g = (double*)malloc(sizeof(double) * (size_t)n);
+    if (!g) return -1;
+    *iters_done = 0;
+    *grad_norm = -1.0;
+    for (int32_t t = 0; t < max_iters; ++t) {
+        double loss, gb;
+        if (oracle_loss_grad(X, y, m, n, w, *b, &loss, g, &gb) != 0) { free(g); return -1; }
+        for (int32_t j = 0; j < n; ++j) w[j] -= lr * g[j];
+        *b -= lr * gb;
+        double q = 0.0;
+        for (int32_t j = 0; j < n; ++j) q += g[j] * g[j];          /* Algorithm 4 */
+        q += gb * gb;
+        double nrm = sqrt(q);
+        if (loss_hist) loss_hist[t] = loss;
+        if (gnorm_hist) gnorm_hist[t] = nrm;
+        *iters_done = t + 1;
+        *grad_norm = nrm;
+        if (nrm <= eps) break;                                      /* Algorithm 7: test after the update */
+    }
+    free(g);
+    return 0;
+}
+
 /* label_i = 1 iff p_i >= thr, decided in logit space: z_i >= log(thr/(1-thr)).  z_out (nullable) gets z. */
 int oracle_predict(const float* X, int64_t m, int32_t n, const double* w, double b, double thr,
                    uint8_t* labels, double* z_out) {

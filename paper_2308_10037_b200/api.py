@@ -21,7 +21,7 @@ LR_ERR_NULL, LR_ERR_SHAPE, LR_ERR_ALIGNMENT, LR_ERR_VALUE, LR_ERR_CUDA, LR_ERR_T
 EXPORTS = ["lr_plan_query", "lr_create", "lr_destroy", "lr_loss_grad", "lr_fit", "lr_predict", "lr_shard_sums",
            "lr_apply_sums", "lr_fit_host",
            "lr_predict_host", "lr_profile_enable", "lr_profile_read", "lr_launch_count", "lr_last_device_status",
-           "lr_last_cuda_error", "lr_status_string", "lr_loss_grad_noalloc"]
+           "lr_last_cuda_error", "lr_status_string", "lr_loss_grad_noalloc", "lr_fit_tol"]
 
 
 class LrPlan(ctypes.Structure):
@@ -58,6 +58,8 @@ def lib() -> ctypes.CDLL:
         L.lr_predict.argtypes = [P, P, I64, I32, P, P, F, P, P]
         L.lr_shard_sums.argtypes = [P, P, P, I64, I32, P, P, P, P]
         L.lr_apply_sums.argtypes = [P, P, I32, I64, I32, F, P, P, P, P]
+        L.lr_fit_tol.argtypes = [P, P, P, I64, I32, F, F, I32, I32, P, P, P, P, ctypes.POINTER(I32),
+                                 ctypes.POINTER(F), P]
         L.lr_loss_grad_noalloc.argtypes = [I32, P, P, I64, I32, P, P, P, P, P, P, P]
         L.lr_fit_host.argtypes = [P, P, P, I64, I32, F, I32, P, P, P]
         L.lr_predict_host.argtypes = [P, P, I64, I32, P, P, F, P]
@@ -160,6 +162,18 @@ class Context:
                           int(iters), _dev_ptr(w, torch.float32, "w"), _dev_ptr(b, torch.float32, "b"),
                           _dev_ptr(loss_hist, torch.float32, "loss_hist"), self._stream())
         self._check(rc, "lr_fit")
+
+    def fit_tol(self, X, y, lr, eps, max_iters, w, b, check_every=16, loss_hist=None, gnorm_hist=None):
+        """GD until ||grad||_2 <= eps (at most ``max_iters`` updates), in place on w, b.  Returns (updates, last norm)."""
+        m, n = X.shape
+        done, nrm = ctypes.c_int32(), ctypes.c_float()
+        rc = lib().lr_fit_tol(self._h, _dev_ptr(X, torch.float32, "X"), _dev_ptr(y, torch.float32, "y"), m, n, float(lr),
+                              float(eps), int(max_iters), int(check_every), _dev_ptr(w, torch.float32, "w"),
+                              _dev_ptr(b, torch.float32, "b"), _dev_ptr(loss_hist, torch.float32, "loss_hist"),
+                              _dev_ptr(gnorm_hist, torch.float32, "gnorm_hist"), ctypes.byref(done), ctypes.byref(nrm),
+                              self._stream())
+        self._check(rc, "lr_fit_tol")
+        return done.value, nrm.value
 
     def predict(self, X, w, b, thr):
         m, n = X.shape

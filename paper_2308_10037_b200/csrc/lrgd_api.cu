@@ -117,6 +117,9 @@ struct lr_ctx {
     int n_max = 0;
     double* d_partial = nullptr;
     int* d_status = nullptr;
+    TolState* d_tol = nullptr;                      // stopping-rule state of lr_fit_tol
+    double* d_gbuf = nullptr;                       // [n_max+1] gradient entries for the norm
+    TolState* h_tol = nullptr;                      // pinned host mirror
     // buffers of the host-pointer entry points (grown on demand)
     void* d_hX = nullptr; size_t hX_bytes = 0;
     void* d_hy = nullptr; size_t hy_bytes = 0;
@@ -190,6 +193,11 @@ cudaError_t launch_split(const lr_plan& P, const SplitParams& sp, cudaStream_t s
 
 struct Pass {
     const float* X; const float* y; int64_t m; int32_t n; const float* w; const float* b;
+    const int* stop = nullptr;                      // device flag that turns the launch into a no-op once set
+};
+
+struct TolArgs {                                    // tolerance mode of the reduction
+    TolState* state; double* gbuf; double eps; float* gnorm_out;
 };
 
 // Enqueues the streaming kernel for one pass (loss/grad partials, or labels when `labels` is set).
@@ -206,24 +214,24 @@ int launch_stream_pass(lr_ctx* ctx, const lr_plan& P, const Pass& a, uint8_t* la
     }
     cudaError_t e;
     if (P.variant == 0) {
-        StreamParams sp;
+        StreamParams sp{};
         sp.X = a.X; sp.y = a.y; sp.m = a.m; sp.n = a.n; sp.w = a.w; sp.b = a.b;
-        sp.partial = ctx->d_partial; sp.labels = labels; sp.cut = cut; sp.status = ctx->d_status;
+        sp.partial = ctx->d_partial; sp.labels = labels; sp.cut = cut; sp.status = ctx->d_status; sp.stop = a.stop;
         sp.depth = P.stages;
         sp.num_batches = (a.m + P.rows_per_batch - 1) / P.rows_per_batch;
         e = predict ? launch_rows<true>(P, sp, st) : launch_rows<false>(P, sp, st);
     } else if (P.variant == 1) {
-        SplitParams sp;
+        SplitParams sp{};
         sp.X = a.X; sp.y = a.y; sp.m = a.m; sp.n = a.n; sp.w = a.w; sp.b = a.b;
-        sp.partial = ctx->d_partial; sp.labels = labels; sp.cut = cut; sp.status = ctx->d_status;
+        sp.partial = ctx->d_partial; sp.labels = labels; sp.cut = cut; sp.status = ctx->d_status; sp.stop = a.stop;
         sp.depth = P.stages;
         sp.cw = (a.n / 4 + kNW - 1) / kNW;
         sp.num_batches = (a.m + P.rows_per_batch - 1) / P.rows_per_batch;
         e = predict ? launch_split<true>(P, sp, st) : launch_split<false>(P, sp, st);
     } else {
-        GenericParams gp;
+        GenericParams gp{};
         gp.X = a.X; gp.y = a.y; gp.m = a.m; gp.n = a.n; gp.w = a.w; gp.b = a.b;
-        gp.partial = ctx->d_partial; gp.labels = labels; gp.cut = cut;
+        gp.partial = ctx->d_partial; gp.labels = labels; gp.cut = cut; gp.stop = a.stop;
         if (predict) k_generic<true><<<P.grid, P.threads, 0, st>>>(gp);
         else k_generic<false><<<P.grid, P.threads, 0, st>>>(gp);
         e = cudaGetLastError();
@@ -238,11 +246,13 @@ int launch_stream_pass(lr_ctx* ctx, const lr_plan& P, const Pass& a, uint8_t* la
 }
 
 int launch_reduce(lr_ctx* ctx, const double* partial, int G, int64_t m, int32_t n, double lr, bool update, float* w,
-                  float* b, float* grad_w, float* grad_b, float* loss_out, double* raw_sums, cudaStream_t st) {
-    ReduceParams rp;
+                  float* b, float* grad_w, float* grad_b, float* loss_out, double* raw_sums, cudaStream_t st,
+                  const TolArgs* tol = nullptr) {
+    ReduceParams rp{};
     rp.partial = partial; rp.G = G; rp.n = n; rp.inv_m = 1.0 / double(m); rp.lr = lr;
     rp.update = update ? 1 : 0; rp.w = w; rp.b = b; rp.grad_w = grad_w; rp.grad_b = grad_b; rp.loss_out = loss_out;
     rp.raw_sums = raw_sums;
+    if (tol) { rp.tol = tol->state; rp.gbuf = tol->gbuf; rp.eps = tol->eps; rp.gnorm_out = tol->gnorm_out; }
     dim3 block(32, kRedSlices);
     k_reduce_update<<<(n + 2 + 31) / 32, block, 0, st>>>(rp);
     LR_CK(ctx, cudaGetLastError());
@@ -295,11 +305,18 @@ int lr_create(lr_ctx** out, int32_t device, int32_t n_max) {
     }
     if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&c->d_status), sizeof(int));
     if (e == cudaSuccess) e = cudaMemset(c->d_status, 0, sizeof(int));
+    if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&c->d_tol), sizeof(TolState));
+    if (e == cudaSuccess) e = cudaMemset(c->d_tol, 0, sizeof(TolState));
+    if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&c->d_gbuf), (size_t(n_max) + 1) * sizeof(double));
+    if (e == cudaSuccess) e = cudaMallocHost(reinterpret_cast<void**>(&c->h_tol), sizeof(TolState));
     if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&c->hstream, cudaStreamNonBlocking);
     if (prev >= 0) cudaSetDevice(prev);
     if (e != cudaSuccess) {
         if (c->d_partial) cudaFree(c->d_partial);
         if (c->d_status) cudaFree(c->d_status);
+        if (c->d_tol) cudaFree(c->d_tol);
+        if (c->d_gbuf) cudaFree(c->d_gbuf);
+        if (c->h_tol) cudaFreeHost(c->h_tol);
         delete c;
         return rc != LR_OK ? rc : LR_ERR_CUDA;
     }
@@ -316,6 +333,9 @@ int lr_destroy(lr_ctx* ctx) {
         if (ctx->hstream) cudaStreamDestroy(ctx->hstream);
         cudaFree(ctx->d_partial);
         cudaFree(ctx->d_status);
+        cudaFree(ctx->d_tol);
+        cudaFree(ctx->d_gbuf);
+        if (ctx->h_tol) cudaFreeHost(ctx->h_tol);
         cudaFree(ctx->d_hX);
         cudaFree(ctx->d_hy);
         cudaFree(ctx->d_hw);
@@ -365,6 +385,48 @@ int lr_fit(lr_ctx* ctx, const float* d_X, const float* d_y, int64_t m, int32_t n
                            d_loss_hist ? d_loss_hist + t : nullptr, nullptr, st);
         if (rc != LR_OK) return rc;
     }
+    return LR_OK;
+}
+
+int lr_fit_tol(lr_ctx* ctx, const float* d_X, const float* d_y, int64_t m, int32_t n, float lr, float eps,
+               int32_t max_iters, int32_t check_every, float* d_w, float* d_b, float* d_loss_hist, float* d_gnorm_hist,
+               int32_t* iters_done, float* grad_norm, void* stream) {
+    int rc = check_common(ctx, d_X, m, n, d_w, d_b);
+    if (rc != LR_OK) return rc;
+    if (!d_y || !iters_done || !grad_norm) return LR_ERR_NULL;
+    if (max_iters < 0 || check_every < 1) return LR_ERR_SHAPE;
+    if (!aligned(d_y, 4) || (d_loss_hist && !aligned(d_loss_hist, 4)) || (d_gnorm_hist && !aligned(d_gnorm_hist, 4)))
+        return LR_ERR_ALIGNMENT;
+    if (!std::isfinite(lr) || !(eps >= 0.f) || !std::isfinite(eps)) return LR_ERR_VALUE;
+    lr_plan P;
+    rc = make_plan(m, n, aligned(d_X, 16), ctx->sm_count, &P);
+    if (rc != LR_OK) return rc;
+    *iters_done = 0;
+    *grad_norm = -1.f;
+    if (max_iters == 0) return LR_OK;
+    DeviceGuard g(ctx);
+    if (!g.ok) return LR_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    LR_CK(ctx, cudaMemsetAsync(ctx->d_tol, 0, sizeof(TolState), st));
+    const int* stop = &ctx->d_tol->stop;
+    for (int32_t t = 0; t < max_iters;) {
+        const int32_t chunk = std::min(check_every, max_iters - t);
+        for (int32_t k = 0; k < chunk; ++k, ++t) {
+            Pass pass{d_X, d_y, m, n, d_w, d_b};
+            pass.stop = stop;
+            rc = launch_stream_pass(ctx, P, pass, nullptr, 0.f, st);
+            if (rc != LR_OK) return rc;
+            TolArgs ta{ctx->d_tol, ctx->d_gbuf, double(eps), d_gnorm_hist ? d_gnorm_hist + t : nullptr};
+            rc = launch_reduce(ctx, ctx->d_partial, P.grid, m, n, double(lr), true, d_w, d_b, nullptr, nullptr,
+                               d_loss_hist ? d_loss_hist + t : nullptr, nullptr, st, &ta);
+            if (rc != LR_OK) return rc;
+        }
+        LR_CK(ctx, cudaMemcpyAsync(ctx->h_tol, ctx->d_tol, sizeof(TolState), cudaMemcpyDeviceToHost, st));
+        LR_CK(ctx, cudaStreamSynchronize(st));
+        if (ctx->h_tol->stop) break;
+    }
+    *iters_done = ctx->h_tol->iters_done;
+    *grad_norm = static_cast<float>(ctx->h_tol->grad_norm);
     return LR_OK;
 }
 
@@ -602,14 +664,14 @@ extern "C" int lr_loss_grad_noalloc(int32_t device, const float* d_X, const floa
     if (cudaMemsetAsync(status, 0, sizeof(int), st) != cudaSuccess) return LR_ERR_CUDA;
     cudaError_t e;
     if (P.variant == 0) {
-        StreamParams sp;
+        StreamParams sp{};
         sp.X = d_X; sp.y = d_y; sp.m = m; sp.n = n; sp.w = d_w; sp.b = d_b;
         sp.partial = partial; sp.labels = nullptr; sp.cut = 0.f; sp.status = status;
         sp.depth = P.stages;
         sp.num_batches = (m + P.rows_per_batch - 1) / P.rows_per_batch;
         e = launch_rows<false>(P, sp, st);
     } else if (P.variant == 1) {
-        SplitParams sp;
+        SplitParams sp{};
         sp.X = d_X; sp.y = d_y; sp.m = m; sp.n = n; sp.w = d_w; sp.b = d_b;
         sp.partial = partial; sp.labels = nullptr; sp.cut = 0.f; sp.status = status;
         sp.depth = P.stages;
@@ -617,14 +679,14 @@ extern "C" int lr_loss_grad_noalloc(int32_t device, const float* d_X, const floa
         sp.num_batches = (m + P.rows_per_batch - 1) / P.rows_per_batch;
         e = launch_split<false>(P, sp, st);
     } else {
-        GenericParams gp;
+        GenericParams gp{};
         gp.X = d_X; gp.y = d_y; gp.m = m; gp.n = n; gp.w = d_w; gp.b = d_b;
         gp.partial = partial; gp.labels = nullptr; gp.cut = 0.f;
         k_generic<false><<<P.grid, P.threads, 0, st>>>(gp);
         e = cudaGetLastError();
     }
     if (e != cudaSuccess) return LR_ERR_CUDA;
-    ReduceParams rp;
+    ReduceParams rp{};
     rp.partial = partial; rp.G = P.grid; rp.n = n; rp.inv_m = 1.0 / double(m); rp.lr = 0.0; rp.update = 0;
     rp.w = nullptr; rp.b = nullptr; rp.grad_w = d_grad_w; rp.grad_b = d_grad_b; rp.loss_out = d_loss; rp.raw_sums = nullptr;
     k_reduce_update<<<(n + 2 + 31) / 32, dim3(32, kRedSlices), 0, st>>>(rp);

@@ -26,10 +26,12 @@ struct GenericParams {
     double* partial;          // [grid][n+2]
     unsigned char* labels;    // predict mode
     float cut;
+    const int* stop;          // nullable: non-zero makes the launch a no-op
 };
 
 template <bool PREDICT>
 __global__ void __launch_bounds__(kGenThreads) k_generic(const GenericParams p) {
+    if (p.stop != nullptr && *reinterpret_cast<const volatile int*>(p.stop) != 0) return;   // a stopping rule was met by an earlier iteration
     __shared__ float err_s[kGenRows];
     __shared__ double red_e[kGenThreads / 32], red_l[kGenThreads / 32];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;

@@ -3,13 +3,27 @@
 // (Algorithm 1's update; descent sign as in Algorithm 7).
 //
 // Block = 32 columns x kRedSlices slices.  Slice s sums partial rows [s*per, (s+1)*per) of its column in
-// index order in fp64; the slices are then added in slice order.  No atomics: bit-reproducible.
+// index order in fp64; the slices are then added in slice order.  No atomics on data: bit-reproducible.
+//
+// Tolerance mode (Algorithm 7's stopping rule, built from Algorithm 4's norm): every block parks its fp64
+// gradient entries in `gbuf`; the block that finishes last (a ticket counter) adds their squares in index
+// order, records ||grad||_2, counts the update, and raises `stop` when ||grad||_2 <= eps.  Kernels enqueued
+// after that see `stop` and return without touching anything, so the parameters stay exactly as they were
+// after the stopping update no matter how many further iterations the host had already enqueued.
 #pragma once
 #include "lrgd_common.cuh"
 
 namespace lrgd {
 
 constexpr int kRedSlices = 8;
+
+struct TolState {             // device-resident, owned by the context
+    int stop;                 // 1 once the tolerance has been met
+    int iters_done;           // updates applied since the state was reset
+    unsigned int ticket;      // blocks of the current reduction that have finished
+    int pad;
+    double grad_norm;         // ||(grad_w, grad_b)||_2 of the last applied update
+};
 
 struct ReduceParams {
     const double* partial;    // [G][n+2]: n column sums, sum err, sum loss
@@ -24,10 +38,17 @@ struct ReduceParams {
     float* grad_b;
     float* loss_out;          // nullable
     double* raw_sums;         // non-null: write the unscaled fp64 sums [n+2] here and nothing else
+    // tolerance mode (all null / zero otherwise)
+    TolState* tol;
+    double* gbuf;             // [n+1] scratch for the gradient entries
+    double eps;
+    float* gnorm_out;         // nullable: ||grad||_2 of this iteration
 };
 
 __global__ void __launch_bounds__(32 * kRedSlices) k_reduce_update(const ReduceParams p) {
     __shared__ double sh[kRedSlices][33];
+    __shared__ int is_last;
+    if (p.tol != nullptr && *reinterpret_cast<volatile int*>(&p.tol->stop) != 0) return;   // uniform: set by an earlier kernel
     const int col = blockIdx.x * 32 + threadIdx.x;
     const int slice = threadIdx.y;
     const int stride = p.n + 2;
@@ -41,23 +62,53 @@ __global__ void __launch_bounds__(32 * kRedSlices) k_reduce_update(const ReduceP
     }
     sh[slice][threadIdx.x] = s;
     __syncthreads();
-    if (slice != 0 || col >= stride) return;
-    double t = 0.0;
+    if (slice == 0 && col < stride) {
+        double t = 0.0;
 #pragma unroll
-    for (int k = 0; k < kRedSlices; ++k) t += sh[k][threadIdx.x];
-    if (p.raw_sums) {
-        p.raw_sums[col] = t;
-        return;
+        for (int k = 0; k < kRedSlices; ++k) t += sh[k][threadIdx.x];
+        if (p.raw_sums) {
+            p.raw_sums[col] = t;
+        } else {
+            const double v = t * p.inv_m;
+            if (col < p.n) {
+                if (p.update) p.w[col] = static_cast<float>(static_cast<double>(p.w[col]) - p.lr * v);
+                else p.grad_w[col] = static_cast<float>(v);
+            } else if (col == p.n) {
+                if (p.update) p.b[0] = static_cast<float>(static_cast<double>(p.b[0]) - p.lr * v);
+                else p.grad_b[0] = static_cast<float>(v);
+            } else {
+                if (p.loss_out) p.loss_out[0] = static_cast<float>(v);
+            }
+            if (p.tol != nullptr && col <= p.n) p.gbuf[col] = v;
+        }
     }
-    const double v = t * p.inv_m;
-    if (col < p.n) {
-        if (p.update) p.w[col] = static_cast<float>(static_cast<double>(p.w[col]) - p.lr * v);
-        else p.grad_w[col] = static_cast<float>(v);
-    } else if (col == p.n) {
-        if (p.update) p.b[0] = static_cast<float>(static_cast<double>(p.b[0]) - p.lr * v);
-        else p.grad_b[0] = static_cast<float>(v);
-    } else {
-        if (p.loss_out) p.loss_out[0] = static_cast<float>(v);
+    if (p.tol == nullptr) return;
+
+    // ---- tolerance mode: the last block to finish forms the norm ----
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0 && threadIdx.y == 0) {
+        const unsigned int t = atomicAdd(&p.tol->ticket, 1u);
+        is_last = (t == gridDim.x - 1) ? 1 : 0;
+    }
+    __syncthreads();
+    if (!is_last || threadIdx.y != 0) return;
+    __threadfence();
+    const volatile double* gb = p.gbuf;
+    double q = 0.0;
+    for (int c = threadIdx.x; c <= p.n; c += 32) {           // lane-strided, then a fixed xor tree: one fixed order
+        const double v = gb[c];
+        q += v * v;
+    }
+#pragma unroll
+    for (int msk = 16; msk >= 1; msk >>= 1) q += __shfl_xor_sync(0xffffffffu, q, msk);
+    if (threadIdx.x == 0) {
+        const double nrm = sqrt(q);
+        p.tol->grad_norm = nrm;
+        p.tol->iters_done += 1;
+        if (p.gnorm_out) p.gnorm_out[0] = static_cast<float>(nrm);
+        if (nrm <= p.eps) p.tol->stop = 1;
+        p.tol->ticket = 0u;
     }
 }
 

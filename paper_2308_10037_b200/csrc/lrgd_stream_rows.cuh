@@ -39,6 +39,7 @@ struct StreamParams {
     unsigned char* labels;    // [m]                   (predict mode)
     float cut;                // predict: logit(thr)
     int* status;              // device status word
+    const int* stop;          // nullable: non-zero means a stopping rule has been met and the launch is a no-op
     int depth;                // stages per warp (1..kMaxDepth)
     long long num_batches;    // ceil(m / rows per batch)
 };
@@ -77,6 +78,7 @@ __global__ void __launch_bounds__(NW * 32, 1) k_stream_rows(const StreamParams p
     static_assert(NW * kMaxDepth * 8 + 16 <= kHeaderBytes, "header too small");
     constexpr unsigned FULL = 0xffffffffu;
 
+    if (p.stop != nullptr && *reinterpret_cast<const volatile int*>(p.stop) != 0) return;   // a stopping rule was met by an earlier iteration
     extern __shared__ __align__(128) unsigned char smem[];
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem);                       // [NW][kMaxDepth]
     volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + NW * kMaxDepth);

@@ -35,6 +35,7 @@ struct SplitParams {
     unsigned char* labels;    // predict mode
     float cut;
     int* status;
+    const int* stop;          // nullable: non-zero makes the launch a no-op
     int depth;                // stages per warp
     int cw;                   // 16-byte column groups per warp slice
     long long num_batches;    // ceil(m / RB)
@@ -48,6 +49,7 @@ __global__ void __launch_bounds__(NW * 32, 1) k_stream_split(const SplitParams p
     static_assert(NW * kMaxDepth * 8 + 16 <= kSplitZOffset, "header too small");
     static_assert(kSplitZOffset + 2 * NW * RB * 4 <= kSplitHeaderBytes, "header too small");
 
+    if (p.stop != nullptr && *reinterpret_cast<const volatile int*>(p.stop) != 0) return;   // a stopping rule was met by an earlier iteration
     extern __shared__ __align__(128) unsigned char smem[];
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + NW * kMaxDepth);

@@ -228,3 +228,29 @@ def test_bad_arguments_are_rejected():
         oracle.predict(X, w, b, 1.0)
     with pytest.raises(ValueError):
         oracle.predict(X, w, b, 0.0)
+
+
+def test_stopping_rule_follows_algorithm_7():
+    X, y, _, _ = datagen.random_problem(2000, 6, seed=12)
+    lr = 0.5
+    # eps = 0 never stops early: identical to the fixed-count fit
+    w0, b0, k0, n0, lh0, gh0 = oracle.fit_tol(X, y, lr, 0.0, 25)
+    wf, bf, lhf = oracle.fit(X, y, lr, 25)
+    assert k0 == 25 and np.array_equal(w0, wf) and b0 == bf and np.array_equal(lh0, lhf)
+    # the recorded norms are the norms of the gradients at the iterates before each update
+    _, _, _, wh, bh = oracle.fit(X, y, lr, 25, history=True)
+    for t in (0, 7, 24):
+        _, g, g_b = oracle.loss_grad(X, y, wh[t], bh[t])
+        assert abs(gh0[t] - math.sqrt(float(g @ g) + g_b * g_b)) < 1e-15
+    # a tolerance between two consecutive norms stops exactly there, after applying that update
+    eps = 0.5 * (gh0[9] + gh0[10])
+    assert gh0[10] < eps < gh0[9]
+    w1, b1, k1, n1, lh1, gh1 = oracle.fit_tol(X, y, lr, eps, 25)
+    assert k1 == 11 and n1 == gh0[10] and np.array_equal(w1, wh[11]) and b1 == bh[11]
+    assert len(lh1) == 11 and np.array_equal(gh1, gh0[:11])
+    # a huge tolerance still applies one update (the test comes after the update)
+    w2, b2, k2, n2, _, _ = oracle.fit_tol(X, y, lr, 1e9, 25)
+    assert k2 == 1 and np.array_equal(w2, wh[1]) and n2 == gh0[0]
+    # no iterations allowed: nothing happens
+    w3, b3, k3, n3, _, _ = oracle.fit_tol(X, y, lr, 1.0, 0)
+    assert k3 == 0 and n3 == -1.0 and not w3.any() and b3 == 0.0
