@@ -71,7 +71,7 @@ int make_plan(int64_t m, int32_t n, bool aligned16, int32_t sms, lr_plan* P) {
         if (per_warp >= (int64_t(1) << 31)) return LR_ERR_SHAPE;
         return LR_OK;
     }
-    if (aligned16 && n % 4 == 0 && n / 4 <= kNW * 64) {
+    if (aligned16 && n % 4 == 0 && n / 4 <= kNW * 64 && m < (int64_t(1) << 31) - 65536) {   // TMA coordinates are int32
         // wide rows: the warps of a CTA split each row by columns
         const int cw = (n / 4 + kNW - 1) / kNW;                                 // 16-byte column groups per warp slice
         const int nv = cw > 32 ? 2 : 1;
@@ -79,8 +79,7 @@ int make_plan(int64_t m, int32_t n, bool aligned16, int32_t sms, lr_plan* P) {
         const int64_t B = (m + rb - 1) / rb;
         const int grid = int(std::min<int64_t>(B, sms));
         const int64_t per_cta = (B + grid - 1) / grid;
-        const int64_t row_stride = (int64_t(cw) * 16 + 127) & ~int64_t(127);
-        const int64_t stage_stride = rb * row_stride;
+        const int64_t stage_stride = (int64_t(cw) * 16 * rb + 127) & ~int64_t(127);   // one densely packed box per stage
         int D = int(std::min<int64_t>(kMaxDepth, kStageBudgetBytes / (kNW * stage_stride)));
         D = int(std::min<int64_t>(D, per_cta));
         if (D < 1) D = 1;
@@ -176,19 +175,48 @@ cudaError_t launch_rows(const lr_plan& P, const StreamParams& sp, cudaStream_t s
     return launch_rows_t<4, 32, 2, PRED>(P, sp, st);
 }
 
+// Tensor map of X for the wide-row kernel: fp32 [m][n] row-major, box = cw*4 floats by rb rows, zero fill outside.
+// The encoder is a driver entry point, resolved at run time so that the library links against the runtime only.
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+cudaError_t make_x_tensor_map(const float* X, int64_t m, int32_t n, int cw, int rb, CUtensorMap* out) {
+    static EncodeTiledFn encode = nullptr;
+    if (!encode) {
+        void* fn = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q);
+        if (e != cudaSuccess) return e;
+        if (q != cudaDriverEntryPointSuccess || !fn) return cudaErrorNotSupported;
+        encode = reinterpret_cast<EncodeTiledFn>(fn);
+    }
+    const cuuint64_t dims[2] = {cuuint64_t(n), cuuint64_t(m)};
+    const cuuint64_t strides[1] = {cuuint64_t(n) * 4};
+    const cuuint32_t box[2] = {cuuint32_t(cw) * 4, cuuint32_t(rb)};
+    const cuuint32_t estr[2] = {1, 1};
+    CUresult r = encode(out, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float*>(X), dims, strides, box, estr,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
+}
+
 template <int NV, int RB, bool PRED>
-cudaError_t launch_split_t(const lr_plan& P, const SplitParams& sp, cudaStream_t st) {
+cudaError_t launch_split_t(const lr_plan& P, const CUtensorMap& tm, const SplitParams& sp, cudaStream_t st) {
     auto kern = k_stream_split<NV, RB, kNW, PRED>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, P.smem_bytes);
     if (e != cudaSuccess) return e;
-    kern<<<P.grid, P.threads, P.smem_bytes, st>>>(sp);
+    kern<<<P.grid, P.threads, P.smem_bytes, st>>>(tm, sp);
     return cudaGetLastError();
 }
 
 template <bool PRED>
-cudaError_t launch_split(const lr_plan& P, const SplitParams& sp, cudaStream_t st) {
-    if (P.vec_per_lane == 2) return launch_split_t<2, 4, PRED>(P, sp, st);
-    return launch_split_t<1, 8, PRED>(P, sp, st);
+cudaError_t launch_split(const lr_plan& P, const float* X, const SplitParams& sp, cudaStream_t st) {
+    CUtensorMap tm;
+    cudaError_t e = make_x_tensor_map(X, sp.m, sp.n, sp.cw, P.rows_per_batch, &tm);
+    if (e != cudaSuccess) return e;
+    if (P.vec_per_lane == 2) return launch_split_t<2, 4, PRED>(P, tm, sp, st);
+    return launch_split_t<1, 8, PRED>(P, tm, sp, st);
 }
 
 struct Pass {
@@ -222,12 +250,12 @@ int launch_stream_pass(lr_ctx* ctx, const lr_plan& P, const Pass& a, uint8_t* la
         e = predict ? launch_rows<true>(P, sp, st) : launch_rows<false>(P, sp, st);
     } else if (P.variant == 1) {
         SplitParams sp{};
-        sp.X = a.X; sp.y = a.y; sp.m = a.m; sp.n = a.n; sp.w = a.w; sp.b = a.b;
+        sp.y = a.y; sp.m = a.m; sp.n = a.n; sp.w = a.w; sp.b = a.b;
         sp.partial = ctx->d_partial; sp.labels = labels; sp.cut = cut; sp.status = ctx->d_status; sp.stop = a.stop;
         sp.depth = P.stages;
         sp.cw = (a.n / 4 + kNW - 1) / kNW;
         sp.num_batches = (a.m + P.rows_per_batch - 1) / P.rows_per_batch;
-        e = predict ? launch_split<true>(P, sp, st) : launch_split<false>(P, sp, st);
+        e = predict ? launch_split<true>(P, a.X, sp, st) : launch_split<false>(P, a.X, sp, st);
     } else {
         GenericParams gp{};
         gp.X = a.X; gp.y = a.y; gp.m = a.m; gp.n = a.n; gp.w = a.w; gp.b = a.b;
@@ -672,12 +700,12 @@ extern "C" int lr_loss_grad_noalloc(int32_t device, const float* d_X, const floa
         e = launch_rows<false>(P, sp, st);
     } else if (P.variant == 1) {
         SplitParams sp{};
-        sp.X = d_X; sp.y = d_y; sp.m = m; sp.n = n; sp.w = d_w; sp.b = d_b;
+        sp.y = d_y; sp.m = m; sp.n = n; sp.w = d_w; sp.b = d_b;
         sp.partial = partial; sp.labels = nullptr; sp.cut = 0.f; sp.status = status;
         sp.depth = P.stages;
         sp.cw = (n / 4 + kNW - 1) / kNW;
         sp.num_batches = (m + P.rows_per_batch - 1) / P.rows_per_batch;
-        e = launch_split<false>(P, sp, st);
+        e = launch_split<false>(P, d_X, sp, st);
     } else {
         GenericParams gp{};
         gp.X = d_X; gp.y = d_y; gp.m = m; gp.n = n; gp.w = d_w; gp.b = d_b;

@@ -85,6 +85,26 @@ __device__ __forceinline__ void bulk_copy_g2s(void* dst, const void* src, uint32
         : "memory");
 }
 
+// Tiled 2-D TMA copy global -> shared through a tensor map (no multicast): the box whose first element has
+// coordinates (x, y) -- x along the contiguous dimension, x*4 bytes a multiple of 16 -- lands densely packed at dst
+// (128-byte aligned); out-of-range elements are written as zeros and count towards the transferred bytes.
+__device__ __forceinline__ void bulk_tensor_2d_g2s(void* dst, const void* tmap, int x, int y, uint64_t* bar, uint64_t policy) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3}], [%4], %5;"
+        ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(x), "r"(y), "r"(smem_u32(bar)), "l"(policy)
+        : "memory");
+}
+
+// err alone (same arithmetic as in logistic_terms, so the two agree bit for bit)
+__device__ __forceinline__ float logistic_err(float z, float y) {
+    const float t = expf(-fabsf(z));
+    const float r = 1.0f / (1.0f + t);
+    const float tr = t * r;
+    const float p = z >= 0.0f ? r : tr;
+    const float q = z >= 0.0f ? tr : r;
+    return (y == 1.0f) ? -q : (p - y);
+}
+
 // Per-row logistic terms in fp32 from the logit z and the target y:
 //   err  = sigmoid(z) - y            (Eq. 1; Algorithm 7's sigmoid followed by Substract(Y, res))
 //   loss = max(z,0) + log1p(exp(-|z|)) - y*z  ( = -[y log p + (1-y) log(1-p)], finite for any z )

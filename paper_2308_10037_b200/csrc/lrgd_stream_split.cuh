@@ -3,19 +3,22 @@
 // A row no longer fits one warp's registers, so the 16 warps of a CTA split every row by columns: warp w owns
 // the contiguous slice of CW = ceil(n/4/16) 16-byte column groups starting at w*CW.  The CTA walks batches of RB
 // rows (batch g belongs to CTA g mod grid).  As in the narrow-row kernel each warp runs its own asynchronous
-// pipeline with `depth` private stages, filled by its elected lane with one 1-D bulk copy per row (the slice of
-// a row is contiguous, slices of consecutive rows are n*4 bytes apart), completing on the warp's own mbarriers.
+// pipeline with `depth` private stages completing on its own mbarriers; a stage is one RB-row by CW-group box of X,
+// fetched by the warp's elected lane with ONE tiled TMA copy (cp.async.bulk.tensor.2d through a tensor map of X;
+// no multicast).  Rows past m and columns past n arrive as zeros, so the loads need no bounds logic.
 // Per batch:
-//   1. every warp moves its slice of the RB rows into registers (conflict-free 128-bit shared loads), re-arms the
-//      stage, and forms its partial dot products (lane FMAs + transposing shuffle reduction);
-//   2. the partials meet in a double-buffered shared array, one __syncthreads per batch; every warp then adds the
-//      16 partials of each row in warp order, so all warps hold bit-identical z = x.w + b  (model equation, II-A);
-//   3. p, err and the loss term are formed (redundantly per warp, counted once by warp 0)   (Eq. 1, Algorithm 7);
+//   1. every warp moves its box into registers (conflict-free 128-bit shared loads), re-arms the stage, and forms
+//      its partial dot products (lane FMAs + transposing shuffle reduction);
+//   2. the partials meet in a double-buffered shared array, one __syncthreads per batch; every warp then adds the 16
+//      partials of each row in one fixed order, so all warps hold bit-identical z = x.w + b  (model equation, II-A);
+//   3. err is formed by every warp, the loss term only by warp 0                            (Eq. 1, Algorithm 7);
 //   4. acc[c] += x[r][c] * err[r] on the registers loaded in step 1                        (Algorithm 1's err.X).
 // Each column belongs to exactly one lane of one warp, so the CTA's partial row needs no cross-warp combine.
 // A warp whose bounded wait expires raises the CTA's abort flag; it (and then every other warp) keeps taking part in
 // the per-batch barrier without touching its stages, so the CTA still retires, with the status word set.
 #pragma once
+#include <cuda.h>
+
 #include "lrgd_common.cuh"
 #include "lrgd_stream_rows.cuh"
 
@@ -25,7 +28,6 @@ constexpr int kSplitHeaderBytes = 2048;   // mbarriers [NW][kMaxDepth], abort fl
 constexpr int kSplitZOffset = 1024;
 
 struct SplitParams {
-    const float* X;
     const float* y;
     long long m;
     int n;
@@ -37,15 +39,18 @@ struct SplitParams {
     int* status;
     const int* stop;          // nullable: non-zero makes the launch a no-op
     int depth;                // stages per warp
-    int cw;                   // 16-byte column groups per warp slice
+    int cw;                   // 16-byte column groups per warp slice (the tensor map's box is cw*4 floats by RB rows)
     long long num_batches;    // ceil(m / RB)
 };
 
 template <int NV, int RB, int NW, bool PREDICT>
-__global__ void __launch_bounds__(NW * 32, 1) k_stream_split(const SplitParams p) {
+__global__ void __launch_bounds__(NW * 32, 1) k_stream_split(const __grid_constant__ CUtensorMap tmap, const SplitParams p) {
     constexpr int LOG_RB = Log2<RB>::value;
-    constexpr int SHIFT = 5 - LOG_RB;              // lanes holding the same row after the reduction = 2^SHIFT
+    constexpr int SHIFT = 5 - LOG_RB;              // log2 of the lanes holding the same row after the reduction
+    constexpr int DUP = 1 << SHIFT;
+    constexpr int PER_DUP = NW / DUP;              // partial logits each of those lanes adds up
     constexpr unsigned FULL = 0xffffffffu;
+    static_assert(NW % DUP == 0, "warps must split evenly over the duplicate lanes");
     static_assert(NW * kMaxDepth * 8 + 16 <= kSplitZOffset, "header too small");
     static_assert(kSplitZOffset + 2 * NW * RB * 4 <= kSplitHeaderBytes, "header too small");
 
@@ -60,9 +65,9 @@ __global__ void __launch_bounds__(NW * 32, 1) k_stream_split(const SplitParams p
     const int D = p.depth, CW = p.cw;
     const int n = p.n, n4 = n >> 2;
     const int c0 = warp * CW;                                                 // first column group of this warp's slice
-    const int mycw = n4 - c0 < CW ? (n4 - c0 > 0 ? n4 - c0 : 0) : CW;         // column groups in the slice (0: idle warp)
-    const uint32_t row_stride = (static_cast<uint32_t>(CW) * 16u + 127u) & ~127u;
-    const uint32_t stage_stride = RB * row_stride;
+    const int mycw = n4 - c0 < CW ? (n4 - c0 > 0 ? n4 - c0 : 0) : CW;         // column groups of the slice inside the matrix
+    const uint32_t box_bytes = static_cast<uint32_t>(CW) * 16u * RB;          // one stage = one box, rows packed densely
+    const uint32_t stage_stride = (box_bytes + 127u) & ~127u;
     unsigned char* my_stages = data + static_cast<size_t>(warp) * D * stage_stride;
     uint64_t* my_bars = bars + warp * kMaxDepth;
 
@@ -77,15 +82,11 @@ __global__ void __launch_bounds__(NW * 32, 1) k_stream_split(const SplitParams p
     __syncthreads();
 
     const uint64_t pol = l2_policy_evict_first();
-    auto issue = [&](int i, int d) {               // lane 0 only, mycw > 0
-        const long long row0 = (static_cast<long long>(i) * gridDim.x + blockIdx.x) * RB;
-        const long long left = p.m - row0;
-        const int rows = left < RB ? static_cast<int>(left) : RB;
-        unsigned char* dst = my_stages + static_cast<size_t>(d) * stage_stride;
-        const uint32_t bytes = static_cast<uint32_t>(mycw) * 16u;
-        mbar_arrive_expect_tx(&my_bars[d], bytes * rows);
-        const float* src = p.X + row0 * n + c0 * 4;
-        for (int r = 0; r < rows; ++r) bulk_copy_g2s(dst + r * row_stride, src + static_cast<long long>(r) * n, bytes, &my_bars[d], pol);
+    const int stride_rows = static_cast<int>(gridDim.x) * RB;                 // rows between this CTA's batches (m < 2^31 here)
+    int row0 = static_cast<int>(blockIdx.x) * RB;                             // first row of the current batch
+    auto issue = [&](int r0, int d) {              // lane 0 of a warp with mycw > 0
+        mbar_arrive_expect_tx(&my_bars[d], box_bytes);
+        bulk_tensor_2d_g2s(my_stages + static_cast<size_t>(d) * stage_stride, &tmap, c0 * 4, r0, &my_bars[d], pol);
     };
 
     float4 acc[NV];
@@ -105,12 +106,14 @@ __global__ void __launch_bounds__(NW * 32, 1) k_stream_split(const SplitParams p
     }
     const float bval = __ldg(p.b);
     const int myr = (lane >> SHIFT) & (RB - 1);    // the row of a batch whose logit ends up on this lane
-    const bool owner = (lane & ((1 << SHIFT) - 1)) == 0;
+    const int dup = lane & (DUP - 1);              // which of the lanes sharing that row this one is
+    const bool owner = dup == 0;
+    const bool full_cw = CW == 32 * NV;            // every lane's column groups lie inside the box
 
     const bool active = mycw > 0;
     if (active && lane == 0) {
         const int pre = cnt < D ? cnt : D;
-        for (int d = 0; d < pre; ++d) issue(d, d);
+        for (int d = 0; d < pre; ++d) issue(row0 + d * stride_rows, d);
     }
     int issued = active ? (cnt < D ? cnt : D) : 0;
     int done = 0;
@@ -118,22 +121,21 @@ __global__ void __launch_bounds__(NW * 32, 1) k_stream_split(const SplitParams p
     int since_flush = 0;
     int d = 0;
     uint32_t phase = 0;
+    float y_next = 0.f;
+    if constexpr (!PREDICT) {
+        if (cnt > 0 && row0 + myr < p.m) y_next = __ldg(p.y + row0 + myr);
+    }
 
     for (int i = 0; i < cnt; ++i) {
-        const long long row0 = (static_cast<long long>(i) * gridDim.x + blockIdx.x) * RB;
-        const long long left = p.m - row0;
-        const int rows = left < RB ? static_cast<int>(left) : RB;
-        const bool myvalid = myr < rows;
-        float yv = 0.f;
+        const bool myvalid = row0 + myr < p.m;
+        const float yv = y_next;
         if constexpr (!PREDICT) {
-            if (myvalid) yv = __ldg(p.y + row0 + myr);
+            const long long rn = static_cast<long long>(row0) + stride_rows + myr;
+            y_next = (i + 1 < cnt && rn < p.m) ? __ldg(p.y + rn) : 0.f;
         }
 
         float4 x[RB][NV];
-#pragma unroll
-        for (int r = 0; r < RB; ++r)
-#pragma unroll
-            for (int k = 0; k < NV; ++k) x[r][k] = make_float4(0.f, 0.f, 0.f, 0.f);
+        bool have = false;
         if (active && !aborted) {
             bool ok = mbar_wait_bounded(&my_bars[d], phase, abort_flag);
             ok = __all_sync(FULL, ok);
@@ -141,26 +143,38 @@ __global__ void __launch_bounds__(NW * 32, 1) k_stream_split(const SplitParams p
                 aborted = true;
             } else {
                 done = i + 1;
-                const unsigned char* stage = my_stages + static_cast<size_t>(d) * stage_stride;
+                have = true;
+                const float4* t4 = reinterpret_cast<const float4*>(my_stages + static_cast<size_t>(d) * stage_stride);
+                if (full_cw) {
 #pragma unroll
-                for (int r = 0; r < RB; ++r) {
-                    const float4* t4 = reinterpret_cast<const float4*>(stage + r * row_stride);
+                    for (int r = 0; r < RB; ++r)
 #pragma unroll
-                    for (int k = 0; k < NV; ++k) {
-                        const int loc = lane + 32 * k;
-                        if (r < rows && loc < mycw) x[r][k] = t4[loc];
-                    }
+                        for (int k = 0; k < NV; ++k) x[r][k] = t4[r * (32 * NV) + lane + 32 * k];
+                } else {
+#pragma unroll
+                    for (int r = 0; r < RB; ++r)
+#pragma unroll
+                        for (int k = 0; k < NV; ++k) {
+                            const int loc = lane + 32 * k;
+                            x[r][k] = loc < CW ? t4[r * CW + loc] : make_float4(0.f, 0.f, 0.f, 0.f);
+                        }
                 }
                 __syncwarp();
                 if (i + D < cnt) {
                     if (lane == 0) {
                         fence_proxy_async_smem();
-                        issue(i + D, d);
+                        issue(row0 + D * stride_rows, d);
                     }
                     issued = i + D + 1;
                 }
                 if (++d == D) { d = 0; phase ^= 1u; }
             }
+        }
+        if (!have) {
+#pragma unroll
+            for (int r = 0; r < RB; ++r)
+#pragma unroll
+                for (int k = 0; k < NV; ++k) x[r][k] = make_float4(0.f, 0.f, 0.f, 0.f);
         }
 
         float v[RB];
@@ -180,17 +194,26 @@ __global__ void __launch_bounds__(NW * 32, 1) k_stream_split(const SplitParams p
         float* zp = zpart + (i & 1) * (NW * RB);
         if (owner) zp[warp * RB + myr] = v[0];
         __syncthreads();
-        float z = bval;
+        // the lanes that share a row add PER_DUP partials each (warp order), then a butterfly: one fixed order, same in every warp
+        float zs = 0.f;
 #pragma unroll
-        for (int wi = 0; wi < NW; ++wi) z += zp[wi * RB + myr];
+        for (int j = 0; j < PER_DUP; ++j) zs += zp[(dup * PER_DUP + j) * RB + myr];
+#pragma unroll
+        for (int msk = DUP / 2; msk >= 1; msk >>= 1) zs += __shfl_xor_sync(FULL, zs, msk);
+        const float z = zs + bval;
 
         if constexpr (PREDICT) {
             if (warp == 0 && owner && myvalid) p.labels[row0 + myr] = z >= p.cut ? 1 : 0;
         } else {
-            float e, L;
-            logistic_terms(z, yv, e, L);
-            if (!myvalid) { e = 0.f; L = 0.f; }
-            if (warp == 0 && owner) { se += e; sl += L; }
+            float e;
+            if (warp == 0) {                       // warp-uniform: the loss term is needed once per row
+                float L;
+                logistic_terms(z, yv, e, L);
+                if (owner && myvalid) { se += e; sl += L; }
+            } else {
+                e = logistic_err(z, yv);
+            }
+            if (!myvalid) e = 0.f;
 #pragma unroll
             for (int r = 0; r < RB; ++r) {
                 const float er = __shfl_sync(FULL, e, r << SHIFT);
@@ -213,6 +236,7 @@ __global__ void __launch_bounds__(NW * 32, 1) k_stream_split(const SplitParams p
                 dse += se; dsl += sl; se = 0.f; sl = 0.f;
             }
         }
+        row0 += stride_rows;
     }
 
     if (aborted) {

@@ -81,7 +81,7 @@ def test_plan_wide_rows_are_split_across_warps(m, n, nv, rb):
     assert p["variant"] == 1 and p["vec_per_lane"] == nv and p["rows_per_batch"] == rb
     assert p["threads"] == 512 and p["grid"] == min(-(-m // rb), 148)
     cw = -(-(n // 4) // 16)
-    stage = rb * (-(-cw * 16 // 128) * 128)
+    stage = -(-rb * cw * 16 // 128) * 128
     assert 1 <= p["stages"] <= 4 and p["smem_bytes"] == 2048 + 16 * p["stages"] * stage <= 227 * 1024
 
 
