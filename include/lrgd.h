@@ -119,6 +119,25 @@ int lr_fit_tol(lr_ctx* ctx, const float* d_X, const float* d_y, int64_t m, int32
                int32_t* iters_done, float* grad_norm, void* stream);
 
 /*
+ * Gradient descent with an L2 penalty and momentum.  The paper lists regularisation and other optimisers as future
+ * work (Section V) without defining them; the textbook definitions are used:
+ *   loss = data loss + (l2/2)*||w||^2 (the bias is not penalised);  g_w = X^T err/m + l2*w,  g_b = sum err/m;
+ *   v <- momentum*v + g;   w, b <- w, b - lr*v,   or with nesterov != 0:  w, b - lr*(g + momentum*v)  (v updated first).
+ * l2 = 0, momentum = 0 reproduces lr_fit bit for bit.  d_velocity is NULL (a context-owned velocity, zeroed at the start of
+ * the call) or a device array [n+1] (w entries, then b) that is read and updated, so a run can be split across calls.
+ * d_loss_hist (NULL or [iters]) receives the penalised loss at the parameters before each update.
+ * Errors as lr_fit, plus LR_ERR_VALUE for l2 < 0 or momentum outside [0, 1).
+ */
+typedef struct lr_opt {
+    float l2;
+    float momentum;
+    int32_t nesterov;
+} lr_opt;
+int lr_fit_opt(lr_ctx* ctx, const float* d_X, const float* d_y, int64_t m, int32_t n,
+               float lr, int32_t iters, const lr_opt* opt,
+               float* d_w, float* d_b, float* d_velocity, float* d_loss_hist, void* stream);
+
+/*
  * d_labels[i] = 1 if sigmoid(x_i.w + b) >= thr else 0, decided in logit space as
  * z_i >= log(thr/(1-thr)) evaluated in fp32 (the paper reports f1 but states no threshold; the
  * caller supplies it).  0 < thr < 1.  d_labels is uint8 [m].

@@ -38,6 +38,7 @@ def _load():
         lib.oracle_loss_grad.argtypes = [P, P, I64, I32, P, D, P, P, P]
         lib.oracle_fit.argtypes = [P, P, I64, I32, D, I32, P, P, P, P, P, ctypes.c_int]
         lib.oracle_predict.argtypes = [P, I64, I32, P, D, D, P, P]
+        lib.oracle_fit_opt.argtypes = [P, P, I64, I32, D, I32, D, D, ctypes.c_int, P, P, P, P]
         lib.oracle_fit_tol.argtypes = [P, P, I64, I32, D, D, I32, P, P, P, P, P, P]
         lib.oracle_f1.argtypes = [P, P, I64, P, P, P, P]
         _lib = lib
@@ -122,6 +123,22 @@ def fit_tol(X, y, lr, eps, max_iters, w0=None, b0=0.0):
         raise ValueError("oracle_fit_tol: bad arguments")
     k = done.value
     return w, float(b[0]), k, nrm.value, lh[:k], gh[:k]
+
+
+def fit_opt(X, y, lr, iters, l2=0.0, momentum=0.0, nesterov=False, w0=None, b0=0.0, vel0=None):
+    """GD with an L2 penalty and momentum.  Returns ``(w, b, vel[n+1], loss_hist)``."""
+    X = _f32(X)
+    m, n = X.shape
+    y = _f32(y, (m,))
+    w = np.zeros(n) if w0 is None else np.array(w0, dtype=np.float64).copy()
+    b = np.array([float(b0)])
+    vel = np.zeros(n + 1) if vel0 is None else np.array(vel0, dtype=np.float64).copy()
+    lh = np.zeros(max(iters, 1))
+    rc = _load().oracle_fit_opt(_ptr(X), _ptr(y), m, n, float(lr), int(iters), float(l2), float(momentum), int(bool(nesterov)),
+                                _ptr(w), _ptr(b), _ptr(vel), _ptr(lh))
+    if rc != 0:
+        raise ValueError("oracle_fit_opt: bad arguments")
+    return w, float(b[0]), vel, lh[:iters]
 
 
 def predict(X, w, b, thr, return_z=False):

@@ -32,7 +32,10 @@
  * Pins (tests, CPU only): ln 2 at w=b=0, X^T(0.5-y)/m at w=b=0, closed-form one- and two-row cases,
  * central finite differences, label-flip symmetry, row duplication, ones-column/bias equivalence,
  * saturation at |z|=40, descent-lemma monotonicity, planted-w* recovery, float64 autograd of a
- * library BCE-with-logits, brute-force predict and hand-counted F1.  No function here is unpinned.
+ * library BCE-with-logits, brute-force predict and hand-counted F1; the stopping rule against the fixed-count
+ * trajectory and its recorded norms; the penalty/momentum update against three steps done by hand from
+ * oracle_loss_grad, central differences of the penalised loss and the vanishing penalised gradient at its fixed
+ * point.  No function here is unpinned.
  */
 #include <math.h>
 #include <stdint.h>
@@ -168,6 +171,37 @@ int oracle_fit_tol(const float* X, const float* y, int64_t m, int32_t n, double 
         *iters_done = t + 1;
         *grad_norm = nrm;
         if (nrm <= eps) break;                                      /* Algorithm 7: test after the update */
+    }
+    free(g);
+    return 0;
+}
+
+/*
+ * Gradient descent with an L2 penalty on w and (optionally Nesterov) momentum.  The paper only names these as future
+ * work (Section V); the definitions are the textbook ones:
+ *   loss = data loss + (l2/2) sum_j w_j^2 ;  g_w = grad_w + l2*w ;  g_b = grad_b   (bias not penalised)
+ *   v <- mu*v + g ;  (w,b) <- (w,b) - lr*v            heavy ball
+ *                    (w,b) <- (w,b) - lr*(g + mu*v)   Nesterov form, v already updated
+ * vel[n+1] (w entries then b) is in/out.  loss_hist (nullable) gets the penalised loss before each update.
+ */
+int oracle_fit_opt(const float* X, const float* y, int64_t m, int32_t n, double lr, int32_t iters, double l2, double mu,
+                   int nesterov, double* w, double* b, double* vel, double* loss_hist) {
+    if (!X || !y || !w || !b || !vel || m < 1 || n < 1 || iters < 0 || !(l2 >= 0.0) || !(mu >= 0.0 && mu < 1.0)) return -1;
+    double* g = (double*)malloc(sizeof(double) * (size_t)n);
+    if (!g) return -1;
+    for (int32_t t = 0; t < iters; ++t) {
+        double loss, gb;
+        if (oracle_loss_grad(X, y, m, n, w, *b, &loss, g, &gb) != 0) { free(g); return -1; }
+        double sq = 0.0;
+        for (int32_t j = 0; j < n; ++j) sq += w[j] * w[j];
+        if (loss_hist) loss_hist[t] = loss + 0.5 * l2 * sq;
+        for (int32_t j = 0; j <= n; ++j) {
+            double gj = j < n ? g[j] + l2 * w[j] : gb;
+            double v = mu * vel[j] + gj;
+            double step = nesterov ? gj + mu * v : v;
+            vel[j] = v;
+            if (j < n) w[j] -= lr * step; else *b -= lr * step;
+        }
     }
     free(g);
     return 0;

@@ -21,7 +21,7 @@ LR_ERR_NULL, LR_ERR_SHAPE, LR_ERR_ALIGNMENT, LR_ERR_VALUE, LR_ERR_CUDA, LR_ERR_T
 EXPORTS = ["lr_plan_query", "lr_create", "lr_destroy", "lr_loss_grad", "lr_fit", "lr_predict", "lr_shard_sums",
            "lr_apply_sums", "lr_fit_host",
            "lr_predict_host", "lr_profile_enable", "lr_profile_read", "lr_launch_count", "lr_last_device_status",
-           "lr_last_cuda_error", "lr_status_string", "lr_loss_grad_noalloc", "lr_fit_tol"]
+           "lr_last_cuda_error", "lr_status_string", "lr_loss_grad_noalloc", "lr_fit_tol", "lr_fit_opt"]
 
 
 class LrPlan(ctypes.Structure):
@@ -30,6 +30,10 @@ class LrPlan(ctypes.Structure):
 
     def as_dict(self):
         return {k: int(getattr(self, k)) for k, _ in self._fields_}
+
+
+class LrOpt(ctypes.Structure):
+    _fields_ = [("l2", ctypes.c_float), ("momentum", ctypes.c_float), ("nesterov", ctypes.c_int32)]
 
 
 class LrError(RuntimeError):
@@ -60,6 +64,7 @@ def lib() -> ctypes.CDLL:
         L.lr_apply_sums.argtypes = [P, P, I32, I64, I32, F, P, P, P, P]
         L.lr_fit_tol.argtypes = [P, P, P, I64, I32, F, F, I32, I32, P, P, P, P, ctypes.POINTER(I32),
                                  ctypes.POINTER(F), P]
+        L.lr_fit_opt.argtypes = [P, P, P, I64, I32, F, I32, ctypes.POINTER(LrOpt), P, P, P, P, P]
         L.lr_loss_grad_noalloc.argtypes = [I32, P, P, I64, I32, P, P, P, P, P, P, P]
         L.lr_fit_host.argtypes = [P, P, P, I64, I32, F, I32, P, P, P]
         L.lr_predict_host.argtypes = [P, P, I64, I32, P, P, F, P]
@@ -174,6 +179,16 @@ class Context:
                               self._stream())
         self._check(rc, "lr_fit_tol")
         return done.value, nrm.value
+
+    def fit_opt(self, X, y, lr, iters, w, b, l2=0.0, momentum=0.0, nesterov=False, velocity=None, loss_hist=None):
+        """GD with an L2 penalty and (Nesterov) momentum, in place on w, b (and ``velocity`` [n+1] when given)."""
+        m, n = X.shape
+        opt = LrOpt(float(l2), float(momentum), int(bool(nesterov)))
+        rc = lib().lr_fit_opt(self._h, _dev_ptr(X, torch.float32, "X"), _dev_ptr(y, torch.float32, "y"), m, n, float(lr),
+                              int(iters), ctypes.byref(opt), _dev_ptr(w, torch.float32, "w"), _dev_ptr(b, torch.float32, "b"),
+                              _dev_ptr(velocity, torch.float32, "velocity"), _dev_ptr(loss_hist, torch.float32, "loss_hist"),
+                              self._stream())
+        self._check(rc, "lr_fit_opt")
 
     def predict(self, X, w, b, thr):
         m, n = X.shape

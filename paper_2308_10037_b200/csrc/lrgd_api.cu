@@ -119,6 +119,9 @@ struct lr_ctx {
     TolState* d_tol = nullptr;                      // stopping-rule state of lr_fit_tol
     double* d_gbuf = nullptr;                       // [n_max+1] gradient entries for the norm
     TolState* h_tol = nullptr;                      // pinned host mirror
+    float* d_vel = nullptr;                         // [n_max+1] velocity of lr_fit_opt when the caller passes none
+    double* d_oscr = nullptr;                       // [n_max+2] scratch of the optimiser reduction
+    unsigned int* d_oticket = nullptr;
     // buffers of the host-pointer entry points (grown on demand)
     void* d_hX = nullptr; size_t hX_bytes = 0;
     void* d_hy = nullptr; size_t hy_bytes = 0;
@@ -337,6 +340,10 @@ int lr_create(lr_ctx** out, int32_t device, int32_t n_max) {
     if (e == cudaSuccess) e = cudaMemset(c->d_tol, 0, sizeof(TolState));
     if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&c->d_gbuf), (size_t(n_max) + 1) * sizeof(double));
     if (e == cudaSuccess) e = cudaMallocHost(reinterpret_cast<void**>(&c->h_tol), sizeof(TolState));
+    if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&c->d_vel), (size_t(n_max) + 1) * sizeof(float));
+    if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&c->d_oscr), (size_t(n_max) + 2) * sizeof(double));
+    if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&c->d_oticket), sizeof(unsigned int));
+    if (e == cudaSuccess) e = cudaMemset(c->d_oticket, 0, sizeof(unsigned int));
     if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&c->hstream, cudaStreamNonBlocking);
     if (prev >= 0) cudaSetDevice(prev);
     if (e != cudaSuccess) {
@@ -345,6 +352,9 @@ int lr_create(lr_ctx** out, int32_t device, int32_t n_max) {
         if (c->d_tol) cudaFree(c->d_tol);
         if (c->d_gbuf) cudaFree(c->d_gbuf);
         if (c->h_tol) cudaFreeHost(c->h_tol);
+        if (c->d_vel) cudaFree(c->d_vel);
+        if (c->d_oscr) cudaFree(c->d_oscr);
+        if (c->d_oticket) cudaFree(c->d_oticket);
         delete c;
         return rc != LR_OK ? rc : LR_ERR_CUDA;
     }
@@ -364,6 +374,9 @@ int lr_destroy(lr_ctx* ctx) {
         cudaFree(ctx->d_tol);
         cudaFree(ctx->d_gbuf);
         if (ctx->h_tol) cudaFreeHost(ctx->h_tol);
+        cudaFree(ctx->d_vel);
+        cudaFree(ctx->d_oscr);
+        cudaFree(ctx->d_oticket);
         cudaFree(ctx->d_hX);
         cudaFree(ctx->d_hy);
         cudaFree(ctx->d_hw);
@@ -455,6 +468,43 @@ int lr_fit_tol(lr_ctx* ctx, const float* d_X, const float* d_y, int64_t m, int32
     }
     *iters_done = ctx->h_tol->iters_done;
     *grad_norm = static_cast<float>(ctx->h_tol->grad_norm);
+    return LR_OK;
+}
+
+int lr_fit_opt(lr_ctx* ctx, const float* d_X, const float* d_y, int64_t m, int32_t n, float lr, int32_t iters,
+               const lr_opt* opt, float* d_w, float* d_b, float* d_velocity, float* d_loss_hist, void* stream) {
+    int rc = check_common(ctx, d_X, m, n, d_w, d_b);
+    if (rc != LR_OK) return rc;
+    if (!d_y || !opt) return LR_ERR_NULL;
+    if (iters < 0) return LR_ERR_SHAPE;
+    if (!aligned(d_y, 4) || (d_loss_hist && !aligned(d_loss_hist, 4)) || (d_velocity && !aligned(d_velocity, 4)))
+        return LR_ERR_ALIGNMENT;
+    if (!std::isfinite(lr) || !(opt->l2 >= 0.f) || !std::isfinite(opt->l2) || !(opt->momentum >= 0.f && opt->momentum < 1.f))
+        return LR_ERR_VALUE;
+    lr_plan P;
+    rc = make_plan(m, n, aligned(d_X, 16), ctx->sm_count, &P);
+    if (rc != LR_OK) return rc;
+    if (iters == 0) return LR_OK;
+    DeviceGuard g(ctx);
+    if (!g.ok) return LR_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    float* vel = d_velocity;
+    if (!vel) {
+        vel = ctx->d_vel;
+        LR_CK(ctx, cudaMemsetAsync(vel, 0, (size_t(n) + 1) * sizeof(float), st));
+    }
+    for (int32_t t = 0; t < iters; ++t) {
+        rc = launch_stream_pass(ctx, P, Pass{d_X, d_y, m, n, d_w, d_b}, nullptr, 0.f, st);
+        if (rc != LR_OK) return rc;
+        OptParams op{};
+        op.partial = ctx->d_partial; op.G = P.grid; op.n = n; op.inv_m = 1.0 / double(m); op.lr = double(lr);
+        op.l2 = double(opt->l2); op.mu = double(opt->momentum); op.nesterov = opt->nesterov ? 1 : 0;
+        op.w = d_w; op.b = d_b; op.vel = vel; op.loss_out = d_loss_hist ? d_loss_hist + t : nullptr;
+        op.scratch = ctx->d_oscr; op.ticket = ctx->d_oticket;
+        k_reduce_opt<<<(n + 2 + 31) / 32, dim3(32, kRedSlices), 0, st>>>(op);
+        LR_CK(ctx, cudaGetLastError());
+        ctx->launches += 1;
+    }
     return LR_OK;
 }
 

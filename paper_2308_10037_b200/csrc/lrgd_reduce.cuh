@@ -113,4 +113,86 @@ __global__ void __launch_bounds__(32 * kRedSlices) k_reduce_update(const ReduceP
     }
 }
 
+// ------------------------------------------------------------------------------------------------------
+// Second stage with an L2 penalty and momentum (the paper names regularisation and other optimisers as future
+// work, Section V, without defining them; the definitions used here are the textbook ones):
+//   loss   = data loss + (l2/2) * ||w||^2                (the bias is not penalised)
+//   g_w    = X^T err / m + l2 * w ,  g_b = sum err / m
+//   v     <- mu * v + g                                   (heavy-ball velocity, one entry per parameter)
+//   w, b  <- w, b - lr * v            or, with nesterov:  w, b - lr * (g + mu * v)   (v already updated)
+// Same fixed-order column reduction as k_reduce_update; the block that finishes last adds the squared old
+// weights in index order and writes the penalised loss.
+struct OptParams {
+    const double* partial;    // [G][n+2]
+    int G;
+    int n;
+    double inv_m;
+    double lr;
+    double l2;
+    double mu;
+    int nesterov;
+    float* w;
+    float* b;
+    float* vel;               // [n+1] in/out
+    float* loss_out;          // nullable
+    double* scratch;          // [n+2]: squared old weights [n], spare, data loss
+    unsigned int* ticket;
+};
+
+__global__ void __launch_bounds__(32 * kRedSlices) k_reduce_opt(const OptParams p) {
+    __shared__ double sh[kRedSlices][33];
+    __shared__ int is_last;
+    const int col = blockIdx.x * 32 + threadIdx.x;
+    const int slice = threadIdx.y;
+    const int stride = p.n + 2;
+    const int per = (p.G + kRedSlices - 1) / kRedSlices;
+    const int g0 = slice * per;
+    const int g1 = g0 + per < p.G ? g0 + per : p.G;
+    double s = 0.0;
+    if (col < stride) {
+        const double* src = p.partial + col;
+#pragma unroll 8
+        for (int g = g0; g < g1; ++g) s += src[static_cast<size_t>(g) * stride];
+    }
+    sh[slice][threadIdx.x] = s;
+    __syncthreads();
+    if (slice == 0 && col < stride) {
+        double t = 0.0;
+#pragma unroll
+        for (int k = 0; k < kRedSlices; ++k) t += sh[k][threadIdx.x];
+        const double mean = t * p.inv_m;
+        if (col <= p.n) {
+            float* param = col < p.n ? p.w + col : p.b;
+            const double old = static_cast<double>(*param);
+            const double g = col < p.n ? mean + p.l2 * old : mean;
+            const double v = p.mu * static_cast<double>(p.vel[col]) + g;
+            const double step = p.nesterov ? g + p.mu * v : v;
+            p.vel[col] = static_cast<float>(v);
+            *param = static_cast<float>(old - p.lr * step);
+            if (col < p.n) p.scratch[col] = old * old;
+        } else {
+            p.scratch[p.n + 1] = mean;            // data loss
+        }
+    }
+    if (p.loss_out == nullptr) return;
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0 && threadIdx.y == 0) {
+        const unsigned int t = atomicAdd(p.ticket, 1u);
+        is_last = (t == gridDim.x - 1) ? 1 : 0;
+    }
+    __syncthreads();
+    if (!is_last || threadIdx.y != 0) return;
+    __threadfence();
+    const volatile double* sc = p.scratch;
+    double q = 0.0;
+    for (int c = threadIdx.x; c < p.n; c += 32) q += sc[c];
+#pragma unroll
+    for (int msk = 16; msk >= 1; msk >>= 1) q += __shfl_xor_sync(0xffffffffu, q, msk);
+    if (threadIdx.x == 0) {
+        p.loss_out[0] = static_cast<float>(sc[p.n + 1] + 0.5 * p.l2 * q);
+        *p.ticket = 0u;
+    }
+}
+
 }  // namespace lrgd

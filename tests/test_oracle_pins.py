@@ -254,3 +254,56 @@ def test_stopping_rule_follows_algorithm_7():
     # no iterations allowed: nothing happens
     w3, b3, k3, n3, _, _ = oracle.fit_tol(X, y, lr, 1.0, 0)
     assert k3 == 0 and n3 == -1.0 and not w3.any() and b3 == 0.0
+
+
+def test_penalty_and_momentum_follow_their_definitions():
+    X, y, _, _ = datagen.random_problem(1200, 5, seed=13)
+    lr, l2, mu = 0.4, 0.3, 0.7
+    # no penalty, no momentum: the plain fit
+    w0, b0, v0, lh0 = oracle.fit_opt(X, y, lr, 9)
+    wf, bf, lhf = oracle.fit(X, y, lr, 9)
+    assert np.array_equal(w0, wf) and b0 == bf and np.array_equal(lh0, lhf)
+    # heavy ball, three steps by hand from the plain loss/gradient routine
+    w, b, v = np.zeros(5), 0.0, np.zeros(6)
+    losses = []
+    for _ in range(3):
+        L, g, gb = oracle.loss_grad(X, y, w, b)
+        losses.append(L + 0.5 * l2 * float(w @ w))
+        gfull = np.concatenate([g + l2 * w, [gb]])           # the bias carries no penalty
+        v = mu * v + gfull
+        w, b = w - lr * v[:5], b - lr * v[5]
+    w1, b1, v1, lh1 = oracle.fit_opt(X, y, lr, 3, l2=l2, momentum=mu)
+    np.testing.assert_allclose(w1, w, atol=1e-15, rtol=0)
+    assert abs(b1 - b) < 1e-15
+    np.testing.assert_allclose(v1, v, atol=1e-15, rtol=0)
+    np.testing.assert_allclose(lh1, losses, atol=1e-15, rtol=0)
+    # Nesterov form, same bookkeeping
+    w, b, v = np.zeros(5), 0.0, np.zeros(6)
+    for _ in range(3):
+        _, g, gb = oracle.loss_grad(X, y, w, b)
+        gfull = np.concatenate([g + l2 * w, [gb]])
+        v = mu * v + gfull
+        step = gfull + mu * v
+        w, b = w - lr * step[:5], b - lr * step[5]
+    w2, b2, v2, _ = oracle.fit_opt(X, y, lr, 3, l2=l2, momentum=mu, nesterov=True)
+    np.testing.assert_allclose(w2, w, atol=1e-15, rtol=0)
+    assert abs(b2 - b) < 1e-15 and not np.allclose(w2, w1)
+    # the penalised gradient is the gradient of the penalised loss (central differences)
+    wp = np.array([0.3, -0.2, 0.5, 0.1, -0.4])
+    _, g, _ = oracle.loss_grad(X, y, wp, 0.2)
+    for j in range(5):
+        d = np.zeros(5)
+        d[j] = 1e-5
+        f = lambda ww: oracle.loss_grad(X, y, ww, 0.2)[0] + 0.5 * l2 * float(ww @ ww)
+        assert abs((f(wp + d) - f(wp - d)) / 2e-5 - (g[j] + l2 * wp[j])) < 1e-8
+    # at the fixed point of the penalised problem the penalised gradient vanishes and ||w|| shrinks with the penalty
+    wa, ba, _, _ = oracle.fit_opt(X, y, 1.0, 400, l2=0.5, momentum=0.5)
+    _, g, gb = oracle.loss_grad(X, y, wa, ba)
+    assert np.linalg.norm(np.concatenate([g + 0.5 * wa, [gb]])) < 1e-10
+    wb, _, _, _ = oracle.fit_opt(X, y, 1.0, 400, l2=0.05, momentum=0.5)
+    assert np.linalg.norm(wa) < np.linalg.norm(wb)
+    # resuming with the returned velocity continues the same trajectory
+    wa1, ba1, va1, _ = oracle.fit_opt(X, y, lr, 4, l2=l2, momentum=mu)
+    wa2, ba2, va2, _ = oracle.fit_opt(X, y, lr, 3, l2=l2, momentum=mu, w0=wa1, b0=ba1, vel0=va1)
+    wa3, ba3, va3, _ = oracle.fit_opt(X, y, lr, 7, l2=l2, momentum=mu)
+    assert np.array_equal(wa2, wa3) and ba2 == ba3 and np.array_equal(va2, va3)
