@@ -185,6 +185,14 @@ int lr_launch_count(lr_ctx* ctx, int64_t* out);
 /* Synchronises the device and returns in *out the device status word: LR_OK or LR_ERR_TIMEOUT.  Clears it. */
 int lr_last_device_status(lr_ctx* ctx, int32_t* out);
 
+/*
+ * Exercises the give-up path of the bounded device-side waits without harming the device: enqueues a one-warp
+ * kernel that waits on an mbarrier which is completed up front (arm != 0) or never (arm == 0), for at most limit_ms
+ * (1..1000) milliseconds.  When the wait runs out the kernel sets the device status word, exactly as a streaming kernel
+ * whose copy never lands would, and returns; lr_last_device_status then reports LR_ERR_TIMEOUT and clears it.
+ */
+int lr_selftest_wait(lr_ctx* ctx, int32_t arm, int32_t limit_ms, void* stream);
+
 /* The cudaError_t value of the most recent failing CUDA call made through this context (0 if none). */
 int lr_last_cuda_error(lr_ctx* ctx);
 

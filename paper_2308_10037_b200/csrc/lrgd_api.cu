@@ -655,6 +655,17 @@ int lr_last_device_status(lr_ctx* ctx, int32_t* out) {
     return LR_OK;
 }
 
+int lr_selftest_wait(lr_ctx* ctx, int32_t arm, int32_t limit_ms, void* stream) {
+    if (!ctx) return LR_ERR_NULL;
+    if (limit_ms < 1 || limit_ms > 1000) return LR_ERR_VALUE;
+    DeviceGuard g(ctx);
+    if (!g.ok) return LR_ERR_CUDA;
+    k_wait_probe<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(ctx->d_status, 1000000ull * unsigned(limit_ms), arm ? 1 : 0);
+    LR_CK(ctx, cudaGetLastError());
+    ctx->launches += 1;
+    return LR_OK;
+}
+
 int lr_last_cuda_error(lr_ctx* ctx) { return ctx ? ctx->last_cuda : 0; }
 
 const char* lr_status_string(int code) {

@@ -53,9 +53,10 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
     return ok != 0;
 }
 
-// Waits for the phase with the given parity to complete, for at most kWaitLimitNs.  On expiry (or when
-// another thread of the CTA has already given up) raises *abort_flag and returns false.
-__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+// Waits for the phase with the given parity to complete, for at most limit_ns.  On expiry (or when another
+// thread of the CTA has already given up) raises *abort_flag and returns false.
+__device__ __forceinline__ bool mbar_wait_bounded_ns(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
+                                                     unsigned long long limit_ns) {
     if (mbar_try_wait(bar, parity)) return true;
     const unsigned long long t0 = global_timer_ns();
     for (;;) {
@@ -63,11 +64,31 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity
         for (int i = 0; i < 32; ++i)
             if (mbar_try_wait(bar, parity)) return true;
         if (*abort_flag) return false;
-        if (global_timer_ns() - t0 > kWaitLimitNs) {
+        if (global_timer_ns() - t0 > limit_ns) {
             *abort_flag = 1;
             return false;
         }
     }
+}
+
+__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+    return mbar_wait_bounded_ns(bar, parity, abort_flag, kWaitLimitNs);
+}
+
+// One warp waits on an mbarrier that is completed up front (arm != 0) or never (arm == 0), with the given limit; on
+// expiry it sets the status word exactly as the streaming kernels do.  Used to exercise the give-up path on purpose.
+__global__ void k_wait_probe(int* status, unsigned long long limit_ns, int arm) {
+    __shared__ uint64_t bar;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) {
+        mbar_init(&bar, 1);
+        abort_flag = 0;
+        fence_mbar_init();
+    }
+    __syncthreads();
+    if (arm && threadIdx.x == 0) mbar_arrive(&bar);
+    const bool ok = mbar_wait_bounded_ns(&bar, 0u, &abort_flag, limit_ns);
+    if (!ok && threadIdx.x == 0) atomicExch(status, kStatusTimeout);
 }
 
 __device__ __forceinline__ uint64_t l2_policy_evict_first() {

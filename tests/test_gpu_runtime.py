@@ -1,0 +1,68 @@
+"""Runtime behaviour around the kernels: the bounded-wait give-up path, and the row-sharded driver on a real
+process group (one rank: the only size a single GPU allows).
+
+Nothing here faults, traps or hangs the device: the give-up test waits a few milliseconds on a barrier that
+nothing completes, the kernel then returns normally with the status word set, and the context stays usable.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from _parity import LOSS_TOL, W_TOL, rel_l2
+from paper_2308_10037_b200 import api, datagen
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    from paper_2308_10037_b200 import build
+    build.build()
+    c = api.Context(n_max=512, device=0)
+    yield c
+    c.close()
+
+
+def test_bounded_wait_gives_up_and_reports(ctx):
+    ctx.selftest_wait(arm=True, limit_ms=20)                 # the barrier completes: no status
+    assert ctx.device_status() == 0
+    ctx.selftest_wait(arm=False, limit_ms=20)                # nothing completes it: the kernel gives up after 20 ms
+    assert ctx.device_status() == api.LR_ERR_TIMEOUT
+    assert api.status_string(api.LR_ERR_TIMEOUT) == "a bounded device-side wait expired"
+    assert ctx.device_status() == 0                          # reading clears the word
+    # the context and the device are still fine
+    X, y, w, b = datagen.random_problem(5000, 64, seed=21)
+    dl, dg, dg0 = ctx.loss_grad(torch.from_numpy(X).cuda(), torch.from_numpy(y).cuda(), torch.from_numpy(w).cuda(),
+                                torch.tensor([b], device="cuda"))
+    L, g, g0 = oracle.loss_grad(X, y, w, b)
+    assert abs(dl.item() - L) <= LOSS_TOL and rel_l2(dg.cpu().numpy(), g) <= 1e-5
+    assert ctx.device_status() == 0
+    with pytest.raises(api.LrError):
+        ctx.selftest_wait(arm=False, limit_ms=5000)          # limits above one second are refused
+
+
+def test_sharded_driver_on_a_one_rank_nccl_group(ctx):
+    import torch.distributed as dist
+    from paper_2308_10037_b200 import parallel
+    if dist.is_initialized():
+        pytest.skip("a process group already exists in this process")
+    dist.init_process_group("nccl", init_method="tcp://127.0.0.1:29871", rank=0, world_size=1,
+                            device_id=torch.device("cuda", 0))
+    try:
+        wl = datagen.scaled(datagen.WORKLOADS["cfg3"], 30_001)
+        X, y, _, _ = datagen.generate(wl)
+        dX, dy = torch.from_numpy(X).cuda(), torch.from_numpy(y).cuda()
+        w = torch.zeros(wl.n, device="cuda")
+        b = torch.zeros(1, device="cuda")
+        hist = torch.empty(8, device="cuda")
+        parallel.fit_sharded_cuda(ctx, dX, dy, wl.m, wl.lr, 8, w, b, loss_hist=hist)
+        torch.cuda.synchronize()
+        w_ref, b_ref, lh_ref = oracle.fit(X, y, wl.lr, 8)
+        assert rel_l2(np.concatenate([w.cpu().numpy(), b.cpu().numpy()]), np.concatenate([w_ref, [b_ref]])) <= W_TOL
+        assert np.max(np.abs(hist.cpu().numpy() - lh_ref)) <= LOSS_TOL
+        # one shard, one rank: the same kernels and the same summation order as lr_fit -> identical bits
+        wf, bf = api.lr_fit(dX, dy, wl.lr, 8, ctx=ctx)
+        assert torch.equal(w, wf) and torch.equal(b, bf)
+    finally:
+        dist.destroy_process_group()
