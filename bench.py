@@ -10,7 +10,8 @@ far larger than L2, so every iteration streams X from HBM).  One JSON line is pr
   value      iterations/s with X, y resident in HBM (CUDA events around one lr_fit call of K steps)
   e2e        the workload's own fit (its configured iteration count) through lr_fit_host: pinned host
              buffers in, parameters out, copies inside the timed region
-  roofline   the streaming kernel alone: (4mn + 4m) bytes per launch / its mean CUDA-event duration
+  roofline   narrow rows: the persistent kernel that runs all K timed iterations in one launch, K(4mn + 4m) bytes over
+             its duration; `single_pass` (and wide rows): one fused pass alone, from CUDA events around each launch
   cpu_baseline  the float64 CPU checker timed on this host on a bounded number of iterations
 
 With --gpus N > 1 (under torchrun) the rows are sharded: every rank holds one workload-sized block of
@@ -215,6 +216,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--rows", type=int, default=0, help="override the workload's row count (profiling on a smaller case)")
     ap.add_argument("--tol", default="", help="ALPHA,EPS: time-to-tolerance mode (Algorithm 7 stopping rule); --steps caps the updates")
+    ap.add_argument("--no-persistent", action="store_true", help="force two kernels per iteration in lr_fit")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
@@ -261,6 +263,8 @@ def main():
     dy = yh.to("cuda", non_blocking=True)
     torch.cuda.synchronize()
     ctx = api.Context(n_max=wl.n, device=local_rank)
+    if args.no_persistent:
+        ctx.set_persistent(False)
     w = torch.zeros(wl.n, dtype=torch.float32, device="cuda")
     b = torch.zeros(1, dtype=torch.float32, device="cuda")
     m_total = wl.m * world
@@ -320,11 +324,22 @@ def main():
     bytes_per_launch = 4 * wl.m * wl.n + 4 * wl.m
     achieved = bytes_per_launch / (k1_ms * 1e-3) / 1e9
     peak, peak_kind = measured_hbm_peak()
-    roofline = {"bound": "hbm", "kernel": "k_stream_rows (fused loss/gradient pass)", "achieved": achieved, "peak": peak,
-                "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
-                "traffic": (NCU_TRAFFIC_BYTES_PER_ROW[args.workload] * wl.m if args.workload in NCU_TRAFFIC_BYTES_PER_ROW else None),
-                "bytes_per_launch": bytes_per_launch, "avg_launch_ms": k1_ms, "launches_timed": n_l,
-                "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS}
+    plan = api.plan_query(wl.m, wl.n, sm_count=torch.cuda.get_device_properties(local_rank).multi_processor_count)
+    pass_kernel = {0: "k_stream_rows", 1: "k_stream_split", 2: "k_generic"}[plan["variant"]]
+    traffic = NCU_TRAFFIC_BYTES_PER_ROW[args.workload] * wl.m if args.workload in NCU_TRAFFIC_BYTES_PER_ROW else None
+    single_pass = {"kernel": f"{pass_kernel} (one fused loss/gradient pass, two-kernel form of lr_fit)", "achieved": achieved,
+                   "unit": "GB/s", "frac": achieved / peak, "bytes_per_launch": bytes_per_launch, "avg_launch_ms": k1_ms,
+                   "launches_timed": n_l, "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS}
+    if world == 1 and launches == 1:
+        # the timed region was ONE launch of the persistent kernel doing all K iterations (pass + reduction + update)
+        ach = bytes_per_launch * args.steps / (ms * 1e-3) / 1e9
+        roofline = {"bound": "hbm", "kernel": "k_fit_rows (persistent: all timed iterations in one cooperative launch)",
+                    "achieved": ach, "peak": peak, "unit": "GB/s", "frac": ach / peak, "peak_kind": f"of {peak_kind}",
+                    "traffic": traffic * args.steps if traffic else None, "bytes_per_launch": bytes_per_launch * args.steps,
+                    "avg_launch_ms": ms, "launches_timed": 1, "iterations_per_launch": args.steps,
+                    "frac_of_nominal_8TBs": ach / NOMINAL_HBM_GBS, "single_pass": single_pass}
+    else:
+        roofline = dict(single_pass, bound="hbm", peak=peak, peak_kind=f"of {peak_kind}", traffic=traffic)
 
     # ---- end to end through the host-pointer entry point ----
     e2e = None

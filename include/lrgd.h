@@ -95,9 +95,14 @@ int lr_loss_grad(lr_ctx* ctx, const float* d_X, const float* d_y, int64_t m, int
  * receives the loss at the parameters BEFORE update t.  iters == 0 is a no-op.
  * Results are bit-reproducible for a given shape and device, and fit(a) followed by fit(b) equals
  * fit(a+b) bit for bit.
+ * For rows of up to 512 columns (16-byte aligned X, n % 4 == 0) and iters >= 2 the whole call is ONE cooperative
+ * launch of a persistent kernel (grid barriers between the pass and the update; the HBM stream continues across
+ * iterations); otherwise two kernels per iteration.  Both give the same bits.  lr_set_persistent(ctx, 0) forces the
+ * two-kernel form (it is also used while lr_profile_enable is on, so that single launches can be timed).
  */
 int lr_fit(lr_ctx* ctx, const float* d_X, const float* d_y, int64_t m, int32_t n,
            float lr, int32_t iters, float* d_w, float* d_b, float* d_loss_hist, void* stream);
+int lr_set_persistent(lr_ctx* ctx, int32_t on);
 
 /*
  * Gradient descent with the paper's stopping rule (Algorithm 7's loop; the norm is Algorithm 4's):

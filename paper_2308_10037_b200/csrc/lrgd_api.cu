@@ -9,6 +9,7 @@
 #include <new>
 #include <vector>
 
+#include "lrgd_fit_rows.cuh"
 #include "lrgd_generic.cuh"
 #include "lrgd_reduce.cuh"
 #include "lrgd_stream_rows.cuh"
@@ -25,6 +26,7 @@ constexpr int kNW = LRGD_NW;                   // warps per CTA of the staged ke
 constexpr int kStageBudgetBytes = 208 * 1024;  // shared memory the warps' stages may take (227 KB per CTA on sm_100)
 constexpr int kMaxGridPerSm = 8;               // widest launch any variant uses, in CTAs per SM
 constexpr int kMaxProfiled = 4096;
+constexpr int kMaxDynamicSmem = 232448;         // opt-in dynamic shared memory per CTA on sm_100
 constexpr int64_t kMaxRows = int64_t(1) << 40;
 #ifndef LRGD_NV2_RB
 #define LRGD_NV2_RB 4                          // register batch (rows per warp) of the 132..256-column instantiation
@@ -122,6 +124,9 @@ struct lr_ctx {
     float* d_vel = nullptr;                         // [n_max+1] velocity of lr_fit_opt when the caller passes none
     double* d_oscr = nullptr;                       // [n_max+2] scratch of the optimiser reduction
     unsigned int* d_oticket = nullptr;
+    unsigned int* d_gbar = nullptr;                 // grid-barrier counter of the persistent fit kernel
+    bool coop = false;                              // device supports cooperative launches
+    bool persistent = true;                         // lr_fit may use the single-launch kernel
     // buffers of the host-pointer entry points (grown on demand)
     void* d_hX = nullptr; size_t hX_bytes = 0;
     void* d_hy = nullptr; size_t hy_bytes = 0;
@@ -220,6 +225,23 @@ cudaError_t launch_split(const lr_plan& P, const float* X, const SplitParams& sp
     if (e != cudaSuccess) return e;
     if (P.vec_per_lane == 2) return launch_split_t<2, 4, PRED>(P, tm, sp, st);
     return launch_split_t<1, 8, PRED>(P, tm, sp, st);
+}
+
+template <int NV, int LPR, int RB>
+cudaError_t launch_fit_t(const lr_plan& P, int smem, FitParams& fp, cudaStream_t st) {
+    auto kern = k_fit_rows<NV, LPR, RB, kNW>;
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) return e;
+    void* args[] = {&fp};
+    return cudaLaunchCooperativeKernel(reinterpret_cast<void*>(kern), dim3(P.grid), dim3(P.threads), args, size_t(smem), st);
+}
+
+cudaError_t launch_fit(const lr_plan& P, int smem, FitParams& fp, cudaStream_t st) {
+    if (P.lanes_per_row == 8) return launch_fit_t<1, 8, 8>(P, smem, fp, st);
+    if (P.lanes_per_row == 16) return launch_fit_t<1, 16, 8>(P, smem, fp, st);
+    if (P.vec_per_lane == 1) return launch_fit_t<1, 32, 8>(P, smem, fp, st);
+    if (P.vec_per_lane == 2) return launch_fit_t<2, 32, LRGD_NV2_RB>(P, smem, fp, st);
+    return launch_fit_t<4, 32, 2>(P, smem, fp, st);
 }
 
 struct Pass {
@@ -344,6 +366,12 @@ int lr_create(lr_ctx** out, int32_t device, int32_t n_max) {
     if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&c->d_oscr), (size_t(n_max) + 2) * sizeof(double));
     if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&c->d_oticket), sizeof(unsigned int));
     if (e == cudaSuccess) e = cudaMemset(c->d_oticket, 0, sizeof(unsigned int));
+    if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&c->d_gbar), sizeof(unsigned int));
+    if (e == cudaSuccess) {
+        int coop = 0;
+        e = cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, device);
+        c->coop = coop != 0;
+    }
     if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&c->hstream, cudaStreamNonBlocking);
     if (prev >= 0) cudaSetDevice(prev);
     if (e != cudaSuccess) {
@@ -355,6 +383,7 @@ int lr_create(lr_ctx** out, int32_t device, int32_t n_max) {
         if (c->d_vel) cudaFree(c->d_vel);
         if (c->d_oscr) cudaFree(c->d_oscr);
         if (c->d_oticket) cudaFree(c->d_oticket);
+        if (c->d_gbar) cudaFree(c->d_gbar);
         delete c;
         return rc != LR_OK ? rc : LR_ERR_CUDA;
     }
@@ -377,6 +406,7 @@ int lr_destroy(lr_ctx* ctx) {
         cudaFree(ctx->d_vel);
         cudaFree(ctx->d_oscr);
         cudaFree(ctx->d_oticket);
+        cudaFree(ctx->d_gbar);
         cudaFree(ctx->d_hX);
         cudaFree(ctx->d_hy);
         cudaFree(ctx->d_hw);
@@ -419,6 +449,23 @@ int lr_fit(lr_ctx* ctx, const float* d_X, const float* d_y, int64_t m, int32_t n
     DeviceGuard g(ctx);
     if (!g.ok) return LR_ERR_CUDA;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    // Narrow rows, several iterations: one cooperative launch runs the whole fit (same bits as the loop below).
+    if (P.variant == 0 && ctx->persistent && ctx->coop && !ctx->prof && iters >= 2 &&
+        2ll * iters * P.grid < (1ll << 32)) {
+        const int64_t stage_stride = (int64_t(P.rows_per_batch) * n * 4 + 127) & ~int64_t(127);
+        const int64_t room = kMaxDynamicSmem - kHeaderBytes - kFitTailBytes;
+        const int depth = int(std::max<int64_t>(1, std::min<int64_t>(P.stages, room / (kNW * stage_stride))));
+        FitParams fp{};
+        fp.X = d_X; fp.y = d_y; fp.m = m; fp.n = n; fp.w = d_w; fp.b = d_b; fp.partial = ctx->d_partial;
+        fp.loss_hist = d_loss_hist; fp.status = ctx->d_status; fp.gbar = ctx->d_gbar; fp.depth = depth;
+        fp.num_batches = (m + P.rows_per_batch - 1) / P.rows_per_batch;
+        fp.iters = iters; fp.lr = double(lr); fp.inv_m = 1.0 / double(m);
+        LR_CK(ctx, cudaMemsetAsync(ctx->d_gbar, 0, sizeof(unsigned int), st));
+        const int smem = int(kHeaderBytes + int64_t(kNW) * depth * stage_stride + kFitTailBytes);
+        LR_CK(ctx, launch_fit(P, smem, fp, st));
+        ctx->launches += 1;
+        return LR_OK;
+    }
     for (int32_t t = 0; t < iters; ++t) {
         rc = launch_stream_pass(ctx, P, Pass{d_X, d_y, m, n, d_w, d_b}, nullptr, 0.f, st);
         if (rc != LR_OK) return rc;
@@ -426,6 +473,12 @@ int lr_fit(lr_ctx* ctx, const float* d_X, const float* d_y, int64_t m, int32_t n
                            d_loss_hist ? d_loss_hist + t : nullptr, nullptr, st);
         if (rc != LR_OK) return rc;
     }
+    return LR_OK;
+}
+
+int lr_set_persistent(lr_ctx* ctx, int32_t on) {
+    if (!ctx) return LR_ERR_NULL;
+    ctx->persistent = on != 0;
     return LR_OK;
 }
 

@@ -1,0 +1,349 @@
+// Persistent whole-fit kernel for rows of up to 512 columns: all `iters` gradient-descent iterations in ONE
+// cooperative launch (one CTA per SM, co-resident), instead of two launches per iteration.
+//
+// Per iteration every CTA runs the same per-warp streaming pass as k_stream_rows (same static batch map, same
+// arithmetic, same summation orders), writes its fp64 partial row, and meets the other CTAs at a grid barrier; the
+// columns of the reduction + update (the arithmetic of k_reduce_update, slice for slice) are then spread over all
+// warps of all CTAs, and a second grid barrier publishes the new parameters.  Results are bit-identical to the two-kernel path.
+//
+// What the single launch buys: no launch gaps, and the HBM stream never drains -- X does not depend on w, so each warp
+// keeps re-arming its stages straight across the iteration boundary (the first batches of iteration t+1 are in flight
+// while the CTAs reduce iteration t).  This matters for short passes (a 400 MB pass lasts ~60 us, of which launch,
+// ramp-up and tail were ~20 %) and most for L2-resident problems.
+//
+// Grid barrier: a monotonic counter in global memory; thread 0 of each CTA adds one and spins (bounded, 2 s) until the
+// counter reaches grid * k.  On expiry, or when another CTA has raised the status word, the CTA stops iterating, waits
+// (bounded) for its own copies in flight and retires with LR_ERR_TIMEOUT in the status word.
+#pragma once
+#include "lrgd_common.cuh"
+#include "lrgd_reduce.cuh"
+#include "lrgd_stream_rows.cuh"
+
+namespace lrgd {
+
+constexpr int kFitCombineCols = 64;            // columns combined per pass through the CTA's combine buffer
+constexpr int kFitTailBytes = 9216;            // combine buffer / reduction slices, after the stages
+
+struct FitParams {
+    const float* X;
+    const float* y;
+    long long m;
+    int n;
+    float* w;                  // [n] in/out
+    float* b;                  // [1] in/out
+    double* partial;           // [grid][n+2]
+    float* loss_hist;          // nullable [iters]
+    int* status;               // device status word
+    unsigned int* gbar;        // grid-barrier counter, zero at launch
+    int depth;
+    long long num_batches;
+    int iters;
+    double lr;
+    double inv_m;
+};
+
+__device__ __forceinline__ unsigned int ld_acquire_u32(const unsigned int* p) {
+    unsigned int v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+
+// All threads of the CTA call this.  Returns false if the barrier gave up (or the CTA had already given up).
+__device__ __forceinline__ bool grid_barrier(unsigned int* counter, unsigned int target, int* status, volatile int* cta_abort) {
+    __syncthreads();
+    if (threadIdx.x == 0 && !*cta_abort) {
+        __threadfence();
+        atomicAdd(counter, 1u);
+        const unsigned long long t0 = global_timer_ns();
+        while (ld_acquire_u32(counter) < target) {
+            if (*reinterpret_cast<volatile int*>(status) != 0 || global_timer_ns() - t0 > kWaitLimitNs) {
+                atomicExch(status, kStatusTimeout);
+                *cta_abort = 1;
+                break;
+            }
+        }
+        __threadfence();
+    }
+    __syncthreads();
+    return *cta_abort == 0;
+}
+
+template <int NV, int LPR, int RB, int NW>
+__global__ void __launch_bounds__(NW * 32, 1) k_fit_rows(const FitParams p) {
+    constexpr int RPW = 32 / LPR;
+    constexpr int RPB = RB * RPW;
+    constexpr int LOG_LPR = Log2<LPR>::value;
+    constexpr int LOG_RB = Log2<RB>::value;
+    constexpr int SHIFT = LOG_LPR - LOG_RB;
+    constexpr unsigned FULL = 0xffffffffu;
+    static_assert(SHIFT >= 0, "rows per batch slot must not exceed lanes per row");
+    static_assert(kRedSlices == 32, "one lane per reduction slice of k_reduce_update");
+    static_assert(NW * kFitCombineCols * 8 + 2 * NW * 8 <= kFitTailBytes, "tail too small");
+
+    extern __shared__ __align__(128) unsigned char smem[];
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + NW * kMaxDepth);
+    unsigned char* data = smem + kHeaderBytes;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int D = p.depth;
+    const int n = p.n, n4 = n >> 2;
+    const int G = gridDim.x;
+    const uint32_t stage_stride = (static_cast<uint32_t>(RPB) * n * 4u + 127u) & ~127u;
+    unsigned char* my_stages = data + static_cast<size_t>(warp) * D * stage_stride;
+    unsigned char* tail = data + static_cast<size_t>(NW) * D * stage_stride;      // combine buffer
+    uint64_t* my_bars = bars + warp * kMaxDepth;
+
+    const long long B = p.num_batches;
+    const long long Bw = B > warp ? (B - warp + NW - 1) / NW : 0;
+    const int cnt = Bw > blockIdx.x ? static_cast<int>((Bw - blockIdx.x + G - 1) / G) : 0;    // batches of this warp per iteration
+    const long long fills_total = static_cast<long long>(cnt) * p.iters;                       // stage fills over the whole fit
+
+    if (threadIdx.x == 0) *abort_flag = 0;
+    if (lane == 0) {
+        for (int d = 0; d < D; ++d) mbar_init(&my_bars[d], 1);
+        fence_mbar_init();
+    }
+    __syncthreads();
+
+    const uint64_t pol = l2_policy_evict_first();
+    const long long stride_rows = static_cast<long long>(G) * NW * RPB;
+    const long long first_row = (static_cast<long long>(blockIdx.x) * NW + warp) * RPB;
+    auto issue = [&](long long r0, int d) {        // lane 0 only
+        const long long left = p.m - r0;
+        const uint32_t rows = left < RPB ? static_cast<uint32_t>(left) : RPB;
+        const uint32_t xbytes = rows * n * 4u;
+        mbar_arrive_expect_tx(&my_bars[d], xbytes);
+        bulk_copy_g2s(my_stages + static_cast<size_t>(d) * stage_stride, p.X + r0 * n, xbytes, &my_bars[d], pol);
+    };
+
+    const int sub = lane & (LPR - 1), slot = lane >> LOG_LPR;
+    const int myr = ((sub >> SHIFT) & (RB - 1)) * RPW + slot;
+    const bool owner = (sub & ((1 << SHIFT) - 1)) == 0;
+    const bool full_cols = n4 == NV * LPR;
+
+    // the fit is one long sequence of fills (iteration-major); fill f lands in stage f % D
+    long long issued = 0;                          // fills whose copy has been issued (warp-uniform)
+    long long consumed = 0;                        // fills whose wait has succeeded
+    int issue_i = 0;                               // batch index (within an iteration) of the next fill to issue
+    {
+        const long long pre = fills_total < D ? fills_total : D;
+        for (long long f = 0; f < pre; ++f) {
+            if (lane == 0) issue(first_row + issue_i * stride_rows, static_cast<int>(f));
+            if (++issue_i == cnt) issue_i = 0;
+        }
+        issued = pre;
+    }
+    int d = 0;
+    uint32_t phase = 0;
+    unsigned int barrier_no = 0;
+    bool alive = true;                             // CTA-uniform after every grid barrier
+
+    for (int t = 0; t < p.iters && alive; ++t) {
+        float4 wv[NV];
+#pragma unroll
+        for (int k = 0; k < NV; ++k) {
+            const int idx = sub + k * LPR;
+            wv[k] = idx < n4 ? make_float4(__ldcg(p.w + 4 * idx), __ldcg(p.w + 4 * idx + 1), __ldcg(p.w + 4 * idx + 2),
+                                           __ldcg(p.w + 4 * idx + 3))
+                             : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+        const float bval = __ldcg(p.b);
+        float4 acc[NV];
+        double dacc[NV][4];
+        float se = 0.f, sl = 0.f;
+        double dse = 0.0, dsl = 0.0;
+#pragma unroll
+        for (int k = 0; k < NV; ++k) {
+            acc[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+            dacc[k][0] = dacc[k][1] = dacc[k][2] = dacc[k][3] = 0.0;
+        }
+        int since_flush = 0;
+        long long row0 = first_row;
+        float y_next = (cnt > 0 && row0 + myr < p.m) ? __ldg(p.y + row0 + myr) : 0.f;
+        bool warp_ok = true;
+
+        for (int i = 0; i < cnt; ++i) {
+            bool ok = mbar_wait_bounded(&my_bars[d], phase, abort_flag);
+            ok = __all_sync(FULL, ok);
+            if (!ok) { warp_ok = false; break; }
+            consumed += 1;
+
+            const long long left = p.m - row0;
+            const int rows = left < RPB ? static_cast<int>(left) : RPB;
+            const float4* t4 = reinterpret_cast<const float4*>(my_stages + static_cast<size_t>(d) * stage_stride);
+            float4 x[RB][NV];
+            if (full_cols && rows == RPB) {
+#pragma unroll
+                for (int r8 = 0; r8 < RB; ++r8)
+#pragma unroll
+                    for (int k2 = 0; k2 < NV; ++k2) x[r8][k2] = t4[(r8 * RPW + slot) * (NV * LPR) + sub + k2 * LPR];
+            } else {
+#pragma unroll
+                for (int r8 = 0; r8 < RB; ++r8) {
+                    const int r = r8 * RPW + slot;
+#pragma unroll
+                    for (int k2 = 0; k2 < NV; ++k2) {
+                        const int idx = sub + k2 * LPR;
+                        x[r8][k2] = (r < rows && idx < n4) ? t4[r * n4 + idx] : make_float4(0.f, 0.f, 0.f, 0.f);
+                    }
+                }
+            }
+            const bool myvalid = myr < rows;
+            const float yv = y_next;
+            {
+                const long long rn = row0 + stride_rows + myr;
+                y_next = (i + 1 < cnt && rn < p.m) ? __ldg(p.y + rn) : 0.f;
+            }
+            // re-arm the stage with the fill `depth` ahead in the fit-long sequence (possibly of the next iteration)
+            __syncwarp();
+            if (issued < fills_total) {
+                if (lane == 0) {
+                    fence_proxy_async_smem();
+                    issue(first_row + issue_i * stride_rows, d);
+                }
+                if (++issue_i == cnt) issue_i = 0;
+                issued += 1;
+            }
+            if (++d == D) { d = 0; phase ^= 1u; }
+
+            float v[RB];
+#pragma unroll
+            for (int r8 = 0; r8 < RB; ++r8) {
+                float dot = 0.f;
+#pragma unroll
+                for (int k2 = 0; k2 < NV; ++k2) {
+                    dot = fmaf(x[r8][k2].x, wv[k2].x, dot);
+                    dot = fmaf(x[r8][k2].y, wv[k2].y, dot);
+                    dot = fmaf(x[r8][k2].z, wv[k2].z, dot);
+                    dot = fmaf(x[r8][k2].w, wv[k2].w, dot);
+                }
+                v[r8] = dot;
+            }
+            lane_reduce<RB, LPR / 2, RB>(v, lane);
+            const float z = v[0] + bval;
+            float e, L;
+            logistic_terms(z, yv, e, L);
+            if (!myvalid) { e = 0.f; L = 0.f; }
+            if (owner) { se += e; sl += L; }
+#pragma unroll
+            for (int r8 = 0; r8 < RB; ++r8) {
+                const float ei = __shfl_sync(FULL, e, r8 << SHIFT, LPR);
+#pragma unroll
+                for (int k2 = 0; k2 < NV; ++k2) {
+                    acc[k2].x = fmaf(x[r8][k2].x, ei, acc[k2].x);
+                    acc[k2].y = fmaf(x[r8][k2].y, ei, acc[k2].y);
+                    acc[k2].z = fmaf(x[r8][k2].z, ei, acc[k2].z);
+                    acc[k2].w = fmaf(x[r8][k2].w, ei, acc[k2].w);
+                }
+            }
+            if (++since_flush == kFlushBatches) {
+                since_flush = 0;
+#pragma unroll
+                for (int k2 = 0; k2 < NV; ++k2) {
+                    dacc[k2][0] += acc[k2].x; dacc[k2][1] += acc[k2].y;
+                    dacc[k2][2] += acc[k2].z; dacc[k2][3] += acc[k2].w;
+                    acc[k2] = make_float4(0.f, 0.f, 0.f, 0.f);
+                }
+                dse += se; dsl += sl; se = 0.f; sl = 0.f;
+            }
+            row0 += stride_rows;
+        }
+        (void)warp_ok;                             // a failed wait has raised the CTA's abort flag; handled at the barrier
+
+#pragma unroll
+        for (int k2 = 0; k2 < NV; ++k2) {
+            dacc[k2][0] += acc[k2].x; dacc[k2][1] += acc[k2].y;
+            dacc[k2][2] += acc[k2].z; dacc[k2][3] += acc[k2].w;
+        }
+        dse += se; dsl += sl;
+
+        // ---- fixed-order combine of the CTA's warps, kFitCombineCols columns at a time (the stages stay in use) ----
+        // row slots of one warp that own the same columns: add in slot order (as k_stream_rows does)
+#pragma unroll
+        for (int k2 = 0; k2 < NV; ++k2)
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                double tsum = 0.0;
+#pragma unroll
+                for (int sidx = 0; sidx < RPW; ++sidx) tsum += __shfl_sync(FULL, dacc[k2][c], sub + sidx * LPR);
+                dacc[k2][c] = tsum;
+            }
+#pragma unroll
+        for (int msk = 16; msk >= 1; msk >>= 1) {
+            dse += __shfl_xor_sync(FULL, dse, msk);
+            dsl += __shfl_xor_sync(FULL, dsl, msk);
+        }
+        double* red = reinterpret_cast<double*>(tail);                 // [NW][kFitCombineCols]
+        double* red_e = red + NW * kFitCombineCols;
+        double* red_l = red_e + NW;
+        double* out = p.partial + static_cast<size_t>(blockIdx.x) * (n + 2);
+        __syncthreads();                                               // previous use of the tail is over
+        if (lane == 0) { red_e[warp] = dse; red_l[warp] = dsl; }
+        for (int c0 = 0; c0 < n; c0 += kFitCombineCols) {
+#pragma unroll
+            for (int k2 = 0; k2 < NV; ++k2) {
+                const int idx = sub + k2 * LPR;
+                const int col = idx * 4 - c0;
+                if (slot == 0 && idx < n4 && col >= 0 && col < kFitCombineCols) {
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) red[warp * kFitCombineCols + col + c] = dacc[k2][c];
+                }
+            }
+            __syncthreads();
+            if (threadIdx.x < kFitCombineCols && c0 + threadIdx.x < n) {
+                double tsum = 0.0;
+                for (int wi = 0; wi < NW; ++wi) tsum += red[wi * kFitCombineCols + threadIdx.x];
+                out[c0 + threadIdx.x] = tsum;
+            }
+            __syncthreads();
+        }
+        if (threadIdx.x < 2) {
+            const double* src = threadIdx.x == 0 ? red_e : red_l;
+            double tsum = 0.0;
+            for (int wi = 0; wi < NW; ++wi) tsum += src[wi];
+            out[n + threadIdx.x] = tsum;
+        }
+
+        barrier_no += 1;
+        alive = grid_barrier(p.gbar, static_cast<unsigned int>(G) * barrier_no, p.status, abort_flag);
+        if (!alive) break;
+
+        // ---- reduction + update: one warp per column, columns spread over all warps of all CTAs.  Lane s plays slice s of
+        // k_reduce_update (rows [s*per, (s+1)*per) in index order); lane 0 then adds the 32 slice sums in slice order ----
+        {
+            const int stride = n + 2;
+            const int per = (G + kRedSlices - 1) / kRedSlices;
+            const int g0 = lane * per;
+            const int g1 = g0 + per < G ? g0 + per : G;
+            for (int col = warp * G + blockIdx.x; col < stride; col += NW * G) {
+                double s = 0.0;
+                const double* src = p.partial + col;
+                for (int g = g0; g < g1; ++g) s += __ldcg(src + static_cast<size_t>(g) * stride);
+                double tsum = 0.0;
+#pragma unroll
+                for (int k = 0; k < kRedSlices; ++k) tsum += __shfl_sync(FULL, s, k);
+                if (lane == 0) {
+                    const double v = tsum * p.inv_m;
+                    if (col < n) p.w[col] = static_cast<float>(static_cast<double>(__ldcg(p.w + col)) - p.lr * v);
+                    else if (col == n) p.b[0] = static_cast<float>(static_cast<double>(__ldcg(p.b)) - p.lr * v);
+                    else if (p.loss_hist) p.loss_hist[t] = static_cast<float>(v);
+                }
+            }
+        }
+        barrier_no += 1;
+        alive = grid_barrier(p.gbar, static_cast<unsigned int>(G) * barrier_no, p.status, abort_flag);
+    }
+
+    if (!alive || *abort_flag) {
+        // gave up: let this warp's copies still in flight land (bounded) before the CTA retires
+        if (lane == 0) {
+            atomicExch(p.status, kStatusTimeout);
+            for (long long f = consumed; f < issued; ++f)
+                mbar_wait_bounded(&my_bars[f % D], static_cast<uint32_t>(f / D) & 1u, abort_flag);
+        }
+        __syncwarp();
+    }
+}
+
+}  // namespace lrgd

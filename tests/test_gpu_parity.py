@@ -210,6 +210,28 @@ def test_argument_errors_with_a_live_context(ctx):
     assert ctx.launch_count() == n0 + 2
 
 
+@pytest.mark.parametrize("name,m,iters", [("cfg1", 10_000, 25), ("cfg2", 150_007, 12), ("cfg3", 120_001, 9), ("cfg5", 300_000, 7),
+                                           ("higgs_like", 200_003, 11), ("cfg1", 37, 5), ("cfg3", 9, 3)])
+def test_single_launch_fit_equals_two_kernel_fit(ctx, name, m, iters):
+    # lr_fit runs narrow-row problems as one persistent cooperative launch; forcing the two-kernels-per-iteration form
+    # must give the same bits (same batch map, same summation orders), including the loss history
+    wl = datagen.scaled(datagen.WORKLOADS[name], m)
+    X, y, _, _ = datagen.generate(wl)
+    dX, dy = dev(X), dev(y)
+    n0 = ctx.launch_count()
+    w1, b1, h1 = api.lr_fit(dX, dy, wl.lr, iters, return_history=True, ctx=ctx)
+    assert ctx.launch_count() == n0 + 1                       # one launch for the whole fit
+    ctx.set_persistent(False)
+    try:
+        n0 = ctx.launch_count()
+        w2, b2, h2 = api.lr_fit(dX, dy, wl.lr, iters, return_history=True, ctx=ctx)
+        assert ctx.launch_count() == n0 + 2 * iters
+    finally:
+        ctx.set_persistent(True)
+    assert torch.equal(w1, w2) and torch.equal(b1, b2) and torch.equal(h1, h2)
+    assert ctx.device_status() == 0
+
+
 def test_row_sharded_entry_points_match_oracle(ctx):
     # three row shards on one GPU, one after the other (no kernel waits on another): lr_shard_sums per shard,
     # lr_apply_sums over the stacked sums, for several steps; against the checker's unsharded fit
