@@ -36,7 +36,8 @@ UNIT = "iterations/s"
 NOMINAL_HBM_GBS = 8000.0
 # dram__bytes_read.sum + dram__bytes_write.sum of the streaming kernel per row of X, from the ncu capture summarised in
 # profiles/ (taken at m = 500,000 and scaled by rows).  Remove an entry when its kernel changes.
-NCU_TRAFFIC_BYTES_PER_ROW = {"cfg3": (514.024192e6 + 3.515648e6) / 500_000}
+NCU_TRAFFIC_BYTES_PER_ROW = {"cfg3": {"k_stream_rows": (514.024192e6 + 3.515648e6) / 500_000,
+                                      "k_fit_rows": (1.538055e9 + 3.601664e6) / 3 / 500_000}}
 FALLBACK_HBM_GBS = 6650.0
 
 
@@ -326,20 +327,22 @@ def main():
     peak, peak_kind = measured_hbm_peak()
     plan = api.plan_query(wl.m, wl.n, sm_count=torch.cuda.get_device_properties(local_rank).multi_processor_count)
     pass_kernel = {0: "k_stream_rows", 1: "k_stream_split", 2: "k_generic"}[plan["variant"]]
-    traffic = NCU_TRAFFIC_BYTES_PER_ROW[args.workload] * wl.m if args.workload in NCU_TRAFFIC_BYTES_PER_ROW else None
+    per_row = NCU_TRAFFIC_BYTES_PER_ROW.get(args.workload, {})
     single_pass = {"kernel": f"{pass_kernel} (one fused loss/gradient pass, two-kernel form of lr_fit)", "achieved": achieved,
                    "unit": "GB/s", "frac": achieved / peak, "bytes_per_launch": bytes_per_launch, "avg_launch_ms": k1_ms,
-                   "launches_timed": n_l, "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS}
+                   "launches_timed": n_l, "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
+                   "traffic": per_row[pass_kernel] * wl.m if pass_kernel in per_row else None}
     if world == 1 and launches == 1:
         # the timed region was ONE launch of the persistent kernel doing all K iterations (pass + reduction + update)
         ach = bytes_per_launch * args.steps / (ms * 1e-3) / 1e9
         roofline = {"bound": "hbm", "kernel": "k_fit_rows (persistent: all timed iterations in one cooperative launch)",
                     "achieved": ach, "peak": peak, "unit": "GB/s", "frac": ach / peak, "peak_kind": f"of {peak_kind}",
-                    "traffic": traffic * args.steps if traffic else None, "bytes_per_launch": bytes_per_launch * args.steps,
+                    "traffic": per_row["k_fit_rows"] * wl.m * args.steps if "k_fit_rows" in per_row else None,
+                    "bytes_per_launch": bytes_per_launch * args.steps,
                     "avg_launch_ms": ms, "launches_timed": 1, "iterations_per_launch": args.steps,
                     "frac_of_nominal_8TBs": ach / NOMINAL_HBM_GBS, "single_pass": single_pass}
     else:
-        roofline = dict(single_pass, bound="hbm", peak=peak, peak_kind=f"of {peak_kind}", traffic=traffic)
+        roofline = dict(single_pass, bound="hbm", peak=peak, peak_kind=f"of {peak_kind}")
 
     # ---- end to end through the host-pointer entry point ----
     e2e = None
