@@ -28,6 +28,9 @@ constexpr int kMaxGridPerSm = 8;               // widest launch any variant uses
 constexpr int kMaxProfiled = 4096;
 constexpr int kMaxDynamicSmem = 232448;         // opt-in dynamic shared memory per CTA on sm_100
 constexpr int64_t kMaxRows = int64_t(1) << 40;
+#ifndef LRGD_NV1_RB
+#define LRGD_NV1_RB 8                          // register batch of the 68..128-column instantiation
+#endif
 #ifndef LRGD_NV2_RB
 #define LRGD_NV2_RB 4                          // register batch (rows per warp) of the 132..256-column instantiation
 #endif
@@ -38,7 +41,7 @@ struct RowShape { int nv, lpr, rb; };
 bool row_shape_for(int n4, RowShape* s) {
     if (n4 <= 8) *s = {1, 8, 8};
     else if (n4 <= 16) *s = {1, 16, 8};
-    else if (n4 <= 32) *s = {1, 32, 8};
+    else if (n4 <= 32) *s = {1, 32, LRGD_NV1_RB};
     else if (n4 <= 64) *s = {2, 32, LRGD_NV2_RB};
     else if (n4 <= 128) *s = {4, 32, 2};
     else return false;
@@ -178,7 +181,7 @@ template <bool PRED>
 cudaError_t launch_rows(const lr_plan& P, const StreamParams& sp, cudaStream_t st) {
     if (P.lanes_per_row == 8) return launch_rows_t<1, 8, 8, PRED>(P, sp, st);
     if (P.lanes_per_row == 16) return launch_rows_t<1, 16, 8, PRED>(P, sp, st);
-    if (P.vec_per_lane == 1) return launch_rows_t<1, 32, 8, PRED>(P, sp, st);
+    if (P.vec_per_lane == 1) return launch_rows_t<1, 32, LRGD_NV1_RB, PRED>(P, sp, st);
     if (P.vec_per_lane == 2) return launch_rows_t<2, 32, LRGD_NV2_RB, PRED>(P, sp, st);
     return launch_rows_t<4, 32, 2, PRED>(P, sp, st);
 }
@@ -239,7 +242,7 @@ cudaError_t launch_fit_t(const lr_plan& P, int smem, FitParams& fp, cudaStream_t
 cudaError_t launch_fit(const lr_plan& P, int smem, FitParams& fp, cudaStream_t st) {
     if (P.lanes_per_row == 8) return launch_fit_t<1, 8, 8>(P, smem, fp, st);
     if (P.lanes_per_row == 16) return launch_fit_t<1, 16, 8>(P, smem, fp, st);
-    if (P.vec_per_lane == 1) return launch_fit_t<1, 32, 8>(P, smem, fp, st);
+    if (P.vec_per_lane == 1) return launch_fit_t<1, 32, LRGD_NV1_RB>(P, smem, fp, st);
     if (P.vec_per_lane == 2) return launch_fit_t<2, 32, LRGD_NV2_RB>(P, smem, fp, st);
     return launch_fit_t<4, 32, 2>(P, smem, fp, st);
 }
