@@ -173,22 +173,7 @@ __global__ void __launch_bounds__(NW * 32, 1) k_fit_rows(const FitParams p) {
             const int rows = left < RPB ? static_cast<int>(left) : RPB;
             const float4* t4 = reinterpret_cast<const float4*>(my_stages + static_cast<size_t>(d) * stage_stride);
             float4 x[RB][NV];
-            if (full_cols && rows == RPB) {
-#pragma unroll
-                for (int r8 = 0; r8 < RB; ++r8)
-#pragma unroll
-                    for (int k2 = 0; k2 < NV; ++k2) x[r8][k2] = t4[(r8 * RPW + slot) * (NV * LPR) + sub + k2 * LPR];
-            } else {
-#pragma unroll
-                for (int r8 = 0; r8 < RB; ++r8) {
-                    const int r = r8 * RPW + slot;
-#pragma unroll
-                    for (int k2 = 0; k2 < NV; ++k2) {
-                        const int idx = sub + k2 * LPR;
-                        x[r8][k2] = (r < rows && idx < n4) ? t4[r * n4 + idx] : make_float4(0.f, 0.f, 0.f, 0.f);
-                    }
-                }
-            }
+            load_row_batch<NV, LPR, RB>(x, t4, rows, n4, full_cols && rows == RPB, sub, slot);
             const bool myvalid = myr < rows;
             const float yv = y_next;
             {
@@ -207,56 +192,21 @@ __global__ void __launch_bounds__(NW * 32, 1) k_fit_rows(const FitParams p) {
             }
             if (++d == D) { d = 0; phase ^= 1u; }
 
-            float v[RB];
-#pragma unroll
-            for (int r8 = 0; r8 < RB; ++r8) {
-                float dot = 0.f;
-#pragma unroll
-                for (int k2 = 0; k2 < NV; ++k2) {
-                    dot = fmaf(x[r8][k2].x, wv[k2].x, dot);
-                    dot = fmaf(x[r8][k2].y, wv[k2].y, dot);
-                    dot = fmaf(x[r8][k2].z, wv[k2].z, dot);
-                    dot = fmaf(x[r8][k2].w, wv[k2].w, dot);
-                }
-                v[r8] = dot;
-            }
-            lane_reduce<RB, LPR / 2, RB>(v, lane);
-            const float z = v[0] + bval;
+            const float z = batch_dot<NV, LPR, RB>(x, wv, lane) + bval;
             float e, L;
             logistic_terms(z, yv, e, L);
             if (!myvalid) { e = 0.f; L = 0.f; }
             if (owner) { se += e; sl += L; }
-#pragma unroll
-            for (int r8 = 0; r8 < RB; ++r8) {
-                const float ei = __shfl_sync(FULL, e, r8 << SHIFT, LPR);
-#pragma unroll
-                for (int k2 = 0; k2 < NV; ++k2) {
-                    acc[k2].x = fmaf(x[r8][k2].x, ei, acc[k2].x);
-                    acc[k2].y = fmaf(x[r8][k2].y, ei, acc[k2].y);
-                    acc[k2].z = fmaf(x[r8][k2].z, ei, acc[k2].z);
-                    acc[k2].w = fmaf(x[r8][k2].w, ei, acc[k2].w);
-                }
-            }
+            batch_accumulate<NV, LPR, RB>(x, e, acc);
             if (++since_flush == kFlushBatches) {
                 since_flush = 0;
-#pragma unroll
-                for (int k2 = 0; k2 < NV; ++k2) {
-                    dacc[k2][0] += acc[k2].x; dacc[k2][1] += acc[k2].y;
-                    dacc[k2][2] += acc[k2].z; dacc[k2][3] += acc[k2].w;
-                    acc[k2] = make_float4(0.f, 0.f, 0.f, 0.f);
-                }
-                dse += se; dsl += sl; se = 0.f; sl = 0.f;
+                fold_into_fp64<NV>(acc, dacc, se, sl, dse, dsl);
             }
             row0 += stride_rows;
         }
         (void)warp_ok;                             // a failed wait has raised the CTA's abort flag; handled at the barrier
 
-#pragma unroll
-        for (int k2 = 0; k2 < NV; ++k2) {
-            dacc[k2][0] += acc[k2].x; dacc[k2][1] += acc[k2].y;
-            dacc[k2][2] += acc[k2].z; dacc[k2][3] += acc[k2].w;
-        }
-        dse += se; dsl += sl;
+        fold_into_fp64<NV>(acc, dacc, se, sl, dse, dsl);
 
         // ---- fixed-order combine of the CTA's warps, kFitCombineCols columns at a time (the stages stay in use) ----
         // row slots of one warp that own the same columns: add in slot order (as k_stream_rows does)

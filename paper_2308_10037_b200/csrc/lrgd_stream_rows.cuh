@@ -67,6 +67,84 @@ __device__ __forceinline__ void lane_reduce(float (&v)[RB], int lane) {
     }
 }
 
+// ---- pieces of the per-batch work shared by the narrow-row, wide-row and persistent kernels ----
+// A batch lives in registers as x[RB][NV]: RB row slots by NV 16-byte column groups per lane; LPR lanes share a row.
+
+// z partials: lane-local FMAs, then the transposing reduction; the returned value is the full dot product of the row
+// (r, with r = (lane_in_group >> (log2 LPR - log2 RB)) & (RB-1)) that ends up on this lane.
+template <int NV, int LPR, int RB>
+__device__ __forceinline__ float batch_dot(const float4 (&x)[RB][NV], const float4 (&wv)[NV], int lane) {
+    float v[RB];
+#pragma unroll
+    for (int r = 0; r < RB; ++r) {
+        float dot = 0.f;
+#pragma unroll
+        for (int k = 0; k < NV; ++k) {
+            dot = fmaf(x[r][k].x, wv[k].x, dot);
+            dot = fmaf(x[r][k].y, wv[k].y, dot);
+            dot = fmaf(x[r][k].z, wv[k].z, dot);
+            dot = fmaf(x[r][k].w, wv[k].w, dot);
+        }
+        v[r] = dot;
+    }
+    lane_reduce<RB, LPR / 2, RB>(v, lane);
+    return v[0];
+}
+
+// acc[c] += x[r][c] * err[r]: each row's err is fetched from the lane that holds it (Algorithm 1's err.X on registers).
+template <int NV, int LPR, int RB>
+__device__ __forceinline__ void batch_accumulate(const float4 (&x)[RB][NV], float e, float4 (&acc)[NV]) {
+    constexpr int SHIFT = Log2<LPR>::value - Log2<RB>::value;
+#pragma unroll
+    for (int r = 0; r < RB; ++r) {
+        const float er = __shfl_sync(0xffffffffu, e, r << SHIFT, LPR);
+#pragma unroll
+        for (int k = 0; k < NV; ++k) {
+            acc[k].x = fmaf(x[r][k].x, er, acc[k].x);
+            acc[k].y = fmaf(x[r][k].y, er, acc[k].y);
+            acc[k].z = fmaf(x[r][k].z, er, acc[k].z);
+            acc[k].w = fmaf(x[r][k].w, er, acc[k].w);
+        }
+    }
+}
+
+// fp32 per-lane sums folded into their fp64 counterparts (keeps the serial fp32 chains short)
+template <int NV>
+__device__ __forceinline__ void fold_into_fp64(float4 (&acc)[NV], double (&dacc)[NV][4], float& se, float& sl, double& dse,
+                                               double& dsl) {
+#pragma unroll
+    for (int k = 0; k < NV; ++k) {
+        dacc[k][0] += acc[k].x; dacc[k][1] += acc[k].y;
+        dacc[k][2] += acc[k].z; dacc[k][3] += acc[k].w;
+        acc[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+    dse += se; dsl += sl; se = 0.f; sl = 0.f;
+}
+
+// one batch from a narrow-row stage into registers (rows packed at n4 groups; lanes beyond the row or rows beyond the
+// matrix read zeros); `full` = every lane's groups exist and the batch is complete: no bounds logic
+template <int NV, int LPR, int RB>
+__device__ __forceinline__ void load_row_batch(float4 (&x)[RB][NV], const float4* t4, int rows, int n4, bool full, int sub,
+                                               int slot) {
+    constexpr int RPW = 32 / LPR;
+    if (full) {
+#pragma unroll
+        for (int r8 = 0; r8 < RB; ++r8)
+#pragma unroll
+            for (int k2 = 0; k2 < NV; ++k2) x[r8][k2] = t4[(r8 * RPW + slot) * (NV * LPR) + sub + k2 * LPR];
+    } else {
+#pragma unroll
+        for (int r8 = 0; r8 < RB; ++r8) {
+            const int r = r8 * RPW + slot;
+#pragma unroll
+            for (int k2 = 0; k2 < NV; ++k2) {
+                const int idx = sub + k2 * LPR;
+                x[r8][k2] = (r < rows && idx < n4) ? t4[r * n4 + idx] : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+        }
+    }
+}
+
 template <int NV, int LPR, int RB, int NW, bool PREDICT>
 __global__ void __launch_bounds__(NW * 32, 1) k_stream_rows(const StreamParams p) {
     constexpr int RPW = 32 / LPR;                  // rows a warp touches with one load instruction
@@ -163,22 +241,7 @@ __global__ void __launch_bounds__(NW * 32, 1) k_stream_rows(const StreamParams p
         const int rows = left < RPB ? static_cast<int>(left) : RPB;
         const float4* t4 = reinterpret_cast<const float4*>(my_stages + static_cast<size_t>(d) * stage_stride);
         float4 x[RB][NV];
-        if (full_cols && rows == RPB) {
-#pragma unroll
-            for (int r8 = 0; r8 < RB; ++r8)
-#pragma unroll
-                for (int k2 = 0; k2 < NV; ++k2) x[r8][k2] = t4[(r8 * RPW + slot) * (NV * LPR) + sub + k2 * LPR];
-        } else {
-#pragma unroll
-            for (int r8 = 0; r8 < RB; ++r8) {
-                const int r = r8 * RPW + slot;
-#pragma unroll
-                for (int k2 = 0; k2 < NV; ++k2) {
-                    const int idx = sub + k2 * LPR;
-                    x[r8][k2] = (r < rows && idx < n4) ? t4[r * n4 + idx] : make_float4(0.f, 0.f, 0.f, 0.f);
-                }
-            }
-        }
+        load_row_batch<NV, LPR, RB>(x, t4, rows, n4, full_cols && rows == RPB, sub, slot);
         const bool myvalid = myr < rows;
         const float yv = y_next;
         if constexpr (!PREDICT) {
@@ -196,21 +259,7 @@ __global__ void __launch_bounds__(NW * 32, 1) k_stream_rows(const StreamParams p
         }
         if (++d == D) { d = 0; phase ^= 1u; }
 
-        float v[RB];
-#pragma unroll
-        for (int r8 = 0; r8 < RB; ++r8) {
-            float dot = 0.f;
-#pragma unroll
-            for (int k2 = 0; k2 < NV; ++k2) {
-                dot = fmaf(x[r8][k2].x, wv[k2].x, dot);
-                dot = fmaf(x[r8][k2].y, wv[k2].y, dot);
-                dot = fmaf(x[r8][k2].z, wv[k2].z, dot);
-                dot = fmaf(x[r8][k2].w, wv[k2].w, dot);
-            }
-            v[r8] = dot;
-        }
-        lane_reduce<RB, LPR / 2, RB>(v, lane);
-        const float z = v[0] + bval;
+        const float z = batch_dot<NV, LPR, RB>(x, wv, lane) + bval;
 
         if constexpr (PREDICT) {
             if (owner && myvalid) p.labels[row0 + myr] = z >= p.cut ? 1 : 0;
@@ -219,26 +268,10 @@ __global__ void __launch_bounds__(NW * 32, 1) k_stream_rows(const StreamParams p
             logistic_terms(z, yv, e, L);
             if (!myvalid) { e = 0.f; L = 0.f; }
             if (owner) { se += e; sl += L; }
-#pragma unroll
-            for (int r8 = 0; r8 < RB; ++r8) {
-                const float ei = __shfl_sync(FULL, e, r8 << SHIFT, LPR);
-#pragma unroll
-                for (int k2 = 0; k2 < NV; ++k2) {
-                    acc[k2].x = fmaf(x[r8][k2].x, ei, acc[k2].x);
-                    acc[k2].y = fmaf(x[r8][k2].y, ei, acc[k2].y);
-                    acc[k2].z = fmaf(x[r8][k2].z, ei, acc[k2].z);
-                    acc[k2].w = fmaf(x[r8][k2].w, ei, acc[k2].w);
-                }
-            }
+            batch_accumulate<NV, LPR, RB>(x, e, acc);
             if (++since_flush == kFlushBatches) {
                 since_flush = 0;
-#pragma unroll
-                for (int k2 = 0; k2 < NV; ++k2) {
-                    dacc[k2][0] += acc[k2].x; dacc[k2][1] += acc[k2].y;
-                    dacc[k2][2] += acc[k2].z; dacc[k2][3] += acc[k2].w;
-                    acc[k2] = make_float4(0.f, 0.f, 0.f, 0.f);
-                }
-                dse += se; dsl += sl; se = 0.f; sl = 0.f;
+                fold_into_fp64<NV>(acc, dacc, se, sl, dse, dsl);
             }
         }
         row0 += stride_rows;
@@ -254,13 +287,7 @@ __global__ void __launch_bounds__(NW * 32, 1) k_stream_rows(const StreamParams p
         __syncwarp();
     }
     if constexpr (!PREDICT) {
-
-#pragma unroll
-        for (int k2 = 0; k2 < NV; ++k2) {
-            dacc[k2][0] += acc[k2].x; dacc[k2][1] += acc[k2].y;
-            dacc[k2][2] += acc[k2].z; dacc[k2][3] += acc[k2].w;
-        }
-        dse += se; dsl += sl;
+        fold_into_fp64<NV>(acc, dacc, se, sl, dse, dsl);
 
         // ---------------- fixed-order combine of the CTA's warps ----------------
         __syncthreads();                               // all stages are idle: reuse them as the combine buffer

@@ -177,22 +177,9 @@ __global__ void __launch_bounds__(NW * 32, 1) k_stream_split(const __grid_consta
                 for (int k = 0; k < NV; ++k) x[r][k] = make_float4(0.f, 0.f, 0.f, 0.f);
         }
 
-        float v[RB];
-#pragma unroll
-        for (int r = 0; r < RB; ++r) {
-            float dot = 0.f;
-#pragma unroll
-            for (int k = 0; k < NV; ++k) {
-                dot = fmaf(x[r][k].x, wv[k].x, dot);
-                dot = fmaf(x[r][k].y, wv[k].y, dot);
-                dot = fmaf(x[r][k].z, wv[k].z, dot);
-                dot = fmaf(x[r][k].w, wv[k].w, dot);
-            }
-            v[r] = dot;
-        }
-        lane_reduce<RB, 16, RB>(v, lane);
+        const float zpartial = batch_dot<NV, 32, RB>(x, wv, lane);
         float* zp = zpart + (i & 1) * (NW * RB);
-        if (owner) zp[warp * RB + myr] = v[0];
+        if (owner) zp[warp * RB + myr] = zpartial;
         __syncthreads();
         // the lanes that share a row add PER_DUP partials each (warp order), then a butterfly: one fixed order, same in every warp
         float zs = 0.f;
@@ -214,26 +201,10 @@ __global__ void __launch_bounds__(NW * 32, 1) k_stream_split(const __grid_consta
                 e = logistic_err(z, yv);
             }
             if (!myvalid) e = 0.f;
-#pragma unroll
-            for (int r = 0; r < RB; ++r) {
-                const float er = __shfl_sync(FULL, e, r << SHIFT);
-#pragma unroll
-                for (int k = 0; k < NV; ++k) {
-                    acc[k].x = fmaf(x[r][k].x, er, acc[k].x);
-                    acc[k].y = fmaf(x[r][k].y, er, acc[k].y);
-                    acc[k].z = fmaf(x[r][k].z, er, acc[k].z);
-                    acc[k].w = fmaf(x[r][k].w, er, acc[k].w);
-                }
-            }
+            batch_accumulate<NV, 32, RB>(x, e, acc);
             if (++since_flush == 2 * kFlushBatches) {
                 since_flush = 0;
-#pragma unroll
-                for (int k = 0; k < NV; ++k) {
-                    dacc[k][0] += acc[k].x; dacc[k][1] += acc[k].y;
-                    dacc[k][2] += acc[k].z; dacc[k][3] += acc[k].w;
-                    acc[k] = make_float4(0.f, 0.f, 0.f, 0.f);
-                }
-                dse += se; dsl += sl; se = 0.f; sl = 0.f;
+                fold_into_fp64<NV>(acc, dacc, se, sl, dse, dsl);
             }
         }
         row0 += stride_rows;
