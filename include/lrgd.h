@@ -143,6 +143,18 @@ int lr_fit_opt(lr_ctx* ctx, const float* d_X, const float* d_y, int64_t m, int32
                float* d_w, float* d_b, float* d_velocity, float* d_loss_hist, void* stream);
 
 /*
+ * Mini-batch gradient descent over contiguous row blocks (one of the "other optimisers" the paper leaves to future
+ * work, Section V; deterministic: no shuffling).  The rows are cut into ceil(m / batch_rows) blocks of batch_rows rows
+ * (the last one may be shorter); step s uses block (first_batch + s) mod that count, forms loss and gradient over that
+ * block alone (scaled by 1 / rows in the block) and applies  w <- w - lr*grad_w, b <- b - lr*grad_b.
+ * batch_rows == m is lr_fit.  d_loss_hist (NULL or [steps]) receives the block's loss before each update.
+ * Errors as lr_fit, plus LR_ERR_SHAPE for batch_rows outside [1, m] or first_batch < 0.
+ */
+int lr_fit_sgd(lr_ctx* ctx, const float* d_X, const float* d_y, int64_t m, int32_t n,
+               float lr, int64_t batch_rows, int32_t steps, int64_t first_batch,
+               float* d_w, float* d_b, float* d_loss_hist, void* stream);
+
+/*
  * d_labels[i] = 1 if sigmoid(x_i.w + b) >= thr else 0, decided in logit space as
  * z_i >= log(thr/(1-thr)) evaluated in fp32 (the paper reports f1 but states no threshold; the
  * caller supplies it).  0 < thr < 1.  d_labels is uint8 [m].

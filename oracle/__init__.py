@@ -39,6 +39,7 @@ def _load():
         lib.oracle_fit.argtypes = [P, P, I64, I32, D, I32, P, P, P, P, P, ctypes.c_int]
         lib.oracle_predict.argtypes = [P, I64, I32, P, D, D, P, P]
         lib.oracle_fit_opt.argtypes = [P, P, I64, I32, D, I32, D, D, ctypes.c_int, P, P, P, P]
+        lib.oracle_fit_sgd.argtypes = [P, P, I64, I32, D, I64, I32, I64, P, P, P]
         lib.oracle_fit_tol.argtypes = [P, P, I64, I32, D, D, I32, P, P, P, P, P, P]
         lib.oracle_f1.argtypes = [P, P, I64, P, P, P, P]
         _lib = lib
@@ -139,6 +140,21 @@ def fit_opt(X, y, lr, iters, l2=0.0, momentum=0.0, nesterov=False, w0=None, b0=0
     if rc != 0:
         raise ValueError("oracle_fit_opt: bad arguments")
     return w, float(b[0]), vel, lh[:iters]
+
+
+def fit_sgd(X, y, lr, batch_rows, steps, first_batch=0, w0=None, b0=0.0):
+    """Mini-batch GD over contiguous row blocks (no shuffling).  Returns ``(w, b, loss_hist)``."""
+    X = _f32(X)
+    m, n = X.shape
+    y = _f32(y, (m,))
+    w = np.zeros(n) if w0 is None else np.array(w0, dtype=np.float64).copy()
+    b = np.array([float(b0)])
+    lh = np.zeros(max(steps, 1))
+    rc = _load().oracle_fit_sgd(_ptr(X), _ptr(y), m, n, float(lr), int(batch_rows), int(steps), int(first_batch), _ptr(w),
+                                _ptr(b), _ptr(lh))
+    if rc != 0:
+        raise ValueError("oracle_fit_sgd: bad arguments")
+    return w, float(b[0]), lh[:steps]
 
 
 def predict(X, w, b, thr, return_z=False):

@@ -35,7 +35,7 @@
  * library BCE-with-logits, brute-force predict and hand-counted F1; the stopping rule against the fixed-count
  * trajectory and its recorded norms; the penalty/momentum update against three steps done by hand from
  * oracle_loss_grad, central differences of the penalised loss and the vanishing penalised gradient at its fixed
- * point.  No function here is unpinned.
+ * point; mini-batch descent against five steps done by hand on row slices.  No function here is unpinned.
  */
 #include <math.h>
 #include <stdint.h>
@@ -202,6 +202,31 @@ int oracle_fit_opt(const float* X, const float* y, int64_t m, int32_t n, double 
             vel[j] = v;
             if (j < n) w[j] -= lr * step; else *b -= lr * step;
         }
+    }
+    free(g);
+    return 0;
+}
+
+/*
+ * Mini-batch gradient descent over contiguous row blocks, no shuffling (an "other optimiser" in the sense of the paper's
+ * Section V, defined here): the rows are cut into ceil(m/batch_rows) blocks; step s uses block (first_batch + s) mod that
+ * count, takes loss and gradient over that block alone (mean over its rows) and applies the Algorithm 1 update.
+ */
+int oracle_fit_sgd(const float* X, const float* y, int64_t m, int32_t n, double lr, int64_t batch_rows, int32_t steps,
+                   int64_t first_batch, double* w, double* b, double* loss_hist) {
+    if (!X || !y || !w || !b || m < 1 || n < 1 || steps < 0 || batch_rows < 1 || batch_rows > m || first_batch < 0) return -1;
+    double* g = (double*)malloc(sizeof(double) * (size_t)n);
+    if (!g) return -1;
+    int64_t nb = (m + batch_rows - 1) / batch_rows;
+    for (int32_t s = 0; s < steps; ++s) {
+        int64_t k = (first_batch + s) % nb;
+        int64_t r0 = k * batch_rows;
+        int64_t rows = batch_rows < m - r0 ? batch_rows : m - r0;
+        double loss, gb;
+        if (oracle_loss_grad(X + r0 * (int64_t)n, y + r0, rows, n, w, *b, &loss, g, &gb) != 0) { free(g); return -1; }
+        if (loss_hist) loss_hist[s] = loss;
+        for (int32_t j = 0; j < n; ++j) w[j] -= lr * g[j];
+        *b -= lr * gb;
     }
     free(g);
     return 0;

@@ -21,7 +21,7 @@ LR_ERR_NULL, LR_ERR_SHAPE, LR_ERR_ALIGNMENT, LR_ERR_VALUE, LR_ERR_CUDA, LR_ERR_T
 EXPORTS = ["lr_plan_query", "lr_create", "lr_destroy", "lr_loss_grad", "lr_fit", "lr_predict", "lr_shard_sums",
            "lr_apply_sums", "lr_fit_host",
            "lr_predict_host", "lr_profile_enable", "lr_profile_read", "lr_launch_count", "lr_last_device_status",
-           "lr_last_cuda_error", "lr_status_string", "lr_loss_grad_noalloc", "lr_fit_tol", "lr_fit_opt", "lr_selftest_wait", "lr_set_persistent"]
+           "lr_last_cuda_error", "lr_status_string", "lr_loss_grad_noalloc", "lr_fit_tol", "lr_fit_opt", "lr_selftest_wait", "lr_set_persistent", "lr_fit_sgd"]
 
 
 class LrPlan(ctypes.Structure):
@@ -66,6 +66,7 @@ def lib() -> ctypes.CDLL:
                                  ctypes.POINTER(F), P]
         L.lr_fit_opt.argtypes = [P, P, P, I64, I32, F, I32, ctypes.POINTER(LrOpt), P, P, P, P, P]
         L.lr_selftest_wait.argtypes = [P, I32, I32, P]
+        L.lr_fit_sgd.argtypes = [P, P, P, I64, I32, F, I64, I32, I64, P, P, P, P]
         L.lr_set_persistent.argtypes = [P, I32]
         L.lr_loss_grad_noalloc.argtypes = [I32, P, P, I64, I32, P, P, P, P, P, P, P]
         L.lr_fit_host.argtypes = [P, P, P, I64, I32, F, I32, P, P, P]
@@ -191,6 +192,14 @@ class Context:
                               _dev_ptr(velocity, torch.float32, "velocity"), _dev_ptr(loss_hist, torch.float32, "loss_hist"),
                               self._stream())
         self._check(rc, "lr_fit_opt")
+
+    def fit_sgd(self, X, y, lr, batch_rows, steps, w, b, first_batch=0, loss_hist=None):
+        """Mini-batch GD over contiguous row blocks (block (first_batch + s) mod count at step s), in place on w, b."""
+        m, n = X.shape
+        rc = lib().lr_fit_sgd(self._h, _dev_ptr(X, torch.float32, "X"), _dev_ptr(y, torch.float32, "y"), m, n, float(lr),
+                              int(batch_rows), int(steps), int(first_batch), _dev_ptr(w, torch.float32, "w"),
+                              _dev_ptr(b, torch.float32, "b"), _dev_ptr(loss_hist, torch.float32, "loss_hist"), self._stream())
+        self._check(rc, "lr_fit_sgd")
 
     def predict(self, X, w, b, thr):
         m, n = X.shape

@@ -564,6 +564,36 @@ int lr_fit_opt(lr_ctx* ctx, const float* d_X, const float* d_y, int64_t m, int32
     return LR_OK;
 }
 
+int lr_fit_sgd(lr_ctx* ctx, const float* d_X, const float* d_y, int64_t m, int32_t n, float lr, int64_t batch_rows,
+               int32_t steps, int64_t first_batch, float* d_w, float* d_b, float* d_loss_hist, void* stream) {
+    int rc = check_common(ctx, d_X, m, n, d_w, d_b);
+    if (rc != LR_OK) return rc;
+    if (!d_y) return LR_ERR_NULL;
+    if (steps < 0 || batch_rows < 1 || batch_rows > m || first_batch < 0) return LR_ERR_SHAPE;
+    if (!aligned(d_y, 4) || (d_loss_hist && !aligned(d_loss_hist, 4))) return LR_ERR_ALIGNMENT;
+    if (!std::isfinite(lr)) return LR_ERR_VALUE;
+    if (steps == 0) return LR_OK;
+    DeviceGuard g(ctx);
+    if (!g.ok) return LR_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int64_t nb = (m + batch_rows - 1) / batch_rows;
+    for (int32_t s = 0; s < steps; ++s) {
+        const int64_t k = (first_batch + s) % nb;
+        const int64_t r0 = k * batch_rows;
+        const int64_t rows = std::min(batch_rows, m - r0);
+        const float* Xb = d_X + r0 * n;
+        lr_plan P;
+        rc = make_plan(rows, n, aligned(Xb, 16), ctx->sm_count, &P);
+        if (rc != LR_OK) return rc;
+        rc = launch_stream_pass(ctx, P, Pass{Xb, d_y + r0, rows, n, d_w, d_b}, nullptr, 0.f, st);
+        if (rc != LR_OK) return rc;
+        rc = launch_reduce(ctx, ctx->d_partial, P.grid, rows, n, double(lr), true, d_w, d_b, nullptr, nullptr,
+                           d_loss_hist ? d_loss_hist + s : nullptr, nullptr, st);
+        if (rc != LR_OK) return rc;
+    }
+    return LR_OK;
+}
+
 int lr_predict(lr_ctx* ctx, const float* d_X, int64_t m, int32_t n, const float* d_w, const float* d_b, float thr,
                uint8_t* d_labels, void* stream) {
     int rc = check_common(ctx, d_X, m, n, d_w, d_b);

@@ -52,6 +52,36 @@ def test_fit_opt_matches_oracle(ctx, name, m, n, opt):
     assert np.max(np.abs(lh.cpu().numpy() - lh_ref)) <= LOSS_TOL
 
 
+@pytest.mark.parametrize("name,m,n,batch", [("cfg3", 50_003, None, 8_192), ("cfg5", 120_001, None, 30_000), ("cfg2", 9_000, 30, 2_500),
+                                            ("cfg3", 6_001, 2048, 1_000), ("cfg1", 10_000, None, 10_000)])
+def test_minibatch_descent_matches_oracle(ctx, name, m, n, batch):
+    import dataclasses
+    wl = datagen.scaled(datagen.WORKLOADS[name], m)
+    if n is not None:
+        wl = dataclasses.replace(wl, n=n)
+    X, y, _, _ = datagen.generate(wl)
+    dX, dy = dev(X), dev(y)
+    steps, lr = 17, 0.2
+    w_ref, b_ref, lh_ref = oracle.fit_sgd(X, y, lr, batch, steps)
+    w = torch.zeros(wl.n, device="cuda")
+    b = torch.zeros(1, device="cuda")
+    lh = torch.empty(steps, device="cuda")
+    ctx.fit_sgd(dX, dy, lr, batch, steps, w, b, loss_hist=lh)
+    assert rel_l2(np.concatenate([w.cpu().numpy(), b.cpu().numpy()]), np.concatenate([w_ref, [b_ref]])) <= W_TOL
+    assert np.max(np.abs(lh.cpu().numpy() - lh_ref)) <= LOSS_TOL
+    # split across two calls with first_batch: the same bits
+    w2 = torch.zeros(wl.n, device="cuda")
+    b2 = torch.zeros(1, device="cuda")
+    ctx.fit_sgd(dX, dy, lr, batch, 6, w2, b2)
+    ctx.fit_sgd(dX, dy, lr, batch, steps - 6, w2, b2, first_batch=6)
+    assert torch.equal(w2, w) and torch.equal(b2, b)
+    if batch == m:
+        wf, bf = api.lr_fit(dX, dy, lr, steps, ctx=ctx)
+        assert torch.equal(wf, w) and torch.equal(bf, b)        # one block per step is the plain fit
+    with pytest.raises(api.LrError):
+        ctx.fit_sgd(dX, dy, lr, m + 1, 1, w2, b2)
+
+
 def test_defaults_reproduce_plain_fit_and_velocity_resumes(ctx):
     wl = datagen.scaled(datagen.WORKLOADS["cfg3"], 20_000)
     X, y, _, _ = datagen.generate(wl)

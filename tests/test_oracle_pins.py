@@ -307,3 +307,29 @@ def test_penalty_and_momentum_follow_their_definitions():
     wa2, ba2, va2, _ = oracle.fit_opt(X, y, lr, 3, l2=l2, momentum=mu, w0=wa1, b0=ba1, vel0=va1)
     wa3, ba3, va3, _ = oracle.fit_opt(X, y, lr, 7, l2=l2, momentum=mu)
     assert np.array_equal(wa2, wa3) and ba2 == ba3 and np.array_equal(va2, va3)
+
+
+def test_minibatch_descent_walks_contiguous_blocks():
+    X, y, _, _ = datagen.random_problem(1000, 4, seed=14)
+    lr = 0.3
+    # one block = the plain fit
+    w0, b0, lh0 = oracle.fit_sgd(X, y, lr, 1000, 6)
+    wf, bf, lhf = oracle.fit(X, y, lr, 6)
+    assert np.array_equal(w0, wf) and b0 == bf and np.array_equal(lh0, lhf)
+    # blocks of 300 rows: 300, 300, 300, 100; five steps by hand with the plain loss/gradient routine on slices
+    w, b, losses = np.zeros(4), 0.0, []
+    spans = [(0, 300), (300, 600), (600, 900), (900, 1000), (0, 300)]
+    for a, c in spans:
+        L, g, gb = oracle.loss_grad(X[a:c], y[a:c], w, b)
+        losses.append(L)
+        w, b = w - lr * g, b - lr * gb
+    w1, b1, lh1 = oracle.fit_sgd(X, y, lr, 300, 5)
+    np.testing.assert_allclose(w1, w, atol=1e-16, rtol=0)
+    assert abs(b1 - b) < 1e-16
+    np.testing.assert_allclose(lh1, losses, atol=1e-16, rtol=0)
+    # resuming at the right block continues the same walk
+    wa, ba, _ = oracle.fit_sgd(X, y, lr, 300, 3)
+    wb, bb, _ = oracle.fit_sgd(X, y, lr, 300, 2, first_batch=3, w0=wa, b0=ba)
+    assert np.array_equal(wb, w1) and bb == b1
+    with pytest.raises(ValueError):
+        oracle.fit_sgd(X, y, lr, 1001, 1)
