@@ -152,6 +152,15 @@ def run_reference(args, wl):
     print(json.dumps(line))
 
 
+def f1_score(labels, y):
+    """F1 of uint8 labels against 0/1 targets, 0 when nothing is predicted positive correctly (plain counting)."""
+    import numpy as np
+    pos = y > 0.5
+    pred = labels != 0
+    tp = int(np.count_nonzero(pred & pos)); fp = int(np.count_nonzero(pred & ~pos)); fn = int(np.count_nonzero(~pred & pos))
+    return (2.0 * tp / (2.0 * tp + fp + fn)) if tp > 0 else 0.0, tp, fp, fn
+
+
 def workload_config(wl, n_gpus):
     return {"workload": f"{wl.name}: m={wl.m} x n={wl.n} fp32 row-major, lr={wl.lr}, {wl.iters} iterations"
                         + (f" (per GPU; {n_gpus} row shards)" if n_gpus > 1 else ""),
@@ -190,7 +199,7 @@ def run_tol(args, wl):
     torch.cuda.synchronize()
     secs = ev0.elapsed_time(ev1) / 1e3
     labels = ctx.predict(dX[m_tr:], w, b, 0.5).cpu().numpy()
-    f1 = oracle.f1_score(labels, y[m_tr:])[0]
+    f1 = f1_score(labels, y[m_tr:])[0]
     k = max(2, min(iters, 40))
     t0 = time.perf_counter()
     oracle.fit(X[:m_tr], y[:m_tr], alpha, k)
@@ -360,6 +369,24 @@ def main():
                "d2h_bytes_per_step": (4 * wl.n + 4) / wl.iters, "seconds_per_fit": t_e2e,
                "what": f"lr_fit_host: pinned X, y copied in, {wl.iters} iterations, w, b copied out; median of 3"}
 
+    # ---- workloads that ask for it: the workload's own fit from zero, then predict at its threshold and F1 against y ----
+    predict = None
+    if wl.predict_thr is not None and world == 1:
+        w.zero_(); b.zero_()
+        ctx.fit(dX, dy, wl.lr, wl.iters, w, b)
+        for _ in range(3):
+            labels = ctx.predict(dX, w, b, wl.predict_thr)
+        pe0, pe1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        pe0.record()
+        for _ in range(10):
+            labels = ctx.predict(dX, w, b, wl.predict_thr)
+        pe1.record()
+        torch.cuda.synchronize()
+        p_ms = pe0.elapsed_time(pe1) / 10
+        f1, tp, fp, fn = f1_score(labels.cpu().numpy(), y_np)
+        predict = {"thr": wl.predict_thr, "f1_vs_y": f1, "tp": tp, "fp": fp, "fn": fn, "ms_per_predict": p_ms,
+                   "gbs": (4 * wl.m * wl.n + wl.m) / (p_ms * 1e-3) / 1e9, "after_iterations": wl.iters}
+
     # ---- CPU checker on this host's cores (reported baseline, not a target) ----
     cpu = None
     if not args.no_cpu_baseline and world == 1:
@@ -370,7 +397,8 @@ def main():
             "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "f32", "data": "synthetic", "config": workload_config(wl, world),
             "achieved_hbm_gbs_whole_step": bytes_per_launch * world * args.steps / (ms * 1e-3) / 1e9,
-            "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches, "clocks": clocks}
+            "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches, "clocks": clocks,
+            "predict": predict}
     print(json.dumps(line))
     ctx.close()
     if world > 1:

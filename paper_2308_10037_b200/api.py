@@ -201,9 +201,9 @@ class Context:
                               _dev_ptr(b, torch.float32, "b"), _dev_ptr(loss_hist, torch.float32, "loss_hist"), self._stream())
         self._check(rc, "lr_fit_sgd")
 
-    def predict(self, X, w, b, thr):
+    def predict(self, X, w, b, thr, out=None):
         m, n = X.shape
-        labels = torch.empty(m, dtype=torch.uint8, device=X.device)
+        labels = torch.empty(m, dtype=torch.uint8, device=X.device) if out is None else out
         rc = lib().lr_predict(self._h, _dev_ptr(X, torch.float32, "X"), m, n, _dev_ptr(w, torch.float32, "w"),
                               _dev_ptr(b, torch.float32, "b"), float(thr), _dev_ptr(labels, torch.uint8, "labels"),
                               self._stream())

@@ -225,6 +225,7 @@ __global__ void __launch_bounds__(NW * 32, 1) k_stream_rows(const StreamParams p
         if (cnt > 0 && row0 + myr < p.m) y_next = __ldg(p.y + row0 + myr);
     }
     const bool full_cols = n4 == NV * LPR;         // every lane's column groups exist
+    const bool labels_word_aligned = PREDICT && (reinterpret_cast<uintptr_t>(p.labels) & 3u) == 0 && RPB % 4 == 0;
     int issued = cnt < D ? cnt : D;                // warp-uniform count of batches whose copies were issued
     int done = 0;                                  // batches whose stage wait has succeeded
     int since_flush = 0;
@@ -262,7 +263,22 @@ __global__ void __launch_bounds__(NW * 32, 1) k_stream_rows(const StreamParams p
         const float z = batch_dot<NV, LPR, RB>(x, wv, lane) + bval;
 
         if constexpr (PREDICT) {
-            if (owner && myvalid) p.labels[row0 + myr] = z >= p.cut ? 1 : 0;
+            // one bit per lane, then RPB/4 lanes each assemble and store four labels as one 32-bit word
+            const unsigned hit = __ballot_sync(FULL, owner && myvalid && z >= p.cut);
+            if (rows == RPB && labels_word_aligned) {
+                if (lane < RPB / 4) {
+                    unsigned word = 0;
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        const int r = 4 * lane + q;                                   // row of the batch
+                        const int src = (r % RPW) * LPR + ((r / RPW) << SHIFT);       // the owner lane of that row
+                        word |= ((hit >> src) & 1u) << (8 * q);
+                    }
+                    *reinterpret_cast<unsigned*>(p.labels + row0 + 4 * lane) = word;
+                }
+            } else if (owner && myvalid) {
+                p.labels[row0 + myr] = z >= p.cut ? 1 : 0;
+            }
         } else {
             float e, L;
             logistic_terms(z, yv, e, L);

@@ -109,6 +109,7 @@ __global__ void __launch_bounds__(NW * 32, 1) k_stream_split(const __grid_consta
     const int dup = lane & (DUP - 1);              // which of the lanes sharing that row this one is
     const bool owner = dup == 0;
     const bool full_cw = CW == 32 * NV;            // every lane's column groups lie inside the box
+    const bool labels_word_aligned = PREDICT && (reinterpret_cast<uintptr_t>(p.labels) & 3u) == 0;
 
     const bool active = mycw > 0;
     if (active && lane == 0) {
@@ -190,7 +191,19 @@ __global__ void __launch_bounds__(NW * 32, 1) k_stream_split(const __grid_consta
         const float z = zs + bval;
 
         if constexpr (PREDICT) {
-            if (warp == 0 && owner && myvalid) p.labels[row0 + myr] = z >= p.cut ? 1 : 0;
+            if (warp == 0) {
+                const unsigned hit = __ballot_sync(FULL, owner && myvalid && z >= p.cut);
+                if (row0 + RB <= p.m && labels_word_aligned) {
+                    if (lane < RB / 4) {
+                        unsigned word = 0;
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) word |= ((hit >> ((4 * lane + q) << SHIFT)) & 1u) << (8 * q);
+                        *reinterpret_cast<unsigned*>(p.labels + row0 + 4 * lane) = word;
+                    }
+                } else if (owner && myvalid) {
+                    p.labels[row0 + myr] = z >= p.cut ? 1 : 0;
+                }
+            }
         } else {
             float e;
             if (warp == 0) {                       // warp-uniform: the loss term is needed once per row

@@ -161,6 +161,23 @@ def test_predict_matches_oracle(ctx, m, n):
         assert (got == ref).mean() >= LABEL_AGREE or m < 10_000 and (got != ref).sum() <= 1
 
 
+@pytest.mark.parametrize("m,n", [(70_003, 64), (9_001, 2048), (40_001, 28)])
+def test_predict_into_an_unaligned_label_buffer(ctx, m, n):
+    # labels are written four at a time as 32-bit words when the buffer allows it; a byte-offset view must fall back to byte
+    # stores, give the same labels, and leave its neighbours alone
+    X, y, w, b = datagen.random_problem(m, n, seed=70 + n, wscale=2.0)
+    dX, dw, db = dev(X), dev(w), dev(np.array([b], dtype=np.float32))
+    ref = ctx.predict(dX, dw, db, 0.5)
+    buf = torch.full((m + 9,), 7, dtype=torch.uint8, device="cuda")
+    for off in (1, 2, 3, 4):
+        buf.fill_(7)
+        ctx.predict(dX, dw, db, 0.5, out=buf[off:off + m])
+        assert torch.equal(buf[off:off + m], ref)
+        assert bool((buf[:off] == 7).all()) and bool((buf[off + m:] == 7).all())
+    lab_ref = oracle.predict(X, w, b, 0.5)
+    assert (ref.cpu().numpy() == lab_ref).mean() >= LABEL_AGREE
+
+
 def test_predict_after_fit_agrees_and_f1_matches(ctx):
     wl = datagen.scaled(datagen.WORKLOADS["cfg2"], 60_000)
     X, y, _, _ = datagen.generate(wl)
