@@ -465,9 +465,13 @@ int lr_fit(lr_ctx* ctx, const float* d_X, const float* d_y, int64_t m, int32_t n
         fp.iters = iters; fp.lr = double(lr); fp.inv_m = 1.0 / double(m);
         LR_CK(ctx, cudaMemsetAsync(ctx->d_gbar, 0, sizeof(unsigned int), st));
         const int smem = int(kHeaderBytes + int64_t(kNW) * depth * stage_stride + kFitTailBytes);
-        LR_CK(ctx, launch_fit(P, smem, fp, st));
-        ctx->launches += 1;
-        return LR_OK;
+        const cudaError_t le = launch_fit(P, smem, fp, st);
+        if (le == cudaSuccess) {
+            ctx->launches += 1;
+            return LR_OK;
+        }
+        if (le != cudaErrorCooperativeLaunchTooLarge) { ctx->last_cuda = int(le); return LR_ERR_CUDA; }
+        cudaGetLastError();                        // the CTAs cannot all be resident here: use the two-kernel form below
     }
     for (int32_t t = 0; t < iters; ++t) {
         rc = launch_stream_pass(ctx, P, Pass{d_X, d_y, m, n, d_w, d_b}, nullptr, 0.f, st);
