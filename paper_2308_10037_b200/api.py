@@ -21,7 +21,7 @@ LR_ERR_NULL, LR_ERR_SHAPE, LR_ERR_ALIGNMENT, LR_ERR_VALUE, LR_ERR_CUDA, LR_ERR_T
 EXPORTS = ["lr_plan_query", "lr_create", "lr_destroy", "lr_loss_grad", "lr_fit", "lr_predict", "lr_shard_sums",
            "lr_apply_sums", "lr_fit_host",
            "lr_predict_host", "lr_profile_enable", "lr_profile_read", "lr_launch_count", "lr_last_device_status",
-           "lr_last_cuda_error", "lr_status_string", "lr_loss_grad_noalloc", "lr_fit_tol", "lr_fit_opt", "lr_selftest_wait", "lr_set_persistent", "lr_fit_sgd"]
+           "lr_last_cuda_error", "lr_status_string", "lr_loss_grad_noalloc", "lr_fit_tol", "lr_fit_opt", "lr_selftest_wait", "lr_set_persistent", "lr_fit_sgd", "lr_set_l2_keep"]
 
 
 class LrPlan(ctypes.Structure):
@@ -68,6 +68,7 @@ def lib() -> ctypes.CDLL:
         L.lr_selftest_wait.argtypes = [P, I32, I32, P]
         L.lr_fit_sgd.argtypes = [P, P, P, I64, I32, F, I64, I32, I64, P, P, P, P]
         L.lr_set_persistent.argtypes = [P, I32]
+        L.lr_set_l2_keep.argtypes = [P, I64]
         L.lr_loss_grad_noalloc.argtypes = [I32, P, P, I64, I32, P, P, P, P, P, P, P]
         L.lr_fit_host.argtypes = [P, P, P, I64, I32, F, I32, P, P, P]
         L.lr_predict_host.argtypes = [P, P, I64, I32, P, P, F, P]
@@ -254,6 +255,10 @@ class Context:
         v = ctypes.c_int64()
         self._check(lib().lr_launch_count(self._h, ctypes.byref(v)), "lr_launch_count")
         return v.value
+
+    def set_l2_keep(self, nbytes: int):
+        """Ask for the first ``nbytes`` of X to be kept in L2 across the passes of a fit (0 = off)."""
+        self._check(lib().lr_set_l2_keep(self._h, int(nbytes)), "lr_set_l2_keep")
 
     def set_persistent(self, on: bool):
         """Allow (default) or forbid the single-launch persistent kernel in ``fit``; results are identical either way."""

@@ -130,6 +130,8 @@ struct lr_ctx {
     unsigned int* d_gbar = nullptr;                 // grid-barrier counter of the persistent fit kernel
     bool coop = false;                              // device supports cooperative launches
     bool persistent = true;                         // lr_fit may use the single-launch kernel
+    int64_t l2_keep_bytes = -1;                     // leading bytes of X fetched with an evict-last hint; -1 = per-kernel default
+    int64_t l2_bytes = 0;                           // size of the device's L2
     // buffers of the host-pointer entry points (grown on demand)
     void* d_hX = nullptr; size_t hX_bytes = 0;
     void* d_hy = nullptr; size_t hy_bytes = 0;
@@ -247,6 +249,14 @@ cudaError_t launch_fit(const lr_plan& P, int smem, FitParams& fp, cudaStream_t s
     return launch_fit_t<4, 32, 2>(P, smem, fp, st);
 }
 
+// Rows of X to fetch with the evict-last hint.  Default: none for the narrow-row kernels (measured: any kept part slows
+// them down), three quarters of the L2 for the wide-row kernel (measured on 100k x 4096: 0.260 -> 0.231 ms per pass).
+int64_t keep_rows_for(const lr_ctx* ctx, int variant, int32_t n) {
+    int64_t bytes = ctx->l2_keep_bytes;
+    if (bytes < 0) bytes = variant == 1 ? ctx->l2_bytes / 4 * 3 : 0;
+    return bytes / (int64_t(n) * 4);
+}
+
 struct Pass {
     const float* X; const float* y; int64_t m; int32_t n; const float* w; const float* b;
     const int* stop = nullptr;                      // device flag that turns the launch into a no-op once set
@@ -275,6 +285,7 @@ int launch_stream_pass(lr_ctx* ctx, const lr_plan& P, const Pass& a, uint8_t* la
         sp.partial = ctx->d_partial; sp.labels = labels; sp.cut = cut; sp.status = ctx->d_status; sp.stop = a.stop;
         sp.depth = P.stages;
         sp.num_batches = (a.m + P.rows_per_batch - 1) / P.rows_per_batch;
+        sp.keep_rows = keep_rows_for(ctx, 0, a.n);
         e = predict ? launch_rows<true>(P, sp, st) : launch_rows<false>(P, sp, st);
     } else if (P.variant == 1) {
         SplitParams sp{};
@@ -283,6 +294,7 @@ int launch_stream_pass(lr_ctx* ctx, const lr_plan& P, const Pass& a, uint8_t* la
         sp.depth = P.stages;
         sp.cw = (a.n / 4 + kNW - 1) / kNW;
         sp.num_batches = (a.m + P.rows_per_batch - 1) / P.rows_per_batch;
+        sp.keep_rows = keep_rows_for(ctx, 1, a.n);
         e = predict ? launch_split<true>(P, a.X, sp, st) : launch_split<false>(P, a.X, sp, st);
     } else {
         GenericParams gp{};
@@ -370,6 +382,11 @@ int lr_create(lr_ctx** out, int32_t device, int32_t n_max) {
     if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&c->d_oticket), sizeof(unsigned int));
     if (e == cudaSuccess) e = cudaMemset(c->d_oticket, 0, sizeof(unsigned int));
     if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&c->d_gbar), sizeof(unsigned int));
+    if (e == cudaSuccess) {
+        int l2 = 0;
+        e = cudaDeviceGetAttribute(&l2, cudaDevAttrL2CacheSize, device);
+        c->l2_bytes = l2;
+    }
     if (e == cudaSuccess) {
         int coop = 0;
         e = cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, device);
@@ -463,6 +480,7 @@ int lr_fit(lr_ctx* ctx, const float* d_X, const float* d_y, int64_t m, int32_t n
         fp.loss_hist = d_loss_hist; fp.status = ctx->d_status; fp.gbar = ctx->d_gbar; fp.depth = depth;
         fp.num_batches = (m + P.rows_per_batch - 1) / P.rows_per_batch;
         fp.iters = iters; fp.lr = double(lr); fp.inv_m = 1.0 / double(m);
+        fp.keep_rows = keep_rows_for(ctx, 0, n);
         LR_CK(ctx, cudaMemsetAsync(ctx->d_gbar, 0, sizeof(unsigned int), st));
         const int smem = int(kHeaderBytes + int64_t(kNW) * depth * stage_stride + kFitTailBytes);
         const cudaError_t le = launch_fit(P, smem, fp, st);
@@ -480,6 +498,13 @@ int lr_fit(lr_ctx* ctx, const float* d_X, const float* d_y, int64_t m, int32_t n
                            d_loss_hist ? d_loss_hist + t : nullptr, nullptr, st);
         if (rc != LR_OK) return rc;
     }
+    return LR_OK;
+}
+
+int lr_set_l2_keep(lr_ctx* ctx, int64_t bytes) {
+    if (!ctx) return LR_ERR_NULL;
+    if (bytes < -1) return LR_ERR_VALUE;
+    ctx->l2_keep_bytes = bytes;
     return LR_OK;
 }
 

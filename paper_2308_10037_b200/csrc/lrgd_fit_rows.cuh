@@ -37,6 +37,7 @@ struct FitParams {
     unsigned int* gbar;        // grid-barrier counter, zero at launch
     int depth;
     long long num_batches;
+    long long keep_rows;       // rows [0, keep_rows) are fetched with an L2 evict-last hint, the rest evict-first
     int iters;
     double lr;
     double inv_m;
@@ -106,7 +107,7 @@ __global__ void __launch_bounds__(NW * 32, 1) k_fit_rows(const FitParams p) {
     }
     __syncthreads();
 
-    const uint64_t pol = l2_policy_evict_first();
+    const uint64_t pol_stream = l2_policy_evict_first(), pol_keep = l2_policy_evict_last();
     const long long stride_rows = static_cast<long long>(G) * NW * RPB;
     const long long first_row = (static_cast<long long>(blockIdx.x) * NW + warp) * RPB;
     auto issue = [&](long long r0, int d) {        // lane 0 only
@@ -114,7 +115,8 @@ __global__ void __launch_bounds__(NW * 32, 1) k_fit_rows(const FitParams p) {
         const uint32_t rows = left < RPB ? static_cast<uint32_t>(left) : RPB;
         const uint32_t xbytes = rows * n * 4u;
         mbar_arrive_expect_tx(&my_bars[d], xbytes);
-        bulk_copy_g2s(my_stages + static_cast<size_t>(d) * stage_stride, p.X + r0 * n, xbytes, &my_bars[d], pol);
+        bulk_copy_g2s(my_stages + static_cast<size_t>(d) * stage_stride, p.X + r0 * n, xbytes, &my_bars[d],
+                      r0 < p.keep_rows ? pol_keep : pol_stream);
     };
 
     const int sub = lane & (LPR - 1), slot = lane >> LOG_LPR;

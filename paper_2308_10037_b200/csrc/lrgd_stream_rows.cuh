@@ -42,6 +42,7 @@ struct StreamParams {
     const int* stop;          // nullable: non-zero means a stopping rule has been met and the launch is a no-op
     int depth;                // stages per warp (1..kMaxDepth)
     long long num_batches;    // ceil(m / rows per batch)
+    long long keep_rows;      // rows [0, keep_rows) are fetched with an L2 evict-last hint (kept across passes), the rest evict-first
 };
 
 // Sums C values per lane across the lanes selected by masks M, M/2, ..., 1.  While more than one value
@@ -181,7 +182,7 @@ __global__ void __launch_bounds__(NW * 32, 1) k_stream_rows(const StreamParams p
     }
     __syncthreads();
 
-    const uint64_t pol = l2_policy_evict_first();
+    const uint64_t pol_stream = l2_policy_evict_first(), pol_keep = l2_policy_evict_last();
     const long long stride_rows = static_cast<long long>(gridDim.x) * NW * RPB;       // rows between this warp's batches
     long long row0 = (static_cast<long long>(blockIdx.x) * NW + warp) * RPB;          // first row of the current batch
     // (re)fills stage d with the batch that starts at row r0; called by lane 0 only
@@ -190,7 +191,8 @@ __global__ void __launch_bounds__(NW * 32, 1) k_stream_rows(const StreamParams p
         const uint32_t rows = left < RPB ? static_cast<uint32_t>(left) : RPB;
         const uint32_t xbytes = rows * n * 4u;
         mbar_arrive_expect_tx(&my_bars[d], xbytes);
-        bulk_copy_g2s(my_stages + static_cast<size_t>(d) * stage_stride, p.X + r0 * n, xbytes, &my_bars[d], pol);
+        bulk_copy_g2s(my_stages + static_cast<size_t>(d) * stage_stride, p.X + r0 * n, xbytes, &my_bars[d],
+                      r0 < p.keep_rows ? pol_keep : pol_stream);
     };
 
     float4 acc[NV];

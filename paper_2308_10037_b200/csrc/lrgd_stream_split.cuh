@@ -41,6 +41,7 @@ struct SplitParams {
     int depth;                // stages per warp
     int cw;                   // 16-byte column groups per warp slice (the tensor map's box is cw*4 floats by RB rows)
     long long num_batches;    // ceil(m / RB)
+    long long keep_rows;      // rows [0, keep_rows) are fetched with an L2 evict-last hint, the rest evict-first
 };
 
 template <int NV, int RB, int NW, bool PREDICT>
@@ -81,12 +82,13 @@ __global__ void __launch_bounds__(NW * 32, 1) k_stream_split(const __grid_consta
     }
     __syncthreads();
 
-    const uint64_t pol = l2_policy_evict_first();
+    const uint64_t pol_stream = l2_policy_evict_first(), pol_keep = l2_policy_evict_last();
     const int stride_rows = static_cast<int>(gridDim.x) * RB;                 // rows between this CTA's batches (m < 2^31 here)
     int row0 = static_cast<int>(blockIdx.x) * RB;                             // first row of the current batch
     auto issue = [&](int r0, int d) {              // lane 0 of a warp with mycw > 0
         mbar_arrive_expect_tx(&my_bars[d], box_bytes);
-        bulk_tensor_2d_g2s(my_stages + static_cast<size_t>(d) * stage_stride, &tmap, c0 * 4, r0, &my_bars[d], pol);
+        bulk_tensor_2d_g2s(my_stages + static_cast<size_t>(d) * stage_stride, &tmap, c0 * 4, r0, &my_bars[d],
+                           r0 < p.keep_rows ? pol_keep : pol_stream);
     };
 
     float4 acc[NV];
