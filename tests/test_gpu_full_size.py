@@ -76,3 +76,25 @@ def test_full_size_workload(ctx, name):
         # and free-running: labels from the GPU's own fit against labels from the checker's own fit
         own = api.lr_predict(dX, w, b, 0.5, ctx=ctx).cpu().numpy()
         assert (own == oracle.predict(X, w_ref, b_ref, 0.5)).mean() >= LABEL_AGREE
+
+
+def test_more_than_2_to_31_elements(ctx):
+    # 36,000,007 x 64 = 2.3e9 elements (9.2 GB): element offsets pass 2^31 and byte offsets pass 2^33, with a ragged tail.
+    # One pass at non-trivial parameters against the checker, and labels on the last rows (the ones with the largest offsets).
+    import dataclasses
+    wl = dataclasses.replace(datagen.WORKLOADS["cfg5"], m=36_000_007, name="cfg5_big")
+    X, y, wstar, bstar = datagen.generate(wl)
+    dX, dy = torch.from_numpy(X).cuda(), torch.from_numpy(y).cuda()
+    w32 = (0.5 * wstar).astype(np.float32)
+    b32 = np.float32(0.5 * bstar)
+    dw, db = torch.from_numpy(w32).cuda(), torch.tensor([b32], device="cuda")
+    L, g, g0 = oracle.loss_grad(X, y, w32.astype(np.float64), float(b32))
+    dl, dg, dg0 = ctx.loss_grad(dX, dy, dw, db)
+    assert abs(dl.item() - L) <= LOSS_TOL
+    assert_grad_close(np.concatenate([dg.cpu().numpy(), dg0.cpu().numpy()]), np.concatenate([g, [g0]]), 0.0, "big")
+    labels = ctx.predict(dX, dw, db, 0.02).cpu().numpy()
+    tail = slice(wl.m - 2_000_000, wl.m)
+    ref = oracle.predict(X[tail], w32.astype(np.float64), float(b32), 0.02)
+    assert (labels[tail] == ref).mean() >= LABEL_AGREE
+    del dX, dy
+    torch.cuda.empty_cache()

@@ -278,3 +278,22 @@ def test_row_sharded_entry_points_match_oracle(ctx):
     L1, g1, g01 = oracle.loss_grad(X[a0:b0], y[a0:b0], w_prev, b_prev)
     got = sums[1].cpu().numpy() / (b0 - a0)
     assert rel_l2(got[:wl.n + 1], np.concatenate([g1, [g01]])) <= 1e-3 and abs(got[wl.n + 1] - L1) <= 1e-5
+
+
+def test_misaligned_pointers_are_rejected(ctx):
+    # float arrays must be 4-byte aligned: a byte-offset view of a byte buffer is not
+    import ctypes
+    X, y, w, b = datagen.random_problem(64, 8, seed=2)
+    dX, dy, dw, db = dev(X), dev(y), dev(w), dev(np.array([b], dtype=np.float32))
+    raw = torch.zeros(64 * 8 * 4 + 8, dtype=torch.uint8, device="cuda")
+    bad = ctypes.c_void_p(raw.data_ptr() + 1)
+    out = torch.zeros(16, device="cuda")
+    L = api.lib()
+    P = lambda t: ctypes.c_void_p(t.data_ptr())
+    rc = L.lr_loss_grad(ctx._h, bad, P(dy), 64, 8, P(dw), P(db), P(out), P(out[1:]), P(out[12:]), None)
+    assert rc == api.LR_ERR_ALIGNMENT
+    rc = L.lr_fit(ctx._h, P(dX), bad, 64, 8, 0.1, 1, P(dw), P(db), None, None)
+    assert rc == api.LR_ERR_ALIGNMENT
+    rc = L.lr_predict(ctx._h, P(dX), 64, 8, bad, P(db), 0.5, P(raw), None)
+    assert rc == api.LR_ERR_ALIGNMENT
+    assert ctx.device_status() == 0
