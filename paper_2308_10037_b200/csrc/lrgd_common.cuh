@@ -112,6 +112,12 @@ __device__ __forceinline__ void bulk_copy_g2s(void* dst, const void* src, uint32
         : "memory");
 }
 
+// Asks the memory system to bring [src, src+bytes) into L2 (no destination, no completion signal).
+// src 16-byte aligned, bytes a multiple of 16.
+__device__ __forceinline__ void bulk_prefetch_l2(const void* src, uint32_t bytes, uint64_t policy) {
+    asm volatile("cp.async.bulk.prefetch.L2.global.L2::cache_hint [%0], %1, %2;" ::"l"(src), "r"(bytes), "l"(policy) : "memory");
+}
+
 // Tiled 2-D TMA copy global -> shared through a tensor map (no multicast): the box whose first element has
 // coordinates (x, y) -- x along the contiguous dimension, x*4 bytes a multiple of 16 -- lands densely packed at dst
 // (128-byte aligned); out-of-range elements are written as zeros and count towards the transferred bytes.

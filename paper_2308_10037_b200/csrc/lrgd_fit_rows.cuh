@@ -22,6 +22,10 @@
 namespace lrgd {
 
 constexpr int kFitCombineCols = 64;            // columns combined per pass through the CTA's combine buffer
+#ifndef LRGD_FIT_L2PF
+#define LRGD_FIT_L2PF 4
+#endif
+constexpr int kFitL2Prefetch = LRGD_FIT_L2PF;   // batches per warp pulled into L2 ahead of the next iteration (beyond the staged ones)
 constexpr int kFitTailBytes = 9216;            // combine buffer / reduction slices, after the stages
 
 struct FitParams {
@@ -207,6 +211,21 @@ __global__ void __launch_bounds__(NW * 32, 1) k_fit_rows(const FitParams p) {
             row0 += stride_rows;
         }
         (void)warp_ok;                             // a failed wait has raised the CTA's abort flag; handled at the barrier
+
+        // The grid barriers, the reduction and the parameter reload below take longer than the staged batches of the next
+        // iteration last; keep HBM busy meanwhile by pulling this warp's following batches of that iteration into L2.
+        if (lane == 0 && t + 1 < p.iters) {
+#pragma unroll
+            for (int j = 0; j < kFitL2Prefetch; ++j) {
+                const int bi = D + j;
+                if (bi < cnt) {
+                    const long long r0 = first_row + bi * stride_rows;
+                    const long long left = p.m - r0;
+                    const uint32_t rows = left < RPB ? static_cast<uint32_t>(left) : RPB;
+                    bulk_prefetch_l2(p.X + r0 * n, rows * n * 4u, r0 < p.keep_rows ? pol_keep : pol_stream);
+                }
+            }
+        }
 
         fold_into_fp64<NV>(acc, dacc, se, sl, dse, dsl);
 
