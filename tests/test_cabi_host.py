@@ -97,3 +97,25 @@ def test_pipeline_depth_follows_the_shared_memory_budget():
     assert api.plan_query(16_000_000, 64)["stages"] == 3
     assert api.plan_query(1_000_000, 100)["stages"] == 4        # 3.2 KB batches
     assert api.plan_query(100, 32)["stages"] == 1               # one batch per warp at most
+
+
+def test_header_is_plain_c_and_the_example_links():
+    # include/lrgd.h must be usable from C (no C++ in the boundary); the example program must compile and link against the
+    # built library (it is only run where a GPU exists)
+    import shutil
+    import subprocess
+    import tempfile
+    gcc = shutil.which("gcc")
+    if gcc is None:
+        pytest.skip("no gcc")
+    inc = os.path.join(ROOT, "include")
+    pkg = os.path.join(ROOT, "paper_2308_10037_b200")
+    with tempfile.TemporaryDirectory() as tmp:
+        probe = os.path.join(tmp, "probe.c")
+        with open(probe, "w") as f:
+            f.write('#include "lrgd.h"\nint main(void) { lr_plan p; return lr_plan_query(10, 4, 1, 148, &p) == LR_OK ? 0 : 1; }\n')
+        subprocess.check_call([gcc, "-std=c99", "-Wall", "-Wextra", "-Werror", "-pedantic", "-I", inc, probe, "-L", pkg, "-llrgd",
+                               f"-Wl,-rpath,{pkg}", "-o", os.path.join(tmp, "probe")])
+        subprocess.check_call([os.path.join(tmp, "probe")])          # pure host entry point: runs without a GPU
+        subprocess.check_call([gcc, "-std=c99", "-Wall", "-Werror", "-O1", "-I", inc, os.path.join(pkg, "examples", "fit_host.c"),
+                               "-L", pkg, "-llrgd", f"-Wl,-rpath,{pkg}", "-lm", "-o", os.path.join(tmp, "fit_host")])

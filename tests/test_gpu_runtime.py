@@ -66,3 +66,23 @@ def test_sharded_driver_on_a_one_rank_nccl_group(ctx):
         assert torch.equal(w, wf) and torch.equal(b, bf)
     finally:
         dist.destroy_process_group()
+
+
+def test_c_example_program_runs():
+    # a plain C program linked against the shared library, no Python in between
+    import os
+    import shutil
+    import subprocess
+    import tempfile
+    gcc = shutil.which("gcc")
+    if gcc is None:
+        pytest.skip("no gcc")
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    pkg = os.path.join(root, "paper_2308_10037_b200")
+    with tempfile.TemporaryDirectory() as tmp:
+        exe = os.path.join(tmp, "fit_host")
+        subprocess.check_call([gcc, "-std=c99", "-O2", "-I", os.path.join(root, "include"), os.path.join(pkg, "examples", "fit_host.c"),
+                               "-L", pkg, "-llrgd", f"-Wl,-rpath,{pkg}", "-lm", "-o", exe])
+        out = subprocess.run([exe], capture_output=True, text=True, timeout=120)
+        assert out.returncode == 0, out.stdout + out.stderr
+        assert "device status 0" in out.stdout
