@@ -37,7 +37,7 @@ NOMINAL_HBM_GBS = 8000.0
 # dram__bytes_read.sum + dram__bytes_write.sum of the streaming kernel per row of X, from the ncu capture summarised in
 # profiles/ (taken at m = 500,000 and scaled by rows).  Remove an entry when its kernel changes.
 NCU_TRAFFIC_BYTES_PER_ROW = {"cfg3": {"k_stream_rows": (514.024192e6 + 3.515648e6) / 500_000,
-                                      "k_fit_rows": (1.538055e9 + 3.601664e6) / 3 / 500_000}}
+                                      "k_fit_rows": (1.501203e9 + 3.725824e6) / 3 / 500_000}}
 FALLBACK_HBM_GBS = 6650.0
 
 
