@@ -120,7 +120,9 @@ int lr_set_l2_keep(lr_ctx* ctx, int64_t bytes);
  * Algorithm 7 -- for at most max_iters updates.  The norm is formed on the device in fp64 from the same
  * sums the update uses; once it is met a device flag turns every later launch of this call into a
  * no-op, so the result does not depend on check_every.  The host enqueues check_every iterations at a
- * time and then synchronises `stream` to read the flag (this call blocks, unlike lr_fit).
+ * time and then synchronises `stream` to read the flag (this call blocks, unlike lr_fit).  For rows of up to
+ * 512 columns the whole run is instead ONE persistent launch in which all CTAs form the norm after every update
+ * and leave the loop together (check_every is not used; no launch is wasted); both forms give the same bits.
  * d_w, d_b in/out as for lr_fit; d_loss_hist / d_gnorm_hist are NULL or [max_iters] (entries past the
  * stopping iteration are left untouched); *iters_done receives the number of updates applied and
  * *grad_norm the norm of the last applied gradient (-1 if max_iters == 0).  The caller tells

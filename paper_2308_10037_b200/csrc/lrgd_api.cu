@@ -534,6 +534,32 @@ int lr_fit_tol(lr_ctx* ctx, const float* d_X, const float* d_y, int64_t m, int32
     if (!g.ok) return LR_ERR_CUDA;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     LR_CK(ctx, cudaMemsetAsync(ctx->d_tol, 0, sizeof(TolState), st));
+    // Narrow rows: one persistent launch that leaves its loop on the device as soon as the norm is small enough.
+    if (P.variant == 0 && ctx->persistent && ctx->coop && !ctx->prof && 2ll * max_iters * P.grid < (1ll << 32)) {
+        const int64_t stage_stride = (int64_t(P.rows_per_batch) * n * 4 + 127) & ~int64_t(127);
+        const int64_t room = kMaxDynamicSmem - kHeaderBytes - kFitTailBytes;
+        const int depth = int(std::max<int64_t>(1, std::min<int64_t>(P.stages, room / (kNW * stage_stride))));
+        FitParams fp{};
+        fp.X = d_X; fp.y = d_y; fp.m = m; fp.n = n; fp.w = d_w; fp.b = d_b; fp.partial = ctx->d_partial;
+        fp.loss_hist = d_loss_hist; fp.status = ctx->d_status; fp.gbar = ctx->d_gbar; fp.depth = depth;
+        fp.num_batches = (m + P.rows_per_batch - 1) / P.rows_per_batch;
+        fp.iters = max_iters; fp.lr = double(lr); fp.inv_m = 1.0 / double(m);
+        fp.keep_rows = keep_rows_for(ctx, 0, n);
+        fp.tol = ctx->d_tol; fp.gbuf = ctx->d_gbuf; fp.eps = double(eps); fp.gnorm_hist = d_gnorm_hist;
+        LR_CK(ctx, cudaMemsetAsync(ctx->d_gbar, 0, sizeof(unsigned int), st));
+        const int smem = int(kHeaderBytes + int64_t(kNW) * depth * stage_stride + kFitTailBytes);
+        const cudaError_t le = launch_fit(P, smem, fp, st);
+        if (le == cudaSuccess) {
+            ctx->launches += 1;
+            LR_CK(ctx, cudaMemcpyAsync(ctx->h_tol, ctx->d_tol, sizeof(TolState), cudaMemcpyDeviceToHost, st));
+            LR_CK(ctx, cudaStreamSynchronize(st));
+            *iters_done = ctx->h_tol->iters_done;
+            *grad_norm = static_cast<float>(ctx->h_tol->grad_norm);
+            return LR_OK;
+        }
+        if (le != cudaErrorCooperativeLaunchTooLarge) { ctx->last_cuda = int(le); return LR_ERR_CUDA; }
+        cudaGetLastError();
+    }
     const int* stop = &ctx->d_tol->stop;
     for (int32_t t = 0; t < max_iters;) {
         const int32_t chunk = std::min(check_every, max_iters - t);

@@ -11,6 +11,9 @@
 // while the CTAs reduce iteration t).  This matters for short passes (a 400 MB pass lasts ~60 us, of which launch,
 // ramp-up and tail were ~20 %) and most for L2-resident problems.
 //
+// With a tolerance (lr_fit_tol) the kernel also forms ||grad||_2 after every update and all CTAs leave the loop together
+// once it is <= eps: the stopping rule of Algorithm 7 with no host round trip and no wasted launch.
+//
 // Grid barrier: a monotonic counter in global memory; thread 0 of each CTA adds one and spins (bounded, 2 s) until the
 // counter reaches grid * k.  On expiry, or when another CTA has raised the status word, the CTA stops iterating, waits
 // (bounded) for its own copies in flight and retires with LR_ERR_TIMEOUT in the status word.
@@ -45,6 +48,11 @@ struct FitParams {
     int iters;
     double lr;
     double inv_m;
+    // stopping rule (all null / zero for a fixed-count fit): as in k_reduce_update's tolerance mode
+    TolState* tol;
+    double* gbuf;              // [n+1] gradient entries of the current iteration
+    double eps;
+    float* gnorm_hist;         // nullable [iters]
 };
 
 __device__ __forceinline__ unsigned int ld_acquire_u32(const unsigned int* p) {
@@ -299,17 +307,41 @@ __global__ void __launch_bounds__(NW * 32, 1) k_fit_rows(const FitParams p) {
                     if (col < n) p.w[col] = static_cast<float>(static_cast<double>(__ldcg(p.w + col)) - p.lr * v);
                     else if (col == n) p.b[0] = static_cast<float>(static_cast<double>(__ldcg(p.b)) - p.lr * v);
                     else if (p.loss_hist) p.loss_hist[t] = static_cast<float>(v);
+                    if (p.tol != nullptr && col <= n) p.gbuf[col] = v;
                 }
             }
         }
         barrier_no += 1;
         alive = grid_barrier(p.gbar, static_cast<unsigned int>(G) * barrier_no, p.status, abort_flag);
+
+        // ---- stopping rule (Algorithm 7): ||(grad_w, grad_b)||_2 of the update just applied, formed by every CTA in the
+        // same order as k_reduce_update's last block (lane-strided squares, xor tree), so all CTAs take the same decision ----
+        if (p.tol != nullptr && alive) {
+            double q = 0.0;
+            for (int c = lane; c <= n; c += 32) {
+                const double v = __ldcg(p.gbuf + c);
+                q += v * v;
+            }
+#pragma unroll
+            for (int msk = 16; msk >= 1; msk >>= 1) q += __shfl_xor_sync(FULL, q, msk);
+            const double nrm = sqrt(q);
+            if (blockIdx.x == 0 && threadIdx.x == 0) {
+                p.tol->grad_norm = nrm;
+                p.tol->iters_done = t + 1;
+                if (p.gnorm_hist) p.gnorm_hist[t] = static_cast<float>(nrm);
+                if (nrm <= p.eps) p.tol->stop = 1;
+            }
+            if (nrm <= p.eps) break;               // uniform over the whole grid: every warp computed the same nrm
+        }
     }
 
+    // Copies still in flight when the loop ends (a give-up, or an early stop with the next iteration already being
+    // prefetched) must land before the CTA retires and its shared memory is handed to another CTA.
     if (!alive || *abort_flag) {
-        // gave up: let this warp's copies still in flight land (bounded) before the CTA retires
+        if (lane == 0) atomicExch(p.status, kStatusTimeout);
+    }
+    if (consumed < issued) {
         if (lane == 0) {
-            atomicExch(p.status, kStatusTimeout);
             for (long long f = consumed; f < issued; ++f)
                 mbar_wait_bounded(&my_bars[f % D], static_cast<uint32_t>(f / D) & 1u, abort_flag);
         }
