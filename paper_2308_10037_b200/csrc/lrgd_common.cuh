@@ -118,7 +118,7 @@ __device__ __forceinline__ void bulk_prefetch_l2(const void* src, uint32_t bytes
     asm volatile("cp.async.bulk.prefetch.L2.global.L2::cache_hint [%0], %1, %2;" ::"l"(src), "r"(bytes), "l"(policy) : "memory");
 }
 
-// Tiled 2-D TMA copy global -> shared through a tensor map (no multicast): the box whose first element has
+// Tiled 2-D TMA copy global -> shared through a tensor map (single destination CTA): the box whose first element has
 // coordinates (x, y) -- x along the contiguous dimension, x*4 bytes a multiple of 16 -- lands densely packed at dst
 // (128-byte aligned); out-of-range elements are written as zeros and count towards the transferred bytes.
 __device__ __forceinline__ void bulk_tensor_2d_g2s(void* dst, const void* tmap, int x, int y, uint64_t* bar, uint64_t policy) {

@@ -4,8 +4,8 @@
 // the contiguous slice of CW = ceil(n/4/16) 16-byte column groups starting at w*CW.  The CTA walks batches of RB
 // rows (batch g belongs to CTA g mod grid).  As in the narrow-row kernel each warp runs its own asynchronous
 // pipeline with `depth` private stages completing on its own mbarriers; a stage is one RB-row by CW-group box of X,
-// fetched by the warp's elected lane with ONE tiled TMA copy (cp.async.bulk.tensor.2d through a tensor map of X;
-// no multicast).  Rows past m and columns past n arrive as zeros, so the loads need no bounds logic.
+// fetched by the warp's elected lane with ONE tiled TMA copy (cp.async.bulk.tensor.2d through a tensor map of X,
+// delivered to this CTA only).  Rows past m and columns past n arrive as zeros, so the loads need no bounds logic.
 // Per batch:
 //   1. every warp moves its box into registers (conflict-free 128-bit shared loads), re-arms the stage, and forms
 //      its partial dot products (lane FMAs + transposing shuffle reduction);
