@@ -50,9 +50,14 @@ def measured_hbm_peak():
 
 
 class ClockSampler:
-    """Samples nvidia-smi clocks and throttle reasons in the background (200 ms period)."""
-    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
-         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+    """Samples nvidia-smi clocks and throttle reasons in the background (100 ms period).
+
+    Every sample carries nvidia-smi's own timestamp; `stop(t0, t1)` keeps the samples taken between the two wall-clock
+    times (the timed region), so the sampler can be started early and its start-up time does not eat the region.
+    """
+    Q = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+    NAMES = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
 
     def __init__(self, gpu_uuid):
         if not gpu_uuid.startswith("GPU-"):
@@ -65,10 +70,50 @@ class ClockSampler:
         except Exception:
             self.p = None
 
-    def stop(self):
-        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+    def wait_first_sample(self, limit_s=5.0):
+        """Blocks until nvidia-smi has written its first line (or the limit passes)."""
+        t_end = time.time() + limit_s
+        while self.p is not None and time.time() < t_end:
+            if os.path.getsize(self.f.name) > 0:
+                return True
+            time.sleep(0.05)
+        return False
+
+    @staticmethod
+    def parse(text, t0=None, t1=None):
+        """Samples of `text` (nvidia-smi csv lines) whose timestamp lies in [t0, t1] (all of them if t0 is None)."""
+        import datetime
+        rows = []
+        for line in text.splitlines():
+            t = [x.strip() for x in line.split(",")]
+            if len(t) < 8:
+                continue
+            try:
+                ts = datetime.datetime.strptime(t[0], "%Y/%m/%d %H:%M:%S.%f").timestamp()
+                row = (ts, float(t[1]), float(t[2]), float(t[3]), t[4:8])
+            except ValueError:
+                continue
+            if t0 is None or (t0 <= ts <= t1):
+                rows.append(row)
+        return rows
+
+    @classmethod
+    def summarise(cls, rows, in_region):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": len(rows), "in_timed_region": in_region}
+        if rows:
+            reasons = set()
+            for r in rows:
+                for name, v in zip(cls.NAMES, r[4]):
+                    if v == "Active":
+                        reasons.add(name)
+            out.update(sm_mhz=statistics.median(r[1] for r in rows), sm_max_mhz=max(r[2] for r in rows),
+                       reasons=sorted(reasons), power_w_max=max(r[3] for r in rows))
+        return out
+
+    def stop(self, t0, t1):
+        """Ends the sampler; summarises the samples taken in the wall-clock window [t0, t1] (time.time() values)."""
         if self.p is None:
-            return out
+            return self.summarise([], True)
         self.p.terminate()
         try:
             self.p.wait(timeout=5)
@@ -76,27 +121,14 @@ class ClockSampler:
             self.p.kill()
         self.f.flush()
         self.f.seek(0)
-        sm, mx, pw, reasons = [], [], [], set()
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for line in self.f.read().splitlines():
-            t = [x.strip() for x in line.split(",")]
-            if len(t) < 7:
-                continue
-            try:
-                sm.append(float(t[0])); mx.append(float(t[1])); pw.append(float(t[2]))
-            except ValueError:
-                continue
-            for name, v in zip(names, t[3:7]):
-                if v == "Active":
-                    reasons.add(name)
+        text = self.f.read()
         self.f.close()
         os.unlink(self.f.name)
-        if sm:
-            # samples under load: upper half of the observed clocks (idle samples before/after pull the median down)
-            busy = sorted(sm)[len(sm) // 2:]
-            out = {"sm_mhz": statistics.median(busy), "sm_max_mhz": max(mx), "reasons": sorted(reasons),
-                   "samples": len(sm), "power_w_max": max(pw)}
-        return out
+        rows = self.parse(text, t0, t1)
+        if rows:
+            return self.summarise(rows, True)
+        # a region shorter than the sampling period: fall back to the samples nearest to it (within half a second)
+        return self.summarise(self.parse(text, t0 - 0.5, t1 + 0.5), False)
 
 
 def oracle_rate(X, y, wl, budget_s, max_rows=None):
@@ -289,26 +321,29 @@ def main():
             parallel.fit_sharded_cuda(ctx, dX, dy, m_total, wl.lr, k, w, b)
 
     # ---- device-resident timing ----
+    sampler = ClockSampler(str(torch.cuda.get_device_properties(local_rank).uuid)) if rank == 0 else None
     run_steps(args.warmup)
     torch.cuda.synchronize()
+    if sampler:
+        sampler.wait_first_sample()                 # nvidia-smi takes a second or so to come up
     if world > 1:
         dist.barrier()
-    sampler = ClockSampler(str(torch.cuda.get_device_properties(local_rank).uuid)) if rank == 0 else None
-    time.sleep(0.25)
     launches0 = ctx.launch_count()
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     torch.cuda.synchronize()
+    wall0 = time.time()
     ev0.record()
     run_steps(args.steps)
     ev1.record()
     torch.cuda.synchronize()
+    wall1 = time.time()
     ms = ev0.elapsed_time(ev1)
     if world > 1:
         dist.barrier()
         t = torch.tensor([ms], dtype=torch.float64, device="cuda")
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
         ms = float(t.item())
-    clocks = sampler.stop() if sampler else None
+    clocks = sampler.stop(wall0, wall1) if sampler else None
     launches = ctx.launch_count() - launches0
     status = ctx.device_status()
     if status != 0:
