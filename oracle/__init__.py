@@ -42,6 +42,7 @@ def _load():
         lib.oracle_fit_sgd.argtypes = [P, P, I64, I32, D, I64, I32, I64, P, P, P]
         lib.oracle_fit_tol.argtypes = [P, P, I64, I32, D, D, I32, P, P, P, P, P, P]
         lib.oracle_f1.argtypes = [P, P, I64, P, P, P, P]
+        lib.oracle_round_bf16.argtypes = [P, I64, P, P]
         _lib = lib
     return _lib
 
@@ -182,3 +183,18 @@ def f1_score(labels, y):
     if rc != 0:
         raise ValueError("oracle_f1: bad arguments")
     return f1.value, tp.value, fp.value, fn.value
+
+
+def round_bf16(x):
+    """Rounds fp32 values to bfloat16 (round to nearest, ties to even).
+
+    Returns ``(bits, values)``: the uint16 patterns and the same numbers widened back to fp32, both shaped like ``x``.
+    The other routines of this module take ``values`` wherever the CUDA path is given the bfloat16 matrix.
+    """
+    x = _f32(x)
+    bits = np.zeros(x.shape, dtype=np.uint16)
+    values = np.zeros(x.shape, dtype=np.float32)
+    rc = _load().oracle_round_bf16(_ptr(x), x.size, _ptr(bits), _ptr(values))
+    if rc != 0:
+        raise ValueError("oracle_round_bf16: bad arguments")
+    return bits, values

@@ -260,3 +260,52 @@ int oracle_f1(const uint8_t* labels, const float* y, int64_t m, int64_t* tp, int
     *f1 = a > 0 ? (2.0 * (double)a) / (2.0 * (double)a + (double)c + (double)d) : 0.0;
     return 0;
 }
+
+/*
+ * Rounding of binary32 values to the bfloat16 format (the reduced-precision storage variant of X; the paper
+ * itself does not discuss storage precision).  bfloat16 is the upper half of binary32: 1 sign bit, the same 8
+ * exponent bits, the top 7 fraction bits; a pattern h stands for the binary32 value with bits h << 16.
+ * Rounding is IEEE 754 roundTiesToEven, written out as the definition: the two neighbouring bfloat16 values
+ * (the truncated pattern and the next pattern away from zero) are decoded to double, the nearer one wins, and an
+ * exact tie goes to the pattern whose last bit is 0.  The pattern past the largest finite value counts as
+ * 2^128 for the distance and yields infinity.  NaN maps to a quiet NaN of the same sign; infinities and zeros
+ * keep their sign.
+ * Pins (tests, CPU only): hand-worked patterns in tests/golden/bf16_rounding_cases.txt, identity on all 65,536
+ * patterns, a library conversion on random and special values, the half-spacing error bound and monotonicity.
+ */
+static double bf16_pattern_magnitude(uint32_t h15) {         /* h15 = pattern without its sign bit */
+    uint32_t e = h15 >> 7, f = h15 & 0x7fu;
+    if (e == 0) return ldexp((double)f / 128.0, -126);       /* subnormal (and zero) */
+    return ldexp(1.0 + (double)f / 128.0, (int)e - 127);     /* e == 255, f == 0 gives 2^128: the overflow threshold */
+}
+
+int oracle_round_bf16(const float* x, int64_t count, uint16_t* bits_out, float* values_out) {
+    if (!x || count < 0 || (!bits_out && !values_out)) return -1;
+#pragma omp parallel for schedule(static)
+    for (int64_t i = 0; i < count; ++i) {
+        uint32_t u;
+        memcpy(&u, &x[i], 4);
+        uint32_t sign = u >> 31, mag = u & 0x7fffffffu;
+        uint32_t h15;
+        if (mag > 0x7f800000u) {
+            h15 = 0x7fc0u;                                   /* NaN -> quiet NaN */
+        } else if (mag == 0x7f800000u) {
+            h15 = 0x7f80u;                                   /* infinity */
+        } else {
+            uint32_t lo = mag >> 16, hi = lo + 1u;           /* neighbours: towards zero, away from zero */
+            double v = fabs((double)x[i]);
+            double d_lo = v - bf16_pattern_magnitude(lo);
+            double d_hi = bf16_pattern_magnitude(hi) - v;
+            if (d_lo < d_hi) h15 = lo;
+            else if (d_hi < d_lo) h15 = hi;
+            else h15 = (lo & 1u) ? hi : lo;                  /* tie: the even pattern */
+        }
+        uint16_t h = (uint16_t)((sign << 15) | h15);
+        if (bits_out) bits_out[i] = h;
+        if (values_out) {
+            uint32_t w = (uint32_t)h << 16;
+            memcpy(&values_out[i], &w, 4);
+        }
+    }
+    return 0;
+}
