@@ -193,12 +193,13 @@ def f1_score(labels, y):
     return (2.0 * tp / (2.0 * tp + fp + fn)) if tp > 0 else 0.0, tp, fp, fn
 
 
-def workload_config(wl, n_gpus):
-    return {"workload": f"{wl.name}: m={wl.m} x n={wl.n} fp32 row-major, lr={wl.lr}, {wl.iters} iterations"
+def workload_config(wl, n_gpus, x_dtype="f32"):
+    eb = 2 if x_dtype == "bf16" else 4
+    return {"workload": f"{wl.name}: m={wl.m} x n={wl.n} {'bfloat16-stored' if eb == 2 else 'fp32'} row-major, lr={wl.lr}, {wl.iters} iterations"
                         + (f" (per GPU; {n_gpus} row shards)" if n_gpus > 1 else ""),
             "m": wl.m, "n": wl.n, "lr": wl.lr, "iters": wl.iters,
-            "l2": f"no flush needed: X is {wl.m * wl.n * 4 / 1e6:.0f} MB per pass against 126 MB of L2"
-                  if wl.m * wl.n * 4 > 4 * 126e6 else "X fits in L2: the pass is launch/L2-bound, not HBM-bound",
+            "l2": f"no flush needed: X is {wl.m * wl.n * eb / 1e6:.0f} MB per pass against 126 MB of L2"
+                  if wl.m * wl.n * eb > 4 * 126e6 else "X fits in L2: the pass is launch/L2-bound, not HBM-bound",
             "parallelism": "single GPU" if n_gpus == 1 else f"dp{n_gpus} row-sharded, all-gather of n+2 fp64 sums per iteration"}
 
 
@@ -260,6 +261,9 @@ def main():
     ap.add_argument("--tol", default="", help="ALPHA,EPS: time-to-tolerance mode (Algorithm 7 stopping rule); --steps caps the updates")
     ap.add_argument("--no-persistent", action="store_true", help="force two kernels per iteration in lr_fit")
     ap.add_argument("--l2-keep-mb", type=float, default=-1.0, help="MB of X to keep in L2 across iterations (-1: library default, 0: off)")
+    ap.add_argument("--x-dtype", default="f32", choices=["f32", "bf16"],
+                    help="storage type of X on the device: bf16 runs the bfloat16 entry points on lr_convert_bf16's output "
+                         "(half the bytes per pass; no end-to-end or CPU leg)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
@@ -313,6 +317,16 @@ def main():
     w = torch.zeros(wl.n, dtype=torch.float32, device="cuda")
     b = torch.zeros(1, dtype=torch.float32, device="cuda")
     m_total = wl.m * world
+    bf16 = args.x_dtype == "bf16"
+    if bf16:
+        if world > 1:
+            raise SystemExit("--x-dtype bf16 is a single-GPU mode")
+        dX32 = dX
+        dX = ctx.convert_bf16(dX32)                 # the fits below read the bfloat16 matrix only
+        torch.cuda.synchronize()
+        del dX32
+        args.no_e2e = args.no_cpu_baseline = True
+    elem_bytes = 2 if bf16 else 4
 
     def run_steps(k):
         if world == 1:
@@ -369,12 +383,12 @@ def main():
     n_l, tot_ms = ctx.profile_read()
     ctx.profile_enable(False)
     k1_ms = tot_ms / max(n_l, 1)
-    bytes_per_launch = 4 * wl.m * wl.n + 4 * wl.m
+    bytes_per_launch = elem_bytes * wl.m * wl.n + 4 * wl.m
     achieved = bytes_per_launch / (k1_ms * 1e-3) / 1e9
     peak, peak_kind = measured_hbm_peak()
-    plan = api.plan_query(wl.m, wl.n, sm_count=torch.cuda.get_device_properties(local_rank).multi_processor_count)
+    plan = api.plan_query(wl.m, wl.n, sm_count=torch.cuda.get_device_properties(local_rank).multi_processor_count, bf16=bf16)
     pass_kernel = {0: "k_stream_rows", 1: "k_stream_split", 2: "k_generic"}[plan["variant"]]
-    per_row = NCU_TRAFFIC_BYTES_PER_ROW.get(args.workload, {})
+    per_row = NCU_TRAFFIC_BYTES_PER_ROW.get(args.workload + ("_bf16" if bf16 else ""), {})
     single_pass = {"kernel": f"{pass_kernel} (one fused loss/gradient pass, two-kernel form of lr_fit)", "achieved": achieved,
                    "unit": "GB/s", "frac": achieved / peak, "bytes_per_launch": bytes_per_launch, "avg_launch_ms": k1_ms,
                    "launches_timed": n_l, "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
@@ -423,7 +437,7 @@ def main():
         p_ms = pe0.elapsed_time(pe1) / 10
         f1, tp, fp, fn = f1_score(labels.cpu().numpy(), y_np)
         predict = {"thr": wl.predict_thr, "f1_vs_y": f1, "tp": tp, "fp": fp, "fn": fn, "ms_per_predict": p_ms,
-                   "gbs": (4 * wl.m * wl.n + wl.m) / (p_ms * 1e-3) / 1e9, "after_iterations": wl.iters}
+                   "gbs": (elem_bytes * wl.m * wl.n + wl.m) / (p_ms * 1e-3) / 1e9, "after_iterations": wl.iters}
 
     # ---- CPU checker on this host's cores (reported baseline, not a target) ----
     cpu = None
@@ -433,7 +447,7 @@ def main():
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-            "dtype": "f32", "data": "synthetic", "config": workload_config(wl, world),
+            "dtype": "f32", "x_storage": args.x_dtype, "data": "synthetic", "config": workload_config(wl, world, args.x_dtype),
             "achieved_hbm_gbs_whole_step": bytes_per_launch * world * args.steps / (ms * 1e-3) / 1e9,
             "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches, "clocks": clocks,
             "predict": predict}

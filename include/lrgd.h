@@ -39,7 +39,7 @@ enum {
     LR_OK = 0,
     LR_ERR_NULL = -1,       /* a required pointer is NULL */
     LR_ERR_SHAPE = -2,      /* m < 1, n < 1, n > n_max of the ctx, iters < 0, m too large */
-    LR_ERR_ALIGNMENT = -3,  /* a float pointer is not 4-byte aligned */
+    LR_ERR_ALIGNMENT = -3,  /* a float pointer is not 4-byte aligned (a bfloat16 pointer: 2-byte) */
     LR_ERR_VALUE = -4,      /* thr outside (0,1), lr not finite */
     LR_ERR_CUDA = -5,       /* a CUDA runtime call failed; see lr_last_cuda_error */
     LR_ERR_TIMEOUT = -6,    /* a bounded device-side wait expired (reported by lr_last_device_status) */
@@ -172,6 +172,30 @@ int lr_fit_sgd(lr_ctx* ctx, const float* d_X, const float* d_y, int64_t m, int32
  */
 int lr_predict(lr_ctx* ctx, const float* d_X, int64_t m, int32_t n,
                const float* d_w, const float* d_b, float thr, uint8_t* d_labels, void* stream);
+
+/*
+ * bfloat16 storage of X (not in the paper, which is silent on storage precision; it halves the bytes the pass has to
+ * stream).  d_Xh is a DEVICE array of m*n bfloat16 patterns (uint16: the upper half of a binary32 pattern), row-major
+ * with leading dimension n, 2-byte aligned.  Only X changes: y, w, b, the gradient and every sum stay as in the fp32
+ * calls, each element of X is widened exactly to fp32 when it is used, so the three calls below compute exactly what
+ * lr_loss_grad / lr_fit / lr_predict would compute on the fp32 matrix holding the same (bfloat16-representable) values.
+ * The staged kernels take rows of n % 8 == 0 columns with d_Xh 16-byte aligned, up to n = 8192; other shapes run on the
+ * unstaged kernel.  lr_fit_bf16 uses the single persistent launch for n <= 512, like lr_fit.  Errors as the fp32 calls.
+ *
+ * lr_convert_bf16 rounds `count` fp32 values to bfloat16 (round to nearest, ties to even; NaN stays NaN, values past
+ * the largest finite bfloat16 become infinity) -- one elementwise kernel on `stream`; d_X and d_Xh must not overlap.
+ * count == 0 is a no-op.
+ * lr_plan_query_bf16 is lr_plan_query for a bfloat16 matrix (lanes and groups then count 8 columns per 16 bytes).
+ */
+int lr_convert_bf16(lr_ctx* ctx, const float* d_X, int64_t count, uint16_t* d_Xh, void* stream);
+int lr_loss_grad_bf16(lr_ctx* ctx, const uint16_t* d_Xh, const float* d_y, int64_t m, int32_t n,
+                      const float* d_w, const float* d_b,
+                      float* d_loss, float* d_grad_w, float* d_grad_b, void* stream);
+int lr_fit_bf16(lr_ctx* ctx, const uint16_t* d_Xh, const float* d_y, int64_t m, int32_t n,
+                float lr, int32_t iters, float* d_w, float* d_b, float* d_loss_hist, void* stream);
+int lr_predict_bf16(lr_ctx* ctx, const uint16_t* d_Xh, int64_t m, int32_t n,
+                    const float* d_w, const float* d_b, float thr, uint8_t* d_labels, void* stream);
+int lr_plan_query_bf16(int64_t m, int32_t n, int32_t x_aligned16, int32_t sm_count, lr_plan* out);
 
 /*
  * Row-sharded data parallelism (the natural split of Algorithm 1's sums over rows; the paper itself

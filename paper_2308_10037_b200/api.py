@@ -21,7 +21,8 @@ LR_ERR_NULL, LR_ERR_SHAPE, LR_ERR_ALIGNMENT, LR_ERR_VALUE, LR_ERR_CUDA, LR_ERR_T
 EXPORTS = ["lr_plan_query", "lr_create", "lr_destroy", "lr_loss_grad", "lr_fit", "lr_predict", "lr_shard_sums",
            "lr_apply_sums", "lr_fit_host",
            "lr_predict_host", "lr_profile_enable", "lr_profile_read", "lr_launch_count", "lr_last_device_status",
-           "lr_last_cuda_error", "lr_status_string", "lr_loss_grad_noalloc", "lr_fit_tol", "lr_fit_opt", "lr_selftest_wait", "lr_set_persistent", "lr_fit_sgd", "lr_set_l2_keep"]
+           "lr_last_cuda_error", "lr_status_string", "lr_loss_grad_noalloc", "lr_fit_tol", "lr_fit_opt", "lr_selftest_wait", "lr_set_persistent", "lr_fit_sgd", "lr_set_l2_keep",
+           "lr_convert_bf16", "lr_loss_grad_bf16", "lr_fit_bf16", "lr_predict_bf16", "lr_plan_query_bf16"]
 
 
 class LrPlan(ctypes.Structure):
@@ -61,6 +62,11 @@ def lib() -> ctypes.CDLL:
         L.lr_fit.argtypes = [P, P, P, I64, I32, F, I32, P, P, P, P]
         L.lr_predict.argtypes = [P, P, I64, I32, P, P, F, P, P]
         L.lr_shard_sums.argtypes = [P, P, P, I64, I32, P, P, P, P]
+        L.lr_convert_bf16.argtypes = [P, P, I64, P, P]
+        L.lr_loss_grad_bf16.argtypes = L.lr_loss_grad.argtypes
+        L.lr_fit_bf16.argtypes = L.lr_fit.argtypes
+        L.lr_predict_bf16.argtypes = L.lr_predict.argtypes
+        L.lr_plan_query_bf16.argtypes = L.lr_plan_query.argtypes
         L.lr_apply_sums.argtypes = [P, P, I32, I64, I32, F, P, P, P, P]
         L.lr_fit_tol.argtypes = [P, P, P, I64, I32, F, F, I32, I32, P, P, P, P, ctypes.POINTER(I32),
                                  ctypes.POINTER(F), P]
@@ -90,10 +96,11 @@ def status_string(code: int) -> str:
     return lib().lr_status_string(int(code)).decode()
 
 
-def plan_query(m: int, n: int, x_aligned16: bool = True, sm_count: int = 148) -> dict:
-    """Host-only view of the launch plan for an m-by-n problem (no CUDA call)."""
+def plan_query(m: int, n: int, x_aligned16: bool = True, sm_count: int = 148, bf16: bool = False) -> dict:
+    """Host-only view of the launch plan for an m-by-n problem (no CUDA call); ``bf16``: X stored as bfloat16."""
     p = LrPlan()
-    rc = lib().lr_plan_query(int(m), int(n), int(bool(x_aligned16)), int(sm_count), ctypes.byref(p))
+    fn = lib().lr_plan_query_bf16 if bf16 else lib().lr_plan_query
+    rc = fn(int(m), int(n), int(bool(x_aligned16)), int(sm_count), ctypes.byref(p))
     if rc != LR_OK:
         raise LrError(rc, "lr_plan_query")
     return p.as_dict()
@@ -152,25 +159,42 @@ class Context:
         return ctypes.c_void_p(torch.cuda.current_stream(self.device).cuda_stream)
 
     # ---- device-pointer entry points -------------------------------------------------------------
+    # X may be a float32 tensor (lr_loss_grad / lr_fit / lr_predict) or a bfloat16 tensor (the *_bf16 entry points).
+    @staticmethod
+    def _x_kind(X):
+        if isinstance(X, torch.Tensor) and X.dtype == torch.bfloat16:
+            return torch.bfloat16, "_bf16"
+        return torch.float32, ""
+
+    def convert_bf16(self, X, out=None):
+        """Rounds a float32 CUDA tensor to bfloat16 (nearest, ties to even) with the library's kernel."""
+        Xh = torch.empty(X.shape, dtype=torch.bfloat16, device=X.device) if out is None else out
+        rc = lib().lr_convert_bf16(self._h, _dev_ptr(X, torch.float32, "X"), X.numel(), _dev_ptr(Xh, torch.bfloat16, "Xh"),
+                                   self._stream())
+        self._check(rc, "lr_convert_bf16")
+        return Xh
+
     def loss_grad(self, X, y, w, b):
         m, n = X.shape
+        xdt, sfx = self._x_kind(X)
         loss = torch.empty(1, dtype=torch.float32, device=X.device)
         gw = torch.empty(n, dtype=torch.float32, device=X.device)
         gb = torch.empty(1, dtype=torch.float32, device=X.device)
-        rc = lib().lr_loss_grad(self._h, _dev_ptr(X, torch.float32, "X"), _dev_ptr(y, torch.float32, "y"), m, n,
+        rc = getattr(lib(), "lr_loss_grad" + sfx)(self._h, _dev_ptr(X, xdt, "X"), _dev_ptr(y, torch.float32, "y"), m, n,
                                 _dev_ptr(w, torch.float32, "w"), _dev_ptr(b, torch.float32, "b"),
                                 _dev_ptr(loss, torch.float32, "loss"), _dev_ptr(gw, torch.float32, "grad_w"),
                                 _dev_ptr(gb, torch.float32, "grad_b"), self._stream())
-        self._check(rc, "lr_loss_grad")
+        self._check(rc, "lr_loss_grad" + sfx)
         return loss, gw, gb
 
     def fit(self, X, y, lr, iters, w, b, loss_hist=None):
         """In place on ``w`` [n] and ``b`` [1]; ``loss_hist`` is None or a float32 CUDA tensor [iters]."""
         m, n = X.shape
-        rc = lib().lr_fit(self._h, _dev_ptr(X, torch.float32, "X"), _dev_ptr(y, torch.float32, "y"), m, n, float(lr),
+        xdt, sfx = self._x_kind(X)
+        rc = getattr(lib(), "lr_fit" + sfx)(self._h, _dev_ptr(X, xdt, "X"), _dev_ptr(y, torch.float32, "y"), m, n, float(lr),
                           int(iters), _dev_ptr(w, torch.float32, "w"), _dev_ptr(b, torch.float32, "b"),
                           _dev_ptr(loss_hist, torch.float32, "loss_hist"), self._stream())
-        self._check(rc, "lr_fit")
+        self._check(rc, "lr_fit" + sfx)
 
     def fit_tol(self, X, y, lr, eps, max_iters, w, b, check_every=16, loss_hist=None, gnorm_hist=None):
         """GD until ||grad||_2 <= eps (at most ``max_iters`` updates), in place on w, b.  Returns (updates, last norm)."""
@@ -205,10 +229,11 @@ class Context:
     def predict(self, X, w, b, thr, out=None):
         m, n = X.shape
         labels = torch.empty(m, dtype=torch.uint8, device=X.device) if out is None else out
-        rc = lib().lr_predict(self._h, _dev_ptr(X, torch.float32, "X"), m, n, _dev_ptr(w, torch.float32, "w"),
+        xdt, sfx = self._x_kind(X)
+        rc = getattr(lib(), "lr_predict" + sfx)(self._h, _dev_ptr(X, xdt, "X"), m, n, _dev_ptr(w, torch.float32, "w"),
                               _dev_ptr(b, torch.float32, "b"), float(thr), _dev_ptr(labels, torch.uint8, "labels"),
                               self._stream())
-        self._check(rc, "lr_predict")
+        self._check(rc, "lr_predict" + sfx)
         return labels
 
     def shard_sums(self, X, y, w, b, sums):

@@ -9,6 +9,7 @@
 #include <new>
 #include <vector>
 
+#include "lrgd_convert.cuh"
 #include "lrgd_fit_rows.cuh"
 #include "lrgd_generic.cuh"
 #include "lrgd_reduce.cuh"
@@ -37,29 +38,32 @@ constexpr int64_t kMaxRows = int64_t(1) << 40;
 
 struct RowShape { int nv, lpr, rb; };
 
-// Which instantiation of the staged kernel covers n4 = n/4 column groups per row.
-bool row_shape_for(int n4, RowShape* s) {
-    if (n4 <= 8) *s = {1, 8, 8};
-    else if (n4 <= 16) *s = {1, 16, 8};
-    else if (n4 <= 32) *s = {1, 32, LRGD_NV1_RB};
-    else if (n4 <= 64) *s = {2, 32, LRGD_NV2_RB};
-    else if (n4 <= 128) *s = {4, 32, 2};
+// Which instantiation of the narrow-row kernel covers ng 16-byte column groups per row.  bfloat16 rows stop at 64
+// groups: a lane that owns four groups of eight columns would need more registers than a 512-thread CTA can give.
+bool row_shape_for(int ng, bool bf16, RowShape* s) {
+    if (ng <= 8) *s = {1, 8, 8};
+    else if (ng <= 16) *s = {1, 16, 8};
+    else if (ng <= 32) *s = {1, 32, LRGD_NV1_RB};
+    else if (ng <= 64) *s = {2, 32, LRGD_NV2_RB};
+    else if (ng <= 128 && !bf16) *s = {4, 32, 2};
     else return false;
     return true;
 }
 
-int make_plan(int64_t m, int32_t n, bool aligned16, int32_t sms, lr_plan* P) {
+// bf16: X holds bfloat16 (2-byte) elements instead of fp32; a 16-byte group is then 8 columns instead of 4.
+int make_plan(int64_t m, int32_t n, bool aligned16, int32_t sms, lr_plan* P, bool bf16 = false) {
     if (!P) return LR_ERR_NULL;
     if (m < 1 || m > kMaxRows || n < 1 || sms < 1) return LR_ERR_SHAPE;
     std::memset(P, 0, sizeof(*P));
+    const int epg = bf16 ? 8 : 4, eb = bf16 ? 2 : 4;
     RowShape rs;
-    if (aligned16 && n % 4 == 0 && row_shape_for(n / 4, &rs)) {
+    if (aligned16 && n % epg == 0 && row_shape_for(n / epg, bf16, &rs)) {
         const int rpb = rs.rb * (32 / rs.lpr);                                  // rows per batch = rows per stage
         const int64_t B = (m + rpb - 1) / rpb;                                  // batches
         const int64_t slots = (B + kNW - 1) / kNW;                              // CTA-level groups of kNW batches
         const int grid = int(std::min<int64_t>(slots, sms));
         const int64_t per_warp = (slots + grid - 1) / grid;                     // most batches any warp handles
-        const int64_t stage_stride = (int64_t(rpb) * n * 4 + 127) & ~int64_t(127);
+        const int64_t stage_stride = (int64_t(rpb) * n * eb + 127) & ~int64_t(127);
         int D = int(std::min<int64_t>(kMaxDepth, kStageBudgetBytes / (kNW * stage_stride)));
         D = int(std::min<int64_t>(D, per_warp));
         if (D < 1) D = 1;
@@ -76,9 +80,9 @@ int make_plan(int64_t m, int32_t n, bool aligned16, int32_t sms, lr_plan* P) {
         if (per_warp >= (int64_t(1) << 31)) return LR_ERR_SHAPE;
         return LR_OK;
     }
-    if (aligned16 && n % 4 == 0 && n / 4 <= kNW * 64 && m < (int64_t(1) << 31) - 65536) {   // TMA coordinates are int32
+    if (aligned16 && n % epg == 0 && n / epg <= kNW * 64 && m < (int64_t(1) << 31) - 65536) {   // TMA coordinates are int32
         // wide rows: the warps of a CTA split each row by columns
-        const int cw = (n / 4 + kNW - 1) / kNW;                                 // 16-byte column groups per warp slice
+        const int cw = (n / epg + kNW - 1) / kNW;                               // 16-byte column groups per warp slice
         const int nv = cw > 32 ? 2 : 1;
         const int rb = nv == 2 ? 4 : 8;
         const int64_t B = (m + rb - 1) / rb;
@@ -170,9 +174,9 @@ struct DeviceGuard {
 
 bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
 
-template <int NV, int LPR, int RB, bool PRED>
+template <class E, int NV, int LPR, int RB, bool PRED>
 cudaError_t launch_rows_t(const lr_plan& P, const StreamParams& sp, cudaStream_t st) {
-    auto kern = k_stream_rows<NV, LPR, RB, kNW, PRED>;
+    auto kern = k_stream_rows<E, NV, LPR, RB, kNW, PRED>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, P.smem_bytes);
     if (e != cudaSuccess) return e;
     kern<<<P.grid, P.threads, P.smem_bytes, st>>>(sp);
@@ -180,21 +184,30 @@ cudaError_t launch_rows_t(const lr_plan& P, const StreamParams& sp, cudaStream_t
 }
 
 template <bool PRED>
-cudaError_t launch_rows(const lr_plan& P, const StreamParams& sp, cudaStream_t st) {
-    if (P.lanes_per_row == 8) return launch_rows_t<1, 8, 8, PRED>(P, sp, st);
-    if (P.lanes_per_row == 16) return launch_rows_t<1, 16, 8, PRED>(P, sp, st);
-    if (P.vec_per_lane == 1) return launch_rows_t<1, 32, LRGD_NV1_RB, PRED>(P, sp, st);
-    if (P.vec_per_lane == 2) return launch_rows_t<2, 32, LRGD_NV2_RB, PRED>(P, sp, st);
-    return launch_rows_t<4, 32, 2, PRED>(P, sp, st);
+cudaError_t launch_rows(const lr_plan& P, const StreamParams& sp, cudaStream_t st, bool bf16 = false) {
+    if (bf16) {
+        if (P.lanes_per_row == 8) return launch_rows_t<ElemBF16, 1, 8, 8, PRED>(P, sp, st);
+        if (P.lanes_per_row == 16) return launch_rows_t<ElemBF16, 1, 16, 8, PRED>(P, sp, st);
+        if (P.vec_per_lane == 1) return launch_rows_t<ElemBF16, 1, 32, LRGD_NV1_RB, PRED>(P, sp, st);
+        if (P.vec_per_lane == 2) return launch_rows_t<ElemBF16, 2, 32, LRGD_NV2_RB, PRED>(P, sp, st);
+        return cudaErrorInvalidValue;              // the plan never asks for four bfloat16 groups per lane
+    }
+    if (P.lanes_per_row == 8) return launch_rows_t<ElemF32, 1, 8, 8, PRED>(P, sp, st);
+    if (P.lanes_per_row == 16) return launch_rows_t<ElemF32, 1, 16, 8, PRED>(P, sp, st);
+    if (P.vec_per_lane == 1) return launch_rows_t<ElemF32, 1, 32, LRGD_NV1_RB, PRED>(P, sp, st);
+    if (P.vec_per_lane == 2) return launch_rows_t<ElemF32, 2, 32, LRGD_NV2_RB, PRED>(P, sp, st);
+    return launch_rows_t<ElemF32, 4, 32, 2, PRED>(P, sp, st);
 }
 
-// Tensor map of X for the wide-row kernel: fp32 [m][n] row-major, box = cw*4 floats by rb rows, zero fill outside.
+// Tensor map of X for the wide-row kernel: [m][n] row-major, box = cw 16-byte groups by rb rows, zero fill outside.
+// The copy moves bytes untouched, and a box may span at most 256 elements per dimension, so a bfloat16 matrix is
+// described as 32-bit words (n/2 per row): the widest slice, 64 groups, is then 256 elements for either storage type.
 // The encoder is a driver entry point, resolved at run time so that the library links against the runtime only.
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
                                   const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
-cudaError_t make_x_tensor_map(const float* X, int64_t m, int32_t n, int cw, int rb, CUtensorMap* out) {
+cudaError_t make_x_tensor_map(const void* X, bool bf16, int64_t m, int32_t n, int cw, int rb, CUtensorMap* out) {
     static EncodeTiledFn encode = nullptr;
     if (!encode) {
         void* fn = nullptr;
@@ -204,19 +217,21 @@ cudaError_t make_x_tensor_map(const float* X, int64_t m, int32_t n, int cw, int 
         if (q != cudaDriverEntryPointSuccess || !fn) return cudaErrorNotSupported;
         encode = reinterpret_cast<EncodeTiledFn>(fn);
     }
-    const cuuint64_t dims[2] = {cuuint64_t(n), cuuint64_t(m)};
-    const cuuint64_t strides[1] = {cuuint64_t(n) * 4};
+    const cuuint64_t words = bf16 ? cuuint64_t(n) / 2 : cuuint64_t(n);            // 32-bit words per row
+    const cuuint64_t dims[2] = {words, cuuint64_t(m)};
+    const cuuint64_t strides[1] = {words * 4};
     const cuuint32_t box[2] = {cuuint32_t(cw) * 4, cuuint32_t(rb)};
     const cuuint32_t estr[2] = {1, 1};
-    CUresult r = encode(out, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float*>(X), dims, strides, box, estr,
+    CUresult r = encode(out, bf16 ? CU_TENSOR_MAP_DATA_TYPE_UINT32 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2,
+                        const_cast<void*>(X), dims, strides, box, estr,
                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
 }
 
-template <int NV, int RB, bool PRED>
+template <class E, int NV, int RB, bool PRED>
 cudaError_t launch_split_t(const lr_plan& P, const CUtensorMap& tm, const SplitParams& sp, cudaStream_t st) {
-    auto kern = k_stream_split<NV, RB, kNW, PRED>;
+    auto kern = k_stream_split<E, NV, RB, kNW, PRED>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, P.smem_bytes);
     if (e != cudaSuccess) return e;
     kern<<<P.grid, P.threads, P.smem_bytes, st>>>(tm, sp);
@@ -224,42 +239,54 @@ cudaError_t launch_split_t(const lr_plan& P, const CUtensorMap& tm, const SplitP
 }
 
 template <bool PRED>
-cudaError_t launch_split(const lr_plan& P, const float* X, const SplitParams& sp, cudaStream_t st) {
+cudaError_t launch_split(const lr_plan& P, const void* X, const SplitParams& sp, cudaStream_t st, bool bf16 = false) {
     CUtensorMap tm;
-    cudaError_t e = make_x_tensor_map(X, sp.m, sp.n, sp.cw, P.rows_per_batch, &tm);
+    cudaError_t e = make_x_tensor_map(X, bf16, sp.m, sp.n, sp.cw, P.rows_per_batch, &tm);
     if (e != cudaSuccess) return e;
-    if (P.vec_per_lane == 2) return launch_split_t<2, 4, PRED>(P, tm, sp, st);
-    return launch_split_t<1, 8, PRED>(P, tm, sp, st);
+    if (bf16) {
+        if (P.vec_per_lane == 2) return launch_split_t<ElemBF16, 2, 4, PRED>(P, tm, sp, st);
+        return launch_split_t<ElemBF16, 1, 8, PRED>(P, tm, sp, st);
+    }
+    if (P.vec_per_lane == 2) return launch_split_t<ElemF32, 2, 4, PRED>(P, tm, sp, st);
+    return launch_split_t<ElemF32, 1, 8, PRED>(P, tm, sp, st);
 }
 
-template <int NV, int LPR, int RB>
+template <class E, int NV, int LPR, int RB>
 cudaError_t launch_fit_t(const lr_plan& P, int smem, FitParams& fp, cudaStream_t st) {
-    auto kern = k_fit_rows<NV, LPR, RB, kNW>;
+    auto kern = k_fit_rows<E, NV, LPR, RB, kNW>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
     void* args[] = {&fp};
     return cudaLaunchCooperativeKernel(reinterpret_cast<void*>(kern), dim3(P.grid), dim3(P.threads), args, size_t(smem), st);
 }
 
-cudaError_t launch_fit(const lr_plan& P, int smem, FitParams& fp, cudaStream_t st) {
-    if (P.lanes_per_row == 8) return launch_fit_t<1, 8, 8>(P, smem, fp, st);
-    if (P.lanes_per_row == 16) return launch_fit_t<1, 16, 8>(P, smem, fp, st);
-    if (P.vec_per_lane == 1) return launch_fit_t<1, 32, LRGD_NV1_RB>(P, smem, fp, st);
-    if (P.vec_per_lane == 2) return launch_fit_t<2, 32, LRGD_NV2_RB>(P, smem, fp, st);
-    return launch_fit_t<4, 32, 2>(P, smem, fp, st);
+cudaError_t launch_fit(const lr_plan& P, int smem, FitParams& fp, cudaStream_t st, bool bf16 = false) {
+    if (bf16) {
+        if (P.lanes_per_row == 8) return launch_fit_t<ElemBF16, 1, 8, 8>(P, smem, fp, st);
+        if (P.lanes_per_row == 16) return launch_fit_t<ElemBF16, 1, 16, 8>(P, smem, fp, st);
+        if (P.vec_per_lane == 1) return launch_fit_t<ElemBF16, 1, 32, LRGD_NV1_RB>(P, smem, fp, st);
+        if (P.vec_per_lane == 2) return launch_fit_t<ElemBF16, 2, 32, LRGD_NV2_RB>(P, smem, fp, st);
+        return cudaErrorInvalidValue;
+    }
+    if (P.lanes_per_row == 8) return launch_fit_t<ElemF32, 1, 8, 8>(P, smem, fp, st);
+    if (P.lanes_per_row == 16) return launch_fit_t<ElemF32, 1, 16, 8>(P, smem, fp, st);
+    if (P.vec_per_lane == 1) return launch_fit_t<ElemF32, 1, 32, LRGD_NV1_RB>(P, smem, fp, st);
+    if (P.vec_per_lane == 2) return launch_fit_t<ElemF32, 2, 32, LRGD_NV2_RB>(P, smem, fp, st);
+    return launch_fit_t<ElemF32, 4, 32, 2>(P, smem, fp, st);
 }
 
 // Rows of X to fetch with the evict-last hint.  Default: none for the narrow-row kernels (measured: any kept part slows
 // them down), three quarters of the L2 for the wide-row kernel (measured on 100k x 4096: 0.260 -> 0.231 ms per pass).
-int64_t keep_rows_for(const lr_ctx* ctx, int variant, int32_t n) {
+int64_t keep_rows_for(const lr_ctx* ctx, int variant, int32_t n, bool bf16 = false) {
     int64_t bytes = ctx->l2_keep_bytes;
     if (bytes < 0) bytes = variant == 1 ? ctx->l2_bytes / 4 * 3 : 0;
-    return bytes / (int64_t(n) * 4);
+    return bytes / (int64_t(n) * (bf16 ? 2 : 4));
 }
 
 struct Pass {
-    const float* X; const float* y; int64_t m; int32_t n; const float* w; const float* b;
+    const void* X; const float* y; int64_t m; int32_t n; const float* w; const float* b;
     const int* stop = nullptr;                      // device flag that turns the launch into a no-op once set
+    bool bf16 = false;                              // X holds bfloat16 elements instead of fp32
 };
 
 struct TolArgs {                                    // tolerance mode of the reduction
@@ -285,23 +312,28 @@ int launch_stream_pass(lr_ctx* ctx, const lr_plan& P, const Pass& a, uint8_t* la
         sp.partial = ctx->d_partial; sp.labels = labels; sp.cut = cut; sp.status = ctx->d_status; sp.stop = a.stop;
         sp.depth = P.stages;
         sp.num_batches = (a.m + P.rows_per_batch - 1) / P.rows_per_batch;
-        sp.keep_rows = keep_rows_for(ctx, 0, a.n);
-        e = predict ? launch_rows<true>(P, sp, st) : launch_rows<false>(P, sp, st);
+        sp.keep_rows = keep_rows_for(ctx, 0, a.n, a.bf16);
+        e = predict ? launch_rows<true>(P, sp, st, a.bf16) : launch_rows<false>(P, sp, st, a.bf16);
     } else if (P.variant == 1) {
         SplitParams sp{};
         sp.y = a.y; sp.m = a.m; sp.n = a.n; sp.w = a.w; sp.b = a.b;
         sp.partial = ctx->d_partial; sp.labels = labels; sp.cut = cut; sp.status = ctx->d_status; sp.stop = a.stop;
         sp.depth = P.stages;
-        sp.cw = (a.n / 4 + kNW - 1) / kNW;
+        sp.cw = (a.n / (a.bf16 ? 8 : 4) + kNW - 1) / kNW;
         sp.num_batches = (a.m + P.rows_per_batch - 1) / P.rows_per_batch;
-        sp.keep_rows = keep_rows_for(ctx, 1, a.n);
-        e = predict ? launch_split<true>(P, a.X, sp, st) : launch_split<false>(P, a.X, sp, st);
+        sp.keep_rows = keep_rows_for(ctx, 1, a.n, a.bf16);
+        e = predict ? launch_split<true>(P, a.X, sp, st, a.bf16) : launch_split<false>(P, a.X, sp, st, a.bf16);
     } else {
         GenericParams gp{};
         gp.X = a.X; gp.y = a.y; gp.m = a.m; gp.n = a.n; gp.w = a.w; gp.b = a.b;
         gp.partial = ctx->d_partial; gp.labels = labels; gp.cut = cut; gp.stop = a.stop;
-        if (predict) k_generic<true><<<P.grid, P.threads, 0, st>>>(gp);
-        else k_generic<false><<<P.grid, P.threads, 0, st>>>(gp);
+        if (a.bf16) {
+            if (predict) k_generic<ElemBF16, true><<<P.grid, P.threads, 0, st>>>(gp);
+            else k_generic<ElemBF16, false><<<P.grid, P.threads, 0, st>>>(gp);
+        } else {
+            if (predict) k_generic<ElemF32, true><<<P.grid, P.threads, 0, st>>>(gp);
+            else k_generic<ElemF32, false><<<P.grid, P.threads, 0, st>>>(gp);
+        }
         e = cudaGetLastError();
     }
     LR_CK(ctx, e);
@@ -328,10 +360,10 @@ int launch_reduce(lr_ctx* ctx, const double* partial, int G, int64_t m, int32_t 
     return LR_OK;
 }
 
-int check_common(lr_ctx* ctx, const void* X, int64_t m, int32_t n, const void* w, const void* b) {
+int check_common(lr_ctx* ctx, const void* X, int64_t m, int32_t n, const void* w, const void* b, bool bf16 = false) {
     if (!ctx || !X || !w || !b) return LR_ERR_NULL;
     if (m < 1 || m > kMaxRows || n < 1 || n > ctx->n_max) return LR_ERR_SHAPE;
-    if (!aligned(X, 4) || !aligned(w, 4) || !aligned(b, 4)) return LR_ERR_ALIGNMENT;
+    if (!aligned(X, bf16 ? 2 : 4) || !aligned(w, 4) || !aligned(b, 4)) return LR_ERR_ALIGNMENT;
     return LR_OK;
 }
 
@@ -344,9 +376,21 @@ int grow(lr_ctx* ctx, void** buf, size_t* have, size_t need) {
     return LR_OK;
 }
 
+int loss_grad_impl(lr_ctx* ctx, const void* d_X, bool bf16, const float* d_y, int64_t m, int32_t n, const float* d_w,
+                   const float* d_b, float* d_loss, float* d_grad_w, float* d_grad_b, void* stream);
+int fit_impl(lr_ctx* ctx, const void* d_X, bool bf16, const float* d_y, int64_t m, int32_t n, float lr, int32_t iters,
+             float* d_w, float* d_b, float* d_loss_hist, void* stream);
+int predict_impl(lr_ctx* ctx, const void* d_X, bool bf16, int64_t m, int32_t n, const float* d_w, const float* d_b, float thr,
+                 uint8_t* d_labels, void* stream);
+
 }  // namespace
 
 extern "C" {
+
+int lr_plan_query_bf16(int64_t m, int32_t n, int32_t x_aligned16, int32_t sm_count, lr_plan* out) {
+    if (!out) return LR_ERR_NULL;
+    return make_plan(m, n, x_aligned16 != 0, sm_count, out, true);
+}
 
 int lr_plan_query(int64_t m, int32_t n, int32_t x_aligned16, int32_t sm_count, lr_plan* out) {
     if (!out) return LR_ERR_NULL;
@@ -438,32 +482,85 @@ int lr_destroy(lr_ctx* ctx) {
 
 int lr_loss_grad(lr_ctx* ctx, const float* d_X, const float* d_y, int64_t m, int32_t n, const float* d_w,
                  const float* d_b, float* d_loss, float* d_grad_w, float* d_grad_b, void* stream) {
-    int rc = check_common(ctx, d_X, m, n, d_w, d_b);
+    return loss_grad_impl(ctx, d_X, false, d_y, m, n, d_w, d_b, d_loss, d_grad_w, d_grad_b, stream);
+}
+
+int lr_loss_grad_bf16(lr_ctx* ctx, const uint16_t* d_Xh, const float* d_y, int64_t m, int32_t n, const float* d_w,
+                      const float* d_b, float* d_loss, float* d_grad_w, float* d_grad_b, void* stream) {
+    return loss_grad_impl(ctx, d_Xh, true, d_y, m, n, d_w, d_b, d_loss, d_grad_w, d_grad_b, stream);
+}
+
+int lr_fit(lr_ctx* ctx, const float* d_X, const float* d_y, int64_t m, int32_t n, float lr, int32_t iters,
+           float* d_w, float* d_b, float* d_loss_hist, void* stream) {
+    return fit_impl(ctx, d_X, false, d_y, m, n, lr, iters, d_w, d_b, d_loss_hist, stream);
+}
+
+int lr_fit_bf16(lr_ctx* ctx, const uint16_t* d_Xh, const float* d_y, int64_t m, int32_t n, float lr, int32_t iters,
+                float* d_w, float* d_b, float* d_loss_hist, void* stream) {
+    return fit_impl(ctx, d_Xh, true, d_y, m, n, lr, iters, d_w, d_b, d_loss_hist, stream);
+}
+
+int lr_predict(lr_ctx* ctx, const float* d_X, int64_t m, int32_t n, const float* d_w, const float* d_b, float thr,
+               uint8_t* d_labels, void* stream) {
+    return predict_impl(ctx, d_X, false, m, n, d_w, d_b, thr, d_labels, stream);
+}
+
+int lr_predict_bf16(lr_ctx* ctx, const uint16_t* d_Xh, int64_t m, int32_t n, const float* d_w, const float* d_b, float thr,
+                    uint8_t* d_labels, void* stream) {
+    return predict_impl(ctx, d_Xh, true, m, n, d_w, d_b, thr, d_labels, stream);
+}
+
+int lr_convert_bf16(lr_ctx* ctx, const float* d_X, int64_t count, uint16_t* d_Xh, void* stream) {
+    if (!ctx) return LR_ERR_NULL;
+    if (count < 0) return LR_ERR_SHAPE;
+    if (count == 0) return LR_OK;                  // nothing to do; the pointers are not looked at
+    if (!d_X || !d_Xh) return LR_ERR_NULL;
+    if (!aligned(d_X, 4) || !aligned(d_Xh, 2)) return LR_ERR_ALIGNMENT;
+    DeviceGuard g(ctx);
+    if (!g.ok) return LR_ERR_CUDA;
+    const bool vec = aligned(d_X, 16) && aligned(d_Xh, 8);
+    const int64_t units = vec ? (count + 3) / 4 : count;
+    const int grid = int(std::min<int64_t>((units + kConvertThreads - 1) / kConvertThreads, int64_t(ctx->sm_count) * 16));
+    k_convert_bf16<<<grid, kConvertThreads, 0, static_cast<cudaStream_t>(stream)>>>(d_X, count, d_Xh, vec ? 1 : 0);
+    LR_CK(ctx, cudaGetLastError());
+    ctx->launches += 1;
+    return LR_OK;
+}
+
+}  // extern "C"
+
+namespace {
+
+int loss_grad_impl(lr_ctx* ctx, const void* d_X, bool bf16, const float* d_y, int64_t m, int32_t n, const float* d_w,
+                   const float* d_b, float* d_loss, float* d_grad_w, float* d_grad_b, void* stream) {
+    int rc = check_common(ctx, d_X, m, n, d_w, d_b, bf16);
     if (rc != LR_OK) return rc;
     if (!d_y || !d_loss || !d_grad_w || !d_grad_b) return LR_ERR_NULL;
     if (!aligned(d_y, 4) || !aligned(d_loss, 4) || !aligned(d_grad_w, 4) || !aligned(d_grad_b, 4)) return LR_ERR_ALIGNMENT;
     lr_plan P;
-    rc = make_plan(m, n, aligned(d_X, 16), ctx->sm_count, &P);
+    rc = make_plan(m, n, aligned(d_X, 16), ctx->sm_count, &P, bf16);
     if (rc != LR_OK) return rc;
     DeviceGuard g(ctx);
     if (!g.ok) return LR_ERR_CUDA;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    rc = launch_stream_pass(ctx, P, Pass{d_X, d_y, m, n, d_w, d_b}, nullptr, 0.f, st);
+    Pass pass{d_X, d_y, m, n, d_w, d_b};
+    pass.bf16 = bf16;
+    rc = launch_stream_pass(ctx, P, pass, nullptr, 0.f, st);
     if (rc != LR_OK) return rc;
     return launch_reduce(ctx, ctx->d_partial, P.grid, m, n, 0.0, false, nullptr, nullptr, d_grad_w, d_grad_b, d_loss,
                          nullptr, st);
 }
 
-int lr_fit(lr_ctx* ctx, const float* d_X, const float* d_y, int64_t m, int32_t n, float lr, int32_t iters,
-           float* d_w, float* d_b, float* d_loss_hist, void* stream) {
-    int rc = check_common(ctx, d_X, m, n, d_w, d_b);
+int fit_impl(lr_ctx* ctx, const void* d_X, bool bf16, const float* d_y, int64_t m, int32_t n, float lr, int32_t iters,
+             float* d_w, float* d_b, float* d_loss_hist, void* stream) {
+    int rc = check_common(ctx, d_X, m, n, d_w, d_b, bf16);
     if (rc != LR_OK) return rc;
     if (!d_y) return LR_ERR_NULL;
     if (iters < 0) return LR_ERR_SHAPE;
     if (!aligned(d_y, 4) || (d_loss_hist && !aligned(d_loss_hist, 4))) return LR_ERR_ALIGNMENT;
     if (!std::isfinite(lr)) return LR_ERR_VALUE;
     lr_plan P;
-    rc = make_plan(m, n, aligned(d_X, 16), ctx->sm_count, &P);
+    rc = make_plan(m, n, aligned(d_X, 16), ctx->sm_count, &P, bf16);
     if (rc != LR_OK) return rc;
     if (iters == 0) return LR_OK;
     DeviceGuard g(ctx);
@@ -472,7 +569,7 @@ int lr_fit(lr_ctx* ctx, const float* d_X, const float* d_y, int64_t m, int32_t n
     // Narrow rows, several iterations: one cooperative launch runs the whole fit (same bits as the loop below).
     if (P.variant == 0 && ctx->persistent && ctx->coop && !ctx->prof && iters >= 2 &&
         2ll * iters * P.grid < (1ll << 32)) {
-        const int64_t stage_stride = (int64_t(P.rows_per_batch) * n * 4 + 127) & ~int64_t(127);
+        const int64_t stage_stride = (int64_t(P.rows_per_batch) * n * (bf16 ? 2 : 4) + 127) & ~int64_t(127);
         const int64_t room = kMaxDynamicSmem - kHeaderBytes - kFitTailBytes;
         const int depth = int(std::max<int64_t>(1, std::min<int64_t>(P.stages, room / (kNW * stage_stride))));
         FitParams fp{};
@@ -480,10 +577,10 @@ int lr_fit(lr_ctx* ctx, const float* d_X, const float* d_y, int64_t m, int32_t n
         fp.loss_hist = d_loss_hist; fp.status = ctx->d_status; fp.gbar = ctx->d_gbar; fp.depth = depth;
         fp.num_batches = (m + P.rows_per_batch - 1) / P.rows_per_batch;
         fp.iters = iters; fp.lr = double(lr); fp.inv_m = 1.0 / double(m);
-        fp.keep_rows = keep_rows_for(ctx, 0, n);
+        fp.keep_rows = keep_rows_for(ctx, 0, n, bf16);
         LR_CK(ctx, cudaMemsetAsync(ctx->d_gbar, 0, sizeof(unsigned int), st));
         const int smem = int(kHeaderBytes + int64_t(kNW) * depth * stage_stride + kFitTailBytes);
-        const cudaError_t le = launch_fit(P, smem, fp, st);
+        const cudaError_t le = launch_fit(P, smem, fp, st, bf16);
         if (le == cudaSuccess) {
             ctx->launches += 1;
             return LR_OK;
@@ -491,8 +588,10 @@ int lr_fit(lr_ctx* ctx, const float* d_X, const float* d_y, int64_t m, int32_t n
         if (le != cudaErrorCooperativeLaunchTooLarge) { ctx->last_cuda = int(le); return LR_ERR_CUDA; }
         cudaGetLastError();                        // the CTAs cannot all be resident here: use the two-kernel form below
     }
+    Pass pass{d_X, d_y, m, n, d_w, d_b};
+    pass.bf16 = bf16;
     for (int32_t t = 0; t < iters; ++t) {
-        rc = launch_stream_pass(ctx, P, Pass{d_X, d_y, m, n, d_w, d_b}, nullptr, 0.f, st);
+        rc = launch_stream_pass(ctx, P, pass, nullptr, 0.f, st);
         if (rc != LR_OK) return rc;
         rc = launch_reduce(ctx, ctx->d_partial, P.grid, m, n, double(lr), true, d_w, d_b, nullptr, nullptr,
                            d_loss_hist ? d_loss_hist + t : nullptr, nullptr, st);
@@ -500,6 +599,27 @@ int lr_fit(lr_ctx* ctx, const float* d_X, const float* d_y, int64_t m, int32_t n
     }
     return LR_OK;
 }
+
+int predict_impl(lr_ctx* ctx, const void* d_X, bool bf16, int64_t m, int32_t n, const float* d_w, const float* d_b, float thr,
+                 uint8_t* d_labels, void* stream) {
+    int rc = check_common(ctx, d_X, m, n, d_w, d_b, bf16);
+    if (rc != LR_OK) return rc;
+    if (!d_labels) return LR_ERR_NULL;
+    if (!(thr > 0.f && thr < 1.f)) return LR_ERR_VALUE;
+    lr_plan P;
+    rc = make_plan(m, n, aligned(d_X, 16), ctx->sm_count, &P, bf16);
+    if (rc != LR_OK) return rc;
+    DeviceGuard g(ctx);
+    if (!g.ok) return LR_ERR_CUDA;
+    const float cut = static_cast<float>(std::log(double(thr) / (1.0 - double(thr))));
+    Pass pass{d_X, nullptr, m, n, d_w, d_b};
+    pass.bf16 = bf16;
+    return launch_stream_pass(ctx, P, pass, d_labels, cut, static_cast<cudaStream_t>(stream));
+}
+
+}  // namespace
+
+extern "C" {
 
 int lr_set_l2_keep(lr_ctx* ctx, int64_t bytes) {
     if (!ctx) return LR_ERR_NULL;
@@ -647,21 +767,6 @@ int lr_fit_sgd(lr_ctx* ctx, const float* d_X, const float* d_y, int64_t m, int32
         if (rc != LR_OK) return rc;
     }
     return LR_OK;
-}
-
-int lr_predict(lr_ctx* ctx, const float* d_X, int64_t m, int32_t n, const float* d_w, const float* d_b, float thr,
-               uint8_t* d_labels, void* stream) {
-    int rc = check_common(ctx, d_X, m, n, d_w, d_b);
-    if (rc != LR_OK) return rc;
-    if (!d_labels) return LR_ERR_NULL;
-    if (!(thr > 0.f && thr < 1.f)) return LR_ERR_VALUE;
-    lr_plan P;
-    rc = make_plan(m, n, aligned(d_X, 16), ctx->sm_count, &P);
-    if (rc != LR_OK) return rc;
-    DeviceGuard g(ctx);
-    if (!g.ok) return LR_ERR_CUDA;
-    const float cut = static_cast<float>(std::log(double(thr) / (1.0 - double(thr))));
-    return launch_stream_pass(ctx, P, Pass{d_X, nullptr, m, n, d_w, d_b}, d_labels, cut, static_cast<cudaStream_t>(stream));
 }
 
 int lr_shard_sums(lr_ctx* ctx, const float* d_X, const float* d_y, int64_t m_local, int32_t n, const float* d_w,
@@ -912,7 +1017,7 @@ extern "C" int lr_loss_grad_noalloc(int32_t device, const float* d_X, const floa
         GenericParams gp{};
         gp.X = d_X; gp.y = d_y; gp.m = m; gp.n = n; gp.w = d_w; gp.b = d_b;
         gp.partial = partial; gp.labels = nullptr; gp.cut = 0.f;
-        k_generic<false><<<P.grid, P.threads, 0, st>>>(gp);
+        k_generic<ElemF32, false><<<P.grid, P.threads, 0, st>>>(gp);
         e = cudaGetLastError();
     }
     if (e != cudaSuccess) return LR_ERR_CUDA;

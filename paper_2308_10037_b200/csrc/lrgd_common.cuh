@@ -152,6 +152,34 @@ __device__ __forceinline__ void logistic_terms(float z, float y, float& err, flo
     loss = fmaxf(z, 0.0f) + log1pf(t) - y * z;
 }
 
+// Storage types of X.  A "group" is 16 bytes of a row -- the unit of every shared-memory load and of the column
+// ownership of a lane: four fp32 values or eight bfloat16 values (bfloat16 = the upper half of a binary32 pattern,
+// so widening is exact: the pattern moves to the upper 16 bits).  All arithmetic is fp32 for both.
+struct ElemF32 {
+    static constexpr int EPG = 4;        // elements per 16-byte group
+    static constexpr int BYTES = 4;      // bytes per element
+    static __device__ __forceinline__ void unpack(const uint4& g, float (&f)[4]) {
+        f[0] = __uint_as_float(g.x); f[1] = __uint_as_float(g.y);
+        f[2] = __uint_as_float(g.z); f[3] = __uint_as_float(g.w);
+    }
+    static __device__ __forceinline__ float load(const void* base, long long i) {
+        return reinterpret_cast<const float*>(base)[i];
+    }
+};
+struct ElemBF16 {
+    static constexpr int EPG = 8;
+    static constexpr int BYTES = 2;
+    static __device__ __forceinline__ void unpack(const uint4& g, float (&f)[8]) {
+        f[0] = __uint_as_float(g.x << 16); f[1] = __uint_as_float(g.x & 0xffff0000u);
+        f[2] = __uint_as_float(g.y << 16); f[3] = __uint_as_float(g.y & 0xffff0000u);
+        f[4] = __uint_as_float(g.z << 16); f[5] = __uint_as_float(g.z & 0xffff0000u);
+        f[6] = __uint_as_float(g.w << 16); f[7] = __uint_as_float(g.w & 0xffff0000u);
+    }
+    static __device__ __forceinline__ float load(const void* base, long long i) {
+        return __uint_as_float(static_cast<uint32_t>(reinterpret_cast<const unsigned short*>(base)[i]) << 16);
+    }
+};
+
 template <int V>
 struct Log2 {
     static constexpr int value = 1 + Log2<V / 2>::value;

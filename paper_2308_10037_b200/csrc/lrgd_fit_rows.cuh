@@ -32,7 +32,7 @@ constexpr int kFitL2Prefetch = LRGD_FIT_L2PF;   // batches per warp pulled into 
 constexpr int kFitTailBytes = 9216;            // combine buffer / reduction slices, after the stages
 
 struct FitParams {
-    const float* X;
+    const void* X;             // fp32 or bfloat16 [m][n], row-major
     const float* y;
     long long m;
     int n;
@@ -81,8 +81,9 @@ __device__ __forceinline__ bool grid_barrier(unsigned int* counter, unsigned int
     return *cta_abort == 0;
 }
 
-template <int NV, int LPR, int RB, int NW>
+template <class E, int NV, int LPR, int RB, int NW>
 __global__ void __launch_bounds__(NW * 32, 1) k_fit_rows(const FitParams p) {
+    constexpr int EPG = E::EPG;
     constexpr int RPW = 32 / LPR;
     constexpr int RPB = RB * RPW;
     constexpr int LOG_LPR = Log2<LPR>::value;
@@ -100,9 +101,10 @@ __global__ void __launch_bounds__(NW * 32, 1) k_fit_rows(const FitParams p) {
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int D = p.depth;
-    const int n = p.n, n4 = n >> 2;
+    const int n = p.n, n4 = n / EPG;                   // n4 = 16-byte groups per row
     const int G = gridDim.x;
-    const uint32_t stage_stride = (static_cast<uint32_t>(RPB) * n * 4u + 127u) & ~127u;
+    const uint32_t row_bytes = static_cast<uint32_t>(n) * E::BYTES;
+    const uint32_t stage_stride = (static_cast<uint32_t>(RPB) * row_bytes + 127u) & ~127u;
     unsigned char* my_stages = data + static_cast<size_t>(warp) * D * stage_stride;
     unsigned char* tail = data + static_cast<size_t>(NW) * D * stage_stride;      // combine buffer
     uint64_t* my_bars = bars + warp * kMaxDepth;
@@ -125,9 +127,10 @@ __global__ void __launch_bounds__(NW * 32, 1) k_fit_rows(const FitParams p) {
     auto issue = [&](long long r0, int d) {        // lane 0 only
         const long long left = p.m - r0;
         const uint32_t rows = left < RPB ? static_cast<uint32_t>(left) : RPB;
-        const uint32_t xbytes = rows * n * 4u;
+        const uint32_t xbytes = rows * row_bytes;
         mbar_arrive_expect_tx(&my_bars[d], xbytes);
-        bulk_copy_g2s(my_stages + static_cast<size_t>(d) * stage_stride, p.X + r0 * n, xbytes, &my_bars[d],
+        bulk_copy_g2s(my_stages + static_cast<size_t>(d) * stage_stride,
+                      static_cast<const unsigned char*>(p.X) + static_cast<size_t>(r0) * row_bytes, xbytes, &my_bars[d],
                       r0 < p.keep_rows ? pol_keep : pol_stream);
     };
 
@@ -154,24 +157,17 @@ __global__ void __launch_bounds__(NW * 32, 1) k_fit_rows(const FitParams p) {
     bool alive = true;                             // CTA-uniform after every grid barrier
 
     for (int t = 0; t < p.iters && alive; ++t) {
-        float4 wv[NV];
-#pragma unroll
-        for (int k = 0; k < NV; ++k) {
-            const int idx = sub + k * LPR;
-            wv[k] = idx < n4 ? make_float4(__ldcg(p.w + 4 * idx), __ldcg(p.w + 4 * idx + 1), __ldcg(p.w + 4 * idx + 2),
-                                           __ldcg(p.w + 4 * idx + 3))
-                             : make_float4(0.f, 0.f, 0.f, 0.f);
-        }
+        float wv[NV][EPG];
+        load_w_slice<NV, EPG>(wv, p.w, sub, LPR, n4, true);
         const float bval = __ldcg(p.b);
-        float4 acc[NV];
-        double dacc[NV][4];
+        float acc[NV][EPG];
+        double dacc[NV][EPG];
         float se = 0.f, sl = 0.f;
         double dse = 0.0, dsl = 0.0;
 #pragma unroll
-        for (int k = 0; k < NV; ++k) {
-            acc[k] = make_float4(0.f, 0.f, 0.f, 0.f);
-            dacc[k][0] = dacc[k][1] = dacc[k][2] = dacc[k][3] = 0.0;
-        }
+        for (int k = 0; k < NV; ++k)
+#pragma unroll
+            for (int c = 0; c < EPG; ++c) { acc[k][c] = 0.f; dacc[k][c] = 0.0; }
         int since_flush = 0;
         long long row0 = first_row;
         float y_next = (cnt > 0 && row0 + myr < p.m) ? __ldg(p.y + row0 + myr) : 0.f;
@@ -185,8 +181,8 @@ __global__ void __launch_bounds__(NW * 32, 1) k_fit_rows(const FitParams p) {
 
             const long long left = p.m - row0;
             const int rows = left < RPB ? static_cast<int>(left) : RPB;
-            const float4* t4 = reinterpret_cast<const float4*>(my_stages + static_cast<size_t>(d) * stage_stride);
-            float4 x[RB][NV];
+            const uint4* t4 = reinterpret_cast<const uint4*>(my_stages + static_cast<size_t>(d) * stage_stride);
+            uint4 x[RB][NV];
             load_row_batch<NV, LPR, RB>(x, t4, rows, n4, full_cols && rows == RPB, sub, slot);
             const bool myvalid = myr < rows;
             const float yv = y_next;
@@ -206,15 +202,15 @@ __global__ void __launch_bounds__(NW * 32, 1) k_fit_rows(const FitParams p) {
             }
             if (++d == D) { d = 0; phase ^= 1u; }
 
-            const float z = batch_dot<NV, LPR, RB>(x, wv, lane) + bval;
+            const float z = batch_dot<E, NV, LPR, RB>(x, wv, lane) + bval;
             float e, L;
             logistic_terms(z, yv, e, L);
             if (!myvalid) { e = 0.f; L = 0.f; }
             if (owner) { se += e; sl += L; }
-            batch_accumulate<NV, LPR, RB>(x, e, acc);
+            batch_accumulate<E, NV, LPR, RB>(x, e, acc);
             if (++since_flush == kFlushBatches) {
                 since_flush = 0;
-                fold_into_fp64<NV>(acc, dacc, se, sl, dse, dsl);
+                fold_into_fp64<NV, EPG>(acc, dacc, se, sl, dse, dsl);
             }
             row0 += stride_rows;
         }
@@ -230,19 +226,20 @@ __global__ void __launch_bounds__(NW * 32, 1) k_fit_rows(const FitParams p) {
                     const long long r0 = first_row + bi * stride_rows;
                     const long long left = p.m - r0;
                     const uint32_t rows = left < RPB ? static_cast<uint32_t>(left) : RPB;
-                    bulk_prefetch_l2(p.X + r0 * n, rows * n * 4u, r0 < p.keep_rows ? pol_keep : pol_stream);
+                    bulk_prefetch_l2(static_cast<const unsigned char*>(p.X) + static_cast<size_t>(r0) * row_bytes, rows * row_bytes,
+                                     r0 < p.keep_rows ? pol_keep : pol_stream);
                 }
             }
         }
 
-        fold_into_fp64<NV>(acc, dacc, se, sl, dse, dsl);
+        fold_into_fp64<NV, EPG>(acc, dacc, se, sl, dse, dsl);
 
         // ---- fixed-order combine of the CTA's warps, kFitCombineCols columns at a time (the stages stay in use) ----
         // row slots of one warp that own the same columns: add in slot order (as k_stream_rows does)
 #pragma unroll
         for (int k2 = 0; k2 < NV; ++k2)
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
+            for (int c = 0; c < EPG; ++c) {
                 double tsum = 0.0;
 #pragma unroll
                 for (int sidx = 0; sidx < RPW; ++sidx) tsum += __shfl_sync(FULL, dacc[k2][c], sub + sidx * LPR);
@@ -263,10 +260,10 @@ __global__ void __launch_bounds__(NW * 32, 1) k_fit_rows(const FitParams p) {
 #pragma unroll
             for (int k2 = 0; k2 < NV; ++k2) {
                 const int idx = sub + k2 * LPR;
-                const int col = idx * 4 - c0;
+                const int col = idx * EPG - c0;
                 if (slot == 0 && idx < n4 && col >= 0 && col < kFitCombineCols) {
 #pragma unroll
-                    for (int c = 0; c < 4; ++c) red[warp * kFitCombineCols + col + c] = dacc[k2][c];
+                    for (int c = 0; c < EPG; ++c) red[warp * kFitCombineCols + col + c] = dacc[k2][c];
                 }
             }
             __syncthreads();

@@ -1,5 +1,5 @@
-// Unstaged kernel for shapes the staged kernels do not take (n not a multiple of 4, X not 16-byte
-// aligned, or rows wider than the staged kernels cover).  Plain coalesced loads; X is read from HBM
+// Unstaged kernel for shapes the staged kernels do not take (a row that is not a whole number of 16-byte
+// groups, X not 16-byte aligned, or rows wider than the staged kernels cover).  E is the storage type of X.  Plain coalesced loads; X is read from HBM
 // once and a second time through the cache hierarchy.
 //
 // A CTA walks chunks of kGenRows rows (chunk c belongs to CTA c mod grid).  Phase 1: one warp per row
@@ -17,7 +17,7 @@ constexpr int kGenRows = 64;
 constexpr int kGenThreads = 256;
 
 struct GenericParams {
-    const float* X;
+    const void* X;            // fp32 or bfloat16 [m][n], row-major
     const float* y;
     long long m;
     int n;
@@ -29,7 +29,7 @@ struct GenericParams {
     const int* stop;          // nullable: non-zero makes the launch a no-op
 };
 
-template <bool PREDICT>
+template <class E, bool PREDICT>
 __global__ void __launch_bounds__(kGenThreads) k_generic(const GenericParams p) {
     if (p.stop != nullptr && *reinterpret_cast<const volatile int*>(p.stop) != 0) return;   // a stopping rule was met by an earlier iteration
     __shared__ float err_s[kGenRows];
@@ -48,9 +48,9 @@ __global__ void __launch_bounds__(kGenThreads) k_generic(const GenericParams p) 
         const long long row0 = chunk * kGenRows;
         const int rows = static_cast<int>(p.m - row0 < kGenRows ? p.m - row0 : kGenRows);
         for (int r = warp; r < rows; r += NWARP) {
-            const float* xr = p.X + (row0 + r) * n;
+            const long long xr = (row0 + r) * n;
             float d = 0.f;
-            for (int c = lane; c < n; c += 32) d = fmaf(xr[c], __ldg(p.w + c), d);
+            for (int c = lane; c < n; c += 32) d = fmaf(E::load(p.X, xr + c), __ldg(p.w + c), d);
 #pragma unroll
             for (int msk = 16; msk >= 1; msk >>= 1) d += __shfl_xor_sync(0xffffffffu, d, msk);
             const float z = d + bval;
@@ -65,9 +65,9 @@ __global__ void __launch_bounds__(kGenThreads) k_generic(const GenericParams p) 
         if constexpr (!PREDICT) {
             __syncthreads();
             for (int c = threadIdx.x; c < n; c += kGenThreads) {
-                const float* xc = p.X + row0 * n + c;
+                const long long xc = row0 * n + c;
                 float a = 0.f;
-                for (int r = 0; r < rows; ++r) a = fmaf(xc[static_cast<size_t>(r) * n], err_s[r], a);
+                for (int r = 0; r < rows; ++r) a = fmaf(E::load(p.X, xc + static_cast<long long>(r) * n), err_s[r], a);
                 out[c] += static_cast<double>(a);
             }
             __syncthreads();

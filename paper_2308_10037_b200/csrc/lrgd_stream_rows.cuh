@@ -1,4 +1,5 @@
-// Fused single-pass streaming kernel for rows of up to 512 columns (n % 4 == 0, X 16-byte aligned).
+// Fused single-pass streaming kernel for rows of up to 128 16-byte groups (512 fp32 or 512 bfloat16 columns; the
+// row length a whole number of groups, X 16-byte aligned).  E is the storage type of X (ElemF32 / ElemBF16).
 //
 // Every warp runs its own small asynchronous pipeline: it owns `depth` shared-memory stages, each the
 // size of one batch of rows, and its elected lane keeps them filled with 1-D bulk asynchronous copies
@@ -29,7 +30,7 @@ constexpr int kHeaderBytes = 1024;     // per-warp mbarriers [NW][kMaxDepth], ab
 constexpr int kFlushBatches = 4;
 
 struct StreamParams {
-    const float* X;
+    const void* X;            // fp32 or bfloat16 [m][n], row-major
     const float* y;
     long long m;
     int n;
@@ -69,22 +70,23 @@ __device__ __forceinline__ void lane_reduce(float (&v)[RB], int lane) {
 }
 
 // ---- pieces of the per-batch work shared by the narrow-row, wide-row and persistent kernels ----
-// A batch lives in registers as x[RB][NV]: RB row slots by NV 16-byte column groups per lane; LPR lanes share a row.
+// A batch lives in registers as x[RB][NV]: RB row slots by NV 16-byte column groups per lane (raw bits; widened to
+// fp32 where they are used); LPR lanes share a row.  EPG = elements per group of the storage type E.
 
 // z partials: lane-local FMAs, then the transposing reduction; the returned value is the full dot product of the row
 // (r, with r = (lane_in_group >> (log2 LPR - log2 RB)) & (RB-1)) that ends up on this lane.
-template <int NV, int LPR, int RB>
-__device__ __forceinline__ float batch_dot(const float4 (&x)[RB][NV], const float4 (&wv)[NV], int lane) {
+template <class E, int NV, int LPR, int RB>
+__device__ __forceinline__ float batch_dot(const uint4 (&x)[RB][NV], const float (&wv)[NV][E::EPG], int lane) {
     float v[RB];
 #pragma unroll
     for (int r = 0; r < RB; ++r) {
         float dot = 0.f;
 #pragma unroll
         for (int k = 0; k < NV; ++k) {
-            dot = fmaf(x[r][k].x, wv[k].x, dot);
-            dot = fmaf(x[r][k].y, wv[k].y, dot);
-            dot = fmaf(x[r][k].z, wv[k].z, dot);
-            dot = fmaf(x[r][k].w, wv[k].w, dot);
+            float xf[E::EPG];
+            E::unpack(x[r][k], xf);
+#pragma unroll
+            for (int c = 0; c < E::EPG; ++c) dot = fmaf(xf[c], wv[k][c], dot);
         }
         v[r] = dot;
     }
@@ -93,39 +95,53 @@ __device__ __forceinline__ float batch_dot(const float4 (&x)[RB][NV], const floa
 }
 
 // acc[c] += x[r][c] * err[r]: each row's err is fetched from the lane that holds it (Algorithm 1's err.X on registers).
-template <int NV, int LPR, int RB>
-__device__ __forceinline__ void batch_accumulate(const float4 (&x)[RB][NV], float e, float4 (&acc)[NV]) {
+template <class E, int NV, int LPR, int RB>
+__device__ __forceinline__ void batch_accumulate(const uint4 (&x)[RB][NV], float e, float (&acc)[NV][E::EPG]) {
     constexpr int SHIFT = Log2<LPR>::value - Log2<RB>::value;
 #pragma unroll
     for (int r = 0; r < RB; ++r) {
         const float er = __shfl_sync(0xffffffffu, e, r << SHIFT, LPR);
 #pragma unroll
         for (int k = 0; k < NV; ++k) {
-            acc[k].x = fmaf(x[r][k].x, er, acc[k].x);
-            acc[k].y = fmaf(x[r][k].y, er, acc[k].y);
-            acc[k].z = fmaf(x[r][k].z, er, acc[k].z);
-            acc[k].w = fmaf(x[r][k].w, er, acc[k].w);
+            float xf[E::EPG];
+            E::unpack(x[r][k], xf);
+#pragma unroll
+            for (int c = 0; c < E::EPG; ++c) acc[k][c] = fmaf(xf[c], er, acc[k][c]);
         }
     }
 }
 
 // fp32 per-lane sums folded into their fp64 counterparts (keeps the serial fp32 chains short)
-template <int NV>
-__device__ __forceinline__ void fold_into_fp64(float4 (&acc)[NV], double (&dacc)[NV][4], float& se, float& sl, double& dse,
-                                               double& dsl) {
+template <int NV, int EPG>
+__device__ __forceinline__ void fold_into_fp64(float (&acc)[NV][EPG], double (&dacc)[NV][EPG], float& se, float& sl,
+                                               double& dse, double& dsl) {
+#pragma unroll
+    for (int k = 0; k < NV; ++k)
+#pragma unroll
+        for (int c = 0; c < EPG; ++c) {
+            dacc[k][c] += acc[k][c];
+            acc[k][c] = 0.f;
+        }
+    dse += se; dsl += sl; se = 0.f; sl = 0.f;
+}
+
+// this lane's slice of w, widened per group: wv[k][c] = w[EPG*(sub + k*LPR) + c] (zero past the row; w needs no alignment)
+template <int NV, int EPG>
+__device__ __forceinline__ void load_w_slice(float (&wv)[NV][EPG], const float* w, int first_group, int group_stride, int ng,
+                                             bool through_l2) {
 #pragma unroll
     for (int k = 0; k < NV; ++k) {
-        dacc[k][0] += acc[k].x; dacc[k][1] += acc[k].y;
-        dacc[k][2] += acc[k].z; dacc[k][3] += acc[k].w;
-        acc[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+        const int idx = first_group + k * group_stride;
+#pragma unroll
+        for (int c = 0; c < EPG; ++c)
+            wv[k][c] = idx < ng ? (through_l2 ? __ldcg(w + EPG * idx + c) : __ldg(w + EPG * idx + c)) : 0.f;
     }
-    dse += se; dsl += sl; se = 0.f; sl = 0.f;
 }
 
 // one batch from a narrow-row stage into registers (rows packed at n4 groups; lanes beyond the row or rows beyond the
 // matrix read zeros); `full` = every lane's groups exist and the batch is complete: no bounds logic
 template <int NV, int LPR, int RB>
-__device__ __forceinline__ void load_row_batch(float4 (&x)[RB][NV], const float4* t4, int rows, int n4, bool full, int sub,
+__device__ __forceinline__ void load_row_batch(uint4 (&x)[RB][NV], const uint4* t4, int rows, int n4, bool full, int sub,
                                                int slot) {
     constexpr int RPW = 32 / LPR;
     if (full) {
@@ -140,14 +156,15 @@ __device__ __forceinline__ void load_row_batch(float4 (&x)[RB][NV], const float4
 #pragma unroll
             for (int k2 = 0; k2 < NV; ++k2) {
                 const int idx = sub + k2 * LPR;
-                x[r8][k2] = (r < rows && idx < n4) ? t4[r * n4 + idx] : make_float4(0.f, 0.f, 0.f, 0.f);
+                x[r8][k2] = (r < rows && idx < n4) ? t4[r * n4 + idx] : make_uint4(0u, 0u, 0u, 0u);
             }
         }
     }
 }
 
-template <int NV, int LPR, int RB, int NW, bool PREDICT>
+template <class E, int NV, int LPR, int RB, int NW, bool PREDICT>
 __global__ void __launch_bounds__(NW * 32, 1) k_stream_rows(const StreamParams p) {
+    constexpr int EPG = E::EPG;
     constexpr int RPW = 32 / LPR;                  // rows a warp touches with one load instruction
     constexpr int RPB = RB * RPW;                  // rows per batch
     constexpr int LOG_LPR = Log2<LPR>::value;
@@ -165,8 +182,9 @@ __global__ void __launch_bounds__(NW * 32, 1) k_stream_rows(const StreamParams p
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int D = p.depth;
-    const int n = p.n, n4 = n >> 2;
-    const uint32_t stage_stride = (static_cast<uint32_t>(RPB) * n * 4u + 127u) & ~127u;
+    const int n = p.n, n4 = n / EPG;                   // n4 = 16-byte groups per row
+    const uint32_t row_bytes = static_cast<uint32_t>(n) * E::BYTES;
+    const uint32_t stage_stride = (static_cast<uint32_t>(RPB) * row_bytes + 127u) & ~127u;
     unsigned char* my_stages = data + static_cast<size_t>(warp) * D * stage_stride;
     uint64_t* my_bars = bars + warp * kMaxDepth;
 
@@ -189,31 +207,25 @@ __global__ void __launch_bounds__(NW * 32, 1) k_stream_rows(const StreamParams p
     auto issue = [&](long long r0, int d) {
         const long long left = p.m - r0;
         const uint32_t rows = left < RPB ? static_cast<uint32_t>(left) : RPB;
-        const uint32_t xbytes = rows * n * 4u;
+        const uint32_t xbytes = rows * row_bytes;
         mbar_arrive_expect_tx(&my_bars[d], xbytes);
-        bulk_copy_g2s(my_stages + static_cast<size_t>(d) * stage_stride, p.X + r0 * n, xbytes, &my_bars[d],
+        bulk_copy_g2s(my_stages + static_cast<size_t>(d) * stage_stride,
+                      static_cast<const unsigned char*>(p.X) + static_cast<size_t>(r0) * row_bytes, xbytes, &my_bars[d],
                       r0 < p.keep_rows ? pol_keep : pol_stream);
     };
 
-    float4 acc[NV];
-    double dacc[NV][4];
+    float acc[NV][EPG];
+    double dacc[NV][EPG];
     float se = 0.f, sl = 0.f;
     double dse = 0.0, dsl = 0.0;
 #pragma unroll
-    for (int k = 0; k < NV; ++k) {
-        acc[k] = make_float4(0.f, 0.f, 0.f, 0.f);
-        dacc[k][0] = dacc[k][1] = dacc[k][2] = dacc[k][3] = 0.0;
-    }
+    for (int k = 0; k < NV; ++k)
+#pragma unroll
+        for (int c = 0; c < EPG; ++c) { acc[k][c] = 0.f; dacc[k][c] = 0.0; }
     const int sub = lane & (LPR - 1), slot = lane >> LOG_LPR;
 
-    float4 wv[NV];                                 // this lane's slice of w (w needs no 16-byte alignment)
-#pragma unroll
-    for (int k = 0; k < NV; ++k) {
-        const int idx = sub + k * LPR;
-        wv[k] = idx < n4 ? make_float4(__ldg(p.w + 4 * idx), __ldg(p.w + 4 * idx + 1), __ldg(p.w + 4 * idx + 2),
-                                       __ldg(p.w + 4 * idx + 3))
-                         : make_float4(0.f, 0.f, 0.f, 0.f);
-    }
+    float wv[NV][EPG];                             // this lane's slice of w
+    load_w_slice<NV, EPG>(wv, p.w, sub, LPR, n4, false);
     const float bval = __ldg(p.b);
     const int myr = ((sub >> SHIFT) & (RB - 1)) * RPW + slot;     // the row of a batch whose logit ends up on this lane
     const bool owner = (sub & ((1 << SHIFT) - 1)) == 0;           // one lane per row does the bookkeeping
@@ -242,8 +254,8 @@ __global__ void __launch_bounds__(NW * 32, 1) k_stream_rows(const StreamParams p
 
         const long long left = p.m - row0;
         const int rows = left < RPB ? static_cast<int>(left) : RPB;
-        const float4* t4 = reinterpret_cast<const float4*>(my_stages + static_cast<size_t>(d) * stage_stride);
-        float4 x[RB][NV];
+        const uint4* t4 = reinterpret_cast<const uint4*>(my_stages + static_cast<size_t>(d) * stage_stride);
+        uint4 x[RB][NV];
         load_row_batch<NV, LPR, RB>(x, t4, rows, n4, full_cols && rows == RPB, sub, slot);
         const bool myvalid = myr < rows;
         const float yv = y_next;
@@ -262,7 +274,7 @@ __global__ void __launch_bounds__(NW * 32, 1) k_stream_rows(const StreamParams p
         }
         if (++d == D) { d = 0; phase ^= 1u; }
 
-        const float z = batch_dot<NV, LPR, RB>(x, wv, lane) + bval;
+        const float z = batch_dot<E, NV, LPR, RB>(x, wv, lane) + bval;
 
         if constexpr (PREDICT) {
             // one bit per lane, then RPB/4 lanes each assemble and store four labels as one 32-bit word
@@ -286,10 +298,10 @@ __global__ void __launch_bounds__(NW * 32, 1) k_stream_rows(const StreamParams p
             logistic_terms(z, yv, e, L);
             if (!myvalid) { e = 0.f; L = 0.f; }
             if (owner) { se += e; sl += L; }
-            batch_accumulate<NV, LPR, RB>(x, e, acc);
+            batch_accumulate<E, NV, LPR, RB>(x, e, acc);
             if (++since_flush == kFlushBatches) {
                 since_flush = 0;
-                fold_into_fp64<NV>(acc, dacc, se, sl, dse, dsl);
+                fold_into_fp64<NV, EPG>(acc, dacc, se, sl, dse, dsl);
             }
         }
         row0 += stride_rows;
@@ -305,7 +317,7 @@ __global__ void __launch_bounds__(NW * 32, 1) k_stream_rows(const StreamParams p
         __syncwarp();
     }
     if constexpr (!PREDICT) {
-        fold_into_fp64<NV>(acc, dacc, se, sl, dse, dsl);
+        fold_into_fp64<NV, EPG>(acc, dacc, se, sl, dse, dsl);
 
         // ---------------- fixed-order combine of the CTA's warps ----------------
         __syncthreads();                               // all stages are idle: reuse them as the combine buffer
@@ -316,12 +328,12 @@ __global__ void __launch_bounds__(NW * 32, 1) k_stream_rows(const StreamParams p
 #pragma unroll
         for (int k2 = 0; k2 < NV; ++k2) {
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
+            for (int c = 0; c < EPG; ++c) {
                 double t = 0.0;
 #pragma unroll
                 for (int sidx = 0; sidx < RPW; ++sidx) t += __shfl_sync(FULL, dacc[k2][c], sub + sidx * LPR);
                 const int idx = sub + k2 * LPR;
-                if (slot == 0 && idx < n4) red[static_cast<size_t>(warp) * n + idx * 4 + c] = t;
+                if (slot == 0 && idx < n4) red[static_cast<size_t>(warp) * n + idx * EPG + c] = t;
             }
         }
 #pragma unroll

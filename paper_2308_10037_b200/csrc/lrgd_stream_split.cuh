@@ -1,4 +1,6 @@
-// Fused single-pass streaming kernel for wide rows (512 < n <= 4096, n % 4 == 0, X 16-byte aligned).
+// Fused single-pass streaming kernel for wide rows (more 16-byte groups per row than the narrow-row kernel takes, up
+// to 1024: 512 < n <= 4096 fp32 columns or 512 < n <= 8192 bfloat16 columns; the row a whole number of groups, X
+// 16-byte aligned).  E is the storage type of X (ElemF32 / ElemBF16).
 //
 // A row no longer fits one warp's registers, so the 16 warps of a CTA split every row by columns: warp w owns
 // the contiguous slice of CW = ceil(n/4/16) 16-byte column groups starting at w*CW.  The CTA walks batches of RB
@@ -39,13 +41,14 @@ struct SplitParams {
     int* status;
     const int* stop;          // nullable: non-zero makes the launch a no-op
     int depth;                // stages per warp
-    int cw;                   // 16-byte column groups per warp slice (the tensor map's box is cw*4 floats by RB rows)
+    int cw;                   // 16-byte column groups per warp slice (the tensor map's box is cw groups by RB rows)
     long long num_batches;    // ceil(m / RB)
     long long keep_rows;      // rows [0, keep_rows) are fetched with an L2 evict-last hint, the rest evict-first
 };
 
-template <int NV, int RB, int NW, bool PREDICT>
+template <class E, int NV, int RB, int NW, bool PREDICT>
 __global__ void __launch_bounds__(NW * 32, 1) k_stream_split(const __grid_constant__ CUtensorMap tmap, const SplitParams p) {
+    constexpr int EPG = E::EPG;
     constexpr int LOG_RB = Log2<RB>::value;
     constexpr int SHIFT = 5 - LOG_RB;              // log2 of the lanes holding the same row after the reduction
     constexpr int DUP = 1 << SHIFT;
@@ -64,7 +67,7 @@ __global__ void __launch_bounds__(NW * 32, 1) k_stream_split(const __grid_consta
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int D = p.depth, CW = p.cw;
-    const int n = p.n, n4 = n >> 2;
+    const int n = p.n, n4 = n / EPG;                                          // 16-byte groups per row
     const int c0 = warp * CW;                                                 // first column group of this warp's slice
     const int mycw = n4 - c0 < CW ? (n4 - c0 > 0 ? n4 - c0 : 0) : CW;         // column groups of the slice inside the matrix
     const uint32_t box_bytes = static_cast<uint32_t>(CW) * 16u * RB;          // one stage = one box, rows packed densely
@@ -87,24 +90,25 @@ __global__ void __launch_bounds__(NW * 32, 1) k_stream_split(const __grid_consta
     int row0 = static_cast<int>(blockIdx.x) * RB;                             // first row of the current batch
     auto issue = [&](int r0, int d) {              // lane 0 of a warp with mycw > 0
         mbar_arrive_expect_tx(&my_bars[d], box_bytes);
-        bulk_tensor_2d_g2s(my_stages + static_cast<size_t>(d) * stage_stride, &tmap, c0 * 4, r0, &my_bars[d],
+        bulk_tensor_2d_g2s(my_stages + static_cast<size_t>(d) * stage_stride, &tmap, c0 * 4, r0, &my_bars[d],   // x in 32-bit words
                            r0 < p.keep_rows ? pol_keep : pol_stream);
     };
 
-    float4 acc[NV];
-    double dacc[NV][4];
+    float acc[NV][EPG];
+    double dacc[NV][EPG];
     float se = 0.f, sl = 0.f;
     double dse = 0.0, dsl = 0.0;
-    float4 wv[NV];
+    float wv[NV][EPG];
 #pragma unroll
     for (int k = 0; k < NV; ++k) {
-        acc[k] = make_float4(0.f, 0.f, 0.f, 0.f);
-        dacc[k][0] = dacc[k][1] = dacc[k][2] = dacc[k][3] = 0.0;
         const int loc = lane + 32 * k;
         const int idx = c0 + loc;
-        wv[k] = loc < mycw ? make_float4(__ldg(p.w + 4 * idx), __ldg(p.w + 4 * idx + 1), __ldg(p.w + 4 * idx + 2),
-                                         __ldg(p.w + 4 * idx + 3))
-                           : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+        for (int c = 0; c < EPG; ++c) {
+            acc[k][c] = 0.f;
+            dacc[k][c] = 0.0;
+            wv[k][c] = loc < mycw ? __ldg(p.w + EPG * idx + c) : 0.f;
+        }
     }
     const float bval = __ldg(p.b);
     const int myr = (lane >> SHIFT) & (RB - 1);    // the row of a batch whose logit ends up on this lane
@@ -137,7 +141,7 @@ __global__ void __launch_bounds__(NW * 32, 1) k_stream_split(const __grid_consta
             y_next = (i + 1 < cnt && rn < p.m) ? __ldg(p.y + rn) : 0.f;
         }
 
-        float4 x[RB][NV];
+        uint4 x[RB][NV];
         bool have = false;
         if (active && !aborted) {
             bool ok = mbar_wait_bounded(&my_bars[d], phase, abort_flag);
@@ -147,7 +151,7 @@ __global__ void __launch_bounds__(NW * 32, 1) k_stream_split(const __grid_consta
             } else {
                 done = i + 1;
                 have = true;
-                const float4* t4 = reinterpret_cast<const float4*>(my_stages + static_cast<size_t>(d) * stage_stride);
+                const uint4* t4 = reinterpret_cast<const uint4*>(my_stages + static_cast<size_t>(d) * stage_stride);
                 if (full_cw) {
 #pragma unroll
                     for (int r = 0; r < RB; ++r)
@@ -159,7 +163,7 @@ __global__ void __launch_bounds__(NW * 32, 1) k_stream_split(const __grid_consta
 #pragma unroll
                         for (int k = 0; k < NV; ++k) {
                             const int loc = lane + 32 * k;
-                            x[r][k] = loc < CW ? t4[r * CW + loc] : make_float4(0.f, 0.f, 0.f, 0.f);
+                            x[r][k] = loc < CW ? t4[r * CW + loc] : make_uint4(0u, 0u, 0u, 0u);
                         }
                 }
                 __syncwarp();
@@ -177,10 +181,10 @@ __global__ void __launch_bounds__(NW * 32, 1) k_stream_split(const __grid_consta
 #pragma unroll
             for (int r = 0; r < RB; ++r)
 #pragma unroll
-                for (int k = 0; k < NV; ++k) x[r][k] = make_float4(0.f, 0.f, 0.f, 0.f);
+                for (int k = 0; k < NV; ++k) x[r][k] = make_uint4(0u, 0u, 0u, 0u);
         }
 
-        const float zpartial = batch_dot<NV, 32, RB>(x, wv, lane);
+        const float zpartial = batch_dot<E, NV, 32, RB>(x, wv, lane);
         float* zp = zpart + (i & 1) * (NW * RB);
         if (owner) zp[warp * RB + myr] = zpartial;
         __syncthreads();
@@ -216,10 +220,10 @@ __global__ void __launch_bounds__(NW * 32, 1) k_stream_split(const __grid_consta
                 e = logistic_err(z, yv);
             }
             if (!myvalid) e = 0.f;
-            batch_accumulate<NV, 32, RB>(x, e, acc);
+            batch_accumulate<E, NV, 32, RB>(x, e, acc);
             if (++since_flush == 2 * kFlushBatches) {
                 since_flush = 0;
-                fold_into_fp64<NV>(acc, dacc, se, sl, dse, dsl);
+                fold_into_fp64<NV, EPG>(acc, dacc, se, sl, dse, dsl);
             }
         }
         row0 += stride_rows;
@@ -239,11 +243,9 @@ __global__ void __launch_bounds__(NW * 32, 1) k_stream_split(const __grid_consta
         for (int k = 0; k < NV; ++k) {
             const int loc = lane + 32 * k;
             if (loc < mycw) {
-                const int col = 4 * (c0 + loc);
-                out[col + 0] = dacc[k][0] + acc[k].x;
-                out[col + 1] = dacc[k][1] + acc[k].y;
-                out[col + 2] = dacc[k][2] + acc[k].z;
-                out[col + 3] = dacc[k][3] + acc[k].w;
+                const int col = EPG * (c0 + loc);
+#pragma unroll
+                for (int c = 0; c < EPG; ++c) out[col + c] = dacc[k][c] + acc[k][c];
             }
         }
         if (warp == 0) {

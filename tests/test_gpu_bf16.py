@@ -1,0 +1,187 @@
+"""GPU parity for the bfloat16 storage variant of X, through the C-ABI binding.
+
+The conversion kernel is compared bit for bit with the checker's rounding.  The three bfloat16 entry points are compared
+with the float64 checker run on the SAME values (the rounded matrix widened back to fp32), so the tolerances are those
+of the fp32 path: gradient relative L2 <= 1e-5, loss absolute <= 1e-6, fitted parameters relative L2 <= 1e-4, labels
+agreeing on >= 99.99 % of rows.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2308_10037_b200 import api, datagen
+
+pytestmark = pytest.mark.gpu
+
+from _parity import GRAD_TOL, LABEL_AGREE, LOSS_TOL, W_TOL, assert_grad_close, grad_noise_floor, rel_l2
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    from paper_2308_10037_b200 import build
+    build.build()
+    c = api.Context(n_max=8200, device=0)
+    yield c
+    assert c.device_status() == 0
+    c.close()
+
+
+def dev(a):
+    return torch.from_numpy(np.ascontiguousarray(a)).cuda()
+
+
+def dev_bf16(bits):
+    """uint16 bfloat16 patterns (numpy) -> a CUDA bfloat16 tensor holding the same bits."""
+    return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).cuda().view(torch.bfloat16)
+
+
+def test_conversion_is_bit_exact(ctx):
+    rng = np.random.default_rng(5)
+    # random patterns (all exponents, subnormals, infinities, NaNs), a sweep across ties, and a ragged tail
+    x = rng.integers(0, 1 << 32, size=1_000_003, dtype=np.uint64).astype(np.uint32)
+    top = rng.integers(0, 1 << 16, size=20_000, dtype=np.uint64).astype(np.uint32) << 16
+    x = np.concatenate([x, top | 0x7FFF, top | 0x8000, top | 0x8001]).view(np.float32)
+    want, _ = oracle.round_bf16(x)
+    got = ctx.convert_bf16(dev(x)).view(torch.int16).cpu().numpy().view(np.uint16)
+    nan = np.isnan(x)
+    assert np.array_equal(got[~nan], want[~nan])
+    assert np.all((got[nan] & 0x7FFF) > 0x7F80) and np.array_equal(got[nan] >> 15, want[nan] >> 15)   # NaN stays NaN, sign kept
+    # unaligned source and destination take the element-wise path; an empty input is accepted
+    buf = torch.zeros(x.size + 1, dtype=torch.float32, device="cuda")
+    buf[1:] = dev(x)
+    out = torch.zeros(x.size + 1, dtype=torch.bfloat16, device="cuda")
+    ctx.convert_bf16(buf[1:], out=out[1:])
+    got2 = out[1:].view(torch.int16).cpu().numpy().view(np.uint16)
+    assert np.array_equal(got2[~nan], want[~nan])
+    ctx.convert_bf16(torch.empty(0, dtype=torch.float32, device="cuda"))
+
+
+def check_loss_grad(ctx, Xv, dXh, y, w, b, loss_tol=LOSS_TOL):
+    L, g, g0 = oracle.loss_grad(Xv, y, np.asarray(w, dtype=np.float64), float(b))
+    dl, dg, dg0 = ctx.loss_grad(dXh, dev(y), dev(np.asarray(w, dtype=np.float32)), dev(np.array([b], dtype=np.float32)))
+    torch.cuda.synchronize()
+    assert abs(dl.item() - L) <= loss_tol, (dl.item(), L)
+    got = np.concatenate([dg.cpu().numpy(), dg0.cpu().numpy()])
+    assert rel_l2(got, np.concatenate([g, [g0]])) <= GRAD_TOL
+    return got
+
+
+# every staged instantiation for 8-column groups (n/8 <= 8, 16, 32, 64), partly filled lane groups, the wide-row kernel
+# (n/8 > 64: full and partly idle warp slices), the unstaged kernel (n % 8 != 0, n > 8192), tiny / ragged / many-tile rows
+SHAPES = [(1, 8), (7, 8), (9, 5), (33, 56), (1000, 64), (4097, 64), (5003, 128), (2500, 72), (3001, 100), (9999, 256),
+          (777, 200), (1500, 512), (2049, 264), (640, 30), (300, 1), (50, 8200), (20011, 16), (1025, 36),
+          (200_003, 256), (400_001, 64), (200_002, 128), (150_001, 24), (60_001, 512), (90_001, 200), (120_007, 104),
+          (5_001, 4096), (20_003, 1024), (2_500, 520), (1_203, 2056), (701, 4088), (9_000, 2048), (3, 8192), (130, 8192),
+          (1_001, 6000)]
+
+
+@pytest.mark.parametrize("m,n", SHAPES)
+def test_loss_grad_matches_oracle(ctx, m, n):
+    X, y, w, b = datagen.random_problem(m, n, seed=2000 + m + n, wscale=1.5)
+    bits, Xv = oracle.round_bf16(X)
+    check_loss_grad(ctx, Xv, dev_bf16(bits), y, w, b)
+
+
+def test_library_conversion_feeds_the_pass(ctx):
+    # fp32 on the device -> lr_convert_bf16 -> lr_loss_grad_bf16, against the checker on its own rounding of the same X
+    X, y, w, b = datagen.random_problem(30_011, 256, seed=31, wscale=1.0)
+    _, Xv = oracle.round_bf16(X)
+    check_loss_grad(ctx, Xv, ctx.convert_bf16(dev(X)), y, w, b)
+
+
+def test_unaligned_bf16_view_uses_the_unstaged_kernel(ctx):
+    X, y, w, b = datagen.random_problem(1201, 64, seed=12)
+    bits, Xv = oracle.round_bf16(X)
+    buf = torch.zeros(bits.size + 1, dtype=torch.bfloat16, device="cuda")
+    buf[1:] = dev_bf16(bits).ravel()
+    Xh = buf[1:].view(1201, 64)
+    assert Xh.data_ptr() % 16 == 2
+    check_loss_grad(ctx, Xv, Xh, y, w, b)
+
+
+SMALL_WORKLOADS = [("cfg1", 10_000), ("cfg3", 30_011), ("cfg4", 3_000), ("cfg5", 100_003)]
+
+
+@pytest.mark.parametrize("name,m", SMALL_WORKLOADS)
+def test_teacher_forced_trajectory(ctx, name, m):
+    wl = datagen.scaled(datagen.WORKLOADS[name], m)
+    X, y, _, _ = datagen.generate(wl)
+    bits, Xv = oracle.round_bf16(X)
+    iters = min(wl.iters, 40)
+    _, _, lh, wh, bh = oracle.fit(Xv, y, wl.lr, iters, history=True)
+    dXh, dy = dev_bf16(bits), dev(y)
+    floor = grad_noise_floor(Xv)
+    for t in sorted({0, 1, 2, iters // 2, iters - 1}):
+        w32 = wh[t].astype(np.float32)
+        b32 = np.float32(bh[t])
+        L, g, g0 = oracle.loss_grad(Xv, y, w32.astype(np.float64), float(b32))
+        dl, dg, dg0 = ctx.loss_grad(dXh, dy, dev(w32), dev(np.array([b32])))
+        assert abs(dl.item() - L) <= LOSS_TOL, (t, dl.item(), L)
+        got = np.concatenate([dg.cpu().numpy(), dg0.cpu().numpy()])
+        assert_grad_close(got, np.concatenate([g, [g0]]), floor, (name, t))
+
+
+@pytest.mark.parametrize("name,m", [("cfg1", 10_000), ("cfg3", 30_011), ("cfg5", 100_003)])
+def test_fit_and_predict_match_oracle(ctx, name, m):
+    wl = datagen.scaled(datagen.WORKLOADS[name], m)
+    X, y, _, _ = datagen.generate(wl)
+    bits, Xv = oracle.round_bf16(X)
+    iters = min(wl.iters, 60)
+    w_ref, b_ref, lh_ref = oracle.fit(Xv, y, wl.lr, iters)
+    dXh, dy = dev_bf16(bits), dev(y)
+    hist = torch.empty(iters, dtype=torch.float32, device="cuda")
+    w = torch.zeros(wl.n, device="cuda")
+    b = torch.zeros(1, device="cuda")
+    ctx.fit(dXh, dy, wl.lr, iters, w, b, hist)                    # one persistent launch
+    got = np.concatenate([w.cpu().numpy(), b.cpu().numpy()])
+    assert rel_l2(got, np.concatenate([w_ref, [b_ref]])) <= W_TOL
+    assert np.max(np.abs(hist.cpu().numpy() - lh_ref)) <= LOSS_TOL
+    # the two-kernel form gives the same bits
+    ctx.set_persistent(False)
+    w2 = torch.zeros(wl.n, device="cuda")
+    b2 = torch.zeros(1, device="cuda")
+    ctx.fit(dXh, dy, wl.lr, iters, w2, b2)
+    ctx.set_persistent(True)
+    assert torch.equal(w, w2) and torch.equal(b, b2)
+    # predict at two thresholds; rows within fp32 noise of the cut may fall on either side
+    for thr in (0.5, 0.3):
+        lab_ref, z = oracle.predict(Xv, w.cpu().numpy().astype(np.float64), float(b.item()), thr, return_z=True)
+        lab = ctx.predict(dXh, w, b, thr).cpu().numpy()
+        cut = np.log(thr / (1 - thr))
+        clear = np.abs(z - cut) > 1e-4 * (1.0 + np.abs(z))
+        assert np.array_equal(lab[clear], lab_ref[clear])
+        assert (lab == lab_ref).mean() >= LABEL_AGREE
+
+
+def test_wide_rows_fit(ctx):
+    # the wide-row kernel iterates as two kernels per step
+    wl = datagen.scaled(datagen.WORKLOADS["cfg4"], 3_000)
+    X, y, _, _ = datagen.generate(wl)
+    bits, Xv = oracle.round_bf16(X)
+    iters = 8
+    w_ref, b_ref, lh_ref = oracle.fit(Xv, y, wl.lr, iters)
+    hist = torch.empty(iters, dtype=torch.float32, device="cuda")
+    w = torch.zeros(wl.n, device="cuda")
+    b = torch.zeros(1, device="cuda")
+    ctx.fit(dev_bf16(bits), dev(y), wl.lr, iters, w, b, hist)
+    # this workload is not a contraction (the iterates oscillate), so early iterates are compared, loosely on w
+    assert np.max(np.abs(hist.cpu().numpy()[:3] - lh_ref[:3])) <= 1e-5 * max(1.0, float(np.max(lh_ref[:3])))
+    assert rel_l2(np.concatenate([w.cpu().numpy(), b.cpu().numpy()]), np.concatenate([w_ref, [b_ref]])) <= 1e-2
+
+
+def test_argument_checks(ctx):
+    Xh = torch.zeros((16, 8), dtype=torch.bfloat16, device="cuda")
+    y = torch.zeros(16, device="cuda")
+    w = torch.zeros(8, device="cuda")
+    b = torch.zeros(1, device="cuda")
+    L = api.lib()
+    import ctypes
+    P = lambda t: ctypes.c_void_p(t.data_ptr() if t is not None else None)
+    out = torch.zeros(10, device="cuda")
+    assert L.lr_loss_grad_bf16(ctx._h, None, P(y), 16, 8, P(w), P(b), P(out), P(out[1:]), P(out[9:]), None) == api.LR_ERR_NULL
+    assert L.lr_loss_grad_bf16(ctx._h, ctypes.c_void_p(Xh.data_ptr() + 1), P(y), 16, 8, P(w), P(b), P(out), P(out[1:]),
+                               P(out[9:]), None) == api.LR_ERR_ALIGNMENT
+    assert L.lr_fit_bf16(ctx._h, P(Xh), P(y), 16, 9000, 0.1, 1, P(w), P(b), None, None) == api.LR_ERR_SHAPE
+    assert L.lr_predict_bf16(ctx._h, P(Xh), 16, 8, P(w), P(b), 1.5, P(out), None) == api.LR_ERR_VALUE
+    assert L.lr_convert_bf16(ctx._h, P(out), -1, P(Xh), None) == api.LR_ERR_SHAPE
