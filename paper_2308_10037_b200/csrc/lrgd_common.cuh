@@ -152,16 +152,157 @@ __device__ __forceinline__ void logistic_terms(float z, float y, float& err, flo
     loss = fmaxf(z, 0.0f) + log1pf(t) - y * z;
 }
 
+// ---- per-lane arithmetic on 16-byte groups of X ----
+// A lane owns NV groups of a row.  Lane<NV> keeps that lane's slice of w and its fp32 gradient accumulators in the form
+// the storage type's arithmetic wants, and offers: load_w, zero, dot (this lane's part of x.w for one row), accumulate
+// (acc += x * err for one row) and fold (acc added into fp64 partners and cleared).
+
+// fp32 storage: four values per group, plain scalar FMAs in element order.
+template <int NV>
+struct LaneF32 {
+    static constexpr int EPG = 4;
+    float wv[NV][4];
+    float acc[NV][4];
+    // wv[k][c] = w[4*(first_group + k*group_stride) + c] for groups below group_limit, else 0 (w needs no alignment)
+    __device__ __forceinline__ void load_w(const float* w, int first_group, int group_stride, int group_limit, bool through_l2) {
+#pragma unroll
+        for (int k = 0; k < NV; ++k) {
+            const int idx = first_group + k * group_stride;
+#pragma unroll
+            for (int c = 0; c < 4; ++c)
+                wv[k][c] = idx < group_limit ? (through_l2 ? __ldcg(w + 4 * idx + c) : __ldg(w + 4 * idx + c)) : 0.f;
+        }
+    }
+    __device__ __forceinline__ void zero() {
+#pragma unroll
+        for (int k = 0; k < NV; ++k)
+#pragma unroll
+            for (int c = 0; c < 4; ++c) acc[k][c] = 0.f;
+    }
+    __device__ __forceinline__ float dot(const uint4 (&xr)[NV]) const {
+        float d = 0.f;
+#pragma unroll
+        for (int k = 0; k < NV; ++k) {
+            d = fmaf(__uint_as_float(xr[k].x), wv[k][0], d);
+            d = fmaf(__uint_as_float(xr[k].y), wv[k][1], d);
+            d = fmaf(__uint_as_float(xr[k].z), wv[k][2], d);
+            d = fmaf(__uint_as_float(xr[k].w), wv[k][3], d);
+        }
+        return d;
+    }
+    __device__ __forceinline__ void accumulate(const uint4 (&xr)[NV], float er) {
+#pragma unroll
+        for (int k = 0; k < NV; ++k) {
+            acc[k][0] = fmaf(__uint_as_float(xr[k].x), er, acc[k][0]);
+            acc[k][1] = fmaf(__uint_as_float(xr[k].y), er, acc[k][1]);
+            acc[k][2] = fmaf(__uint_as_float(xr[k].z), er, acc[k][2]);
+            acc[k][3] = fmaf(__uint_as_float(xr[k].w), er, acc[k][3]);
+        }
+    }
+    __device__ __forceinline__ void fold(double (&dacc)[NV][4]) {
+#pragma unroll
+        for (int k = 0; k < NV; ++k)
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                dacc[k][c] += acc[k][c];
+                acc[k][c] = 0.f;
+            }
+    }
+};
+
+// Two fp32 values in one 64-bit register, and the packed fused multiply-add on such pairs (fma.rn.f32x2, sm_100):
+// each half is an ordinary round-to-nearest fp32 FMA, so a pair of independent accumulators costs one instruction.
+__device__ __forceinline__ uint64_t f32x2_pack(float lo, float hi) {
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void f32x2_unpack(uint64_t v, float& lo, float& hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t f32x2_fma(uint64_t a, uint64_t b, uint64_t c) {
+    uint64_t d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+
+// bfloat16 storage: eight values per group, two per 32-bit word (element 2j in the low half).  bfloat16 is the upper
+// half of a binary32 pattern, so widening is exact: low element = word << 16, high element = word & 0xffff0000.  The
+// widened pair goes straight into a packed FMA against the matching pair of w (dot) or against (err, err)
+// (accumulate).  The dot product therefore runs as two chains (even and odd columns) that are added at the end.
+template <int NV>
+struct LaneBF16 {
+    static constexpr int EPG = 8;
+    uint64_t wv[NV][4];                  // (w[8g + 2j], w[8g + 2j + 1])
+    uint64_t acc[NV][4];                 // accumulators of the same column pairs
+    static __device__ __forceinline__ uint64_t widen(uint32_t word) {
+        return f32x2_pack(__uint_as_float(word << 16), __uint_as_float(word & 0xffff0000u));
+    }
+    __device__ __forceinline__ void load_w(const float* w, int first_group, int group_stride, int group_limit, bool through_l2) {
+#pragma unroll
+        for (int k = 0; k < NV; ++k) {
+            const int idx = first_group + k * group_stride;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                float lo = 0.f, hi = 0.f;
+                if (idx < group_limit) {
+                    lo = through_l2 ? __ldcg(w + 8 * idx + 2 * j) : __ldg(w + 8 * idx + 2 * j);
+                    hi = through_l2 ? __ldcg(w + 8 * idx + 2 * j + 1) : __ldg(w + 8 * idx + 2 * j + 1);
+                }
+                wv[k][j] = f32x2_pack(lo, hi);
+            }
+        }
+    }
+    __device__ __forceinline__ void zero() {
+#pragma unroll
+        for (int k = 0; k < NV; ++k)
+#pragma unroll
+            for (int j = 0; j < 4; ++j) acc[k][j] = 0ull;
+    }
+    __device__ __forceinline__ float dot(const uint4 (&xr)[NV]) const {
+        uint64_t d = 0ull;
+#pragma unroll
+        for (int k = 0; k < NV; ++k) {
+            d = f32x2_fma(widen(xr[k].x), wv[k][0], d);
+            d = f32x2_fma(widen(xr[k].y), wv[k][1], d);
+            d = f32x2_fma(widen(xr[k].z), wv[k][2], d);
+            d = f32x2_fma(widen(xr[k].w), wv[k][3], d);
+        }
+        float even, odd;
+        f32x2_unpack(d, even, odd);
+        return even + odd;
+    }
+    __device__ __forceinline__ void accumulate(const uint4 (&xr)[NV], float er) {
+        const uint64_t e2 = f32x2_pack(er, er);
+#pragma unroll
+        for (int k = 0; k < NV; ++k) {
+            acc[k][0] = f32x2_fma(widen(xr[k].x), e2, acc[k][0]);
+            acc[k][1] = f32x2_fma(widen(xr[k].y), e2, acc[k][1]);
+            acc[k][2] = f32x2_fma(widen(xr[k].z), e2, acc[k][2]);
+            acc[k][3] = f32x2_fma(widen(xr[k].w), e2, acc[k][3]);
+        }
+    }
+    __device__ __forceinline__ void fold(double (&dacc)[NV][8]) {
+#pragma unroll
+        for (int k = 0; k < NV; ++k)
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                float lo, hi;
+                f32x2_unpack(acc[k][j], lo, hi);
+                dacc[k][2 * j] += lo;
+                dacc[k][2 * j + 1] += hi;
+                acc[k][j] = 0ull;
+            }
+    }
+};
+
 // Storage types of X.  A "group" is 16 bytes of a row -- the unit of every shared-memory load and of the column
-// ownership of a lane: four fp32 values or eight bfloat16 values (bfloat16 = the upper half of a binary32 pattern,
-// so widening is exact: the pattern moves to the upper 16 bits).  All arithmetic is fp32 for both.
+// ownership of a lane: four fp32 values or eight bfloat16 values.  All arithmetic is fp32 for both.
 struct ElemF32 {
     static constexpr int EPG = 4;        // elements per 16-byte group
     static constexpr int BYTES = 4;      // bytes per element
-    static __device__ __forceinline__ void unpack(const uint4& g, float (&f)[4]) {
-        f[0] = __uint_as_float(g.x); f[1] = __uint_as_float(g.y);
-        f[2] = __uint_as_float(g.z); f[3] = __uint_as_float(g.w);
-    }
+    template <int NV>
+    using Lane = LaneF32<NV>;
     static __device__ __forceinline__ float load(const void* base, long long i) {
         return reinterpret_cast<const float*>(base)[i];
     }
@@ -169,12 +310,8 @@ struct ElemF32 {
 struct ElemBF16 {
     static constexpr int EPG = 8;
     static constexpr int BYTES = 2;
-    static __device__ __forceinline__ void unpack(const uint4& g, float (&f)[8]) {
-        f[0] = __uint_as_float(g.x << 16); f[1] = __uint_as_float(g.x & 0xffff0000u);
-        f[2] = __uint_as_float(g.y << 16); f[3] = __uint_as_float(g.y & 0xffff0000u);
-        f[4] = __uint_as_float(g.z << 16); f[5] = __uint_as_float(g.z & 0xffff0000u);
-        f[6] = __uint_as_float(g.w << 16); f[7] = __uint_as_float(g.w & 0xffff0000u);
-    }
+    template <int NV>
+    using Lane = LaneBF16<NV>;
     static __device__ __forceinline__ float load(const void* base, long long i) {
         return __uint_as_float(static_cast<uint32_t>(reinterpret_cast<const unsigned short*>(base)[i]) << 16);
     }

@@ -157,17 +157,17 @@ __global__ void __launch_bounds__(NW * 32, 1) k_fit_rows(const FitParams p) {
     bool alive = true;                             // CTA-uniform after every grid barrier
 
     for (int t = 0; t < p.iters && alive; ++t) {
-        float wv[NV][EPG];
-        load_w_slice<NV, EPG>(wv, p.w, sub, LPR, n4, true);
+        typename E::template Lane<NV> lm;          // this lane's slice of the current w and its fp32 accumulators
+        lm.load_w(p.w, sub, LPR, n4, true);
+        lm.zero();
         const float bval = __ldcg(p.b);
-        float acc[NV][EPG];
         double dacc[NV][EPG];
         float se = 0.f, sl = 0.f;
         double dse = 0.0, dsl = 0.0;
 #pragma unroll
         for (int k = 0; k < NV; ++k)
 #pragma unroll
-            for (int c = 0; c < EPG; ++c) { acc[k][c] = 0.f; dacc[k][c] = 0.0; }
+            for (int c = 0; c < EPG; ++c) dacc[k][c] = 0.0;
         int since_flush = 0;
         long long row0 = first_row;
         float y_next = (cnt > 0 && row0 + myr < p.m) ? __ldg(p.y + row0 + myr) : 0.f;
@@ -202,15 +202,15 @@ __global__ void __launch_bounds__(NW * 32, 1) k_fit_rows(const FitParams p) {
             }
             if (++d == D) { d = 0; phase ^= 1u; }
 
-            const float z = batch_dot<E, NV, LPR, RB>(x, wv, lane) + bval;
+            const float z = batch_dot<E, NV, LPR, RB>(x, lm, lane) + bval;
             float e, L;
             logistic_terms(z, yv, e, L);
             if (!myvalid) { e = 0.f; L = 0.f; }
             if (owner) { se += e; sl += L; }
-            batch_accumulate<E, NV, LPR, RB>(x, e, acc);
+            batch_accumulate<E, NV, LPR, RB>(x, e, lm);
             if (++since_flush == kFlushBatches) {
                 since_flush = 0;
-                fold_into_fp64<NV, EPG>(acc, dacc, se, sl, dse, dsl);
+                fold_into_fp64<E, NV>(lm, dacc, se, sl, dse, dsl);
             }
             row0 += stride_rows;
         }
@@ -232,7 +232,7 @@ __global__ void __launch_bounds__(NW * 32, 1) k_fit_rows(const FitParams p) {
             }
         }
 
-        fold_into_fp64<NV, EPG>(acc, dacc, se, sl, dse, dsl);
+        fold_into_fp64<E, NV>(lm, dacc, se, sl, dse, dsl);
 
         // ---- fixed-order combine of the CTA's warps, kFitCombineCols columns at a time (the stages stay in use) ----
         // row slots of one warp that own the same columns: add in slot order (as k_stream_rows does)

@@ -76,66 +76,31 @@ __device__ __forceinline__ void lane_reduce(float (&v)[RB], int lane) {
 // z partials: lane-local FMAs, then the transposing reduction; the returned value is the full dot product of the row
 // (r, with r = (lane_in_group >> (log2 LPR - log2 RB)) & (RB-1)) that ends up on this lane.
 template <class E, int NV, int LPR, int RB>
-__device__ __forceinline__ float batch_dot(const uint4 (&x)[RB][NV], const float (&wv)[NV][E::EPG], int lane) {
+__device__ __forceinline__ float batch_dot(const uint4 (&x)[RB][NV], const typename E::template Lane<NV>& lm, int lane) {
     float v[RB];
 #pragma unroll
-    for (int r = 0; r < RB; ++r) {
-        float dot = 0.f;
-#pragma unroll
-        for (int k = 0; k < NV; ++k) {
-            float xf[E::EPG];
-            E::unpack(x[r][k], xf);
-#pragma unroll
-            for (int c = 0; c < E::EPG; ++c) dot = fmaf(xf[c], wv[k][c], dot);
-        }
-        v[r] = dot;
-    }
+    for (int r = 0; r < RB; ++r) v[r] = lm.dot(x[r]);
     lane_reduce<RB, LPR / 2, RB>(v, lane);
     return v[0];
 }
 
 // acc[c] += x[r][c] * err[r]: each row's err is fetched from the lane that holds it (Algorithm 1's err.X on registers).
 template <class E, int NV, int LPR, int RB>
-__device__ __forceinline__ void batch_accumulate(const uint4 (&x)[RB][NV], float e, float (&acc)[NV][E::EPG]) {
+__device__ __forceinline__ void batch_accumulate(const uint4 (&x)[RB][NV], float e, typename E::template Lane<NV>& lm) {
     constexpr int SHIFT = Log2<LPR>::value - Log2<RB>::value;
 #pragma unroll
     for (int r = 0; r < RB; ++r) {
         const float er = __shfl_sync(0xffffffffu, e, r << SHIFT, LPR);
-#pragma unroll
-        for (int k = 0; k < NV; ++k) {
-            float xf[E::EPG];
-            E::unpack(x[r][k], xf);
-#pragma unroll
-            for (int c = 0; c < E::EPG; ++c) acc[k][c] = fmaf(xf[c], er, acc[k][c]);
-        }
+        lm.accumulate(x[r], er);
     }
 }
 
 // fp32 per-lane sums folded into their fp64 counterparts (keeps the serial fp32 chains short)
-template <int NV, int EPG>
-__device__ __forceinline__ void fold_into_fp64(float (&acc)[NV][EPG], double (&dacc)[NV][EPG], float& se, float& sl,
+template <class E, int NV>
+__device__ __forceinline__ void fold_into_fp64(typename E::template Lane<NV>& lm, double (&dacc)[NV][E::EPG], float& se, float& sl,
                                                double& dse, double& dsl) {
-#pragma unroll
-    for (int k = 0; k < NV; ++k)
-#pragma unroll
-        for (int c = 0; c < EPG; ++c) {
-            dacc[k][c] += acc[k][c];
-            acc[k][c] = 0.f;
-        }
+    lm.fold(dacc);
     dse += se; dsl += sl; se = 0.f; sl = 0.f;
-}
-
-// this lane's slice of w, widened per group: wv[k][c] = w[EPG*(sub + k*LPR) + c] (zero past the row; w needs no alignment)
-template <int NV, int EPG>
-__device__ __forceinline__ void load_w_slice(float (&wv)[NV][EPG], const float* w, int first_group, int group_stride, int ng,
-                                             bool through_l2) {
-#pragma unroll
-    for (int k = 0; k < NV; ++k) {
-        const int idx = first_group + k * group_stride;
-#pragma unroll
-        for (int c = 0; c < EPG; ++c)
-            wv[k][c] = idx < ng ? (through_l2 ? __ldcg(w + EPG * idx + c) : __ldg(w + EPG * idx + c)) : 0.f;
-    }
 }
 
 // one batch from a narrow-row stage into registers (rows packed at n4 groups; lanes beyond the row or rows beyond the
@@ -214,18 +179,17 @@ __global__ void __launch_bounds__(NW * 32, 1) k_stream_rows(const StreamParams p
                       r0 < p.keep_rows ? pol_keep : pol_stream);
     };
 
-    float acc[NV][EPG];
+    typename E::template Lane<NV> lm;              // this lane's slice of w and its fp32 accumulators
     double dacc[NV][EPG];
     float se = 0.f, sl = 0.f;
     double dse = 0.0, dsl = 0.0;
+    lm.zero();
 #pragma unroll
     for (int k = 0; k < NV; ++k)
 #pragma unroll
-        for (int c = 0; c < EPG; ++c) { acc[k][c] = 0.f; dacc[k][c] = 0.0; }
+        for (int c = 0; c < EPG; ++c) dacc[k][c] = 0.0;
     const int sub = lane & (LPR - 1), slot = lane >> LOG_LPR;
-
-    float wv[NV][EPG];                             // this lane's slice of w
-    load_w_slice<NV, EPG>(wv, p.w, sub, LPR, n4, false);
+    lm.load_w(p.w, sub, LPR, n4, false);
     const float bval = __ldg(p.b);
     const int myr = ((sub >> SHIFT) & (RB - 1)) * RPW + slot;     // the row of a batch whose logit ends up on this lane
     const bool owner = (sub & ((1 << SHIFT) - 1)) == 0;           // one lane per row does the bookkeeping
@@ -274,7 +238,7 @@ __global__ void __launch_bounds__(NW * 32, 1) k_stream_rows(const StreamParams p
         }
         if (++d == D) { d = 0; phase ^= 1u; }
 
-        const float z = batch_dot<E, NV, LPR, RB>(x, wv, lane) + bval;
+        const float z = batch_dot<E, NV, LPR, RB>(x, lm, lane) + bval;
 
         if constexpr (PREDICT) {
             // one bit per lane, then RPB/4 lanes each assemble and store four labels as one 32-bit word
@@ -298,10 +262,10 @@ __global__ void __launch_bounds__(NW * 32, 1) k_stream_rows(const StreamParams p
             logistic_terms(z, yv, e, L);
             if (!myvalid) { e = 0.f; L = 0.f; }
             if (owner) { se += e; sl += L; }
-            batch_accumulate<E, NV, LPR, RB>(x, e, acc);
+            batch_accumulate<E, NV, LPR, RB>(x, e, lm);
             if (++since_flush == kFlushBatches) {
                 since_flush = 0;
-                fold_into_fp64<NV, EPG>(acc, dacc, se, sl, dse, dsl);
+                fold_into_fp64<E, NV>(lm, dacc, se, sl, dse, dsl);
             }
         }
         row0 += stride_rows;
@@ -317,7 +281,7 @@ __global__ void __launch_bounds__(NW * 32, 1) k_stream_rows(const StreamParams p
         __syncwarp();
     }
     if constexpr (!PREDICT) {
-        fold_into_fp64<NV, EPG>(acc, dacc, se, sl, dse, dsl);
+        fold_into_fp64<E, NV>(lm, dacc, se, sl, dse, dsl);
 
         // ---------------- fixed-order combine of the CTA's warps ----------------
         __syncthreads();                               // all stages are idle: reuse them as the combine buffer

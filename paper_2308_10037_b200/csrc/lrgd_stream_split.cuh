@@ -94,22 +94,16 @@ __global__ void __launch_bounds__(NW * 32, 1) k_stream_split(const __grid_consta
                            r0 < p.keep_rows ? pol_keep : pol_stream);
     };
 
-    float acc[NV][EPG];
+    typename E::template Lane<NV> lm;              // this lane's slice of w (groups c0 + lane + 32k) and its fp32 accumulators
     double dacc[NV][EPG];
     float se = 0.f, sl = 0.f;
     double dse = 0.0, dsl = 0.0;
-    float wv[NV][EPG];
+    lm.zero();
+    lm.load_w(p.w, c0 + lane, 32, c0 + mycw, false);
 #pragma unroll
-    for (int k = 0; k < NV; ++k) {
-        const int loc = lane + 32 * k;
-        const int idx = c0 + loc;
+    for (int k = 0; k < NV; ++k)
 #pragma unroll
-        for (int c = 0; c < EPG; ++c) {
-            acc[k][c] = 0.f;
-            dacc[k][c] = 0.0;
-            wv[k][c] = loc < mycw ? __ldg(p.w + EPG * idx + c) : 0.f;
-        }
-    }
+        for (int c = 0; c < EPG; ++c) dacc[k][c] = 0.0;
     const float bval = __ldg(p.b);
     const int myr = (lane >> SHIFT) & (RB - 1);    // the row of a batch whose logit ends up on this lane
     const int dup = lane & (DUP - 1);              // which of the lanes sharing that row this one is
@@ -184,7 +178,7 @@ __global__ void __launch_bounds__(NW * 32, 1) k_stream_split(const __grid_consta
                 for (int k = 0; k < NV; ++k) x[r][k] = make_uint4(0u, 0u, 0u, 0u);
         }
 
-        const float zpartial = batch_dot<E, NV, 32, RB>(x, wv, lane);
+        const float zpartial = batch_dot<E, NV, 32, RB>(x, lm, lane);
         float* zp = zpart + (i & 1) * (NW * RB);
         if (owner) zp[warp * RB + myr] = zpartial;
         __syncthreads();
@@ -220,10 +214,10 @@ __global__ void __launch_bounds__(NW * 32, 1) k_stream_split(const __grid_consta
                 e = logistic_err(z, yv);
             }
             if (!myvalid) e = 0.f;
-            batch_accumulate<E, NV, 32, RB>(x, e, acc);
+            batch_accumulate<E, NV, 32, RB>(x, e, lm);
             if (++since_flush == 2 * kFlushBatches) {
                 since_flush = 0;
-                fold_into_fp64<NV, EPG>(acc, dacc, se, sl, dse, dsl);
+                fold_into_fp64<E, NV>(lm, dacc, se, sl, dse, dsl);
             }
         }
         row0 += stride_rows;
@@ -239,17 +233,17 @@ __global__ void __launch_bounds__(NW * 32, 1) k_stream_split(const __grid_consta
     }
     if constexpr (!PREDICT) {
         double* out = p.partial + static_cast<size_t>(blockIdx.x) * (n + 2);
+        fold_into_fp64<E, NV>(lm, dacc, se, sl, dse, dsl);
 #pragma unroll
         for (int k = 0; k < NV; ++k) {
             const int loc = lane + 32 * k;
             if (loc < mycw) {
                 const int col = EPG * (c0 + loc);
 #pragma unroll
-                for (int c = 0; c < EPG; ++c) out[col + c] = dacc[k][c] + acc[k][c];
+                for (int c = 0; c < EPG; ++c) out[col + c] = dacc[k][c];
             }
         }
         if (warp == 0) {
-            dse += se; dsl += sl;
 #pragma unroll
             for (int msk = 16; msk >= 1; msk >>= 1) {
                 dse += __shfl_xor_sync(FULL, dse, msk);
