@@ -8,6 +8,7 @@ namespace lrgd {
 
 constexpr int kStatusTimeout = -6;                 // LR_ERR_TIMEOUT
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s per wait, then the kernel gives up
+constexpr unsigned long long kDrainLimitNs = 500000000ull;   // 0.5 s per copy still in flight when a CTA winds down
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
     return static_cast<uint32_t>(__cvta_generic_to_shared(p));
@@ -73,6 +74,19 @@ __device__ __forceinline__ bool mbar_wait_bounded_ns(uint64_t* bar, uint32_t par
 
 __device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
     return mbar_wait_bounded_ns(bar, parity, abort_flag, kWaitLimitNs);
+}
+
+// Wait used when a CTA winds down with copies of its own still in flight: it does not look at the abort flag (which
+// is what ends the run), only at the clock, so that the copies really land before the shared memory is given up.
+__device__ __forceinline__ bool mbar_wait_drain(uint64_t* bar, uint32_t parity) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const unsigned long long t0 = global_timer_ns();
+    for (;;) {
+#pragma unroll 1
+        for (int i = 0; i < 32; ++i)
+            if (mbar_try_wait(bar, parity)) return true;
+        if (global_timer_ns() - t0 > kDrainLimitNs) return false;
+    }
 }
 
 // One warp waits on an mbarrier that is completed up front (arm != 0) or never (arm == 0), with the given limit; on

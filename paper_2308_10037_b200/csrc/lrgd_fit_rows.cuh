@@ -112,7 +112,7 @@ __global__ void __launch_bounds__(NW * 32, 1) k_fit_rows(const FitParams p) {
     const long long B = p.num_batches;
     const long long Bw = B > warp ? (B - warp + NW - 1) / NW : 0;
     const int cnt = Bw > blockIdx.x ? static_cast<int>((Bw - blockIdx.x + G - 1) / G) : 0;    // batches of this warp per iteration
-    const long long fills_total = static_cast<long long>(cnt) * p.iters;                       // stage fills over the whole fit
+    const int fill_iters = cnt > 0 ? p.iters : 0;  // the fit is cnt * fill_iters stage fills for this warp, iteration-major
 
     if (threadIdx.x == 0) *abort_flag = 0;
     if (lane == 0) {
@@ -139,17 +139,18 @@ __global__ void __launch_bounds__(NW * 32, 1) k_fit_rows(const FitParams p) {
     const bool owner = (sub & ((1 << SHIFT) - 1)) == 0;
     const bool full_cols = n4 == NV * LPR;
 
-    // the fit is one long sequence of fills (iteration-major); fill f lands in stage f % D
-    long long issued = 0;                          // fills whose copy has been issued (warp-uniform)
-    long long consumed = 0;                        // fills whose wait has succeeded
-    int issue_i = 0;                               // batch index (within an iteration) of the next fill to issue
-    {
-        const long long pre = fills_total < D ? fills_total : D;
-        for (long long f = 0; f < pre; ++f) {
-            if (lane == 0) issue(first_row + issue_i * stride_rows, static_cast<int>(f));
-            if (++issue_i == cnt) issue_i = 0;
-        }
-        issued = pre;
+    // the fit is one long sequence of fills (iteration-major); consecutive fills land in consecutive stages (mod D)
+    int issue_i = 0, issue_t = 0;                  // batch index and iteration of the next fill to issue (warp-uniform)
+    long long issue_row = first_row;               // its first row
+    int inflight = 0;                              // fills issued and not yet consumed
+    auto next_fill = [&]() {
+        issue_row += stride_rows;
+        if (++issue_i == cnt) { issue_i = 0; issue_row = first_row; ++issue_t; }
+    };
+    for (int f = 0; f < D && issue_t < fill_iters; ++f) {
+        if (lane == 0) issue(issue_row, f);
+        next_fill();
+        ++inflight;
     }
     int d = 0;
     uint32_t phase = 0;
@@ -177,7 +178,6 @@ __global__ void __launch_bounds__(NW * 32, 1) k_fit_rows(const FitParams p) {
             bool ok = mbar_wait_bounded(&my_bars[d], phase, abort_flag);
             ok = __all_sync(FULL, ok);
             if (!ok) { warp_ok = false; break; }
-            consumed += 1;
 
             const long long left = p.m - row0;
             const int rows = left < RPB ? static_cast<int>(left) : RPB;
@@ -192,13 +192,14 @@ __global__ void __launch_bounds__(NW * 32, 1) k_fit_rows(const FitParams p) {
             }
             // re-arm the stage with the fill `depth` ahead in the fit-long sequence (possibly of the next iteration)
             __syncwarp();
-            if (issued < fills_total) {
+            if (issue_t < fill_iters) {
                 if (lane == 0) {
                     fence_proxy_async_smem();
-                    issue(first_row + issue_i * stride_rows, d);
+                    issue(issue_row, d);
                 }
-                if (++issue_i == cnt) issue_i = 0;
-                issued += 1;
+                next_fill();
+            } else {
+                --inflight;
             }
             if (++d == D) { d = 0; phase ^= 1u; }
 
@@ -337,10 +338,12 @@ __global__ void __launch_bounds__(NW * 32, 1) k_fit_rows(const FitParams p) {
     if (!alive || *abort_flag) {
         if (lane == 0) atomicExch(p.status, kStatusTimeout);
     }
-    if (consumed < issued) {
+    if (inflight > 0) {
         if (lane == 0) {
-            for (long long f = consumed; f < issued; ++f)
-                mbar_wait_bounded(&my_bars[f % D], static_cast<uint32_t>(f / D) & 1u, abort_flag);
+            for (int f = 0; f < inflight; ++f) {           // the oldest fill in flight sits in stage d, phase parity `phase`
+                mbar_wait_drain(&my_bars[d], phase);
+                if (++d == D) { d = 0; phase ^= 1u; }
+            }
         }
         __syncwarp();
     }

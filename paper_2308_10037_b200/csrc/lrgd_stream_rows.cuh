@@ -276,7 +276,7 @@ __global__ void __launch_bounds__(NW * 32, 1) k_stream_rows(const StreamParams p
         // before the CTA retires and its shared memory is handed to another CTA
         if (lane == 0) {
             atomicExch(p.status, kStatusTimeout);
-            for (int i = done; i < issued; ++i) mbar_wait_bounded(&my_bars[i % D], static_cast<uint32_t>(i / D) & 1u, abort_flag);
+            for (int i = done; i < issued; ++i) mbar_wait_drain(&my_bars[i % D], static_cast<uint32_t>(i / D) & 1u);
         }
         __syncwarp();
     }

@@ -185,3 +185,44 @@ def test_argument_checks(ctx):
     assert L.lr_fit_bf16(ctx._h, P(Xh), P(y), 16, 9000, 0.1, 1, P(w), P(b), None, None) == api.LR_ERR_SHAPE
     assert L.lr_predict_bf16(ctx._h, P(Xh), 16, 8, P(w), P(b), 1.5, P(out), None) == api.LR_ERR_VALUE
     assert L.lr_convert_bf16(ctx._h, P(out), -1, P(Xh), None) == api.LR_ERR_SHAPE
+
+
+@pytest.mark.parametrize("name", ["cfg3", "cfg5"])
+def test_full_size_workload_bf16(ctx, name):
+    """The benchmark's bfloat16 runs at full size: conversion on the device, the workload's own fit, labels."""
+    wl = datagen.WORKLOADS[name]
+    X, y, _, _ = datagen.generate(wl)
+    dX32 = torch.from_numpy(X).cuda()
+    dXh = ctx.convert_bf16(dX32)
+    del dX32
+    bits, Xv = oracle.round_bf16(X)
+    del X
+    # conversion: bit-exact on a strided sample of rows plus the last rows (largest offsets)
+    got_bits = dXh.view(torch.int16)
+    for sl in (slice(0, wl.m, 997), slice(wl.m - 4096, wl.m)):
+        assert np.array_equal(got_bits[sl].cpu().numpy().view(np.uint16), bits[sl])
+    del bits
+    dy = dev(y)
+    iters = wl.iters
+    hist = torch.empty(iters, dtype=torch.float32, device="cuda")
+    w = torch.zeros(wl.n, device="cuda")
+    b = torch.zeros(1, device="cuda")
+    ctx.fit(dXh, dy, wl.lr, iters, w, b, hist)
+    torch.cuda.synchronize()
+    w_ref, b_ref, hist_ref, wh, bh = oracle.fit(Xv, y, wl.lr, iters, history=True)
+    assert rel_l2(np.concatenate([w.cpu().numpy(), b.cpu().numpy()]), np.concatenate([w_ref, [b_ref]])) <= W_TOL
+    assert np.max(np.abs(hist.cpu().numpy().astype(np.float64) - hist_ref)) <= LOSS_TOL
+    floor = grad_noise_floor(Xv)
+    for t in sorted({0, 1, iters // 2, iters - 1}):
+        w32, b32 = wh[t].astype(np.float32), np.float32(bh[t])
+        L, g, g0 = oracle.loss_grad(Xv, y, w32.astype(np.float64), float(b32))
+        dl, dg, dg0 = ctx.loss_grad(dXh, dy, dev(w32), dev(np.array([b32])))
+        assert abs(dl.item() - L) <= LOSS_TOL, (name, t)
+        assert_grad_close(np.concatenate([dg.cpu().numpy(), dg0.cpu().numpy()]), np.concatenate([g, [g0]]), floor, (name, t))
+    w32, b32 = w_ref.astype(np.float32), np.float32(b_ref)
+    for thr in ([0.5] + ([0.05] if name == "cfg5" else [])):
+        labels = ctx.predict(dXh, dev(w32), dev(np.array([b32])), thr).cpu().numpy()
+        lab_ref = oracle.predict(Xv, w32.astype(np.float64), float(b32), thr)
+        assert (labels == lab_ref).mean() >= LABEL_AGREE, (name, thr)
+    del dXh
+    torch.cuda.empty_cache()
