@@ -169,60 +169,8 @@ __device__ __forceinline__ void logistic_terms(float z, float y, float& err, flo
 // ---- per-lane arithmetic on 16-byte groups of X ----
 // A lane owns NV groups of a row.  Lane<NV> keeps that lane's slice of w and its fp32 gradient accumulators in the form
 // the storage type's arithmetic wants, and offers: load_w, zero, dot (this lane's part of x.w for one row), accumulate
-// (acc += x * err for one row) and fold (acc added into fp64 partners and cleared).
-
-// fp32 storage: four values per group, plain scalar FMAs in element order.
-template <int NV>
-struct LaneF32 {
-    static constexpr int EPG = 4;
-    float wv[NV][4];
-    float acc[NV][4];
-    // wv[k][c] = w[4*(first_group + k*group_stride) + c] for groups below group_limit, else 0 (w needs no alignment)
-    __device__ __forceinline__ void load_w(const float* w, int first_group, int group_stride, int group_limit, bool through_l2) {
-#pragma unroll
-        for (int k = 0; k < NV; ++k) {
-            const int idx = first_group + k * group_stride;
-#pragma unroll
-            for (int c = 0; c < 4; ++c)
-                wv[k][c] = idx < group_limit ? (through_l2 ? __ldcg(w + 4 * idx + c) : __ldg(w + 4 * idx + c)) : 0.f;
-        }
-    }
-    __device__ __forceinline__ void zero() {
-#pragma unroll
-        for (int k = 0; k < NV; ++k)
-#pragma unroll
-            for (int c = 0; c < 4; ++c) acc[k][c] = 0.f;
-    }
-    __device__ __forceinline__ float dot(const uint4 (&xr)[NV]) const {
-        float d = 0.f;
-#pragma unroll
-        for (int k = 0; k < NV; ++k) {
-            d = fmaf(__uint_as_float(xr[k].x), wv[k][0], d);
-            d = fmaf(__uint_as_float(xr[k].y), wv[k][1], d);
-            d = fmaf(__uint_as_float(xr[k].z), wv[k][2], d);
-            d = fmaf(__uint_as_float(xr[k].w), wv[k][3], d);
-        }
-        return d;
-    }
-    __device__ __forceinline__ void accumulate(const uint4 (&xr)[NV], float er) {
-#pragma unroll
-        for (int k = 0; k < NV; ++k) {
-            acc[k][0] = fmaf(__uint_as_float(xr[k].x), er, acc[k][0]);
-            acc[k][1] = fmaf(__uint_as_float(xr[k].y), er, acc[k][1]);
-            acc[k][2] = fmaf(__uint_as_float(xr[k].z), er, acc[k][2]);
-            acc[k][3] = fmaf(__uint_as_float(xr[k].w), er, acc[k][3]);
-        }
-    }
-    __device__ __forceinline__ void fold(double (&dacc)[NV][4]) {
-#pragma unroll
-        for (int k = 0; k < NV; ++k)
-#pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                dacc[k][c] += acc[k][c];
-                acc[k][c] = 0.f;
-            }
-    }
-};
+// (acc += x * err for one row) and fold (acc added into fp64 partners and cleared).  Both storage types work on pairs
+// of adjacent columns held in 64-bit registers, so that one packed instruction does two fp32 FMAs.
 
 // Two fp32 values in one 64-bit register, and the packed fused multiply-add on such pairs (fma.rn.f32x2, sm_100):
 // each half is an ordinary round-to-nearest fp32 FMA, so a pair of independent accumulators costs one instruction.
@@ -239,6 +187,70 @@ __device__ __forceinline__ uint64_t f32x2_fma(uint64_t a, uint64_t b, uint64_t c
     asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
     return d;
 }
+
+// fp32 storage: four values per group; the group's (x, y) and (z, w) words are the two pairs of the packed FMAs, so
+// the dot product runs as two chains (even and odd columns) that are added at the end.
+template <int NV>
+struct LaneF32 {
+    static constexpr int EPG = 4;
+    uint64_t wv[NV][2];
+    uint64_t acc[NV][2];
+    __device__ __forceinline__ void load_w(const float* w, int first_group, int group_stride, int group_limit, bool through_l2) {
+#pragma unroll
+        for (int k = 0; k < NV; ++k) {
+            const int idx = first_group + k * group_stride;
+#pragma unroll
+            for (int j = 0; j < 2; ++j) {
+                float lo = 0.f, hi = 0.f;
+                if (idx < group_limit) {
+                    lo = through_l2 ? __ldcg(w + 4 * idx + 2 * j) : __ldg(w + 4 * idx + 2 * j);
+                    hi = through_l2 ? __ldcg(w + 4 * idx + 2 * j + 1) : __ldg(w + 4 * idx + 2 * j + 1);
+                }
+                wv[k][j] = f32x2_pack(lo, hi);
+            }
+        }
+    }
+    __device__ __forceinline__ void zero() {
+#pragma unroll
+        for (int k = 0; k < NV; ++k) { acc[k][0] = 0ull; acc[k][1] = 0ull; }
+    }
+    static __device__ __forceinline__ uint64_t pair(uint32_t a, uint32_t b) {
+        uint64_t r;
+        asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "r"(a), "r"(b));
+        return r;
+    }
+    __device__ __forceinline__ float dot(const uint4 (&xr)[NV]) const {
+        uint64_t d = 0ull;
+#pragma unroll
+        for (int k = 0; k < NV; ++k) {
+            d = f32x2_fma(pair(xr[k].x, xr[k].y), wv[k][0], d);
+            d = f32x2_fma(pair(xr[k].z, xr[k].w), wv[k][1], d);
+        }
+        float even, odd;
+        f32x2_unpack(d, even, odd);
+        return even + odd;
+    }
+    __device__ __forceinline__ void accumulate(const uint4 (&xr)[NV], float er) {
+        const uint64_t e2 = f32x2_pack(er, er);
+#pragma unroll
+        for (int k = 0; k < NV; ++k) {
+            acc[k][0] = f32x2_fma(pair(xr[k].x, xr[k].y), e2, acc[k][0]);
+            acc[k][1] = f32x2_fma(pair(xr[k].z, xr[k].w), e2, acc[k][1]);
+        }
+    }
+    __device__ __forceinline__ void fold(double (&dacc)[NV][4]) {
+#pragma unroll
+        for (int k = 0; k < NV; ++k)
+#pragma unroll
+            for (int j = 0; j < 2; ++j) {
+                float lo, hi;
+                f32x2_unpack(acc[k][j], lo, hi);
+                dacc[k][2 * j] += lo;
+                dacc[k][2 * j + 1] += hi;
+                acc[k][j] = 0ull;
+            }
+    }
+};
 
 // bfloat16 storage: eight values per group, two per 32-bit word (element 2j in the low half).  bfloat16 is the upper
 // half of a binary32 pattern, so widening is exact: low element = word << 16, high element = word & 0xffff0000.  The
