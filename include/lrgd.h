@@ -196,6 +196,21 @@ int lr_fit_bf16(lr_ctx* ctx, const uint16_t* d_Xh, const float* d_y, int64_t m, 
 int lr_predict_bf16(lr_ctx* ctx, const uint16_t* d_Xh, int64_t m, int32_t n,
                     const float* d_w, const float* d_b, float thr, uint8_t* d_labels, void* stream);
 int lr_plan_query_bf16(int64_t m, int32_t n, int32_t x_aligned16, int32_t sm_count, lr_plan* out);
+/* lr_fit_tol, lr_fit_opt, lr_fit_sgd and lr_shard_sums on a bfloat16-stored X: same contracts, same arithmetic, d_Xh as above
+ * (lr_fit_sgd_bf16's row blocks start at d_Xh + block*batch_rows*n; a block that does not start on a 16-byte boundary
+ * runs on the unstaged kernel).  lr_apply_sums is independent of the storage type. */
+int lr_fit_tol_bf16(lr_ctx* ctx, const uint16_t* d_Xh, const float* d_y, int64_t m, int32_t n,
+                    float lr, float eps, int32_t max_iters, int32_t check_every,
+                    float* d_w, float* d_b, float* d_loss_hist, float* d_gnorm_hist,
+                    int32_t* iters_done, float* grad_norm, void* stream);
+int lr_fit_opt_bf16(lr_ctx* ctx, const uint16_t* d_Xh, const float* d_y, int64_t m, int32_t n,
+                    float lr, int32_t iters, const lr_opt* opt,
+                    float* d_w, float* d_b, float* d_velocity, float* d_loss_hist, void* stream);
+int lr_fit_sgd_bf16(lr_ctx* ctx, const uint16_t* d_Xh, const float* d_y, int64_t m, int32_t n,
+                    float lr, int64_t batch_rows, int32_t steps, int64_t first_batch,
+                    float* d_w, float* d_b, float* d_loss_hist, void* stream);
+int lr_shard_sums_bf16(lr_ctx* ctx, const uint16_t* d_Xh, const float* d_y, int64_t m_local, int32_t n,
+                       const float* d_w, const float* d_b, double* d_sums, void* stream);
 
 /*
  * Row-sharded data parallelism (the natural split of Algorithm 1's sums over rows; the paper itself

@@ -22,7 +22,8 @@ EXPORTS = ["lr_plan_query", "lr_create", "lr_destroy", "lr_loss_grad", "lr_fit",
            "lr_apply_sums", "lr_fit_host",
            "lr_predict_host", "lr_profile_enable", "lr_profile_read", "lr_launch_count", "lr_last_device_status",
            "lr_last_cuda_error", "lr_status_string", "lr_loss_grad_noalloc", "lr_fit_tol", "lr_fit_opt", "lr_selftest_wait", "lr_set_persistent", "lr_fit_sgd", "lr_set_l2_keep",
-           "lr_convert_bf16", "lr_loss_grad_bf16", "lr_fit_bf16", "lr_predict_bf16", "lr_plan_query_bf16"]
+           "lr_convert_bf16", "lr_loss_grad_bf16", "lr_fit_bf16", "lr_predict_bf16", "lr_plan_query_bf16",
+           "lr_fit_tol_bf16", "lr_fit_opt_bf16", "lr_fit_sgd_bf16", "lr_shard_sums_bf16"]
 
 
 class LrPlan(ctypes.Structure):
@@ -73,6 +74,10 @@ def lib() -> ctypes.CDLL:
         L.lr_fit_opt.argtypes = [P, P, P, I64, I32, F, I32, ctypes.POINTER(LrOpt), P, P, P, P, P]
         L.lr_selftest_wait.argtypes = [P, I32, I32, P]
         L.lr_fit_sgd.argtypes = [P, P, P, I64, I32, F, I64, I32, I64, P, P, P, P]
+        L.lr_fit_tol_bf16.argtypes = L.lr_fit_tol.argtypes
+        L.lr_fit_opt_bf16.argtypes = L.lr_fit_opt.argtypes
+        L.lr_fit_sgd_bf16.argtypes = L.lr_fit_sgd.argtypes
+        L.lr_shard_sums_bf16.argtypes = L.lr_shard_sums.argtypes
         L.lr_set_persistent.argtypes = [P, I32]
         L.lr_set_l2_keep.argtypes = [P, I64]
         L.lr_loss_grad_noalloc.argtypes = [I32, P, P, I64, I32, P, P, P, P, P, P, P]
@@ -200,31 +205,34 @@ class Context:
         """GD until ||grad||_2 <= eps (at most ``max_iters`` updates), in place on w, b.  Returns (updates, last norm)."""
         m, n = X.shape
         done, nrm = ctypes.c_int32(), ctypes.c_float()
-        rc = lib().lr_fit_tol(self._h, _dev_ptr(X, torch.float32, "X"), _dev_ptr(y, torch.float32, "y"), m, n, float(lr),
+        xdt, sfx = self._x_kind(X)
+        rc = getattr(lib(), "lr_fit_tol" + sfx)(self._h, _dev_ptr(X, xdt, "X"), _dev_ptr(y, torch.float32, "y"), m, n, float(lr),
                               float(eps), int(max_iters), int(check_every), _dev_ptr(w, torch.float32, "w"),
                               _dev_ptr(b, torch.float32, "b"), _dev_ptr(loss_hist, torch.float32, "loss_hist"),
                               _dev_ptr(gnorm_hist, torch.float32, "gnorm_hist"), ctypes.byref(done), ctypes.byref(nrm),
                               self._stream())
-        self._check(rc, "lr_fit_tol")
+        self._check(rc, "lr_fit_tol" + sfx)
         return done.value, nrm.value
 
     def fit_opt(self, X, y, lr, iters, w, b, l2=0.0, momentum=0.0, nesterov=False, velocity=None, loss_hist=None):
         """GD with an L2 penalty and (Nesterov) momentum, in place on w, b (and ``velocity`` [n+1] when given)."""
         m, n = X.shape
         opt = LrOpt(float(l2), float(momentum), int(bool(nesterov)))
-        rc = lib().lr_fit_opt(self._h, _dev_ptr(X, torch.float32, "X"), _dev_ptr(y, torch.float32, "y"), m, n, float(lr),
+        xdt, sfx = self._x_kind(X)
+        rc = getattr(lib(), "lr_fit_opt" + sfx)(self._h, _dev_ptr(X, xdt, "X"), _dev_ptr(y, torch.float32, "y"), m, n, float(lr),
                               int(iters), ctypes.byref(opt), _dev_ptr(w, torch.float32, "w"), _dev_ptr(b, torch.float32, "b"),
                               _dev_ptr(velocity, torch.float32, "velocity"), _dev_ptr(loss_hist, torch.float32, "loss_hist"),
                               self._stream())
-        self._check(rc, "lr_fit_opt")
+        self._check(rc, "lr_fit_opt" + sfx)
 
     def fit_sgd(self, X, y, lr, batch_rows, steps, w, b, first_batch=0, loss_hist=None):
         """Mini-batch GD over contiguous row blocks (block (first_batch + s) mod count at step s), in place on w, b."""
         m, n = X.shape
-        rc = lib().lr_fit_sgd(self._h, _dev_ptr(X, torch.float32, "X"), _dev_ptr(y, torch.float32, "y"), m, n, float(lr),
+        xdt, sfx = self._x_kind(X)
+        rc = getattr(lib(), "lr_fit_sgd" + sfx)(self._h, _dev_ptr(X, xdt, "X"), _dev_ptr(y, torch.float32, "y"), m, n, float(lr),
                               int(batch_rows), int(steps), int(first_batch), _dev_ptr(w, torch.float32, "w"),
                               _dev_ptr(b, torch.float32, "b"), _dev_ptr(loss_hist, torch.float32, "loss_hist"), self._stream())
-        self._check(rc, "lr_fit_sgd")
+        self._check(rc, "lr_fit_sgd" + sfx)
 
     def predict(self, X, w, b, thr, out=None):
         m, n = X.shape
@@ -239,10 +247,11 @@ class Context:
     def shard_sums(self, X, y, w, b, sums):
         """Unnormalised fp64 sums [n+2] of the local rows into ``sums`` (float64 CUDA tensor)."""
         m, n = X.shape
-        rc = lib().lr_shard_sums(self._h, _dev_ptr(X, torch.float32, "X"), _dev_ptr(y, torch.float32, "y"), m, n,
+        xdt, sfx = self._x_kind(X)
+        rc = getattr(lib(), "lr_shard_sums" + sfx)(self._h, _dev_ptr(X, xdt, "X"), _dev_ptr(y, torch.float32, "y"), m, n,
                                  _dev_ptr(w, torch.float32, "w"), _dev_ptr(b, torch.float32, "b"),
                                  _dev_ptr(sums, torch.float64, "sums"), self._stream())
-        self._check(rc, "lr_shard_sums")
+        self._check(rc, "lr_shard_sums" + sfx)
 
     def apply_sums(self, sums_all, m_total, lr, w, b, loss=None):
         """Adds the ``parts`` rows of ``sums_all`` [parts, n+2] in order and applies the update to w, b in place."""

@@ -634,10 +634,14 @@ int lr_set_persistent(lr_ctx* ctx, int32_t on) {
     return LR_OK;
 }
 
-int lr_fit_tol(lr_ctx* ctx, const float* d_X, const float* d_y, int64_t m, int32_t n, float lr, float eps,
-               int32_t max_iters, int32_t check_every, float* d_w, float* d_b, float* d_loss_hist, float* d_gnorm_hist,
-               int32_t* iters_done, float* grad_norm, void* stream) {
-    int rc = check_common(ctx, d_X, m, n, d_w, d_b);
+}  // extern "C"
+
+namespace {
+
+int fit_tol_impl(lr_ctx* ctx, const void* d_X, bool bf16, const float* d_y, int64_t m, int32_t n, float lr, float eps,
+                 int32_t max_iters, int32_t check_every, float* d_w, float* d_b, float* d_loss_hist, float* d_gnorm_hist,
+                 int32_t* iters_done, float* grad_norm, void* stream) {
+    int rc = check_common(ctx, d_X, m, n, d_w, d_b, bf16);
     if (rc != LR_OK) return rc;
     if (!d_y || !iters_done || !grad_norm) return LR_ERR_NULL;
     if (max_iters < 0 || check_every < 1) return LR_ERR_SHAPE;
@@ -645,7 +649,7 @@ int lr_fit_tol(lr_ctx* ctx, const float* d_X, const float* d_y, int64_t m, int32
         return LR_ERR_ALIGNMENT;
     if (!std::isfinite(lr) || !(eps >= 0.f) || !std::isfinite(eps)) return LR_ERR_VALUE;
     lr_plan P;
-    rc = make_plan(m, n, aligned(d_X, 16), ctx->sm_count, &P);
+    rc = make_plan(m, n, aligned(d_X, 16), ctx->sm_count, &P, bf16);
     if (rc != LR_OK) return rc;
     *iters_done = 0;
     *grad_norm = -1.f;
@@ -656,7 +660,7 @@ int lr_fit_tol(lr_ctx* ctx, const float* d_X, const float* d_y, int64_t m, int32
     LR_CK(ctx, cudaMemsetAsync(ctx->d_tol, 0, sizeof(TolState), st));
     // Narrow rows: one persistent launch that leaves its loop on the device as soon as the norm is small enough.
     if (P.variant == 0 && ctx->persistent && ctx->coop && !ctx->prof && 2ll * max_iters * P.grid < (1ll << 32)) {
-        const int64_t stage_stride = (int64_t(P.rows_per_batch) * n * 4 + 127) & ~int64_t(127);
+        const int64_t stage_stride = (int64_t(P.rows_per_batch) * n * (bf16 ? 2 : 4) + 127) & ~int64_t(127);
         const int64_t room = kMaxDynamicSmem - kHeaderBytes - kFitTailBytes;
         const int depth = int(std::max<int64_t>(1, std::min<int64_t>(P.stages, room / (kNW * stage_stride))));
         FitParams fp{};
@@ -664,11 +668,11 @@ int lr_fit_tol(lr_ctx* ctx, const float* d_X, const float* d_y, int64_t m, int32
         fp.loss_hist = d_loss_hist; fp.status = ctx->d_status; fp.gbar = ctx->d_gbar; fp.depth = depth;
         fp.num_batches = (m + P.rows_per_batch - 1) / P.rows_per_batch;
         fp.iters = max_iters; fp.lr = double(lr); fp.inv_m = 1.0 / double(m);
-        fp.keep_rows = keep_rows_for(ctx, 0, n);
+        fp.keep_rows = keep_rows_for(ctx, 0, n, bf16);
         fp.tol = ctx->d_tol; fp.gbuf = ctx->d_gbuf; fp.eps = double(eps); fp.gnorm_hist = d_gnorm_hist;
         LR_CK(ctx, cudaMemsetAsync(ctx->d_gbar, 0, sizeof(unsigned int), st));
         const int smem = int(kHeaderBytes + int64_t(kNW) * depth * stage_stride + kFitTailBytes);
-        const cudaError_t le = launch_fit(P, smem, fp, st);
+        const cudaError_t le = launch_fit(P, smem, fp, st, bf16);
         if (le == cudaSuccess) {
             ctx->launches += 1;
             LR_CK(ctx, cudaMemcpyAsync(ctx->h_tol, ctx->d_tol, sizeof(TolState), cudaMemcpyDeviceToHost, st));
@@ -686,6 +690,7 @@ int lr_fit_tol(lr_ctx* ctx, const float* d_X, const float* d_y, int64_t m, int32
         for (int32_t k = 0; k < chunk; ++k, ++t) {
             Pass pass{d_X, d_y, m, n, d_w, d_b};
             pass.stop = stop;
+            pass.bf16 = bf16;
             rc = launch_stream_pass(ctx, P, pass, nullptr, 0.f, st);
             if (rc != LR_OK) return rc;
             TolArgs ta{ctx->d_tol, ctx->d_gbuf, double(eps), d_gnorm_hist ? d_gnorm_hist + t : nullptr};
@@ -702,9 +707,9 @@ int lr_fit_tol(lr_ctx* ctx, const float* d_X, const float* d_y, int64_t m, int32
     return LR_OK;
 }
 
-int lr_fit_opt(lr_ctx* ctx, const float* d_X, const float* d_y, int64_t m, int32_t n, float lr, int32_t iters,
-               const lr_opt* opt, float* d_w, float* d_b, float* d_velocity, float* d_loss_hist, void* stream) {
-    int rc = check_common(ctx, d_X, m, n, d_w, d_b);
+int fit_opt_impl(lr_ctx* ctx, const void* d_X, bool bf16, const float* d_y, int64_t m, int32_t n, float lr, int32_t iters,
+                 const lr_opt* opt, float* d_w, float* d_b, float* d_velocity, float* d_loss_hist, void* stream) {
+    int rc = check_common(ctx, d_X, m, n, d_w, d_b, bf16);
     if (rc != LR_OK) return rc;
     if (!d_y || !opt) return LR_ERR_NULL;
     if (iters < 0) return LR_ERR_SHAPE;
@@ -713,7 +718,7 @@ int lr_fit_opt(lr_ctx* ctx, const float* d_X, const float* d_y, int64_t m, int32
     if (!std::isfinite(lr) || !(opt->l2 >= 0.f) || !std::isfinite(opt->l2) || !(opt->momentum >= 0.f && opt->momentum < 1.f))
         return LR_ERR_VALUE;
     lr_plan P;
-    rc = make_plan(m, n, aligned(d_X, 16), ctx->sm_count, &P);
+    rc = make_plan(m, n, aligned(d_X, 16), ctx->sm_count, &P, bf16);
     if (rc != LR_OK) return rc;
     if (iters == 0) return LR_OK;
     DeviceGuard g(ctx);
@@ -724,8 +729,10 @@ int lr_fit_opt(lr_ctx* ctx, const float* d_X, const float* d_y, int64_t m, int32
         vel = ctx->d_vel;
         LR_CK(ctx, cudaMemsetAsync(vel, 0, (size_t(n) + 1) * sizeof(float), st));
     }
+    Pass pass{d_X, d_y, m, n, d_w, d_b};
+    pass.bf16 = bf16;
     for (int32_t t = 0; t < iters; ++t) {
-        rc = launch_stream_pass(ctx, P, Pass{d_X, d_y, m, n, d_w, d_b}, nullptr, 0.f, st);
+        rc = launch_stream_pass(ctx, P, pass, nullptr, 0.f, st);
         if (rc != LR_OK) return rc;
         OptParams op{};
         op.partial = ctx->d_partial; op.G = P.grid; op.n = n; op.inv_m = 1.0 / double(m); op.lr = double(lr);
@@ -739,9 +746,9 @@ int lr_fit_opt(lr_ctx* ctx, const float* d_X, const float* d_y, int64_t m, int32
     return LR_OK;
 }
 
-int lr_fit_sgd(lr_ctx* ctx, const float* d_X, const float* d_y, int64_t m, int32_t n, float lr, int64_t batch_rows,
-               int32_t steps, int64_t first_batch, float* d_w, float* d_b, float* d_loss_hist, void* stream) {
-    int rc = check_common(ctx, d_X, m, n, d_w, d_b);
+int fit_sgd_impl(lr_ctx* ctx, const void* d_X, bool bf16, const float* d_y, int64_t m, int32_t n, float lr, int64_t batch_rows,
+                 int32_t steps, int64_t first_batch, float* d_w, float* d_b, float* d_loss_hist, void* stream) {
+    int rc = check_common(ctx, d_X, m, n, d_w, d_b, bf16);
     if (rc != LR_OK) return rc;
     if (!d_y) return LR_ERR_NULL;
     if (steps < 0 || batch_rows < 1 || batch_rows > m || first_batch < 0) return LR_ERR_SHAPE;
@@ -756,11 +763,13 @@ int lr_fit_sgd(lr_ctx* ctx, const float* d_X, const float* d_y, int64_t m, int32
         const int64_t k = (first_batch + s) % nb;
         const int64_t r0 = k * batch_rows;
         const int64_t rows = std::min(batch_rows, m - r0);
-        const float* Xb = d_X + r0 * n;
+        const void* Xb = static_cast<const unsigned char*>(d_X) + size_t(r0) * n * (bf16 ? 2 : 4);
         lr_plan P;
-        rc = make_plan(rows, n, aligned(Xb, 16), ctx->sm_count, &P);
+        rc = make_plan(rows, n, aligned(Xb, 16), ctx->sm_count, &P, bf16);
         if (rc != LR_OK) return rc;
-        rc = launch_stream_pass(ctx, P, Pass{Xb, d_y + r0, rows, n, d_w, d_b}, nullptr, 0.f, st);
+        Pass pass{Xb, d_y + r0, rows, n, d_w, d_b};
+        pass.bf16 = bf16;
+        rc = launch_stream_pass(ctx, P, pass, nullptr, 0.f, st);
         if (rc != LR_OK) return rc;
         rc = launch_reduce(ctx, ctx->d_partial, P.grid, rows, n, double(lr), true, d_w, d_b, nullptr, nullptr,
                            d_loss_hist ? d_loss_hist + s : nullptr, nullptr, st);
@@ -769,22 +778,72 @@ int lr_fit_sgd(lr_ctx* ctx, const float* d_X, const float* d_y, int64_t m, int32
     return LR_OK;
 }
 
-int lr_shard_sums(lr_ctx* ctx, const float* d_X, const float* d_y, int64_t m_local, int32_t n, const float* d_w,
-                  const float* d_b, double* d_sums, void* stream) {
-    int rc = check_common(ctx, d_X, m_local, n, d_w, d_b);
+int shard_sums_impl(lr_ctx* ctx, const void* d_X, bool bf16, const float* d_y, int64_t m_local, int32_t n, const float* d_w,
+                    const float* d_b, double* d_sums, void* stream) {
+    int rc = check_common(ctx, d_X, m_local, n, d_w, d_b, bf16);
     if (rc != LR_OK) return rc;
     if (!d_y || !d_sums) return LR_ERR_NULL;
     if (!aligned(d_y, 4) || !aligned(d_sums, 8)) return LR_ERR_ALIGNMENT;
     lr_plan P;
-    rc = make_plan(m_local, n, aligned(d_X, 16), ctx->sm_count, &P);
+    rc = make_plan(m_local, n, aligned(d_X, 16), ctx->sm_count, &P, bf16);
     if (rc != LR_OK) return rc;
     DeviceGuard g(ctx);
     if (!g.ok) return LR_ERR_CUDA;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    rc = launch_stream_pass(ctx, P, Pass{d_X, d_y, m_local, n, d_w, d_b}, nullptr, 0.f, st);
+    Pass pass{d_X, d_y, m_local, n, d_w, d_b};
+    pass.bf16 = bf16;
+    rc = launch_stream_pass(ctx, P, pass, nullptr, 0.f, st);
     if (rc != LR_OK) return rc;
     return launch_reduce(ctx, ctx->d_partial, P.grid, m_local, n, 0.0, false, nullptr, nullptr, nullptr, nullptr, nullptr,
                          d_sums, st);
+}
+
+}  // namespace
+
+extern "C" {
+
+int lr_fit_tol(lr_ctx* ctx, const float* d_X, const float* d_y, int64_t m, int32_t n, float lr, float eps,
+               int32_t max_iters, int32_t check_every, float* d_w, float* d_b, float* d_loss_hist, float* d_gnorm_hist,
+               int32_t* iters_done, float* grad_norm, void* stream) {
+    return fit_tol_impl(ctx, d_X, false, d_y, m, n, lr, eps, max_iters, check_every, d_w, d_b, d_loss_hist, d_gnorm_hist,
+                        iters_done, grad_norm, stream);
+}
+
+int lr_fit_tol_bf16(lr_ctx* ctx, const uint16_t* d_Xh, const float* d_y, int64_t m, int32_t n, float lr, float eps,
+                    int32_t max_iters, int32_t check_every, float* d_w, float* d_b, float* d_loss_hist, float* d_gnorm_hist,
+                    int32_t* iters_done, float* grad_norm, void* stream) {
+    return fit_tol_impl(ctx, d_Xh, true, d_y, m, n, lr, eps, max_iters, check_every, d_w, d_b, d_loss_hist, d_gnorm_hist,
+                        iters_done, grad_norm, stream);
+}
+
+int lr_fit_opt(lr_ctx* ctx, const float* d_X, const float* d_y, int64_t m, int32_t n, float lr, int32_t iters,
+               const lr_opt* opt, float* d_w, float* d_b, float* d_velocity, float* d_loss_hist, void* stream) {
+    return fit_opt_impl(ctx, d_X, false, d_y, m, n, lr, iters, opt, d_w, d_b, d_velocity, d_loss_hist, stream);
+}
+
+int lr_fit_opt_bf16(lr_ctx* ctx, const uint16_t* d_Xh, const float* d_y, int64_t m, int32_t n, float lr, int32_t iters,
+                    const lr_opt* opt, float* d_w, float* d_b, float* d_velocity, float* d_loss_hist, void* stream) {
+    return fit_opt_impl(ctx, d_Xh, true, d_y, m, n, lr, iters, opt, d_w, d_b, d_velocity, d_loss_hist, stream);
+}
+
+int lr_fit_sgd(lr_ctx* ctx, const float* d_X, const float* d_y, int64_t m, int32_t n, float lr, int64_t batch_rows,
+               int32_t steps, int64_t first_batch, float* d_w, float* d_b, float* d_loss_hist, void* stream) {
+    return fit_sgd_impl(ctx, d_X, false, d_y, m, n, lr, batch_rows, steps, first_batch, d_w, d_b, d_loss_hist, stream);
+}
+
+int lr_fit_sgd_bf16(lr_ctx* ctx, const uint16_t* d_Xh, const float* d_y, int64_t m, int32_t n, float lr, int64_t batch_rows,
+                    int32_t steps, int64_t first_batch, float* d_w, float* d_b, float* d_loss_hist, void* stream) {
+    return fit_sgd_impl(ctx, d_Xh, true, d_y, m, n, lr, batch_rows, steps, first_batch, d_w, d_b, d_loss_hist, stream);
+}
+
+int lr_shard_sums(lr_ctx* ctx, const float* d_X, const float* d_y, int64_t m_local, int32_t n, const float* d_w,
+                  const float* d_b, double* d_sums, void* stream) {
+    return shard_sums_impl(ctx, d_X, false, d_y, m_local, n, d_w, d_b, d_sums, stream);
+}
+
+int lr_shard_sums_bf16(lr_ctx* ctx, const uint16_t* d_Xh, const float* d_y, int64_t m_local, int32_t n, const float* d_w,
+                       const float* d_b, double* d_sums, void* stream) {
+    return shard_sums_impl(ctx, d_Xh, true, d_y, m_local, n, d_w, d_b, d_sums, stream);
 }
 
 int lr_apply_sums(lr_ctx* ctx, const double* d_sums_all, int32_t parts, int64_t m_total, int32_t n, float lr, float* d_w,

@@ -226,3 +226,94 @@ def test_full_size_workload_bf16(ctx, name):
         assert (labels == lab_ref).mean() >= LABEL_AGREE, (name, thr)
     del dXh
     torch.cuda.empty_cache()
+
+
+# ---- the other fits on a bfloat16-stored X: stopping rule, penalty + momentum, mini-batches, row shards ----
+
+def test_stopping_rule_bf16(ctx):
+    wl = datagen.scaled(datagen.WORKLOADS["cfg3"], 40_003)
+    X, y, _, _ = datagen.generate(wl)
+    bits, Xv = oracle.round_bf16(X)
+    max_iters = 40
+    _, _, _, _, _, gh_all = oracle.fit_tol(Xv, y, wl.lr, 0.0, max_iters)
+    run_min = np.minimum.accumulate(gh_all)
+    cands = [t for t in range(2, max_iters) if gh_all[t] < 0.98 * run_min[t - 1]]
+    t_stop = cands[len(cands) // 2]
+    eps = float(np.sqrt(gh_all[t_stop] * run_min[t_stop - 1]))      # clearly between two consecutive norms
+    w_ref, b_ref, k_ref, n_ref, lh_ref, gh_ref = oracle.fit_tol(Xv, y, wl.lr, eps, max_iters)
+    dXh, dy = dev_bf16(bits), dev(y)
+    results = []
+    for persistent in (True, False):
+        ctx.set_persistent(persistent)
+        try:
+            w = torch.zeros(wl.n, device="cuda")
+            b = torch.zeros(1, device="cuda")
+            lh = torch.full((max_iters,), float("nan"), device="cuda")
+            k, nrm = ctx.fit_tol(dXh, dy, wl.lr, eps, max_iters, w, b, check_every=7, loss_hist=lh)
+        finally:
+            ctx.set_persistent(True)
+        assert k == k_ref == t_stop + 1 and abs(nrm - n_ref) <= 1e-4 * n_ref
+        assert rel_l2(np.concatenate([w.cpu().numpy(), b.cpu().numpy()]), np.concatenate([w_ref, [b_ref]])) <= W_TOL
+        lhc = lh.cpu().numpy()
+        assert np.max(np.abs(lhc[:k] - lh_ref)) <= LOSS_TOL and np.isnan(lhc[k:]).all()
+        results.append((w, b))
+    assert torch.equal(results[0][0], results[1][0]) and torch.equal(results[0][1], results[1][1])   # both forms, same bits
+
+
+@pytest.mark.parametrize("name,m,n,opt", [("cfg3", 40_003, None, dict(l2=0.01, momentum=0.5, nesterov=True)),
+                                          ("cfg5", 90_001, None, dict(l2=0.1, momentum=0.9)),
+                                          ("cfg3", 5_003, 4096, dict(l2=0.05, momentum=0.6))])
+def test_fit_opt_bf16(ctx, name, m, n, opt):
+    import dataclasses
+    wl = datagen.scaled(datagen.WORKLOADS[name], m)
+    if n is not None:
+        wl = dataclasses.replace(wl, n=n)
+    lr, iters = min(wl.lr, 0.25), 30
+    X, y, _, _ = datagen.generate(wl)
+    bits, Xv = oracle.round_bf16(X)
+    w_ref, b_ref, _, lh_ref = oracle.fit_opt(Xv, y, lr, iters, **opt)
+    w = torch.zeros(wl.n, device="cuda")
+    b = torch.zeros(1, device="cuda")
+    lh = torch.empty(iters, device="cuda")
+    ctx.fit_opt(dev_bf16(bits), dev(y), lr, iters, w, b, loss_hist=lh, **opt)
+    assert rel_l2(np.concatenate([w.cpu().numpy(), b.cpu().numpy()]), np.concatenate([w_ref, [b_ref]])) <= W_TOL
+    assert np.max(np.abs(lh.cpu().numpy() - lh_ref)) <= LOSS_TOL
+
+
+@pytest.mark.parametrize("m,n,batch", [(50_003, 256, 8_192), (9_000, 24, 2_501), (6_001, 2048, 1_000)])
+def test_minibatch_descent_bf16(ctx, m, n, batch):
+    # 2,501 rows of 24 bfloat16 columns: the second block starts 8 bytes off a 16-byte boundary (unstaged kernel)
+    import dataclasses
+    wl = dataclasses.replace(datagen.scaled(datagen.WORKLOADS["cfg3"], m), n=n)
+    X, y, _, _ = datagen.generate(wl)
+    bits, Xv = oracle.round_bf16(X)
+    steps, lr = 12, 0.2
+    w_ref, b_ref, lh_ref = oracle.fit_sgd(Xv, y, lr, batch, steps, first_batch=1)
+    w = torch.zeros(n, device="cuda")
+    b = torch.zeros(1, device="cuda")
+    lh = torch.empty(steps, device="cuda")
+    ctx.fit_sgd(dev_bf16(bits), dev(y), lr, batch, steps, w, b, first_batch=1, loss_hist=lh)
+    assert rel_l2(np.concatenate([w.cpu().numpy(), b.cpu().numpy()]), np.concatenate([w_ref, [b_ref]])) <= W_TOL
+    assert np.max(np.abs(lh.cpu().numpy() - lh_ref)) <= LOSS_TOL
+
+
+def test_row_shards_bf16(ctx):
+    from paper_2308_10037_b200.parallel import shard_rows
+    wl = datagen.scaled(datagen.WORKLOADS["cfg3"], 50_003)
+    X, y, _, _ = datagen.generate(wl)
+    bits, Xv = oracle.round_bf16(X)
+    parts, steps = 3, 5
+    shards = [shard_rows(wl.m, r, parts) for r in range(parts)]
+    dXs = [dev_bf16(bits[a:b]) for a, b in shards]
+    dys = [dev(y[a:b]) for a, b in shards]
+    w = torch.zeros(wl.n, device="cuda")
+    b = torch.zeros(1, device="cuda")
+    sums = torch.empty((parts, wl.n + 2), dtype=torch.float64, device="cuda")
+    loss = torch.empty(steps, device="cuda")
+    for t in range(steps):
+        for r in range(parts):
+            ctx.shard_sums(dXs[r], dys[r], w, b, sums[r])
+        ctx.apply_sums(sums, wl.m, wl.lr, w, b, loss[t:t + 1])
+    w_ref, b_ref, lh_ref = oracle.fit(Xv, y, wl.lr, steps)
+    assert rel_l2(np.concatenate([w.cpu().numpy(), b.cpu().numpy()]), np.concatenate([w_ref, [b_ref]])) <= W_TOL
+    assert np.max(np.abs(loss.cpu().numpy() - lh_ref)) <= LOSS_TOL
