@@ -105,6 +105,16 @@ int lr_fit(lr_ctx* ctx, const float* d_X, const float* d_y, int64_t m, int32_t n
 int lr_set_persistent(lr_ctx* ctx, int32_t on);
 
 /*
+ * Overlap between the kernels of one call (on by default).  Every iteration of the two-kernel form is a pass followed by
+ * the reduction; with overlap on, each of them is launched as the programmatic dependent of the one before it: it is
+ * scheduled while its predecessor drains, the pass stages its first rows of X (an input nothing in this library
+ * writes) meanwhile, and it waits on the device for the predecessor to complete before it reads the parameters.  The
+ * first kernel of a call is always an ordinary launch, so work the caller enqueued earlier on the stream is complete
+ * before anything is read.  Results do not change.  lr_set_overlap(ctx, 0) launches every kernel the ordinary way.
+ */
+int lr_set_overlap(lr_ctx* ctx, int32_t on);
+
+/*
  * L2 residency hint for iterated passes over the same X: the first `bytes` bytes of X (whole rows) are fetched with an
  * L2 evict-last hint and everything else with evict-first, so that across the iterations of a fit that leading part
  * of X is served from the 126 MB L2 instead of HBM.  Results do not change.  0 turns the hint off; -1 (the default)

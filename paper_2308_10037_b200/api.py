@@ -23,7 +23,7 @@ EXPORTS = ["lr_plan_query", "lr_create", "lr_destroy", "lr_loss_grad", "lr_fit",
            "lr_predict_host", "lr_profile_enable", "lr_profile_read", "lr_launch_count", "lr_last_device_status",
            "lr_last_cuda_error", "lr_status_string", "lr_loss_grad_noalloc", "lr_fit_tol", "lr_fit_opt", "lr_selftest_wait", "lr_set_persistent", "lr_fit_sgd", "lr_set_l2_keep",
            "lr_convert_bf16", "lr_loss_grad_bf16", "lr_fit_bf16", "lr_predict_bf16", "lr_plan_query_bf16",
-           "lr_fit_tol_bf16", "lr_fit_opt_bf16", "lr_fit_sgd_bf16", "lr_shard_sums_bf16"]
+           "lr_fit_tol_bf16", "lr_fit_opt_bf16", "lr_fit_sgd_bf16", "lr_shard_sums_bf16", "lr_set_overlap"]
 
 
 class LrPlan(ctypes.Structure):
@@ -79,6 +79,7 @@ def lib() -> ctypes.CDLL:
         L.lr_fit_sgd_bf16.argtypes = L.lr_fit_sgd.argtypes
         L.lr_shard_sums_bf16.argtypes = L.lr_shard_sums.argtypes
         L.lr_set_persistent.argtypes = [P, I32]
+        L.lr_set_overlap.argtypes = [P, I32]
         L.lr_set_l2_keep.argtypes = [P, I64]
         L.lr_loss_grad_noalloc.argtypes = [I32, P, P, I64, I32, P, P, P, P, P, P, P]
         L.lr_fit_host.argtypes = [P, P, P, I64, I32, F, I32, P, P, P]
@@ -297,6 +298,10 @@ class Context:
     def set_persistent(self, on: bool):
         """Allow (default) or forbid the single-launch persistent kernel in ``fit``; results are identical either way."""
         self._check(lib().lr_set_persistent(self._h, int(bool(on))), "lr_set_persistent")
+
+    def set_overlap(self, on: bool):
+        """Allow (default) or forbid launching consecutive kernels of a call as programmatic dependents; same results."""
+        self._check(lib().lr_set_overlap(self._h, int(bool(on))), "lr_set_overlap")
 
     def selftest_wait(self, arm: bool, limit_ms: int = 20):
         """Enqueue the bounded-wait probe (see ``lr_selftest_wait``); read the outcome with ``device_status``."""

@@ -7,6 +7,7 @@
 #include <cstring>
 #include <mutex>
 #include <new>
+#include <utility>
 #include <vector>
 
 #include "lrgd_convert.cuh"
@@ -134,6 +135,7 @@ struct lr_ctx {
     unsigned int* d_gbar = nullptr;                 // grid-barrier counter of the persistent fit kernel
     bool coop = false;                              // device supports cooperative launches
     bool persistent = true;                         // lr_fit may use the single-launch kernel
+    bool overlap = true;                            // consecutive kernels of one call are launched as programmatic dependents
     int64_t l2_keep_bytes = -1;                     // leading bytes of X fetched with an evict-last hint; -1 = per-kernel default
     int64_t l2_bytes = 0;                           // size of the device's L2
     // buffers of the host-pointer entry points (grown on demand)
@@ -174,29 +176,46 @@ struct DeviceGuard {
 
 bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
 
+// Launches `kern`; with `dependent` set, as a programmatic dependent launch: the kernel may start while the kernel
+// before it in the stream is still draining, and synchronises with it on the device (grid_dependency_wait).
+template <typename... KArgs, typename... Args>
+cudaError_t launch_kernel(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, bool dependent,
+                          Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = dependent ? attr : nullptr;
+    cfg.numAttrs = dependent ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kern, std::forward<Args>(args)...);
+}
+
 template <class E, int NV, int LPR, int RB, bool PRED>
-cudaError_t launch_rows_t(const lr_plan& P, const StreamParams& sp, cudaStream_t st) {
+cudaError_t launch_rows_t(const lr_plan& P, const StreamParams& sp, cudaStream_t st, bool dependent) {
     auto kern = k_stream_rows<E, NV, LPR, RB, kNW, PRED>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, P.smem_bytes);
     if (e != cudaSuccess) return e;
-    kern<<<P.grid, P.threads, P.smem_bytes, st>>>(sp);
-    return cudaGetLastError();
+    return launch_kernel(kern, dim3(P.grid), dim3(P.threads), size_t(P.smem_bytes), st, dependent, sp);
 }
 
 template <bool PRED>
-cudaError_t launch_rows(const lr_plan& P, const StreamParams& sp, cudaStream_t st, bool bf16 = false) {
+cudaError_t launch_rows(const lr_plan& P, const StreamParams& sp, cudaStream_t st, bool bf16 = false, bool dependent = false) {
     if (bf16) {
-        if (P.lanes_per_row == 8) return launch_rows_t<ElemBF16, 1, 8, 8, PRED>(P, sp, st);
-        if (P.lanes_per_row == 16) return launch_rows_t<ElemBF16, 1, 16, 8, PRED>(P, sp, st);
-        if (P.vec_per_lane == 1) return launch_rows_t<ElemBF16, 1, 32, LRGD_NV1_RB, PRED>(P, sp, st);
-        if (P.vec_per_lane == 2) return launch_rows_t<ElemBF16, 2, 32, LRGD_NV2_RB, PRED>(P, sp, st);
+        if (P.lanes_per_row == 8) return launch_rows_t<ElemBF16, 1, 8, 8, PRED>(P, sp, st, dependent);
+        if (P.lanes_per_row == 16) return launch_rows_t<ElemBF16, 1, 16, 8, PRED>(P, sp, st, dependent);
+        if (P.vec_per_lane == 1) return launch_rows_t<ElemBF16, 1, 32, LRGD_NV1_RB, PRED>(P, sp, st, dependent);
+        if (P.vec_per_lane == 2) return launch_rows_t<ElemBF16, 2, 32, LRGD_NV2_RB, PRED>(P, sp, st, dependent);
         return cudaErrorInvalidValue;              // the plan never asks for four bfloat16 groups per lane
     }
-    if (P.lanes_per_row == 8) return launch_rows_t<ElemF32, 1, 8, 8, PRED>(P, sp, st);
-    if (P.lanes_per_row == 16) return launch_rows_t<ElemF32, 1, 16, 8, PRED>(P, sp, st);
-    if (P.vec_per_lane == 1) return launch_rows_t<ElemF32, 1, 32, LRGD_NV1_RB, PRED>(P, sp, st);
-    if (P.vec_per_lane == 2) return launch_rows_t<ElemF32, 2, 32, LRGD_NV2_RB, PRED>(P, sp, st);
-    return launch_rows_t<ElemF32, 4, 32, 2, PRED>(P, sp, st);
+    if (P.lanes_per_row == 8) return launch_rows_t<ElemF32, 1, 8, 8, PRED>(P, sp, st, dependent);
+    if (P.lanes_per_row == 16) return launch_rows_t<ElemF32, 1, 16, 8, PRED>(P, sp, st, dependent);
+    if (P.vec_per_lane == 1) return launch_rows_t<ElemF32, 1, 32, LRGD_NV1_RB, PRED>(P, sp, st, dependent);
+    if (P.vec_per_lane == 2) return launch_rows_t<ElemF32, 2, 32, LRGD_NV2_RB, PRED>(P, sp, st, dependent);
+    return launch_rows_t<ElemF32, 4, 32, 2, PRED>(P, sp, st, dependent);
 }
 
 // Tensor map of X for the wide-row kernel: [m][n] row-major, box = cw 16-byte groups by rb rows, zero fill outside.
@@ -230,25 +249,25 @@ cudaError_t make_x_tensor_map(const void* X, bool bf16, int64_t m, int32_t n, in
 }
 
 template <class E, int NV, int RB, bool PRED>
-cudaError_t launch_split_t(const lr_plan& P, const CUtensorMap& tm, const SplitParams& sp, cudaStream_t st) {
+cudaError_t launch_split_t(const lr_plan& P, const CUtensorMap& tm, const SplitParams& sp, cudaStream_t st, bool dependent) {
     auto kern = k_stream_split<E, NV, RB, kNW, PRED>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, P.smem_bytes);
     if (e != cudaSuccess) return e;
-    kern<<<P.grid, P.threads, P.smem_bytes, st>>>(tm, sp);
-    return cudaGetLastError();
+    return launch_kernel(kern, dim3(P.grid), dim3(P.threads), size_t(P.smem_bytes), st, dependent, tm, sp);
 }
 
 template <bool PRED>
-cudaError_t launch_split(const lr_plan& P, const void* X, const SplitParams& sp, cudaStream_t st, bool bf16 = false) {
+cudaError_t launch_split(const lr_plan& P, const void* X, const SplitParams& sp, cudaStream_t st, bool bf16 = false,
+                         bool dependent = false) {
     CUtensorMap tm;
     cudaError_t e = make_x_tensor_map(X, bf16, sp.m, sp.n, sp.cw, P.rows_per_batch, &tm);
     if (e != cudaSuccess) return e;
     if (bf16) {
-        if (P.vec_per_lane == 2) return launch_split_t<ElemBF16, 2, 4, PRED>(P, tm, sp, st);
-        return launch_split_t<ElemBF16, 1, 8, PRED>(P, tm, sp, st);
+        if (P.vec_per_lane == 2) return launch_split_t<ElemBF16, 2, 4, PRED>(P, tm, sp, st, dependent);
+        return launch_split_t<ElemBF16, 1, 8, PRED>(P, tm, sp, st, dependent);
     }
-    if (P.vec_per_lane == 2) return launch_split_t<ElemF32, 2, 4, PRED>(P, tm, sp, st);
-    return launch_split_t<ElemF32, 1, 8, PRED>(P, tm, sp, st);
+    if (P.vec_per_lane == 2) return launch_split_t<ElemF32, 2, 4, PRED>(P, tm, sp, st, dependent);
+    return launch_split_t<ElemF32, 1, 8, PRED>(P, tm, sp, st, dependent);
 }
 
 template <class E, int NV, int LPR, int RB>
@@ -287,6 +306,8 @@ struct Pass {
     const void* X; const float* y; int64_t m; int32_t n; const float* w; const float* b;
     const int* stop = nullptr;                      // device flag that turns the launch into a no-op once set
     bool bf16 = false;                              // X holds bfloat16 elements instead of fp32
+    bool dependent = false;                         // the kernel before this one in the stream is this library's own reduction:
+                                                    // launch as its programmatic dependent (X is staged while it drains)
 };
 
 struct TolArgs {                                    // tolerance mode of the reduction
@@ -297,6 +318,7 @@ struct TolArgs {                                    // tolerance mode of the red
 int launch_stream_pass(lr_ctx* ctx, const lr_plan& P, const Pass& a, uint8_t* labels, float cut, cudaStream_t st) {
     const bool predict = labels != nullptr;
     const bool timed = ctx->prof && ctx->prof_used < kMaxProfiled;
+    const bool dep = a.dependent && ctx->overlap && !ctx->prof;      // event records between launches would split the pair
     if (timed) {
         while (int(ctx->ev.size()) < 2 * (ctx->prof_used + 1)) {
             cudaEvent_t e;
@@ -313,7 +335,7 @@ int launch_stream_pass(lr_ctx* ctx, const lr_plan& P, const Pass& a, uint8_t* la
         sp.depth = P.stages;
         sp.num_batches = (a.m + P.rows_per_batch - 1) / P.rows_per_batch;
         sp.keep_rows = keep_rows_for(ctx, 0, a.n, a.bf16);
-        e = predict ? launch_rows<true>(P, sp, st, a.bf16) : launch_rows<false>(P, sp, st, a.bf16);
+        e = predict ? launch_rows<true>(P, sp, st, a.bf16, dep) : launch_rows<false>(P, sp, st, a.bf16, dep);
     } else if (P.variant == 1) {
         SplitParams sp{};
         sp.y = a.y; sp.m = a.m; sp.n = a.n; sp.w = a.w; sp.b = a.b;
@@ -322,19 +344,16 @@ int launch_stream_pass(lr_ctx* ctx, const lr_plan& P, const Pass& a, uint8_t* la
         sp.cw = (a.n / (a.bf16 ? 8 : 4) + kNW - 1) / kNW;
         sp.num_batches = (a.m + P.rows_per_batch - 1) / P.rows_per_batch;
         sp.keep_rows = keep_rows_for(ctx, 1, a.n, a.bf16);
-        e = predict ? launch_split<true>(P, a.X, sp, st, a.bf16) : launch_split<false>(P, a.X, sp, st, a.bf16);
+        e = predict ? launch_split<true>(P, a.X, sp, st, a.bf16, dep) : launch_split<false>(P, a.X, sp, st, a.bf16, dep);
     } else {
         GenericParams gp{};
         gp.X = a.X; gp.y = a.y; gp.m = a.m; gp.n = a.n; gp.w = a.w; gp.b = a.b;
         gp.partial = ctx->d_partial; gp.labels = labels; gp.cut = cut; gp.stop = a.stop;
-        if (a.bf16) {
-            if (predict) k_generic<ElemBF16, true><<<P.grid, P.threads, 0, st>>>(gp);
-            else k_generic<ElemBF16, false><<<P.grid, P.threads, 0, st>>>(gp);
-        } else {
-            if (predict) k_generic<ElemF32, true><<<P.grid, P.threads, 0, st>>>(gp);
-            else k_generic<ElemF32, false><<<P.grid, P.threads, 0, st>>>(gp);
-        }
-        e = cudaGetLastError();
+        const dim3 g(P.grid), t(P.threads);
+        if (a.bf16) e = predict ? launch_kernel(k_generic<ElemBF16, true>, g, t, 0, st, dep, gp)
+                                : launch_kernel(k_generic<ElemBF16, false>, g, t, 0, st, dep, gp);
+        else e = predict ? launch_kernel(k_generic<ElemF32, true>, g, t, 0, st, dep, gp)
+                         : launch_kernel(k_generic<ElemF32, false>, g, t, 0, st, dep, gp);
     }
     LR_CK(ctx, e);
     ctx->launches += 1;
@@ -353,9 +372,10 @@ int launch_reduce(lr_ctx* ctx, const double* partial, int G, int64_t m, int32_t 
     rp.update = update ? 1 : 0; rp.w = w; rp.b = b; rp.grad_w = grad_w; rp.grad_b = grad_b; rp.loss_out = loss_out;
     rp.raw_sums = raw_sums;
     if (tol) { rp.tol = tol->state; rp.gbuf = tol->gbuf; rp.eps = tol->eps; rp.gnorm_out = tol->gnorm_out; }
-    dim3 block(32, kRedSlices);
-    k_reduce_update<<<(n + 2 + 31) / 32, block, 0, st>>>(rp);
-    LR_CK(ctx, cudaGetLastError());
+    // always preceded in the stream by the pass that wrote `partial` (or, for lr_apply_sums, by whatever the caller ran:
+    // the kernel waits for it on the device either way), so it is launched as that kernel's programmatic dependent
+    LR_CK(ctx, launch_kernel(k_reduce_update, dim3((n + 2 + 31) / 32), dim3(32, kRedSlices), 0, st,
+                             ctx->overlap && !ctx->prof, rp));
     ctx->launches += 1;
     return LR_OK;
 }
@@ -591,6 +611,7 @@ int fit_impl(lr_ctx* ctx, const void* d_X, bool bf16, const float* d_y, int64_t 
     Pass pass{d_X, d_y, m, n, d_w, d_b};
     pass.bf16 = bf16;
     for (int32_t t = 0; t < iters; ++t) {
+        pass.dependent = t > 0;                    // follows this call's own reduction
         rc = launch_stream_pass(ctx, P, pass, nullptr, 0.f, st);
         if (rc != LR_OK) return rc;
         rc = launch_reduce(ctx, ctx->d_partial, P.grid, m, n, double(lr), true, d_w, d_b, nullptr, nullptr,
@@ -625,6 +646,12 @@ int lr_set_l2_keep(lr_ctx* ctx, int64_t bytes) {
     if (!ctx) return LR_ERR_NULL;
     if (bytes < -1) return LR_ERR_VALUE;
     ctx->l2_keep_bytes = bytes;
+    return LR_OK;
+}
+
+int lr_set_overlap(lr_ctx* ctx, int32_t on) {
+    if (!ctx) return LR_ERR_NULL;
+    ctx->overlap = on != 0;
     return LR_OK;
 }
 
@@ -691,6 +718,7 @@ int fit_tol_impl(lr_ctx* ctx, const void* d_X, bool bf16, const float* d_y, int6
             Pass pass{d_X, d_y, m, n, d_w, d_b};
             pass.stop = stop;
             pass.bf16 = bf16;
+            pass.dependent = k > 0;                // within a chunk it follows this call's own reduction
             rc = launch_stream_pass(ctx, P, pass, nullptr, 0.f, st);
             if (rc != LR_OK) return rc;
             TolArgs ta{ctx->d_tol, ctx->d_gbuf, double(eps), d_gnorm_hist ? d_gnorm_hist + t : nullptr};
@@ -732,6 +760,7 @@ int fit_opt_impl(lr_ctx* ctx, const void* d_X, bool bf16, const float* d_y, int6
     Pass pass{d_X, d_y, m, n, d_w, d_b};
     pass.bf16 = bf16;
     for (int32_t t = 0; t < iters; ++t) {
+        pass.dependent = t > 0;                    // follows this call's own reduction
         rc = launch_stream_pass(ctx, P, pass, nullptr, 0.f, st);
         if (rc != LR_OK) return rc;
         OptParams op{};
@@ -739,8 +768,8 @@ int fit_opt_impl(lr_ctx* ctx, const void* d_X, bool bf16, const float* d_y, int6
         op.l2 = double(opt->l2); op.mu = double(opt->momentum); op.nesterov = opt->nesterov ? 1 : 0;
         op.w = d_w; op.b = d_b; op.vel = vel; op.loss_out = d_loss_hist ? d_loss_hist + t : nullptr;
         op.scratch = ctx->d_oscr; op.ticket = ctx->d_oticket;
-        k_reduce_opt<<<(n + 2 + 31) / 32, dim3(32, kRedSlices), 0, st>>>(op);
-        LR_CK(ctx, cudaGetLastError());
+        LR_CK(ctx, launch_kernel(k_reduce_opt, dim3((n + 2 + 31) / 32), dim3(32, kRedSlices), 0, st,
+                                 ctx->overlap && !ctx->prof, op));
         ctx->launches += 1;
     }
     return LR_OK;
@@ -769,6 +798,7 @@ int fit_sgd_impl(lr_ctx* ctx, const void* d_X, bool bf16, const float* d_y, int6
         if (rc != LR_OK) return rc;
         Pass pass{Xb, d_y + r0, rows, n, d_w, d_b};
         pass.bf16 = bf16;
+        pass.dependent = s > 0;                    // follows this call's own reduction
         rc = launch_stream_pass(ctx, P, pass, nullptr, 0.f, st);
         if (rc != LR_OK) return rc;
         rc = launch_reduce(ctx, ctx->d_partial, P.grid, rows, n, double(lr), true, d_w, d_b, nullptr, nullptr,
@@ -1076,8 +1106,7 @@ extern "C" int lr_loss_grad_noalloc(int32_t device, const float* d_X, const floa
         GenericParams gp{};
         gp.X = d_X; gp.y = d_y; gp.m = m; gp.n = n; gp.w = d_w; gp.b = d_b;
         gp.partial = partial; gp.labels = nullptr; gp.cut = 0.f;
-        k_generic<ElemF32, false><<<P.grid, P.threads, 0, st>>>(gp);
-        e = cudaGetLastError();
+        e = launch_kernel(k_generic<ElemF32, false>, dim3(P.grid), dim3(P.threads), 0, st, false, gp);
     }
     if (e != cudaSuccess) return LR_ERR_CUDA;
     ReduceParams rp{};

@@ -105,6 +105,18 @@ __global__ void k_wait_probe(int* status, unsigned long long limit_ns, int arm) 
     if (!ok && threadIdx.x == 0) atomicExch(status, kStatusTimeout);
 }
 
+// Programmatic dependent launch (sm_90+).  A kernel launched with the programmatic-stream-serialization attribute may
+// start as soon as every CTA of the kernel before it in the stream has called grid_dependency_release() (or exited);
+// whatever it does before grid_dependency_wait() overlaps the tail of that kernel and must not touch anything that
+// kernel (or any earlier one) writes.  grid_dependency_wait() returns once all earlier kernels have completed and their
+// writes are visible.  Without the attribute both are no-ops and the launch is an ordinary one.
+__device__ __forceinline__ void grid_dependency_release() {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+__device__ __forceinline__ void grid_dependency_wait() {
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
 __device__ __forceinline__ uint64_t l2_policy_evict_first() {
     uint64_t pol;
     asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));

@@ -31,13 +31,15 @@ struct GenericParams {
 
 template <class E, bool PREDICT>
 __global__ void __launch_bounds__(kGenThreads) k_generic(const GenericParams p) {
+    grid_dependency_release();
+    grid_dependency_wait();                        // the parameters and the stop flag come from the kernel before this one
     if (p.stop != nullptr && *reinterpret_cast<const volatile int*>(p.stop) != 0) return;   // a stopping rule was met by an earlier iteration
     __shared__ float err_s[kGenRows];
     __shared__ double red_e[kGenThreads / 32], red_l[kGenThreads / 32];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     constexpr int NWARP = kGenThreads / 32;
     const int n = p.n;
-    const float bval = __ldg(p.b);
+    const float bval = __ldcg(p.b);
     double* out = PREDICT ? nullptr : p.partial + static_cast<size_t>(blockIdx.x) * (n + 2);
     if constexpr (!PREDICT) {
         for (int c = threadIdx.x; c < n + 2; c += kGenThreads) out[c] = 0.0;
@@ -50,7 +52,7 @@ __global__ void __launch_bounds__(kGenThreads) k_generic(const GenericParams p) 
         for (int r = warp; r < rows; r += NWARP) {
             const long long xr = (row0 + r) * n;
             float d = 0.f;
-            for (int c = lane; c < n; c += 32) d = fmaf(E::load(p.X, xr + c), __ldg(p.w + c), d);
+            for (int c = lane; c < n; c += 32) d = fmaf(E::load(p.X, xr + c), __ldcg(p.w + c), d);
 #pragma unroll
             for (int msk = 16; msk >= 1; msk >>= 1) d += __shfl_xor_sync(0xffffffffu, d, msk);
             const float z = d + bval;

@@ -48,6 +48,8 @@ struct ReduceParams {
 __global__ void __launch_bounds__(32 * kRedSlices) k_reduce_update(const ReduceParams p) {
     __shared__ double sh[kRedSlices][33];
     __shared__ int is_last;
+    grid_dependency_release();
+    grid_dependency_wait();                        // the partial rows come from the kernel before this one
     if (p.tol != nullptr && *reinterpret_cast<volatile int*>(&p.tol->stop) != 0) return;   // uniform: set by an earlier kernel
     const int col = blockIdx.x * 32 + threadIdx.x;
     const int slice = threadIdx.y;
@@ -59,7 +61,7 @@ __global__ void __launch_bounds__(32 * kRedSlices) k_reduce_update(const ReduceP
     if (col < stride) {
         const double* src = p.partial + col;
 #pragma unroll 8
-        for (int g = g0; g < g1; ++g) s += src[static_cast<size_t>(g) * stride];
+        for (int g = g0; g < g1; ++g) s += __ldcg(src + static_cast<size_t>(g) * stride);   // straight from L2
     }
     sh[slice][threadIdx.x] = s;
     __syncthreads();
@@ -142,6 +144,8 @@ struct OptParams {
 __global__ void __launch_bounds__(32 * kRedSlices) k_reduce_opt(const OptParams p) {
     __shared__ double sh[kRedSlices][33];
     __shared__ int is_last;
+    grid_dependency_release();
+    grid_dependency_wait();                        // the partial rows come from the kernel before this one
     const int col = blockIdx.x * 32 + threadIdx.x;
     const int slice = threadIdx.y;
     const int stride = p.n + 2;
@@ -152,7 +156,7 @@ __global__ void __launch_bounds__(32 * kRedSlices) k_reduce_opt(const OptParams 
     if (col < stride) {
         const double* src = p.partial + col;
 #pragma unroll 8
-        for (int g = g0; g < g1; ++g) s += src[static_cast<size_t>(g) * stride];
+        for (int g = g0; g < g1; ++g) s += __ldcg(src + static_cast<size_t>(g) * stride);   // straight from L2
     }
     sh[slice][threadIdx.x] = s;
     __syncthreads();

@@ -139,7 +139,6 @@ __global__ void __launch_bounds__(NW * 32, 1) k_stream_rows(const StreamParams p
     static_assert(NW * kMaxDepth * 8 + 16 <= kHeaderBytes, "header too small");
     constexpr unsigned FULL = 0xffffffffu;
 
-    if (p.stop != nullptr && *reinterpret_cast<const volatile int*>(p.stop) != 0) return;   // a stopping rule was met by an earlier iteration
     extern __shared__ __align__(128) unsigned char smem[];
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem);                       // [NW][kMaxDepth]
     volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + NW * kMaxDepth);
@@ -189,8 +188,6 @@ __global__ void __launch_bounds__(NW * 32, 1) k_stream_rows(const StreamParams p
 #pragma unroll
         for (int c = 0; c < EPG; ++c) dacc[k][c] = 0.0;
     const int sub = lane & (LPR - 1), slot = lane >> LOG_LPR;
-    lm.load_w(p.w, sub, LPR, n4, false);
-    const float bval = __ldg(p.b);
     const int myr = ((sub >> SHIFT) & (RB - 1)) * RPW + slot;     // the row of a batch whose logit ends up on this lane
     const bool owner = (sub & ((1 << SHIFT) - 1)) == 0;           // one lane per row does the bookkeeping
 
@@ -202,6 +199,21 @@ __global__ void __launch_bounds__(NW * 32, 1) k_stream_rows(const StreamParams p
     if constexpr (!PREDICT) {
         if (cnt > 0 && row0 + myr < p.m) y_next = __ldg(p.y + row0 + myr);
     }
+    // X and y are inputs that no kernel of this library writes, so the first stages are already on their way; the
+    // parameters (and the stop flag) come from the kernel before this one: wait for it only now.
+    grid_dependency_release();
+    grid_dependency_wait();
+    if (p.stop != nullptr && *reinterpret_cast<const volatile int*>(p.stop) != 0) {
+        // a stopping rule was met by an earlier iteration: let the copies just issued land, then leave
+        if (lane == 0) {
+            const int pre = cnt < D ? cnt : D;
+            for (int d = 0; d < pre; ++d) mbar_wait_drain(&my_bars[d], 0u);
+        }
+        __syncwarp();
+        return;
+    }
+    lm.load_w(p.w, sub, LPR, n4, true);            // through L2: the kernel before this one may just have written them
+    const float bval = __ldcg(p.b);
     const bool full_cols = n4 == NV * LPR;         // every lane's column groups exist
     const bool labels_word_aligned = PREDICT && (reinterpret_cast<uintptr_t>(p.labels) & 3u) == 0 && RPB % 4 == 0;
     int issued = cnt < D ? cnt : D;                // warp-uniform count of batches whose copies were issued

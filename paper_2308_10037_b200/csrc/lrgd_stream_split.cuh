@@ -58,7 +58,6 @@ __global__ void __launch_bounds__(NW * 32, 1) k_stream_split(const __grid_consta
     static_assert(NW * kMaxDepth * 8 + 16 <= kSplitZOffset, "header too small");
     static_assert(kSplitZOffset + 2 * NW * RB * 4 <= kSplitHeaderBytes, "header too small");
 
-    if (p.stop != nullptr && *reinterpret_cast<const volatile int*>(p.stop) != 0) return;   // a stopping rule was met by an earlier iteration
     extern __shared__ __align__(128) unsigned char smem[];
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + NW * kMaxDepth);
@@ -99,12 +98,10 @@ __global__ void __launch_bounds__(NW * 32, 1) k_stream_split(const __grid_consta
     float se = 0.f, sl = 0.f;
     double dse = 0.0, dsl = 0.0;
     lm.zero();
-    lm.load_w(p.w, c0 + lane, 32, c0 + mycw, false);
 #pragma unroll
     for (int k = 0; k < NV; ++k)
 #pragma unroll
         for (int c = 0; c < EPG; ++c) dacc[k][c] = 0.0;
-    const float bval = __ldg(p.b);
     const int myr = (lane >> SHIFT) & (RB - 1);    // the row of a batch whose logit ends up on this lane
     const int dup = lane & (DUP - 1);              // which of the lanes sharing that row this one is
     const bool owner = dup == 0;
@@ -126,6 +123,20 @@ __global__ void __launch_bounds__(NW * 32, 1) k_stream_split(const __grid_consta
     if constexpr (!PREDICT) {
         if (cnt > 0 && row0 + myr < p.m) y_next = __ldg(p.y + row0 + myr);
     }
+    // X and y are inputs that no kernel of this library writes, so the first stages are already on their way; the
+    // parameters (and the stop flag) come from the kernel before this one: wait for it only now.
+    grid_dependency_release();
+    grid_dependency_wait();
+    if (p.stop != nullptr && *reinterpret_cast<const volatile int*>(p.stop) != 0) {
+        // a stopping rule was met by an earlier iteration: let the copies just issued land, then leave
+        if (lane == 0) {
+            for (int d2 = 0; d2 < issued; ++d2) mbar_wait_drain(&my_bars[d2], 0u);
+        }
+        __syncwarp();
+        return;
+    }
+    lm.load_w(p.w, c0 + lane, 32, c0 + mycw, true);    // through L2: the kernel before this one may just have written them
+    const float bval = __ldcg(p.b);
 
     for (int i = 0; i < cnt; ++i) {
         const bool myvalid = row0 + myr < p.m;
