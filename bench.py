@@ -267,6 +267,7 @@ def main():
     ap.add_argument("--rows", type=int, default=0, help="override the workload's row count (profiling on a smaller case)")
     ap.add_argument("--tol", default="", help="ALPHA,EPS: time-to-tolerance mode (Algorithm 7 stopping rule); --steps caps the updates")
     ap.add_argument("--no-persistent", action="store_true", help="force two kernels per iteration in lr_fit")
+    ap.add_argument("--force-persistent", action="store_true", help="force the single-launch persistent kernel in lr_fit")
     ap.add_argument("--no-overlap", action="store_true", help="ordinary launches only (no programmatic dependent launches)")
     ap.add_argument("--l2-keep-mb", type=float, default=-1.0, help="MB of X to keep in L2 across iterations (-1: library default, 0: off)")
     ap.add_argument("--x-dtype", default="f32", choices=["f32", "bf16"],
@@ -320,6 +321,8 @@ def main():
     ctx = api.Context(n_max=wl.n, device=local_rank)
     if args.no_persistent:
         ctx.set_persistent(False)
+    if args.force_persistent:
+        ctx.set_persistent(True)
     if args.no_overlap:
         ctx.set_overlap(False)
     if args.l2_keep_mb >= 0:

@@ -95,10 +95,14 @@ int lr_loss_grad(lr_ctx* ctx, const float* d_X, const float* d_y, int64_t m, int
  * receives the loss at the parameters BEFORE update t.  iters == 0 is a no-op.
  * Results are bit-reproducible for a given shape and device, and fit(a) followed by fit(b) equals
  * fit(a+b) bit for bit.
- * For rows of up to 512 columns (16-byte aligned X, n % 4 == 0) and iters >= 2 the whole call is ONE cooperative
- * launch of a persistent kernel (grid barriers between the pass and the update; the HBM stream continues across
- * iterations); otherwise two kernels per iteration.  Both give the same bits.  lr_set_persistent(ctx, 0) forces the
- * two-kernel form (it is also used while lr_profile_enable is on, so that single launches can be timed).
+ * Two forms give the same bits.  Two kernels per iteration (the pass, then the reduction with the update), each
+ * launched as the programmatic dependent of the one before it (see lr_set_overlap); or, for rows of up to 512 columns
+ * (16-byte aligned X, n % 4 == 0) and iters >= 2, ONE cooperative launch of a persistent kernel for the whole call (grid
+ * barriers between the pass and the update; the HBM stream continues across iterations).  By default the library takes
+ * the persistent kernel for fp32 matrices of 64 MB and more, where it measures faster, and two kernels otherwise.
+ * lr_set_persistent(ctx, 0) forces two kernels (also used while lr_profile_enable is on, so that single launches can
+ * be timed), lr_set_persistent(ctx, 1) the persistent kernel wherever the shape allows it, a negative value restores
+ * the default.  The same choice applies to lr_fit_tol and the bfloat16 calls.
  */
 int lr_fit(lr_ctx* ctx, const float* d_X, const float* d_y, int64_t m, int32_t n,
            float lr, int32_t iters, float* d_w, float* d_b, float* d_loss_hist, void* stream);

@@ -295,9 +295,10 @@ class Context:
         """Ask for the first ``nbytes`` of X to be kept in L2 across the passes of a fit (0 = off)."""
         self._check(lib().lr_set_l2_keep(self._h, int(nbytes)), "lr_set_l2_keep")
 
-    def set_persistent(self, on: bool):
-        """Allow (default) or forbid the single-launch persistent kernel in ``fit``; results are identical either way."""
-        self._check(lib().lr_set_persistent(self._h, int(bool(on))), "lr_set_persistent")
+    def set_persistent(self, on: bool | None):
+        """Form of ``fit`` / ``fit_tol``: True = the single-launch persistent kernel wherever the shape allows, False = two
+        kernels per iteration, None = the library chooses (default).  Results are identical either way."""
+        self._check(lib().lr_set_persistent(self._h, -1 if on is None else int(bool(on))), "lr_set_persistent")
 
     def set_overlap(self, on: bool):
         """Allow (default) or forbid launching consecutive kernels of a call as programmatic dependents; same results."""

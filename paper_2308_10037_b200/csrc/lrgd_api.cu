@@ -134,7 +134,7 @@ struct lr_ctx {
     unsigned int* d_oticket = nullptr;
     unsigned int* d_gbar = nullptr;                 // grid-barrier counter of the persistent fit kernel
     bool coop = false;                              // device supports cooperative launches
-    bool persistent = true;                         // lr_fit may use the single-launch kernel
+    int persistent_mode = -1;                       // single-launch fit kernel: -1 the library chooses, 0 never, 1 whenever the shape allows
     bool overlap = true;                            // consecutive kernels of one call are launched as programmatic dependents
     int64_t l2_keep_bytes = -1;                     // leading bytes of X fetched with an evict-last hint; -1 = per-kernel default
     int64_t l2_bytes = 0;                           // size of the device's L2
@@ -300,6 +300,19 @@ int64_t keep_rows_for(const lr_ctx* ctx, int variant, int32_t n, bool bf16 = fal
     int64_t bytes = ctx->l2_keep_bytes;
     if (bytes < 0) bytes = variant == 1 ? ctx->l2_bytes / 4 * 3 : 0;
     return bytes / (int64_t(n) * (bf16 ? 2 : 4));
+}
+
+// Which form a multi-iteration fit on narrow rows takes.  Measured on B200 (ms per iteration, persistent launch against
+// two dependent-launched kernels): fp32 4M x 256 0.5759 / 0.5823, 16M x 64 0.594 / 0.608, 500k x 256 0.0832 / 0.0858,
+// 125k x 256 (128 MB) 0.0265 / 0.0271, 32k x 256 (32 MB) 0.0167 / 0.0153, 1k x 256 0.0092 / 0.0063; bfloat16 4M x 256
+// 0.3259 / 0.3163, 125k x 256 0.0247 / 0.0219.  The persistent kernel wins where the pass is bound by HBM and long enough
+// for the stages filled during its iteration boundary to matter: fp32 matrices from about half the L2 upwards.
+constexpr int64_t kPersistentMinBytes = int64_t(64) << 20;
+bool want_persistent(const lr_ctx* ctx, const lr_plan& P, bool bf16, int64_t m, int32_t n, int64_t iters) {
+    if (P.variant != 0 || !ctx->coop || ctx->prof || ctx->persistent_mode == 0) return false;
+    if (2 * iters * P.grid >= (int64_t(1) << 32)) return false;       // the grid-barrier counter is 32 bits
+    if (ctx->persistent_mode > 0) return true;
+    return !bf16 && m * n * 4 >= kPersistentMinBytes;
 }
 
 struct Pass {
@@ -587,8 +600,7 @@ int fit_impl(lr_ctx* ctx, const void* d_X, bool bf16, const float* d_y, int64_t 
     if (!g.ok) return LR_ERR_CUDA;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     // Narrow rows, several iterations: one cooperative launch runs the whole fit (same bits as the loop below).
-    if (P.variant == 0 && ctx->persistent && ctx->coop && !ctx->prof && iters >= 2 &&
-        2ll * iters * P.grid < (1ll << 32)) {
+    if (iters >= 2 && want_persistent(ctx, P, bf16, m, n, iters)) {
         const int64_t stage_stride = (int64_t(P.rows_per_batch) * n * (bf16 ? 2 : 4) + 127) & ~int64_t(127);
         const int64_t room = kMaxDynamicSmem - kHeaderBytes - kFitTailBytes;
         const int depth = int(std::max<int64_t>(1, std::min<int64_t>(P.stages, room / (kNW * stage_stride))));
@@ -657,7 +669,7 @@ int lr_set_overlap(lr_ctx* ctx, int32_t on) {
 
 int lr_set_persistent(lr_ctx* ctx, int32_t on) {
     if (!ctx) return LR_ERR_NULL;
-    ctx->persistent = on != 0;
+    ctx->persistent_mode = on < 0 ? -1 : (on > 0 ? 1 : 0);
     return LR_OK;
 }
 
@@ -686,7 +698,7 @@ int fit_tol_impl(lr_ctx* ctx, const void* d_X, bool bf16, const float* d_y, int6
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     LR_CK(ctx, cudaMemsetAsync(ctx->d_tol, 0, sizeof(TolState), st));
     // Narrow rows: one persistent launch that leaves its loop on the device as soon as the norm is small enough.
-    if (P.variant == 0 && ctx->persistent && ctx->coop && !ctx->prof && 2ll * max_iters * P.grid < (1ll << 32)) {
+    if (want_persistent(ctx, P, bf16, m, n, max_iters)) {
         const int64_t stage_stride = (int64_t(P.rows_per_batch) * n * (bf16 ? 2 : 4) + 127) & ~int64_t(127);
         const int64_t room = kMaxDynamicSmem - kHeaderBytes - kFitTailBytes;
         const int depth = int(std::max<int64_t>(1, std::min<int64_t>(P.stages, room / (kNW * stage_stride))));

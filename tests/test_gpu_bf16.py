@@ -133,6 +133,7 @@ def test_fit_and_predict_match_oracle(ctx, name, m):
     hist = torch.empty(iters, dtype=torch.float32, device="cuda")
     w = torch.zeros(wl.n, device="cuda")
     b = torch.zeros(1, device="cuda")
+    ctx.set_persistent(True)
     ctx.fit(dXh, dy, wl.lr, iters, w, b, hist)                    # one persistent launch
     got = np.concatenate([w.cpu().numpy(), b.cpu().numpy()])
     assert rel_l2(got, np.concatenate([w_ref, [b_ref]])) <= W_TOL
@@ -142,7 +143,7 @@ def test_fit_and_predict_match_oracle(ctx, name, m):
     w2 = torch.zeros(wl.n, device="cuda")
     b2 = torch.zeros(1, device="cuda")
     ctx.fit(dXh, dy, wl.lr, iters, w2, b2)
-    ctx.set_persistent(True)
+    ctx.set_persistent(None)
     assert torch.equal(w, w2) and torch.equal(b, b2)
     # predict at two thresholds; rows within fp32 noise of the cut may fall on either side
     for thr in (0.5, 0.3):
@@ -251,7 +252,7 @@ def test_stopping_rule_bf16(ctx):
             lh = torch.full((max_iters,), float("nan"), device="cuda")
             k, nrm = ctx.fit_tol(dXh, dy, wl.lr, eps, max_iters, w, b, check_every=7, loss_hist=lh)
         finally:
-            ctx.set_persistent(True)
+            ctx.set_persistent(None)
         assert k == k_ref == t_stop + 1 and abs(nrm - n_ref) <= 1e-4 * n_ref
         assert rel_l2(np.concatenate([w.cpu().numpy(), b.cpu().numpy()]), np.concatenate([w_ref, [b_ref]])) <= W_TOL
         lhc = lh.cpu().numpy()

@@ -56,7 +56,13 @@ def test_random_shape(ctx, m, n, iters, seed):
     # a short fit from that point (lr small enough for any of these shapes)
     lr = 0.05
     w_ref, b_ref, lh_ref = oracle.fit(X, y, lr, iters, w0=w, b0=b)
-    wf, bf, hf = api.lr_fit(dX, dy, lr, iters, w0=dw, b0=db, return_history=True, ctx=ctx)
+    ctx.set_persistent(True)                       # the persistent kernel wherever the shape allows it ...
+    try:
+        wf, bf, hf = api.lr_fit(dX, dy, lr, iters, w0=dw, b0=db, return_history=True, ctx=ctx)
+    finally:
+        ctx.set_persistent(None)
+    wa, ba, ha = api.lr_fit(dX, dy, lr, iters, w0=dw, b0=db, return_history=True, ctx=ctx)   # ... and the library's own choice
+    assert torch.equal(wf, wa) and torch.equal(bf, ba) and torch.equal(hf, ha)
     assert rel_l2(np.concatenate([wf.cpu().numpy(), bf.cpu().numpy()]), np.concatenate([w_ref, [b_ref]])) <= W_TOL
     assert np.max(np.abs(hf.cpu().numpy() - lh_ref)) <= LOSS_TOL
     # labels at the checker's parameters

@@ -230,22 +230,27 @@ def test_argument_errors_with_a_live_context(ctx):
 @pytest.mark.parametrize("name,m,iters", [("cfg1", 10_000, 25), ("cfg2", 150_007, 12), ("cfg3", 120_001, 9), ("cfg5", 300_000, 7),
                                            ("higgs_like", 200_003, 11), ("cfg1", 37, 5), ("cfg3", 9, 3)])
 def test_single_launch_fit_equals_two_kernel_fit(ctx, name, m, iters):
-    # lr_fit runs narrow-row problems as one persistent cooperative launch; forcing the two-kernels-per-iteration form
+    # lr_fit can run narrow-row problems as one persistent cooperative launch; the two-kernels-per-iteration form
     # must give the same bits (same batch map, same summation orders), including the loss history
     wl = datagen.scaled(datagen.WORKLOADS[name], m)
     X, y, _, _ = datagen.generate(wl)
     dX, dy = dev(X), dev(y)
-    n0 = ctx.launch_count()
-    w1, b1, h1 = api.lr_fit(dX, dy, wl.lr, iters, return_history=True, ctx=ctx)
-    assert ctx.launch_count() == n0 + 1                       # one launch for the whole fit
-    ctx.set_persistent(False)
     try:
+        ctx.set_persistent(True)
+        n0 = ctx.launch_count()
+        w1, b1, h1 = api.lr_fit(dX, dy, wl.lr, iters, return_history=True, ctx=ctx)
+        assert ctx.launch_count() == n0 + 1                       # one launch for the whole fit
+        ctx.set_persistent(False)
         n0 = ctx.launch_count()
         w2, b2, h2 = api.lr_fit(dX, dy, wl.lr, iters, return_history=True, ctx=ctx)
         assert ctx.launch_count() == n0 + 2 * iters
+        ctx.set_overlap(False)                                    # ordinary launches instead of dependent ones: same bits again
+        w3, b3, h3 = api.lr_fit(dX, dy, wl.lr, iters, return_history=True, ctx=ctx)
     finally:
-        ctx.set_persistent(True)
+        ctx.set_persistent(None)
+        ctx.set_overlap(True)
     assert torch.equal(w1, w2) and torch.equal(b1, b2) and torch.equal(h1, h2)
+    assert torch.equal(w3, w2) and torch.equal(b3, b2) and torch.equal(h3, h2)
     assert ctx.device_status() == 0
 
 

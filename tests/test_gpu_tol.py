@@ -64,7 +64,11 @@ def test_stops_at_the_same_iteration_as_the_checker(ctx, name, m, max_iters, n):
     w_ref, b_ref, k_ref, n_ref, lh_ref, gh_ref = oracle.fit_tol(X, y, wl.lr, eps, max_iters)
     assert k_ref == t_stop + 1
 
-    w, b, k, nrm, lh, gh = run_gpu(ctx, dX, dy, wl.n, wl.lr, eps, max_iters)
+    ctx.set_persistent(True)                                               # the rule inside the persistent kernel (narrow rows)
+    try:
+        w, b, k, nrm, lh, gh = run_gpu(ctx, dX, dy, wl.n, wl.lr, eps, max_iters)
+    finally:
+        ctx.set_persistent(None)
     assert k == k_ref
     assert abs(nrm - n_ref) <= 1e-4 * n_ref
     assert rel_l2(np.concatenate([w.cpu().numpy(), b.cpu().numpy()]), np.concatenate([w_ref, [b_ref]])) <= W_TOL
@@ -82,7 +86,7 @@ def test_stops_at_the_same_iteration_as_the_checker(ctx, name, m, max_iters, n):
             assert np.array_equal(gh2[:k], gh[:k]) and np.isnan(gh2[k:]).all()
             assert np.array_equal(lh2[:k], lh[:k]) and np.isnan(lh2[k:]).all()
     finally:
-        ctx.set_persistent(True)
+        ctx.set_persistent(None)
 
 
 def test_limits_of_the_rule(ctx):
