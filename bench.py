@@ -10,8 +10,9 @@ far larger than L2, so every iteration streams X from HBM).  One JSON line is pr
   value      iterations/s with X, y resident in HBM (CUDA events around one lr_fit call of K steps)
   e2e        the workload's own fit (its configured iteration count) through lr_fit_host: pinned host
              buffers in, parameters out, copies inside the timed region
-  roofline   narrow rows: the persistent kernel that runs all K timed iterations in one launch, K(4mn + 4m) bytes over
-             its duration; `single_pass` (and wide rows): one fused pass alone, from CUDA events around each launch
+  roofline   where lr_fit runs as one persistent launch (fp32 matrices of 64 MB and more with narrow rows): that kernel,
+             K(4mn + 4m) bytes over its duration; `single_pass` (and every other case): one fused pass alone, from CUDA
+             events around each launch
   cpu_baseline  the float64 CPU checker timed on this host on a bounded number of iterations
 
 With --gpus N > 1 (under torchrun) the rows are sharded: every rank holds one workload-sized block of
@@ -462,6 +463,9 @@ def main():
             "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "f32", "x_storage": args.x_dtype, "data": "synthetic", "config": workload_config(wl, world, args.x_dtype),
             "achieved_hbm_gbs_whole_step": bytes_per_launch * world * args.steps / (ms * 1e-3) / 1e9,
+            "fit_form": ("one persistent launch for all timed iterations" if launches == 1 and args.steps > 1 else
+                         f"{launches // max(args.steps, 1)} kernels per iteration"
+                         + ("" if args.no_overlap else ", each the programmatic dependent of the one before")),
             "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches, "clocks": clocks,
             "predict": predict}
     print(json.dumps(line))

@@ -134,9 +134,9 @@ int lr_set_l2_keep(lr_ctx* ctx, int64_t bytes);
  * Algorithm 7 -- for at most max_iters updates.  The norm is formed on the device in fp64 from the same
  * sums the update uses; once it is met a device flag turns every later launch of this call into a
  * no-op, so the result does not depend on check_every.  The host enqueues check_every iterations at a
- * time and then synchronises `stream` to read the flag (this call blocks, unlike lr_fit).  For rows of up to
- * 512 columns the whole run is instead ONE persistent launch in which all CTAs form the norm after every update
- * and leave the loop together (check_every is not used; no launch is wasted); both forms give the same bits.
+ * time and then synchronises `stream` to read the flag (this call blocks, unlike lr_fit).  Where lr_fit would take its
+ * persistent kernel (see lr_fit) the whole run is instead ONE persistent launch in which all CTAs form the norm after
+ * every update and leave the loop together (check_every is not used; no launch is wasted); both forms give the same bits.
  * d_w, d_b in/out as for lr_fit; d_loss_hist / d_gnorm_hist are NULL or [max_iters] (entries past the
  * stopping iteration are left untouched); *iters_done receives the number of updates applied and
  * *grad_norm the norm of the last applied gradient (-1 if max_iters == 0).  The caller tells
@@ -194,7 +194,8 @@ int lr_predict(lr_ctx* ctx, const float* d_X, int64_t m, int32_t n,
  * calls, each element of X is widened exactly to fp32 when it is used, so the three calls below compute exactly what
  * lr_loss_grad / lr_fit / lr_predict would compute on the fp32 matrix holding the same (bfloat16-representable) values.
  * The staged kernels take rows of n % 8 == 0 columns with d_Xh 16-byte aligned, up to n = 8192; other shapes run on the
- * unstaged kernel.  lr_fit_bf16 uses the single persistent launch for n <= 512, like lr_fit.  Errors as the fp32 calls.
+ * unstaged kernel.  lr_fit_bf16 runs as two dependent-launched kernels per iteration unless lr_set_persistent(ctx, 1) asks for
+ * the persistent kernel (n <= 512).  Errors as the fp32 calls.
  *
  * lr_convert_bf16 rounds `count` fp32 values to bfloat16 (round to nearest, ties to even; NaN stays NaN, values past
  * the largest finite bfloat16 become infinity) -- one elementwise kernel on `stream`; d_X and d_Xh must not overlap.
