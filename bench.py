@@ -39,12 +39,12 @@ NOMINAL_HBM_GBS = 8000.0
 # smaller row count of the same workload and scaled by rows; k_fit_rows: per row and iteration).  Keys: workload, with
 # "_bf16" for bfloat16 storage.  Remove an entry when its kernel changes.
 NCU_TRAFFIC_BYTES_PER_ROW = {
-    "cfg3": {"k_stream_rows": (514.024192e6 + 3.718656e6) / 500_000,
-             "k_fit_rows": (1.501455e9 + 3.736832e6) / 3 / 500_000},
-    "cfg4": {"k_stream_split": (491.679744e6 + 3.951616e6) / 30_000},
-    "cfg3_bf16": {"k_stream_rows": (516.048896e6 + 4.382976e6) / 1_000_000,
-                  "k_fit_rows": (1.503418e9 + 5.269504e6) / 3 / 1_000_000},
-    "cfg4_bf16": {"k_stream_split": (491.802624e6 + 4.932864e6) / 60_000},
+    "cfg3": {"k_stream_rows": (514.067712e6 + 4.353792e6) / 500_000,
+             "k_fit_rows": (1.501335e9 + 3.986176e6) / 3 / 500_000},
+    "cfg4": {"k_stream_split": (491.691264e6 + 4.271616e6) / 30_000},
+    "cfg3_bf16": {"k_stream_rows": (516.026112e6 + 3.413504e6) / 1_000_000,
+                  "k_fit_rows": (1.503216e9 + 5.057536e6) / 3 / 1_000_000},
+    "cfg4_bf16": {"k_stream_split": (491.804160e6 + 3.820032e6) / 60_000},
 }
 FALLBACK_HBM_GBS = 6650.0
 
