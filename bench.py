@@ -401,7 +401,7 @@ def main():
     achieved = bytes_per_launch / (k1_ms * 1e-3) / 1e9
     peak, peak_kind = measured_hbm_peak()
     plan = api.plan_query(wl.m, wl.n, sm_count=torch.cuda.get_device_properties(local_rank).multi_processor_count, bf16=bf16)
-    pass_kernel = {0: "k_stream_rows", 1: "k_stream_split", 2: "k_generic"}[plan["variant"]]
+    pass_kernel = {0: "k_stream_rows", 1: "k_stream_split", 2: "k_generic", 3: "k_stream_rows"}[plan["variant"]]
     per_row = NCU_TRAFFIC_BYTES_PER_ROW.get(args.workload + ("_bf16" if bf16 else ""), {})
     single_pass = {"kernel": f"{pass_kernel} (one fused loss/gradient pass, two-kernel form of lr_fit)", "achieved": achieved,
                    "unit": "GB/s", "frac": achieved / peak, "bytes_per_launch": bytes_per_launch, "avg_launch_ms": k1_ms,

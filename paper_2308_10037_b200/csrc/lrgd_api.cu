@@ -51,6 +51,19 @@ bool row_shape_for(int ng, bool bf16, RowShape* s) {
     return true;
 }
 
+// Narrow fp32 rows whose length is not a multiple of four: a lane owns single elements (nv of them per row).
+bool any_row_shape_for(int n, RowShape* s) {
+    if (n <= 8) *s = {1, 8, 8};
+    else if (n <= 16) *s = {1, 16, 8};
+    else if (n <= 32) *s = {1, 32, 16};
+    else if (n <= 64) *s = {2, 32, 16};
+    else if (n <= 128) *s = {4, 32, 8};
+    else if (n <= 256) *s = {8, 32, 4};
+    else if (n <= 512) *s = {16, 32, 2};
+    else return false;
+    return true;
+}
+
 // bf16: X holds bfloat16 (2-byte) elements instead of fp32; a 16-byte group is then 8 columns instead of 4.
 int make_plan(int64_t m, int32_t n, bool aligned16, int32_t sms, lr_plan* P, bool bf16 = false) {
     if (!P) return LR_ERR_NULL;
@@ -58,18 +71,20 @@ int make_plan(int64_t m, int32_t n, bool aligned16, int32_t sms, lr_plan* P, boo
     std::memset(P, 0, sizeof(*P));
     const int epg = bf16 ? 8 : 4, eb = bf16 ? 2 : 4;
     RowShape rs;
-    if (aligned16 && n % epg == 0 && row_shape_for(n / epg, bf16, &rs)) {
+    const bool grouped = aligned16 && n % epg == 0 && row_shape_for(n / epg, bf16, &rs);
+    const bool any_len = !grouped && aligned16 && !bf16 && n % 4 != 0 && any_row_shape_for(n, &rs);
+    if (grouped || any_len) {
         const int rpb = rs.rb * (32 / rs.lpr);                                  // rows per batch = rows per stage
         const int64_t B = (m + rpb - 1) / rpb;                                  // batches
         const int64_t slots = (B + kNW - 1) / kNW;                              // CTA-level groups of kNW batches
         const int grid = int(std::min<int64_t>(slots, sms));
         const int64_t per_warp = (slots + grid - 1) / grid;                     // most batches any warp handles
-        const int64_t stage_stride = (int64_t(rpb) * n * eb + 127) & ~int64_t(127);
+        const int64_t stage_stride = (int64_t(rpb) * n * eb + (any_len ? 16 : 0) + 127) & ~int64_t(127);   // as the kernel lays it out
         int D = int(std::min<int64_t>(kMaxDepth, kStageBudgetBytes / (kNW * stage_stride)));
         D = int(std::min<int64_t>(D, per_warp));
         if (D < 1) D = 1;
         const int64_t combine = int64_t(kNW) * n * 8 + 2 * kNW * 8;
-        P->variant = 0;
+        P->variant = grouped ? 0 : 3;
         P->lanes_per_row = rs.lpr;
         P->vec_per_lane = rs.nv;
         P->rows_per_batch = rpb;
@@ -204,6 +219,15 @@ cudaError_t launch_rows_t(const lr_plan& P, const StreamParams& sp, cudaStream_t
 
 template <bool PRED>
 cudaError_t launch_rows(const lr_plan& P, const StreamParams& sp, cudaStream_t st, bool bf16 = false, bool dependent = false) {
+    if (P.variant == 3) {                          // fp32 rows of any length: (lanes per row, elements per lane) picks the instantiation
+        if (P.lanes_per_row == 8) return launch_rows_t<ElemF32Any, 1, 8, 8, PRED>(P, sp, st, dependent);
+        if (P.lanes_per_row == 16) return launch_rows_t<ElemF32Any, 1, 16, 8, PRED>(P, sp, st, dependent);
+        if (P.vec_per_lane == 1) return launch_rows_t<ElemF32Any, 1, 32, 16, PRED>(P, sp, st, dependent);
+        if (P.vec_per_lane == 2) return launch_rows_t<ElemF32Any, 2, 32, 16, PRED>(P, sp, st, dependent);
+        if (P.vec_per_lane == 4) return launch_rows_t<ElemF32Any, 4, 32, 8, PRED>(P, sp, st, dependent);
+        if (P.vec_per_lane == 8) return launch_rows_t<ElemF32Any, 8, 32, 4, PRED>(P, sp, st, dependent);
+        return launch_rows_t<ElemF32Any, 16, 32, 2, PRED>(P, sp, st, dependent);
+    }
     if (bf16) {
         if (P.lanes_per_row == 8) return launch_rows_t<ElemBF16, 1, 8, 8, PRED>(P, sp, st, dependent);
         if (P.lanes_per_row == 16) return launch_rows_t<ElemBF16, 1, 16, 8, PRED>(P, sp, st, dependent);
@@ -341,7 +365,7 @@ int launch_stream_pass(lr_ctx* ctx, const lr_plan& P, const Pass& a, uint8_t* la
         LR_CK(ctx, cudaEventRecord(ctx->ev[2 * ctx->prof_used], st));
     }
     cudaError_t e;
-    if (P.variant == 0) {
+    if (P.variant == 0 || P.variant == 3) {
         StreamParams sp{};
         sp.X = a.X; sp.y = a.y; sp.m = a.m; sp.n = a.n; sp.w = a.w; sp.b = a.b;
         sp.partial = ctx->d_partial; sp.labels = labels; sp.cut = cut; sp.status = ctx->d_status; sp.stop = a.stop;
@@ -1099,7 +1123,7 @@ extern "C" int lr_loss_grad_noalloc(int32_t device, const float* d_X, const floa
     // fully rewritten by the CTAs that the reduction reads)
     if (cudaMemsetAsync(status, 0, sizeof(int), st) != cudaSuccess) return LR_ERR_CUDA;
     cudaError_t e;
-    if (P.variant == 0) {
+    if (P.variant == 0 || P.variant == 3) {
         StreamParams sp{};
         sp.X = d_X; sp.y = d_y; sp.m = m; sp.n = n; sp.w = d_w; sp.b = d_b;
         sp.partial = partial; sp.labels = nullptr; sp.cut = 0.f; sp.status = status;

@@ -334,11 +334,52 @@ struct LaneBF16 {
     }
 };
 
+// Rows of any length (fp32): the unit a lane owns is a single element, so a row needs no particular length.  Loads are
+// 32-bit (consecutive lanes read consecutive words: conflict-free), arithmetic is scalar FMAs in ownership order.
+template <int NV>
+struct LaneF32Any {
+    static constexpr int EPG = 1;
+    float wv[NV];
+    float acc[NV];
+    __device__ __forceinline__ void load_w(const float* w, int first_group, int group_stride, int group_limit, bool through_l2) {
+#pragma unroll
+        for (int k = 0; k < NV; ++k) {
+            const int idx = first_group + k * group_stride;
+            wv[k] = idx < group_limit ? (through_l2 ? __ldcg(w + idx) : __ldg(w + idx)) : 0.f;
+        }
+    }
+    __device__ __forceinline__ void zero() {
+#pragma unroll
+        for (int k = 0; k < NV; ++k) acc[k] = 0.f;
+    }
+    __device__ __forceinline__ float dot(const uint32_t (&xr)[NV]) const {
+        float d0 = 0.f, d1 = 0.f;                  // two chains: NV goes up to 16
+#pragma unroll
+        for (int k = 0; k < NV; ++k) {
+            if (k & 1) d1 = fmaf(__uint_as_float(xr[k]), wv[k], d1);
+            else d0 = fmaf(__uint_as_float(xr[k]), wv[k], d0);
+        }
+        return d0 + d1;
+    }
+    __device__ __forceinline__ void accumulate(const uint32_t (&xr)[NV], float er) {
+#pragma unroll
+        for (int k = 0; k < NV; ++k) acc[k] = fmaf(__uint_as_float(xr[k]), er, acc[k]);
+    }
+    __device__ __forceinline__ void fold(double (&dacc)[NV][1]) {
+#pragma unroll
+        for (int k = 0; k < NV; ++k) {
+            dacc[k][0] += acc[k];
+            acc[k] = 0.f;
+        }
+    }
+};
+
 // Storage types of X.  A "group" is 16 bytes of a row -- the unit of every shared-memory load and of the column
 // ownership of a lane: four fp32 values or eight bfloat16 values.  All arithmetic is fp32 for both.
 struct ElemF32 {
     static constexpr int EPG = 4;        // elements per 16-byte group
     static constexpr int BYTES = 4;      // bytes per element
+    using Raw = uint4;                   // a group as it sits in shared memory and registers
     template <int NV>
     using Lane = LaneF32<NV>;
     static __device__ __forceinline__ float load(const void* base, long long i) {
@@ -348,10 +389,23 @@ struct ElemF32 {
 struct ElemBF16 {
     static constexpr int EPG = 8;
     static constexpr int BYTES = 2;
+    using Raw = uint4;
     template <int NV>
     using Lane = LaneBF16<NV>;
     static __device__ __forceinline__ float load(const void* base, long long i) {
         return __uint_as_float(static_cast<uint32_t>(reinterpret_cast<const unsigned short*>(base)[i]) << 16);
+    }
+};
+
+// fp32 rows whose length is not a multiple of four: the "group" degenerates to one element (see LaneF32Any).
+struct ElemF32Any {
+    static constexpr int EPG = 1;
+    static constexpr int BYTES = 4;
+    using Raw = uint32_t;
+    template <int NV>
+    using Lane = LaneF32Any<NV>;
+    static __device__ __forceinline__ float load(const void* base, long long i) {
+        return reinterpret_cast<const float*>(base)[i];
     }
 };
 

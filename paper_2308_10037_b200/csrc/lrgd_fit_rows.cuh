@@ -91,6 +91,7 @@ __global__ void __launch_bounds__(NW * 32, 1) k_fit_rows(const FitParams p) {
     constexpr int SHIFT = LOG_LPR - LOG_RB;
     constexpr unsigned FULL = 0xffffffffu;
     static_assert(SHIFT >= 0, "rows per batch slot must not exceed lanes per row");
+    static_assert(E::EPG > 1, "rows of 16-byte groups only");
     static_assert(kRedSlices == 32, "one lane per reduction slice of k_reduce_update");
     static_assert(NW * kFitCombineCols * 8 + 2 * NW * 8 <= kFitTailBytes, "tail too small");
 
@@ -183,7 +184,7 @@ __global__ void __launch_bounds__(NW * 32, 1) k_fit_rows(const FitParams p) {
             const int rows = left < RPB ? static_cast<int>(left) : RPB;
             const uint4* t4 = reinterpret_cast<const uint4*>(my_stages + static_cast<size_t>(d) * stage_stride);
             uint4 x[RB][NV];
-            load_row_batch<NV, LPR, RB>(x, t4, rows, n4, full_cols && rows == RPB, sub, slot);
+            load_row_batch<uint4, NV, LPR, RB>(x, t4, rows, n4, full_cols && rows == RPB, sub, slot);
             const bool myvalid = myr < rows;
             const float yv = y_next;
             {

@@ -76,7 +76,7 @@ __device__ __forceinline__ void lane_reduce(float (&v)[RB], int lane) {
 // z partials: lane-local FMAs, then the transposing reduction; the returned value is the full dot product of the row
 // (r, with r = (lane_in_group >> (log2 LPR - log2 RB)) & (RB-1)) that ends up on this lane.
 template <class E, int NV, int LPR, int RB>
-__device__ __forceinline__ float batch_dot(const uint4 (&x)[RB][NV], const typename E::template Lane<NV>& lm, int lane) {
+__device__ __forceinline__ float batch_dot(const typename E::Raw (&x)[RB][NV], const typename E::template Lane<NV>& lm, int lane) {
     float v[RB];
 #pragma unroll
     for (int r = 0; r < RB; ++r) v[r] = lm.dot(x[r]);
@@ -86,7 +86,7 @@ __device__ __forceinline__ float batch_dot(const uint4 (&x)[RB][NV], const typen
 
 // acc[c] += x[r][c] * err[r]: each row's err is fetched from the lane that holds it (Algorithm 1's err.X on registers).
 template <class E, int NV, int LPR, int RB>
-__device__ __forceinline__ void batch_accumulate(const uint4 (&x)[RB][NV], float e, typename E::template Lane<NV>& lm) {
+__device__ __forceinline__ void batch_accumulate(const typename E::Raw (&x)[RB][NV], float e, typename E::template Lane<NV>& lm) {
     constexpr int SHIFT = Log2<LPR>::value - Log2<RB>::value;
 #pragma unroll
     for (int r = 0; r < RB; ++r) {
@@ -105,8 +105,8 @@ __device__ __forceinline__ void fold_into_fp64(typename E::template Lane<NV>& lm
 
 // one batch from a narrow-row stage into registers (rows packed at n4 groups; lanes beyond the row or rows beyond the
 // matrix read zeros); `full` = every lane's groups exist and the batch is complete: no bounds logic
-template <int NV, int LPR, int RB>
-__device__ __forceinline__ void load_row_batch(uint4 (&x)[RB][NV], const uint4* t4, int rows, int n4, bool full, int sub,
+template <class Raw, int NV, int LPR, int RB>
+__device__ __forceinline__ void load_row_batch(Raw (&x)[RB][NV], const Raw* t4, int rows, int n4, bool full, int sub,
                                                int slot) {
     constexpr int RPW = 32 / LPR;
     if (full) {
@@ -121,7 +121,7 @@ __device__ __forceinline__ void load_row_batch(uint4 (&x)[RB][NV], const uint4* 
 #pragma unroll
             for (int k2 = 0; k2 < NV; ++k2) {
                 const int idx = sub + k2 * LPR;
-                x[r8][k2] = (r < rows && idx < n4) ? t4[r * n4 + idx] : make_uint4(0u, 0u, 0u, 0u);
+                x[r8][k2] = (r < rows && idx < n4) ? t4[r * n4 + idx] : Raw{};
             }
         }
     }
@@ -148,7 +148,9 @@ __global__ void __launch_bounds__(NW * 32, 1) k_stream_rows(const StreamParams p
     const int D = p.depth;
     const int n = p.n, n4 = n / EPG;                   // n4 = 16-byte groups per row
     const uint32_t row_bytes = static_cast<uint32_t>(n) * E::BYTES;
-    const uint32_t stage_stride = (static_cast<uint32_t>(RPB) * row_bytes + 127u) & ~127u;
+    // rows of any length: a batch need not start on a 16-byte boundary; its copy then starts up to 12 bytes early
+    constexpr uint32_t kSlack = E::EPG == 1 ? 16u : 0u;
+    const uint32_t stage_stride = (static_cast<uint32_t>(RPB) * row_bytes + kSlack + 127u) & ~127u;
     unsigned char* my_stages = data + static_cast<size_t>(warp) * D * stage_stride;
     uint64_t* my_bars = bars + warp * kMaxDepth;
 
@@ -172,10 +174,29 @@ __global__ void __launch_bounds__(NW * 32, 1) k_stream_rows(const StreamParams p
         const long long left = p.m - r0;
         const uint32_t rows = left < RPB ? static_cast<uint32_t>(left) : RPB;
         const uint32_t xbytes = rows * row_bytes;
-        mbar_arrive_expect_tx(&my_bars[d], xbytes);
-        bulk_copy_g2s(my_stages + static_cast<size_t>(d) * stage_stride,
-                      static_cast<const unsigned char*>(p.X) + static_cast<size_t>(r0) * row_bytes, xbytes, &my_bars[d],
-                      r0 < p.keep_rows ? pol_keep : pol_stream);
+        unsigned char* dst = my_stages + static_cast<size_t>(d) * stage_stride;
+        const unsigned char* src = static_cast<const unsigned char*>(p.X) + static_cast<size_t>(r0) * row_bytes;
+        if constexpr (E::EPG == 1) {
+            static_assert(E::EPG != 1 || E::BYTES == 4, "the tail is moved in 32-bit words");
+            // rows of any length: neither the start nor the size of a batch need be a multiple of 16 bytes.  The bulk copy
+            // covers the 16-byte-aligned span that starts at or up to 12 bytes before the batch (those bytes belong to the
+            // row before it) and ends at or before its last byte; the few words left over at the end are moved by this
+            // lane with plain loads and stores.  Nothing outside [X, X + m*n) is read.  The batch then sits at dst + off.
+            const uint32_t off = static_cast<uint32_t>(reinterpret_cast<uintptr_t>(src)) & 15u;
+            const uint32_t span = off + xbytes;
+            const uint32_t bulk = span & ~15u;
+            if (bulk != 0u) {
+                mbar_arrive_expect_tx(&my_bars[d], bulk);
+                bulk_copy_g2s(dst, src - off, bulk, &my_bars[d], r0 < p.keep_rows ? pol_keep : pol_stream);
+            } else {
+                mbar_arrive(&my_bars[d]);
+            }
+            for (uint32_t o = bulk; o < span; o += 4u)
+                *reinterpret_cast<uint32_t*>(dst + o) = *reinterpret_cast<const uint32_t*>(src - off + o);
+        } else {
+            mbar_arrive_expect_tx(&my_bars[d], xbytes);
+            bulk_copy_g2s(dst, src, xbytes, &my_bars[d], r0 < p.keep_rows ? pol_keep : pol_stream);
+        }
     };
 
     typename E::template Lane<NV> lm;              // this lane's slice of w and its fp32 accumulators
@@ -195,6 +216,7 @@ __global__ void __launch_bounds__(NW * 32, 1) k_stream_rows(const StreamParams p
         const int pre = cnt < D ? cnt : D;
         for (int d = 0; d < pre; ++d) issue(row0 + d * stride_rows, d);
     }
+    __syncwarp();                                  // orders the plain stores a ragged tail may have needed before the warp's reads
     float y_next = 0.f;                            // y of this lane's row in the next batch, loaded one batch ahead
     if constexpr (!PREDICT) {
         if (cnt > 0 && row0 + myr < p.m) y_next = __ldg(p.y + row0 + myr);
@@ -227,12 +249,16 @@ __global__ void __launch_bounds__(NW * 32, 1) k_stream_rows(const StreamParams p
         ok = __all_sync(FULL, ok);
         if (!ok) break;
         done = i + 1;
+        if constexpr (E::EPG == 1) __syncwarp();   // lane 0 may have completed this stage with plain stores
 
         const long long left = p.m - row0;
         const int rows = left < RPB ? static_cast<int>(left) : RPB;
-        const uint4* t4 = reinterpret_cast<const uint4*>(my_stages + static_cast<size_t>(d) * stage_stride);
-        uint4 x[RB][NV];
-        load_row_batch<NV, LPR, RB>(x, t4, rows, n4, full_cols && rows == RPB, sub, slot);
+        using Raw = typename E::Raw;
+        // (rows of any length: the batch sits where its first byte fell within the 16-byte-aligned copy; X itself is aligned)
+        const uint32_t off = E::EPG == 1 ? static_cast<uint32_t>((row0 * row_bytes) & 15) : 0u;
+        const Raw* t4 = reinterpret_cast<const Raw*>(my_stages + static_cast<size_t>(d) * stage_stride + off);
+        Raw x[RB][NV];
+        load_row_batch<Raw, NV, LPR, RB>(x, t4, rows, n4, full_cols && rows == RPB, sub, slot);
         const bool myvalid = myr < rows;
         const float yv = y_next;
         if constexpr (!PREDICT) {

@@ -68,11 +68,25 @@ def test_plan_staged_shapes(m, n, lpr, nv):
 
 
 def test_plan_falls_back_for_unaligned_or_odd_shapes():
-    assert api.plan_query(1000, 30)["variant"] == 2          # n not a multiple of 4
+    assert api.plan_query(1000, 515)["variant"] == 2         # n not a multiple of 4 and wider than 512
     assert api.plan_query(1000, 32, x_aligned16=False)["variant"] == 2
+    assert api.plan_query(1000, 30, x_aligned16=False)["variant"] == 2
     assert api.plan_query(1000, 8192)["variant"] == 2         # wider than any staged kernel
-    g = api.plan_query(100, 30)
+    assert api.plan_query(1000, 30, bf16=True)["variant"] == 2   # bfloat16 rows must be whole 16-byte groups
+    g = api.plan_query(100, 515)
     assert g["grid"] == 2 and g["threads"] == 256
+
+
+@pytest.mark.parametrize("n,lpr,nv,rb", [(1, 8, 1, 8), (7, 8, 1, 8), (13, 16, 1, 8), (30, 32, 1, 16), (33, 32, 2, 16), (101, 32, 4, 8),
+                                         (255, 32, 8, 4), (258, 32, 16, 2), (511, 32, 16, 2)])
+def test_plan_rows_of_any_length(n, lpr, nv, rb):
+    # fp32 rows whose length is not a multiple of four still take a staged kernel: a lane owns single elements
+    p = api.plan_query(200_003, n)
+    assert p["variant"] == 3 and p["lanes_per_row"] == lpr and p["vec_per_lane"] == nv
+    assert p["rows_per_batch"] == rb * (32 // lpr)
+    assert nv * lpr >= n and p["smem_bytes"] <= 227 * 1024
+    stage = -(-(p["tile_rows"] * n * 4 + 16) // 128) * 128      # a batch may start up to 12 bytes into its stage
+    assert 1024 + 16 * p["stages"] * stage <= p["smem_bytes"]
 
 
 @pytest.mark.parametrize("m,n,nv,rb", [(100_000, 4096, 2, 4), (5000, 1024, 1, 8), (5000, 516, 1, 8), (5000, 2052, 2, 4)])
@@ -119,3 +133,34 @@ def test_header_is_plain_c_and_the_example_links():
         subprocess.check_call([os.path.join(tmp, "probe")])          # pure host entry point: runs without a GPU
         subprocess.check_call([gcc, "-std=c99", "-Wall", "-Werror", "-O1", "-I", inc, os.path.join(pkg, "examples", "fit_host.c"),
                                "-L", pkg, "-llrgd", f"-Wl,-rpath,{pkg}", "-lm", "-o", os.path.join(tmp, "fit_host")])
+
+
+def test_any_length_copies_stay_inside_the_matrix():
+    """The staged kernel for rows of any length copies, per batch, the 16-byte-aligned span that starts at or just before
+    the batch and ends at or before its last byte, and moves the few words left over with plain loads.  This replays
+    that arithmetic for every batch of many shapes: aligned bulk copies, nothing read outside the matrix, every byte of
+    the matrix covered once, nothing written outside the stage."""
+    import random
+    rnd = random.Random(1)
+    shapes = [(2758, 449), (1, 1), (7, 3), (300, 1), (640, 30), (1025, 101), (526, 255), (999, 511), (5, 510), (3, 258),
+              (17, 257), (2, 449), (1, 511)]
+    shapes += [(rnd.randint(1, 3000), rnd.choice([n for n in range(1, 513) if n % 4])) for _ in range(200)]
+    for m, n in shapes:
+        p = api.plan_query(m, n)
+        assert p["variant"] == 3
+        rpb, row_bytes, total = p["rows_per_batch"], 4 * n, 4 * m * n
+        stage = -(-(rpb * row_bytes + 16) // 128) * 128
+        assert 1024 + 16 * p["stages"] * stage <= p["smem_bytes"]
+        covered = 0
+        for g in range(-(-m // rpb)):
+            r0 = g * rpb
+            xbytes = min(rpb, m - r0) * row_bytes
+            src = r0 * row_bytes                         # X itself is 16-byte aligned: offsets stand for addresses
+            off = src & 15
+            span = off + xbytes
+            bulk = span & ~15
+            assert (src - off) % 16 == 0 and src - off >= 0 and src - off + bulk <= total
+            assert span <= stage and span - bulk < 16 and (span - bulk) % 4 == 0
+            assert all(0 <= src - off + o < total for o in range(bulk, span, 4))
+            covered += xbytes
+        assert covered == total

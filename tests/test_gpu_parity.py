@@ -43,8 +43,9 @@ def check_loss_grad(ctx, X, y, w, b, grad_tol=GRAD_TOL, loss_tol=LOSS_TOL):
 
 
 # shapes: every staged instantiation (n/4 <= 8, 16, 32, 64, 128), partly filled lane groups (28, 100, 200, 36),
-# the unstaged kernel (n % 4 != 0, n > 512), and row counts that are tiny, ragged, or span many tiles
-SHAPES = [(1, 4), (7, 4), (8, 3), (33, 28), (1000, 32), (4097, 32), (5003, 64), (2500, 36), (3001, 100), (9999, 256),
+# rows of any length (n % 4 != 0, n <= 512), the unstaged kernel (n % 4 != 0 and n > 512, n > 4096), and row counts that
+# are tiny, ragged, or span many tiles
+SHAPES = [(777, 515), (301, 1001), (1, 4), (7, 4), (8, 3), (33, 28), (1000, 32), (4097, 32), (5003, 64), (2500, 36), (3001, 100), (9999, 256),
           (777, 200), (1500, 512), (2049, 260), (640, 30), (1025, 101), (300, 1), (130, 4096), (50, 8192), (20011, 8),
           # enough rows that every warp refills its shared-memory stages many times, with a ragged last batch
           (200_003, 256), (400_001, 32), (200_002, 64), (120_007, 100), (150_001, 28), (60_001, 512), (90_001, 200),
@@ -159,6 +160,32 @@ def test_predict_matches_oracle(ctx, m, n):
         clear = np.abs(z - cut) > 1e-4 * (1 + np.abs(z))   # rows whose decision is not within fp32 noise of the cut
         assert np.array_equal(got[clear], ref[clear])
         assert (got == ref).mean() >= LABEL_AGREE or m < 10_000 and (got != ref).sum() <= 1
+
+
+# fp32 rows whose length is not a multiple of four (a lane owns single elements): every instantiation (n <= 8, 16, 32, 64,
+# 128, 256, 512), batches that do not start on a 16-byte boundary (two-row batches of odd-length rows), ragged tails whose
+# byte count is not a multiple of 16, stage reuse
+ANY_LENGTH = [(33, 7), (1, 3), (20_011, 5), (40_003, 13), (150_001, 30), (90_001, 49), (100_001, 101), (200_003, 255),
+              (2_758, 449), (60_001, 449), (50_002, 511), (5, 510), (3, 258), (17, 257), (70_001, 258), (1, 511)]
+
+
+@pytest.mark.parametrize("m,n", ANY_LENGTH)
+def test_rows_of_any_length(ctx, m, n):
+    assert api.plan_query(m, n)["variant"] == 3
+    X, y, w, b = datagen.random_problem(m, n, seed=3000 + m + n, wscale=1.5)
+    check_loss_grad(ctx, X, y, w, b)
+    # labels, including the word-packed stores
+    dX, dw, db = dev(X), dev(w), dev(np.array([b], dtype=np.float32))
+    ref, z = oracle.predict(X, w, b, 0.4, return_z=True)
+    got = ctx.predict(dX, dw, db, 0.4).cpu().numpy()
+    clear = np.abs(z - math.log(0.4 / 0.6)) > 1e-4 * (1 + np.abs(z))
+    assert np.array_equal(got[clear], ref[clear])
+    # a short fit (two dependent-launched kernels per iteration: these shapes have no persistent form)
+    iters, lr = 6, 0.1
+    w_ref, b_ref, lh_ref = oracle.fit(X, y, lr, iters, w0=w, b0=b)
+    wf, bf, hf = api.lr_fit(dX, dev(y), lr, iters, w0=dw, b0=db, return_history=True, ctx=ctx)
+    assert rel_l2(np.concatenate([wf.cpu().numpy(), bf.cpu().numpy()]), np.concatenate([w_ref, [b_ref]])) <= W_TOL
+    assert np.max(np.abs(hf.cpu().numpy() - lh_ref)) <= LOSS_TOL
 
 
 @pytest.mark.parametrize("m,n", [(70_003, 64), (9_001, 2048), (40_001, 28)])
