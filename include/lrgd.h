@@ -51,8 +51,8 @@ typedef struct lr_ctx lr_ctx;
 /* Launch plan for a given shape, as chosen by the host logic (pure host code, no CUDA call). */
 typedef struct lr_plan {
     int32_t variant;       /* 0 = row-per-lane-group staged kernel, 1 = row-split staged kernel, 2 = unstaged generic kernel,
-                              3 = row-per-lane-group staged kernel for fp32 rows of any length up to 512 (a lane owns single
-                              elements: vec_per_lane counts elements, not 16-byte groups) */
+                              3 = row-per-lane-group staged kernel for fp32 rows of any length up to 512 and any 4-byte aligned
+                              matrix (a lane owns single elements: vec_per_lane counts elements, not 16-byte groups) */
     int32_t lanes_per_row; /* staged kernels: lanes that share one row (8, 16, 32; 512 for the row-split kernel) */
     int32_t vec_per_lane;  /* staged kernels: 16-byte column groups owned by one lane */
     int32_t rows_per_batch;/* rows one warp (or one CTA for the row-split kernel) holds in registers at a time */
@@ -85,9 +85,9 @@ int lr_destroy(lr_ctx* ctx);
  *   d_loss[0] = loss, d_grad_w[0..n) = X^T err / m, d_grad_b[0] = sum err / m.
  * Inputs d_X [m*n], d_y [m], d_w [n], d_b [1] are read only.  Two kernels are enqueued: the fused
  * streaming kernel (reads X once) and the fixed-order cross-CTA reduction.
- * Which streaming kernel runs depends on the shape (lr_plan_query tells): with d_X 16-byte aligned, rows of up to 512
- * columns of any length and rows of up to 4096 columns with n % 4 == 0 take the staged kernels that run at HBM speed;
- * anything else (unaligned d_X, wider rows, 512 < n with n % 4 != 0) runs on a slower unstaged kernel.
+ * Which streaming kernel runs depends on the shape (lr_plan_query tells): rows of up to 512 columns always take a staged
+ * kernel that runs at or near HBM speed (fastest with d_X 16-byte aligned and n % 4 == 0); so do rows of up to 4096
+ * columns with n % 4 == 0 and d_X 16-byte aligned; anything else runs on a slower unstaged kernel.
  */
 int lr_loss_grad(lr_ctx* ctx, const float* d_X, const float* d_y, int64_t m, int32_t n,
                  const float* d_w, const float* d_b,

@@ -51,7 +51,8 @@ bool row_shape_for(int ng, bool bf16, RowShape* s) {
     return true;
 }
 
-// Narrow fp32 rows whose length is not a multiple of four: a lane owns single elements (nv of them per row).
+// Narrow fp32 rows whose length is not a multiple of four, or whose matrix is not 16-byte aligned: a lane owns single
+// elements (nv of them per row).
 bool any_row_shape_for(int n, RowShape* s) {
     if (n <= 8) *s = {1, 8, 8};
     else if (n <= 16) *s = {1, 16, 8};
@@ -72,7 +73,8 @@ int make_plan(int64_t m, int32_t n, bool aligned16, int32_t sms, lr_plan* P, boo
     const int epg = bf16 ? 8 : 4, eb = bf16 ? 2 : 4;
     RowShape rs;
     const bool grouped = aligned16 && n % epg == 0 && row_shape_for(n / epg, bf16, &rs);
-    const bool any_len = !grouped && aligned16 && !bf16 && n % 4 != 0 && any_row_shape_for(n, &rs);
+    // fp32 rows that cannot be cut into aligned 16-byte groups (length not a multiple of four, or X only 4-byte aligned)
+    const bool any_len = !grouped && !bf16 && any_row_shape_for(n, &rs);
     if (grouped || any_len) {
         const int rpb = rs.rb * (32 / rs.lpr);                                  // rows per batch = rows per stage
         const int64_t B = (m + rpb - 1) / rpb;                                  // batches

@@ -178,20 +178,25 @@ __global__ void __launch_bounds__(NW * 32, 1) k_stream_rows(const StreamParams p
         const unsigned char* src = static_cast<const unsigned char*>(p.X) + static_cast<size_t>(r0) * row_bytes;
         if constexpr (E::EPG == 1) {
             static_assert(E::EPG != 1 || E::BYTES == 4, "the tail is moved in 32-bit words");
-            // rows of any length: neither the start nor the size of a batch need be a multiple of 16 bytes.  The bulk copy
-            // covers the 16-byte-aligned span that starts at or up to 12 bytes before the batch (those bytes belong to the
-            // row before it) and ends at or before its last byte; the few words left over at the end are moved by this
-            // lane with plain loads and stores.  Nothing outside [X, X + m*n) is read.  The batch then sits at dst + off.
+            // rows of any length, X 4-byte aligned: neither the start nor the size of a batch need be a multiple of 16
+            // bytes.  The batch lands at dst + off, off = its address mod 16.  The bulk copy covers the 16-byte-aligned span
+            // that starts at or up to 12 bytes before the batch (bytes of the row before it) and ends at or before its last
+            // byte; for the very first batch of a matrix that is itself not 16-byte aligned it starts at the first boundary
+            // inside the batch instead.  The few words left over at either end are moved by this lane with plain loads and
+            // stores.  Nothing outside [X, X + m*n) is read.
             const uint32_t off = static_cast<uint32_t>(reinterpret_cast<uintptr_t>(src)) & 15u;
-            const uint32_t span = off + xbytes;
-            const uint32_t bulk = span & ~15u;
+            const uint32_t span = off + xbytes;                                   // stage bytes [off, span) hold the batch
+            const uint32_t lo = (r0 == 0 && off != 0u) ? 16u : 0u;                // first stage byte the bulk copy writes
+            const uint32_t bulk = span > lo ? (span - lo) & ~15u : 0u;
             if (bulk != 0u) {
                 mbar_arrive_expect_tx(&my_bars[d], bulk);
-                bulk_copy_g2s(dst, src - off, bulk, &my_bars[d], r0 < p.keep_rows ? pol_keep : pol_stream);
+                bulk_copy_g2s(dst + lo, src - off + lo, bulk, &my_bars[d], r0 < p.keep_rows ? pol_keep : pol_stream);
             } else {
                 mbar_arrive(&my_bars[d]);
             }
-            for (uint32_t o = bulk; o < span; o += 4u)
+            for (uint32_t o = off; o < lo && o < span; o += 4u)                   // head (first batch of an unaligned matrix only)
+                *reinterpret_cast<uint32_t*>(dst + o) = *reinterpret_cast<const uint32_t*>(src - off + o);
+            for (uint32_t o = lo + bulk; o < span; o += 4u)                       // tail
                 *reinterpret_cast<uint32_t*>(dst + o) = *reinterpret_cast<const uint32_t*>(src - off + o);
         } else {
             mbar_arrive_expect_tx(&my_bars[d], xbytes);
@@ -254,8 +259,8 @@ __global__ void __launch_bounds__(NW * 32, 1) k_stream_rows(const StreamParams p
         const long long left = p.m - row0;
         const int rows = left < RPB ? static_cast<int>(left) : RPB;
         using Raw = typename E::Raw;
-        // (rows of any length: the batch sits where its first byte fell within the 16-byte-aligned copy; X itself is aligned)
-        const uint32_t off = E::EPG == 1 ? static_cast<uint32_t>((row0 * row_bytes) & 15) : 0u;
+        // (rows of any length: the batch sits at its address mod 16 within the stage)
+        const uint32_t off = E::EPG == 1 ? static_cast<uint32_t>((reinterpret_cast<uintptr_t>(p.X) + row0 * row_bytes) & 15u) : 0u;
         const Raw* t4 = reinterpret_cast<const Raw*>(my_stages + static_cast<size_t>(d) * stage_stride + off);
         Raw x[RB][NV];
         load_row_batch<Raw, NV, LPR, RB>(x, t4, rows, n4, full_cols && rows == RPB, sub, slot);

@@ -69,8 +69,10 @@ def test_plan_staged_shapes(m, n, lpr, nv):
 
 def test_plan_falls_back_for_unaligned_or_odd_shapes():
     assert api.plan_query(1000, 515)["variant"] == 2         # n not a multiple of 4 and wider than 512
-    assert api.plan_query(1000, 32, x_aligned16=False)["variant"] == 2
-    assert api.plan_query(1000, 30, x_aligned16=False)["variant"] == 2
+    assert api.plan_query(1000, 516, x_aligned16=False)["variant"] == 2    # wide rows need a 16-byte aligned matrix
+    assert api.plan_query(1000, 32, x_aligned16=False)["variant"] == 3     # narrow rows do not: element-wise staged kernel
+    assert api.plan_query(1000, 30, x_aligned16=False)["variant"] == 3
+    assert api.plan_query(1000, 32, x_aligned16=False, bf16=True)["variant"] == 2
     assert api.plan_query(1000, 8192)["variant"] == 2         # wider than any staged kernel
     assert api.plan_query(1000, 30, bf16=True)["variant"] == 2   # bfloat16 rows must be whole 16-byte groups
     g = api.plan_query(100, 515)
@@ -137,30 +139,42 @@ def test_header_is_plain_c_and_the_example_links():
 
 def test_any_length_copies_stay_inside_the_matrix():
     """The staged kernel for rows of any length copies, per batch, the 16-byte-aligned span that starts at or just before
-    the batch and ends at or before its last byte, and moves the few words left over with plain loads.  This replays
-    that arithmetic for every batch of many shapes: aligned bulk copies, nothing read outside the matrix, every byte of
-    the matrix covered once, nothing written outside the stage."""
+    the batch (at the first boundary inside it for the first batch of a matrix that is not 16-byte aligned) and ends at or
+    before its last byte, and moves the few words left over with plain loads.  This replays that arithmetic for every
+    batch of many shapes and base alignments: aligned bulk copies, nothing read outside the matrix, every byte of the
+    matrix covered exactly once, nothing written outside the stage."""
     import random
     rnd = random.Random(1)
     shapes = [(2758, 449), (1, 1), (7, 3), (300, 1), (640, 30), (1025, 101), (526, 255), (999, 511), (5, 510), (3, 258),
               (17, 257), (2, 449), (1, 511)]
     shapes += [(rnd.randint(1, 3000), rnd.choice([n for n in range(1, 513) if n % 4])) for _ in range(200)]
-    for m, n in shapes:
-        p = api.plan_query(m, n)
+    cases = [(m, n, 0) for m, n in shapes]
+    cases += [(m, n, base) for (m, n) in shapes[:60] + [(1, 1), (2, 2), (3, 1), (40, 32), (999, 256), (77, 512)] for base in (4, 8, 12)]
+    for m, n, base in cases:
+        p = api.plan_query(m, n, x_aligned16=(base == 0))
         assert p["variant"] == 3
-        rpb, row_bytes, total = p["rows_per_batch"], 4 * n, 4 * m * n
+        rpb, row_bytes = p["rows_per_batch"], 4 * n
+        lo_x, hi_x = 4096 + base, 4096 + base + 4 * m * n          # the matrix occupies the addresses [lo_x, hi_x)
         stage = -(-(rpb * row_bytes + 16) // 128) * 128
         assert 1024 + 16 * p["stages"] * stage <= p["smem_bytes"]
-        covered = 0
+        seen = 0
         for g in range(-(-m // rpb)):
             r0 = g * rpb
             xbytes = min(rpb, m - r0) * row_bytes
-            src = r0 * row_bytes                         # X itself is 16-byte aligned: offsets stand for addresses
+            src = lo_x + r0 * row_bytes
             off = src & 15
             span = off + xbytes
-            bulk = span & ~15
-            assert (src - off) % 16 == 0 and src - off >= 0 and src - off + bulk <= total
-            assert span <= stage and span - bulk < 16 and (span - bulk) % 4 == 0
-            assert all(0 <= src - off + o < total for o in range(bulk, span, 4))
-            covered += xbytes
-        assert covered == total
+            lo = 16 if (r0 == 0 and off != 0) else 0
+            bulk = ((span - lo) & ~15) if span > lo else 0
+            assert span <= stage
+            if bulk:
+                assert (src - off + lo) % 16 == 0 and lo_x <= src - off + lo and src - off + lo + bulk <= hi_x
+            head = list(range(off, min(lo, span), 4))
+            tail = list(range(lo + bulk, span, 4))
+            assert len(head) <= 3 and len(tail) <= 3
+            assert all(lo_x <= src - off + o and src - off + o + 4 <= hi_x for o in head + tail)
+            # every byte of the batch is written exactly once: head, bulk and tail tile [off, span) of the stage
+            written = sorted(head + tail + list(range(lo, lo + bulk, 4)))
+            assert [o for o in written if o >= off] == list(range(off, span, 4))
+            seen += xbytes
+        assert seen == 4 * m * n

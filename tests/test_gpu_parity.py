@@ -76,7 +76,28 @@ def test_saturated_rows_stay_finite(ctx):
     assert np.isfinite(got).all()
 
 
-def test_unaligned_views_use_the_unstaged_kernel(ctx):
+@pytest.mark.parametrize("m,n,shift", [(1201, 32, 1), (150_003, 30, 1), (60_001, 256, 2), (40_001, 449, 3), (9, 5, 3), (1, 1, 1),
+                                       (2_001, 516, 1), (301, 1001, 2)])
+def test_matrices_that_are_only_4_byte_aligned(ctx, m, n, shift):
+    # a view that starts `shift` floats into an allocation: narrow rows stay on a staged kernel (element-wise groups; the
+    # first batch is completed with plain loads instead of reading in front of the matrix), wide rows run unstaged
+    X, y, w, b = datagen.random_problem(m, n, seed=4000 + m + n)
+    buf = torch.full((X.size + 8,), float("nan"), dtype=torch.float32, device="cuda")      # NaN all around the view
+    buf[shift:shift + X.size] = dev(X).ravel()
+    Xv = buf[shift:shift + X.size].view(m, n)
+    assert Xv.data_ptr() % 16 == 4 * shift
+    assert api.plan_query(m, n, x_aligned16=False)["variant"] == (3 if n <= 512 else 2)
+    L, g, g0 = oracle.loss_grad(X, y, w, b)
+    dl, dg, dg0 = ctx.loss_grad(Xv, dev(y), dev(w), dev(np.array([b], dtype=np.float32)))
+    assert abs(dl.item() - L) <= LOSS_TOL
+    assert rel_l2(np.concatenate([dg.cpu().numpy(), dg0.cpu().numpy()]), np.concatenate([g, [g0]])) <= GRAD_TOL
+    ref, z = oracle.predict(X, w, b, 0.5, return_z=True)
+    got = ctx.predict(Xv, dev(w), dev(np.array([b], dtype=np.float32)), 0.5).cpu().numpy()
+    clear = np.abs(z) > 1e-4 * (1 + np.abs(z))
+    assert np.array_equal(got[clear], ref[clear])
+
+
+def test_unaligned_views(ctx):
     X, y, w, b = datagen.random_problem(1201, 32, seed=11)
     buf = torch.zeros(X.size + 1, dtype=torch.float32, device="cuda")
     buf[1:] = dev(X).ravel()
