@@ -37,16 +37,19 @@ constexpr int64_t kMaxRows = int64_t(1) << 40;
 #define LRGD_NV2_RB 4                          // register batch (rows per warp) of the 132..256-column instantiation
 #endif
 
-struct RowShape { int nv, lpr, rb; };
+struct RowShape { int nv, lpr, rb; int nw = kNW; };    // nw = warps per CTA
 
 // Which instantiation of the narrow-row kernel covers ng 16-byte column groups per row.  bfloat16 rows stop at 64
 // groups: a lane that owns four groups of eight columns would need more registers than a 512-thread CTA can give.
+// fp32 rows of 129..256 groups (516..1024 columns) run with eight warps per CTA, so that a thread may hold the eight
+// groups of its row slice, their weights and accumulators (up to 255 registers); the bytes in flight per SM stay the same.
 bool row_shape_for(int ng, bool bf16, RowShape* s) {
     if (ng <= 8) *s = {1, 8, 8};
     else if (ng <= 16) *s = {1, 16, 8};
     else if (ng <= 32) *s = {1, 32, LRGD_NV1_RB};
     else if (ng <= 64) *s = {2, 32, LRGD_NV2_RB};
     else if (ng <= 128 && !bf16) *s = {4, 32, 2};
+    else if (ng <= 256 && !bf16) *s = {8, 32, 2, 8};
     else return false;
     return true;
 }
@@ -78,14 +81,14 @@ int make_plan(int64_t m, int32_t n, bool aligned16, int32_t sms, lr_plan* P, boo
     if (grouped || any_len) {
         const int rpb = rs.rb * (32 / rs.lpr);                                  // rows per batch = rows per stage
         const int64_t B = (m + rpb - 1) / rpb;                                  // batches
-        const int64_t slots = (B + kNW - 1) / kNW;                              // CTA-level groups of kNW batches
+        const int64_t slots = (B + rs.nw - 1) / rs.nw;                              // CTA-level groups of nw batches
         const int grid = int(std::min<int64_t>(slots, sms));
         const int64_t per_warp = (slots + grid - 1) / grid;                     // most batches any warp handles
         const int64_t stage_stride = (int64_t(rpb) * n * eb + (any_len ? 16 : 0) + 127) & ~int64_t(127);   // as the kernel lays it out
-        int D = int(std::min<int64_t>(kMaxDepth, kStageBudgetBytes / (kNW * stage_stride)));
+        int D = int(std::min<int64_t>(kMaxDepth, kStageBudgetBytes / (rs.nw * stage_stride)));
         D = int(std::min<int64_t>(D, per_warp));
         if (D < 1) D = 1;
-        const int64_t combine = int64_t(kNW) * n * 8 + 2 * kNW * 8;
+        const int64_t combine = int64_t(rs.nw) * n * 8 + 2 * rs.nw * 8;
         P->variant = grouped ? 0 : 3;
         P->lanes_per_row = rs.lpr;
         P->vec_per_lane = rs.nv;
@@ -93,8 +96,8 @@ int make_plan(int64_t m, int32_t n, bool aligned16, int32_t sms, lr_plan* P, boo
         P->tile_rows = rpb;
         P->stages = D;
         P->grid = grid;
-        P->threads = kNW * 32;
-        P->smem_bytes = int(kHeaderBytes + std::max<int64_t>(int64_t(kNW) * D * stage_stride, combine));
+        P->threads = rs.nw * 32;
+        P->smem_bytes = int(kHeaderBytes + std::max<int64_t>(int64_t(rs.nw) * D * stage_stride, combine));
         if (per_warp >= (int64_t(1) << 31)) return LR_ERR_SHAPE;
         return LR_OK;
     }
@@ -211,9 +214,9 @@ cudaError_t launch_kernel(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t 
     return cudaLaunchKernelEx(&cfg, kern, std::forward<Args>(args)...);
 }
 
-template <class E, int NV, int LPR, int RB, bool PRED>
+template <class E, int NV, int LPR, int RB, bool PRED, int NW = kNW>
 cudaError_t launch_rows_t(const lr_plan& P, const StreamParams& sp, cudaStream_t st, bool dependent) {
-    auto kern = k_stream_rows<E, NV, LPR, RB, kNW, PRED>;
+    auto kern = k_stream_rows<E, NV, LPR, RB, NW, PRED>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, P.smem_bytes);
     if (e != cudaSuccess) return e;
     return launch_kernel(kern, dim3(P.grid), dim3(P.threads), size_t(P.smem_bytes), st, dependent, sp);
@@ -241,6 +244,7 @@ cudaError_t launch_rows(const lr_plan& P, const StreamParams& sp, cudaStream_t s
     if (P.lanes_per_row == 16) return launch_rows_t<ElemF32, 1, 16, 8, PRED>(P, sp, st, dependent);
     if (P.vec_per_lane == 1) return launch_rows_t<ElemF32, 1, 32, LRGD_NV1_RB, PRED>(P, sp, st, dependent);
     if (P.vec_per_lane == 2) return launch_rows_t<ElemF32, 2, 32, LRGD_NV2_RB, PRED>(P, sp, st, dependent);
+    if (P.vec_per_lane == 8) return launch_rows_t<ElemF32, 8, 32, 2, PRED, 8>(P, sp, st, dependent);      // eight warps per CTA
     return launch_rows_t<ElemF32, 4, 32, 2, PRED>(P, sp, st, dependent);
 }
 
@@ -335,7 +339,7 @@ int64_t keep_rows_for(const lr_ctx* ctx, int variant, int32_t n, bool bf16 = fal
 // for the stages filled during its iteration boundary to matter: fp32 matrices from about half the L2 upwards.
 constexpr int64_t kPersistentMinBytes = int64_t(64) << 20;
 bool want_persistent(const lr_ctx* ctx, const lr_plan& P, bool bf16, int64_t m, int32_t n, int64_t iters) {
-    if (P.variant != 0 || !ctx->coop || ctx->prof || ctx->persistent_mode == 0) return false;
+    if (P.variant != 0 || P.threads != kNW * 32 || !ctx->coop || ctx->prof || ctx->persistent_mode == 0) return false;
     if (2 * iters * P.grid >= (int64_t(1) << 32)) return false;       // the grid-barrier counter is 32 bits
     if (ctx->persistent_mode > 0) return true;
     return !bf16 && m * n * 4 >= kPersistentMinBytes;

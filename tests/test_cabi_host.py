@@ -91,7 +91,18 @@ def test_plan_rows_of_any_length(n, lpr, nv, rb):
     assert 1024 + 16 * p["stages"] * stage <= p["smem_bytes"]
 
 
-@pytest.mark.parametrize("m,n,nv,rb", [(100_000, 4096, 2, 4), (5000, 1024, 1, 8), (5000, 516, 1, 8), (5000, 2052, 2, 4)])
+def test_plan_rows_of_516_to_1024_columns_use_eight_warps():
+    for m, n in [(5000, 516), (5000, 1024), (200_000, 1000)]:
+        p = api.plan_query(m, n)
+        assert p["variant"] == 0 and p["threads"] == 256 and p["vec_per_lane"] == 8 and p["rows_per_batch"] == 2
+        stage = -(-2 * n * 4 // 128) * 128
+        assert 1024 + 8 * p["stages"] * stage <= p["smem_bytes"] <= 227 * 1024
+        assert p["smem_bytes"] >= 1024 + 8 * n * 8 + 2 * 8 * 8         # room for the end-of-kernel combine of eight warps
+        assert p["grid"] == min(-(-(-(-m // 2)) // 8), 148)
+    assert api.plan_query(5000, 1024, bf16=True)["variant"] == 1     # bfloat16 rows of more than 64 groups stay on the split kernel
+
+
+@pytest.mark.parametrize("m,n,nv,rb", [(100_000, 4096, 2, 4), (5000, 1028, 1, 8), (5000, 1540, 1, 8), (5000, 2052, 2, 4)])
 def test_plan_wide_rows_are_split_across_warps(m, n, nv, rb):
     p = api.plan_query(m, n)
     assert p["variant"] == 1 and p["vec_per_lane"] == nv and p["rows_per_batch"] == rb
