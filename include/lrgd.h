@@ -198,7 +198,8 @@ int lr_predict(lr_ctx* ctx, const float* d_X, int64_t m, int32_t n,
  * with leading dimension n, 2-byte aligned.  Only X changes: y, w, b, the gradient and every sum stay as in the fp32
  * calls, each element of X is widened exactly to fp32 when it is used, so the three calls below compute exactly what
  * lr_loss_grad / lr_fit / lr_predict would compute on the fp32 matrix holding the same (bfloat16-representable) values.
- * The staged kernels take rows of n % 8 == 0 columns with d_Xh 16-byte aligned, up to n = 8192; other shapes run on the
+ * Rows of up to 512 columns always take a staged kernel (fastest with n % 8 == 0 and d_Xh 16-byte aligned); so do rows of
+ * up to 8192 columns with n % 8 == 0 and d_Xh 16-byte aligned; other shapes run on the
  * unstaged kernel.  lr_fit_bf16 runs as two dependent-launched kernels per iteration unless lr_set_persistent(ctx, 1) asks for
  * the persistent kernel (n <= 512).  Errors as the fp32 calls.
  *

@@ -54,8 +54,8 @@ bool row_shape_for(int ng, bool bf16, RowShape* s) {
     return true;
 }
 
-// Narrow fp32 rows whose length is not a multiple of four, or whose matrix is not 16-byte aligned: a lane owns single
-// elements (nv of them per row).
+// Narrow rows whose length is not a whole number of 16-byte groups, or whose matrix is not 16-byte aligned: a lane owns
+// single elements (nv of them per row).
 bool any_row_shape_for(int n, RowShape* s) {
     if (n <= 8) *s = {1, 8, 8};
     else if (n <= 16) *s = {1, 16, 8};
@@ -76,8 +76,9 @@ int make_plan(int64_t m, int32_t n, bool aligned16, int32_t sms, lr_plan* P, boo
     const int epg = bf16 ? 8 : 4, eb = bf16 ? 2 : 4;
     RowShape rs;
     const bool grouped = aligned16 && n % epg == 0 && row_shape_for(n / epg, bf16, &rs);
-    // fp32 rows that cannot be cut into aligned 16-byte groups (length not a multiple of four, or X only 4-byte aligned)
-    const bool any_len = !grouped && !bf16 && any_row_shape_for(n, &rs);
+    // rows of up to 512 columns that cannot be cut into aligned 16-byte groups (length not a whole number of groups, or X
+    // aligned to its element size only)
+    const bool any_len = !grouped && any_row_shape_for(n, &rs);
     if (grouped || any_len) {
         const int rpb = rs.rb * (32 / rs.lpr);                                  // rows per batch = rows per stage
         const int64_t B = (m + rpb - 1) / rpb;                                  // batches
@@ -224,7 +225,16 @@ cudaError_t launch_rows_t(const lr_plan& P, const StreamParams& sp, cudaStream_t
 
 template <bool PRED>
 cudaError_t launch_rows(const lr_plan& P, const StreamParams& sp, cudaStream_t st, bool bf16 = false, bool dependent = false) {
-    if (P.variant == 3) {                          // fp32 rows of any length: (lanes per row, elements per lane) picks the instantiation
+    if (P.variant == 3 && bf16) {                  // rows of any length: (lanes per row, elements per lane) picks the instantiation
+        if (P.lanes_per_row == 8) return launch_rows_t<ElemBF16Any, 1, 8, 8, PRED>(P, sp, st, dependent);
+        if (P.lanes_per_row == 16) return launch_rows_t<ElemBF16Any, 1, 16, 8, PRED>(P, sp, st, dependent);
+        if (P.vec_per_lane == 1) return launch_rows_t<ElemBF16Any, 1, 32, 16, PRED>(P, sp, st, dependent);
+        if (P.vec_per_lane == 2) return launch_rows_t<ElemBF16Any, 2, 32, 16, PRED>(P, sp, st, dependent);
+        if (P.vec_per_lane == 4) return launch_rows_t<ElemBF16Any, 4, 32, 8, PRED>(P, sp, st, dependent);
+        if (P.vec_per_lane == 8) return launch_rows_t<ElemBF16Any, 8, 32, 4, PRED>(P, sp, st, dependent);
+        return launch_rows_t<ElemBF16Any, 16, 32, 2, PRED>(P, sp, st, dependent);
+    }
+    if (P.variant == 3) {
         if (P.lanes_per_row == 8) return launch_rows_t<ElemF32Any, 1, 8, 8, PRED>(P, sp, st, dependent);
         if (P.lanes_per_row == 16) return launch_rows_t<ElemF32Any, 1, 16, 8, PRED>(P, sp, st, dependent);
         if (P.vec_per_lane == 1) return launch_rows_t<ElemF32Any, 1, 32, 16, PRED>(P, sp, st, dependent);

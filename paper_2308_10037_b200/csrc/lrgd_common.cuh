@@ -334,10 +334,14 @@ struct LaneBF16 {
     }
 };
 
-// Rows of any length (fp32): the unit a lane owns is a single element, so a row needs no particular length.  Loads are
-// 32-bit (consecutive lanes read consecutive words: conflict-free), arithmetic is scalar FMAs in ownership order.
-template <int NV>
-struct LaneF32Any {
+// Rows of any length: the unit a lane owns is a single element, so a row needs no particular length.  Loads are one
+// element wide (consecutive lanes read consecutive elements: conflict-free), arithmetic is scalar FMAs in ownership
+// order.  Raw is the element as stored: a 32-bit word holding an fp32 value, or a 16-bit bfloat16 pattern.
+__device__ __forceinline__ float widen_element(uint32_t v) { return __uint_as_float(v); }
+__device__ __forceinline__ float widen_element(unsigned short v) { return __uint_as_float(static_cast<uint32_t>(v) << 16); }
+
+template <class Raw, int NV>
+struct LaneAny {
     static constexpr int EPG = 1;
     float wv[NV];
     float acc[NV];
@@ -352,18 +356,18 @@ struct LaneF32Any {
 #pragma unroll
         for (int k = 0; k < NV; ++k) acc[k] = 0.f;
     }
-    __device__ __forceinline__ float dot(const uint32_t (&xr)[NV]) const {
+    __device__ __forceinline__ float dot(const Raw (&xr)[NV]) const {
         float d0 = 0.f, d1 = 0.f;                  // two chains: NV goes up to 16
 #pragma unroll
         for (int k = 0; k < NV; ++k) {
-            if (k & 1) d1 = fmaf(__uint_as_float(xr[k]), wv[k], d1);
-            else d0 = fmaf(__uint_as_float(xr[k]), wv[k], d0);
+            if (k & 1) d1 = fmaf(widen_element(xr[k]), wv[k], d1);
+            else d0 = fmaf(widen_element(xr[k]), wv[k], d0);
         }
         return d0 + d1;
     }
-    __device__ __forceinline__ void accumulate(const uint32_t (&xr)[NV], float er) {
+    __device__ __forceinline__ void accumulate(const Raw (&xr)[NV], float er) {
 #pragma unroll
-        for (int k = 0; k < NV; ++k) acc[k] = fmaf(__uint_as_float(xr[k]), er, acc[k]);
+        for (int k = 0; k < NV; ++k) acc[k] = fmaf(widen_element(xr[k]), er, acc[k]);
     }
     __device__ __forceinline__ void fold(double (&dacc)[NV][1]) {
 #pragma unroll
@@ -397,15 +401,26 @@ struct ElemBF16 {
     }
 };
 
-// fp32 rows whose length is not a multiple of four: the "group" degenerates to one element (see LaneF32Any).
+// Rows that cannot be cut into aligned 16-byte groups (any length, matrix aligned to its element size only): the
+// "group" degenerates to one element (see LaneAny).
 struct ElemF32Any {
     static constexpr int EPG = 1;
     static constexpr int BYTES = 4;
     using Raw = uint32_t;
     template <int NV>
-    using Lane = LaneF32Any<NV>;
+    using Lane = LaneAny<uint32_t, NV>;
     static __device__ __forceinline__ float load(const void* base, long long i) {
         return reinterpret_cast<const float*>(base)[i];
+    }
+};
+struct ElemBF16Any {
+    static constexpr int EPG = 1;
+    static constexpr int BYTES = 2;
+    using Raw = unsigned short;
+    template <int NV>
+    using Lane = LaneAny<unsigned short, NV>;
+    static __device__ __forceinline__ float load(const void* base, long long i) {
+        return __uint_as_float(static_cast<uint32_t>(reinterpret_cast<const unsigned short*>(base)[i]) << 16);
     }
 };
 

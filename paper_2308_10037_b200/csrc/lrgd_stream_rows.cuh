@@ -177,13 +177,12 @@ __global__ void __launch_bounds__(NW * 32, 1) k_stream_rows(const StreamParams p
         unsigned char* dst = my_stages + static_cast<size_t>(d) * stage_stride;
         const unsigned char* src = static_cast<const unsigned char*>(p.X) + static_cast<size_t>(r0) * row_bytes;
         if constexpr (E::EPG == 1) {
-            static_assert(E::EPG != 1 || E::BYTES == 4, "the tail is moved in 32-bit words");
-            // rows of any length, X 4-byte aligned: neither the start nor the size of a batch need be a multiple of 16
+            // rows of any length, X aligned to its element size: neither the start nor the size of a batch need be a multiple of 16
             // bytes.  The batch lands at dst + off, off = its address mod 16.  The bulk copy covers the 16-byte-aligned span
             // that starts at or up to 12 bytes before the batch (bytes of the row before it) and ends at or before its last
             // byte; for the very first batch of a matrix that is itself not 16-byte aligned it starts at the first boundary
-            // inside the batch instead.  The few words left over at either end are moved by this lane with plain loads and
-            // stores.  Nothing outside [X, X + m*n) is read.
+            // inside the batch instead.  The few elements left over at either end are moved by this lane with plain loads
+            // and stores.  Nothing outside [X, X + m*n) is read.
             const uint32_t off = static_cast<uint32_t>(reinterpret_cast<uintptr_t>(src)) & 15u;
             const uint32_t span = off + xbytes;                                   // stage bytes [off, span) hold the batch
             const uint32_t lo = (r0 == 0 && off != 0u) ? 16u : 0u;                // first stage byte the bulk copy writes
@@ -194,10 +193,11 @@ __global__ void __launch_bounds__(NW * 32, 1) k_stream_rows(const StreamParams p
             } else {
                 mbar_arrive(&my_bars[d]);
             }
-            for (uint32_t o = off; o < lo && o < span; o += 4u)                   // head (first batch of an unaligned matrix only)
-                *reinterpret_cast<uint32_t*>(dst + o) = *reinterpret_cast<const uint32_t*>(src - off + o);
-            for (uint32_t o = lo + bulk; o < span; o += 4u)                       // tail
-                *reinterpret_cast<uint32_t*>(dst + o) = *reinterpret_cast<const uint32_t*>(src - off + o);
+            using Raw = typename E::Raw;                                          // one element
+            for (uint32_t o = off; o < lo && o < span; o += E::BYTES)             // head (first batch of an unaligned matrix only)
+                *reinterpret_cast<Raw*>(dst + o) = *reinterpret_cast<const Raw*>(src - off + o);
+            for (uint32_t o = lo + bulk; o < span; o += E::BYTES)                 // tail
+                *reinterpret_cast<Raw*>(dst + o) = *reinterpret_cast<const Raw*>(src - off + o);
         } else {
             mbar_arrive_expect_tx(&my_bars[d], xbytes);
             bulk_copy_g2s(dst, src, xbytes, &my_bars[d], r0 < p.keep_rows ? pol_keep : pol_stream);

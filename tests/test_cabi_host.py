@@ -72,9 +72,10 @@ def test_plan_falls_back_for_unaligned_or_odd_shapes():
     assert api.plan_query(1000, 516, x_aligned16=False)["variant"] == 2    # wide rows need a 16-byte aligned matrix
     assert api.plan_query(1000, 32, x_aligned16=False)["variant"] == 3     # narrow rows do not: element-wise staged kernel
     assert api.plan_query(1000, 30, x_aligned16=False)["variant"] == 3
-    assert api.plan_query(1000, 32, x_aligned16=False, bf16=True)["variant"] == 2
+    assert api.plan_query(1000, 32, x_aligned16=False, bf16=True)["variant"] == 3
     assert api.plan_query(1000, 8192)["variant"] == 2         # wider than any staged kernel
-    assert api.plan_query(1000, 30, bf16=True)["variant"] == 2   # bfloat16 rows must be whole 16-byte groups
+    assert api.plan_query(1000, 30, bf16=True)["variant"] == 3   # element-wise staged kernel, bfloat16 too
+    assert api.plan_query(1000, 516, bf16=True)["variant"] == 2  # 516 % 8 != 0 and wider than 512
     g = api.plan_query(100, 515)
     assert g["grid"] == 2 and g["threads"] == 256
 
@@ -159,13 +160,16 @@ def test_any_length_copies_stay_inside_the_matrix():
     shapes = [(2758, 449), (1, 1), (7, 3), (300, 1), (640, 30), (1025, 101), (526, 255), (999, 511), (5, 510), (3, 258),
               (17, 257), (2, 449), (1, 511)]
     shapes += [(rnd.randint(1, 3000), rnd.choice([n for n in range(1, 513) if n % 4])) for _ in range(200)]
-    cases = [(m, n, 0) for m, n in shapes]
-    cases += [(m, n, base) for (m, n) in shapes[:60] + [(1, 1), (2, 2), (3, 1), (40, 32), (999, 256), (77, 512)] for base in (4, 8, 12)]
-    for m, n, base in cases:
-        p = api.plan_query(m, n, x_aligned16=(base == 0))
+    cases = [(m, n, 0, 4) for m, n in shapes]
+    extra = shapes[:60] + [(1, 1), (2, 2), (3, 1), (40, 32), (999, 256), (77, 512)]
+    cases += [(m, n, base, 4) for (m, n) in extra for base in (4, 8, 12)]
+    # bfloat16 (2-byte elements): lengths that are not a multiple of eight, and bases on every even offset
+    cases += [(m, n, 0, 2) for (m, n) in shapes[:80] if n % 8] + [(m, n, base, 2) for (m, n) in extra[:40] for base in (2, 6, 10, 14)]
+    for m, n, base, eb in cases:
+        p = api.plan_query(m, n, x_aligned16=(base == 0), bf16=(eb == 2))
         assert p["variant"] == 3
-        rpb, row_bytes = p["rows_per_batch"], 4 * n
-        lo_x, hi_x = 4096 + base, 4096 + base + 4 * m * n          # the matrix occupies the addresses [lo_x, hi_x)
+        rpb, row_bytes = p["rows_per_batch"], eb * n
+        lo_x, hi_x = 4096 + base, 4096 + base + eb * m * n         # the matrix occupies the addresses [lo_x, hi_x)
         stage = -(-(rpb * row_bytes + 16) // 128) * 128
         assert 1024 + 16 * p["stages"] * stage <= p["smem_bytes"]
         seen = 0
@@ -180,12 +184,12 @@ def test_any_length_copies_stay_inside_the_matrix():
             assert span <= stage
             if bulk:
                 assert (src - off + lo) % 16 == 0 and lo_x <= src - off + lo and src - off + lo + bulk <= hi_x
-            head = list(range(off, min(lo, span), 4))
-            tail = list(range(lo + bulk, span, 4))
-            assert len(head) <= 3 and len(tail) <= 3
-            assert all(lo_x <= src - off + o and src - off + o + 4 <= hi_x for o in head + tail)
+            head = list(range(off, min(lo, span), eb))
+            tail = list(range(lo + bulk, span, eb))
+            assert len(head) <= 16 // eb - 1 and len(tail) <= 16 // eb - 1
+            assert all(lo_x <= src - off + o and src - off + o + eb <= hi_x for o in head + tail)
             # every byte of the batch is written exactly once: head, bulk and tail tile [off, span) of the stage
-            written = sorted(head + tail + list(range(lo, lo + bulk, 4)))
-            assert [o for o in written if o >= off] == list(range(off, span, 4))
+            written = sorted(head + tail + list(range(lo, lo + bulk, eb)))
+            assert [o for o in written if o >= off] == list(range(off, span, eb))
             seen += xbytes
-        assert seen == 4 * m * n
+        assert seen == eb * m * n

@@ -90,14 +90,41 @@ def test_library_conversion_feeds_the_pass(ctx):
     check_loss_grad(ctx, Xv, ctx.convert_bf16(dev(X)), y, w, b)
 
 
-def test_unaligned_bf16_view_uses_the_unstaged_kernel(ctx):
-    X, y, w, b = datagen.random_problem(1201, 64, seed=12)
+@pytest.mark.parametrize("m,n,shift", [(1201, 64, 1), (90_001, 30, 3), (40_001, 449, 5), (7, 3, 7), (2_001, 520, 1)])
+def test_bf16_views_that_are_only_2_byte_aligned(ctx, m, n, shift):
+    # narrow rows stay on a staged kernel (element-wise; the first batch is completed with plain loads instead of reading
+    # in front of the matrix, which is surrounded by NaN here); wide rows run unstaged
+    X, y, w, b = datagen.random_problem(m, n, seed=13 + m + n)
     bits, Xv = oracle.round_bf16(X)
-    buf = torch.zeros(bits.size + 1, dtype=torch.bfloat16, device="cuda")
-    buf[1:] = dev_bf16(bits).ravel()
-    Xh = buf[1:].view(1201, 64)
-    assert Xh.data_ptr() % 16 == 2
+    buf = torch.full((bits.size + 16,), float("nan"), dtype=torch.bfloat16, device="cuda")
+    buf[shift:shift + bits.size] = dev_bf16(bits).ravel()
+    Xh = buf[shift:shift + bits.size].view(m, n)
+    assert Xh.data_ptr() % 16 == 2 * shift
+    assert api.plan_query(m, n, x_aligned16=False, bf16=True)["variant"] == (3 if n <= 512 else 2)
     check_loss_grad(ctx, Xv, Xh, y, w, b)
+
+
+# bfloat16 rows whose length is not a multiple of eight: every element-wise instantiation, batches that start off a
+# 16-byte boundary, ragged tails, stage reuse; pass, labels and a short fit
+@pytest.mark.parametrize("m,n", [(33, 7), (1, 3), (40_003, 13), (150_001, 30), (100_001, 100), (200_003, 255), (2_758, 449),
+                                 (60_001, 449), (50_002, 508), (5, 510), (17, 257)])
+def test_bf16_rows_of_any_length(ctx, m, n):
+    assert api.plan_query(m, n, bf16=True)["variant"] == 3
+    X, y, w, b = datagen.random_problem(m, n, seed=3500 + m + n, wscale=1.5)
+    bits, Xv = oracle.round_bf16(X)
+    dXh = dev_bf16(bits)
+    check_loss_grad(ctx, Xv, dXh, y, w, b)
+    dw, db = dev(w), dev(np.array([b], dtype=np.float32))
+    ref, z = oracle.predict(Xv, w, b, 0.4, return_z=True)
+    got = ctx.predict(dXh, dw, db, 0.4).cpu().numpy()
+    clear = np.abs(z - np.log(0.4 / 0.6)) > 1e-4 * (1 + np.abs(z))
+    assert np.array_equal(got[clear], ref[clear])
+    iters, lr = 6, 0.1
+    w_ref, b_ref, lh_ref = oracle.fit(Xv, y, lr, iters, w0=w, b0=b)
+    hist = torch.empty(iters, device="cuda")
+    ctx.fit(dXh, dev(y), lr, iters, dw, db, hist)
+    assert rel_l2(np.concatenate([dw.cpu().numpy(), db.cpu().numpy()]), np.concatenate([w_ref, [b_ref]])) <= W_TOL
+    assert np.max(np.abs(hist.cpu().numpy() - lh_ref)) <= LOSS_TOL
 
 
 SMALL_WORKLOADS = [("cfg1", 10_000), ("cfg3", 30_011), ("cfg4", 3_000), ("cfg5", 100_003)]
