@@ -39,16 +39,17 @@ constexpr int64_t kMaxRows = int64_t(1) << 40;
 
 struct RowShape { int nv, lpr, rb; int nw = kNW; };    // nw = warps per CTA
 
-// Which instantiation of the narrow-row kernel covers ng 16-byte column groups per row.  bfloat16 rows stop at 64
-// groups: a lane that owns four groups of eight columns would need more registers than a 512-thread CTA can give.
-// fp32 rows of 129..256 groups (516..1024 columns) run with eight warps per CTA, so that a thread may hold the eight
-// groups of its row slice, their weights and accumulators (up to 255 registers); the bytes in flight per SM stay the same.
+// Which instantiation of the narrow-row kernel covers ng 16-byte column groups per row.  The widest shapes -- fp32
+// rows of 129..256 groups (516..1024 columns), bfloat16 rows of 65..128 groups (520..1024 columns) -- run with eight
+// warps per CTA, so that a thread may hold its 32 columns of a row slice, their weights and accumulators (up to 255
+// registers; a 512-thread CTA gives 128); the bytes in flight per SM stay the same.
 bool row_shape_for(int ng, bool bf16, RowShape* s) {
     if (ng <= 8) *s = {1, 8, 8};
     else if (ng <= 16) *s = {1, 16, 8};
     else if (ng <= 32) *s = {1, 32, LRGD_NV1_RB};
     else if (ng <= 64) *s = {2, 32, LRGD_NV2_RB};
     else if (ng <= 128 && !bf16) *s = {4, 32, 2};
+    else if (ng <= 128 && bf16) *s = {4, 32, 2, 8};         // 520..1024 bfloat16 columns: eight warps, as below
     else if (ng <= 256 && !bf16) *s = {8, 32, 2, 8};
     else return false;
     return true;
@@ -248,7 +249,8 @@ cudaError_t launch_rows(const lr_plan& P, const StreamParams& sp, cudaStream_t s
         if (P.lanes_per_row == 16) return launch_rows_t<ElemBF16, 1, 16, 8, PRED>(P, sp, st, dependent);
         if (P.vec_per_lane == 1) return launch_rows_t<ElemBF16, 1, 32, LRGD_NV1_RB, PRED>(P, sp, st, dependent);
         if (P.vec_per_lane == 2) return launch_rows_t<ElemBF16, 2, 32, LRGD_NV2_RB, PRED>(P, sp, st, dependent);
-        return cudaErrorInvalidValue;              // the plan never asks for four bfloat16 groups per lane
+        if (P.vec_per_lane == 4) return launch_rows_t<ElemBF16, 4, 32, 2, PRED, 8>(P, sp, st, dependent);     // eight warps per CTA
+        return cudaErrorInvalidValue;
     }
     if (P.lanes_per_row == 8) return launch_rows_t<ElemF32, 1, 8, 8, PRED>(P, sp, st, dependent);
     if (P.lanes_per_row == 16) return launch_rows_t<ElemF32, 1, 16, 8, PRED>(P, sp, st, dependent);

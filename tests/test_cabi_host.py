@@ -100,7 +100,9 @@ def test_plan_rows_of_516_to_1024_columns_use_eight_warps():
         assert 1024 + 8 * p["stages"] * stage <= p["smem_bytes"] <= 227 * 1024
         assert p["smem_bytes"] >= 1024 + 8 * n * 8 + 2 * 8 * 8         # room for the end-of-kernel combine of eight warps
         assert p["grid"] == min(-(-(-(-m // 2)) // 8), 148)
-    assert api.plan_query(5000, 1024, bf16=True)["variant"] == 1     # bfloat16 rows of more than 64 groups stay on the split kernel
+    pb = api.plan_query(5000, 1024, bf16=True)                        # bfloat16: 65..128 groups per row, eight warps too
+    assert pb["variant"] == 0 and pb["threads"] == 256 and pb["vec_per_lane"] == 4 and pb["rows_per_batch"] == 2
+    assert api.plan_query(5000, 1032, bf16=True)["variant"] == 1     # wider bfloat16 rows stay on the split kernel
 
 
 @pytest.mark.parametrize("m,n,nv,rb", [(100_000, 4096, 2, 4), (5000, 1028, 1, 8), (5000, 1540, 1, 8), (5000, 2052, 2, 4)])
