@@ -107,7 +107,12 @@ int make_plan(int64_t m, int32_t n, bool aligned16, int32_t sms, lr_plan* P, boo
         // wide rows: the warps of a CTA split each row by columns
         const int cw = (n / epg + kNW - 1) / kNW;                               // 16-byte column groups per warp slice
         const int nv = cw > 32 ? 2 : 1;
-        const int rb = nv == 2 ? 4 : 8;
+        // Rows per batch.  All warps of a CTA meet once per batch, so a batch must carry enough bytes to cover that
+        // round trip: slices of up to 24 groups per warp take 16 rows at a time and slices of 33..48 groups 8 rows, where 8
+        // and 4 left the pass latency-bound (1028 columns: 3.6 TB/s, 2052: 4.2 TB/s); wider slices would leave room for
+        // one stage only.
+        const int rb = nv == 2 ? (cw <= 48 && !bf16 ? 8 : 4)             // (the bfloat16 kernels would spill registers with the
+                               : (cw <= 24 && !bf16 ? 16 : 8);          //  larger batches)
         const int64_t B = (m + rb - 1) / rb;
         const int grid = int(std::min<int64_t>(B, sms));
         const int64_t per_cta = (B + grid - 1) / grid;
@@ -308,7 +313,9 @@ cudaError_t launch_split(const lr_plan& P, const void* X, const SplitParams& sp,
         if (P.vec_per_lane == 2) return launch_split_t<ElemBF16, 2, 4, PRED>(P, tm, sp, st, dependent);
         return launch_split_t<ElemBF16, 1, 8, PRED>(P, tm, sp, st, dependent);
     }
+    if (P.vec_per_lane == 2 && P.rows_per_batch == 8) return launch_split_t<ElemF32, 2, 8, PRED>(P, tm, sp, st, dependent);
     if (P.vec_per_lane == 2) return launch_split_t<ElemF32, 2, 4, PRED>(P, tm, sp, st, dependent);
+    if (P.rows_per_batch == 16) return launch_split_t<ElemF32, 1, 16, PRED>(P, tm, sp, st, dependent);
     return launch_split_t<ElemF32, 1, 8, PRED>(P, tm, sp, st, dependent);
 }
 

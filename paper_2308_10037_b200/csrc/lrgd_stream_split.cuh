@@ -26,7 +26,7 @@
 
 namespace lrgd {
 
-constexpr int kSplitHeaderBytes = 2048;   // mbarriers [NW][kMaxDepth], abort flag, partial logits [2][NW][RB]
+constexpr int kSplitHeaderBytes = 4096;   // mbarriers [NW][kMaxDepth], abort flag, partial logits [2][NW][RB] (RB up to 16)
 constexpr int kSplitZOffset = 1024;
 
 struct SplitParams {

@@ -105,14 +105,14 @@ def test_plan_rows_of_516_to_1024_columns_use_eight_warps():
     assert api.plan_query(5000, 1032, bf16=True)["variant"] == 1     # wider bfloat16 rows stay on the split kernel
 
 
-@pytest.mark.parametrize("m,n,nv,rb", [(100_000, 4096, 2, 4), (5000, 1028, 1, 8), (5000, 1540, 1, 8), (5000, 2052, 2, 4)])
+@pytest.mark.parametrize("m,n,nv,rb", [(100_000, 4096, 2, 4), (5000, 1028, 1, 16), (5000, 1540, 1, 8), (5000, 2052, 2, 8), (5000, 3200, 2, 4)])
 def test_plan_wide_rows_are_split_across_warps(m, n, nv, rb):
     p = api.plan_query(m, n)
     assert p["variant"] == 1 and p["vec_per_lane"] == nv and p["rows_per_batch"] == rb
     assert p["threads"] == 512 and p["grid"] == min(-(-m // rb), 148)
     cw = -(-(n // 4) // 16)
     stage = -(-rb * cw * 16 // 128) * 128
-    assert 1 <= p["stages"] <= 4 and p["smem_bytes"] == 2048 + 16 * p["stages"] * stage <= 227 * 1024
+    assert 1 <= p["stages"] <= 4 and p["smem_bytes"] == 4096 + 16 * p["stages"] * stage <= 227 * 1024
 
 
 def test_plan_rejects_bad_shapes():
