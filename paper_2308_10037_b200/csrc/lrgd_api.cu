@@ -103,15 +103,15 @@ int make_plan(int64_t m, int32_t n, bool aligned16, int32_t sms, lr_plan* P, boo
         if (per_warp >= (int64_t(1) << 31)) return LR_ERR_SHAPE;
         return LR_OK;
     }
-    if (aligned16 && n % epg == 0 && n / epg <= kNW * 64 && m < (int64_t(1) << 31) - 65536) {   // TMA coordinates are int32
+    if (aligned16 && n % epg == 0 && n / epg <= kNW * (bf16 ? 64 : 128) && m < (int64_t(1) << 31) - 65536) {   // TMA coordinates are int32
         // wide rows: the warps of a CTA split each row by columns
         const int cw = (n / epg + kNW - 1) / kNW;                               // 16-byte column groups per warp slice
-        const int nv = cw > 32 ? 2 : 1;
+        const int nv = cw > 64 ? 4 : (cw > 32 ? 2 : 1);            // fp32 rows of 4100..8192 columns: four groups per lane, two rows
         // Rows per batch.  All warps of a CTA meet once per batch, so a batch must carry enough bytes to cover that
         // round trip: slices of up to 24 groups per warp take 16 rows at a time and slices of 33..48 groups 8 rows, where 8
         // and 4 left the pass latency-bound (1028 columns: 3.6 TB/s, 2052: 4.2 TB/s); wider slices would leave room for
         // one stage only.
-        const int rb = nv == 2 ? (cw <= 48 && !bf16 ? 8 : 4)             // (the bfloat16 kernels would spill registers with the
+        const int rb = nv == 4 ? 2 : nv == 2 ? (cw <= 48 && !bf16 ? 8 : 4)             // (the bfloat16 kernels would spill registers with the
                                : (cw <= 24 && !bf16 ? 16 : 8);          //  larger batches)
         const int64_t B = (m + rb - 1) / rb;
         const int grid = int(std::min<int64_t>(B, sms));
@@ -269,6 +269,8 @@ cudaError_t launch_rows(const lr_plan& P, const StreamParams& sp, cudaStream_t s
 // The copy moves bytes untouched, and a box may span at most 256 elements per dimension, so a bfloat16 matrix is
 // described as 32-bit words (n/2 per row): the widest slice, 64 groups, is then 256 elements for either storage type.
 // The encoder is a driver entry point, resolved at run time so that the library links against the runtime only.
+bool split_words64(bool bf16, int cw) { return !bf16 && cw > 64; }
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
                                   const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -283,12 +285,15 @@ cudaError_t make_x_tensor_map(const void* X, bool bf16, int64_t m, int32_t n, in
         if (q != cudaDriverEntryPointSuccess || !fn) return cudaErrorNotSupported;
         encode = reinterpret_cast<EncodeTiledFn>(fn);
     }
-    const cuuint64_t words = bf16 ? cuuint64_t(n) / 2 : cuuint64_t(n);            // 32-bit words per row
-    const cuuint64_t dims[2] = {words, cuuint64_t(m)};
-    const cuuint64_t strides[1] = {words * 4};
-    const cuuint32_t box[2] = {cuuint32_t(cw) * 4, cuuint32_t(rb)};
+    // (fp32 slices of more than 64 groups -- rows of more than 4096 columns -- are described as 64-bit words for the same reason)
+    const bool wide64 = split_words64(bf16, cw);
+    const cuuint64_t row_bytes = cuuint64_t(n) * (bf16 ? 2 : 4);
+    const cuuint32_t wbytes = wide64 ? 8 : 4;
+    const cuuint64_t dims[2] = {row_bytes / wbytes, cuuint64_t(m)};
+    const cuuint64_t strides[1] = {row_bytes};
+    const cuuint32_t box[2] = {cuuint32_t(cw) * (16 / wbytes), cuuint32_t(rb)};
     const cuuint32_t estr[2] = {1, 1};
-    CUresult r = encode(out, bf16 ? CU_TENSOR_MAP_DATA_TYPE_UINT32 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2,
+    CUresult r = encode(out, wide64 ? CU_TENSOR_MAP_DATA_TYPE_UINT64 : bf16 ? CU_TENSOR_MAP_DATA_TYPE_UINT32 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2,
                         const_cast<void*>(X), dims, strides, box, estr,
                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
@@ -313,6 +318,7 @@ cudaError_t launch_split(const lr_plan& P, const void* X, const SplitParams& sp,
         if (P.vec_per_lane == 2) return launch_split_t<ElemBF16, 2, 4, PRED>(P, tm, sp, st, dependent);
         return launch_split_t<ElemBF16, 1, 8, PRED>(P, tm, sp, st, dependent);
     }
+    if (P.vec_per_lane == 4) return launch_split_t<ElemF32, 4, 2, PRED>(P, tm, sp, st, dependent);
     if (P.vec_per_lane == 2 && P.rows_per_batch == 8) return launch_split_t<ElemF32, 2, 8, PRED>(P, tm, sp, st, dependent);
     if (P.vec_per_lane == 2) return launch_split_t<ElemF32, 2, 4, PRED>(P, tm, sp, st, dependent);
     if (P.rows_per_batch == 16) return launch_split_t<ElemF32, 1, 16, PRED>(P, tm, sp, st, dependent);
@@ -404,6 +410,7 @@ int launch_stream_pass(lr_ctx* ctx, const lr_plan& P, const Pass& a, uint8_t* la
         sp.partial = ctx->d_partial; sp.labels = labels; sp.cut = cut; sp.status = ctx->d_status; sp.stop = a.stop;
         sp.depth = P.stages;
         sp.cw = (a.n / (a.bf16 ? 8 : 4) + kNW - 1) / kNW;
+        sp.x_per_group = split_words64(a.bf16, sp.cw) ? 2 : 4;
         sp.num_batches = (a.m + P.rows_per_batch - 1) / P.rows_per_batch;
         sp.keep_rows = keep_rows_for(ctx, 1, a.n, a.bf16);
         e = predict ? launch_split<true>(P, a.X, sp, st, a.bf16, dep) : launch_split<false>(P, a.X, sp, st, a.bf16, dep);
@@ -1161,6 +1168,7 @@ extern "C" int lr_loss_grad_noalloc(int32_t device, const float* d_X, const floa
         sp.partial = partial; sp.labels = nullptr; sp.cut = 0.f; sp.status = status;
         sp.depth = P.stages;
         sp.cw = (n / 4 + kNW - 1) / kNW;
+        sp.x_per_group = split_words64(false, sp.cw) ? 2 : 4;
         sp.num_batches = (m + P.rows_per_batch - 1) / P.rows_per_batch;
         e = launch_split<false>(P, d_X, sp, st);
     } else {

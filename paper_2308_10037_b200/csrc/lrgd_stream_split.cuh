@@ -42,6 +42,7 @@ struct SplitParams {
     const int* stop;          // nullable: non-zero makes the launch a no-op
     int depth;                // stages per warp
     int cw;                   // 16-byte column groups per warp slice (the tensor map's box is cw groups by RB rows)
+    int x_per_group;          // tensor-map elements per 16-byte group: 4 (32-bit words) or 2 (64-bit words)
     long long num_batches;    // ceil(m / RB)
     long long keep_rows;      // rows [0, keep_rows) are fetched with an L2 evict-last hint, the rest evict-first
 };
@@ -89,7 +90,7 @@ __global__ void __launch_bounds__(NW * 32, 1) k_stream_split(const __grid_consta
     int row0 = static_cast<int>(blockIdx.x) * RB;                             // first row of the current batch
     auto issue = [&](int r0, int d) {              // lane 0 of a warp with mycw > 0
         mbar_arrive_expect_tx(&my_bars[d], box_bytes);
-        bulk_tensor_2d_g2s(my_stages + static_cast<size_t>(d) * stage_stride, &tmap, c0 * 4, r0, &my_bars[d],   // x in 32-bit words
+        bulk_tensor_2d_g2s(my_stages + static_cast<size_t>(d) * stage_stride, &tmap, c0 * p.x_per_group, r0, &my_bars[d],
                            r0 < p.keep_rows ? pol_keep : pol_stream);
     };
 
@@ -106,7 +107,7 @@ __global__ void __launch_bounds__(NW * 32, 1) k_stream_split(const __grid_consta
     const int dup = lane & (DUP - 1);              // which of the lanes sharing that row this one is
     const bool owner = dup == 0;
     const bool full_cw = CW == 32 * NV;            // every lane's column groups lie inside the box
-    const bool labels_word_aligned = PREDICT && (reinterpret_cast<uintptr_t>(p.labels) & 3u) == 0;
+    const bool labels_word_aligned = PREDICT && RB % 4 == 0 && (reinterpret_cast<uintptr_t>(p.labels) & 3u) == 0;
 
     const bool active = mycw > 0;
     if (active && lane == 0) {

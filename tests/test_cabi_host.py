@@ -73,7 +73,8 @@ def test_plan_falls_back_for_unaligned_or_odd_shapes():
     assert api.plan_query(1000, 32, x_aligned16=False)["variant"] == 3     # narrow rows do not: element-wise staged kernel
     assert api.plan_query(1000, 30, x_aligned16=False)["variant"] == 3
     assert api.plan_query(1000, 32, x_aligned16=False, bf16=True)["variant"] == 3
-    assert api.plan_query(1000, 8192)["variant"] == 2         # wider than any staged kernel
+    assert api.plan_query(1000, 8196)["variant"] == 2         # wider than any staged kernel
+    assert api.plan_query(1000, 8200, bf16=True)["variant"] == 2
     assert api.plan_query(1000, 30, bf16=True)["variant"] == 3   # element-wise staged kernel, bfloat16 too
     assert api.plan_query(1000, 516, bf16=True)["variant"] == 2  # 516 % 8 != 0 and wider than 512
     g = api.plan_query(100, 515)
@@ -105,7 +106,7 @@ def test_plan_rows_of_516_to_1024_columns_use_eight_warps():
     assert api.plan_query(5000, 1032, bf16=True)["variant"] == 1     # wider bfloat16 rows stay on the split kernel
 
 
-@pytest.mark.parametrize("m,n,nv,rb", [(100_000, 4096, 2, 4), (5000, 1028, 1, 16), (5000, 1540, 1, 8), (5000, 2052, 2, 8), (5000, 3200, 2, 4)])
+@pytest.mark.parametrize("m,n,nv,rb", [(100_000, 4096, 2, 4), (5000, 1028, 1, 16), (5000, 1540, 1, 8), (5000, 2052, 2, 8), (5000, 3200, 2, 4), (5000, 4100, 4, 2), (5000, 8192, 4, 2)])
 def test_plan_wide_rows_are_split_across_warps(m, n, nv, rb):
     p = api.plan_query(m, n)
     assert p["variant"] == 1 and p["vec_per_lane"] == nv and p["rows_per_batch"] == rb

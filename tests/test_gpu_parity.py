@@ -45,7 +45,7 @@ def check_loss_grad(ctx, X, y, w, b, grad_tol=GRAD_TOL, loss_tol=LOSS_TOL):
 # shapes: every staged instantiation (n/4 <= 8, 16, 32, 64, 128), partly filled lane groups (28, 100, 200, 36),
 # rows of any length (n % 4 != 0, n <= 512), the unstaged kernel (n % 4 != 0 and n > 512, n > 4096), and row counts that
 # are tiny, ragged, or span many tiles
-SHAPES = [(777, 515), (301, 1001), (1, 4), (7, 4), (8, 3), (33, 28), (1000, 32), (4097, 32), (5003, 64), (2500, 36), (3001, 100), (9999, 256),
+SHAPES = [(777, 515), (301, 1001), (3_001, 8192), (1_001, 5000), (777, 6148), (20, 8196), (1, 4), (7, 4), (8, 3), (33, 28), (1000, 32), (4097, 32), (5003, 64), (2500, 36), (3001, 100), (9999, 256),
           (777, 200), (1500, 512), (2049, 260), (640, 30), (1025, 101), (300, 1), (130, 4096), (50, 8192), (20011, 8),
           # enough rows that every warp refills its shared-memory stages many times, with a ragged last batch
           (200_003, 256), (400_001, 32), (200_002, 64), (120_007, 100), (150_001, 28), (60_001, 512), (90_001, 200),
