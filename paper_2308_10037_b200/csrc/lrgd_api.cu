@@ -47,7 +47,9 @@ bool row_shape_for(int ng, bool bf16, RowShape* s) {
     if (ng <= 8) *s = {1, 8, 8};
     else if (ng <= 16) *s = {1, 16, 8};
     else if (ng <= 32) *s = {1, 32, LRGD_NV1_RB};
-    else if (ng <= 64) *s = {2, 32, LRGD_NV2_RB};
+    else if (ng <= 64 && !bf16) *s = {2, 32, LRGD_NV2_RB};
+    else if (ng <= 64 && bf16) *s = {2, 32, 8, 8};          // 264..512 bfloat16 columns: eight warps, eight rows (no spills)
+    else if (ng <= 96 && !bf16) *s = {4, 32, 4, 8};         // 260..384 fp32 columns: eight warps, four rows (4..6 KB batches)
     else if (ng <= 128 && !bf16) *s = {4, 32, 2};
     else if (ng <= 128 && bf16) *s = {4, 32, 2, 8};         // 520..1024 bfloat16 columns: eight warps, as below
     else if (ng <= 256 && !bf16) *s = {8, 32, 2, 8};
@@ -253,6 +255,7 @@ cudaError_t launch_rows(const lr_plan& P, const StreamParams& sp, cudaStream_t s
         if (P.lanes_per_row == 8) return launch_rows_t<ElemBF16, 1, 8, 8, PRED>(P, sp, st, dependent);
         if (P.lanes_per_row == 16) return launch_rows_t<ElemBF16, 1, 16, 8, PRED>(P, sp, st, dependent);
         if (P.vec_per_lane == 1) return launch_rows_t<ElemBF16, 1, 32, LRGD_NV1_RB, PRED>(P, sp, st, dependent);
+        if (P.vec_per_lane == 2 && P.threads == 256) return launch_rows_t<ElemBF16, 2, 32, 8, PRED, 8>(P, sp, st, dependent);
         if (P.vec_per_lane == 2) return launch_rows_t<ElemBF16, 2, 32, LRGD_NV2_RB, PRED>(P, sp, st, dependent);
         if (P.vec_per_lane == 4) return launch_rows_t<ElemBF16, 4, 32, 2, PRED, 8>(P, sp, st, dependent);     // eight warps per CTA
         return cudaErrorInvalidValue;
@@ -262,6 +265,7 @@ cudaError_t launch_rows(const lr_plan& P, const StreamParams& sp, cudaStream_t s
     if (P.vec_per_lane == 1) return launch_rows_t<ElemF32, 1, 32, LRGD_NV1_RB, PRED>(P, sp, st, dependent);
     if (P.vec_per_lane == 2) return launch_rows_t<ElemF32, 2, 32, LRGD_NV2_RB, PRED>(P, sp, st, dependent);
     if (P.vec_per_lane == 8) return launch_rows_t<ElemF32, 8, 32, 2, PRED, 8>(P, sp, st, dependent);      // eight warps per CTA
+    if (P.vec_per_lane == 4 && P.threads == 256) return launch_rows_t<ElemF32, 4, 32, 4, PRED, 8>(P, sp, st, dependent);
     return launch_rows_t<ElemF32, 4, 32, 2, PRED>(P, sp, st, dependent);
 }
 
