@@ -39,12 +39,12 @@ NOMINAL_HBM_GBS = 8000.0
 # smaller row count of the same workload and scaled by rows; k_fit_rows: per row and iteration).  Keys: workload, with
 # "_bf16" for bfloat16 storage.  Remove an entry when its kernel changes.
 NCU_TRAFFIC_BYTES_PER_ROW = {
-    "cfg3": {"k_stream_rows": (514.067712e6 + 4.353792e6) / 500_000,
-             "k_fit_rows": (1.501335e9 + 3.986176e6) / 3 / 500_000},
-    "cfg4": {"k_stream_split": (491.691264e6 + 4.271616e6) / 30_000},
-    "cfg3_bf16": {"k_stream_rows": (516.026112e6 + 3.413504e6) / 1_000_000,
-                  "k_fit_rows": (1.503216e9 + 5.057536e6) / 3 / 1_000_000},
-    "cfg4_bf16": {"k_stream_split": (491.804160e6 + 3.820032e6) / 60_000},
+    "cfg3": {"k_stream_rows": (514.040064e6 + 3.598336e6) / 500_000,
+             "k_fit_rows": (1.501257e9 + 3.482880e6) / 3 / 500_000},
+    "cfg4": {"k_stream_split": (491.682048e6 + 3.577600e6) / 30_000},
+    "cfg3_bf16": {"k_stream_rows": (516.026624e6 + 3.481088e6) / 1_000_000,
+                  "k_fit_rows": (1.503338e9 + 5.044224e6) / 3 / 1_000_000},
+    "cfg4_bf16": {"k_stream_split": (491.803904e6 + 5.702400e6) / 60_000},
 }
 FALLBACK_HBM_GBS = 6650.0
 
