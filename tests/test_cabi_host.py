@@ -196,3 +196,39 @@ def test_any_length_copies_stay_inside_the_matrix():
             assert [o for o in written if o >= off] == list(range(off, span, eb))
             seen += xbytes
         assert seen == eb * m * n
+
+
+def test_every_row_length_gets_a_launchable_plan():
+    """Sweeps n = 1 .. 8300 for both storage types and both alignments: the plan always names a kernel shape that exists,
+    fits the shared memory of a CTA, keeps at least one stage, and (staged kernels) sizes its stages as the kernels do."""
+    for bf16 in (False, True):
+        eb, epg = (2, 8) if bf16 else (4, 4)
+        for aligned in (True, False):
+            for n in list(range(1, 1100)) + list(range(1100, 8301, 4)) + [4097, 8191, 8193]:
+                p = api.plan_query(70_001, n, x_aligned16=aligned, bf16=bf16)
+                v = p["variant"]
+                assert p["smem_bytes"] <= 227 * 1024 and p["grid"] >= 1 and p["threads"] in (256, 512)
+                if v in (0, 3):
+                    nw = p["threads"] // 32
+                    assert nw in (8, 16) and 1 <= p["stages"] <= 4
+                    lanes = p["lanes_per_row"]
+                    groups = n if v == 3 else n // epg
+                    assert lanes in (8, 16, 32) and p["vec_per_lane"] * lanes >= groups
+                    assert p["rows_per_batch"] % (32 // lanes) == 0
+                    stage = -(-(p["rows_per_batch"] * n * eb + (16 if v == 3 else 0)) // 128) * 128
+                    assert 1024 + nw * p["stages"] * stage <= p["smem_bytes"]
+                    assert p["smem_bytes"] >= 1024 + nw * n * 8 + 2 * nw * 8          # the end-of-kernel combine
+                    if v == 0:
+                        assert aligned and n % epg == 0
+                    else:
+                        assert n <= 512
+                elif v == 1:
+                    assert aligned and n % epg == 0 and p["threads"] == 512
+                    cw = -(-(n // epg) // 16)
+                    assert p["vec_per_lane"] * 32 >= cw and p["vec_per_lane"] in (1, 2, 4)
+                    assert cw * (2 if (not bf16 and cw > 64) else 4) <= 256                # tensor-map box limit
+                    stage = -(-p["rows_per_batch"] * cw * 16 // 128) * 128
+                    assert 1 <= p["stages"] <= 4 and p["smem_bytes"] == 4096 + 16 * p["stages"] * stage
+                else:
+                    assert v == 2 and p["threads"] == 256
+                    assert n > 512 and (not aligned or n % epg != 0 or n > 8192)

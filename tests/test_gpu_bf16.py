@@ -83,6 +83,16 @@ def test_loss_grad_matches_oracle(ctx, m, n):
     check_loss_grad(ctx, Xv, dev_bf16(bits), y, w, b)
 
 
+# both sides of every boundary between the bfloat16 kernel shapes
+@pytest.mark.parametrize("n", [8, 16, 64, 72, 128, 136, 256, 264, 512, 520, 1024, 1032, 2048, 2056, 4096, 4104, 8192, 8200, 9, 65,
+                               257, 511, 516])
+def test_shape_boundaries_bf16(ctx, n):
+    m = max(40, min(60_001, 24_000_000 // n)) + 3
+    X, y, w, b = datagen.random_problem(m, n, seed=6500 + n, wscale=1.0)
+    bits, Xv = oracle.round_bf16(X)
+    check_loss_grad(ctx, Xv, dev_bf16(bits), y, w, b)
+
+
 def test_library_conversion_feeds_the_pass(ctx):
     # fp32 on the device -> lr_convert_bf16 -> lr_loss_grad_bf16, against the checker on its own rounding of the same X
     X, y, w, b = datagen.random_problem(30_011, 256, seed=31, wscale=1.0)

@@ -59,6 +59,24 @@ def test_loss_grad_matches_oracle(ctx, m, n):
     check_loss_grad(ctx, X, y, w, b)
 
 
+# both sides of every boundary between kernel shapes (lanes per row, groups per lane, warps per CTA, rows per batch,
+# narrow / split / unstaged), for a row count that gives every warp several batches with a ragged last one
+BOUNDARY_N = [4, 8, 12, 32, 36, 64, 68, 128, 132, 256, 260, 384, 388, 512, 516, 1024, 1028, 1536, 1540, 2048, 2052, 3072, 3076,
+              4096, 4100, 8192, 8196, 9, 17, 33, 65, 129, 257, 513]
+
+
+@pytest.mark.parametrize("n", BOUNDARY_N)
+def test_shape_boundaries(ctx, n):
+    m = max(40, min(60_001, 24_000_000 // n)) + 3
+    X, y, w, b = datagen.random_problem(m, n, seed=6000 + n, wscale=1.0)
+    check_loss_grad(ctx, X, y, w, b)
+    dX, dw, db = dev(X), dev(w), dev(np.array([b], dtype=np.float32))
+    ref, z = oracle.predict(X, w, b, 0.5, return_z=True)
+    got = ctx.predict(dX, dw, db, 0.5).cpu().numpy()
+    clear = np.abs(z) > 1e-4 * (1 + np.abs(z))
+    assert np.array_equal(got[clear], ref[clear])
+
+
 @pytest.mark.parametrize("m,n", [(1000, 32), (3001, 100), (9999, 256), (640, 30)])
 def test_zero_parameters_give_ln2(ctx, m, n):
     X, y, _, _ = datagen.random_problem(m, n, seed=7)
