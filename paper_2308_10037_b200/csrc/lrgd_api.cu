@@ -107,30 +107,33 @@ int make_plan(int64_t m, int32_t n, bool aligned16, int32_t sms, lr_plan* P, boo
     }
     if (aligned16 && n % epg == 0 && n / epg <= kNW * (bf16 ? 64 : 128) && m < (int64_t(1) << 31) - 65536) {   // TMA coordinates are int32
         // wide rows: the warps of a CTA split each row by columns
-        const int cw = (n / epg + kNW - 1) / kNW;                               // 16-byte column groups per warp slice
+        // bfloat16 rows of up to 256 groups (1032..2048 columns) are split across eight warps instead of sixteen: slices of
+        // 17..32 groups, and 255 registers per thread, which 16-row batches need
+        const int nw = (bf16 && n / epg <= 256) ? 8 : kNW;
+        const int cw = (n / epg + nw - 1) / nw;                                 // 16-byte column groups per warp slice
         const int nv = cw > 64 ? 4 : (cw > 32 ? 2 : 1);            // fp32 rows of 4100..8192 columns: four groups per lane, two rows
         // Rows per batch.  All warps of a CTA meet once per batch, so a batch must carry enough bytes to cover that
         // round trip: slices of up to 24 groups per warp take 16 rows at a time and slices of 33..48 groups 8 rows, where 8
         // and 4 left the pass latency-bound (1028 columns: 3.6 TB/s, 2052: 4.2 TB/s); wider slices would leave room for
         // one stage only.
-        const int rb = nv == 4 ? 2 : nv == 2 ? (cw <= 48 && !bf16 ? 8 : 4)             // (the bfloat16 kernels would spill registers with the
-                               : (cw <= 24 && !bf16 ? 16 : 8);          //  larger batches)
+        const int rb = nv == 4 ? 2 : nv == 2 ? (cw <= 48 && !bf16 ? 8 : 4)             // (the 16-warp bfloat16 kernels would spill
+                               : (nw == 8 || (cw <= 24 && !bf16) ? 16 : 8);          //  registers with the larger batches)
         const int64_t B = (m + rb - 1) / rb;
         const int grid = int(std::min<int64_t>(B, sms));
         const int64_t per_cta = (B + grid - 1) / grid;
         const int64_t stage_stride = (int64_t(cw) * 16 * rb + 127) & ~int64_t(127);   // one densely packed box per stage
-        int D = int(std::min<int64_t>(kMaxDepth, kStageBudgetBytes / (kNW * stage_stride)));
+        int D = int(std::min<int64_t>(kMaxDepth, kStageBudgetBytes / (nw * stage_stride)));
         D = int(std::min<int64_t>(D, per_cta));
         if (D < 1) D = 1;
         P->variant = 1;
-        P->lanes_per_row = kNW * 32;
+        P->lanes_per_row = nw * 32;
         P->vec_per_lane = nv;
         P->rows_per_batch = rb;
         P->tile_rows = rb;
         P->stages = D;
         P->grid = grid;
-        P->threads = kNW * 32;
-        P->smem_bytes = int(kSplitHeaderBytes + int64_t(kNW) * D * stage_stride);
+        P->threads = nw * 32;
+        P->smem_bytes = int(kSplitHeaderBytes + int64_t(nw) * D * stage_stride);
         if (per_cta >= (int64_t(1) << 31)) return LR_ERR_SHAPE;
         return LR_OK;
     }
@@ -304,9 +307,9 @@ cudaError_t make_x_tensor_map(const void* X, bool bf16, int64_t m, int32_t n, in
     return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
 }
 
-template <class E, int NV, int RB, bool PRED>
+template <class E, int NV, int RB, bool PRED, int NW = kNW>
 cudaError_t launch_split_t(const lr_plan& P, const CUtensorMap& tm, const SplitParams& sp, cudaStream_t st, bool dependent) {
-    auto kern = k_stream_split<E, NV, RB, kNW, PRED>;
+    auto kern = k_stream_split<E, NV, RB, NW, PRED>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, P.smem_bytes);
     if (e != cudaSuccess) return e;
     return launch_kernel(kern, dim3(P.grid), dim3(P.threads), size_t(P.smem_bytes), st, dependent, tm, sp);
@@ -319,6 +322,7 @@ cudaError_t launch_split(const lr_plan& P, const void* X, const SplitParams& sp,
     cudaError_t e = make_x_tensor_map(X, bf16, sp.m, sp.n, sp.cw, P.rows_per_batch, &tm);
     if (e != cudaSuccess) return e;
     if (bf16) {
+        if (P.threads == 256) return launch_split_t<ElemBF16, 1, 16, PRED, 8>(P, tm, sp, st, dependent);    // eight warps per CTA
         if (P.vec_per_lane == 2) return launch_split_t<ElemBF16, 2, 4, PRED>(P, tm, sp, st, dependent);
         return launch_split_t<ElemBF16, 1, 8, PRED>(P, tm, sp, st, dependent);
     }
@@ -413,7 +417,7 @@ int launch_stream_pass(lr_ctx* ctx, const lr_plan& P, const Pass& a, uint8_t* la
         sp.y = a.y; sp.m = a.m; sp.n = a.n; sp.w = a.w; sp.b = a.b;
         sp.partial = ctx->d_partial; sp.labels = labels; sp.cut = cut; sp.status = ctx->d_status; sp.stop = a.stop;
         sp.depth = P.stages;
-        sp.cw = (a.n / (a.bf16 ? 8 : 4) + kNW - 1) / kNW;
+        sp.cw = (a.n / (a.bf16 ? 8 : 4) + P.threads / 32 - 1) / (P.threads / 32);      // groups per warp slice, as planned
         sp.x_per_group = split_words64(a.bf16, sp.cw) ? 2 : 4;
         sp.num_batches = (a.m + P.rows_per_batch - 1) / P.rows_per_batch;
         sp.keep_rows = keep_rows_for(ctx, 1, a.n, a.bf16);
@@ -1171,7 +1175,7 @@ extern "C" int lr_loss_grad_noalloc(int32_t device, const float* d_X, const floa
         sp.y = d_y; sp.m = m; sp.n = n; sp.w = d_w; sp.b = d_b;
         sp.partial = partial; sp.labels = nullptr; sp.cut = 0.f; sp.status = status;
         sp.depth = P.stages;
-        sp.cw = (n / 4 + kNW - 1) / kNW;
+        sp.cw = (n / 4 + P.threads / 32 - 1) / (P.threads / 32);
         sp.x_per_group = split_words64(false, sp.cw) ? 2 : 4;
         sp.num_batches = (m + P.rows_per_batch - 1) / P.rows_per_batch;
         e = launch_split<false>(P, d_X, sp, st);

@@ -223,12 +223,14 @@ def test_every_row_length_gets_a_launchable_plan():
                     else:
                         assert n <= 512
                 elif v == 1:
-                    assert aligned and n % epg == 0 and p["threads"] == 512
-                    cw = -(-(n // epg) // 16)
+                    nw = p["threads"] // 32
+                    assert aligned and n % epg == 0 and nw == (8 if bf16 and n // epg <= 256 else 16)
+                    cw = -(-(n // epg) // nw)
                     assert p["vec_per_lane"] * 32 >= cw and p["vec_per_lane"] in (1, 2, 4)
                     assert cw * (2 if (not bf16 and cw > 64) else 4) <= 256                # tensor-map box limit
+                    assert 2 * nw * p["rows_per_batch"] * 4 <= 4096 - 1024                   # the logit exchange fits the header
                     stage = -(-p["rows_per_batch"] * cw * 16 // 128) * 128
-                    assert 1 <= p["stages"] <= 4 and p["smem_bytes"] == 4096 + 16 * p["stages"] * stage
+                    assert 1 <= p["stages"] <= 4 and p["smem_bytes"] == 4096 + nw * p["stages"] * stage
                 else:
                     assert v == 2 and p["threads"] == 256
                     assert n > 512 and (not aligned or n % epg != 0 or n > 8192)
