@@ -107,16 +107,16 @@ int make_plan(int64_t m, int32_t n, bool aligned16, int32_t sms, lr_plan* P, boo
     }
     if (aligned16 && n % epg == 0 && n / epg <= kNW * (bf16 ? 64 : 128) && m < (int64_t(1) << 31) - 65536) {   // TMA coordinates are int32
         // wide rows: the warps of a CTA split each row by columns
-        // bfloat16 rows of up to 256 groups (1032..2048 columns) are split across eight warps instead of sixteen: slices of
-        // 17..32 groups, and 255 registers per thread, which 16-row batches need
-        const int nw = (bf16 && n / epg <= 256) ? 8 : kNW;
+        // bfloat16 rows of up to 384 groups (1032..3072 columns) are split across eight warps instead of sixteen: wider
+        // slices, and 255 registers per thread, which batches of 16 (one group per lane) or 8 rows (two groups) need
+        const int nw = (bf16 && n / epg <= 384) ? 8 : kNW;
         const int cw = (n / epg + nw - 1) / nw;                                 // 16-byte column groups per warp slice
         const int nv = cw > 64 ? 4 : (cw > 32 ? 2 : 1);            // fp32 rows of 4100..8192 columns: four groups per lane, two rows
         // Rows per batch.  All warps of a CTA meet once per batch, so a batch must carry enough bytes to cover that
         // round trip: slices of up to 24 groups per warp take 16 rows at a time and slices of 33..48 groups 8 rows, where 8
         // and 4 left the pass latency-bound (1028 columns: 3.6 TB/s, 2052: 4.2 TB/s); wider slices would leave room for
         // one stage only.
-        const int rb = nv == 4 ? 2 : nv == 2 ? (cw <= 48 && !bf16 ? 8 : 4)             // (the 16-warp bfloat16 kernels would spill
+        const int rb = nv == 4 ? 2 : nv == 2 ? (nw == 8 || (cw <= 48 && !bf16) ? 8 : 4)  // (the 16-warp bfloat16 kernels would spill
                                : (nw == 8 || (cw <= 24 && !bf16) ? 16 : 8);          //  registers with the larger batches)
         const int64_t B = (m + rb - 1) / rb;
         const int grid = int(std::min<int64_t>(B, sms));
@@ -322,6 +322,7 @@ cudaError_t launch_split(const lr_plan& P, const void* X, const SplitParams& sp,
     cudaError_t e = make_x_tensor_map(X, bf16, sp.m, sp.n, sp.cw, P.rows_per_batch, &tm);
     if (e != cudaSuccess) return e;
     if (bf16) {
+        if (P.threads == 256 && P.vec_per_lane == 2) return launch_split_t<ElemBF16, 2, 8, PRED, 8>(P, tm, sp, st, dependent);
         if (P.threads == 256) return launch_split_t<ElemBF16, 1, 16, PRED, 8>(P, tm, sp, st, dependent);    // eight warps per CTA
         if (P.vec_per_lane == 2) return launch_split_t<ElemBF16, 2, 4, PRED>(P, tm, sp, st, dependent);
         return launch_split_t<ElemBF16, 1, 8, PRED>(P, tm, sp, st, dependent);

@@ -224,7 +224,7 @@ def test_every_row_length_gets_a_launchable_plan():
                         assert n <= 512
                 elif v == 1:
                     nw = p["threads"] // 32
-                    assert aligned and n % epg == 0 and nw == (8 if bf16 and n // epg <= 256 else 16)
+                    assert aligned and n % epg == 0 and nw == (8 if bf16 and n // epg <= 384 else 16)
                     cw = -(-(n // epg) // nw)
                     assert p["vec_per_lane"] * 32 >= cw and p["vec_per_lane"] in (1, 2, 4)
                     assert cw * (2 if (not bf16 and cw > 64) else 4) <= 256                # tensor-map box limit
