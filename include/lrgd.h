@@ -51,15 +51,15 @@ typedef struct lr_ctx lr_ctx;
 /* Launch plan for a given shape, as chosen by the host logic (pure host code, no CUDA call). */
 typedef struct lr_plan {
     int32_t variant;       /* 0 = row-per-lane-group staged kernel, 1 = row-split staged kernel, 2 = unstaged generic kernel,
-                              3 = row-per-lane-group staged kernel for fp32 rows of any length up to 512 and any 4-byte aligned
-                              matrix (a lane owns single elements: vec_per_lane counts elements, not 16-byte groups) */
-    int32_t lanes_per_row; /* staged kernels: lanes that share one row (8, 16, 32; 512 for the row-split kernel) */
+                              3 = row-per-lane-group staged kernel for rows of any length up to 512 in a matrix aligned to its
+                              element size only (a lane owns single elements: vec_per_lane counts elements, not 16-byte groups) */
+    int32_t lanes_per_row; /* staged kernels: lanes that share one row (8, 16, 32; all threads of the CTA for the row-split kernel) */
     int32_t vec_per_lane;  /* staged kernels: 16-byte column groups owned by one lane */
     int32_t rows_per_batch;/* rows one warp (or one CTA for the row-split kernel) holds in registers at a time */
     int32_t tile_rows;     /* rows per asynchronously staged shared-memory stage */
     int32_t stages;        /* stages (copies in flight) per warp; per CTA for the row-split kernel */
     int32_t grid;          /* CTAs */
-    int32_t threads;       /* threads per CTA */
+    int32_t threads;       /* threads per CTA: 512, or 256 for the shapes whose threads need more than 128 registers */
     int32_t smem_bytes;    /* dynamic shared memory per CTA */
 } lr_plan;
 
