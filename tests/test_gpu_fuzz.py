@@ -1,7 +1,7 @@
 """Seeded random shapes through every entry point that computes, against the float64 checker.
 
 The shape list is drawn once from a fixed seed, so the test is reproducible; it mixes the three kernel families
-(narrow staged rows, wide split rows, unstaged), tiny and ragged row counts, and iteration counts that make the
+(narrow staged rows of whole groups and of any length, wide rows, unstaged), tiny and ragged row counts, and iteration counts that make the
 persistent fit kernel wrap its stages across iteration boundaries in every phase.
 """
 import numpy as np
@@ -23,7 +23,7 @@ def _shapes():
         if family == 0:
             n = int(g.integers(1, 129)) * 4                     # staged narrow rows: 4 .. 512
         elif family == 1:
-            n = int(g.integers(129, 1025)) * 4                  # split wide rows: 516 .. 4096
+            n = int(g.integers(129, 2049)) * 4                  # wide rows: 516 .. 8192 (eight-warp and row-split kernels)
         else:
             n = int(g.integers(1, 700))                         # anything, mostly not a multiple of 4
         budget = 6_000_000 // n                                 # keep each case at a few MB
@@ -37,7 +37,7 @@ def _shapes():
 def ctx():
     from paper_2308_10037_b200 import build
     build.build()
-    c = api.Context(n_max=4096, device=0)
+    c = api.Context(n_max=8192, device=0)
     yield c
     assert c.device_status() == 0
     c.close()
