@@ -67,6 +67,7 @@ bool any_row_shape_for(int n, RowShape* s) {
     else if (n <= 128) *s = {4, 32, 8};
     else if (n <= 256) *s = {8, 32, 4};
     else if (n <= 512) *s = {16, 32, 2};
+    else if (n <= 1024) *s = {32, 32, 1, 8};                // eight warps per CTA, one row at a time (up to 4 KB)
     else return false;
     return true;
 }
@@ -243,6 +244,7 @@ cudaError_t launch_rows(const lr_plan& P, const StreamParams& sp, cudaStream_t s
         if (P.vec_per_lane == 2) return launch_rows_t<ElemBF16Any, 2, 32, 16, PRED>(P, sp, st, dependent);
         if (P.vec_per_lane == 4) return launch_rows_t<ElemBF16Any, 4, 32, 8, PRED>(P, sp, st, dependent);
         if (P.vec_per_lane == 8) return launch_rows_t<ElemBF16Any, 8, 32, 4, PRED>(P, sp, st, dependent);
+        if (P.vec_per_lane == 32) return launch_rows_t<ElemBF16Any, 32, 32, 1, PRED, 8>(P, sp, st, dependent);
         return launch_rows_t<ElemBF16Any, 16, 32, 2, PRED>(P, sp, st, dependent);
     }
     if (P.variant == 3) {
@@ -252,6 +254,7 @@ cudaError_t launch_rows(const lr_plan& P, const StreamParams& sp, cudaStream_t s
         if (P.vec_per_lane == 2) return launch_rows_t<ElemF32Any, 2, 32, 16, PRED>(P, sp, st, dependent);
         if (P.vec_per_lane == 4) return launch_rows_t<ElemF32Any, 4, 32, 8, PRED>(P, sp, st, dependent);
         if (P.vec_per_lane == 8) return launch_rows_t<ElemF32Any, 8, 32, 4, PRED>(P, sp, st, dependent);
+        if (P.vec_per_lane == 32) return launch_rows_t<ElemF32Any, 32, 32, 1, PRED, 8>(P, sp, st, dependent);
         return launch_rows_t<ElemF32Any, 16, 32, 2, PRED>(P, sp, st, dependent);
     }
     if (bf16) {

@@ -68,16 +68,17 @@ def test_plan_staged_shapes(m, n, lpr, nv):
 
 
 def test_plan_falls_back_for_unaligned_or_odd_shapes():
-    assert api.plan_query(1000, 515)["variant"] == 2         # n not a multiple of 4 and wider than 512
-    assert api.plan_query(1000, 516, x_aligned16=False)["variant"] == 2    # wide rows need a 16-byte aligned matrix
+    assert api.plan_query(1000, 1027)["variant"] == 2        # n not a multiple of 4 and wider than 1024
+    assert api.plan_query(1000, 1028, x_aligned16=False)["variant"] == 2   # wide rows need a 16-byte aligned matrix
+    assert api.plan_query(1000, 515)["variant"] == 3 and api.plan_query(1000, 516, x_aligned16=False)["variant"] == 3
     assert api.plan_query(1000, 32, x_aligned16=False)["variant"] == 3     # narrow rows do not: element-wise staged kernel
     assert api.plan_query(1000, 30, x_aligned16=False)["variant"] == 3
     assert api.plan_query(1000, 32, x_aligned16=False, bf16=True)["variant"] == 3
     assert api.plan_query(1000, 8196)["variant"] == 2         # wider than any staged kernel
     assert api.plan_query(1000, 8200, bf16=True)["variant"] == 2
     assert api.plan_query(1000, 30, bf16=True)["variant"] == 3   # element-wise staged kernel, bfloat16 too
-    assert api.plan_query(1000, 516, bf16=True)["variant"] == 2  # 516 % 8 != 0 and wider than 512
-    g = api.plan_query(100, 515)
+    assert api.plan_query(1000, 1036, bf16=True)["variant"] == 2 # 1036 % 8 != 0 and wider than 1024
+    g = api.plan_query(100, 1027)
     assert g["grid"] == 2 and g["threads"] == 256
 
 
@@ -163,6 +164,7 @@ def test_any_length_copies_stay_inside_the_matrix():
     shapes = [(2758, 449), (1, 1), (7, 3), (300, 1), (640, 30), (1025, 101), (526, 255), (999, 511), (5, 510), (3, 258),
               (17, 257), (2, 449), (1, 511)]
     shapes += [(rnd.randint(1, 3000), rnd.choice([n for n in range(1, 513) if n % 4])) for _ in range(200)]
+    shapes += [(3, 513), (1, 1023), (77, 1021), (500, 777), (2, 1022)] + [(rnd.randint(1, 400), rnd.choice([n for n in range(513, 1025) if n % 4])) for _ in range(40)]
     cases = [(m, n, 0, 4) for m, n in shapes]
     extra = shapes[:60] + [(1, 1), (2, 2), (3, 1), (40, 32), (999, 256), (77, 512)]
     cases += [(m, n, base, 4) for (m, n) in extra for base in (4, 8, 12)]
@@ -174,7 +176,7 @@ def test_any_length_copies_stay_inside_the_matrix():
         rpb, row_bytes = p["rows_per_batch"], eb * n
         lo_x, hi_x = 4096 + base, 4096 + base + eb * m * n         # the matrix occupies the addresses [lo_x, hi_x)
         stage = -(-(rpb * row_bytes + 16) // 128) * 128
-        assert 1024 + 16 * p["stages"] * stage <= p["smem_bytes"]
+        assert 1024 + (p["threads"] // 32) * p["stages"] * stage <= p["smem_bytes"]
         seen = 0
         for g in range(-(-m // rpb)):
             r0 = g * rpb
@@ -221,7 +223,7 @@ def test_every_row_length_gets_a_launchable_plan():
                     if v == 0:
                         assert aligned and n % epg == 0
                     else:
-                        assert n <= 512
+                        assert n <= 1024
                 elif v == 1:
                     nw = p["threads"] // 32
                     assert aligned and n % epg == 0 and nw == (8 if bf16 and n // epg <= 384 else 16)
@@ -233,4 +235,4 @@ def test_every_row_length_gets_a_launchable_plan():
                     assert 1 <= p["stages"] <= 4 and p["smem_bytes"] == 4096 + nw * p["stages"] * stage
                 else:
                     assert v == 2 and p["threads"] == 256
-                    assert n > 512 and (not aligned or n % epg != 0 or n > 8192)
+                    assert n > 1024 and (not aligned or n % epg != 0 or n > 8192)

@@ -45,7 +45,7 @@ def check_loss_grad(ctx, X, y, w, b, grad_tol=GRAD_TOL, loss_tol=LOSS_TOL):
 # shapes: every staged instantiation (n/4 <= 8, 16, 32, 64, 128), partly filled lane groups (28, 100, 200, 36),
 # rows of any length (n % 4 != 0, n <= 512), the unstaged kernel (n % 4 != 0 and n > 512, n > 4096), and row counts that
 # are tiny, ragged, or span many tiles
-SHAPES = [(777, 515), (301, 1001), (3_001, 8192), (1_001, 5000), (777, 6148), (20, 8196), (1, 4), (7, 4), (8, 3), (33, 28), (1000, 32), (4097, 32), (5003, 64), (2500, 36), (3001, 100), (9999, 256),
+SHAPES = [(777, 515), (301, 1001), (301, 1027), (200, 2050), (3_001, 8192), (1_001, 5000), (777, 6148), (20, 8196), (1, 4), (7, 4), (8, 3), (33, 28), (1000, 32), (4097, 32), (5003, 64), (2500, 36), (3001, 100), (9999, 256),
           (777, 200), (1500, 512), (2049, 260), (640, 30), (1025, 101), (300, 1), (130, 4096), (50, 8192), (20011, 8),
           # enough rows that every warp refills its shared-memory stages many times, with a ragged last batch
           (200_003, 256), (400_001, 32), (200_002, 64), (120_007, 100), (150_001, 28), (60_001, 512), (90_001, 200),
@@ -95,7 +95,7 @@ def test_saturated_rows_stay_finite(ctx):
 
 
 @pytest.mark.parametrize("m,n,shift", [(1201, 32, 1), (150_003, 30, 1), (60_001, 256, 2), (40_001, 449, 3), (9, 5, 3), (1, 1, 1),
-                                       (2_001, 516, 1), (301, 1001, 2)])
+                                       (20_001, 516, 1), (20_003, 1024, 3), (2_001, 1028, 1), (301, 2001, 2)])
 def test_matrices_that_are_only_4_byte_aligned(ctx, m, n, shift):
     # a view that starts `shift` floats into an allocation: narrow rows stay on a staged kernel (element-wise groups; the
     # first batch is completed with plain loads instead of reading in front of the matrix), wide rows run unstaged
@@ -104,7 +104,7 @@ def test_matrices_that_are_only_4_byte_aligned(ctx, m, n, shift):
     buf[shift:shift + X.size] = dev(X).ravel()
     Xv = buf[shift:shift + X.size].view(m, n)
     assert Xv.data_ptr() % 16 == 4 * shift
-    assert api.plan_query(m, n, x_aligned16=False)["variant"] == (3 if n <= 512 else 2)
+    assert api.plan_query(m, n, x_aligned16=False)["variant"] == (3 if n <= 1024 else 2)
     L, g, g0 = oracle.loss_grad(X, y, w, b)
     dl, dg, dg0 = ctx.loss_grad(Xv, dev(y), dev(w), dev(np.array([b], dtype=np.float32)))
     assert abs(dl.item() - L) <= LOSS_TOL
@@ -204,7 +204,7 @@ def test_predict_matches_oracle(ctx, m, n):
 # fp32 rows whose length is not a multiple of four (a lane owns single elements): every instantiation (n <= 8, 16, 32, 64,
 # 128, 256, 512), batches that do not start on a 16-byte boundary (two-row batches of odd-length rows), ragged tails whose
 # byte count is not a multiple of 16, stage reuse
-ANY_LENGTH = [(33, 7), (1, 3), (20_011, 5), (40_003, 13), (150_001, 30), (90_001, 49), (100_001, 101), (200_003, 255),
+ANY_LENGTH = [(40_001, 513), (30_003, 777), (25_001, 1023), (3, 1001), (33, 7), (1, 3), (20_011, 5), (40_003, 13), (150_001, 30), (90_001, 49), (100_001, 101), (200_003, 255),
               (2_758, 449), (60_001, 449), (50_002, 511), (5, 510), (3, 258), (17, 257), (70_001, 258), (1, 511)]
 
 
