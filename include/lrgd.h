@@ -86,8 +86,8 @@ int lr_destroy(lr_ctx* ctx);
  * Inputs d_X [m*n], d_y [m], d_w [n], d_b [1] are read only.  Two kernels are enqueued: the fused
  * streaming kernel (reads X once) and the fixed-order cross-CTA reduction.
  * Which streaming kernel runs depends on the shape (lr_plan_query tells): rows of up to 1024 columns always take a staged
- * kernel that runs at or near HBM speed (fastest with d_X 16-byte aligned and n % 4 == 0); so do rows of up to 8192
- * columns with n % 4 == 0 and d_X 16-byte aligned; anything else runs on a slower unstaged kernel.
+ * kernel (at HBM speed with d_X 16-byte aligned and n % 4 == 0, at a half to nine tenths of it otherwise); so do rows
+ * of up to 8192 columns with n % 4 == 0 and d_X 16-byte aligned; anything else runs on a slower unstaged kernel.
  */
 int lr_loss_grad(lr_ctx* ctx, const float* d_X, const float* d_y, int64_t m, int32_t n,
                  const float* d_w, const float* d_b,
