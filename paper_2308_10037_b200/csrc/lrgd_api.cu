@@ -224,13 +224,38 @@ cudaError_t launch_kernel(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t 
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = dependent ? attr : nullptr;
     cfg.numAttrs = dependent ? 1 : 0;
-    return cudaLaunchKernelEx(&cfg, kern, std::forward<Args>(args)...);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, kern, args...);
+    if (dependent && (e == cudaErrorNotSupported || e == cudaErrorInvalidValue)) {
+        // a driver or stream that does not take the attribute: the ordinary launch computes the same thing
+        cudaGetLastError();
+        cfg.attrs = nullptr;
+        cfg.numAttrs = 0;
+        e = cudaLaunchKernelEx(&cfg, kern, args...);
+    }
+    return e;
 }
+
+// Raises a kernel's dynamic shared-memory limit to `smem` on the current device, once: the limit is remembered per
+// kernel instantiation (Tag) and device, so that the thousands of launches of a fit do not repeat the runtime call.
+template <class Tag>
+cudaError_t ensure_dynamic_smem(const void* kern, int smem) {
+    constexpr int kDevices = 64;
+    static int have[kDevices] = {};
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev >= 0 && dev < kDevices && have[dev] >= smem) return cudaSuccess;
+    e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e == cudaSuccess && dev >= 0 && dev < kDevices) have[dev] = smem;
+    return e;
+}
+template <class E, int A, int B, int C, int D, bool F>
+struct KernelTag {};
 
 template <class E, int NV, int LPR, int RB, bool PRED, int NW = kNW>
 cudaError_t launch_rows_t(const lr_plan& P, const StreamParams& sp, cudaStream_t st, bool dependent) {
     auto kern = k_stream_rows<E, NV, LPR, RB, NW, PRED>;
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, P.smem_bytes);
+    cudaError_t e = ensure_dynamic_smem<KernelTag<E, NV, LPR, RB, NW, PRED>>(reinterpret_cast<const void*>(kern), P.smem_bytes);
     if (e != cudaSuccess) return e;
     return launch_kernel(kern, dim3(P.grid), dim3(P.threads), size_t(P.smem_bytes), st, dependent, sp);
 }
@@ -313,7 +338,7 @@ cudaError_t make_x_tensor_map(const void* X, bool bf16, int64_t m, int32_t n, in
 template <class E, int NV, int RB, bool PRED, int NW = kNW>
 cudaError_t launch_split_t(const lr_plan& P, const CUtensorMap& tm, const SplitParams& sp, cudaStream_t st, bool dependent) {
     auto kern = k_stream_split<E, NV, RB, NW, PRED>;
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, P.smem_bytes);
+    cudaError_t e = ensure_dynamic_smem<KernelTag<E, NV, -1, RB, NW, PRED>>(reinterpret_cast<const void*>(kern), P.smem_bytes);
     if (e != cudaSuccess) return e;
     return launch_kernel(kern, dim3(P.grid), dim3(P.threads), size_t(P.smem_bytes), st, dependent, tm, sp);
 }

@@ -57,6 +57,9 @@ __global__ void __launch_bounds__(32 * kRedSlices) k_reduce_update(const ReduceP
     const int per = (p.G + kRedSlices - 1) / kRedSlices;
     const int g0 = slice * per;
     const int g1 = g0 + per < p.G ? g0 + per : p.G;
+    // the parameter this thread will update is fetched together with the partial rows (one round trip instead of two)
+    float old_param = 0.f;
+    if (p.update && slice == 0 && col <= p.n) old_param = col < p.n ? __ldcg(p.w + col) : __ldcg(p.b);
     double s = 0.0;
     if (col < stride) {
         const double* src = p.partial + col;
@@ -74,10 +77,10 @@ __global__ void __launch_bounds__(32 * kRedSlices) k_reduce_update(const ReduceP
         } else {
             const double v = t * p.inv_m;
             if (col < p.n) {
-                if (p.update) p.w[col] = static_cast<float>(static_cast<double>(p.w[col]) - p.lr * v);
+                if (p.update) p.w[col] = static_cast<float>(static_cast<double>(old_param) - p.lr * v);
                 else p.grad_w[col] = static_cast<float>(v);
             } else if (col == p.n) {
-                if (p.update) p.b[0] = static_cast<float>(static_cast<double>(p.b[0]) - p.lr * v);
+                if (p.update) p.b[0] = static_cast<float>(static_cast<double>(old_param) - p.lr * v);
                 else p.grad_b[0] = static_cast<float>(v);
             } else {
                 if (p.loss_out) p.loss_out[0] = static_cast<float>(v);
