@@ -32,7 +32,8 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
-METRIC = "GD iterations/sec (full-batch, m x n fp32)"
+# value is the iterations/sec part; the GB/s and the fraction of peak are in `achieved_hbm_gbs_whole_step` and `roofline`
+METRIC = "GD iterations/sec and achieved HBM GB/s (fraction of B200 peak) at m\u00d7n fp32"
 UNIT = "iterations/s"
 NOMINAL_HBM_GBS = 8000.0
 # dram__bytes_read.sum + dram__bytes_write.sum per row of X, from the ncu captures summarised in profiles/ (taken on a
