@@ -101,13 +101,16 @@ int lr_loss_grad(lr_ctx* ctx, const float* d_X, const float* d_y, int64_t m, int
  * Results are bit-reproducible for a given shape and device, and fit(a) followed by fit(b) equals
  * fit(a+b) bit for bit.
  * Two forms give the same bits.  Two kernels per iteration (the pass, then the reduction with the update), each
- * launched as the programmatic dependent of the one before it (see lr_set_overlap); or, for rows of up to 512 columns
- * (16-byte aligned X, n % 4 == 0) and iters >= 2, ONE cooperative launch of a persistent kernel for the whole call (grid
- * barriers between the pass and the update; the HBM stream continues across iterations).  By default the library takes
- * the persistent kernel for fp32 matrices of 64 MB and more, where it measures faster, and two kernels otherwise.
+ * launched as the programmatic dependent of the one before it (see lr_set_overlap); or, for rows of up to 256 or of
+ * 388..512 columns (the shapes whose kernel runs 16 warps per CTA; 16-byte aligned X, n % 4 == 0) and iters >= 2, ONE cooperative
+ * launch of a persistent kernel for the whole call: one grid barrier per iteration, after which every CTA adds up the
+ * partial sums for itself and keeps its own copy of the parameters; the HBM stream continues across iterations, and a
+ * problem whose rows all fit the CTAs' shared memory (up to ~28 MB) is fetched once and kept there for the whole call.
+ * The library takes the persistent kernel wherever the shape allows it (it measures at least as fast everywhere).
  * lr_set_persistent(ctx, 0) forces two kernels (also used while lr_profile_enable is on, so that single launches can
- * be timed), lr_set_persistent(ctx, 1) the persistent kernel wherever the shape allows it, a negative value restores
- * the default.  The same choice applies to lr_fit_tol and the bfloat16 calls.
+ * be timed), any other value restores the default.  The same choice applies to lr_fit_tol and the bfloat16 calls.
+ * If a bounded wait inside the persistent kernel expires, the kernel stops, the status word reports LR_ERR_TIMEOUT and
+ * d_w, d_b are left as they were on entry.
  */
 int lr_fit(lr_ctx* ctx, const float* d_X, const float* d_y, int64_t m, int32_t n,
            float lr, int32_t iters, float* d_w, float* d_b, float* d_loss_hist, void* stream);
@@ -200,8 +203,8 @@ int lr_predict(lr_ctx* ctx, const float* d_X, int64_t m, int32_t n,
  * lr_loss_grad / lr_fit / lr_predict would compute on the fp32 matrix holding the same (bfloat16-representable) values.
  * Rows of up to 1024 columns always take a staged kernel (fastest with n % 8 == 0 and d_Xh 16-byte aligned); so do rows of
  * up to 8192 columns with n % 8 == 0 and d_Xh 16-byte aligned; other shapes run on the
- * unstaged kernel.  lr_fit_bf16 runs as two dependent-launched kernels per iteration unless lr_set_persistent(ctx, 1) asks for
- * the persistent kernel (n <= 512).  Errors as the fp32 calls.
+ * unstaged kernel.  lr_fit_bf16 takes the persistent kernel of lr_fit for rows of up to 512 columns with n % 8 == 0 and
+ * d_Xh 16-byte aligned.  Errors as the fp32 calls.
  *
  * lr_convert_bf16 rounds `count` fp32 values to bfloat16 (round to nearest, ties to even; NaN stays NaN, values past
  * the largest finite bfloat16 become infinity) -- one elementwise kernel on `stream`; d_X and d_Xh must not overlap.

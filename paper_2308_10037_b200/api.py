@@ -112,24 +112,45 @@ def plan_query(m: int, n: int, x_aligned16: bool = True, sm_count: int = 148, bf
     return p.as_dict()
 
 
-def _dev_ptr(t: torch.Tensor | None, dtype, name: str):
+def _dev_ptr(t: torch.Tensor | None, dtype, name: str, count: int | None = None, device: int | None = None):
+    """Device address of ``t`` after checking what the C side cannot see behind a bare pointer.
+
+    ``count`` is the number of elements the call reads or writes through the pointer: a shorter tensor would be an
+    out-of-bounds access on the device, so it is refused here with ValueError.  ``device`` is the index of the device
+    the call runs on; a tensor that lives on another one is refused as well.  None passes through (optional arguments).
+    """
     if t is None:
         return None
     if not (isinstance(t, torch.Tensor) and t.is_cuda and t.dtype == dtype and t.is_contiguous()):
         raise TypeError(f"{name}: expected a contiguous CUDA tensor of dtype {dtype}")
+    if count is not None and t.numel() < count:
+        raise ValueError(f"{name}: {t.numel()} elements, the call needs {count}")
+    if device is not None and t.device.index != device:
+        raise ValueError(f"{name}: lives on cuda:{t.device.index}, the call runs on cuda:{device}")
     return ctypes.c_void_p(t.data_ptr())
 
 
-def _host_ptr(a, dtype, name: str):
+def _shape2(X, name: str = "X"):
+    if not isinstance(X, (torch.Tensor, np.ndarray)) or X.ndim != 2 or X.shape[0] < 1 or X.shape[1] < 1:
+        raise ValueError(f"{name}: expected a 2-D array with at least one row and one column")
+    return int(X.shape[0]), int(X.shape[1])
+
+
+def _host_ptr(a, dtype, name: str, count: int | None = None):
+    """Host address of a CPU tensor or numpy array holding at least ``count`` elements of ``dtype``."""
     if a is None:
         return None
     if isinstance(a, torch.Tensor):
         if a.is_cuda or not a.is_contiguous() or a.dtype != dtype:
             raise TypeError(f"{name}: expected a contiguous CPU tensor of dtype {dtype}")
+        if count is not None and a.numel() < count:
+            raise ValueError(f"{name}: {a.numel()} elements, the call needs {count}")
         return ctypes.c_void_p(a.data_ptr())
     npdt = {torch.float32: np.float32, torch.uint8: np.uint8}[dtype]
     if not (isinstance(a, np.ndarray) and a.dtype == npdt and a.flags.c_contiguous):
         raise TypeError(f"{name}: expected a C-contiguous numpy array of dtype {npdt}")
+    if count is not None and a.size < count:
+        raise ValueError(f"{name}: {a.size} elements, the call needs {count}")
     return ctypes.c_void_p(a.ctypes.data)
 
 
@@ -172,109 +193,124 @@ class Context:
             return torch.bfloat16, "_bf16"
         return torch.float32, ""
 
+    def _p(self, t, dtype, name, count=None):
+        """``_dev_ptr`` for an argument of a call on this context: also checks that the tensor is on the context's device."""
+        return _dev_ptr(t, dtype, name, count, self.device)
+
     def convert_bf16(self, X, out=None):
         """Rounds a float32 CUDA tensor to bfloat16 (nearest, ties to even) with the library's kernel."""
+        px = self._p(X, torch.float32, "X")
+        count = X.numel()
         Xh = torch.empty(X.shape, dtype=torch.bfloat16, device=X.device) if out is None else out
-        rc = lib().lr_convert_bf16(self._h, _dev_ptr(X, torch.float32, "X"), X.numel(), _dev_ptr(Xh, torch.bfloat16, "Xh"),
-                                   self._stream())
+        rc = lib().lr_convert_bf16(self._h, px, count, self._p(Xh, torch.bfloat16, "Xh", count), self._stream())
         self._check(rc, "lr_convert_bf16")
         return Xh
 
     def loss_grad(self, X, y, w, b):
-        m, n = X.shape
+        m, n = _shape2(X)
         xdt, sfx = self._x_kind(X)
-        loss = torch.empty(1, dtype=torch.float32, device=X.device)
-        gw = torch.empty(n, dtype=torch.float32, device=X.device)
-        gb = torch.empty(1, dtype=torch.float32, device=X.device)
-        rc = getattr(lib(), "lr_loss_grad" + sfx)(self._h, _dev_ptr(X, xdt, "X"), _dev_ptr(y, torch.float32, "y"), m, n,
-                                _dev_ptr(w, torch.float32, "w"), _dev_ptr(b, torch.float32, "b"),
-                                _dev_ptr(loss, torch.float32, "loss"), _dev_ptr(gw, torch.float32, "grad_w"),
-                                _dev_ptr(gb, torch.float32, "grad_b"), self._stream())
+        F32 = torch.float32
+        inputs = (self._p(X, xdt, "X"), self._p(y, F32, "y", m), m, n, self._p(w, F32, "w", n), self._p(b, F32, "b", 1))
+        loss = torch.empty(1, dtype=F32, device=X.device)
+        gw = torch.empty(n, dtype=F32, device=X.device)
+        gb = torch.empty(1, dtype=F32, device=X.device)
+        rc = getattr(lib(), "lr_loss_grad" + sfx)(self._h, *inputs, self._p(loss, F32, "loss", 1),
+                                self._p(gw, F32, "grad_w", n), self._p(gb, F32, "grad_b", 1), self._stream())
         self._check(rc, "lr_loss_grad" + sfx)
         return loss, gw, gb
 
     def fit(self, X, y, lr, iters, w, b, loss_hist=None):
         """In place on ``w`` [n] and ``b`` [1]; ``loss_hist`` is None or a float32 CUDA tensor [iters]."""
-        m, n = X.shape
+        m, n = _shape2(X)
         xdt, sfx = self._x_kind(X)
-        rc = getattr(lib(), "lr_fit" + sfx)(self._h, _dev_ptr(X, xdt, "X"), _dev_ptr(y, torch.float32, "y"), m, n, float(lr),
-                          int(iters), _dev_ptr(w, torch.float32, "w"), _dev_ptr(b, torch.float32, "b"),
-                          _dev_ptr(loss_hist, torch.float32, "loss_hist"), self._stream())
+        F32, iters = torch.float32, int(iters)
+        rc = getattr(lib(), "lr_fit" + sfx)(self._h, self._p(X, xdt, "X"), self._p(y, F32, "y", m), m, n, float(lr), iters,
+                          self._p(w, F32, "w", n), self._p(b, F32, "b", 1), self._p(loss_hist, F32, "loss_hist", max(iters, 0)),
+                          self._stream())
         self._check(rc, "lr_fit" + sfx)
 
     def fit_tol(self, X, y, lr, eps, max_iters, w, b, check_every=16, loss_hist=None, gnorm_hist=None):
         """GD until ||grad||_2 <= eps (at most ``max_iters`` updates), in place on w, b.  Returns (updates, last norm)."""
-        m, n = X.shape
+        m, n = _shape2(X)
         done, nrm = ctypes.c_int32(), ctypes.c_float()
         xdt, sfx = self._x_kind(X)
-        rc = getattr(lib(), "lr_fit_tol" + sfx)(self._h, _dev_ptr(X, xdt, "X"), _dev_ptr(y, torch.float32, "y"), m, n, float(lr),
-                              float(eps), int(max_iters), int(check_every), _dev_ptr(w, torch.float32, "w"),
-                              _dev_ptr(b, torch.float32, "b"), _dev_ptr(loss_hist, torch.float32, "loss_hist"),
-                              _dev_ptr(gnorm_hist, torch.float32, "gnorm_hist"), ctypes.byref(done), ctypes.byref(nrm),
-                              self._stream())
+        F32, cap = torch.float32, max(int(max_iters), 0)
+        rc = getattr(lib(), "lr_fit_tol" + sfx)(self._h, self._p(X, xdt, "X"), self._p(y, F32, "y", m), m, n, float(lr),
+                              float(eps), int(max_iters), int(check_every), self._p(w, F32, "w", n), self._p(b, F32, "b", 1),
+                              self._p(loss_hist, F32, "loss_hist", cap), self._p(gnorm_hist, F32, "gnorm_hist", cap),
+                              ctypes.byref(done), ctypes.byref(nrm), self._stream())
         self._check(rc, "lr_fit_tol" + sfx)
         return done.value, nrm.value
 
     def fit_opt(self, X, y, lr, iters, w, b, l2=0.0, momentum=0.0, nesterov=False, velocity=None, loss_hist=None):
         """GD with an L2 penalty and (Nesterov) momentum, in place on w, b (and ``velocity`` [n+1] when given)."""
-        m, n = X.shape
+        m, n = _shape2(X)
         opt = LrOpt(float(l2), float(momentum), int(bool(nesterov)))
         xdt, sfx = self._x_kind(X)
-        rc = getattr(lib(), "lr_fit_opt" + sfx)(self._h, _dev_ptr(X, xdt, "X"), _dev_ptr(y, torch.float32, "y"), m, n, float(lr),
-                              int(iters), ctypes.byref(opt), _dev_ptr(w, torch.float32, "w"), _dev_ptr(b, torch.float32, "b"),
-                              _dev_ptr(velocity, torch.float32, "velocity"), _dev_ptr(loss_hist, torch.float32, "loss_hist"),
+        F32, iters = torch.float32, int(iters)
+        rc = getattr(lib(), "lr_fit_opt" + sfx)(self._h, self._p(X, xdt, "X"), self._p(y, F32, "y", m), m, n, float(lr),
+                              iters, ctypes.byref(opt), self._p(w, F32, "w", n), self._p(b, F32, "b", 1),
+                              self._p(velocity, F32, "velocity", n + 1), self._p(loss_hist, F32, "loss_hist", max(iters, 0)),
                               self._stream())
         self._check(rc, "lr_fit_opt" + sfx)
 
     def fit_sgd(self, X, y, lr, batch_rows, steps, w, b, first_batch=0, loss_hist=None):
         """Mini-batch GD over contiguous row blocks (block (first_batch + s) mod count at step s), in place on w, b."""
-        m, n = X.shape
+        m, n = _shape2(X)
         xdt, sfx = self._x_kind(X)
-        rc = getattr(lib(), "lr_fit_sgd" + sfx)(self._h, _dev_ptr(X, xdt, "X"), _dev_ptr(y, torch.float32, "y"), m, n, float(lr),
-                              int(batch_rows), int(steps), int(first_batch), _dev_ptr(w, torch.float32, "w"),
-                              _dev_ptr(b, torch.float32, "b"), _dev_ptr(loss_hist, torch.float32, "loss_hist"), self._stream())
+        F32, steps = torch.float32, int(steps)
+        rc = getattr(lib(), "lr_fit_sgd" + sfx)(self._h, self._p(X, xdt, "X"), self._p(y, F32, "y", m), m, n, float(lr),
+                              int(batch_rows), steps, int(first_batch), self._p(w, F32, "w", n), self._p(b, F32, "b", 1),
+                              self._p(loss_hist, F32, "loss_hist", max(steps, 0)), self._stream())
         self._check(rc, "lr_fit_sgd" + sfx)
 
     def predict(self, X, w, b, thr, out=None):
-        m, n = X.shape
-        labels = torch.empty(m, dtype=torch.uint8, device=X.device) if out is None else out
+        m, n = _shape2(X)
         xdt, sfx = self._x_kind(X)
-        rc = getattr(lib(), "lr_predict" + sfx)(self._h, _dev_ptr(X, xdt, "X"), m, n, _dev_ptr(w, torch.float32, "w"),
-                              _dev_ptr(b, torch.float32, "b"), float(thr), _dev_ptr(labels, torch.uint8, "labels"),
-                              self._stream())
+        F32 = torch.float32
+        px, pw, pb = self._p(X, xdt, "X"), self._p(w, F32, "w", n), self._p(b, F32, "b", 1)
+        labels = torch.empty(m, dtype=torch.uint8, device=X.device) if out is None else out
+        rc = getattr(lib(), "lr_predict" + sfx)(self._h, px, m, n, pw, pb, float(thr),
+                                                self._p(labels, torch.uint8, "labels", m), self._stream())
         self._check(rc, "lr_predict" + sfx)
         return labels
 
     def shard_sums(self, X, y, w, b, sums):
         """Unnormalised fp64 sums [n+2] of the local rows into ``sums`` (float64 CUDA tensor)."""
-        m, n = X.shape
+        m, n = _shape2(X)
         xdt, sfx = self._x_kind(X)
-        rc = getattr(lib(), "lr_shard_sums" + sfx)(self._h, _dev_ptr(X, xdt, "X"), _dev_ptr(y, torch.float32, "y"), m, n,
-                                 _dev_ptr(w, torch.float32, "w"), _dev_ptr(b, torch.float32, "b"),
-                                 _dev_ptr(sums, torch.float64, "sums"), self._stream())
+        F32 = torch.float32
+        rc = getattr(lib(), "lr_shard_sums" + sfx)(self._h, self._p(X, xdt, "X"), self._p(y, F32, "y", m), m, n,
+                                 self._p(w, F32, "w", n), self._p(b, F32, "b", 1),
+                                 self._p(sums, torch.float64, "sums", n + 2), self._stream())
         self._check(rc, "lr_shard_sums" + sfx)
 
     def apply_sums(self, sums_all, m_total, lr, w, b, loss=None):
         """Adds the ``parts`` rows of ``sums_all`` [parts, n+2] in order and applies the update to w, b in place."""
-        parts, n2 = sums_all.shape
-        rc = lib().lr_apply_sums(self._h, _dev_ptr(sums_all, torch.float64, "sums_all"), parts, int(m_total), n2 - 2,
-                                 float(lr), _dev_ptr(w, torch.float32, "w"), _dev_ptr(b, torch.float32, "b"),
-                                 _dev_ptr(loss, torch.float32, "loss"), self._stream())
+        parts, n2 = _shape2(sums_all, "sums_all")
+        if n2 < 3:
+            raise ValueError("sums_all: expected [parts, n+2] with n >= 1")
+        F32, n = torch.float32, n2 - 2
+        rc = lib().lr_apply_sums(self._h, self._p(sums_all, torch.float64, "sums_all"), parts, int(m_total), n,
+                                 float(lr), self._p(w, F32, "w", n), self._p(b, F32, "b", 1), self._p(loss, F32, "loss", 1),
+                                 self._stream())
         self._check(rc, "lr_apply_sums")
 
     # ---- host-pointer entry points ---------------------------------------------------------------
     def fit_host(self, X, y, lr, iters, w, b, loss_hist=None):
         """X, y, w, b (and loss_hist) are CPU tensors or numpy arrays; w, b are updated in place."""
-        m, n = X.shape
-        rc = lib().lr_fit_host(self._h, _host_ptr(X, torch.float32, "X"), _host_ptr(y, torch.float32, "y"), m, n,
-                               float(lr), int(iters), _host_ptr(w, torch.float32, "w"), _host_ptr(b, torch.float32, "b"),
-                               _host_ptr(loss_hist, torch.float32, "loss_hist"))
+        m, n = _shape2(X)
+        F32, iters = torch.float32, int(iters)
+        rc = lib().lr_fit_host(self._h, _host_ptr(X, F32, "X"), _host_ptr(y, F32, "y", m), m, n, float(lr), iters,
+                               _host_ptr(w, F32, "w", n), _host_ptr(b, F32, "b", 1),
+                               _host_ptr(loss_hist, F32, "loss_hist", max(iters, 0)))
         self._check(rc, "lr_fit_host")
 
     def predict_host(self, X, w, b, thr, labels):
-        m, n = X.shape
-        rc = lib().lr_predict_host(self._h, _host_ptr(X, torch.float32, "X"), m, n, _host_ptr(w, torch.float32, "w"),
-                                   _host_ptr(b, torch.float32, "b"), float(thr), _host_ptr(labels, torch.uint8, "labels"))
+        m, n = _shape2(X)
+        F32 = torch.float32
+        rc = lib().lr_predict_host(self._h, _host_ptr(X, F32, "X"), m, n, _host_ptr(w, F32, "w", n), _host_ptr(b, F32, "b", 1),
+                                   float(thr), _host_ptr(labels, torch.uint8, "labels", m))
         self._check(rc, "lr_predict_host")
 
     # ---- measurement / status --------------------------------------------------------------------
@@ -368,12 +404,15 @@ def lr_loss_grad_noalloc(X, y, w, b, loss, grad_w, grad_b, status=None):
     optionally ``status`` [1] int32, all CUDA tensors that already exist.  Scratch lives in a fixed array
     inside the library (n <= LR_NOALLOC_MAX_N); calls that overlap on the GPU race on it.
     """
-    m, n = X.shape
+    m, n = _shape2(X)
+    if not (isinstance(X, torch.Tensor) and X.is_cuda):
+        raise TypeError("X: expected a contiguous CUDA tensor of dtype torch.float32")
     dev = X.device.index if X.device.index is not None else torch.cuda.current_device()
-    rc = lib().lr_loss_grad_noalloc(int(dev), _dev_ptr(X, torch.float32, "X"), _dev_ptr(y, torch.float32, "y"), m, n,
-                                    _dev_ptr(w, torch.float32, "w"), _dev_ptr(b, torch.float32, "b"),
-                                    _dev_ptr(loss, torch.float32, "loss"), _dev_ptr(grad_w, torch.float32, "grad_w"),
-                                    _dev_ptr(grad_b, torch.float32, "grad_b"), _dev_ptr(status, torch.int32, "status"),
+    F32 = torch.float32
+    rc = lib().lr_loss_grad_noalloc(int(dev), _dev_ptr(X, F32, "X", None, dev), _dev_ptr(y, F32, "y", m, dev), m, n,
+                                    _dev_ptr(w, F32, "w", n, dev), _dev_ptr(b, F32, "b", 1, dev),
+                                    _dev_ptr(loss, F32, "loss", 1, dev), _dev_ptr(grad_w, F32, "grad_w", n, dev),
+                                    _dev_ptr(grad_b, F32, "grad_b", 1, dev), _dev_ptr(status, torch.int32, "status", 1, dev),
                                     ctypes.c_void_p(torch.cuda.current_stream(dev).cuda_stream))
     if rc != LR_OK:
         raise LrError(rc, "lr_loss_grad_noalloc")

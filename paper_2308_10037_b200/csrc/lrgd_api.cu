@@ -2,6 +2,9 @@
 // The declarations and their contracts are in include/lrgd.h.
 #include "../../include/lrgd.h"
 
+#include <nvtx3/nvToolsExt.h>
+
+#include <algorithm>
 #include <cmath>
 #include <cstdlib>
 #include <cstring>
@@ -162,10 +165,11 @@ struct lr_ctx {
     TolState* d_tol = nullptr;                      // stopping-rule state of lr_fit_tol
     double* d_gbuf = nullptr;                       // [n_max+1] gradient entries for the norm
     TolState* h_tol = nullptr;                      // pinned host mirror
+    int* h_words = nullptr;                         // pinned: [0] status word before a blocking call, [1] after it, [2] abort word of a persistent launch
     float* d_vel = nullptr;                         // [n_max+1] velocity of lr_fit_opt when the caller passes none
     double* d_oscr = nullptr;                       // [n_max+2] scratch of the optimiser reduction
     unsigned int* d_oticket = nullptr;
-    unsigned int* d_gbar = nullptr;                 // grid-barrier counter of the persistent fit kernel
+    unsigned int* d_gbar = nullptr;                 // persistent fit kernel: [0] grid-barrier counter, [1] abort flag of the launch
     bool coop = false;                              // device supports cooperative launches
     int persistent_mode = -1;                       // single-launch fit kernel: -1 the library chooses, 0 never, 1 whenever the shape allows
     bool overlap = true;                            // consecutive kernels of one call are launched as programmatic dependents
@@ -186,6 +190,12 @@ struct lr_ctx {
 };
 
 namespace {
+
+// A named range around a whole library call, visible on a profiler's timeline (costs nothing when no tool is attached).
+struct NvtxRange {
+    explicit NvtxRange(const char* name) { nvtxRangePushA(name); }
+    ~NvtxRange() { nvtxRangePop(); }
+};
 
 struct DeviceGuard {
     int prev = -1;
@@ -241,9 +251,11 @@ template <class Tag>
 cudaError_t ensure_dynamic_smem(const void* kern, int smem) {
     constexpr int kDevices = 64;
     static int have[kDevices] = {};
+    static std::mutex mu;                          // contexts on different host threads may share an instantiation
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
+    std::lock_guard<std::mutex> lock(mu);
     if (dev >= 0 && dev < kDevices && have[dev] >= smem) return cudaSuccess;
     e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e == cudaSuccess && dev >= 0 && dev < kDevices) have[dev] = smem;
@@ -311,15 +323,19 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
 cudaError_t make_x_tensor_map(const void* X, bool bf16, int64_t m, int32_t n, int cw, int rb, CUtensorMap* out) {
-    static EncodeTiledFn encode = nullptr;
-    if (!encode) {
+    // resolved once per process; the initialisation of a function-local static is thread-safe
+    struct Resolved { EncodeTiledFn fn = nullptr; cudaError_t err = cudaSuccess; };
+    static const Resolved resolved = [] {
+        Resolved r;
         void* fn = nullptr;
         cudaDriverEntryPointQueryResult q;
-        cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q);
-        if (e != cudaSuccess) return e;
-        if (q != cudaDriverEntryPointSuccess || !fn) return cudaErrorNotSupported;
-        encode = reinterpret_cast<EncodeTiledFn>(fn);
-    }
+        r.err = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q);
+        if (r.err == cudaSuccess && (q != cudaDriverEntryPointSuccess || !fn)) r.err = cudaErrorNotSupported;
+        if (r.err == cudaSuccess) r.fn = reinterpret_cast<EncodeTiledFn>(fn);
+        return r;
+    }();
+    if (resolved.err != cudaSuccess) return resolved.err;
+    const EncodeTiledFn encode = resolved.fn;
     // (fp32 slices of more than 64 groups -- rows of more than 4096 columns -- are described as 64-bit words for the same reason)
     const bool wide64 = split_words64(bf16, cw);
     const cuuint64_t row_bytes = cuuint64_t(n) * (bf16 ? 2 : 4);
@@ -363,27 +379,29 @@ cudaError_t launch_split(const lr_plan& P, const void* X, const SplitParams& sp,
 }
 
 template <class E, int NV, int LPR, int RB>
-cudaError_t launch_fit_t(const lr_plan& P, int smem, FitParams& fp, cudaStream_t st) {
-    auto kern = k_fit_rows<E, NV, LPR, RB, kNW>;
+cudaError_t launch_fit_t(const lr_plan& P, int smem, bool resident, FitParams& fp, cudaStream_t st) {
+    const void* kern = resident ? reinterpret_cast<const void*>(k_fit_rows<E, NV, LPR, RB, kNW, true>)
+                                : reinterpret_cast<const void*>(k_fit_rows<E, NV, LPR, RB, kNW, false>);
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
     void* args[] = {&fp};
-    return cudaLaunchCooperativeKernel(reinterpret_cast<void*>(kern), dim3(P.grid), dim3(P.threads), args, size_t(smem), st);
+    return cudaLaunchCooperativeKernel(kern, dim3(P.grid), dim3(P.threads), args, size_t(smem), st);
 }
 
-cudaError_t launch_fit(const lr_plan& P, int smem, FitParams& fp, cudaStream_t st, bool bf16 = false) {
+// resident: every warp's share of X fits its stages, which are then filled once and kept for the whole fit
+cudaError_t launch_fit(const lr_plan& P, int smem, bool resident, FitParams& fp, cudaStream_t st, bool bf16 = false) {
     if (bf16) {
-        if (P.lanes_per_row == 8) return launch_fit_t<ElemBF16, 1, 8, 8>(P, smem, fp, st);
-        if (P.lanes_per_row == 16) return launch_fit_t<ElemBF16, 1, 16, 8>(P, smem, fp, st);
-        if (P.vec_per_lane == 1) return launch_fit_t<ElemBF16, 1, 32, LRGD_NV1_RB>(P, smem, fp, st);
-        if (P.vec_per_lane == 2) return launch_fit_t<ElemBF16, 2, 32, LRGD_NV2_RB>(P, smem, fp, st);
+        if (P.lanes_per_row == 8) return launch_fit_t<ElemBF16, 1, 8, 8>(P, smem, resident, fp, st);
+        if (P.lanes_per_row == 16) return launch_fit_t<ElemBF16, 1, 16, 8>(P, smem, resident, fp, st);
+        if (P.vec_per_lane == 1) return launch_fit_t<ElemBF16, 1, 32, LRGD_NV1_RB>(P, smem, resident, fp, st);
+        if (P.vec_per_lane == 2) return launch_fit_t<ElemBF16, 2, 32, LRGD_NV2_RB>(P, smem, resident, fp, st);
         return cudaErrorInvalidValue;
     }
-    if (P.lanes_per_row == 8) return launch_fit_t<ElemF32, 1, 8, 8>(P, smem, fp, st);
-    if (P.lanes_per_row == 16) return launch_fit_t<ElemF32, 1, 16, 8>(P, smem, fp, st);
-    if (P.vec_per_lane == 1) return launch_fit_t<ElemF32, 1, 32, LRGD_NV1_RB>(P, smem, fp, st);
-    if (P.vec_per_lane == 2) return launch_fit_t<ElemF32, 2, 32, LRGD_NV2_RB>(P, smem, fp, st);
-    return launch_fit_t<ElemF32, 4, 32, 2>(P, smem, fp, st);
+    if (P.lanes_per_row == 8) return launch_fit_t<ElemF32, 1, 8, 8>(P, smem, resident, fp, st);
+    if (P.lanes_per_row == 16) return launch_fit_t<ElemF32, 1, 16, 8>(P, smem, resident, fp, st);
+    if (P.vec_per_lane == 1) return launch_fit_t<ElemF32, 1, 32, LRGD_NV1_RB>(P, smem, resident, fp, st);
+    if (P.vec_per_lane == 2) return launch_fit_t<ElemF32, 2, 32, LRGD_NV2_RB>(P, smem, resident, fp, st);
+    return launch_fit_t<ElemF32, 4, 32, 2>(P, smem, resident, fp, st);
 }
 
 // Rows of X to fetch with the evict-last hint.  Default: none for the narrow-row kernels (measured: any kept part slows
@@ -394,17 +412,46 @@ int64_t keep_rows_for(const lr_ctx* ctx, int variant, int32_t n, bool bf16 = fal
     return bytes / (int64_t(n) * (bf16 ? 2 : 4));
 }
 
-// Which form a multi-iteration fit on narrow rows takes.  Measured on B200 (ms per iteration, persistent launch against
-// two dependent-launched kernels): fp32 4M x 256 0.5759 / 0.5823, 16M x 64 0.594 / 0.608, 500k x 256 0.0832 / 0.0858,
-// 125k x 256 (128 MB) 0.0265 / 0.0271, 32k x 256 (32 MB) 0.0167 / 0.0153, 1k x 256 0.0092 / 0.0063; bfloat16 4M x 256
-// 0.3259 / 0.3163, 125k x 256 0.0247 / 0.0219.  The persistent kernel wins where the pass is bound by HBM and long enough
-// for the stages filled during its iteration boundary to matter: fp32 matrices from about half the L2 upwards.
-constexpr int64_t kPersistentMinBytes = int64_t(64) << 20;
+// Which form a multi-iteration fit on narrow rows takes.  Measured on B200 (us per iteration, persistent launch against
+// two dependent-launched kernels): fp32 300 x 256 4.1 / 5.3, 1k x 256 4.7 / 6.1, 3k x 32 3.6 / 4.5, 10k x 32 4.6 / 4.7,
+// 100k x 64 (26 MB, resident in shared memory) 6.7 / 11.5, 28k x 256 (29 MB, resident) 10.5 / 14.5, 32k x 256 12.2 / 15.0,
+// 250k x 64 11.9 / 16.1, 125k x 256 24.7 / 26.9, 1M x 100 64.3 / 68.0, 4M x 256 577.9 / 584.4; bfloat16 4M x 256
+// 328.5 / 328.6, 16M x 64 323.8 / 337.3.  With one grid barrier per iteration and the reduction done by every CTA for
+// itself the persistent kernel is at least as fast everywhere, so it is the default wherever the shape allows it.
 bool want_persistent(const lr_ctx* ctx, const lr_plan& P, bool bf16, int64_t m, int32_t n, int64_t iters) {
+    (void)bf16; (void)m; (void)n;
     if (P.variant != 0 || P.threads != kNW * 32 || !ctx->coop || ctx->prof || ctx->persistent_mode == 0) return false;
-    if (2 * iters * P.grid >= (int64_t(1) << 32)) return false;       // the grid-barrier counter is 32 bits
-    if (ctx->persistent_mode > 0) return true;
-    return !bf16 && m * n * 4 >= kPersistentMinBytes;
+    if (iters * P.grid >= (int64_t(1) << 32)) return false;           // the grid-barrier counter is 32 bits
+    return true;
+}
+
+// Enqueues the persistent kernel for a whole fit (fixed count, or with the stopping rule when `tol` is given).
+// Returns cudaErrorCooperativeLaunchTooLarge when the CTAs cannot all be resident (the caller then iterates with two
+// kernels), any other error as it comes.
+struct PersistentTol { TolState* state; double eps; float* gnorm_hist; };
+cudaError_t launch_persistent_fit(lr_ctx* ctx, const lr_plan& P, bool bf16, const void* d_X, const float* d_y, int64_t m,
+                                  int32_t n, float lr, int32_t iters, float* d_w, float* d_b, float* d_loss_hist,
+                                  const PersistentTol* tol, cudaStream_t st) {
+    const int64_t stage_stride = (int64_t(P.rows_per_batch) * n * (bf16 ? 2 : 4) + 127) & ~int64_t(127);
+    const int64_t room = kMaxDynamicSmem - kHeaderBytes - kFitTailBytes;
+    const int64_t B = (m + P.rows_per_batch - 1) / P.rows_per_batch;
+    const int64_t slots = (B + kNW - 1) / kNW;
+    const int64_t per_warp = (slots + P.grid - 1) / P.grid;                    // most batches any warp handles per iteration
+    const int depth = int(std::max<int64_t>(1, std::min<int64_t>({int64_t(kMaxDepth), room / (kNW * stage_stride), per_warp})));
+    FitParams fp{};
+    fp.X = d_X; fp.y = d_y; fp.m = m; fp.n = n; fp.w = d_w; fp.b = d_b; fp.partial = ctx->d_partial;
+    fp.loss_hist = d_loss_hist; fp.status = ctx->d_status; fp.gbar = ctx->d_gbar; fp.depth = depth;
+    const bool resident = per_warp <= depth;       // every warp's share of X fits its stages: filled once, kept for the fit
+    fp.num_batches = B;
+    fp.iters = iters; fp.lr = double(lr); fp.inv_m = 1.0 / double(m);
+    fp.keep_rows = keep_rows_for(ctx, 0, n, bf16);
+    if (tol) { fp.tol = tol->state; fp.eps = tol->eps; fp.gnorm_hist = tol->gnorm_hist; }
+    cudaError_t e = cudaMemsetAsync(ctx->d_gbar, 0, 2 * sizeof(unsigned int), st);   // barrier counter and abort flag
+    if (e != cudaSuccess) return e;
+    const int smem = int(kHeaderBytes + int64_t(kNW) * depth * stage_stride + kFitTailBytes);
+    e = launch_fit(P, smem, resident, fp, st, bf16);
+    if (e == cudaSuccess) ctx->launches += 1;
+    return e;
 }
 
 struct Pass {
@@ -547,11 +594,12 @@ int lr_create(lr_ctx** out, int32_t device, int32_t n_max) {
     if (e == cudaSuccess) e = cudaMemset(c->d_tol, 0, sizeof(TolState));
     if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&c->d_gbuf), (size_t(n_max) + 1) * sizeof(double));
     if (e == cudaSuccess) e = cudaMallocHost(reinterpret_cast<void**>(&c->h_tol), sizeof(TolState));
+    if (e == cudaSuccess) e = cudaMallocHost(reinterpret_cast<void**>(&c->h_words), 4 * sizeof(int));
     if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&c->d_vel), (size_t(n_max) + 1) * sizeof(float));
     if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&c->d_oscr), (size_t(n_max) + 2) * sizeof(double));
     if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&c->d_oticket), sizeof(unsigned int));
     if (e == cudaSuccess) e = cudaMemset(c->d_oticket, 0, sizeof(unsigned int));
-    if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&c->d_gbar), sizeof(unsigned int));
+    if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&c->d_gbar), 2 * sizeof(unsigned int));
     if (e == cudaSuccess) {
         int l2 = 0;
         e = cudaDeviceGetAttribute(&l2, cudaDevAttrL2CacheSize, device);
@@ -570,6 +618,7 @@ int lr_create(lr_ctx** out, int32_t device, int32_t n_max) {
         if (c->d_tol) cudaFree(c->d_tol);
         if (c->d_gbuf) cudaFree(c->d_gbuf);
         if (c->h_tol) cudaFreeHost(c->h_tol);
+        if (c->h_words) cudaFreeHost(c->h_words);
         if (c->d_vel) cudaFree(c->d_vel);
         if (c->d_oscr) cudaFree(c->d_oscr);
         if (c->d_oticket) cudaFree(c->d_oticket);
@@ -593,6 +642,7 @@ int lr_destroy(lr_ctx* ctx) {
         cudaFree(ctx->d_tol);
         cudaFree(ctx->d_gbuf);
         if (ctx->h_tol) cudaFreeHost(ctx->h_tol);
+        if (ctx->h_words) cudaFreeHost(ctx->h_words);
         cudaFree(ctx->d_vel);
         cudaFree(ctx->d_oscr);
         cudaFree(ctx->d_oticket);
@@ -694,22 +744,8 @@ int fit_impl(lr_ctx* ctx, const void* d_X, bool bf16, const float* d_y, int64_t 
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     // Narrow rows, several iterations: one cooperative launch runs the whole fit (same bits as the loop below).
     if (iters >= 2 && want_persistent(ctx, P, bf16, m, n, iters)) {
-        const int64_t stage_stride = (int64_t(P.rows_per_batch) * n * (bf16 ? 2 : 4) + 127) & ~int64_t(127);
-        const int64_t room = kMaxDynamicSmem - kHeaderBytes - kFitTailBytes;
-        const int depth = int(std::max<int64_t>(1, std::min<int64_t>(P.stages, room / (kNW * stage_stride))));
-        FitParams fp{};
-        fp.X = d_X; fp.y = d_y; fp.m = m; fp.n = n; fp.w = d_w; fp.b = d_b; fp.partial = ctx->d_partial;
-        fp.loss_hist = d_loss_hist; fp.status = ctx->d_status; fp.gbar = ctx->d_gbar; fp.depth = depth;
-        fp.num_batches = (m + P.rows_per_batch - 1) / P.rows_per_batch;
-        fp.iters = iters; fp.lr = double(lr); fp.inv_m = 1.0 / double(m);
-        fp.keep_rows = keep_rows_for(ctx, 0, n, bf16);
-        LR_CK(ctx, cudaMemsetAsync(ctx->d_gbar, 0, sizeof(unsigned int), st));
-        const int smem = int(kHeaderBytes + int64_t(kNW) * depth * stage_stride + kFitTailBytes);
-        const cudaError_t le = launch_fit(P, smem, fp, st, bf16);
-        if (le == cudaSuccess) {
-            ctx->launches += 1;
-            return LR_OK;
-        }
+        const cudaError_t le = launch_persistent_fit(ctx, P, bf16, d_X, d_y, m, n, lr, iters, d_w, d_b, d_loss_hist, nullptr, st);
+        if (le == cudaSuccess) return LR_OK;
         if (le != cudaErrorCooperativeLaunchTooLarge) { ctx->last_cuda = int(le); return LR_ERR_CUDA; }
         cudaGetLastError();                        // the CTAs cannot all be resident here: use the two-kernel form below
     }
@@ -790,28 +826,19 @@ int fit_tol_impl(lr_ctx* ctx, const void* d_X, bool bf16, const float* d_y, int6
     if (!g.ok) return LR_ERR_CUDA;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     LR_CK(ctx, cudaMemsetAsync(ctx->d_tol, 0, sizeof(TolState), st));
+    // the status word before this call's kernels, so that a give-up during the call can be told from an older, unread one
+    LR_CK(ctx, cudaMemcpyAsync(&ctx->h_words[0], ctx->d_status, sizeof(int), cudaMemcpyDeviceToHost, st));
     // Narrow rows: one persistent launch that leaves its loop on the device as soon as the norm is small enough.
     if (want_persistent(ctx, P, bf16, m, n, max_iters)) {
-        const int64_t stage_stride = (int64_t(P.rows_per_batch) * n * (bf16 ? 2 : 4) + 127) & ~int64_t(127);
-        const int64_t room = kMaxDynamicSmem - kHeaderBytes - kFitTailBytes;
-        const int depth = int(std::max<int64_t>(1, std::min<int64_t>(P.stages, room / (kNW * stage_stride))));
-        FitParams fp{};
-        fp.X = d_X; fp.y = d_y; fp.m = m; fp.n = n; fp.w = d_w; fp.b = d_b; fp.partial = ctx->d_partial;
-        fp.loss_hist = d_loss_hist; fp.status = ctx->d_status; fp.gbar = ctx->d_gbar; fp.depth = depth;
-        fp.num_batches = (m + P.rows_per_batch - 1) / P.rows_per_batch;
-        fp.iters = max_iters; fp.lr = double(lr); fp.inv_m = 1.0 / double(m);
-        fp.keep_rows = keep_rows_for(ctx, 0, n, bf16);
-        fp.tol = ctx->d_tol; fp.gbuf = ctx->d_gbuf; fp.eps = double(eps); fp.gnorm_hist = d_gnorm_hist;
-        LR_CK(ctx, cudaMemsetAsync(ctx->d_gbar, 0, sizeof(unsigned int), st));
-        const int smem = int(kHeaderBytes + int64_t(kNW) * depth * stage_stride + kFitTailBytes);
-        const cudaError_t le = launch_fit(P, smem, fp, st, bf16);
+        const PersistentTol pt{ctx->d_tol, double(eps), d_gnorm_hist};
+        const cudaError_t le = launch_persistent_fit(ctx, P, bf16, d_X, d_y, m, n, lr, max_iters, d_w, d_b, d_loss_hist, &pt, st);
         if (le == cudaSuccess) {
-            ctx->launches += 1;
             LR_CK(ctx, cudaMemcpyAsync(ctx->h_tol, ctx->d_tol, sizeof(TolState), cudaMemcpyDeviceToHost, st));
+            LR_CK(ctx, cudaMemcpyAsync(&ctx->h_words[2], ctx->d_gbar + 1, sizeof(int), cudaMemcpyDeviceToHost, st));
             LR_CK(ctx, cudaStreamSynchronize(st));
             *iters_done = ctx->h_tol->iters_done;
             *grad_norm = static_cast<float>(ctx->h_tol->grad_norm);
-            return LR_OK;
+            return ctx->h_words[2] != 0 ? LR_ERR_TIMEOUT : LR_OK;     // the launch's own abort flag: a bounded wait expired
         }
         if (le != cudaErrorCooperativeLaunchTooLarge) { ctx->last_cuda = int(le); return LR_ERR_CUDA; }
         cudaGetLastError();
@@ -832,7 +859,13 @@ int fit_tol_impl(lr_ctx* ctx, const void* d_X, bool bf16, const float* d_y, int6
             if (rc != LR_OK) return rc;
         }
         LR_CK(ctx, cudaMemcpyAsync(ctx->h_tol, ctx->d_tol, sizeof(TolState), cudaMemcpyDeviceToHost, st));
+        LR_CK(ctx, cudaMemcpyAsync(&ctx->h_words[1], ctx->d_status, sizeof(int), cudaMemcpyDeviceToHost, st));
         LR_CK(ctx, cudaStreamSynchronize(st));
+        if (ctx->h_words[1] != 0 && ctx->h_words[0] == 0) {           // a bounded wait expired in one of this call's kernels
+            *iters_done = ctx->h_tol->iters_done;
+            *grad_norm = static_cast<float>(ctx->h_tol->grad_norm);
+            return LR_ERR_TIMEOUT;
+        }
         if (ctx->h_tol->stop) break;
     }
     *iters_done = ctx->h_tol->iters_done;
@@ -1113,7 +1146,7 @@ const char* lr_status_string(int code) {
         case LR_OK: return "ok";
         case LR_ERR_NULL: return "a required pointer is NULL";
         case LR_ERR_SHAPE: return "shape out of range (m, n, iters) or larger than the context allows";
-        case LR_ERR_ALIGNMENT: return "a float pointer is not 4-byte aligned";
+        case LR_ERR_ALIGNMENT: return "a pointer is not aligned to its element size (4 bytes for float, 2 for bfloat16, 8 for double)";
         case LR_ERR_VALUE: return "value out of range (thr must be in (0,1), lr finite)";
         case LR_ERR_CUDA: return "a CUDA runtime call failed";
         case LR_ERR_TIMEOUT: return "a bounded device-side wait expired";
@@ -1181,39 +1214,24 @@ extern "C" int lr_loss_grad_noalloc(int32_t device, const float* d_X, const floa
     NoAllocDevice* dev = nullptr;
     int rc = noalloc_setup(device, &dev);
     if (rc != LR_OK) return rc;
+    // n <= LR_NOALLOC_MAX_N, so the plan is always one of the two narrow-row staged kernels (16-byte groups, or single
+    // elements for odd lengths and 4-byte-aligned matrices), whose grid never exceeds the SM count given here
     lr_plan P;
-    rc = make_plan(m, n, aligned(d_X, 16), dev->sm_count, &P);
+    rc = make_plan(m, n, aligned(d_X, 16), std::min(dev->sm_count, kNoAllocMaxGrid), &P);
     if (rc != LR_OK) return rc;
-    if (P.grid > kNoAllocMaxGrid) P.grid = kNoAllocMaxGrid;            // only the unstaged kernel asks for more; it strides over its chunks
+    if ((P.variant != 0 && P.variant != 3) || P.grid > kNoAllocMaxGrid) return LR_ERR_SHAPE;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     double* partial = dev->scratch;
     int* status = d_status ? d_status : reinterpret_cast<int*>(dev->scratch + size_t(kNoAllocMaxGrid) * kNoAllocRowDoubles);
     // the array keeps whatever the previous call left: the status word must start at zero (the partial rows are
     // fully rewritten by the CTAs that the reduction reads)
     if (cudaMemsetAsync(status, 0, sizeof(int), st) != cudaSuccess) return LR_ERR_CUDA;
-    cudaError_t e;
-    if (P.variant == 0 || P.variant == 3) {
-        StreamParams sp{};
-        sp.X = d_X; sp.y = d_y; sp.m = m; sp.n = n; sp.w = d_w; sp.b = d_b;
-        sp.partial = partial; sp.labels = nullptr; sp.cut = 0.f; sp.status = status;
-        sp.depth = P.stages;
-        sp.num_batches = (m + P.rows_per_batch - 1) / P.rows_per_batch;
-        e = launch_rows<false>(P, sp, st);
-    } else if (P.variant == 1) {
-        SplitParams sp{};
-        sp.y = d_y; sp.m = m; sp.n = n; sp.w = d_w; sp.b = d_b;
-        sp.partial = partial; sp.labels = nullptr; sp.cut = 0.f; sp.status = status;
-        sp.depth = P.stages;
-        sp.cw = (n / 4 + P.threads / 32 - 1) / (P.threads / 32);
-        sp.x_per_group = split_words64(false, sp.cw) ? 2 : 4;
-        sp.num_batches = (m + P.rows_per_batch - 1) / P.rows_per_batch;
-        e = launch_split<false>(P, d_X, sp, st);
-    } else {
-        GenericParams gp{};
-        gp.X = d_X; gp.y = d_y; gp.m = m; gp.n = n; gp.w = d_w; gp.b = d_b;
-        gp.partial = partial; gp.labels = nullptr; gp.cut = 0.f;
-        e = launch_kernel(k_generic<ElemF32, false>, dim3(P.grid), dim3(P.threads), 0, st, false, gp);
-    }
+    StreamParams sp{};
+    sp.X = d_X; sp.y = d_y; sp.m = m; sp.n = n; sp.w = d_w; sp.b = d_b;
+    sp.partial = partial; sp.labels = nullptr; sp.cut = 0.f; sp.status = status;
+    sp.depth = P.stages;
+    sp.num_batches = (m + P.rows_per_batch - 1) / P.rows_per_batch;
+    const cudaError_t e = launch_rows<false>(P, sp, st);
     if (e != cudaSuccess) return LR_ERR_CUDA;
     ReduceParams rp{};
     rp.partial = partial; rp.G = P.grid; rp.n = n; rp.inv_m = 1.0 / double(m); rp.lr = 0.0; rp.update = 0;

@@ -178,6 +178,15 @@ __device__ __forceinline__ void logistic_terms(float z, float y, float& err, flo
     loss = fmaxf(z, 0.0f) + log1pf(t) - y * z;
 }
 
+// Where a lane fetches its slice of w from: global memory through L2 (the kernel before this one may just have written
+// it), or the CTA's own shared-memory copy (the persistent kernel keeps the current parameters there).
+enum class WSource { GlobalL2, Shared };
+template <WSource S>
+__device__ __forceinline__ float load_param(const float* p) {
+    if constexpr (S == WSource::GlobalL2) return __ldcg(p);
+    else return *p;
+}
+
 // ---- per-lane arithmetic on 16-byte groups of X ----
 // A lane owns NV groups of a row.  Lane<NV> keeps that lane's slice of w and its fp32 gradient accumulators in the form
 // the storage type's arithmetic wants, and offers: load_w, zero, dot (this lane's part of x.w for one row), accumulate
@@ -207,7 +216,8 @@ struct LaneF32 {
     static constexpr int EPG = 4;
     uint64_t wv[NV][2];
     uint64_t acc[NV][2];
-    __device__ __forceinline__ void load_w(const float* w, int first_group, int group_stride, int group_limit, bool through_l2) {
+    template <WSource S>
+    __device__ __forceinline__ void load_w(const float* w, int first_group, int group_stride, int group_limit) {
 #pragma unroll
         for (int k = 0; k < NV; ++k) {
             const int idx = first_group + k * group_stride;
@@ -215,8 +225,8 @@ struct LaneF32 {
             for (int j = 0; j < 2; ++j) {
                 float lo = 0.f, hi = 0.f;
                 if (idx < group_limit) {
-                    lo = through_l2 ? __ldcg(w + 4 * idx + 2 * j) : __ldg(w + 4 * idx + 2 * j);
-                    hi = through_l2 ? __ldcg(w + 4 * idx + 2 * j + 1) : __ldg(w + 4 * idx + 2 * j + 1);
+                    lo = load_param<S>(w + 4 * idx + 2 * j);
+                    hi = load_param<S>(w + 4 * idx + 2 * j + 1);
                 }
                 wv[k][j] = f32x2_pack(lo, hi);
             }
@@ -276,7 +286,8 @@ struct LaneBF16 {
     static __device__ __forceinline__ uint64_t widen(uint32_t word) {
         return f32x2_pack(__uint_as_float(word << 16), __uint_as_float(word & 0xffff0000u));
     }
-    __device__ __forceinline__ void load_w(const float* w, int first_group, int group_stride, int group_limit, bool through_l2) {
+    template <WSource S>
+    __device__ __forceinline__ void load_w(const float* w, int first_group, int group_stride, int group_limit) {
 #pragma unroll
         for (int k = 0; k < NV; ++k) {
             const int idx = first_group + k * group_stride;
@@ -284,8 +295,8 @@ struct LaneBF16 {
             for (int j = 0; j < 4; ++j) {
                 float lo = 0.f, hi = 0.f;
                 if (idx < group_limit) {
-                    lo = through_l2 ? __ldcg(w + 8 * idx + 2 * j) : __ldg(w + 8 * idx + 2 * j);
-                    hi = through_l2 ? __ldcg(w + 8 * idx + 2 * j + 1) : __ldg(w + 8 * idx + 2 * j + 1);
+                    lo = load_param<S>(w + 8 * idx + 2 * j);
+                    hi = load_param<S>(w + 8 * idx + 2 * j + 1);
                 }
                 wv[k][j] = f32x2_pack(lo, hi);
             }
@@ -345,11 +356,12 @@ struct LaneAny {
     static constexpr int EPG = 1;
     float wv[NV];
     float acc[NV];
-    __device__ __forceinline__ void load_w(const float* w, int first_group, int group_stride, int group_limit, bool through_l2) {
+    template <WSource S>
+    __device__ __forceinline__ void load_w(const float* w, int first_group, int group_stride, int group_limit) {
 #pragma unroll
         for (int k = 0; k < NV; ++k) {
             const int idx = first_group + k * group_stride;
-            wv[k] = idx < group_limit ? (through_l2 ? __ldcg(w + idx) : __ldg(w + idx)) : 0.f;
+            wv[k] = idx < group_limit ? load_param<S>(w + idx) : 0.f;
         }
     }
     __device__ __forceinline__ void zero() {

@@ -2,21 +2,31 @@
 // cooperative launch (one CTA per SM, co-resident), instead of two launches per iteration.
 //
 // Per iteration every CTA runs the same per-warp streaming pass as k_stream_rows (same static batch map, same
-// arithmetic, same summation orders), writes its fp64 partial row, and meets the other CTAs at a grid barrier; the
-// columns of the reduction + update (the arithmetic of k_reduce_update, slice for slice) are then spread over all
-// warps of all CTAs, and a second grid barrier publishes the new parameters.  Results are bit-identical to the two-kernel path.
+// arithmetic, same summation orders), writes its fp64 partial row, and meets the other CTAs at ONE grid barrier.  After
+// it every CTA adds up all partial rows for itself -- the arithmetic of k_reduce_update, slice for slice, so every CTA
+// gets the same bits -- and updates its own shared-memory copy of the parameters: there is no second barrier and no
+// reload of the parameters through global memory.  The partial rows are double-buffered by iteration parity, so a CTA
+// that is already writing the rows of iteration t+1 cannot disturb one that still reads those of iteration t (it
+// cannot get to iteration t+2 before everybody has passed the barrier of t+1).  CTA 0 writes the loss history and, at
+// the end, the parameters.  Results are bit-identical to the two-kernel path.
 //
 // What the single launch buys: no launch gaps, and the HBM stream never drains -- X does not depend on w, so each warp
 // keeps re-arming its stages straight across the iteration boundary (the first batches of iteration t+1 are in flight
 // while the CTAs reduce iteration t).  This matters for short passes (a 400 MB pass lasts ~60 us, of which launch,
 // ramp-up and tail were ~20 %) and most for L2-resident problems.
 //
+// Resident form: when every warp's share of X fits its stages (a problem of up to ~28 MB on 148 SMs), the stages are
+// filled once and kept for the whole fit; an iteration is then arithmetic on shared memory plus the boundary, with no
+// copy, no re-arming and no mbarrier wait after the first pass.
+//
 // With a tolerance (lr_fit_tol) the kernel also forms ||grad||_2 after every update and all CTAs leave the loop together
 // once it is <= eps: the stopping rule of Algorithm 7 with no host round trip and no wasted launch.
 //
 // Grid barrier: a monotonic counter in global memory; thread 0 of each CTA adds one and spins (bounded, 2 s) until the
-// counter reaches grid * k.  On expiry, or when another CTA has raised the status word, the CTA stops iterating, waits
-// (bounded) for its own copies in flight and retires with LR_ERR_TIMEOUT in the status word.
+// counter reaches grid * k.  A second word next to the counter is the run's abort flag: a CTA whose wait expires (here
+// or on a stage) raises it, every other CTA sees it in its own wait, and all of them stop iterating, wait (bounded) for
+// their own copies in flight and retire with LR_ERR_TIMEOUT in the context's status word.  Both words are cleared by the
+// host before every launch, so a status left unread by an earlier call cannot end this one.
 #pragma once
 #include "lrgd_common.cuh"
 #include "lrgd_reduce.cuh"
@@ -24,12 +34,22 @@
 
 namespace lrgd {
 
-constexpr int kFitCombineCols = 64;            // columns combined per pass through the CTA's combine buffer
+constexpr int kFitCombineCols = 128;           // columns combined per pass through the CTA's combine buffer
 #ifndef LRGD_FIT_L2PF
 #define LRGD_FIT_L2PF 4
 #endif
 constexpr int kFitL2Prefetch = LRGD_FIT_L2PF;   // batches per warp pulled into L2 ahead of the next iteration (beyond the staged ones)
-constexpr int kFitTailBytes = 9216;            // combine buffer / reduction slices, after the stages
+constexpr int kFitMaxCols = 512;               // widest row the persistent kernel takes
+constexpr int kFitWarps = 16;
+// after the stages: combine buffer [warps][kFitCombineCols] fp64, sum err / sum loss per warp, the CTA's copy of the
+// parameters (w[n], b) in fp32, and the reduced sums / gradient entries [n+2] in fp64
+constexpr int kFitRedBytes = kFitWarps * kFitCombineCols * 8 + 2 * kFitWarps * 8;
+constexpr int kFitParamBytes = (kFitMaxCols + 4) * 4;
+constexpr int kFitSumBytes = (kFitMaxCols + 2) * 8;
+constexpr int kFitTailBytes = (kFitRedBytes + kFitParamBytes + kFitSumBytes + 127) / 128 * 128;
+constexpr int kFitRowChunk = 5;                // partial rows of one slice a thread has in flight (grids of up to 160 CTAs: the whole slice)
+constexpr int kFitChunkPairs = 32;             // column pairs per chunk of the reduction: one per lane, 512 contiguous bytes per row
+static_assert(2 * kFitWarps * 2 * kFitChunkPairs <= kFitWarps * kFitCombineCols, "the reduction reuses the combine buffer for two chunks");
 
 struct FitParams {
     const void* X;             // fp32 or bfloat16 [m][n], row-major
@@ -38,10 +58,10 @@ struct FitParams {
     int n;
     float* w;                  // [n] in/out
     float* b;                  // [1] in/out
-    double* partial;           // [grid][n+2]
+    double* partial;           // [2][grid][n+2]: the per-CTA sums of even and odd iterations
     float* loss_hist;          // nullable [iters]
-    int* status;               // device status word
-    unsigned int* gbar;        // grid-barrier counter, zero at launch
+    int* status;               // device status word (sticky report; never read here)
+    unsigned int* gbar;        // [0] grid-barrier counter, [1] abort flag of this launch; both zero at launch
     int depth;
     long long num_batches;
     long long keep_rows;       // rows [0, keep_rows) are fetched with an L2 evict-last hint, the rest evict-first
@@ -50,38 +70,139 @@ struct FitParams {
     double inv_m;
     // stopping rule (all null / zero for a fixed-count fit): as in k_reduce_update's tolerance mode
     TolState* tol;
-    double* gbuf;              // [n+1] gradient entries of the current iteration
     double eps;
     float* gnorm_hist;         // nullable [iters]
 };
 
-__device__ __forceinline__ unsigned int ld_acquire_u32(const unsigned int* p) {
+__device__ __forceinline__ unsigned int ld_relaxed_u32(const unsigned int* p) {
     unsigned int v;
-    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
     return v;
 }
 
-// All threads of the CTA call this.  Returns false if the barrier gave up (or the CTA had already given up).
-__device__ __forceinline__ bool grid_barrier(unsigned int* counter, unsigned int target, int* status, volatile int* cta_abort) {
+// All threads of the CTA call this.  Returns false if the barrier gave up (or the CTA, or another one, had already
+// given up).  Writes of the CTA before the call are visible to every CTA after it (release: fence, then the add; acquire:
+// relaxed polling loads, then a fence; the CTA's other threads are ordered through the two __syncthreads).
+__device__ __forceinline__ bool grid_barrier(unsigned int* gbar, unsigned int target, int* status, volatile int* cta_abort) {
     __syncthreads();
-    if (threadIdx.x == 0 && !*cta_abort) {
-        __threadfence();
-        atomicAdd(counter, 1u);
-        const unsigned long long t0 = global_timer_ns();
-        while (ld_acquire_u32(counter) < target) {
-            if (*reinterpret_cast<volatile int*>(status) != 0 || global_timer_ns() - t0 > kWaitLimitNs) {
-                atomicExch(status, kStatusTimeout);
-                *cta_abort = 1;
-                break;
+    if (threadIdx.x == 0) {
+        if (*cta_abort) {
+            atomicExch(gbar + 1, 1u);              // a stage wait of this CTA expired: tell the others
+        } else {
+            __threadfence();
+            atomicAdd(gbar, 1u);
+            if (ld_relaxed_u32(gbar) < target) {
+                const unsigned long long t0 = global_timer_ns();
+                for (;;) {
+                    bool there = false;
+#pragma unroll 1
+                    for (int i = 0; i < 64 && !there; ++i) there = ld_relaxed_u32(gbar) >= target;
+                    if (there) break;
+                    const bool told = ld_relaxed_u32(gbar + 1) != 0u;
+                    if (told || global_timer_ns() - t0 > kWaitLimitNs) {
+                        if (!told) atomicExch(gbar + 1, 1u);
+                        atomicExch(status, kStatusTimeout);
+                        *cta_abort = 1;
+                        break;
+                    }
+                }
             }
+            __threadfence();                       // acquire side: the other CTAs' rows are read after this
         }
-        __threadfence();
     }
     __syncthreads();
     return *cta_abort == 0;
 }
 
-template <class E, int NV, int LPR, int RB, int NW>
+// Adds up the G partial rows [G][stride] column by column into sums[stride] (shared memory); called by all threads of a
+// CTA, with the order of k_reduce_update so that the result has that kernel's bits: slice s = rows [s*per, (s+1)*per) in
+// index order, then the 32 slice sums in the fixed tree (s with s+16, then distance 8, 4, 2, 1).
+// Warp w owns slices w and w+16 -- the two that the first tree level adds -- and a lane owns one pair of adjacent columns,
+// so every load instruction of a warp reads 512 contiguous bytes of one partial row (all CTAs read the same rows at
+// the same time: scattered 16-byte reads cost L2 eight times the requests).  The 16 per-warp sums of a chunk of 64 columns
+// meet in `buf` and one thread per column finishes the tree.  Two chunks are in flight together.  Kept out of line: its
+// registers (twenty 16-byte loads in flight per thread) must not weigh on the streaming loop of the caller.
+template <int NW>
+__device__ __noinline__ void reduce_partial_rows(const double* pbuf, int G, int stride, double* buf, double* sums) {
+    static_assert(2 * NW == kRedSlices, "one warp per pair of slices");
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int per = (G + kRedSlices - 1) / kRedSlices;
+    const int npairs = stride / 2;
+    const int nchunks = (npairs + kFitChunkPairs - 1) / kFitChunkPairs;
+    const int lo0 = warp * per, hi0 = (warp + NW) * per;               // first rows of slices `warp` and `warp + 16`
+    const int lo1 = lo0 + per < G ? lo0 + per : G, hi1 = hi0 + per < G ? hi0 + per : G;
+    const double2 zero = make_double2(0.0, 0.0);
+    if (per == 1) {
+        // grids of up to 32 CTAs (small problems, where this call is most of the iteration): a slice is a single row, so one
+        // thread per column pair holds all of them at once -- one round trip to L2, no exchange through shared memory
+        for (int q = threadIdx.x; q < npairs; q += NW * 32) {
+            double2 a[NW];
+#pragma unroll
+            for (int i = 0; i < NW; ++i)
+                a[i] = i < G ? __ldcg(reinterpret_cast<const double2*>(pbuf + static_cast<size_t>(i) * stride) + q) : zero;
+            if (G > NW) {
+#pragma unroll
+                for (int i = 0; i < NW; ++i) {
+                    const double2 hi = i + NW < G ? __ldcg(reinterpret_cast<const double2*>(pbuf + static_cast<size_t>(i + NW) * stride) + q) : zero;
+                    a[i] = make_double2(a[i].x + hi.x, a[i].y + hi.y);
+                }
+            }
+#pragma unroll
+            for (int h = NW / 2; h >= 1; h >>= 1)
+#pragma unroll
+                for (int i = 0; i < h; ++i) a[i] = make_double2(a[i].x + a[i + h].x, a[i].y + a[i + h].y);
+            sums[2 * q] = a[0].x;
+            sums[2 * q + 1] = a[0].y;
+        }
+        __syncthreads();
+        return;
+    }
+    for (int c0 = 0; c0 < nchunks; c0 += 2) {
+        double2 slo[2] = {zero, zero}, shi[2] = {zero, zero};
+        for (int r0 = 0; r0 < per; r0 += kFitRowChunk) {
+            double2 vlo[2][kFitRowChunk], vhi[2][kFitRowChunk];
+#pragma unroll
+            for (int u = 0; u < 2; ++u) {
+                const int q = (c0 + u) * kFitChunkPairs + lane;
+                const bool live = q < npairs;
+#pragma unroll
+                for (int r = 0; r < kFitRowChunk; ++r) {
+                    const int gl = lo0 + r0 + r, gh = hi0 + r0 + r;
+                    vlo[u][r] = (live && gl < lo1) ? __ldcg(reinterpret_cast<const double2*>(pbuf + static_cast<size_t>(gl) * stride) + q) : zero;
+                    vhi[u][r] = (live && gh < hi1) ? __ldcg(reinterpret_cast<const double2*>(pbuf + static_cast<size_t>(gh) * stride) + q) : zero;
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < 2; ++u)
+#pragma unroll
+                for (int r = 0; r < kFitRowChunk; ++r) {               // (+0.0 where there is no row: changes nothing)
+                    slo[u].x += vlo[u][r].x; slo[u].y += vlo[u][r].y;
+                    shi[u].x += vhi[u][r].x; shi[u].y += vhi[u][r].y;
+                }
+        }
+#pragma unroll
+        for (int u = 0; u < 2; ++u)                                    // first tree level: slice w + slice w+16
+            reinterpret_cast<double2*>(buf)[(u * NW + warp) * kFitChunkPairs + lane] = make_double2(slo[u].x + shi[u].x, slo[u].y + shi[u].y);
+        __syncthreads();
+        if (threadIdx.x < 4 * kFitChunkPairs) {
+            const int u = threadIdx.x / (2 * kFitChunkPairs), c = threadIdx.x % (2 * kFitChunkPairs);
+            const int col = (c0 + u) * 2 * kFitChunkPairs + c;
+            if (col < stride) {
+                double v[NW];
+#pragma unroll
+                for (int i = 0; i < NW; ++i) v[i] = buf[(u * NW + i) * 2 * kFitChunkPairs + c];
+#pragma unroll
+                for (int h = NW / 2; h >= 1; h >>= 1)
+#pragma unroll
+                    for (int i = 0; i < h; ++i) v[i] = v[i] + v[i + h];
+                sums[col] = v[0];
+            }
+        }
+        __syncthreads();
+    }
+}
+
+template <class E, int NV, int LPR, int RB, int NW, bool RESIDENT>
 __global__ void __launch_bounds__(NW * 32, 1) k_fit_rows(const FitParams p) {
     constexpr int EPG = E::EPG;
     constexpr int RPW = 32 / LPR;
@@ -93,7 +214,8 @@ __global__ void __launch_bounds__(NW * 32, 1) k_fit_rows(const FitParams p) {
     static_assert(SHIFT >= 0, "rows per batch slot must not exceed lanes per row");
     static_assert(E::EPG > 1, "rows of 16-byte groups only");
     static_assert(kRedSlices == 32, "one lane per reduction slice of k_reduce_update");
-    static_assert(NW * kFitCombineCols * 8 + 2 * NW * 8 <= kFitTailBytes, "tail too small");
+    static_assert(NW == kFitWarps, "tail layout is sized for this many warps");
+    static_assert(NV * LPR * EPG <= kFitMaxCols, "row wider than the parameter copy");
 
     extern __shared__ __align__(128) unsigned char smem[];
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem);
@@ -103,28 +225,37 @@ __global__ void __launch_bounds__(NW * 32, 1) k_fit_rows(const FitParams p) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int D = p.depth;
     const int n = p.n, n4 = n / EPG;                   // n4 = 16-byte groups per row
-    const int G = gridDim.x;
+    const int G = gridDim.x, cta = blockIdx.x;
+    const int stride = n + 2;                          // doubles per partial row (even: n is a multiple of four)
     const uint32_t row_bytes = static_cast<uint32_t>(n) * E::BYTES;
     const uint32_t stage_stride = (static_cast<uint32_t>(RPB) * row_bytes + 127u) & ~127u;
     unsigned char* my_stages = data + static_cast<size_t>(warp) * D * stage_stride;
-    unsigned char* tail = data + static_cast<size_t>(NW) * D * stage_stride;      // combine buffer
+    unsigned char* tail = data + static_cast<size_t>(NW) * D * stage_stride;
+    double* red = reinterpret_cast<double*>(tail);                     // [NW][kFitCombineCols]
+    double* red_e = red + NW * kFitCombineCols;
+    double* red_l = red_e + NW;
+    float* w_s = reinterpret_cast<float*>(tail + kFitRedBytes);        // w[0..n), then b
+    double* sum_s = reinterpret_cast<double*>(tail + kFitRedBytes + kFitParamBytes);   // [n+2]
     uint64_t* my_bars = bars + warp * kMaxDepth;
 
     const long long B = p.num_batches;
     const long long Bw = B > warp ? (B - warp + NW - 1) / NW : 0;
-    const int cnt = Bw > blockIdx.x ? static_cast<int>((Bw - blockIdx.x + G - 1) / G) : 0;    // batches of this warp per iteration
-    const int fill_iters = cnt > 0 ? p.iters : 0;  // the fit is cnt * fill_iters stage fills for this warp, iteration-major
+    const int cnt = Bw > cta ? static_cast<int>((Bw - cta + G - 1) / G) : 0;    // batches of this warp per iteration
+    constexpr bool resident = RESIDENT;            // cnt <= D for every warp of the grid (the host checked)
+    const int fill_iters = cnt > 0 ? (resident ? 1 : p.iters) : 0;   // the fit is cnt * fill_iters stage fills for this warp, iteration-major
 
     if (threadIdx.x == 0) *abort_flag = 0;
     if (lane == 0) {
         for (int d = 0; d < D; ++d) mbar_init(&my_bars[d], 1);
         fence_mbar_init();
     }
+    // the CTA's own copy of the parameters
+    for (int c = threadIdx.x; c <= n; c += NW * 32) w_s[c] = c < n ? __ldcg(p.w + c) : __ldcg(p.b);
     __syncthreads();
 
     const uint64_t pol_stream = l2_policy_evict_first(), pol_keep = l2_policy_evict_last();
     const long long stride_rows = static_cast<long long>(G) * NW * RPB;
-    const long long first_row = (static_cast<long long>(blockIdx.x) * NW + warp) * RPB;
+    const long long first_row = (static_cast<long long>(cta) * NW + warp) * RPB;
     auto issue = [&](long long r0, int d) {        // lane 0 only
         const long long left = p.m - r0;
         const uint32_t rows = left < RPB ? static_cast<uint32_t>(left) : RPB;
@@ -153,6 +284,8 @@ __global__ void __launch_bounds__(NW * 32, 1) k_fit_rows(const FitParams p) {
         next_fill();
         ++inflight;
     }
+    // y of this lane's row in the first batch: the same in every iteration
+    const float y_first = (cnt > 0 && first_row + myr < p.m) ? __ldg(p.y + first_row + myr) : 0.f;
     int d = 0;
     uint32_t phase = 0;
     unsigned int barrier_no = 0;
@@ -160,9 +293,9 @@ __global__ void __launch_bounds__(NW * 32, 1) k_fit_rows(const FitParams p) {
 
     for (int t = 0; t < p.iters && alive; ++t) {
         typename E::template Lane<NV> lm;          // this lane's slice of the current w and its fp32 accumulators
-        lm.load_w(p.w, sub, LPR, n4, true);
+        lm.template load_w<WSource::Shared>(w_s, sub, LPR, n4);
         lm.zero();
-        const float bval = __ldcg(p.b);
+        const float bval = w_s[n];
         double dacc[NV][EPG];
         float se = 0.f, sl = 0.f;
         double dse = 0.0, dsl = 0.0;
@@ -172,13 +305,15 @@ __global__ void __launch_bounds__(NW * 32, 1) k_fit_rows(const FitParams p) {
             for (int c = 0; c < EPG; ++c) dacc[k][c] = 0.0;
         int since_flush = 0;
         long long row0 = first_row;
-        float y_next = (cnt > 0 && row0 + myr < p.m) ? __ldg(p.y + row0 + myr) : 0.f;
-        bool warp_ok = true;
+        float y_next = y_first;
+        const bool waits = !resident || t == 0;    // a resident stage is complete once and for all after the first pass
 
         for (int i = 0; i < cnt; ++i) {
-            bool ok = mbar_wait_bounded(&my_bars[d], phase, abort_flag);
-            ok = __all_sync(FULL, ok);
-            if (!ok) { warp_ok = false; break; }
+            if (waits) {
+                bool ok = mbar_wait_bounded(&my_bars[d], phase, abort_flag);
+                ok = __all_sync(FULL, ok);
+                if (!ok) break;                    // the CTA's abort flag is up; handled at the barrier
+            }
 
             const long long left = p.m - row0;
             const int rows = left < RPB ? static_cast<int>(left) : RPB;
@@ -191,18 +326,23 @@ __global__ void __launch_bounds__(NW * 32, 1) k_fit_rows(const FitParams p) {
                 const long long rn = row0 + stride_rows + myr;
                 y_next = (i + 1 < cnt && rn < p.m) ? __ldg(p.y + rn) : 0.f;
             }
-            // re-arm the stage with the fill `depth` ahead in the fit-long sequence (possibly of the next iteration)
-            __syncwarp();
-            if (issue_t < fill_iters) {
-                if (lane == 0) {
-                    fence_proxy_async_smem();
-                    issue(issue_row, d);
-                }
-                next_fill();
+            if constexpr (resident) {
+                if (waits) --inflight;
+                if (++d == cnt) d = 0;             // stage i holds batch i in every iteration
             } else {
-                --inflight;
+                // re-arm the stage with the fill `depth` ahead in the fit-long sequence (possibly of the next iteration)
+                __syncwarp();
+                if (issue_t < fill_iters) {
+                    if (lane == 0) {
+                        fence_proxy_async_smem();
+                        issue(issue_row, d);
+                    }
+                    next_fill();
+                } else {
+                    --inflight;
+                }
+                if (++d == D) { d = 0; phase ^= 1u; }
             }
-            if (++d == D) { d = 0; phase ^= 1u; }
 
             const float z = batch_dot<E, NV, LPR, RB>(x, lm, lane) + bval;
             float e, L;
@@ -216,11 +356,10 @@ __global__ void __launch_bounds__(NW * 32, 1) k_fit_rows(const FitParams p) {
             }
             row0 += stride_rows;
         }
-        (void)warp_ok;                             // a failed wait has raised the CTA's abort flag; handled at the barrier
 
-        // The grid barriers, the reduction and the parameter reload below take longer than the staged batches of the next
-        // iteration last; keep HBM busy meanwhile by pulling this warp's following batches of that iteration into L2.
-        if (lane == 0 && t + 1 < p.iters) {
+        // The grid barrier and the reduction below take longer than the staged batches of the next iteration last; keep
+        // HBM busy meanwhile by pulling this warp's following batches of that iteration into L2.
+        if (!resident && lane == 0 && t + 1 < p.iters) {
 #pragma unroll
             for (int j = 0; j < kFitL2Prefetch; ++j) {
                 const int bi = D + j;
@@ -252,12 +391,8 @@ __global__ void __launch_bounds__(NW * 32, 1) k_fit_rows(const FitParams p) {
             dse += __shfl_xor_sync(FULL, dse, msk);
             dsl += __shfl_xor_sync(FULL, dsl, msk);
         }
-        double* red = reinterpret_cast<double*>(tail);                 // [NW][kFitCombineCols]
-        double* red_e = red + NW * kFitCombineCols;
-        double* red_l = red_e + NW;
-        double* out = p.partial + static_cast<size_t>(blockIdx.x) * (n + 2);
-        __syncthreads();                                               // previous use of the tail is over
-        if (lane == 0) { red_e[warp] = dse; red_l[warp] = dsl; }
+        double* out = p.partial + (static_cast<size_t>(t & 1) * G + cta) * stride;
+        if (lane == 0) { red_e[warp] = dse; red_l[warp] = dsl; }       // (the last reader of these was before the previous barrier)
         for (int c0 = 0; c0 < n; c0 += kFitCombineCols) {
 #pragma unroll
             for (int k2 = 0; k2 < NV; ++k2) {
@@ -287,44 +422,33 @@ __global__ void __launch_bounds__(NW * 32, 1) k_fit_rows(const FitParams p) {
         alive = grid_barrier(p.gbar, static_cast<unsigned int>(G) * barrier_no, p.status, abort_flag);
         if (!alive) break;
 
-        // ---- reduction + update: one warp per column, columns spread over all warps of all CTAs.  Lane s plays slice s of
-        // k_reduce_update (rows [s*per, (s+1)*per) in index order); lane 0 then adds the 32 slice sums in slice order ----
-        {
-            const int stride = n + 2;
-            const int per = (G + kRedSlices - 1) / kRedSlices;
-            const int g0 = lane * per;
-            const int g1 = g0 + per < G ? g0 + per : G;
-            for (int col = warp * G + blockIdx.x; col < stride; col += NW * G) {
-                double s = 0.0;
-                const double* src = p.partial + col;
-                for (int g = g0; g < g1; ++g) s += __ldcg(src + static_cast<size_t>(g) * stride);
-                double tsum = 0.0;
-#pragma unroll
-                for (int k = 0; k < kRedSlices; ++k) tsum += __shfl_sync(FULL, s, k);
-                if (lane == 0) {
-                    const double v = tsum * p.inv_m;
-                    if (col < n) p.w[col] = static_cast<float>(static_cast<double>(__ldcg(p.w + col)) - p.lr * v);
-                    else if (col == n) p.b[0] = static_cast<float>(static_cast<double>(__ldcg(p.b)) - p.lr * v);
-                    else if (p.loss_hist) p.loss_hist[t] = static_cast<float>(v);
-                    if (p.tol != nullptr && col <= n) p.gbuf[col] = v;
-                }
+        // ---- reduction, by every CTA for itself (see reduce_partial_rows) ----
+        reduce_partial_rows<NW>(p.partial + static_cast<size_t>(t & 1) * G * stride, G, stride, red, sum_s);
+
+        // ---- update (the arithmetic of k_reduce_update), every CTA on its own copy; CTA 0 keeps the history ----
+        for (int c = threadIdx.x; c < stride; c += NW * 32) {
+            const double v = sum_s[c] * p.inv_m;
+            if (c <= n) {
+                w_s[c] = static_cast<float>(static_cast<double>(w_s[c]) - p.lr * v);
+                sum_s[c] = v;                                           // gradient entry, for the norm below
+            } else if (cta == 0 && p.loss_hist) {
+                p.loss_hist[t] = static_cast<float>(v);
             }
         }
-        barrier_no += 1;
-        alive = grid_barrier(p.gbar, static_cast<unsigned int>(G) * barrier_no, p.status, abort_flag);
+        __syncthreads();
 
-        // ---- stopping rule (Algorithm 7): ||(grad_w, grad_b)||_2 of the update just applied, formed by every CTA in the
+        // ---- stopping rule (Algorithm 7): ||(grad_w, grad_b)||_2 of the update just applied, formed by every warp in the
         // same order as k_reduce_update's last block (lane-strided squares, xor tree), so all CTAs take the same decision ----
-        if (p.tol != nullptr && alive) {
+        if (p.tol != nullptr) {
             double q = 0.0;
             for (int c = lane; c <= n; c += 32) {
-                const double v = __ldcg(p.gbuf + c);
+                const double v = sum_s[c];
                 q += v * v;
             }
 #pragma unroll
             for (int msk = 16; msk >= 1; msk >>= 1) q += __shfl_xor_sync(FULL, q, msk);
             const double nrm = sqrt(q);
-            if (blockIdx.x == 0 && threadIdx.x == 0) {
+            if (cta == 0 && threadIdx.x == 0) {
                 p.tol->grad_norm = nrm;
                 p.tol->iters_done = t + 1;
                 if (p.gnorm_hist) p.gnorm_hist[t] = static_cast<float>(nrm);
@@ -334,11 +458,18 @@ __global__ void __launch_bounds__(NW * 32, 1) k_fit_rows(const FitParams p) {
         }
     }
 
+    if (alive && *abort_flag == 0) {
+        if (cta == 0)                              // every CTA holds the same parameters; one of them stores them
+            for (int c = threadIdx.x; c <= n; c += NW * 32) {
+                if (c < n) p.w[c] = w_s[c];
+                else p.b[0] = w_s[n];
+            }
+    } else if (lane == 0) {
+        atomicExch(p.status, kStatusTimeout);      // the parameters are left as they were at launch
+        atomicExch(p.gbar + 1, 1u);
+    }
     // Copies still in flight when the loop ends (a give-up, or an early stop with the next iteration already being
     // prefetched) must land before the CTA retires and its shared memory is handed to another CTA.
-    if (!alive || *abort_flag) {
-        if (lane == 0) atomicExch(p.status, kStatusTimeout);
-    }
     if (inflight > 0) {
         if (lane == 0) {
             for (int f = 0; f < inflight; ++f) {           // the oldest fill in flight sits in stage d, phase parity `phase`

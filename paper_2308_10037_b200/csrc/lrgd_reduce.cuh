@@ -3,7 +3,8 @@
 // (Algorithm 1's update; descent sign as in Algorithm 7).
 //
 // Block = 32 columns x kRedSlices slices.  Slice s sums partial rows [s*per, (s+1)*per) of its column in
-// index order in fp64; the slices are then added in slice order.  No atomics on data: bit-reproducible.
+// index order in fp64; the 32 slice sums are then added pairwise in a fixed tree (slice s with s+16, then
+// with s+8, s+4, s+2, s+1).  No atomics on data: bit-reproducible.
 //
 // Tolerance mode (Algorithm 7's stopping rule, built from Algorithm 4's norm): every block parks its fp64
 // gradient entries in `gbuf`; the block that finishes last (a ticket counter) adds their squares in index
@@ -16,6 +17,23 @@
 namespace lrgd {
 
 constexpr int kRedSlices = 32;           // 1024 threads: few dependent L2 reads per thread keeps this stage at ~2 us
+
+// The fixed tree in which the 32 slice sums of a column are added: v[s] + v[s+16] for s < 16, then the 16 results
+// pairwise at distance 8, and so on.  slice_tree_sum works on the 32 values held by one thread; slice_tree_sum_warp
+// on one value per lane (a butterfly of xor shuffles: every lane ends with the value slice_tree_sum returns, because
+// each step adds the same two numbers on both partners).  Depth five instead of a chain of 32 dependent additions.
+__device__ __forceinline__ double slice_tree_sum(double (&v)[kRedSlices]) {
+#pragma unroll
+    for (int h = kRedSlices / 2; h >= 1; h >>= 1)
+#pragma unroll
+        for (int i = 0; i < h; ++i) v[i] = v[i] + v[i + h];
+    return v[0];
+}
+__device__ __forceinline__ double slice_tree_sum_warp(double v) {
+#pragma unroll
+    for (int msk = kRedSlices / 2; msk >= 1; msk >>= 1) v = v + __shfl_xor_sync(0xffffffffu, v, msk);
+    return v;
+}
 
 struct TolState {             // device-resident, owned by the context
     int stop;                 // 1 once the tolerance has been met
@@ -69,9 +87,10 @@ __global__ void __launch_bounds__(32 * kRedSlices) k_reduce_update(const ReduceP
     sh[slice][threadIdx.x] = s;
     __syncthreads();
     if (slice == 0 && col < stride) {
-        double t = 0.0;
+        double sl[kRedSlices];
 #pragma unroll
-        for (int k = 0; k < kRedSlices; ++k) t += sh[k][threadIdx.x];
+        for (int k = 0; k < kRedSlices; ++k) sl[k] = sh[k][threadIdx.x];
+        const double t = slice_tree_sum(sl);
         if (p.raw_sums) {
             p.raw_sums[col] = t;
         } else {
@@ -164,10 +183,10 @@ __global__ void __launch_bounds__(32 * kRedSlices) k_reduce_opt(const OptParams 
     sh[slice][threadIdx.x] = s;
     __syncthreads();
     if (slice == 0 && col < stride) {
-        double t = 0.0;
+        double sl[kRedSlices];
 #pragma unroll
-        for (int k = 0; k < kRedSlices; ++k) t += sh[k][threadIdx.x];
-        const double mean = t * p.inv_m;
+        for (int k = 0; k < kRedSlices; ++k) sl[k] = sh[k][threadIdx.x];
+        const double mean = slice_tree_sum(sl) * p.inv_m;
         if (col <= p.n) {
             float* param = col < p.n ? p.w + col : p.b;
             const double old = static_cast<double>(*param);

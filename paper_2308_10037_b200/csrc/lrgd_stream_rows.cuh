@@ -239,7 +239,7 @@ __global__ void __launch_bounds__(NW * 32, 1) k_stream_rows(const StreamParams p
         __syncwarp();
         return;
     }
-    lm.load_w(p.w, sub, LPR, n4, true);            // through L2: the kernel before this one may just have written them
+    lm.template load_w<WSource::GlobalL2>(p.w, sub, LPR, n4);   // through L2: the kernel before this one may just have written them
     const float bval = __ldcg(p.b);
     const bool full_cols = n4 == NV * LPR;         // every lane's column groups exist
     const bool labels_word_aligned = PREDICT && (reinterpret_cast<uintptr_t>(p.labels) & 3u) == 0 && RPB % 4 == 0;

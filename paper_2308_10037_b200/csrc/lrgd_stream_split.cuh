@@ -136,7 +136,7 @@ __global__ void __launch_bounds__(NW * 32, 1) k_stream_split(const __grid_consta
         __syncwarp();
         return;
     }
-    lm.load_w(p.w, c0 + lane, 32, c0 + mycw, true);    // through L2: the kernel before this one may just have written them
+    lm.template load_w<WSource::GlobalL2>(p.w, c0 + lane, 32, c0 + mycw);    // through L2: the kernel before this one may just have written them
     const float bval = __ldcg(p.b);
 
     for (int i = 0; i < cnt; ++i) {

@@ -15,9 +15,30 @@ where the second term only matters at iterates whose gradient norm is below ~1e5
 iterations of the fast-converging workloads).  ``test_fp32_floor.py`` shows on the CPU that even an idealised fp32
 evaluation (float32 logits and sigmoid, exact float64 accumulation) misses the relative bar at such an iterate.
 """
+import json
+import os
+
 import numpy as np
 
+import oracle
+
 GRAD_TOL, LOSS_TOL, W_TOL, LABEL_AGREE = 1e-5, 1e-6, 1e-4, 0.9999
+
+
+def record(kind, **fields):
+    """Appends one JSON line with the achieved errors of a parity check to the file named by LRGD_PARITY_RECORD.
+
+    The GPU tests call this with what they measured (error, the bound that applied, which bound was binding), so that a
+    run leaves a table of achieved figures behind and not only a pass mark.  Without the variable nothing is written.
+    """
+    path = os.environ.get("LRGD_PARITY_RECORD")
+    if not path:
+        return
+    clean = {k: (float(v) if isinstance(v, (np.floating, float)) else int(v) if isinstance(v, (np.integer,)) else v)
+             for k, v in fields.items()}
+    os.makedirs(os.path.dirname(os.path.abspath(path)), exist_ok=True)
+    with open(path, "a") as f:
+        f.write(json.dumps({"kind": kind, **clean}) + "\n")
 
 
 def rel_l2(a, b):
@@ -41,8 +62,40 @@ def grad_noise_floor(X, fro=None):
     return 8.0 * 2.0 ** -24 * fro / X.shape[0]
 
 
-def assert_grad_close(got, ref, floor, what=""):
+def assert_grad_close(got, ref, floor, what="", floor_allowed=True):
+    """The gradient bar.  Returns (relative error, True if the absolute floor and not 1e-5 * ||g|| was the binding bound).
+
+    The floor can only be the binding bound where ||g_ref|| < 1e5 * floor (that is what max() means); with
+    floor_allowed=False the plain relative bar has to hold on its own and a converged iterate is a test failure.
+    """
     got, ref = np.asarray(got, dtype=np.float64).ravel(), np.asarray(ref, dtype=np.float64).ravel()
     err = float(np.linalg.norm(got - ref))
-    bound = max(GRAD_TOL * float(np.linalg.norm(ref)), floor)
-    assert err <= bound, (what, err, bound, float(np.linalg.norm(ref)))
+    norm = float(np.linalg.norm(ref))
+    plain = GRAD_TOL * norm
+    used_floor = err > plain
+    if used_floor:
+        assert floor_allowed, (what, "plain 1e-5 bar missed where no floor is allowed", err, plain)
+        assert norm < 1e5 * floor, (what, "floor used although the gradient is not small", norm, floor)
+    assert err <= max(plain, floor), (what, err, max(plain, floor), norm)
+    return err / max(norm, 1e-300), used_floor
+
+
+def allowed_drift(X, y, wl, ref, hist_ref):
+    """What a fit that meets the per-iteration gradient bar may still drift by, measured on the checker itself.
+
+    The gradient bar lets every update differ from the exact one by lr * 1e-5 * ||g||.  One such deviation is injected
+    into the checker at the first update (start point moved by that much, in two random directions and along the
+    all-ones direction, the dominant eigenvector of an uncentred design) and the checker is rerun in float64.  The
+    largest movement of its final parameters (relative L2) and of its loss history (absolute) is the scale below which
+    a free-running comparison says nothing about the kernels.  Returns (drift_w, drift_loss).
+    """
+    _, g, g0 = oracle.loss_grad(X, y, np.zeros(wl.n), 0.0)
+    eps = wl.lr * GRAD_TOL * float(np.linalg.norm(np.concatenate([g, [g0]])))
+    rng = np.random.default_rng(7)
+    drift_w = drift_l = 0.0
+    for d in (rng.standard_normal(wl.n + 1), rng.standard_normal(wl.n + 1), np.ones(wl.n + 1)):
+        d = d / np.linalg.norm(d) * eps
+        w_p, b_p, lh_p = oracle.fit(X, y, wl.lr, wl.iters, w0=d[:-1], b0=d[-1])
+        drift_w = max(drift_w, rel_l2(np.concatenate([w_p, [b_p]]), ref))
+        drift_l = max(drift_l, float(np.max(np.abs(lh_p - hist_ref))))
+    return drift_w, drift_l

@@ -15,7 +15,8 @@ from paper_2308_10037_b200 import api, datagen
 
 pytestmark = pytest.mark.gpu
 
-from _parity import GRAD_TOL, LABEL_AGREE, LOSS_TOL, W_TOL, assert_grad_close, grad_noise_floor, rel_l2
+from _parity import (GRAD_TOL, LABEL_AGREE, LOSS_TOL, W_TOL, allowed_drift, assert_grad_close, grad_noise_floor, record,
+                     rel_l2)
 
 
 @pytest.fixture(scope="module")
@@ -151,7 +152,9 @@ def test_teacher_forced_trajectory(ctx, name, m):
         dl, dg, dg0 = ctx.loss_grad(dX, dy, dev(w32), dev(np.array([b32])))
         assert abs(dl.item() - L) <= LOSS_TOL, (t, dl.item(), L)
         got = np.concatenate([dg.cpu().numpy(), dg0.cpu().numpy()])
-        assert_grad_close(got, np.concatenate([g, [g0]]), floor, (name, t))
+        rel, used_floor = assert_grad_close(got, np.concatenate([g, [g0]]), floor, (name, t), floor_allowed=name == "cfg2")
+        record("small_iterate", workload=wl.name, t=t, grad_rel_l2=rel, bound="floor" if used_floor else "1e-5*|g|",
+               loss_abs_err=abs(dl.item() - L))
 
 
 @pytest.mark.parametrize("name,m", SMALL_WORKLOADS)
@@ -162,15 +165,18 @@ def test_fit_matches_oracle(ctx, name, m):
     w, b, lh = api.lr_fit(dev(X), dev(y), wl.lr, wl.iters, return_history=True, ctx=ctx)
     got = np.concatenate([w.cpu().numpy(), b.cpu().numpy()])
     ref = np.concatenate([w_ref, [b_ref]])
+    w_rel = rel_l2(got, ref)
+    hist_err = float(np.max(np.abs(lh.cpu().numpy().astype(np.float64) - lh_ref)))
+    hist_bound = LOSS_TOL
     if name == "cfg4":
-        # lr = 0.05 is above 2/L for uncentred U[0,1) features: the iteration is not a contraction, so rounding
-        # differences are amplified; the checker's own fp32-rounded rerun sets the scale of what is attainable
-        w_r, b_r, _ = oracle.fit(X, y, wl.lr, wl.iters, round_to_fp32=True)
-        own = rel_l2(np.concatenate([w_r, [b_r]]), ref)
-        assert rel_l2(got, ref) <= max(W_TOL, 20 * own)
-    else:
-        assert rel_l2(got, ref) <= W_TOL
-        assert np.max(np.abs(lh.cpu().numpy().astype(np.float64) - lh_ref)) <= LOSS_TOL
+        # lr = 0.05 is above 2/L for uncentred U[0,1) features: the iteration is not a contraction and the loss swings
+        # between ~4 and ~8.  The final parameters still meet the plain bar; the loss history is held to the drift the
+        # checker itself shows under one tolerance-sized deviation, and to one fp32 spacing of the stored values
+        _, drift_l = allowed_drift(X, y, wl, ref, lh_ref)
+        hist_bound = max(LOSS_TOL, float(np.max(np.abs(lh_ref))) * 2.0 ** -23, drift_l)
+    record("small_fit", workload=wl.name, w_rel_l2=w_rel, loss_hist_max_abs_err=hist_err, loss_hist_bound=hist_bound)
+    assert w_rel <= W_TOL
+    assert hist_err <= hist_bound
 
 
 def test_fit_is_deterministic_and_resumable(ctx):
@@ -293,8 +299,12 @@ def test_argument_errors_with_a_live_context(ctx):
     assert ctx.launch_count() == n0 + 2
 
 
+# 148 SMs x 16 warps x 4 rows per batch x 3 stages = 28,416 rows of 256 columns is the largest problem of that shape whose
+# rows all stay in shared memory for the whole fit (the resident form of the persistent kernel); one more row and it streams
 @pytest.mark.parametrize("name,m,iters", [("cfg1", 10_000, 25), ("cfg2", 150_007, 12), ("cfg3", 120_001, 9), ("cfg5", 300_000, 7),
-                                           ("higgs_like", 200_003, 11), ("cfg1", 37, 5), ("cfg3", 9, 3)])
+                                           ("higgs_like", 200_003, 11), ("cfg1", 37, 5), ("cfg3", 9, 3), ("cfg3", 28_416, 6),
+                                           ("cfg3", 28_417, 6), ("cfg3", 20_003, 7), ("cfg5", 100_001, 5), ("cfg2", 50_001, 8),
+                                           ("higgs_like", 150_000, 6)])
 def test_single_launch_fit_equals_two_kernel_fit(ctx, name, m, iters):
     # lr_fit can run narrow-row problems as one persistent cooperative launch; the two-kernels-per-iteration form
     # must give the same bits (same batch map, same summation orders), including the loss history

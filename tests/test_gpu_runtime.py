@@ -42,6 +42,34 @@ def test_bounded_wait_gives_up_and_reports(ctx):
         ctx.selftest_wait(arm=False, limit_ms=5000)          # limits above one second are refused
 
 
+def test_an_unread_status_does_not_disturb_later_fits(ctx):
+    # the status word is a sticky report: a give-up that nobody has read yet must not end the persistent kernel of a later
+    # call (which has an abort flag of its own, cleared at every launch), nor change any result
+    wl = datagen.scaled(datagen.WORKLOADS["cfg3"], 40_001)
+    X, y, _, _ = datagen.generate(wl)
+    dX, dy = torch.from_numpy(X).cuda(), torch.from_numpy(y).cuda()
+    ctx.set_persistent(False)
+    w_ref, b_ref, h_ref = api.lr_fit(dX, dy, wl.lr, 6, return_history=True, ctx=ctx)
+    assert ctx.device_status() == 0
+    ctx.selftest_wait(arm=False, limit_ms=20)                # leaves LR_ERR_TIMEOUT in the status word, unread
+    try:
+        ctx.set_persistent(True)
+        w, b, h = api.lr_fit(dX, dy, wl.lr, 6, return_history=True, ctx=ctx)
+        assert torch.equal(w, w_ref) and torch.equal(b, b_ref) and torch.equal(h, h_ref)
+        wt = torch.zeros(wl.n, device="cuda")
+        bt = torch.zeros(1, device="cuda")
+        done, nrm = ctx.fit_tol(dX, dy, wl.lr, 0.0, 6, wt, bt)     # eps = 0 never stops early: six updates, same bits
+        assert done == 6 and torch.equal(wt, w_ref) and torch.equal(bt, b_ref)
+        ctx.set_persistent(False)
+        wt.zero_(); bt.zero_()
+        done, nrm = ctx.fit_tol(dX, dy, wl.lr, 0.0, 6, wt, bt, check_every=2)
+        assert done == 6 and torch.equal(wt, w_ref) and torch.equal(bt, b_ref)
+    finally:
+        ctx.set_persistent(None)
+    assert ctx.device_status() == api.LR_ERR_TIMEOUT         # the old report is still there, and reading clears it
+    assert ctx.device_status() == 0
+
+
 def test_sharded_driver_on_a_one_rank_nccl_group(ctx):
     import torch.distributed as dist
     from paper_2308_10037_b200 import parallel
