@@ -130,8 +130,10 @@ int lr_set_overlap(lr_ctx* ctx, int32_t on);
  * L2 residency hint for iterated passes over the same X: the first `bytes` bytes of X (whole rows) are fetched with an
  * L2 evict-last hint and everything else with evict-first, so that across the iterations of a fit that leading part
  * of X is served from the 126 MB L2 instead of HBM.  Results do not change.  0 turns the hint off; -1 (the default)
- * lets the library choose: three quarters of the L2 for the wide-row kernel (n > 512), where it is worth 12 % per pass
- * on 100k x 4096, and nothing for the narrow-row kernels, which measure slower with any part kept.
+ * lets the library choose: three quarters of the L2 for the wide-row kernel (n > 1024), where it is worth 12 % per pass
+ * on 100k x 4096; a quarter of the L2 for the persistent narrow-row kernel, where the kept rows are the first ones every
+ * warp needs after an iteration boundary (3 % per iteration on 1M x 100, 10 % on 250k x 256); and nothing for single
+ * narrow-row passes, which measure slower with any part kept.
  */
 int lr_set_l2_keep(lr_ctx* ctx, int64_t bytes);
 

@@ -33,27 +33,23 @@ constexpr int kMaxGridPerSm = 8;               // widest launch any variant uses
 constexpr int kMaxProfiled = 4096;
 constexpr int kMaxDynamicSmem = 232448;         // opt-in dynamic shared memory per CTA on sm_100
 constexpr int64_t kMaxRows = int64_t(1) << 40;
-#ifndef LRGD_NV1_RB
-#define LRGD_NV1_RB 8                          // register batch of the 68..128-column instantiation
-#endif
-#ifndef LRGD_NV2_RB
-#define LRGD_NV2_RB 4                          // register batch (rows per warp) of the 132..256-column instantiation
-#endif
 
 struct RowShape { int nv, lpr, rb; int nw = kNW; };    // nw = warps per CTA
 
-// Which instantiation of the narrow-row kernel covers ng 16-byte column groups per row.  The widest shapes -- fp32
-// rows of 129..256 groups (516..1024 columns), bfloat16 rows of 65..128 groups (520..1024 columns) -- run with eight
-// warps per CTA, so that a thread may hold its 32 columns of a row slice, their weights and accumulators (up to 255
-// registers; a 512-thread CTA gives 128); the bytes in flight per SM stay the same.
+// Which instantiation of the narrow-row kernel covers ng 16-byte column groups per row.  The shapes whose threads hold
+// more than a 512-thread CTA's 128 registers run with eight warps per CTA (255 registers): fp32 rows of 17..32 groups
+// (68..128 columns) with 16-row batches -- the per-batch work (the logistic terms, the reduction, the stage bookkeeping) is
+// then shared by twice the rows, which is what these issue-bound rows need --, fp32 rows of 65..96 and 129..256 groups and
+// bfloat16 rows of 33..128 groups (a thread holds its 32 columns of a row slice, their weights and accumulators).  The
+// bytes in flight per SM stay the same.
 bool row_shape_for(int ng, bool bf16, RowShape* s) {
     if (ng <= 8) *s = {1, 8, 8};
     else if (ng <= 16) *s = {1, 16, 8};
-    else if (ng <= 32) *s = {1, 32, LRGD_NV1_RB};
-    else if (ng <= 64 && !bf16) *s = {2, 32, LRGD_NV2_RB};
+    else if (ng <= 32 && !bf16) *s = {1, 32, 16, 8};        // 68..128 fp32 columns: eight warps, sixteen rows
+    else if (ng <= 32) *s = {1, 32, 8};
+    else if (ng <= 64 && !bf16) *s = {2, 32, 4};
     else if (ng <= 64 && bf16) *s = {2, 32, 8, 8};          // 264..512 bfloat16 columns: eight warps, eight rows (no spills)
-    else if (ng <= 96 && !bf16) *s = {4, 32, 4, 8};         // 260..384 fp32 columns: eight warps, four rows (4..6 KB batches)
-    else if (ng <= 128 && !bf16) *s = {4, 32, 2};
+    else if (ng <= 128 && !bf16) *s = {4, 32, 4, 8};        // 260..512 fp32 columns: eight warps, four rows (4..8 KB batches)
     else if (ng <= 128 && bf16) *s = {4, 32, 2, 8};         // 520..1024 bfloat16 columns: eight warps, as below
     else if (ng <= 256 && !bf16) *s = {8, 32, 2, 8};
     else return false;
@@ -264,52 +260,52 @@ cudaError_t ensure_dynamic_smem(const void* kern, int smem) {
 template <class E, int A, int B, int C, int D, bool F>
 struct KernelTag {};
 
-template <class E, int NV, int LPR, int RB, bool PRED, int NW = kNW>
-cudaError_t launch_rows_t(const lr_plan& P, const StreamParams& sp, cudaStream_t st, bool dependent) {
-    auto kern = k_stream_rows<E, NV, LPR, RB, NW, PRED>;
-    cudaError_t e = ensure_dynamic_smem<KernelTag<E, NV, LPR, RB, NW, PRED>>(reinterpret_cast<const void*>(kern), P.smem_bytes);
-    if (e != cudaSuccess) return e;
-    return launch_kernel(kern, dim3(P.grid), dim3(P.threads), size_t(P.smem_bytes), st, dependent, sp);
+// One instantiation of the narrow-row kernels: storage type, groups per lane, lanes per row, rows per batch slot, warps.
+template <class E, int NV, int LPR, int RB, int NW>
+struct RowKernelShape {
+    using Elem = E;
+    static constexpr int nv = NV, lpr = LPR, rb = RB, nw = NW;
+};
+
+// Calls f(RowKernelShape<...>{}) for the instantiation a plan of variant 0 or 3 names; every shape the planner can
+// produce is listed here once, and the two launchers below (single pass, persistent fit) share the list.
+template <class F>
+cudaError_t for_row_shape(const lr_plan& P, bool bf16, F&& f) {
+    const int nw = P.threads / 32, lpr = P.lanes_per_row, nv = P.vec_per_lane, rb = P.rows_per_batch / (32 / lpr);
+    auto is = [&](int a, int b, int c, int d) { return nv == a && lpr == b && rb == c && nw == d; };
+#define LRGD_SHAPE(E, a, b, c, d) if (is(a, b, c, d)) return f(RowKernelShape<E, a, b, c, d>{});
+    if (P.variant == 3) {                          // rows of any length: a lane owns single elements
+        if (bf16) {
+            LRGD_SHAPE(ElemBF16Any, 1, 8, 8, 16) LRGD_SHAPE(ElemBF16Any, 1, 16, 8, 16) LRGD_SHAPE(ElemBF16Any, 1, 32, 16, 16)
+            LRGD_SHAPE(ElemBF16Any, 2, 32, 16, 16) LRGD_SHAPE(ElemBF16Any, 4, 32, 8, 16) LRGD_SHAPE(ElemBF16Any, 8, 32, 4, 16)
+            LRGD_SHAPE(ElemBF16Any, 16, 32, 2, 16) LRGD_SHAPE(ElemBF16Any, 32, 32, 1, 8)
+        } else {
+            LRGD_SHAPE(ElemF32Any, 1, 8, 8, 16) LRGD_SHAPE(ElemF32Any, 1, 16, 8, 16) LRGD_SHAPE(ElemF32Any, 1, 32, 16, 16)
+            LRGD_SHAPE(ElemF32Any, 2, 32, 16, 16) LRGD_SHAPE(ElemF32Any, 4, 32, 8, 16) LRGD_SHAPE(ElemF32Any, 8, 32, 4, 16)
+            LRGD_SHAPE(ElemF32Any, 16, 32, 2, 16) LRGD_SHAPE(ElemF32Any, 32, 32, 1, 8)
+        }
+    } else if (bf16) {
+        LRGD_SHAPE(ElemBF16, 1, 8, 8, 16) LRGD_SHAPE(ElemBF16, 1, 16, 8, 16) LRGD_SHAPE(ElemBF16, 1, 32, 8, 16)
+        LRGD_SHAPE(ElemBF16, 2, 32, 8, 8) LRGD_SHAPE(ElemBF16, 4, 32, 2, 8)
+    } else {
+        LRGD_SHAPE(ElemF32, 1, 8, 8, 16) LRGD_SHAPE(ElemF32, 1, 16, 8, 16) LRGD_SHAPE(ElemF32, 1, 32, 16, 8)
+        LRGD_SHAPE(ElemF32, 2, 32, 4, 16) LRGD_SHAPE(ElemF32, 4, 32, 4, 8)
+        LRGD_SHAPE(ElemF32, 8, 32, 2, 8)
+    }
+#undef LRGD_SHAPE
+    return cudaErrorInvalidValue;
 }
 
 template <bool PRED>
 cudaError_t launch_rows(const lr_plan& P, const StreamParams& sp, cudaStream_t st, bool bf16 = false, bool dependent = false) {
-    if (P.variant == 3 && bf16) {                  // rows of any length: (lanes per row, elements per lane) picks the instantiation
-        if (P.lanes_per_row == 8) return launch_rows_t<ElemBF16Any, 1, 8, 8, PRED>(P, sp, st, dependent);
-        if (P.lanes_per_row == 16) return launch_rows_t<ElemBF16Any, 1, 16, 8, PRED>(P, sp, st, dependent);
-        if (P.vec_per_lane == 1) return launch_rows_t<ElemBF16Any, 1, 32, 16, PRED>(P, sp, st, dependent);
-        if (P.vec_per_lane == 2) return launch_rows_t<ElemBF16Any, 2, 32, 16, PRED>(P, sp, st, dependent);
-        if (P.vec_per_lane == 4) return launch_rows_t<ElemBF16Any, 4, 32, 8, PRED>(P, sp, st, dependent);
-        if (P.vec_per_lane == 8) return launch_rows_t<ElemBF16Any, 8, 32, 4, PRED>(P, sp, st, dependent);
-        if (P.vec_per_lane == 32) return launch_rows_t<ElemBF16Any, 32, 32, 1, PRED, 8>(P, sp, st, dependent);
-        return launch_rows_t<ElemBF16Any, 16, 32, 2, PRED>(P, sp, st, dependent);
-    }
-    if (P.variant == 3) {
-        if (P.lanes_per_row == 8) return launch_rows_t<ElemF32Any, 1, 8, 8, PRED>(P, sp, st, dependent);
-        if (P.lanes_per_row == 16) return launch_rows_t<ElemF32Any, 1, 16, 8, PRED>(P, sp, st, dependent);
-        if (P.vec_per_lane == 1) return launch_rows_t<ElemF32Any, 1, 32, 16, PRED>(P, sp, st, dependent);
-        if (P.vec_per_lane == 2) return launch_rows_t<ElemF32Any, 2, 32, 16, PRED>(P, sp, st, dependent);
-        if (P.vec_per_lane == 4) return launch_rows_t<ElemF32Any, 4, 32, 8, PRED>(P, sp, st, dependent);
-        if (P.vec_per_lane == 8) return launch_rows_t<ElemF32Any, 8, 32, 4, PRED>(P, sp, st, dependent);
-        if (P.vec_per_lane == 32) return launch_rows_t<ElemF32Any, 32, 32, 1, PRED, 8>(P, sp, st, dependent);
-        return launch_rows_t<ElemF32Any, 16, 32, 2, PRED>(P, sp, st, dependent);
-    }
-    if (bf16) {
-        if (P.lanes_per_row == 8) return launch_rows_t<ElemBF16, 1, 8, 8, PRED>(P, sp, st, dependent);
-        if (P.lanes_per_row == 16) return launch_rows_t<ElemBF16, 1, 16, 8, PRED>(P, sp, st, dependent);
-        if (P.vec_per_lane == 1) return launch_rows_t<ElemBF16, 1, 32, LRGD_NV1_RB, PRED>(P, sp, st, dependent);
-        if (P.vec_per_lane == 2 && P.threads == 256) return launch_rows_t<ElemBF16, 2, 32, 8, PRED, 8>(P, sp, st, dependent);
-        if (P.vec_per_lane == 2) return launch_rows_t<ElemBF16, 2, 32, LRGD_NV2_RB, PRED>(P, sp, st, dependent);
-        if (P.vec_per_lane == 4) return launch_rows_t<ElemBF16, 4, 32, 2, PRED, 8>(P, sp, st, dependent);     // eight warps per CTA
-        return cudaErrorInvalidValue;
-    }
-    if (P.lanes_per_row == 8) return launch_rows_t<ElemF32, 1, 8, 8, PRED>(P, sp, st, dependent);
-    if (P.lanes_per_row == 16) return launch_rows_t<ElemF32, 1, 16, 8, PRED>(P, sp, st, dependent);
-    if (P.vec_per_lane == 1) return launch_rows_t<ElemF32, 1, 32, LRGD_NV1_RB, PRED>(P, sp, st, dependent);
-    if (P.vec_per_lane == 2) return launch_rows_t<ElemF32, 2, 32, LRGD_NV2_RB, PRED>(P, sp, st, dependent);
-    if (P.vec_per_lane == 8) return launch_rows_t<ElemF32, 8, 32, 2, PRED, 8>(P, sp, st, dependent);      // eight warps per CTA
-    if (P.vec_per_lane == 4 && P.threads == 256) return launch_rows_t<ElemF32, 4, 32, 4, PRED, 8>(P, sp, st, dependent);
-    return launch_rows_t<ElemF32, 4, 32, 2, PRED>(P, sp, st, dependent);
+    return for_row_shape(P, bf16, [&](auto shape) {
+        using S = decltype(shape);
+        auto kern = k_stream_rows<typename S::Elem, S::nv, S::lpr, S::rb, S::nw, PRED>;
+        cudaError_t e = ensure_dynamic_smem<KernelTag<typename S::Elem, S::nv, S::lpr, S::rb, S::nw, PRED>>(
+            reinterpret_cast<const void*>(kern), P.smem_bytes);
+        if (e != cudaSuccess) return e;
+        return launch_kernel(kern, dim3(P.grid), dim3(P.threads), size_t(P.smem_bytes), st, dependent, sp);
+    });
 }
 
 // Tensor map of X for the wide-row kernel: [m][n] row-major, box = cw 16-byte groups by rb rows, zero fill outside.
@@ -378,37 +374,33 @@ cudaError_t launch_split(const lr_plan& P, const void* X, const SplitParams& sp,
     return launch_split_t<ElemF32, 1, 8, PRED>(P, tm, sp, st, dependent);
 }
 
-template <class E, int NV, int LPR, int RB>
-cudaError_t launch_fit_t(const lr_plan& P, int smem, bool resident, FitParams& fp, cudaStream_t st) {
-    const void* kern = resident ? reinterpret_cast<const void*>(k_fit_rows<E, NV, LPR, RB, kNW, true>)
-                                : reinterpret_cast<const void*>(k_fit_rows<E, NV, LPR, RB, kNW, false>);
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-    if (e != cudaSuccess) return e;
-    void* args[] = {&fp};
-    return cudaLaunchCooperativeKernel(kern, dim3(P.grid), dim3(P.threads), args, size_t(smem), st);
-}
-
-// resident: every warp's share of X fits its stages, which are then filled once and kept for the whole fit
+// The persistent whole-fit kernel of a variant-0 plan; resident: every warp's share of X fits its stages, which are then
+// filled once and kept for the whole fit.
 cudaError_t launch_fit(const lr_plan& P, int smem, bool resident, FitParams& fp, cudaStream_t st, bool bf16 = false) {
-    if (bf16) {
-        if (P.lanes_per_row == 8) return launch_fit_t<ElemBF16, 1, 8, 8>(P, smem, resident, fp, st);
-        if (P.lanes_per_row == 16) return launch_fit_t<ElemBF16, 1, 16, 8>(P, smem, resident, fp, st);
-        if (P.vec_per_lane == 1) return launch_fit_t<ElemBF16, 1, 32, LRGD_NV1_RB>(P, smem, resident, fp, st);
-        if (P.vec_per_lane == 2) return launch_fit_t<ElemBF16, 2, 32, LRGD_NV2_RB>(P, smem, resident, fp, st);
-        return cudaErrorInvalidValue;
-    }
-    if (P.lanes_per_row == 8) return launch_fit_t<ElemF32, 1, 8, 8>(P, smem, resident, fp, st);
-    if (P.lanes_per_row == 16) return launch_fit_t<ElemF32, 1, 16, 8>(P, smem, resident, fp, st);
-    if (P.vec_per_lane == 1) return launch_fit_t<ElemF32, 1, 32, LRGD_NV1_RB>(P, smem, resident, fp, st);
-    if (P.vec_per_lane == 2) return launch_fit_t<ElemF32, 2, 32, LRGD_NV2_RB>(P, smem, resident, fp, st);
-    return launch_fit_t<ElemF32, 4, 32, 2>(P, smem, resident, fp, st);
+    if (P.variant != 0) return cudaErrorInvalidValue;
+    return for_row_shape(P, bf16, [&](auto shape) {
+        using S = decltype(shape);
+        if constexpr (S::Elem::EPG > 1) {
+            const void* kern = resident ? reinterpret_cast<const void*>(k_fit_rows<typename S::Elem, S::nv, S::lpr, S::rb, S::nw, true>)
+                                        : reinterpret_cast<const void*>(k_fit_rows<typename S::Elem, S::nv, S::lpr, S::rb, S::nw, false>);
+            cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+            if (e != cudaSuccess) return e;
+            void* args[] = {&fp};
+            return cudaLaunchCooperativeKernel(kern, dim3(P.grid), dim3(P.threads), args, size_t(smem), st);
+        } else {
+            return cudaErrorInvalidValue;
+        }
+    });
 }
 
-// Rows of X to fetch with the evict-last hint.  Default: none for the narrow-row kernels (measured: any kept part slows
-// them down), three quarters of the L2 for the wide-row kernel (measured on 100k x 4096: 0.260 -> 0.231 ms per pass).
-int64_t keep_rows_for(const lr_ctx* ctx, int variant, int32_t n, bool bf16 = false) {
+// Rows of X to fetch with the evict-last hint.  Defaults: three quarters of the L2 for the wide-row kernel (measured on
+// 100k x 4096: 0.260 -> 0.231 ms per pass); a quarter of the L2 for the persistent narrow-row kernel -- the leading rows are
+// every warp's first batches of an iteration, so the stream restarts from L2 after each grid barrier (measured per
+// iteration with 0 / 32 / 64 MB kept: 1M x 100 62.2 / 60.7 / 60.4 us, 250k x 256 44.3 / 39.8 / 42.1, 125k x 256 25.2 / 22.8 /
+// 24.6, 4M x 256 572.3 / - / 566.9); nothing for single narrow-row passes, which measure slower with any part kept.
+int64_t keep_rows_for(const lr_ctx* ctx, int variant, int32_t n, bool bf16 = false, bool persistent = false) {
     int64_t bytes = ctx->l2_keep_bytes;
-    if (bytes < 0) bytes = variant == 1 ? ctx->l2_bytes / 4 * 3 : 0;
+    if (bytes < 0) bytes = variant == 1 ? ctx->l2_bytes / 4 * 3 : (persistent ? ctx->l2_bytes / 4 : 0);
     return bytes / (int64_t(n) * (bf16 ? 2 : 4));
 }
 
@@ -420,7 +412,7 @@ int64_t keep_rows_for(const lr_ctx* ctx, int variant, int32_t n, bool bf16 = fal
 // itself the persistent kernel is at least as fast everywhere, so it is the default wherever the shape allows it.
 bool want_persistent(const lr_ctx* ctx, const lr_plan& P, bool bf16, int64_t m, int32_t n, int64_t iters) {
     (void)bf16; (void)m; (void)n;
-    if (P.variant != 0 || P.threads != kNW * 32 || !ctx->coop || ctx->prof || ctx->persistent_mode == 0) return false;
+    if (P.variant != 0 || !ctx->coop || ctx->prof || ctx->persistent_mode == 0) return false;
     if (iters * P.grid >= (int64_t(1) << 32)) return false;           // the grid-barrier counter is 32 bits
     return true;
 }
@@ -432,23 +424,25 @@ struct PersistentTol { TolState* state; double eps; float* gnorm_hist; };
 cudaError_t launch_persistent_fit(lr_ctx* ctx, const lr_plan& P, bool bf16, const void* d_X, const float* d_y, int64_t m,
                                   int32_t n, float lr, int32_t iters, float* d_w, float* d_b, float* d_loss_hist,
                                   const PersistentTol* tol, cudaStream_t st) {
+    const int nw = P.threads / 32;
     const int64_t stage_stride = (int64_t(P.rows_per_batch) * n * (bf16 ? 2 : 4) + 127) & ~int64_t(127);
-    const int64_t room = kMaxDynamicSmem - kHeaderBytes - kFitTailBytes;
+    const int64_t tail = fit_tail_bytes(n);
+    const int64_t room = kMaxDynamicSmem - kHeaderBytes - tail;
     const int64_t B = (m + P.rows_per_batch - 1) / P.rows_per_batch;
-    const int64_t slots = (B + kNW - 1) / kNW;
+    const int64_t slots = (B + nw - 1) / nw;
     const int64_t per_warp = (slots + P.grid - 1) / P.grid;                    // most batches any warp handles per iteration
-    const int depth = int(std::max<int64_t>(1, std::min<int64_t>({int64_t(kMaxDepth), room / (kNW * stage_stride), per_warp})));
+    const int depth = int(std::max<int64_t>(1, std::min<int64_t>({int64_t(kMaxDepth), room / (nw * stage_stride), per_warp})));
     FitParams fp{};
     fp.X = d_X; fp.y = d_y; fp.m = m; fp.n = n; fp.w = d_w; fp.b = d_b; fp.partial = ctx->d_partial;
     fp.loss_hist = d_loss_hist; fp.status = ctx->d_status; fp.gbar = ctx->d_gbar; fp.depth = depth;
     const bool resident = per_warp <= depth;       // every warp's share of X fits its stages: filled once, kept for the fit
     fp.num_batches = B;
     fp.iters = iters; fp.lr = double(lr); fp.inv_m = 1.0 / double(m);
-    fp.keep_rows = keep_rows_for(ctx, 0, n, bf16);
+    fp.keep_rows = keep_rows_for(ctx, 0, n, bf16, true);
     if (tol) { fp.tol = tol->state; fp.eps = tol->eps; fp.gnorm_hist = tol->gnorm_hist; }
     cudaError_t e = cudaMemsetAsync(ctx->d_gbar, 0, 2 * sizeof(unsigned int), st);   // barrier counter and abort flag
     if (e != cudaSuccess) return e;
-    const int smem = int(kHeaderBytes + int64_t(kNW) * depth * stage_stride + kFitTailBytes);
+    const int smem = int(kHeaderBytes + int64_t(nw) * depth * stage_stride + tail);
     e = launch_fit(P, smem, resident, fp, st, bf16);
     if (e == cudaSuccess) ctx->launches += 1;
     return e;

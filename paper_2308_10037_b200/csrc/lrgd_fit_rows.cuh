@@ -39,17 +39,22 @@ constexpr int kFitCombineCols = 128;           // columns combined per pass thro
 #define LRGD_FIT_L2PF 4
 #endif
 constexpr int kFitL2Prefetch = LRGD_FIT_L2PF;   // batches per warp pulled into L2 ahead of the next iteration (beyond the staged ones)
-constexpr int kFitMaxCols = 512;               // widest row the persistent kernel takes
-constexpr int kFitWarps = 16;
-// after the stages: combine buffer [warps][kFitCombineCols] fp64, sum err / sum loss per warp, the CTA's copy of the
-// parameters (w[n], b) in fp32, and the reduced sums / gradient entries [n+2] in fp64
-constexpr int kFitRedBytes = kFitWarps * kFitCombineCols * 8 + 2 * kFitWarps * 8;
-constexpr int kFitParamBytes = (kFitMaxCols + 4) * 4;
-constexpr int kFitSumBytes = (kFitMaxCols + 2) * 8;
-constexpr int kFitTailBytes = (kFitRedBytes + kFitParamBytes + kFitSumBytes + 127) / 128 * 128;
+constexpr int kFitMaxCols = 1024;              // widest row the persistent kernel takes
+constexpr int kFitMaxWarps = 16;
+// after the stages: combine buffer [warps][kFitCombineCols] fp64 (sized for 16 warps) and sum err / sum loss per warp, then
+// the CTA's copy of the parameters (w[n], b) in fp32, then the reduced sums / gradient entries [n+2] in fp64
+constexpr int kFitRedBytes = kFitMaxWarps * kFitCombineCols * 8 + 2 * kFitMaxWarps * 8;
+__host__ __device__ constexpr int fit_param_bytes(int n) { return ((n + 1) * 4 + 15) / 16 * 16; }
+__host__ __device__ constexpr int fit_tail_bytes(int n) { return (kFitRedBytes + fit_param_bytes(n) + (n + 2) * 8 + 127) / 128 * 128; }
 constexpr int kFitRowChunk = 5;                // partial rows of one slice a thread has in flight (grids of up to 160 CTAs: the whole slice)
 constexpr int kFitChunkPairs = 32;             // column pairs per chunk of the reduction: one per lane, 512 contiguous bytes per row
-static_assert(2 * kFitWarps * 2 * kFitChunkPairs <= kFitWarps * kFitCombineCols, "the reduction reuses the combine buffer for two chunks");
+#ifndef LRGD_FIT_RED_INLINE
+#define LRGD_FIT_RED_INLINE __noinline__       // out of line: the streaming loop of the caller then keeps all its registers
+#endif
+#ifndef LRGD_FIT_RED_CHUNKS
+#define LRGD_FIT_RED_CHUNKS 2                  // 64-column chunks of the reduction in flight per round (where the registers allow)
+#endif
+static_assert(LRGD_FIT_RED_CHUNKS * kFitMaxWarps * 2 * kFitChunkPairs <= kFitMaxWarps * kFitCombineCols, "the reduction reuses the combine buffer");
 
 struct FitParams {
     const void* X;             // fp32 or bfloat16 [m][n], row-major
@@ -117,85 +122,100 @@ __device__ __forceinline__ bool grid_barrier(unsigned int* gbar, unsigned int ta
 // Adds up the G partial rows [G][stride] column by column into sums[stride] (shared memory); called by all threads of a
 // CTA, with the order of k_reduce_update so that the result has that kernel's bits: slice s = rows [s*per, (s+1)*per) in
 // index order, then the 32 slice sums in the fixed tree (s with s+16, then distance 8, 4, 2, 1).
-// Warp w owns slices w and w+16 -- the two that the first tree level adds -- and a lane owns one pair of adjacent columns,
-// so every load instruction of a warp reads 512 contiguous bytes of one partial row (all CTAs read the same rows at
-// the same time: scattered 16-byte reads cost L2 eight times the requests).  The 16 per-warp sums of a chunk of 64 columns
-// meet in `buf` and one thread per column finishes the tree.  Two chunks are in flight together.  Kept out of line: its
-// registers (twenty 16-byte loads in flight per thread) must not weigh on the streaming loop of the caller.
+// Warp w owns the slices w, w + NW, w + 2 NW, ... -- the ones the first tree levels add to each other -- and a lane owns
+// one pair of adjacent columns, so every load instruction of a warp reads 512 contiguous bytes of one partial row (all
+// CTAs read the same rows at the same time: scattered 16-byte reads cost L2 eight times the requests).  The NW per-warp
+// sums of a chunk of 64 columns meet in `buf` and one thread per column finishes the tree.  A thread has at most
+// (32 / NW) * kFitRowChunk 16-byte loads in flight: few enough to live in the registers the streaming loop leaves free.
+// Grids of up to 32 CTAs (small problems, where this call is most of the iteration): a slice is a single row, a lane
+// plays a slice and the tree is a butterfly of shuffles; several column pairs are in flight per warp.
 template <int NW>
-__device__ __noinline__ void reduce_partial_rows(const double* pbuf, int G, int stride, double* buf, double* sums) {
-    static_assert(2 * NW == kRedSlices, "one warp per pair of slices");
+__device__ LRGD_FIT_RED_INLINE void reduce_partial_rows(const double* pbuf, int G, int stride, double* buf, double* sums) {
+    constexpr int K = kRedSlices / NW;             // slices per warp
+    static_assert(K * NW == kRedSlices && (K & (K - 1)) == 0, "slices must split evenly over the warps");
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int per = (G + kRedSlices - 1) / kRedSlices;
     const int npairs = stride / 2;
-    const int nchunks = (npairs + kFitChunkPairs - 1) / kFitChunkPairs;
-    const int lo0 = warp * per, hi0 = (warp + NW) * per;               // first rows of slices `warp` and `warp + 16`
-    const int lo1 = lo0 + per < G ? lo0 + per : G, hi1 = hi0 + per < G ? hi0 + per : G;
     const double2 zero = make_double2(0.0, 0.0);
     if (per == 1) {
-        // grids of up to 32 CTAs (small problems, where this call is most of the iteration): a slice is a single row, so one
-        // thread per column pair holds all of them at once -- one round trip to L2, no exchange through shared memory
-        for (int q = threadIdx.x; q < npairs; q += NW * 32) {
-            double2 a[NW];
+        constexpr int U = 4;                       // column pairs in flight per warp
+        for (int q0 = warp; q0 < npairs; q0 += NW * U) {
+            double2 v[U];
 #pragma unroll
-            for (int i = 0; i < NW; ++i)
-                a[i] = i < G ? __ldcg(reinterpret_cast<const double2*>(pbuf + static_cast<size_t>(i) * stride) + q) : zero;
-            if (G > NW) {
-#pragma unroll
-                for (int i = 0; i < NW; ++i) {
-                    const double2 hi = i + NW < G ? __ldcg(reinterpret_cast<const double2*>(pbuf + static_cast<size_t>(i + NW) * stride) + q) : zero;
-                    a[i] = make_double2(a[i].x + hi.x, a[i].y + hi.y);
-                }
+            for (int u = 0; u < U; ++u) {
+                const int q = q0 + u * NW;
+                v[u] = (q < npairs && lane < G) ? __ldcg(reinterpret_cast<const double2*>(pbuf + static_cast<size_t>(lane) * stride) + q) : zero;
             }
 #pragma unroll
-            for (int h = NW / 2; h >= 1; h >>= 1)
-#pragma unroll
-                for (int i = 0; i < h; ++i) a[i] = make_double2(a[i].x + a[i + h].x, a[i].y + a[i + h].y);
-            sums[2 * q] = a[0].x;
-            sums[2 * q + 1] = a[0].y;
+            for (int u = 0; u < U; ++u) {
+                const int q = q0 + u * NW;         // warp-uniform
+                if (q < npairs) {
+                    const double tx = slice_tree_sum_warp(v[u].x), ty = slice_tree_sum_warp(v[u].y);
+                    if (lane == 0) { sums[2 * q] = tx; sums[2 * q + 1] = ty; }
+                }
+            }
         }
         __syncthreads();
         return;
     }
-    for (int c0 = 0; c0 < nchunks; c0 += 2) {
-        double2 slo[2] = {zero, zero}, shi[2] = {zero, zero};
-        for (int r0 = 0; r0 < per; r0 += kFitRowChunk) {
-            double2 vlo[2][kFitRowChunk], vhi[2][kFitRowChunk];
+    constexpr int CH = LRGD_FIT_RED_CHUNKS * K <= 4 ? LRGD_FIT_RED_CHUNKS : 1;   // chunks of 64 columns in flight (two with 16 warps)
+    const int nchunks = (npairs + kFitChunkPairs - 1) / kFitChunkPairs;
+    for (int c0 = 0; c0 < nchunks; c0 += CH) {
+        double2 acc[CH][K];
 #pragma unroll
-            for (int u = 0; u < 2; ++u) {
+        for (int u = 0; u < CH; ++u)
+#pragma unroll
+            for (int k = 0; k < K; ++k) acc[u][k] = zero;
+        for (int r0 = 0; r0 < per; r0 += kFitRowChunk) {
+            double2 v[CH][K][kFitRowChunk];
+#pragma unroll
+            for (int u = 0; u < CH; ++u) {
                 const int q = (c0 + u) * kFitChunkPairs + lane;
                 const bool live = q < npairs;
 #pragma unroll
-                for (int r = 0; r < kFitRowChunk; ++r) {
-                    const int gl = lo0 + r0 + r, gh = hi0 + r0 + r;
-                    vlo[u][r] = (live && gl < lo1) ? __ldcg(reinterpret_cast<const double2*>(pbuf + static_cast<size_t>(gl) * stride) + q) : zero;
-                    vhi[u][r] = (live && gh < hi1) ? __ldcg(reinterpret_cast<const double2*>(pbuf + static_cast<size_t>(gh) * stride) + q) : zero;
+                for (int k = 0; k < K; ++k) {
+                    const int first = (warp + k * NW) * per;               // slice warp + k NW
+                    const int last = first + per < G ? first + per : G;
+#pragma unroll
+                    for (int r = 0; r < kFitRowChunk; ++r) {
+                        const int g = first + r0 + r;
+                        v[u][k][r] = (live && r0 + r < per && g < last)
+                                         ? __ldcg(reinterpret_cast<const double2*>(pbuf + static_cast<size_t>(g) * stride) + q) : zero;
+                    }
                 }
             }
 #pragma unroll
-            for (int u = 0; u < 2; ++u)
+            for (int u = 0; u < CH; ++u)
 #pragma unroll
-                for (int r = 0; r < kFitRowChunk; ++r) {               // (+0.0 where there is no row: changes nothing)
-                    slo[u].x += vlo[u][r].x; slo[u].y += vlo[u][r].y;
-                    shi[u].x += vhi[u][r].x; shi[u].y += vhi[u][r].y;
-                }
+                for (int k = 0; k < K; ++k)
+#pragma unroll
+                    for (int r = 0; r < kFitRowChunk; ++r) {               // (+0.0 where there is no row: changes nothing)
+                        acc[u][k].x += v[u][k][r].x;
+                        acc[u][k].y += v[u][k][r].y;
+                    }
         }
 #pragma unroll
-        for (int u = 0; u < 2; ++u)                                    // first tree level: slice w + slice w+16
-            reinterpret_cast<double2*>(buf)[(u * NW + warp) * kFitChunkPairs + lane] = make_double2(slo[u].x + shi[u].x, slo[u].y + shi[u].y);
+        for (int u = 0; u < CH; ++u) {
+            // the tree levels inside this warp's slices: distance 16, 8, ... down to NW (in slices), i.e. K/2, ..., 1 here
+#pragma unroll
+            for (int h = K / 2; h >= 1; h >>= 1)
+#pragma unroll
+                for (int k = 0; k < h; ++k) { acc[u][k].x += acc[u][k + h].x; acc[u][k].y += acc[u][k + h].y; }
+            reinterpret_cast<double2*>(buf)[(u * NW + warp) * kFitChunkPairs + lane] = acc[u][0];
+        }
         __syncthreads();
-        if (threadIdx.x < 4 * kFitChunkPairs) {
+        if (threadIdx.x < CH * 2 * kFitChunkPairs) {
             const int u = threadIdx.x / (2 * kFitChunkPairs), c = threadIdx.x % (2 * kFitChunkPairs);
             const int col = (c0 + u) * 2 * kFitChunkPairs + c;
             if (col < stride) {
-                double v[NW];
+                double t[NW];
 #pragma unroll
-                for (int i = 0; i < NW; ++i) v[i] = buf[(u * NW + i) * 2 * kFitChunkPairs + c];
+                for (int i = 0; i < NW; ++i) t[i] = buf[(u * NW + i) * 2 * kFitChunkPairs + c];
 #pragma unroll
                 for (int h = NW / 2; h >= 1; h >>= 1)
 #pragma unroll
-                    for (int i = 0; i < h; ++i) v[i] = v[i] + v[i + h];
-                sums[col] = v[0];
+                    for (int i = 0; i < h; ++i) t[i] = t[i] + t[i + h];
+                sums[col] = t[0];
             }
         }
         __syncthreads();
@@ -214,7 +234,7 @@ __global__ void __launch_bounds__(NW * 32, 1) k_fit_rows(const FitParams p) {
     static_assert(SHIFT >= 0, "rows per batch slot must not exceed lanes per row");
     static_assert(E::EPG > 1, "rows of 16-byte groups only");
     static_assert(kRedSlices == 32, "one lane per reduction slice of k_reduce_update");
-    static_assert(NW == kFitWarps, "tail layout is sized for this many warps");
+    static_assert(NW <= kFitMaxWarps && kRedSlices % NW == 0, "tail layout and reduction are sized for up to 16 warps");
     static_assert(NV * LPR * EPG <= kFitMaxCols, "row wider than the parameter copy");
 
     extern __shared__ __align__(128) unsigned char smem[];
@@ -235,7 +255,7 @@ __global__ void __launch_bounds__(NW * 32, 1) k_fit_rows(const FitParams p) {
     double* red_e = red + NW * kFitCombineCols;
     double* red_l = red_e + NW;
     float* w_s = reinterpret_cast<float*>(tail + kFitRedBytes);        // w[0..n), then b
-    double* sum_s = reinterpret_cast<double*>(tail + kFitRedBytes + kFitParamBytes);   // [n+2]
+    double* sum_s = reinterpret_cast<double*>(tail + kFitRedBytes + fit_param_bytes(n));   // [n+2]
     uint64_t* my_bars = bars + warp * kMaxDepth;
 
     const long long B = p.num_batches;

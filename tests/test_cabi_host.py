@@ -51,20 +51,23 @@ def test_null_context_is_rejected_before_any_cuda_call():
     assert L.lr_destroy(None) == api.LR_OK
 
 
-@pytest.mark.parametrize("m,n,lpr,nv", [(10_000, 32, 8, 1), (16_000_000, 64, 16, 1), (1_000_000, 100, 32, 1),
-                                         (4_000_000, 256, 32, 2), (11_000_000, 28, 8, 1), (5000, 512, 32, 4)])
-def test_plan_staged_shapes(m, n, lpr, nv):
+@pytest.mark.parametrize("m,n,lpr,nv,nw", [(10_000, 32, 8, 1, 16), (16_000_000, 64, 16, 1, 16), (1_000_000, 100, 32, 1, 8),
+                                            (4_000_000, 256, 32, 2, 16), (11_000_000, 28, 8, 1, 16), (5000, 512, 32, 4, 8),
+                                            (70_000, 128, 32, 1, 8), (9_000, 68, 32, 1, 8)])
+def test_plan_staged_shapes(m, n, lpr, nv, nw):
     p = api.plan_query(m, n)
     assert p["variant"] == 0 and p["lanes_per_row"] == lpr and p["vec_per_lane"] == nv
-    assert p["threads"] == 512 and 1 <= p["grid"] <= 148
+    assert p["threads"] == 32 * nw and 1 <= p["grid"] <= 148
     assert p["tile_rows"] == p["rows_per_batch"]              # one stage holds one register batch
     assert 1 <= p["stages"] <= 4
     assert p["smem_bytes"] <= 227 * 1024
     stage = -(-p["tile_rows"] * n * 4 // 128) * 128
-    assert 1024 + 16 * p["stages"] * stage <= p["smem_bytes"]
-    # 16 warps per CTA take one batch each per round; the grid never exceeds the rounds available
+    assert 1024 + nw * p["stages"] * stage <= p["smem_bytes"]
+    # the warps of a CTA take one batch each per round; the grid never exceeds the rounds available
     batches = -(-m // p["rows_per_batch"])
-    assert p["grid"] == min(-(-batches // 16), 148)
+    assert p["grid"] == min(-(-batches // nw), 148)
+    if nw == 8 and nv == 1:
+        assert p["rows_per_batch"] == 16                      # 68..128 fp32 columns: sixteen rows per batch, eight warps
 
 
 def test_plan_falls_back_for_unaligned_or_odd_shapes():

@@ -330,6 +330,37 @@ def test_single_launch_fit_equals_two_kernel_fit(ctx, name, m, iters):
     assert ctx.device_status() == 0
 
 
+# the other shapes of the narrow-row kernels, eight-warp ones included (68..128, 260..384 and 516..1024 columns), resident
+# (every row stays in shared memory) and streaming; bfloat16 storage of the same matrices too
+@pytest.mark.parametrize("m,n", [(50_001, 128), (300_001, 100), (30_001, 320), (9_001, 1024), (60_001, 516), (40_001, 388),
+                                 (120_001, 260), (2_001, 68), (200_003, 16), (33, 1000)])
+@pytest.mark.parametrize("bf16", [False, True])
+def test_single_launch_fit_equals_two_kernel_fit_all_shapes(ctx, m, n, bf16):
+    X, y, w0, b0 = datagen.random_problem(m, n, seed=8000 + m + n, wscale=0.5)
+    if bf16:
+        if n % 8:
+            pytest.skip("bfloat16 rows of 16-byte groups need n % 8 == 0")
+        bits, X = oracle.round_bf16(X)
+        dX = torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16)
+    else:
+        dX = dev(X)
+    dy, iters, lr = dev(y), 7, 0.2
+    try:
+        ctx.set_persistent(True)
+        n0 = ctx.launch_count()
+        w1, b1, h1 = api.lr_fit(dX, dy, lr, iters, w0=dev(w0), b0=float(b0), return_history=True, ctx=ctx)
+        assert ctx.launch_count() == n0 + 1
+        ctx.set_persistent(False)
+        w2, b2, h2 = api.lr_fit(dX, dy, lr, iters, w0=dev(w0), b0=float(b0), return_history=True, ctx=ctx)
+    finally:
+        ctx.set_persistent(None)
+    assert torch.equal(w1, w2) and torch.equal(b1, b2) and torch.equal(h1, h2)
+    w_ref, b_ref, lh_ref = oracle.fit(X, y, lr, iters, w0=w0, b0=b0)
+    assert rel_l2(np.concatenate([w1.cpu().numpy(), b1.cpu().numpy()]), np.concatenate([w_ref, [b_ref]])) <= W_TOL
+    assert np.max(np.abs(h1.cpu().numpy() - lh_ref)) <= LOSS_TOL
+    assert ctx.device_status() == 0
+
+
 def test_row_sharded_entry_points_match_oracle(ctx):
     # three row shards on one GPU, one after the other (no kernel waits on another): lr_shard_sums per shard,
     # lr_apply_sums over the stacked sums, for several steps; against the checker's unsharded fit
