@@ -215,7 +215,7 @@ def workload_config(wl, n_gpus, x_dtype="f32"):
                    f"X is {wl.m * wl.n * eb / 1e6:.0f} MB, not larger than twice the 126 MB L2: part of every pass is served from L2"
                    if wl.m * wl.n * eb > 126e6 else
                    "X fits in L2: the pass is launch/L2-bound, not HBM-bound"),
-            "parallelism": "single GPU" if n_gpus == 1 else f"dp{n_gpus} row-sharded, all-gather of n+2 fp64 sums per iteration"}
+            "parallelism": "single GPU" if n_gpus == 1 else f"dp{n_gpus} row-sharded, n+2 fp64 sums exchanged per iteration"}
 
 
 def run_tol(args, wl):
@@ -281,6 +281,9 @@ def main():
     ap.add_argument("--x-dtype", default="f32", choices=["f32", "bf16"],
                     help="storage type of X on the device: bf16 runs the bfloat16 entry points on lr_convert_bf16's output "
                          "(half the bytes per pass; no end-to-end or CPU leg)")
+    ap.add_argument("--fused-exchange", action="store_true",
+                    help="--gpus N > 1: exchange the sums inside the persistent kernel (lr_fit_sharded over symmetric memory) "
+                         "instead of one NCCL all-gather per iteration")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
@@ -349,9 +352,13 @@ def main():
         args.no_e2e = args.no_cpu_baseline = True
     elem_bytes = 2 if bf16 else 4
 
+    exchange = parallel.ExchangeBuffers(wl.n, torch.device("cuda", local_rank)) if world > 1 and args.fused_exchange else None
+
     def run_steps(k):
         if world == 1:
             ctx.fit(dX, dy, wl.lr, k, w, b)
+        elif exchange is not None:
+            parallel.fit_sharded_fused(ctx, dX, dy, m_total, wl.lr, k, w, b, exchange)
         else:
             parallel.fit_sharded_cuda(ctx, dX, dy, m_total, wl.lr, k, w, b)
 

@@ -243,14 +243,70 @@ int lr_shard_sums_bf16(lr_ctx* ctx, const uint16_t* d_Xh, const float* d_y, int6
  * runs on one device).  Each shard holds a contiguous block of rows.  lr_shard_sums runs the fused
  * pass on the local rows and writes the UNNORMALISED fp64 sums d_sums[0..n) = X^T err,
  * d_sums[n] = sum err, d_sums[n+1] = sum of per-row loss terms.  After the caller has gathered the
- * `parts` sum vectors into d_sums_all [parts][n+2] (rank order), lr_apply_sums adds them in index
- * order, scales by 1/m_total and applies  w <- w - lr*grad_w, b <- b - lr*grad_b  (every rank gets
+ * `parts` sum vectors into d_sums_all [parts][n+2] (rank order), lr_apply_sums adds them in a fixed
+ * order (a pairwise tree over the parts), scales by 1/m_total and applies  w <- w - lr*grad_w, b <- b - lr*grad_b  (every rank gets
  * bit-identical parameters); d_loss (nullable) receives the global loss before the update.
  */
 int lr_shard_sums(lr_ctx* ctx, const float* d_X, const float* d_y, int64_t m_local, int32_t n,
                   const float* d_w, const float* d_b, double* d_sums, void* stream);
 int lr_apply_sums(lr_ctx* ctx, const double* d_sums_all, int32_t parts, int64_t m_total, int32_t n,
                   float lr, float* d_w, float* d_b, float* d_loss, void* stream);
+
+/*
+ * Row-sharded fit with the exchange inside the kernel (same split of Algorithm 1's sums over rows as lr_shard_sums /
+ * lr_apply_sums, without a host round trip or a collective call per iteration).  Every rank calls lr_fit_sharded with
+ * its own rows (m_local of the m_total rows), the same n, lr and iters, and the same start point in d_w, d_b.  Each
+ * iteration a rank forms the n+2 sums of its rows in one persistent launch (see lr_fit), stores them into slot
+ * [step parity][rank] of EVERY rank's exchange buffer with plain stores, publishes the step number in flag [rank] of
+ * every buffer (system-scope release), waits until the flags of all ranks in its own buffer show the step, adds the
+ * `world` vectors in the fixed order lr_apply_sums uses and applies the update.  All ranks end with bit-identical
+ * parameters, and with the bits the lr_shard_sums / all-gather / lr_apply_sums loop gives.  With world == 1 the result is
+ * lr_fit's, bit for bit.  d_loss_hist (NULL or [iters]) receives the global loss on every rank.
+ *
+ * Exchange buffers: one per rank, in that rank's own device memory, lr_exchange_bytes(world, n) bytes, 128-byte aligned,
+ * ZEROED ONCE before the first use (followed by a barrier among the ranks), and mapped into every other rank's address
+ * space (peer access within a process, CUDA IPC or a symmetric-memory allocation between processes).  d_exchange is a HOST
+ * array of `world` device pointers as THIS rank addresses them; d_exchange[rank] is its own buffer.  Only plain loads
+ * and stores touch a peer's memory.
+ * epoch: the number of steps these buffers have carried so far -- 0 for the first call, then the sum of the iters of the
+ * earlier calls; it must be the same on every rank (the flags count steps monotonically across calls).
+ * wait_ms (1..60000): bound on every wait for the other ranks.  When it expires (a rank that died or never called), the
+ * kernel stops, d_w and d_b keep their values from before the call and lr_last_device_status reports LR_ERR_TIMEOUT;
+ * the buffers must then be zeroed and the epoch restarted before they are used again.
+ * Shapes: those lr_fit runs as one persistent launch (rows of up to 1024 columns, 16-byte aligned X, n % 4 == 0; n % 8 for
+ * bfloat16) on a device with cooperative launches; anything else returns LR_ERR_SHAPE (use lr_shard_sums / lr_apply_sums).
+ * Errors: as lr_fit, plus LR_ERR_SHAPE for world outside 1..32, rank outside [0, world), m_total < m_local, epoch < 0;
+ * LR_ERR_VALUE for wait_ms out of range; LR_ERR_ALIGNMENT for an exchange buffer that is not 128-byte aligned.
+ */
+int lr_exchange_bytes(int32_t world, int32_t n, int64_t* bytes);
+int lr_fit_sharded(lr_ctx* ctx, const float* d_X, const float* d_y, int64_t m_local, int64_t m_total, int32_t n,
+                   float lr, int32_t iters, float* d_w, float* d_b, float* d_loss_hist,
+                   int32_t rank, int32_t world, void* const* d_exchange, int64_t epoch, int32_t wait_ms, void* stream);
+int lr_fit_sharded_bf16(lr_ctx* ctx, const uint16_t* d_Xh, const float* d_y, int64_t m_local, int64_t m_total, int32_t n,
+                        float lr, int32_t iters, float* d_w, float* d_b, float* d_loss_hist,
+                        int32_t rank, int32_t world, void* const* d_exchange, int64_t epoch, int32_t wait_ms, void* stream);
+
+/*
+ * The ranks of lr_fit_sharded on ONE GPU: `world` (2..32) row shards run as `world` groups of CTAs of a single cooperative
+ * launch, each group with its own rows, parameters and exchange buffer, exchanging exactly as ranks on different GPUs do.
+ * Because all CTAs of a cooperative launch are resident together, ranks that wait on one another cannot starve each
+ * other -- which separate launches, streams or processes on one GPU could not guarantee.  This is the way to run and
+ * test the multi-rank path where a single GPU is available; it is not faster than lr_fit.
+ * d_X, d_y, m_local, d_w, d_b, d_loss_hist (nullable, entries nullable) and d_exchange are HOST arrays of `world`
+ * entries (device pointers / row counts); d_w[r], d_b[r] hold the common start point and receive rank r's result.
+ * Every rank takes plan-SMs / world SMs (see lr_set_sm_limit).  Built for fp32 rows of up to 32 and of 132..256 columns
+ * with 16-byte aligned shards; other shapes return LR_ERR_SHAPE.  The call blocks until its parameter block is on the device.
+ */
+int lr_fit_sharded_local(lr_ctx* ctx, int32_t world, const float* const* d_X, const float* const* d_y, const int64_t* m_local,
+                         int32_t n, float lr, int32_t iters, float* const* d_w, float* const* d_b, float* const* d_loss_hist,
+                         void* const* d_exchange, int64_t epoch, int32_t wait_ms, void* stream);
+
+/*
+ * Limits the SMs (CTAs) the launch plans of this context use to `sms`; 0 restores the device's count.  The per-CTA
+ * partial sums, hence the low bits of every result, depend on the grid: two contexts with the same limit on the same
+ * kind of device give the same bits.
+ */
+int lr_set_sm_limit(lr_ctx* ctx, int32_t sms);
 
 /*
  * Host-buffer variants: copy h_X, h_y (and h_w, h_b) to device buffers owned by the context

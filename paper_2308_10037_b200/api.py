@@ -23,7 +23,8 @@ EXPORTS = ["lr_plan_query", "lr_create", "lr_destroy", "lr_loss_grad", "lr_fit",
            "lr_predict_host", "lr_profile_enable", "lr_profile_read", "lr_launch_count", "lr_last_device_status",
            "lr_last_cuda_error", "lr_status_string", "lr_loss_grad_noalloc", "lr_fit_tol", "lr_fit_opt", "lr_selftest_wait", "lr_set_persistent", "lr_fit_sgd", "lr_set_l2_keep",
            "lr_convert_bf16", "lr_loss_grad_bf16", "lr_fit_bf16", "lr_predict_bf16", "lr_plan_query_bf16",
-           "lr_fit_tol_bf16", "lr_fit_opt_bf16", "lr_fit_sgd_bf16", "lr_shard_sums_bf16", "lr_set_overlap"]
+           "lr_fit_tol_bf16", "lr_fit_opt_bf16", "lr_fit_sgd_bf16", "lr_shard_sums_bf16", "lr_set_overlap",
+           "lr_exchange_bytes", "lr_fit_sharded", "lr_fit_sharded_bf16", "lr_fit_sharded_local", "lr_set_sm_limit"]
 
 
 class LrPlan(ctypes.Structure):
@@ -81,6 +82,12 @@ def lib() -> ctypes.CDLL:
         L.lr_set_persistent.argtypes = [P, I32]
         L.lr_set_overlap.argtypes = [P, I32]
         L.lr_set_l2_keep.argtypes = [P, I64]
+        L.lr_set_sm_limit.argtypes = [P, I32]
+        L.lr_exchange_bytes.argtypes = [I32, I32, ctypes.POINTER(I64)]
+        L.lr_fit_sharded.argtypes = [P, P, P, I64, I64, I32, F, I32, P, P, P, I32, I32, ctypes.POINTER(P), I64, I32, P]
+        L.lr_fit_sharded_bf16.argtypes = L.lr_fit_sharded.argtypes
+        L.lr_fit_sharded_local.argtypes = [P, I32, ctypes.POINTER(P), ctypes.POINTER(P), ctypes.POINTER(I64), I32, F, I32,
+                                           ctypes.POINTER(P), ctypes.POINTER(P), ctypes.POINTER(P), ctypes.POINTER(P), I64, I32, P]
         L.lr_loss_grad_noalloc.argtypes = [I32, P, P, I64, I32, P, P, P, P, P, P, P]
         L.lr_fit_host.argtypes = [P, P, P, I64, I32, F, I32, P, P, P]
         L.lr_predict_host.argtypes = [P, P, I64, I32, P, P, F, P]
@@ -110,6 +117,15 @@ def plan_query(m: int, n: int, x_aligned16: bool = True, sm_count: int = 148, bf
     if rc != LR_OK:
         raise LrError(rc, "lr_plan_query")
     return p.as_dict()
+
+
+def exchange_bytes(world: int, n: int) -> int:
+    """Size of one rank's exchange buffer for a row-sharded fit over ``world`` ranks and ``n`` columns."""
+    v = ctypes.c_int64()
+    rc = lib().lr_exchange_bytes(int(world), int(n), ctypes.byref(v))
+    if rc != LR_OK:
+        raise LrError(rc, "lr_exchange_bytes")
+    return v.value
 
 
 def _dev_ptr(t: torch.Tensor | None, dtype, name: str, count: int | None = None, device: int | None = None):
@@ -295,6 +311,68 @@ class Context:
                                  float(lr), self._p(w, F32, "w", n), self._p(b, F32, "b", 1), self._p(loss, F32, "loss", 1),
                                  self._stream())
         self._check(rc, "lr_apply_sums")
+
+    # ---- row shards with the exchange inside the kernel ------------------------------------------
+    def fit_sharded(self, X, y, m_total, lr, iters, w, b, rank, world, exchange_ptrs, epoch=0, wait_ms=10_000, loss_hist=None):
+        """This rank's part of a row-sharded fit (see ``lr_fit_sharded``), in place on w, b.
+
+        ``exchange_ptrs``: the ``world`` exchange buffers as this rank addresses them (integers, or CUDA tensors for
+        buffers of this process); ``exchange_ptrs[rank]`` is this rank's own.  ``epoch``: steps these buffers have carried.
+        """
+        m, n = _shape2(X)
+        xdt, sfx = self._x_kind(X)
+        F32, iters = torch.float32, int(iters)
+        if len(exchange_ptrs) != int(world):
+            raise ValueError("exchange_ptrs: one buffer per rank")
+        need = exchange_bytes(int(world), n)
+        ptrs = (ctypes.c_void_p * int(world))()
+        for r, e in enumerate(exchange_ptrs):
+            if isinstance(e, torch.Tensor):
+                if not e.is_cuda or e.numel() * e.element_size() < need:
+                    raise ValueError(f"exchange_ptrs[{r}]: a CUDA tensor of at least {need} bytes is needed")
+                e = e.data_ptr()
+            ptrs[r] = ctypes.c_void_p(int(e))
+        rc = getattr(lib(), "lr_fit_sharded" + sfx)(self._h, self._p(X, xdt, "X"), self._p(y, F32, "y", m), m, int(m_total), n,
+                                  float(lr), iters, self._p(w, F32, "w", n), self._p(b, F32, "b", 1),
+                                  self._p(loss_hist, F32, "loss_hist", max(iters, 0)), int(rank), int(world), ptrs,
+                                  int(epoch), int(wait_ms), self._stream())
+        self._check(rc, "lr_fit_sharded" + sfx)
+
+    def fit_sharded_local(self, Xs, ys, lr, iters, ws, bs, exchange, epoch=0, wait_ms=10_000, loss_hists=None):
+        """All ranks of a row-sharded fit as CTA groups of one launch on this GPU (see ``lr_fit_sharded_local``).
+
+        ``Xs``, ``ys``, ``ws``, ``bs``, ``exchange`` (and ``loss_hists``) are lists with one CUDA tensor per rank.
+        """
+        world = len(Xs)
+        if not (len(ys) == len(ws) == len(bs) == len(exchange) == world) or (loss_hists is not None and len(loss_hists) != world):
+            raise ValueError("one entry per rank in every list")
+        F32, iters = torch.float32, int(iters)
+        n = _shape2(Xs[0])[1]
+        need = exchange_bytes(world, n)
+        PA = ctypes.c_void_p * world
+        pX, py, pw, pb, ph, pe = PA(), PA(), PA(), PA(), PA(), PA()
+        ms = (ctypes.c_int64 * world)()
+        for r in range(world):
+            m, nr = _shape2(Xs[r], f"Xs[{r}]")
+            if nr != n:
+                raise ValueError("all shards need the same number of columns")
+            ms[r] = m
+            pX[r] = self._p(Xs[r], F32, f"Xs[{r}]")
+            py[r] = self._p(ys[r], F32, f"ys[{r}]", m)
+            pw[r] = self._p(ws[r], F32, f"ws[{r}]", n)
+            pb[r] = self._p(bs[r], F32, f"bs[{r}]", 1)
+            ph[r] = self._p(loss_hists[r], F32, f"loss_hists[{r}]", max(iters, 0)) if loss_hists is not None else None
+            e = exchange[r]
+            if not (isinstance(e, torch.Tensor) and e.is_cuda and e.numel() * e.element_size() >= need):
+                raise ValueError(f"exchange[{r}]: a CUDA tensor of at least {need} bytes is needed")
+            pe[r] = ctypes.c_void_p(e.data_ptr())
+        rc = lib().lr_fit_sharded_local(self._h, world, pX, py, ms, n, float(lr), iters, pw, pb,
+                                        ph if loss_hists is not None else None, pe, int(epoch), int(wait_ms), self._stream())
+        self._check(rc, "lr_fit_sharded_local")
+
+    def set_sm_limit(self, sms: int | None):
+        """Launch plans of this context use at most ``sms`` SMs (None or 0: all of them)."""
+        self._check(lib().lr_set_sm_limit(self._h, int(sms or 0)), "lr_set_sm_limit")
 
     # ---- host-pointer entry points ---------------------------------------------------------------
     def fit_host(self, X, y, lr, iters, w, b, loss_hist=None):

@@ -10,6 +10,7 @@
 #include <cstring>
 #include <mutex>
 #include <new>
+#include <type_traits>
 #include <utility>
 #include <vector>
 
@@ -166,6 +167,9 @@ struct lr_ctx {
     double* d_oscr = nullptr;                       // [n_max+2] scratch of the optimiser reduction
     unsigned int* d_oticket = nullptr;
     unsigned int* d_gbar = nullptr;                 // persistent fit kernel: [0] grid-barrier counter, [1] abort flag of the launch
+                                                    // (one such pair per rank when several ranks run as one launch)
+    FitParams* d_rank_params = nullptr;             // [kMaxWorld] parameters of the ranks of lr_fit_sharded_local
+    int sm_limit = 0;                               // > 0: plans use at most this many SMs (lr_set_sm_limit)
     bool coop = false;                              // device supports cooperative launches
     int persistent_mode = -1;                       // single-launch fit kernel: -1 the library chooses, 0 never, 1 whenever the shape allows
     bool overlap = true;                            // consecutive kernels of one call are launched as programmatic dependents
@@ -214,6 +218,9 @@ struct DeviceGuard {
     } while (0)
 
 bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
+
+// SMs the launch plans of this context may use (lr_set_sm_limit)
+int plan_sms(const lr_ctx* ctx) { return ctx->sm_limit > 0 ? std::min(ctx->sm_limit, ctx->sm_count) : ctx->sm_count; }
 
 // Launches `kern`; with `dependent` set, as a programmatic dependent launch: the kernel may start while the kernel
 // before it in the stream is still draining, and synchronises with it on the device (grid_dependency_wait).
@@ -393,6 +400,28 @@ cudaError_t launch_fit(const lr_plan& P, int smem, bool resident, FitParams& fp,
     });
 }
 
+// The same kernel with several ranks of a row-sharded fit as CTA groups of one cooperative launch (lr_fit_sharded_local).
+// Built for two shapes only -- fp32 rows of up to 32 and of 132..256 columns -- which is what exercising the exchange needs.
+cudaError_t launch_fit_ranks(const lr_plan& P, int smem, bool resident, const FitParams* d_ranks, int world, int ctas_per_rank,
+                             cudaStream_t st) {
+    if (P.variant != 0) return cudaErrorInvalidValue;
+    return for_row_shape(P, false, [&](auto shape) {
+        using S = decltype(shape);
+        constexpr bool built = std::is_same<typename S::Elem, ElemF32>::value && S::nw == 16 &&
+                               ((S::nv == 2 && S::lpr == 32 && S::rb == 4) || (S::nv == 1 && S::lpr == 8 && S::rb == 8));
+        if constexpr (built) {
+            const void* kern = resident ? reinterpret_cast<const void*>(k_fit_rows_ranks<ElemF32, S::nv, S::lpr, S::rb, S::nw, true>)
+                                        : reinterpret_cast<const void*>(k_fit_rows_ranks<ElemF32, S::nv, S::lpr, S::rb, S::nw, false>);
+            cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+            if (e != cudaSuccess) return e;
+            void* args[] = {&d_ranks, &ctas_per_rank};
+            return cudaLaunchCooperativeKernel(kern, dim3(world * ctas_per_rank), dim3(P.threads), args, size_t(smem), st);
+        } else {
+            return cudaErrorInvalidValue;
+        }
+    });
+}
+
 // Rows of X to fetch with the evict-last hint.  Defaults: three quarters of the L2 for the wide-row kernel (measured on
 // 100k x 4096: 0.260 -> 0.231 ms per pass); a quarter of the L2 for the persistent narrow-row kernel -- the leading rows are
 // every warp's first batches of an iteration, so the stream restarts from L2 after each grid barrier (measured per
@@ -417,33 +446,57 @@ bool want_persistent(const lr_ctx* ctx, const lr_plan& P, bool bf16, int64_t m, 
     return true;
 }
 
-// Enqueues the persistent kernel for a whole fit (fixed count, or with the stopping rule when `tol` is given).
-// Returns cudaErrorCooperativeLaunchTooLarge when the CTAs cannot all be resident (the caller then iterates with two
-// kernels), any other error as it comes.
-struct PersistentTol { TolState* state; double eps; float* gnorm_hist; };
-cudaError_t launch_persistent_fit(lr_ctx* ctx, const lr_plan& P, bool bf16, const void* d_X, const float* d_y, int64_t m,
-                                  int32_t n, float lr, int32_t iters, float* d_w, float* d_b, float* d_loss_hist,
-                                  const PersistentTol* tol, cudaStream_t st) {
+// Shared-memory shape of the persistent kernel for a plan and a grid of G CTAs: stages per warp, whether every warp's
+// share of X stays resident in them, and the dynamic shared memory of a CTA.
+struct FitLayout { int depth; bool resident; int smem; };
+FitLayout fit_layout(const lr_plan& P, bool bf16, int64_t m, int32_t n, int G) {
     const int nw = P.threads / 32;
     const int64_t stage_stride = (int64_t(P.rows_per_batch) * n * (bf16 ? 2 : 4) + 127) & ~int64_t(127);
     const int64_t tail = fit_tail_bytes(n);
     const int64_t room = kMaxDynamicSmem - kHeaderBytes - tail;
     const int64_t B = (m + P.rows_per_batch - 1) / P.rows_per_batch;
     const int64_t slots = (B + nw - 1) / nw;
-    const int64_t per_warp = (slots + P.grid - 1) / P.grid;                    // most batches any warp handles per iteration
-    const int depth = int(std::max<int64_t>(1, std::min<int64_t>({int64_t(kMaxDepth), room / (nw * stage_stride), per_warp})));
+    const int64_t per_warp = (slots + G - 1) / G;                              // most batches any warp handles per iteration
+    FitLayout L;
+    L.depth = int(std::max<int64_t>(1, std::min<int64_t>({int64_t(kMaxDepth), room / (nw * stage_stride), per_warp})));
+    L.resident = per_warp <= L.depth;              // every warp's share of X fits its stages: filled once, kept for the fit
+    L.smem = int(kHeaderBytes + int64_t(nw) * L.depth * stage_stride + tail);
+    return L;
+}
+
+struct PersistentTol { TolState* state; double eps; float* gnorm_hist; };
+struct PersistentShard {                           // row shards: this rank, the exchange buffers, the bound on waits for peers
+    int rank, world; int64_t m_total; uint64_t epoch; uint64_t wait_ns; void* const* xbuf;
+};
+
+FitParams fit_params(lr_ctx* ctx, const lr_plan& P, bool bf16, const void* d_X, const float* d_y, int64_t m, int32_t n, float lr,
+                     int32_t iters, float* d_w, float* d_b, float* d_loss_hist, int depth, const PersistentTol* tol,
+                     const PersistentShard* shard) {
     FitParams fp{};
     fp.X = d_X; fp.y = d_y; fp.m = m; fp.n = n; fp.w = d_w; fp.b = d_b; fp.partial = ctx->d_partial;
     fp.loss_hist = d_loss_hist; fp.status = ctx->d_status; fp.gbar = ctx->d_gbar; fp.depth = depth;
-    const bool resident = per_warp <= depth;       // every warp's share of X fits its stages: filled once, kept for the fit
-    fp.num_batches = B;
-    fp.iters = iters; fp.lr = double(lr); fp.inv_m = 1.0 / double(m);
+    fp.num_batches = (m + P.rows_per_batch - 1) / P.rows_per_batch;
+    fp.iters = iters; fp.lr = double(lr); fp.inv_m = 1.0 / double(shard ? shard->m_total : m);
     fp.keep_rows = keep_rows_for(ctx, 0, n, bf16, true);
     if (tol) { fp.tol = tol->state; fp.eps = tol->eps; fp.gnorm_hist = tol->gnorm_hist; }
+    if (shard) {
+        fp.rank = shard->rank; fp.world = shard->world; fp.epoch = shard->epoch; fp.wait_ns = shard->wait_ns;
+        for (int r = 0; r < shard->world; ++r) fp.xbuf[r] = static_cast<unsigned char*>(shard->xbuf[r]);
+    }
+    return fp;
+}
+
+// Enqueues the persistent kernel for a whole fit (fixed count, or with the stopping rule when `tol` is given, or as one
+// rank of a row-sharded fit when `shard` is given).  Returns cudaErrorCooperativeLaunchTooLarge when the CTAs cannot all
+// be resident (the caller then iterates with two kernels), any other error as it comes.
+cudaError_t launch_persistent_fit(lr_ctx* ctx, const lr_plan& P, bool bf16, const void* d_X, const float* d_y, int64_t m,
+                                  int32_t n, float lr, int32_t iters, float* d_w, float* d_b, float* d_loss_hist,
+                                  const PersistentTol* tol, cudaStream_t st, const PersistentShard* shard = nullptr) {
+    const FitLayout L = fit_layout(P, bf16, m, n, P.grid);
+    FitParams fp = fit_params(ctx, P, bf16, d_X, d_y, m, n, lr, iters, d_w, d_b, d_loss_hist, L.depth, tol, shard);
     cudaError_t e = cudaMemsetAsync(ctx->d_gbar, 0, 2 * sizeof(unsigned int), st);   // barrier counter and abort flag
     if (e != cudaSuccess) return e;
-    const int smem = int(kHeaderBytes + int64_t(nw) * depth * stage_stride + tail);
-    e = launch_fit(P, smem, resident, fp, st, bf16);
+    e = launch_fit(P, L.smem, L.resident, fp, st, bf16);
     if (e == cudaSuccess) ctx->launches += 1;
     return e;
 }
@@ -593,7 +646,8 @@ int lr_create(lr_ctx** out, int32_t device, int32_t n_max) {
     if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&c->d_oscr), (size_t(n_max) + 2) * sizeof(double));
     if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&c->d_oticket), sizeof(unsigned int));
     if (e == cudaSuccess) e = cudaMemset(c->d_oticket, 0, sizeof(unsigned int));
-    if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&c->d_gbar), 2 * sizeof(unsigned int));
+    if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&c->d_gbar), 2 * kMaxWorld * sizeof(unsigned int));
+    if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&c->d_rank_params), kMaxWorld * sizeof(FitParams));
     if (e == cudaSuccess) {
         int l2 = 0;
         e = cudaDeviceGetAttribute(&l2, cudaDevAttrL2CacheSize, device);
@@ -617,6 +671,7 @@ int lr_create(lr_ctx** out, int32_t device, int32_t n_max) {
         if (c->d_oscr) cudaFree(c->d_oscr);
         if (c->d_oticket) cudaFree(c->d_oticket);
         if (c->d_gbar) cudaFree(c->d_gbar);
+        if (c->d_rank_params) cudaFree(c->d_rank_params);
         delete c;
         return rc != LR_OK ? rc : LR_ERR_CUDA;
     }
@@ -641,6 +696,7 @@ int lr_destroy(lr_ctx* ctx) {
         cudaFree(ctx->d_oscr);
         cudaFree(ctx->d_oticket);
         cudaFree(ctx->d_gbar);
+        cudaFree(ctx->d_rank_params);
         cudaFree(ctx->d_hX);
         cudaFree(ctx->d_hy);
         cudaFree(ctx->d_hw);
@@ -708,7 +764,7 @@ int loss_grad_impl(lr_ctx* ctx, const void* d_X, bool bf16, const float* d_y, in
     if (!d_y || !d_loss || !d_grad_w || !d_grad_b) return LR_ERR_NULL;
     if (!aligned(d_y, 4) || !aligned(d_loss, 4) || !aligned(d_grad_w, 4) || !aligned(d_grad_b, 4)) return LR_ERR_ALIGNMENT;
     lr_plan P;
-    rc = make_plan(m, n, aligned(d_X, 16), ctx->sm_count, &P, bf16);
+    rc = make_plan(m, n, aligned(d_X, 16), plan_sms(ctx), &P, bf16);
     if (rc != LR_OK) return rc;
     DeviceGuard g(ctx);
     if (!g.ok) return LR_ERR_CUDA;
@@ -730,7 +786,7 @@ int fit_impl(lr_ctx* ctx, const void* d_X, bool bf16, const float* d_y, int64_t 
     if (!aligned(d_y, 4) || (d_loss_hist && !aligned(d_loss_hist, 4))) return LR_ERR_ALIGNMENT;
     if (!std::isfinite(lr)) return LR_ERR_VALUE;
     lr_plan P;
-    rc = make_plan(m, n, aligned(d_X, 16), ctx->sm_count, &P, bf16);
+    rc = make_plan(m, n, aligned(d_X, 16), plan_sms(ctx), &P, bf16);
     if (rc != LR_OK) return rc;
     if (iters == 0) return LR_OK;
     DeviceGuard g(ctx);
@@ -763,7 +819,7 @@ int predict_impl(lr_ctx* ctx, const void* d_X, bool bf16, int64_t m, int32_t n, 
     if (!d_labels) return LR_ERR_NULL;
     if (!(thr > 0.f && thr < 1.f)) return LR_ERR_VALUE;
     lr_plan P;
-    rc = make_plan(m, n, aligned(d_X, 16), ctx->sm_count, &P, bf16);
+    rc = make_plan(m, n, aligned(d_X, 16), plan_sms(ctx), &P, bf16);
     if (rc != LR_OK) return rc;
     DeviceGuard g(ctx);
     if (!g.ok) return LR_ERR_CUDA;
@@ -811,7 +867,7 @@ int fit_tol_impl(lr_ctx* ctx, const void* d_X, bool bf16, const float* d_y, int6
         return LR_ERR_ALIGNMENT;
     if (!std::isfinite(lr) || !(eps >= 0.f) || !std::isfinite(eps)) return LR_ERR_VALUE;
     lr_plan P;
-    rc = make_plan(m, n, aligned(d_X, 16), ctx->sm_count, &P, bf16);
+    rc = make_plan(m, n, aligned(d_X, 16), plan_sms(ctx), &P, bf16);
     if (rc != LR_OK) return rc;
     *iters_done = 0;
     *grad_norm = -1.f;
@@ -878,7 +934,7 @@ int fit_opt_impl(lr_ctx* ctx, const void* d_X, bool bf16, const float* d_y, int6
     if (!std::isfinite(lr) || !(opt->l2 >= 0.f) || !std::isfinite(opt->l2) || !(opt->momentum >= 0.f && opt->momentum < 1.f))
         return LR_ERR_VALUE;
     lr_plan P;
-    rc = make_plan(m, n, aligned(d_X, 16), ctx->sm_count, &P, bf16);
+    rc = make_plan(m, n, aligned(d_X, 16), plan_sms(ctx), &P, bf16);
     if (rc != LR_OK) return rc;
     if (iters == 0) return LR_OK;
     DeviceGuard g(ctx);
@@ -926,7 +982,7 @@ int fit_sgd_impl(lr_ctx* ctx, const void* d_X, bool bf16, const float* d_y, int6
         const int64_t rows = std::min(batch_rows, m - r0);
         const void* Xb = static_cast<const unsigned char*>(d_X) + size_t(r0) * n * (bf16 ? 2 : 4);
         lr_plan P;
-        rc = make_plan(rows, n, aligned(Xb, 16), ctx->sm_count, &P, bf16);
+        rc = make_plan(rows, n, aligned(Xb, 16), plan_sms(ctx), &P, bf16);
         if (rc != LR_OK) return rc;
         Pass pass{Xb, d_y + r0, rows, n, d_w, d_b};
         pass.bf16 = bf16;
@@ -947,7 +1003,7 @@ int shard_sums_impl(lr_ctx* ctx, const void* d_X, bool bf16, const float* d_y, i
     if (!d_y || !d_sums) return LR_ERR_NULL;
     if (!aligned(d_y, 4) || !aligned(d_sums, 8)) return LR_ERR_ALIGNMENT;
     lr_plan P;
-    rc = make_plan(m_local, n, aligned(d_X, 16), ctx->sm_count, &P, bf16);
+    rc = make_plan(m_local, n, aligned(d_X, 16), plan_sms(ctx), &P, bf16);
     if (rc != LR_OK) return rc;
     DeviceGuard g(ctx);
     if (!g.ok) return LR_ERR_CUDA;
@@ -1147,6 +1203,134 @@ const char* lr_status_string(int code) {
         case LR_ERR_NOMEM: return "allocation failed";
         default: return "unknown status";
     }
+}
+
+}  // extern "C"
+
+// ------------------------------------------------------------------------------------------------------
+// Row-sharded fits with the exchange inside the persistent kernel.
+// ------------------------------------------------------------------------------------------------------
+namespace {
+
+int fit_sharded_impl(lr_ctx* ctx, const void* d_X, bool bf16, const float* d_y, int64_t m_local, int64_t m_total, int32_t n,
+                     float lr, int32_t iters, float* d_w, float* d_b, float* d_loss_hist, int32_t rank, int32_t world,
+                     void* const* d_exchange, int64_t epoch, int32_t wait_ms, void* stream) {
+    int rc = check_common(ctx, d_X, m_local, n, d_w, d_b, bf16);
+    if (rc != LR_OK) return rc;
+    if (!d_y || !d_exchange) return LR_ERR_NULL;
+    if (iters < 0 || world < 1 || world > kMaxWorld || rank < 0 || rank >= world || m_total < m_local || epoch < 0) return LR_ERR_SHAPE;
+    if (wait_ms < 1 || wait_ms > 60000 || !std::isfinite(lr)) return LR_ERR_VALUE;
+    for (int r = 0; r < world; ++r) {
+        if (!d_exchange[r]) return LR_ERR_NULL;
+        if (!aligned(d_exchange[r], 128)) return LR_ERR_ALIGNMENT;
+    }
+    if (!aligned(d_y, 4) || (d_loss_hist && !aligned(d_loss_hist, 4))) return LR_ERR_ALIGNMENT;
+    lr_plan P;
+    rc = make_plan(m_local, n, aligned(d_X, 16), plan_sms(ctx), &P, bf16);
+    if (rc != LR_OK) return rc;
+    if (P.variant != 0 || !ctx->coop || int64_t(iters) * P.grid >= (int64_t(1) << 32)) return LR_ERR_SHAPE;   // no persistent kernel for this shape
+    if (iters == 0) return LR_OK;
+    NvtxRange range("lr_fit_sharded");
+    DeviceGuard g(ctx);
+    if (!g.ok) return LR_ERR_CUDA;
+    const PersistentShard shard{rank, world, m_total, uint64_t(epoch), uint64_t(wait_ms) * 1000000ull, d_exchange};
+    const cudaError_t e = launch_persistent_fit(ctx, P, bf16, d_X, d_y, m_local, n, lr, iters, d_w, d_b, d_loss_hist, nullptr,
+                                                static_cast<cudaStream_t>(stream), &shard);
+    if (e != cudaSuccess) { ctx->last_cuda = int(e); cudaGetLastError(); return LR_ERR_CUDA; }
+    return LR_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int lr_exchange_bytes(int32_t world, int32_t n, int64_t* bytes) {
+    if (!bytes) return LR_ERR_NULL;
+    if (world < 1 || world > kMaxWorld || n < 1) return LR_ERR_SHAPE;
+    *bytes = exchange_buffer_bytes(world, n);
+    return LR_OK;
+}
+
+int lr_set_sm_limit(lr_ctx* ctx, int32_t sms) {
+    if (!ctx) return LR_ERR_NULL;
+    if (sms < 0) return LR_ERR_VALUE;
+    ctx->sm_limit = sms;
+    return LR_OK;
+}
+
+int lr_fit_sharded(lr_ctx* ctx, const float* d_X, const float* d_y, int64_t m_local, int64_t m_total, int32_t n, float lr,
+                   int32_t iters, float* d_w, float* d_b, float* d_loss_hist, int32_t rank, int32_t world,
+                   void* const* d_exchange, int64_t epoch, int32_t wait_ms, void* stream) {
+    return fit_sharded_impl(ctx, d_X, false, d_y, m_local, m_total, n, lr, iters, d_w, d_b, d_loss_hist, rank, world, d_exchange,
+                            epoch, wait_ms, stream);
+}
+
+int lr_fit_sharded_bf16(lr_ctx* ctx, const uint16_t* d_Xh, const float* d_y, int64_t m_local, int64_t m_total, int32_t n, float lr,
+                        int32_t iters, float* d_w, float* d_b, float* d_loss_hist, int32_t rank, int32_t world,
+                        void* const* d_exchange, int64_t epoch, int32_t wait_ms, void* stream) {
+    return fit_sharded_impl(ctx, d_Xh, true, d_y, m_local, m_total, n, lr, iters, d_w, d_b, d_loss_hist, rank, world, d_exchange,
+                            epoch, wait_ms, stream);
+}
+
+int lr_fit_sharded_local(lr_ctx* ctx, int32_t world, const float* const* d_X, const float* const* d_y, const int64_t* m_local,
+                         int32_t n, float lr, int32_t iters, float* const* d_w, float* const* d_b, float* const* d_loss_hist,
+                         void* const* d_exchange, int64_t epoch, int32_t wait_ms, void* stream) {
+    if (!ctx || !d_X || !d_y || !m_local || !d_w || !d_b || !d_exchange) return LR_ERR_NULL;
+    if (world < 2 || world > kMaxWorld || n < 1 || n > ctx->n_max || iters < 0 || epoch < 0) return LR_ERR_SHAPE;
+    if (wait_ms < 1 || wait_ms > 60000 || !std::isfinite(lr)) return LR_ERR_VALUE;
+    const int sms = plan_sms(ctx) / world;                                      // SMs (= CTAs) a rank may take
+    if (sms < 1 || !ctx->coop) return LR_ERR_SHAPE;
+    int64_t m_total = 0;
+    lr_plan P{};
+    int ctas = 0;
+    for (int r = 0; r < world; ++r) {
+        if (!d_X[r] || !d_y[r] || !d_w[r] || !d_b[r] || !d_exchange[r]) return LR_ERR_NULL;
+        if (m_local[r] < 1 || m_local[r] > kMaxRows) return LR_ERR_SHAPE;
+        if (!aligned(d_X[r], 16) || !aligned(d_y[r], 4) || !aligned(d_w[r], 4) || !aligned(d_b[r], 4) || !aligned(d_exchange[r], 128) ||
+            (d_loss_hist && d_loss_hist[r] && !aligned(d_loss_hist[r], 4)))
+            return LR_ERR_ALIGNMENT;
+        lr_plan Pr;
+        const int rc = make_plan(m_local[r], n, true, sms, &Pr);
+        if (rc != LR_OK) return rc;
+        if (Pr.variant != 0) return LR_ERR_SHAPE;
+        if (r == 0) P = Pr;
+        ctas = std::max(ctas, int(Pr.grid));
+        m_total += m_local[r];
+    }
+    if (int64_t(iters) * ctas >= (int64_t(1) << 32)) return LR_ERR_SHAPE;
+    if (size_t(world) * 2 * ctas * (size_t(n) + 2) > size_t(ctx->sm_count) * kMaxGridPerSm * (size_t(ctx->n_max) + 2)) return LR_ERR_SHAPE;
+    if (iters == 0) return LR_OK;
+    NvtxRange range("lr_fit_sharded_local");
+    DeviceGuard g(ctx);
+    if (!g.ok) return LR_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    // one shared-memory shape for all ranks: the deepest pipeline any of them wants; resident only if all of them are
+    FitLayout L{1, true, 0};
+    for (int r = 0; r < world; ++r) {
+        const FitLayout Lr = fit_layout(P, false, m_local[r], n, ctas);
+        L.depth = std::max(L.depth, Lr.depth);
+        L.resident = L.resident && Lr.resident;
+        L.smem = std::max(L.smem, Lr.smem);
+    }
+    std::vector<FitParams> h(static_cast<size_t>(world));
+    for (int r = 0; r < world; ++r) {
+        const PersistentShard shard{r, world, m_total, uint64_t(epoch), uint64_t(wait_ms) * 1000000ull, d_exchange};
+        h[r] = fit_params(ctx, P, false, d_X[r], d_y[r], m_local[r], n, lr, iters, d_w[r], d_b[r],
+                          d_loss_hist ? d_loss_hist[r] : nullptr, L.depth, nullptr, &shard);
+        h[r].partial = ctx->d_partial + size_t(r) * 2 * ctas * (size_t(n) + 2);   // every rank its own partial rows ...
+        h[r].gbar = ctx->d_gbar + 2 * r;                                         // ... and barrier words
+        h[r].keep_rows = 0;
+    }
+    LR_CK(ctx, cudaMemsetAsync(ctx->d_gbar, 0, 2 * kMaxWorld * sizeof(unsigned int), st));
+    LR_CK(ctx, cudaMemcpyAsync(ctx->d_rank_params, h.data(), sizeof(FitParams) * world, cudaMemcpyHostToDevice, st));
+    LR_CK(ctx, cudaStreamSynchronize(st));          // the host copy of the parameters must outlive the (pageable) transfer
+    lr_plan Pl = P;
+    Pl.grid = ctas;
+    const cudaError_t e = launch_fit_ranks(Pl, L.smem, L.resident, ctx->d_rank_params, world, ctas, st);
+    if (e == cudaErrorInvalidValue) { cudaGetLastError(); return LR_ERR_SHAPE; }
+    if (e != cudaSuccess) { ctx->last_cuda = int(e); cudaGetLastError(); return LR_ERR_CUDA; }
+    ctx->launches += 1;
+    return LR_OK;
 }
 
 }  // extern "C"

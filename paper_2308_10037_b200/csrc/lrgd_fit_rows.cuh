@@ -22,6 +22,15 @@
 // With a tolerance (lr_fit_tol) the kernel also forms ||grad||_2 after every update and all CTAs leave the loop together
 // once it is <= eps: the stopping rule of Algorithm 7 with no host round trip and no wasted launch.
 //
+// Row shards on several GPUs (lr_fit_sharded): every rank runs this kernel on its own rows.  After the grid barrier CTA 0
+// of a rank adds up the rank's partial rows, stores the n+2 sums into slot [t & 1][rank] of EVERY rank's exchange buffer
+// (plain stores through peer mappings; no multicast, no bulk copies from or to a peer) and then publishes the step
+// number in flag [rank] of every buffer with a system-scope release.  All CTAs of a rank wait (bounded) until the flags
+// of all ranks in their own buffer show the step, add the `world` vectors in k_reduce_update's fixed order -- the order
+// lr_apply_sums uses, so every rank gets the same bits -- and update their copy of the parameters.  The slots alternate
+// with the parity of the step: a rank can only be one step ahead of the slowest one (it needs that rank's flag to go
+// on), so the slot it overwrites has been read by everybody.
+//
 // Grid barrier: a monotonic counter in global memory; thread 0 of each CTA adds one and spins (bounded, 2 s) until the
 // counter reaches grid * k.  A second word next to the counter is the run's abort flag: a CTA whose wait expires (here
 // or on a stage) raises it, every other CTA sees it in its own wait, and all of them stop iterating, wait (bounded) for
@@ -56,6 +65,9 @@ constexpr int kFitChunkPairs = 32;             // column pairs per chunk of the 
 #endif
 static_assert(LRGD_FIT_RED_CHUNKS * kFitMaxWarps * 2 * kFitChunkPairs <= kFitMaxWarps * kFitCombineCols, "the reduction reuses the combine buffer");
 
+constexpr int kMaxWorld = 32;                  // ranks of a row-sharded fit (one slice of the fixed summation tree each)
+static_assert(kMaxWorld <= kRedSlices, "one reduction slice per rank");
+
 struct FitParams {
     const void* X;             // fp32 or bfloat16 [m][n], row-major
     const float* y;
@@ -77,7 +89,30 @@ struct FitParams {
     TolState* tol;
     double eps;
     float* gnorm_hist;         // nullable [iters]
+    // row shards (world == 0: a fit on one GPU, nothing below is used)
+    int rank, world;
+    unsigned long long epoch;  // steps exchanged through these buffers before this launch (the same on every rank)
+    unsigned long long wait_ns;               // bound on each wait for the other ranks
+    unsigned char* xbuf[kMaxWorld];           // exchange buffer of every rank as this rank addresses it; [rank] is its own
 };
+
+// Layout of one rank's exchange buffer: one 8-byte step flag per source rank, 128 bytes apart; then two slots
+// (step parity) of `world` vectors of n+2 doubles, each vector padded to a multiple of 128 bytes.
+__host__ __device__ constexpr long long exchange_vector_bytes(int n) { return ((n + 2) * 8LL + 127) / 128 * 128; }
+__host__ __device__ constexpr long long exchange_flag_offset(int src) { return 128LL * src; }
+__host__ __device__ constexpr long long exchange_slot_offset(int world, int n, int parity, int src) {
+    return 128LL * world + (static_cast<long long>(parity) * world + src) * exchange_vector_bytes(n);
+}
+__host__ __device__ constexpr long long exchange_buffer_bytes(int world, int n) { return exchange_slot_offset(world, n, 2, 0); }
+
+__device__ __forceinline__ unsigned long long ld_relaxed_sys_u64(const unsigned long long* p) {
+    unsigned long long v;
+    asm volatile("ld.relaxed.sys.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_release_sys_u64(unsigned long long* p, unsigned long long v) {
+    asm volatile("st.release.sys.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
+}
 
 __device__ __forceinline__ unsigned int ld_relaxed_u32(const unsigned int* p) {
     unsigned int v;
@@ -222,8 +257,66 @@ __device__ LRGD_FIT_RED_INLINE void reduce_partial_rows(const double* pbuf, int 
     }
 }
 
+// The exchange of a row-sharded step, called by all threads of every CTA after the rank's grid barrier; leaves the global
+// sums in sums[stride].  Returns false if a wait for another rank expired (the CTA's abort flag is then up).
+template <int NW>
+__device__ LRGD_FIT_RED_INLINE bool exchange_rank_sums(const FitParams& p, int cta, int G, int stride, int t, double* buf, double* sums,
+                                                      volatile int* cta_abort) {
+    const unsigned long long step = p.epoch + static_cast<unsigned long long>(t) + 1ull;
+    const int parity = static_cast<int>(step & 1ull);
+    if (cta == 0) {
+        // this rank's sums, then one copy of them into every rank's buffer, then the flags
+        reduce_partial_rows<NW>(p.partial + static_cast<size_t>(t & 1) * G * stride, G, stride, buf, sums);
+        for (int r = 0; r < p.world; ++r) {
+            double* dst = reinterpret_cast<double*>(p.xbuf[r] + exchange_slot_offset(p.world, p.n, parity, p.rank));
+            for (int c = threadIdx.x; c < stride; c += NW * 32) dst[c] = sums[c];
+        }
+        __syncthreads();
+        if (threadIdx.x < p.world) {
+            __threadfence_system();                // the stores of the whole CTA (ordered by the barrier above) before the flag
+            st_release_sys_u64(reinterpret_cast<unsigned long long*>(p.xbuf[threadIdx.x] + exchange_flag_offset(p.rank)), step);
+        }
+    }
+    // wait for every rank's flag in this rank's own buffer
+    if (threadIdx.x < p.world) {
+        const unsigned long long* flag = reinterpret_cast<const unsigned long long*>(p.xbuf[p.rank] + exchange_flag_offset(threadIdx.x));
+        if (ld_relaxed_sys_u64(flag) < step) {
+            const unsigned long long t0 = global_timer_ns();
+            for (;;) {
+                bool there = false;
+#pragma unroll 1
+                for (int i = 0; i < 64 && !there; ++i) there = ld_relaxed_sys_u64(flag) >= step;
+                if (there) break;
+                if (*cta_abort || ld_relaxed_u32(p.gbar + 1) != 0u || global_timer_ns() - t0 > p.wait_ns) {
+                    atomicExch(p.gbar + 1, 1u);
+                    atomicExch(p.status, kStatusTimeout);
+                    *cta_abort = 1;
+                    break;
+                }
+            }
+        }
+        __threadfence_system();                    // acquire side: the other ranks' vectors are read after this
+    }
+    __syncthreads();
+    if (*cta_abort) return false;
+    // the `world` vectors in k_reduce_update's order for `world` rows: one row per slice, then the fixed tree
+    const unsigned char* own = p.xbuf[p.rank];
+    for (int c = threadIdx.x; c < stride; c += NW * 32) {
+        double sl[kRedSlices];
+#pragma unroll
+        for (int r = 0; r < kRedSlices; ++r) {
+            double v = 0.0;
+            if (r < p.world) v += __ldcg(reinterpret_cast<const double*>(own + exchange_slot_offset(p.world, p.n, parity, r)) + c);
+            sl[r] = v;
+        }
+        sums[c] = slice_tree_sum(sl);
+    }
+    __syncthreads();
+    return true;
+}
+
 template <class E, int NV, int LPR, int RB, int NW, bool RESIDENT>
-__global__ void __launch_bounds__(NW * 32, 1) k_fit_rows(const FitParams p) {
+__device__ __forceinline__ void fit_rows_body(const FitParams& p, const int cta, const int G) {
     constexpr int EPG = E::EPG;
     constexpr int RPW = 32 / LPR;
     constexpr int RPB = RB * RPW;
@@ -245,7 +338,6 @@ __global__ void __launch_bounds__(NW * 32, 1) k_fit_rows(const FitParams p) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int D = p.depth;
     const int n = p.n, n4 = n / EPG;                   // n4 = 16-byte groups per row
-    const int G = gridDim.x, cta = blockIdx.x;
     const int stride = n + 2;                          // doubles per partial row (even: n is a multiple of four)
     const uint32_t row_bytes = static_cast<uint32_t>(n) * E::BYTES;
     const uint32_t stage_stride = (static_cast<uint32_t>(RPB) * row_bytes + 127u) & ~127u;
@@ -442,8 +534,13 @@ __global__ void __launch_bounds__(NW * 32, 1) k_fit_rows(const FitParams p) {
         alive = grid_barrier(p.gbar, static_cast<unsigned int>(G) * barrier_no, p.status, abort_flag);
         if (!alive) break;
 
-        // ---- reduction, by every CTA for itself (see reduce_partial_rows) ----
-        reduce_partial_rows<NW>(p.partial + static_cast<size_t>(t & 1) * G * stride, G, stride, red, sum_s);
+        // ---- reduction, by every CTA for itself (see reduce_partial_rows); with row shards on several GPUs the exchange ----
+        if (p.world == 0) {
+            reduce_partial_rows<NW>(p.partial + static_cast<size_t>(t & 1) * G * stride, G, stride, red, sum_s);
+        } else {
+            alive = exchange_rank_sums<NW>(p, cta, G, stride, t, red, sum_s, abort_flag);
+            if (!alive) break;
+        }
 
         // ---- update (the arithmetic of k_reduce_update), every CTA on its own copy; CTA 0 keeps the history ----
         for (int c = threadIdx.x; c < stride; c += NW * 32) {
@@ -499,6 +596,22 @@ __global__ void __launch_bounds__(NW * 32, 1) k_fit_rows(const FitParams p) {
         }
         __syncwarp();
     }
+}
+
+template <class E, int NV, int LPR, int RB, int NW, bool RESIDENT>
+__global__ void __launch_bounds__(NW * 32, 1) k_fit_rows(const __grid_constant__ FitParams p) {
+    // (__grid_constant__: the exchange takes the parameters by reference; without it the kernel would keep a copy of the
+    // whole block in local memory and read its fields from there)
+    fit_rows_body<E, NV, LPR, RB, NW, RESIDENT>(p, blockIdx.x, gridDim.x);
+}
+
+// Several ranks of a row-sharded fit as groups of CTAs of ONE cooperative launch on one GPU: CTAs
+// [r * ctas_per_rank, (r + 1) * ctas_per_rank) play rank r with the parameters ranks[r] (its own rows, partial rows, barrier
+// words and exchange buffer).  All CTAs are co-resident, so ranks that wait on one another cannot starve each other; the
+// exchange runs exactly as it does between GPUs.  This is how the multi-rank path is exercised where only one GPU is there.
+template <class E, int NV, int LPR, int RB, int NW, bool RESIDENT>
+__global__ void __launch_bounds__(NW * 32, 1) k_fit_rows_ranks(const FitParams* ranks, int ctas_per_rank) {
+    fit_rows_body<E, NV, LPR, RB, NW, RESIDENT>(ranks[blockIdx.x / ctas_per_rank], blockIdx.x % ctas_per_rank, ctas_per_rank);
 }
 
 }  // namespace lrgd

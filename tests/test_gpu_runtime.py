@@ -92,6 +92,20 @@ def test_sharded_driver_on_a_one_rank_nccl_group(ctx):
         # one shard, one rank: the same kernels and the same summation order as lr_fit -> identical bits
         wf, bf = api.lr_fit(dX, dy, wl.lr, 8, ctx=ctx)
         assert torch.equal(w, wf) and torch.equal(b, bf)
+        # and the fused form on the same one-rank group: exchange buffer in symmetric memory, one launch for all steps
+        try:
+            ex = parallel.ExchangeBuffers(wl.n, torch.device("cuda", 0))
+        except Exception as err:                                  # symmetric memory is not available everywhere
+            ex = None
+            print("symmetric memory unavailable:", err)
+        if ex is not None:
+            w2 = torch.zeros(wl.n, device="cuda")
+            b2 = torch.zeros(1, device="cuda")
+            parallel.fit_sharded_fused(ctx, dX, dy, wl.m, wl.lr, 5, w2, b2, ex)
+            parallel.fit_sharded_fused(ctx, dX, dy, wl.m, wl.lr, 3, w2, b2, ex)
+            torch.cuda.synchronize()
+            assert ex.epoch == 8 and torch.equal(w2, wf) and torch.equal(b2, bf)
+            assert ctx.device_status() == 0
     finally:
         dist.destroy_process_group()
 
