@@ -280,7 +280,7 @@ def main():
     ap.add_argument("--l2-keep-mb", type=float, default=-1.0, help="MB of X to keep in L2 across iterations (-1: library default, 0: off)")
     ap.add_argument("--x-dtype", default="f32", choices=["f32", "bf16"],
                     help="storage type of X on the device: bf16 runs the bfloat16 entry points on lr_convert_bf16's output "
-                         "(half the bytes per pass; no end-to-end or CPU leg)")
+                         "(half the bytes per pass)")
     ap.add_argument("--fused-exchange", action="store_true",
                     help="--gpus N > 1: exchange the sums inside the persistent kernel (lr_fit_sharded over symmetric memory) "
                          "instead of one NCCL all-gather per iteration")
@@ -349,7 +349,6 @@ def main():
         dX = ctx.convert_bf16(dX32)                 # the fits below read the bfloat16 matrix only
         torch.cuda.synchronize()
         del dX32
-        args.no_e2e = args.no_cpu_baseline = True
     elem_bytes = 2 if bf16 else 4
 
     exchange = parallel.ExchangeBuffers(wl.n, torch.device("cuda", local_rank)) if world > 1 and args.fused_exchange else None
@@ -462,12 +461,13 @@ def main():
         for rep in range(4):
             wh.zero_(); bh.zero_()
             t0 = time.perf_counter()
-            ctx.fit_host(Xh, yh, wl.lr, wl.iters, wh, bh)
+            ctx.fit_host(Xh, yh, wl.lr, wl.iters, wh, bh, store_bf16=bf16)
             times.append(time.perf_counter() - t0)
         t_e2e = statistics.median(times[1:])
-        e2e = {"value": wl.iters / t_e2e, "unit": UNIT, "h2d_bytes_per_step": (bytes_per_launch + 4 * wl.n + 4) / wl.iters,
+        e2e = {"value": wl.iters / t_e2e, "unit": UNIT, "h2d_bytes_per_step": (4 * wl.m * wl.n + 4 * wl.m + 4 * wl.n + 4) / wl.iters,
                "d2h_bytes_per_step": (4 * wl.n + 4) / wl.iters, "seconds_per_fit": t_e2e,
-               "what": f"lr_fit_host: pinned X, y copied in, {wl.iters} iterations, w, b copied out; median of 3"}
+               "what": (f"lr_fit_host{'_bf16' if bf16 else ''}: pinned fp32 X, y copied in, "
+                        + ("X rounded to bfloat16 on the device, " if bf16 else "") + f"{wl.iters} iterations, w, b copied out; median of 3")}
 
     # ---- workloads that ask for it: the workload's own fit from zero, then predict at its threshold and F1 against y ----
     predict = None
@@ -490,7 +490,13 @@ def main():
     # ---- CPU checker on this host's cores (reported baseline, not a target) ----
     cpu = None
     if not args.no_cpu_baseline and world == 1:
-        rate, what, threads = oracle_rate(X_np, y_np, wl, budget_s=15.0)
+        X_cpu = X_np
+        if bf16:                                    # the checker runs on the values the device streams: X rounded to bfloat16
+            import oracle
+            X_cpu = oracle.round_bf16(X_np)[1]
+        rate, what, threads = oracle_rate(X_cpu, y_np, wl, budget_s=15.0)
+        if bf16:
+            what += " (X rounded to bfloat16 by the checker)"
         cpu = {"value": rate, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": what}
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,

@@ -72,7 +72,9 @@ int lr_plan_query(int64_t m, int32_t n, int32_t x_aligned16, int32_t sm_count, l
 
 /*
  * Creates a context on CUDA device `device` with workspace for problems of up to n_max columns
- * (any m).  Allocates the per-CTA partial-sum buffer and the device status word.
+ * (any m: the workspace is one row of n_max + 2 sums per CTA and a few words of state, so the number of rows
+ * of a problem needs no bound here).  Allocates the per-CTA partial-sum buffer and the device status word.
+ * Every computing call runs inside a named NVTX range (lr_fit, lr_fit_tol, ...), visible on a profiler's timeline.
  * Errors: LR_ERR_NULL (out), LR_ERR_SHAPE (n_max < 1), LR_ERR_CUDA, LR_ERR_NOMEM.
  */
 int lr_create(lr_ctx** out, int32_t device, int32_t n_max);
@@ -318,6 +320,13 @@ int lr_fit_host(lr_ctx* ctx, const float* h_X, const float* h_y, int64_t m, int3
                 float lr, int32_t iters, float* h_w, float* h_b, float* h_loss_hist);
 int lr_predict_host(lr_ctx* ctx, const float* h_X, int64_t m, int32_t n,
                     const float* h_w, const float* h_b, float thr, uint8_t* h_labels);
+/* The same with X stored as bfloat16 on the device: h_X is fp32 as above, it is copied in and rounded once on the device
+ * (lr_convert_bf16), and the bfloat16 entry points run on the rounded matrix (half the bytes per pass; the result is what
+ * lr_fit / lr_predict give on the matrix of rounded values). */
+int lr_fit_host_bf16(lr_ctx* ctx, const float* h_X, const float* h_y, int64_t m, int32_t n,
+                     float lr, int32_t iters, float* h_w, float* h_b, float* h_loss_hist);
+int lr_predict_host_bf16(lr_ctx* ctx, const float* h_X, int64_t m, int32_t n,
+                         const float* h_w, const float* h_b, float thr, uint8_t* h_labels);
 
 /*
  * Per-kernel timing for measurement.  While enabled, lr_loss_grad / lr_fit / lr_predict bracket every

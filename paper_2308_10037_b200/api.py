@@ -24,7 +24,7 @@ EXPORTS = ["lr_plan_query", "lr_create", "lr_destroy", "lr_loss_grad", "lr_fit",
            "lr_last_cuda_error", "lr_status_string", "lr_loss_grad_noalloc", "lr_fit_tol", "lr_fit_opt", "lr_selftest_wait", "lr_set_persistent", "lr_fit_sgd", "lr_set_l2_keep",
            "lr_convert_bf16", "lr_loss_grad_bf16", "lr_fit_bf16", "lr_predict_bf16", "lr_plan_query_bf16",
            "lr_fit_tol_bf16", "lr_fit_opt_bf16", "lr_fit_sgd_bf16", "lr_shard_sums_bf16", "lr_set_overlap",
-           "lr_exchange_bytes", "lr_fit_sharded", "lr_fit_sharded_bf16", "lr_fit_sharded_local", "lr_set_sm_limit"]
+           "lr_fit_host_bf16", "lr_predict_host_bf16", "lr_exchange_bytes", "lr_fit_sharded", "lr_fit_sharded_bf16", "lr_fit_sharded_local", "lr_set_sm_limit"]
 
 
 class LrPlan(ctypes.Structure):
@@ -91,6 +91,8 @@ def lib() -> ctypes.CDLL:
         L.lr_loss_grad_noalloc.argtypes = [I32, P, P, I64, I32, P, P, P, P, P, P, P]
         L.lr_fit_host.argtypes = [P, P, P, I64, I32, F, I32, P, P, P]
         L.lr_predict_host.argtypes = [P, P, I64, I32, P, P, F, P]
+        L.lr_fit_host_bf16.argtypes = L.lr_fit_host.argtypes
+        L.lr_predict_host_bf16.argtypes = L.lr_predict_host.argtypes
         L.lr_profile_enable.argtypes = [P, I32]
         L.lr_profile_read.argtypes = [P, ctypes.POINTER(I32), ctypes.POINTER(ctypes.c_double)]
         L.lr_launch_count.argtypes = [P, ctypes.POINTER(I64)]
@@ -375,21 +377,25 @@ class Context:
         self._check(lib().lr_set_sm_limit(self._h, int(sms or 0)), "lr_set_sm_limit")
 
     # ---- host-pointer entry points ---------------------------------------------------------------
-    def fit_host(self, X, y, lr, iters, w, b, loss_hist=None):
-        """X, y, w, b (and loss_hist) are CPU tensors or numpy arrays; w, b are updated in place."""
+    def fit_host(self, X, y, lr, iters, w, b, loss_hist=None, store_bf16=False):
+        """X, y, w, b (and loss_hist) are CPU tensors or numpy arrays; w, b are updated in place.
+
+        ``store_bf16``: X (fp32 on the host) is rounded to bfloat16 on the device after the copy and the fit streams that.
+        """
         m, n = _shape2(X)
         F32, iters = torch.float32, int(iters)
-        rc = lib().lr_fit_host(self._h, _host_ptr(X, F32, "X"), _host_ptr(y, F32, "y", m), m, n, float(lr), iters,
-                               _host_ptr(w, F32, "w", n), _host_ptr(b, F32, "b", 1),
-                               _host_ptr(loss_hist, F32, "loss_hist", max(iters, 0)))
-        self._check(rc, "lr_fit_host")
+        fn = lib().lr_fit_host_bf16 if store_bf16 else lib().lr_fit_host
+        rc = fn(self._h, _host_ptr(X, F32, "X"), _host_ptr(y, F32, "y", m), m, n, float(lr), iters,
+                _host_ptr(w, F32, "w", n), _host_ptr(b, F32, "b", 1), _host_ptr(loss_hist, F32, "loss_hist", max(iters, 0)))
+        self._check(rc, "lr_fit_host_bf16" if store_bf16 else "lr_fit_host")
 
-    def predict_host(self, X, w, b, thr, labels):
+    def predict_host(self, X, w, b, thr, labels, store_bf16=False):
         m, n = _shape2(X)
         F32 = torch.float32
-        rc = lib().lr_predict_host(self._h, _host_ptr(X, F32, "X"), m, n, _host_ptr(w, F32, "w", n), _host_ptr(b, F32, "b", 1),
-                                   float(thr), _host_ptr(labels, torch.uint8, "labels", m))
-        self._check(rc, "lr_predict_host")
+        fn = lib().lr_predict_host_bf16 if store_bf16 else lib().lr_predict_host
+        rc = fn(self._h, _host_ptr(X, F32, "X"), m, n, _host_ptr(w, F32, "w", n), _host_ptr(b, F32, "b", 1),
+                float(thr), _host_ptr(labels, torch.uint8, "labels", m))
+        self._check(rc, "lr_predict_host_bf16" if store_bf16 else "lr_predict_host")
 
     # ---- measurement / status --------------------------------------------------------------------
     def profile_enable(self, on: bool = True):

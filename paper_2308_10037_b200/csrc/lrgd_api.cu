@@ -180,6 +180,7 @@ struct lr_ctx {
     void* d_hy = nullptr; size_t hy_bytes = 0;
     void* d_hw = nullptr; size_t hw_bytes = 0;      // w[n] | b | loss_hist
     void* d_hl = nullptr; size_t hl_bytes = 0;      // labels
+    void* d_hXh = nullptr; size_t hXh_bytes = 0;    // bfloat16 copy of X (lr_fit_host_bf16, lr_predict_host_bf16)
     cudaStream_t hstream = nullptr;
     // profiling
     bool prof = false;
@@ -701,6 +702,7 @@ int lr_destroy(lr_ctx* ctx) {
         cudaFree(ctx->d_hy);
         cudaFree(ctx->d_hw);
         cudaFree(ctx->d_hl);
+        cudaFree(ctx->d_hXh);
     }
     delete ctx;
     return LR_OK;
@@ -789,6 +791,7 @@ int fit_impl(lr_ctx* ctx, const void* d_X, bool bf16, const float* d_y, int64_t 
     rc = make_plan(m, n, aligned(d_X, 16), plan_sms(ctx), &P, bf16);
     if (rc != LR_OK) return rc;
     if (iters == 0) return LR_OK;
+    NvtxRange range(bf16 ? "lr_fit_bf16" : "lr_fit");
     DeviceGuard g(ctx);
     if (!g.ok) return LR_ERR_CUDA;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -872,6 +875,7 @@ int fit_tol_impl(lr_ctx* ctx, const void* d_X, bool bf16, const float* d_y, int6
     *iters_done = 0;
     *grad_norm = -1.f;
     if (max_iters == 0) return LR_OK;
+    NvtxRange range(bf16 ? "lr_fit_tol_bf16" : "lr_fit_tol");
     DeviceGuard g(ctx);
     if (!g.ok) return LR_ERR_CUDA;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -937,6 +941,7 @@ int fit_opt_impl(lr_ctx* ctx, const void* d_X, bool bf16, const float* d_y, int6
     rc = make_plan(m, n, aligned(d_X, 16), plan_sms(ctx), &P, bf16);
     if (rc != LR_OK) return rc;
     if (iters == 0) return LR_OK;
+    NvtxRange range(bf16 ? "lr_fit_opt_bf16" : "lr_fit_opt");
     DeviceGuard g(ctx);
     if (!g.ok) return LR_ERR_CUDA;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -972,6 +977,7 @@ int fit_sgd_impl(lr_ctx* ctx, const void* d_X, bool bf16, const float* d_y, int6
     if (!aligned(d_y, 4) || (d_loss_hist && !aligned(d_loss_hist, 4))) return LR_ERR_ALIGNMENT;
     if (!std::isfinite(lr)) return LR_ERR_VALUE;
     if (steps == 0) return LR_OK;
+    NvtxRange range(bf16 ? "lr_fit_sgd_bf16" : "lr_fit_sgd");
     DeviceGuard g(ctx);
     if (!g.ok) return LR_ERR_CUDA;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -1014,6 +1020,83 @@ int shard_sums_impl(lr_ctx* ctx, const void* d_X, bool bf16, const float* d_y, i
     if (rc != LR_OK) return rc;
     return launch_reduce(ctx, ctx->d_partial, P.grid, m_local, n, 0.0, false, nullptr, nullptr, nullptr, nullptr, nullptr,
                          d_sums, st);
+}
+
+// Host-pointer fits and predictions: copy in, run the device entry points on the context's own stream, copy out.
+// store_bf16: X arrives as fp32 and is rounded to bfloat16 on the device right after the copy (lr_convert_bf16); the
+// bfloat16 entry points then stream half the bytes per pass.
+int stage_host_x(lr_ctx* ctx, const float* h_X, int64_t m, int32_t n, bool store_bf16, cudaStream_t st, const void** d_X) {
+    const size_t xb = size_t(m) * n * 4;
+    int rc;
+    if ((rc = grow(ctx, &ctx->d_hX, &ctx->hX_bytes, xb)) != LR_OK) return rc;
+    LR_CK(ctx, cudaMemcpyAsync(ctx->d_hX, h_X, xb, cudaMemcpyHostToDevice, st));
+    *d_X = ctx->d_hX;
+    if (store_bf16) {
+        if ((rc = grow(ctx, &ctx->d_hXh, &ctx->hXh_bytes, xb / 2)) != LR_OK) return rc;
+        rc = lr_convert_bf16(ctx, static_cast<const float*>(ctx->d_hX), m * n, static_cast<uint16_t*>(ctx->d_hXh), st);
+        if (rc != LR_OK) return rc;
+        *d_X = ctx->d_hXh;
+    }
+    return LR_OK;
+}
+
+int fit_host_impl(lr_ctx* ctx, const float* h_X, bool store_bf16, const float* h_y, int64_t m, int32_t n, float lr, int32_t iters,
+                  float* h_w, float* h_b, float* h_loss_hist) {
+    int rc = check_common(ctx, h_X, m, n, h_w, h_b);
+    if (rc != LR_OK) return rc;
+    if (!h_y) return LR_ERR_NULL;
+    if (iters < 0) return LR_ERR_SHAPE;
+    if (!std::isfinite(lr)) return LR_ERR_VALUE;
+    NvtxRange range(store_bf16 ? "lr_fit_host_bf16" : "lr_fit_host");
+    DeviceGuard g(ctx);
+    if (!g.ok) return LR_ERR_CUDA;
+    const size_t yb = size_t(m) * 4;
+    const size_t wb = (size_t(n) + 1 + size_t(iters)) * 4;
+    if ((rc = grow(ctx, &ctx->d_hy, &ctx->hy_bytes, yb)) != LR_OK) return rc;
+    if ((rc = grow(ctx, &ctx->d_hw, &ctx->hw_bytes, wb)) != LR_OK) return rc;
+    float* dy = static_cast<float*>(ctx->d_hy);
+    float* dw = static_cast<float*>(ctx->d_hw);
+    float* db = dw + n;
+    float* dh = db + 1;
+    cudaStream_t st = ctx->hstream;
+    const void* dX = nullptr;
+    if ((rc = stage_host_x(ctx, h_X, m, n, store_bf16, st, &dX)) != LR_OK) return rc;
+    LR_CK(ctx, cudaMemcpyAsync(dy, h_y, yb, cudaMemcpyHostToDevice, st));
+    LR_CK(ctx, cudaMemcpyAsync(dw, h_w, size_t(n) * 4, cudaMemcpyHostToDevice, st));
+    LR_CK(ctx, cudaMemcpyAsync(db, h_b, 4, cudaMemcpyHostToDevice, st));
+    rc = fit_impl(ctx, dX, store_bf16, dy, m, n, lr, iters, dw, db, h_loss_hist ? dh : nullptr, st);
+    if (rc != LR_OK) return rc;
+    LR_CK(ctx, cudaMemcpyAsync(h_w, dw, size_t(n) * 4, cudaMemcpyDeviceToHost, st));
+    LR_CK(ctx, cudaMemcpyAsync(h_b, db, 4, cudaMemcpyDeviceToHost, st));
+    if (h_loss_hist && iters > 0) LR_CK(ctx, cudaMemcpyAsync(h_loss_hist, dh, size_t(iters) * 4, cudaMemcpyDeviceToHost, st));
+    LR_CK(ctx, cudaStreamSynchronize(st));
+    return LR_OK;
+}
+
+int predict_host_impl(lr_ctx* ctx, const float* h_X, bool store_bf16, int64_t m, int32_t n, const float* h_w, const float* h_b,
+                      float thr, uint8_t* h_labels) {
+    int rc = check_common(ctx, h_X, m, n, h_w, h_b);
+    if (rc != LR_OK) return rc;
+    if (!h_labels) return LR_ERR_NULL;
+    if (!(thr > 0.f && thr < 1.f)) return LR_ERR_VALUE;
+    NvtxRange range(store_bf16 ? "lr_predict_host_bf16" : "lr_predict_host");
+    DeviceGuard g(ctx);
+    if (!g.ok) return LR_ERR_CUDA;
+    if ((rc = grow(ctx, &ctx->d_hw, &ctx->hw_bytes, (size_t(n) + 1) * 4)) != LR_OK) return rc;
+    if ((rc = grow(ctx, &ctx->d_hl, &ctx->hl_bytes, size_t(m))) != LR_OK) return rc;
+    float* dw = static_cast<float*>(ctx->d_hw);
+    float* db = dw + n;
+    uint8_t* dl = static_cast<uint8_t*>(ctx->d_hl);
+    cudaStream_t st = ctx->hstream;
+    const void* dX = nullptr;
+    if ((rc = stage_host_x(ctx, h_X, m, n, store_bf16, st, &dX)) != LR_OK) return rc;
+    LR_CK(ctx, cudaMemcpyAsync(dw, h_w, size_t(n) * 4, cudaMemcpyHostToDevice, st));
+    LR_CK(ctx, cudaMemcpyAsync(db, h_b, 4, cudaMemcpyHostToDevice, st));
+    rc = predict_impl(ctx, dX, store_bf16, m, n, dw, db, thr, dl, st);
+    if (rc != LR_OK) return rc;
+    LR_CK(ctx, cudaMemcpyAsync(h_labels, dl, size_t(m), cudaMemcpyDeviceToHost, st));
+    LR_CK(ctx, cudaStreamSynchronize(st));
+    return LR_OK;
 }
 
 }  // namespace
@@ -1078,62 +1161,22 @@ int lr_apply_sums(lr_ctx* ctx, const double* d_sums_all, int32_t parts, int64_t 
 
 int lr_fit_host(lr_ctx* ctx, const float* h_X, const float* h_y, int64_t m, int32_t n, float lr, int32_t iters,
                 float* h_w, float* h_b, float* h_loss_hist) {
-    int rc = check_common(ctx, h_X, m, n, h_w, h_b);
-    if (rc != LR_OK) return rc;
-    if (!h_y) return LR_ERR_NULL;
-    if (iters < 0) return LR_ERR_SHAPE;
-    if (!std::isfinite(lr)) return LR_ERR_VALUE;
-    DeviceGuard g(ctx);
-    if (!g.ok) return LR_ERR_CUDA;
-    const size_t xb = size_t(m) * n * 4, yb = size_t(m) * 4;
-    const size_t wb = (size_t(n) + 1 + size_t(iters)) * 4;
-    if ((rc = grow(ctx, &ctx->d_hX, &ctx->hX_bytes, xb)) != LR_OK) return rc;
-    if ((rc = grow(ctx, &ctx->d_hy, &ctx->hy_bytes, yb)) != LR_OK) return rc;
-    if ((rc = grow(ctx, &ctx->d_hw, &ctx->hw_bytes, wb)) != LR_OK) return rc;
-    float* dX = static_cast<float*>(ctx->d_hX);
-    float* dy = static_cast<float*>(ctx->d_hy);
-    float* dw = static_cast<float*>(ctx->d_hw);
-    float* db = dw + n;
-    float* dh = db + 1;
-    cudaStream_t st = ctx->hstream;
-    LR_CK(ctx, cudaMemcpyAsync(dX, h_X, xb, cudaMemcpyHostToDevice, st));
-    LR_CK(ctx, cudaMemcpyAsync(dy, h_y, yb, cudaMemcpyHostToDevice, st));
-    LR_CK(ctx, cudaMemcpyAsync(dw, h_w, size_t(n) * 4, cudaMemcpyHostToDevice, st));
-    LR_CK(ctx, cudaMemcpyAsync(db, h_b, 4, cudaMemcpyHostToDevice, st));
-    rc = lr_fit(ctx, dX, dy, m, n, lr, iters, dw, db, h_loss_hist ? dh : nullptr, st);
-    if (rc != LR_OK) return rc;
-    LR_CK(ctx, cudaMemcpyAsync(h_w, dw, size_t(n) * 4, cudaMemcpyDeviceToHost, st));
-    LR_CK(ctx, cudaMemcpyAsync(h_b, db, 4, cudaMemcpyDeviceToHost, st));
-    if (h_loss_hist && iters > 0) LR_CK(ctx, cudaMemcpyAsync(h_loss_hist, dh, size_t(iters) * 4, cudaMemcpyDeviceToHost, st));
-    LR_CK(ctx, cudaStreamSynchronize(st));
-    return LR_OK;
+    return fit_host_impl(ctx, h_X, false, h_y, m, n, lr, iters, h_w, h_b, h_loss_hist);
+}
+
+int lr_fit_host_bf16(lr_ctx* ctx, const float* h_X, const float* h_y, int64_t m, int32_t n, float lr, int32_t iters,
+                     float* h_w, float* h_b, float* h_loss_hist) {
+    return fit_host_impl(ctx, h_X, true, h_y, m, n, lr, iters, h_w, h_b, h_loss_hist);
 }
 
 int lr_predict_host(lr_ctx* ctx, const float* h_X, int64_t m, int32_t n, const float* h_w, const float* h_b, float thr,
                     uint8_t* h_labels) {
-    int rc = check_common(ctx, h_X, m, n, h_w, h_b);
-    if (rc != LR_OK) return rc;
-    if (!h_labels) return LR_ERR_NULL;
-    if (!(thr > 0.f && thr < 1.f)) return LR_ERR_VALUE;
-    DeviceGuard g(ctx);
-    if (!g.ok) return LR_ERR_CUDA;
-    const size_t xb = size_t(m) * n * 4;
-    if ((rc = grow(ctx, &ctx->d_hX, &ctx->hX_bytes, xb)) != LR_OK) return rc;
-    if ((rc = grow(ctx, &ctx->d_hw, &ctx->hw_bytes, (size_t(n) + 1) * 4)) != LR_OK) return rc;
-    if ((rc = grow(ctx, &ctx->d_hl, &ctx->hl_bytes, size_t(m))) != LR_OK) return rc;
-    float* dX = static_cast<float*>(ctx->d_hX);
-    float* dw = static_cast<float*>(ctx->d_hw);
-    float* db = dw + n;
-    uint8_t* dl = static_cast<uint8_t*>(ctx->d_hl);
-    cudaStream_t st = ctx->hstream;
-    LR_CK(ctx, cudaMemcpyAsync(dX, h_X, xb, cudaMemcpyHostToDevice, st));
-    LR_CK(ctx, cudaMemcpyAsync(dw, h_w, size_t(n) * 4, cudaMemcpyHostToDevice, st));
-    LR_CK(ctx, cudaMemcpyAsync(db, h_b, 4, cudaMemcpyHostToDevice, st));
-    rc = lr_predict(ctx, dX, m, n, dw, db, thr, dl, st);
-    if (rc != LR_OK) return rc;
-    LR_CK(ctx, cudaMemcpyAsync(h_labels, dl, size_t(m), cudaMemcpyDeviceToHost, st));
-    LR_CK(ctx, cudaStreamSynchronize(st));
-    return LR_OK;
+    return predict_host_impl(ctx, h_X, false, m, n, h_w, h_b, thr, h_labels);
+}
+
+int lr_predict_host_bf16(lr_ctx* ctx, const float* h_X, int64_t m, int32_t n, const float* h_w, const float* h_b, float thr,
+                         uint8_t* h_labels) {
+    return predict_host_impl(ctx, h_X, true, m, n, h_w, h_b, thr, h_labels);
 }
 
 int lr_profile_enable(lr_ctx* ctx, int32_t on) {

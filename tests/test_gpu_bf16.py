@@ -192,6 +192,32 @@ def test_fit_and_predict_match_oracle(ctx, name, m):
         assert (lab == lab_ref).mean() >= LABEL_AGREE
 
 
+def test_host_entry_points_with_bfloat16_storage(ctx):
+    # fp32 rows on the host, rounded to bfloat16 on the device after the copy: the result is the device-pointer fit on the
+    # library's own conversion, bit for bit, and the checker's fit on its own rounding within the tolerances
+    wl = datagen.scaled(datagen.WORKLOADS["cfg3"], 30_011)
+    X, y, _, _ = datagen.generate(wl)
+    iters = 9
+    w = np.zeros(wl.n, dtype=np.float32)
+    b = np.zeros(1, dtype=np.float32)
+    hist = np.zeros(iters, dtype=np.float32)
+    ctx.fit_host(X, y, wl.lr, iters, w, b, hist, store_bf16=True)
+    dXh = ctx.convert_bf16(dev(X))
+    dw = torch.zeros(wl.n, device="cuda")
+    db = torch.zeros(1, device="cuda")
+    dh = torch.empty(iters, device="cuda")
+    ctx.fit(dXh, dev(y), wl.lr, iters, dw, db, dh)
+    assert np.array_equal(w, dw.cpu().numpy()) and np.array_equal(b, db.cpu().numpy()) and np.array_equal(hist, dh.cpu().numpy())
+    _, Xv = oracle.round_bf16(X)
+    w_ref, b_ref, lh_ref = oracle.fit(Xv, y, wl.lr, iters)
+    assert rel_l2(np.concatenate([w, b]), np.concatenate([w_ref, [b_ref]])) <= W_TOL
+    assert np.max(np.abs(hist - lh_ref)) <= LOSS_TOL
+    labels = np.zeros(wl.m, dtype=np.uint8)
+    ctx.predict_host(X, w, b, 0.4, labels, store_bf16=True)
+    assert np.array_equal(labels, ctx.predict(dXh, dw, db, 0.4).cpu().numpy())
+    assert (labels == oracle.predict(Xv, w.astype(np.float64), float(b[0]), 0.4)).mean() >= LABEL_AGREE
+
+
 def test_wide_rows_fit(ctx):
     # the wide-row kernel iterates as two kernels per step
     wl = datagen.scaled(datagen.WORKLOADS["cfg4"], 3_000)
