@@ -37,19 +37,34 @@ METRIC = "GD iterations/sec and achieved HBM GB/s (fraction of B200 peak) at m\u
 UNIT = "iterations/s"
 NOMINAL_HBM_GBS = 8000.0
 # dram__bytes_read.sum + dram__bytes_write.sum per row of X, from the ncu captures summarised in profiles/ (taken on a
-# smaller row count of the same workload and scaled by rows; k_fit_rows: per row and iteration).  Keys: workload, with
-# "_bf16" for bfloat16 storage.  Remove an entry when its kernel changes.
+# smaller row count of the same workload and scaled by rows).  k_stream_rows / k_stream_split: one pass.  k_fit_rows: per
+# row and iteration with nothing kept in L2 -- the captures ran three iterations with the default quarter of the L2
+# (KEPT_BYTES of X) kept, so two of the three served those bytes from L2; the figure here has them added back, and
+# `fit_traffic` takes the kept bytes off again for the iterations after the first.  Keys: workload, with "_bf16" for
+# bfloat16 storage.  Remove an entry when its kernel changes.
+KEPT_BYTES = 33_030_144                         # a quarter of the 126 MB L2, as lr_set_l2_keep's default for the persistent kernel
 NCU_TRAFFIC_BYTES_PER_ROW = {
-    "cfg2": {"k_stream_rows": (404.024832e6 + 3.117056e6) / 1_000_000},
-    "cfg5": {"k_stream_rows": (520.023552e6 + 3.864576e6) / 2_000_000},
-    "higgs_like": {"k_stream_rows": (464.036864e6 + 3.543040e6) / 4_000_000},
+    "cfg2": {"k_stream_rows": (404.024832e6 + 3.117056e6) / 1_000_000,
+             "k_fit_rows": (1.111132e9 + 4.197632e6 + 2 * KEPT_BYTES) / 3 / 1_000_000},
+    "cfg5": {"k_stream_rows": (520.023552e6 + 3.864576e6) / 2_000_000,
+             "k_fit_rows": (1.446715e9 + 7.011840e6 + 2 * KEPT_BYTES) / 3 / 2_000_000},
+    "higgs_like": {"k_stream_rows": (464.036864e6 + 3.543040e6) / 4_000_000,
+                   "k_fit_rows": (1.269865e9 + 5.956608e6 + 2 * KEPT_BYTES) / 3 / 4_000_000},
     "cfg3": {"k_stream_rows": (514.040064e6 + 3.598336e6) / 500_000,
-             "k_fit_rows": (1.501257e9 + 3.482880e6) / 3 / 500_000},
+             "k_fit_rows": (1.439553e9 + 3.939840e6 + 2 * KEPT_BYTES) / 3 / 500_000},
     "cfg4": {"k_stream_split": (491.682048e6 + 3.577600e6) / 30_000},
     "cfg3_bf16": {"k_stream_rows": (516.026624e6 + 3.481088e6) / 1_000_000,
-                  "k_fit_rows": (1.503338e9 + 5.044224e6) / 3 / 1_000_000},
+                  "k_fit_rows": (1.441246e9 + 4.163328e6 + 2 * KEPT_BYTES) / 3 / 1_000_000},
     "cfg4_bf16": {"k_stream_split": (491.803904e6 + 5.702400e6) / 60_000},
 }
+
+
+def fit_traffic(per_row, m, steps, x_bytes, keep_bytes):
+    """DRAM bytes of one persistent launch of `steps` iterations over m rows: every iteration after the first finds the kept
+    part of X (at most all of it) in L2."""
+    return per_row * m * steps - (steps - 1) * min(keep_bytes, x_bytes)
+
+
 FALLBACK_HBM_GBS = 6650.0
 
 
@@ -443,7 +458,9 @@ def main():
         ach = bytes_per_launch * args.steps / (ms * 1e-3) / 1e9
         roofline = {"bound": "hbm", "kernel": "k_fit_rows (persistent: all timed iterations in one cooperative launch)",
                     "achieved": ach, "peak": peak, "unit": "GB/s", "frac": ach / peak, "peak_kind": f"of {peak_kind}",
-                    "traffic": per_row["k_fit_rows"] * wl.m * args.steps if "k_fit_rows" in per_row else None,
+                    "traffic": (fit_traffic(per_row["k_fit_rows"], wl.m, args.steps, elem_bytes * wl.m * wl.n,
+                                            KEPT_BYTES if args.l2_keep_mb < 0 else int(args.l2_keep_mb * 1e6))
+                                if "k_fit_rows" in per_row and args.rows == 0 else None),
                     "bytes_per_launch": bytes_per_launch * args.steps,
                     "avg_launch_ms": ms, "launches_timed": 1, "iterations_per_launch": args.steps,
                     "frac_of_nominal_8TBs": ach / NOMINAL_HBM_GBS, "single_pass": single_pass}
