@@ -44,7 +44,7 @@ NOMINAL_HBM_GBS = 8000.0
 # bfloat16 storage.  Remove an entry when its kernel changes.
 KEPT_BYTES = 33_030_144                         # a quarter of the 126 MB L2, as lr_set_l2_keep's default for the persistent kernel
 NCU_TRAFFIC_BYTES_PER_ROW = {
-    "cfg2": {"k_stream_rows": (404.024832e6 + 3.117056e6) / 1_000_000,
+    "cfg2": {"k_stream_rows": (404.025344e6 + 3.488768e6) / 1_000_000,
              "k_fit_rows": (1.111132e9 + 4.197632e6 + 2 * KEPT_BYTES) / 3 / 1_000_000},
     "cfg5": {"k_stream_rows": (520.023552e6 + 3.864576e6) / 2_000_000,
              "k_fit_rows": (1.446715e9 + 7.011840e6 + 2 * KEPT_BYTES) / 3 / 2_000_000},
