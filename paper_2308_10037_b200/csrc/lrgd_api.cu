@@ -20,6 +20,7 @@
 #include "lrgd_reduce.cuh"
 #include "lrgd_stream_rows.cuh"
 #include "lrgd_stream_split.cuh"
+#include "lrgd_stream_wide.cuh"
 
 using namespace lrgd;
 
@@ -34,6 +35,7 @@ constexpr int kMaxGridPerSm = 8;               // widest launch any variant uses
 constexpr int kMaxProfiled = 4096;
 constexpr int kMaxDynamicSmem = 232448;         // opt-in dynamic shared memory per CTA on sm_100
 constexpr int64_t kMaxRows = int64_t(1) << 40;
+constexpr int kWideAnyMaxCols = 8192;           // widest row of the CTA-wide staged kernel for rows of any length
 
 struct RowShape { int nv, lpr, rb; int nw = kNW; };    // nw = warps per CTA
 
@@ -67,8 +69,7 @@ bool any_row_shape_for(int n, RowShape* s) {
     else if (n <= 128) *s = {4, 32, 8};
     else if (n <= 256) *s = {8, 32, 4};
     else if (n <= 512) *s = {16, 32, 2};
-    else if (n <= 1024) *s = {32, 32, 1, 8};                // eight warps per CTA, one row at a time (up to 4 KB)
-    else return false;
+    else return false;                                      // wider rows of any length: the CTA-wide staged kernel (variant 4)
     return true;
 }
 
@@ -135,6 +136,40 @@ int make_plan(int64_t m, int32_t n, bool aligned16, int32_t sms, lr_plan* P, boo
         P->grid = grid;
         P->threads = nw * 32;
         P->smem_bytes = int(kSplitHeaderBytes + int64_t(nw) * D * stage_stride);
+        if (per_cta >= (int64_t(1) << 31)) return LR_ERR_SHAPE;
+        return LR_OK;
+    }
+    if (n > 512 && n <= kWideAnyMaxCols) {
+        // wide rows of any length, matrix aligned to its element size: the warps of a CTA split each row by columns and the
+        // stages, whole batches of contiguous rows, belong to the CTA.  A lane holds NV elements of each of RB rows (32 in
+        // all); a batch is at most ~64 KB so that two to four of them are in flight.
+        // rows of up to 1024 elements are split over eight warps (slices of 65..128 elements: three or four per lane, sixteen
+        // rows per batch in 255 registers), wider ones over sixteen
+        const int nw = n <= 1024 ? 8 : kNW;
+        const int cw = (n + nw - 1) / nw;                                       // elements per warp slice
+        // elements per lane and row: the smallest of 2, 3, 4, 6, 8, 12, 16 that covers the slice (a lane's slots beyond the
+        // slice are dead work, so the steps are kept fine); rows per batch: as many as the registers hold (32 or 48 elements
+        // of a batch per lane), because all warps meet once per batch
+        static const int kNv[7] = {2, 3, 4, 6, 8, 12, 16}, kRb[7] = {16, 16, 8, 8, 4, 4, 2};
+        int pick = 0;
+        while (pick < 6 && kNv[pick] * 32 < cw) ++pick;
+        const int nv = kNv[pick], rb = nw == 8 ? 16 : kRb[pick];
+        const int64_t B = (m + rb - 1) / rb;
+        const int grid = int(std::min<int64_t>(B, sms));
+        const int64_t per_cta = (B + grid - 1) / grid;
+        const int64_t stage_stride = (int64_t(rb) * n * eb + 16 + 127) & ~int64_t(127);
+        int D = int(std::min<int64_t>(kMaxDepth, (kStageBudgetBytes + 12 * 1024) / stage_stride));
+        D = int(std::min<int64_t>(D, per_cta));
+        if (D < 1) D = 1;
+        P->variant = 4;
+        P->lanes_per_row = nw * 32;
+        P->vec_per_lane = nv;
+        P->rows_per_batch = rb;
+        P->tile_rows = rb;
+        P->stages = D;
+        P->grid = grid;
+        P->threads = nw * 32;
+        P->smem_bytes = int(kSplitHeaderBytes + int64_t(D) * stage_stride);
         if (per_cta >= (int64_t(1) << 31)) return LR_ERR_SHAPE;
         return LR_OK;
     }
@@ -286,11 +321,11 @@ cudaError_t for_row_shape(const lr_plan& P, bool bf16, F&& f) {
         if (bf16) {
             LRGD_SHAPE(ElemBF16Any, 1, 8, 8, 16) LRGD_SHAPE(ElemBF16Any, 1, 16, 8, 16) LRGD_SHAPE(ElemBF16Any, 1, 32, 16, 16)
             LRGD_SHAPE(ElemBF16Any, 2, 32, 16, 16) LRGD_SHAPE(ElemBF16Any, 4, 32, 8, 16) LRGD_SHAPE(ElemBF16Any, 8, 32, 4, 16)
-            LRGD_SHAPE(ElemBF16Any, 16, 32, 2, 16) LRGD_SHAPE(ElemBF16Any, 32, 32, 1, 8)
+            LRGD_SHAPE(ElemBF16Any, 16, 32, 2, 16)
         } else {
             LRGD_SHAPE(ElemF32Any, 1, 8, 8, 16) LRGD_SHAPE(ElemF32Any, 1, 16, 8, 16) LRGD_SHAPE(ElemF32Any, 1, 32, 16, 16)
             LRGD_SHAPE(ElemF32Any, 2, 32, 16, 16) LRGD_SHAPE(ElemF32Any, 4, 32, 8, 16) LRGD_SHAPE(ElemF32Any, 8, 32, 4, 16)
-            LRGD_SHAPE(ElemF32Any, 16, 32, 2, 16) LRGD_SHAPE(ElemF32Any, 32, 32, 1, 8)
+            LRGD_SHAPE(ElemF32Any, 16, 32, 2, 16)
         }
     } else if (bf16) {
         LRGD_SHAPE(ElemBF16, 1, 8, 8, 16) LRGD_SHAPE(ElemBF16, 1, 16, 8, 16) LRGD_SHAPE(ElemBF16, 1, 32, 8, 16)
@@ -380,6 +415,34 @@ cudaError_t launch_split(const lr_plan& P, const void* X, const SplitParams& sp,
     if (P.vec_per_lane == 2) return launch_split_t<ElemF32, 2, 4, PRED>(P, tm, sp, st, dependent);
     if (P.rows_per_batch == 16) return launch_split_t<ElemF32, 1, 16, PRED>(P, tm, sp, st, dependent);
     return launch_split_t<ElemF32, 1, 8, PRED>(P, tm, sp, st, dependent);
+}
+
+template <class E, int NV, int RB, bool PRED, int NW = kNW>
+cudaError_t launch_wide_t(const lr_plan& P, const WideParams& wp, cudaStream_t st, bool dependent) {
+    auto kern = k_stream_wide<E, NV, RB, NW, PRED>;
+    cudaError_t e = ensure_dynamic_smem<KernelTag<E, NV, -2, RB, NW, PRED>>(reinterpret_cast<const void*>(kern), P.smem_bytes);
+    if (e != cudaSuccess) return e;
+    return launch_kernel(kern, dim3(P.grid), dim3(P.threads), size_t(P.smem_bytes), st, dependent, wp);
+}
+
+template <bool PRED>
+cudaError_t launch_wide(const lr_plan& P, const WideParams& wp, cudaStream_t st, bool bf16, bool dependent) {
+#define LRGD_WIDE(E, nv, rb) if (P.vec_per_lane == nv && P.rows_per_batch == rb) return launch_wide_t<E, nv, rb, PRED>(P, wp, st, dependent);
+    if (P.threads == 256) {                        // rows of 513..1024 elements: eight warps
+        if (bf16) return P.vec_per_lane == 3 ? launch_wide_t<ElemBF16Any, 3, 16, PRED, 8>(P, wp, st, dependent)
+                                             : launch_wide_t<ElemBF16Any, 4, 16, PRED, 8>(P, wp, st, dependent);
+        return P.vec_per_lane == 3 ? launch_wide_t<ElemF32Any, 3, 16, PRED, 8>(P, wp, st, dependent)
+                                   : launch_wide_t<ElemF32Any, 4, 16, PRED, 8>(P, wp, st, dependent);
+    }
+    if (bf16) {
+        LRGD_WIDE(ElemBF16Any, 2, 16) LRGD_WIDE(ElemBF16Any, 3, 16) LRGD_WIDE(ElemBF16Any, 4, 8) LRGD_WIDE(ElemBF16Any, 6, 8)
+        LRGD_WIDE(ElemBF16Any, 8, 4) LRGD_WIDE(ElemBF16Any, 12, 4) LRGD_WIDE(ElemBF16Any, 16, 2)
+    } else {
+        LRGD_WIDE(ElemF32Any, 2, 16) LRGD_WIDE(ElemF32Any, 3, 16) LRGD_WIDE(ElemF32Any, 4, 8) LRGD_WIDE(ElemF32Any, 6, 8)
+        LRGD_WIDE(ElemF32Any, 8, 4) LRGD_WIDE(ElemF32Any, 12, 4) LRGD_WIDE(ElemF32Any, 16, 2)
+    }
+#undef LRGD_WIDE
+    return cudaErrorInvalidValue;
 }
 
 // The persistent whole-fit kernel of a variant-0 plan; resident: every warp's share of X fits its stages, which are then
@@ -546,6 +609,15 @@ int launch_stream_pass(lr_ctx* ctx, const lr_plan& P, const Pass& a, uint8_t* la
         sp.num_batches = (a.m + P.rows_per_batch - 1) / P.rows_per_batch;
         sp.keep_rows = keep_rows_for(ctx, 1, a.n, a.bf16);
         e = predict ? launch_split<true>(P, a.X, sp, st, a.bf16, dep) : launch_split<false>(P, a.X, sp, st, a.bf16, dep);
+    } else if (P.variant == 4) {
+        WideParams wp{};
+        wp.X = a.X; wp.y = a.y; wp.m = a.m; wp.n = a.n; wp.w = a.w; wp.b = a.b;
+        wp.partial = ctx->d_partial; wp.labels = labels; wp.cut = cut; wp.status = ctx->d_status; wp.stop = a.stop;
+        wp.depth = P.stages;
+        wp.cw = (a.n + P.threads / 32 - 1) / (P.threads / 32);
+        wp.num_batches = (a.m + P.rows_per_batch - 1) / P.rows_per_batch;
+        wp.keep_rows = keep_rows_for(ctx, 1, a.n, a.bf16);
+        e = predict ? launch_wide<true>(P, wp, st, a.bf16, dep) : launch_wide<false>(P, wp, st, a.bf16, dep);
     } else {
         GenericParams gp{};
         gp.X = a.X; gp.y = a.y; gp.m = a.m; gp.n = a.n; gp.w = a.w; gp.b = a.b;

@@ -70,19 +70,28 @@ def test_plan_staged_shapes(m, n, lpr, nv, nw):
         assert p["rows_per_batch"] == 16                      # 68..128 fp32 columns: sixteen rows per batch, eight warps
 
 
-def test_plan_falls_back_for_unaligned_or_odd_shapes():
-    assert api.plan_query(1000, 1027)["variant"] == 2        # n not a multiple of 4 and wider than 1024
-    assert api.plan_query(1000, 1028, x_aligned16=False)["variant"] == 2   # wide rows need a 16-byte aligned matrix
-    assert api.plan_query(1000, 515)["variant"] == 3 and api.plan_query(1000, 516, x_aligned16=False)["variant"] == 3
-    assert api.plan_query(1000, 32, x_aligned16=False)["variant"] == 3     # narrow rows do not: element-wise staged kernel
+def test_plan_for_unaligned_or_odd_shapes():
+    # rows of any length in a matrix aligned to its element size: per-warp stages up to 512 columns (variant 3), CTA-wide
+    # stages of whole rows up to 8192 (variant 4); only wider rows run unstaged (variant 2)
+    assert api.plan_query(1000, 1027)["variant"] == 4        # n not a multiple of 4 and wider than 1024
+    assert api.plan_query(1000, 1028, x_aligned16=False)["variant"] == 4   # the row-split kernel needs a 16-byte aligned matrix
+    assert api.plan_query(1000, 515)["variant"] == 4 and api.plan_query(1000, 516, x_aligned16=False)["variant"] == 4
+    assert api.plan_query(1000, 511)["variant"] == 3 and api.plan_query(1000, 512, x_aligned16=False)["variant"] == 3
+    assert api.plan_query(1000, 32, x_aligned16=False)["variant"] == 3     # narrow rows: element-wise staged kernel
     assert api.plan_query(1000, 30, x_aligned16=False)["variant"] == 3
     assert api.plan_query(1000, 32, x_aligned16=False, bf16=True)["variant"] == 3
+    assert api.plan_query(1000, 8191)["variant"] == 4 and api.plan_query(1000, 8192, x_aligned16=False)["variant"] == 4
     assert api.plan_query(1000, 8196)["variant"] == 2         # wider than any staged kernel
     assert api.plan_query(1000, 8200, bf16=True)["variant"] == 2
     assert api.plan_query(1000, 30, bf16=True)["variant"] == 3   # element-wise staged kernel, bfloat16 too
-    assert api.plan_query(1000, 1036, bf16=True)["variant"] == 2 # 1036 % 8 != 0 and wider than 1024
-    g = api.plan_query(100, 1027)
-    assert g["grid"] == 2 and g["threads"] == 256
+    assert api.plan_query(1000, 1036, bf16=True)["variant"] == 4 # 1036 % 8 != 0 and wider than 1024
+    g = api.plan_query(100, 8197)
+    assert g["variant"] == 2 and g["grid"] == 2 and g["threads"] == 256
+    w = api.plan_query(100_000, 1027)
+    assert w["vec_per_lane"] == 3 and w["rows_per_batch"] == 16 and w["stages"] == 3 and w["threads"] == 512
+    assert api.plan_query(100_000, 8191)["rows_per_batch"] == 2
+    n513 = api.plan_query(100_000, 513)
+    assert n513["rows_per_batch"] == 16 and n513["threads"] == 256 and n513["vec_per_lane"] == 3
 
 
 @pytest.mark.parametrize("n,lpr,nv,rb", [(1, 8, 1, 8), (7, 8, 1, 8), (13, 16, 1, 8), (30, 32, 1, 16), (33, 32, 2, 16), (101, 32, 4, 8),
@@ -167,7 +176,8 @@ def test_any_length_copies_stay_inside_the_matrix():
     shapes = [(2758, 449), (1, 1), (7, 3), (300, 1), (640, 30), (1025, 101), (526, 255), (999, 511), (5, 510), (3, 258),
               (17, 257), (2, 449), (1, 511)]
     shapes += [(rnd.randint(1, 3000), rnd.choice([n for n in range(1, 513) if n % 4])) for _ in range(200)]
-    shapes += [(3, 513), (1, 1023), (77, 1021), (500, 777), (2, 1022)] + [(rnd.randint(1, 400), rnd.choice([n for n in range(513, 1025) if n % 4])) for _ in range(40)]
+    shapes += [(3, 513), (1, 1023), (77, 1021), (500, 777), (2, 1022), (9, 8191), (33, 4099), (5, 2049), (64, 1025)]
+    shapes += [(rnd.randint(1, 400), rnd.choice([n for n in range(513, 8192) if n % 4])) for _ in range(60)]
     cases = [(m, n, 0, 4) for m, n in shapes]
     extra = shapes[:60] + [(1, 1), (2, 2), (3, 1), (40, 32), (999, 256), (77, 512)]
     cases += [(m, n, base, 4) for (m, n) in extra for base in (4, 8, 12)]
@@ -175,11 +185,14 @@ def test_any_length_copies_stay_inside_the_matrix():
     cases += [(m, n, 0, 2) for (m, n) in shapes[:80] if n % 8] + [(m, n, base, 2) for (m, n) in extra[:40] for base in (2, 6, 10, 14)]
     for m, n, base, eb in cases:
         p = api.plan_query(m, n, x_aligned16=(base == 0), bf16=(eb == 2))
-        assert p["variant"] == 3
+        assert p["variant"] == (3 if n <= 512 else 4)             # per-warp stages up to 512 columns, CTA-wide stages beyond
         rpb, row_bytes = p["rows_per_batch"], eb * n
         lo_x, hi_x = 4096 + base, 4096 + base + eb * m * n         # the matrix occupies the addresses [lo_x, hi_x)
         stage = -(-(rpb * row_bytes + 16) // 128) * 128
-        assert 1024 + (p["threads"] // 32) * p["stages"] * stage <= p["smem_bytes"]
+        if p["variant"] == 3:
+            assert 1024 + (p["threads"] // 32) * p["stages"] * stage <= p["smem_bytes"]
+        else:
+            assert 4096 + p["stages"] * stage == p["smem_bytes"] <= 227 * 1024
         seen = 0
         for g in range(-(-m // rpb)):
             r0 = g * rpb
@@ -226,7 +239,17 @@ def test_every_row_length_gets_a_launchable_plan():
                     if v == 0:
                         assert aligned and n % epg == 0
                     else:
-                        assert n <= 1024
+                        assert n <= 512
+                elif v == 4:
+                    # wide rows of any length: CTA-wide stages of whole rows; eight warps up to 1024 elements, sixteen beyond
+                    nw = p["threads"] // 32
+                    assert 512 < n <= 8192 and nw == (8 if n <= 1024 else 16)
+                    cw = -(-n // nw)
+                    assert p["vec_per_lane"] in (2, 3, 4, 6, 8, 12, 16) and p["vec_per_lane"] * 32 >= cw
+                    assert p["vec_per_lane"] * p["rows_per_batch"] in (32, 48, 64) and p["rows_per_batch"] in (2, 4, 8, 16)
+                    assert 2 * nw * p["rows_per_batch"] * 4 <= 4096 - 1024                   # the logit exchange fits the header
+                    stage = -(-(p["rows_per_batch"] * n * eb + 16) // 128) * 128
+                    assert 1 <= p["stages"] <= 4 and p["smem_bytes"] == 4096 + p["stages"] * stage
                 elif v == 1:
                     nw = p["threads"] // 32
                     assert aligned and n % epg == 0 and nw == (8 if bf16 and n // epg <= 384 else 16)
@@ -237,5 +260,5 @@ def test_every_row_length_gets_a_launchable_plan():
                     stage = -(-p["rows_per_batch"] * cw * 16 // 128) * 128
                     assert 1 <= p["stages"] <= 4 and p["smem_bytes"] == 4096 + nw * p["stages"] * stage
                 else:
-                    assert v == 2 and p["threads"] == 256
+                    assert v == 2 and p["threads"] == 256 and n > 8192
                     assert n > 1024 and (not aligned or n % epg != 0 or n > 8192)

@@ -110,16 +110,17 @@ def test_bf16_views_that_are_only_2_byte_aligned(ctx, m, n, shift):
     buf[shift:shift + bits.size] = dev_bf16(bits).ravel()
     Xh = buf[shift:shift + bits.size].view(m, n)
     assert Xh.data_ptr() % 16 == 2 * shift
-    assert api.plan_query(m, n, x_aligned16=False, bf16=True)["variant"] == (3 if n <= 1024 else 2)
+    assert api.plan_query(m, n, x_aligned16=False, bf16=True)["variant"] == (3 if n <= 512 else 4)
     check_loss_grad(ctx, Xv, Xh, y, w, b)
 
 
 # bfloat16 rows whose length is not a multiple of eight: every element-wise instantiation, batches that start off a
 # 16-byte boundary, ragged tails, stage reuse; pass, labels and a short fit
 @pytest.mark.parametrize("m,n", [(33, 7), (1, 3), (40_003, 13), (150_001, 30), (100_001, 100), (200_003, 255), (2_758, 449),
-                                 (60_001, 449), (50_002, 508), (5, 510), (17, 257), (30_001, 1020), (20_003, 777)])
+                                 (60_001, 449), (50_002, 508), (5, 510), (17, 257), (30_001, 1020), (20_003, 777),
+                                 (9_001, 4100), (3_001, 8191), (20_001, 1025), (7, 8190), (12_001, 2049)])
 def test_bf16_rows_of_any_length(ctx, m, n):
-    assert api.plan_query(m, n, bf16=True)["variant"] == 3
+    assert api.plan_query(m, n, bf16=True)["variant"] == (3 if n <= 512 else 4)
     X, y, w, b = datagen.random_problem(m, n, seed=3500 + m + n, wscale=1.5)
     bits, Xv = oracle.round_bf16(X)
     dXh = dev_bf16(bits)

@@ -105,7 +105,7 @@ def test_matrices_that_are_only_4_byte_aligned(ctx, m, n, shift):
     buf[shift:shift + X.size] = dev(X).ravel()
     Xv = buf[shift:shift + X.size].view(m, n)
     assert Xv.data_ptr() % 16 == 4 * shift
-    assert api.plan_query(m, n, x_aligned16=False)["variant"] == (3 if n <= 1024 else 2)
+    assert api.plan_query(m, n, x_aligned16=False)["variant"] == (3 if n <= 512 else 4)
     L, g, g0 = oracle.loss_grad(X, y, w, b)
     dl, dg, dg0 = ctx.loss_grad(Xv, dev(y), dev(w), dev(np.array([b], dtype=np.float32)))
     assert abs(dl.item() - L) <= LOSS_TOL
@@ -210,13 +210,14 @@ def test_predict_matches_oracle(ctx, m, n):
 # fp32 rows whose length is not a multiple of four (a lane owns single elements): every instantiation (n <= 8, 16, 32, 64,
 # 128, 256, 512), batches that do not start on a 16-byte boundary (two-row batches of odd-length rows), ragged tails whose
 # byte count is not a multiple of 16, stage reuse
-ANY_LENGTH = [(40_001, 513), (30_003, 777), (25_001, 1023), (3, 1001), (33, 7), (1, 3), (20_011, 5), (40_003, 13), (150_001, 30), (90_001, 49), (100_001, 101), (200_003, 255),
+ANY_LENGTH = [(9_001, 4099), (3_001, 8191), (20_001, 1025), (7, 8191), (2, 6001), (1, 2049), (12_001, 2050),
+              (40_001, 513), (30_003, 777), (25_001, 1023), (3, 1001), (33, 7), (1, 3), (20_011, 5), (40_003, 13), (150_001, 30), (90_001, 49), (100_001, 101), (200_003, 255),
               (2_758, 449), (60_001, 449), (50_002, 511), (5, 510), (3, 258), (17, 257), (70_001, 258), (1, 511)]
 
 
 @pytest.mark.parametrize("m,n", ANY_LENGTH)
 def test_rows_of_any_length(ctx, m, n):
-    assert api.plan_query(m, n)["variant"] == 3
+    assert api.plan_query(m, n)["variant"] == (3 if n <= 512 else 4)
     X, y, w, b = datagen.random_problem(m, n, seed=3000 + m + n, wscale=1.5)
     check_loss_grad(ctx, X, y, w, b)
     # labels, including the word-packed stores
