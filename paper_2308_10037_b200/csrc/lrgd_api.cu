@@ -107,7 +107,10 @@ int make_plan(int64_t m, int32_t n, bool aligned16, int32_t sms, lr_plan* P, boo
         if (per_warp >= (int64_t(1) << 31)) return LR_ERR_SHAPE;
         return LR_OK;
     }
-    if (aligned16 && n % epg == 0 && n / epg <= kNW * (bf16 ? 64 : 128) && m < (int64_t(1) << 31) - 65536) {   // TMA coordinates are int32
+    // (fp32 rows of 4100..6144 columns are the exception: slices of 65..96 groups per warp leave the row-split kernel with two
+    // rows per batch and half-empty lanes, 3.7-5.1 TB/s, where the CTA-wide stages of variant 4 below reach 4.7-5.9)
+    const bool split_weak = !bf16 && n / epg > 1024 && n / epg <= 1536;
+    if (aligned16 && n % epg == 0 && n / epg <= kNW * (bf16 ? 64 : 128) && !split_weak && m < (int64_t(1) << 31) - 65536) {   // TMA coordinates are int32
         // wide rows: the warps of a CTA split each row by columns
         // bfloat16 rows of up to 384 groups (1032..3072 columns) are split across eight warps instead of sixteen: wider
         // slices, and 255 registers per thread, which batches of 16 (one group per lane) or 8 rows (two groups) need

@@ -63,7 +63,7 @@ def test_loss_grad_matches_oracle(ctx, m, n):
 # both sides of every boundary between kernel shapes (lanes per row, groups per lane, warps per CTA, rows per batch,
 # narrow / split / unstaged), for a row count that gives every warp several batches with a ragged last one
 BOUNDARY_N = [4, 8, 12, 32, 36, 64, 68, 128, 132, 256, 260, 384, 388, 512, 516, 1024, 1028, 1536, 1540, 2048, 2052, 3072, 3076,
-              4096, 4100, 8192, 8196, 9, 17, 33, 65, 129, 257, 513]
+              4096, 4100, 6144, 6148, 8192, 8196, 9, 17, 33, 65, 129, 257, 513, 1025, 8191]
 
 
 @pytest.mark.parametrize("n", BOUNDARY_N)
