@@ -292,6 +292,7 @@ def main():
     ap.add_argument("--no-persistent", action="store_true", help="force two kernels per iteration in lr_fit")
     ap.add_argument("--force-persistent", action="store_true", help="force the single-launch persistent kernel in lr_fit")
     ap.add_argument("--no-overlap", action="store_true", help="ordinary launches only (no programmatic dependent launches)")
+    ap.add_argument("--no-cluster", action="store_true", help="tiny problems: the grid-wide persistent kernel instead of the single-cluster one")
     ap.add_argument("--l2-keep-mb", type=float, default=-1.0, help="MB of X to keep in L2 across iterations (-1: library default, 0: off)")
     ap.add_argument("--x-dtype", default="f32", choices=["f32", "bf16"],
                     help="storage type of X on the device: bf16 runs the bfloat16 entry points on lr_convert_bf16's output "
@@ -351,6 +352,8 @@ def main():
         ctx.set_persistent(True)
     if args.no_overlap:
         ctx.set_overlap(False)
+    if args.no_cluster:
+        ctx.set_cluster(False)
     if args.l2_keep_mb >= 0:
         ctx.set_l2_keep(int(args.l2_keep_mb * 1e6))
     w = torch.zeros(wl.n, dtype=torch.float32, device="cuda")
@@ -456,11 +459,14 @@ def main():
     if world == 1 and launches == 1:
         # the timed region was ONE launch of the persistent kernel doing all K iterations (pass + reduction + update)
         ach = bytes_per_launch * args.steps / (ms * 1e-3) / 1e9
-        roofline = {"bound": "hbm", "kernel": "k_fit_rows (persistent: all timed iterations in one cooperative launch)",
+        cluster_c = 0 if args.no_cluster else api.cluster_ctas(wl.m, wl.n, bf16=bf16)
+        roofline = {"bound": "hbm", "kernel": (f"k_fit_cluster (all timed iterations in one launch on one cluster of {cluster_c} CTAs; X stays in "
+                                               "their shared memory, so the algorithmic bytes below never reach HBM after the first pass)"
+                                               if cluster_c else "k_fit_rows (persistent: all timed iterations in one cooperative launch)"),
                     "achieved": ach, "peak": peak, "unit": "GB/s", "frac": ach / peak, "peak_kind": f"of {peak_kind}",
                     "traffic": (fit_traffic(per_row["k_fit_rows"], wl.m, args.steps, elem_bytes * wl.m * wl.n,
                                             KEPT_BYTES if args.l2_keep_mb < 0 else int(args.l2_keep_mb * 1e6))
-                                if "k_fit_rows" in per_row and args.rows == 0 else None),
+                                if "k_fit_rows" in per_row and args.rows == 0 and not cluster_c else None),
                     "bytes_per_launch": bytes_per_launch * args.steps,
                     "avg_launch_ms": ms, "launches_timed": 1, "iterations_per_launch": args.steps,
                     "frac_of_nominal_8TBs": ach / NOMINAL_HBM_GBS, "single_pass": single_pass}
@@ -520,7 +526,9 @@ def main():
             "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "f32", "x_storage": args.x_dtype, "data": "synthetic", "config": workload_config(wl, world, args.x_dtype),
             "achieved_hbm_gbs_whole_step": bytes_per_launch * world * args.steps / (ms * 1e-3) / 1e9,
-            "fit_form": ("one persistent launch for all timed iterations" if launches == 1 and args.steps > 1 else
+            "fit_form": ("one launch on one thread-block cluster for all timed iterations"
+                         if launches == 1 and args.steps > 1 and not args.no_cluster and api.cluster_ctas(wl.m, wl.n, bf16=bf16) else
+                         "one persistent launch for all timed iterations" if launches == 1 and args.steps > 1 else
                          f"{launches // max(args.steps, 1)} kernels per iteration"
                          + ("" if args.no_overlap else ", each the programmatic dependent of the one before")),
             "timed_regions": {"repeats": repeats, "ms_median": ms, "ms_min": min(region_ms), "ms_max": max(region_ms),

@@ -118,6 +118,20 @@ int lr_loss_grad(lr_ctx* ctx, const float* d_X, const float* d_y, int64_t m, int
 int lr_fit(lr_ctx* ctx, const float* d_X, const float* d_y, int64_t m, int32_t n,
            float lr, int32_t iters, float* d_w, float* d_b, float* d_loss_hist, void* stream);
 int lr_set_persistent(lr_ctx* ctx, int32_t on);
+/*
+ * Third form of lr_fit, for problems whose X fits the shared memory of ONE thread-block cluster of 16 (or 8) CTAs (up to
+ * ~3 MB; rows of 16-byte groups as for the persistent kernel; at least one batch of rows for every CTA): X is fetched
+ * once, and in every iteration each CTA pushes its partial sums into the shared memory of all CTAs of the cluster with
+ * asynchronous remote stores that complete on the receiver's mbarrier, so an iteration never touches global memory.
+ * Taken by default where it applies and no SM limit is set.  The result has the bits of the other forms run under
+ * lr_set_sm_limit(ctx, C), C the cluster size -- the rows are divided among C CTAs instead of all SMs, which changes
+ * the order of the sums.  lr_set_cluster(ctx, 0) switches the form off, any other value restores the default.
+ * lr_fit_tol and lr_fit_sharded do not use it.  A wait that expires ends the kernel as it ends the persistent one.
+ * lr_cluster_ctas (host only, no CUDA call) returns the cluster size the form would use for a shape, 0 if none;
+ * whether a cluster of that size can be resident is known at launch only (if not, the persistent kernel runs).
+ */
+int lr_set_cluster(lr_ctx* ctx, int32_t on);
+int32_t lr_cluster_ctas(int64_t m, int32_t n, int32_t x_aligned16, int32_t bf16);
 
 /*
  * Overlap between the kernels of one call (on by default).  Every iteration of the two-kernel form is a pass followed by

@@ -24,7 +24,8 @@ EXPORTS = ["lr_plan_query", "lr_create", "lr_destroy", "lr_loss_grad", "lr_fit",
            "lr_last_cuda_error", "lr_status_string", "lr_loss_grad_noalloc", "lr_fit_tol", "lr_fit_opt", "lr_selftest_wait", "lr_set_persistent", "lr_fit_sgd", "lr_set_l2_keep",
            "lr_convert_bf16", "lr_loss_grad_bf16", "lr_fit_bf16", "lr_predict_bf16", "lr_plan_query_bf16",
            "lr_fit_tol_bf16", "lr_fit_opt_bf16", "lr_fit_sgd_bf16", "lr_shard_sums_bf16", "lr_set_overlap",
-           "lr_fit_host_bf16", "lr_predict_host_bf16", "lr_exchange_bytes", "lr_fit_sharded", "lr_fit_sharded_bf16", "lr_fit_sharded_local", "lr_set_sm_limit"]
+           "lr_fit_host_bf16", "lr_predict_host_bf16", "lr_exchange_bytes", "lr_fit_sharded", "lr_fit_sharded_bf16", "lr_fit_sharded_local", "lr_set_sm_limit",
+           "lr_set_cluster", "lr_cluster_ctas"]
 
 
 class LrPlan(ctypes.Structure):
@@ -83,6 +84,9 @@ def lib() -> ctypes.CDLL:
         L.lr_set_overlap.argtypes = [P, I32]
         L.lr_set_l2_keep.argtypes = [P, I64]
         L.lr_set_sm_limit.argtypes = [P, I32]
+        L.lr_set_cluster.argtypes = [P, I32]
+        L.lr_cluster_ctas.argtypes = [I64, I32, I32, I32]
+        L.lr_cluster_ctas.restype = I32
         L.lr_exchange_bytes.argtypes = [I32, I32, ctypes.POINTER(I64)]
         L.lr_fit_sharded.argtypes = [P, P, P, I64, I64, I32, F, I32, P, P, P, I32, I32, ctypes.POINTER(P), I64, I32, P]
         L.lr_fit_sharded_bf16.argtypes = L.lr_fit_sharded.argtypes
@@ -119,6 +123,11 @@ def plan_query(m: int, n: int, x_aligned16: bool = True, sm_count: int = 148, bf
     if rc != LR_OK:
         raise LrError(rc, "lr_plan_query")
     return p.as_dict()
+
+
+def cluster_ctas(m: int, n: int, x_aligned16: bool = True, bf16: bool = False) -> int:
+    """Cluster size the single-cluster form of ``fit`` would use for an m-by-n problem, 0 if it has none (host only)."""
+    return int(lib().lr_cluster_ctas(int(m), int(n), int(bool(x_aligned16)), int(bool(bf16))))
 
 
 def exchange_bytes(world: int, n: int) -> int:
@@ -419,6 +428,11 @@ class Context:
         """Form of ``fit`` / ``fit_tol``: True = the single-launch persistent kernel wherever the shape allows, False = two
         kernels per iteration, None = the library chooses (default).  Results are identical either way."""
         self._check(lib().lr_set_persistent(self._h, -1 if on is None else int(bool(on))), "lr_set_persistent")
+
+    def set_cluster(self, on: bool):
+        """Allow (default) or forbid the single-cluster form of ``fit``.  Its results are those of the other forms under
+        ``set_sm_limit(cluster_ctas(m, n))``."""
+        self._check(lib().lr_set_cluster(self._h, int(bool(on))), "lr_set_cluster")
 
     def set_overlap(self, on: bool):
         """Allow (default) or forbid launching consecutive kernels of a call as programmatic dependents; same results."""

@@ -15,6 +15,7 @@
 #include <vector>
 
 #include "lrgd_convert.cuh"
+#include "lrgd_fit_cluster.cuh"
 #include "lrgd_fit_rows.cuh"
 #include "lrgd_generic.cuh"
 #include "lrgd_reduce.cuh"
@@ -208,6 +209,7 @@ struct lr_ctx {
                                                     // (one such pair per rank when several ranks run as one launch)
     FitParams* d_rank_params = nullptr;             // [kMaxWorld] parameters of the ranks of lr_fit_sharded_local
     int sm_limit = 0;                               // > 0: plans use at most this many SMs (lr_set_sm_limit)
+    int cluster_mode = -1;                          // single-cluster fit kernel for tiny problems: -1 the library chooses, 0 never
     bool coop = false;                              // device supports cooperative launches
     int persistent_mode = -1;                       // single-launch fit kernel: -1 the library chooses, 0 never, 1 whenever the shape allows
     bool overlap = true;                            // consecutive kernels of one call are launched as programmatic dependents
@@ -553,6 +555,72 @@ FitParams fit_params(lr_ctx* ctx, const lr_plan& P, bool bf16, const void* d_X, 
     return fp;
 }
 
+// Cluster sizes the single-cluster fit tries, largest first (sixteen needs the non-portable opt-in).
+constexpr int kClusterSizes[] = {16, 8};
+
+// The plan of the single-cluster fit on a cluster of C CTAs, if the problem allows one: the narrow-row plan for a grid of C
+// CTAs, all of them busy, in which every warp keeps all its batches in shared memory.  The result has the bits of any
+// other form of the fit run under lr_set_sm_limit(C).
+bool cluster_plan(int64_t m, int32_t n, bool aligned16, bool bf16, int C, lr_plan* P, FitLayout* L, int* smem) {
+    if (make_plan(m, n, aligned16, C, P, bf16) != LR_OK || P->variant != 0 || P->grid != C) return false;
+    *L = fit_layout(*P, bf16, m, n, C);
+    const int64_t stage_stride = (int64_t(P->rows_per_batch) * n * (bf16 ? 2 : 4) + 127) & ~int64_t(127);
+    const int64_t need = cluster_fit_smem(n, P->threads / 32, L->depth, int(stage_stride), C);
+    if (!L->resident || need > kMaxDynamicSmem) return false;
+    *smem = int(need);
+    return true;
+}
+
+// Problems whose X fits the shared memory of one thread-block cluster: the whole fit without leaving the cluster (see
+// k_fit_cluster).  Returns cudaErrorNotSupported when the problem or the device does not allow it (the caller then takes
+// the grid-wide persistent kernel).
+cudaError_t launch_cluster_fit(lr_ctx* ctx, bool bf16, const void* d_X, const float* d_y, int64_t m, int32_t n,
+                               float lr, int32_t iters, float* d_w, float* d_b, float* d_loss_hist, cudaStream_t st) {
+    if (ctx->cluster_mode == 0 || ctx->sm_limit > 0) return cudaErrorNotSupported;
+    for (const int C : kClusterSizes) {
+        lr_plan P;
+        FitLayout L;
+        int smem = 0;
+        if (!cluster_plan(m, n, aligned(d_X, 16), bf16, C, &P, &L, &smem)) continue;
+        const cudaError_t e = for_row_shape(P, bf16, [&](auto shape) {
+            using S = decltype(shape);
+            if constexpr (S::Elem::EPG > 1) {
+                auto kern = k_fit_cluster<typename S::Elem, S::nv, S::lpr, S::rb, S::nw>;
+                cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+                if (e == cudaSuccess && C > 8) e = cudaFuncSetAttribute(kern, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+                if (e != cudaSuccess) return e;
+                cudaLaunchConfig_t cfg = {};
+                cfg.gridDim = dim3(C);
+                cfg.blockDim = dim3(P.threads);
+                cfg.dynamicSmemBytes = size_t(smem);
+                cfg.stream = st;
+                cudaLaunchAttribute attr[1];
+                attr[0].id = cudaLaunchAttributeClusterDimension;
+                attr[0].val.clusterDim.x = unsigned(C);
+                attr[0].val.clusterDim.y = 1;
+                attr[0].val.clusterDim.z = 1;
+                cfg.attrs = attr;
+                cfg.numAttrs = 1;
+                int clusters = 0;
+                e = cudaOccupancyMaxActiveClusters(&clusters, kern, &cfg);
+                if (e != cudaSuccess) return e;
+                if (clusters < 1) return cudaErrorNotSupported;   // a cluster of this size cannot be resident here
+                ClusterFitParams cp{};
+                cp.X = d_X; cp.y = d_y; cp.m = m; cp.n = n; cp.w = d_w; cp.b = d_b; cp.loss_hist = d_loss_hist;
+                cp.status = ctx->d_status; cp.depth = L.depth;
+                cp.num_batches = (m + P.rows_per_batch - 1) / P.rows_per_batch;
+                cp.iters = iters; cp.lr = double(lr); cp.inv_m = 1.0 / double(m);
+                return cudaLaunchKernelEx(&cfg, kern, cp);
+            } else {
+                return cudaErrorNotSupported;
+            }
+        });
+        if (e == cudaSuccess) { ctx->launches += 1; return cudaSuccess; }
+        cudaGetLastError();
+    }
+    return cudaErrorNotSupported;
+}
+
 // Enqueues the persistent kernel for a whole fit (fixed count, or with the stopping rule when `tol` is given, or as one
 // rank of a row-sharded fit when `shard` is given).  Returns cudaErrorCooperativeLaunchTooLarge when the CTAs cannot all
 // be resident (the caller then iterates with two kernels), any other error as it comes.
@@ -872,6 +940,7 @@ int fit_impl(lr_ctx* ctx, const void* d_X, bool bf16, const float* d_y, int64_t 
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     // Narrow rows, several iterations: one cooperative launch runs the whole fit (same bits as the loop below).
     if (iters >= 2 && want_persistent(ctx, P, bf16, m, n, iters)) {
+        if (launch_cluster_fit(ctx, bf16, d_X, d_y, m, n, lr, iters, d_w, d_b, d_loss_hist, st) == cudaSuccess) return LR_OK;
         const cudaError_t le = launch_persistent_fit(ctx, P, bf16, d_X, d_y, m, n, lr, iters, d_w, d_b, d_loss_hist, nullptr, st);
         if (le == cudaSuccess) return LR_OK;
         if (le != cudaErrorCooperativeLaunchTooLarge) { ctx->last_cuda = int(le); return LR_ERR_CUDA; }
@@ -927,6 +996,22 @@ int lr_set_overlap(lr_ctx* ctx, int32_t on) {
 int lr_set_persistent(lr_ctx* ctx, int32_t on) {
     if (!ctx) return LR_ERR_NULL;
     ctx->persistent_mode = on < 0 ? -1 : (on > 0 ? 1 : 0);
+    return LR_OK;
+}
+
+int32_t lr_cluster_ctas(int64_t m, int32_t n, int32_t x_aligned16, int32_t bf16) {
+    for (const int C : kClusterSizes) {
+        lr_plan P;
+        FitLayout L;
+        int smem = 0;
+        if (cluster_plan(m, n, x_aligned16 != 0, bf16 != 0, C, &P, &L, &smem)) return C;
+    }
+    return 0;
+}
+
+int lr_set_cluster(lr_ctx* ctx, int32_t on) {
+    if (!ctx) return LR_ERR_NULL;
+    ctx->cluster_mode = on == 0 ? 0 : -1;
     return LR_OK;
 }
 

@@ -154,6 +154,32 @@ __device__ __forceinline__ bool grid_barrier(unsigned int* gbar, unsigned int ta
     return *cta_abort == 0;
 }
 
+// One column of up to 32 partial rows in k_reduce_update's order: a slice is a single row (an absent one counts as 0.0),
+// then the fixed tree (s with s+16, then distance 8, 4, 2, 1).  `row_value(g)` yields the entry of row g; all of them are
+// requested before the first addition.  NW only shapes the loop (slices i, i + NW, ... first: the tree levels of distance >= NW).
+template <int NW, class F>
+__device__ __forceinline__ double single_row_slices_sum(int G, F&& row_value) {
+    constexpr int K = kRedSlices / NW;
+    static_assert(K * NW == kRedSlices && (K & (K - 1)) == 0, "slices must split evenly");
+    double a[NW];
+#pragma unroll
+    for (int i = 0; i < NW; ++i) {
+        double r[K];
+#pragma unroll
+        for (int k = 0; k < K; ++k) r[k] = i + k * NW < G ? row_value(i + k * NW) : 0.0;
+#pragma unroll
+        for (int h = K / 2; h >= 1; h >>= 1)
+#pragma unroll
+            for (int k = 0; k < h; ++k) r[k] += r[k + h];
+        a[i] = r[0];
+    }
+#pragma unroll
+    for (int h = NW / 2; h >= 1; h >>= 1)
+#pragma unroll
+        for (int i = 0; i < h; ++i) a[i] += a[i + h];
+    return a[0];
+}
+
 // Adds up the G partial rows [G][stride] column by column into sums[stride] (shared memory); called by all threads of a
 // CTA, with the order of k_reduce_update so that the result has that kernel's bits: slice s = rows [s*per, (s+1)*per) in
 // index order, then the 32 slice sums in the fixed tree (s with s+16, then distance 8, 4, 2, 1).
@@ -162,8 +188,8 @@ __device__ __forceinline__ bool grid_barrier(unsigned int* gbar, unsigned int ta
 // CTAs read the same rows at the same time: scattered 16-byte reads cost L2 eight times the requests).  The NW per-warp
 // sums of a chunk of 64 columns meet in `buf` and one thread per column finishes the tree.  A thread has at most
 // (32 / NW) * kFitRowChunk 16-byte loads in flight: few enough to live in the registers the streaming loop leaves free.
-// Grids of up to 32 CTAs (small problems, where this call is most of the iteration): a slice is a single row, a lane
-// plays a slice and the tree is a butterfly of shuffles; several column pairs are in flight per warp.
+// Grids of up to 32 CTAs (small problems, where this call is most of the iteration): a slice is a single row and one
+// thread per column holds all rows at once.
 template <int NW>
 __device__ LRGD_FIT_RED_INLINE void reduce_partial_rows(const double* pbuf, int G, int stride, double* buf, double* sums) {
     constexpr int K = kRedSlices / NW;             // slices per warp
@@ -173,23 +199,11 @@ __device__ LRGD_FIT_RED_INLINE void reduce_partial_rows(const double* pbuf, int 
     const int npairs = stride / 2;
     const double2 zero = make_double2(0.0, 0.0);
     if (per == 1) {
-        constexpr int U = 4;                       // column pairs in flight per warp
-        for (int q0 = warp; q0 < npairs; q0 += NW * U) {
-            double2 v[U];
-#pragma unroll
-            for (int u = 0; u < U; ++u) {
-                const int q = q0 + u * NW;
-                v[u] = (q < npairs && lane < G) ? __ldcg(reinterpret_cast<const double2*>(pbuf + static_cast<size_t>(lane) * stride) + q) : zero;
-            }
-#pragma unroll
-            for (int u = 0; u < U; ++u) {
-                const int q = q0 + u * NW;         // warp-uniform
-                if (q < npairs) {
-                    const double tx = slice_tree_sum_warp(v[u].x), ty = slice_tree_sum_warp(v[u].y);
-                    if (lane == 0) { sums[2 * q] = tx; sums[2 * q + 1] = ty; }
-                }
-            }
-        }
+        // a slice is a single row: one thread per column holds all of them at once -- one round trip to L2 and a tree in
+        // registers, no exchange through shared memory or shuffles (at 256 columns a butterfly per column pair took 2.5 us
+        // more; a thread per PAIR of columns needs twice the registers, which the caller's streaming loop pays for)
+        for (int col = threadIdx.x; col < stride; col += NW * 32)
+            sums[col] = single_row_slices_sum<NW>(G, [&](int g) { return __ldcg(pbuf + static_cast<size_t>(g) * stride + col); });
         __syncthreads();
         return;
     }

@@ -143,6 +143,36 @@ def test_pipeline_depth_follows_the_shared_memory_budget():
     assert api.plan_query(100, 32)["stages"] == 1               # one batch per warp at most
 
 
+@pytest.mark.parametrize("m,n,bf16,aligned,want", [
+    (10_000, 32, False, True, 16),      # two batches of 32 rows for most warps of 16 CTAs
+    (4_100, 32, False, True, 8),        # 9 CTA-loads of batches: not enough for sixteen CTAs, enough for eight
+    (3_000, 32, False, True, 0),        # 6 CTA-loads: too few even for a cluster of eight
+    (24_000, 32, False, True, 16),      # three stages per warp
+    (30_001, 32, False, True, 0),       # four stages of 4 KB per warp do not fit beside the received rows
+    (30_001, 32, True, True, 16),       # ... with bfloat16 rows they do
+    (60_000, 32, False, True, 0),       # more rows than a cluster's shared memory holds
+    (1_500, 256, False, True, 16),
+    (3_000, 256, False, True, 0),
+    (3_000, 100, False, True, 16),      # an eight-warp shape
+    (10_000, 32, False, False, 0),      # rows that are not 16-byte groups
+    (10_000, 30, False, True, 0),
+    (2_000, 1028, False, True, 0),      # wide rows have no persistent form
+])
+def test_cluster_plan(m, n, bf16, aligned, want):
+    C = api.cluster_ctas(m, n, x_aligned16=aligned, bf16=bf16)
+    assert C == want
+    if C:
+        # the plan is the narrow-row plan for C SMs with every CTA busy and all batches of a warp resident at once
+        p = api.plan_query(m, n, sm_count=C, bf16=bf16)
+        assert p["variant"] == 0 and p["grid"] == C
+        warps = p["threads"] // 32
+        batches = -(-m // p["rows_per_batch"])
+        per_warp = -(-(-(-batches // warps)) // C)
+        assert per_warp <= 4
+        stage = -(-(p["rows_per_batch"] * n * (2 if bf16 else 4)) // 128) * 128
+        assert warps * per_warp * stage + 2 * C * (n + 2) * 8 < 227 * 1024
+
+
 def test_header_is_plain_c_and_the_example_links():
     # include/lrgd.h must be usable from C (no C++ in the boundary); the example program must compile and link against the
     # built library (it is only run where a GPU exists)

@@ -362,6 +362,66 @@ def test_single_launch_fit_equals_two_kernel_fit_all_shapes(ctx, m, n, bf16):
     assert ctx.device_status() == 0
 
 
+# problems that fit the shared memory of one thread-block cluster run lr_fit there (partial sums pushed from CTA to CTA);
+# clusters of 16 and of 8, one to four batches per warp, ragged last batches, idle warps, and bfloat16 storage.  The bits are
+# those of the other forms with the rows divided among as many CTAs as the cluster has.
+CLUSTER_CASES = [("cfg1", 10_000, False), ("cfg1", 4_100, False), ("cfg1", 7_777, False), ("cfg1", 24_000, False),
+                 ("cfg3", 1_500, False), ("cfg3", 600, False), ("cfg5", 2_000, False), ("cfg5", 12_001, False),
+                 ("higgs_like", 20_003, False), ("cfg2", 3_000, False),
+                 ("cfg1", 10_000, True), ("cfg1", 30_001, True), ("cfg3", 3_000, True), ("cfg3", 1_500, True), ("cfg5", 12_001, True)]
+
+
+@pytest.mark.parametrize("name,m,bf16", CLUSTER_CASES)
+def test_cluster_form_equals_the_other_forms(ctx, name, m, bf16):
+    wl = datagen.scaled(datagen.WORKLOADS[name], m)
+    X, y, _, _ = datagen.generate(wl)
+    if bf16:
+        bits, X = oracle.round_bf16(X)
+        dX = torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16)
+    else:
+        dX = dev(X)
+    C = api.cluster_ctas(wl.m, wl.n, bf16=bf16)
+    assert C in (8, 16), "every case here is meant to have a cluster plan"
+    dy, iters = dev(y), 9
+    try:
+        n0 = ctx.launch_count()
+        w1, b1, h1 = api.lr_fit(dX, dy, wl.lr, iters, return_history=True, ctx=ctx)          # default: the cluster form
+        assert ctx.launch_count() == n0 + 1
+        ctx.set_cluster(False)
+        ctx.set_sm_limit(C)
+        w2, b2, h2 = api.lr_fit(dX, dy, wl.lr, iters, return_history=True, ctx=ctx)          # grid-wide persistent kernel on C CTAs
+        assert ctx.launch_count() == n0 + 2
+        ctx.set_persistent(False)
+        w3, b3, h3 = api.lr_fit(dX, dy, wl.lr, iters, return_history=True, ctx=ctx)          # two kernels per iteration
+        assert ctx.launch_count() == n0 + 2 + 2 * iters
+    finally:
+        ctx.set_cluster(True)
+        ctx.set_sm_limit(0)
+        ctx.set_persistent(None)
+    assert torch.equal(w1, w2) and torch.equal(b1, b2) and torch.equal(h1, h2)
+    assert torch.equal(w1, w3) and torch.equal(b1, b3) and torch.equal(h1, h3)
+    w_ref, b_ref, lh_ref = oracle.fit(X, y, wl.lr, iters)
+    assert rel_l2(np.concatenate([w1.cpu().numpy(), b1.cpu().numpy()]), np.concatenate([w_ref, [b_ref]])) <= W_TOL
+    assert np.max(np.abs(h1.cpu().numpy() - lh_ref)) <= LOSS_TOL
+    assert ctx.device_status() == 0
+
+
+# a fit continued in a second call, and a start point other than zero, on the cluster form
+def test_cluster_form_continues_a_fit(ctx):
+    wl = datagen.scaled(datagen.WORKLOADS["cfg1"], 7_777)
+    X, y, _, _ = datagen.generate(wl)
+    assert api.cluster_ctas(wl.m, wl.n) == 16
+    dX, dy = dev(X), dev(y)
+    w_a, b_a, h_a = api.lr_fit(dX, dy, wl.lr, 12, return_history=True, ctx=ctx)
+    w_b = torch.zeros(wl.n, device="cuda")
+    b_b = torch.zeros(1, device="cuda")
+    h_b = torch.empty(12, device="cuda")
+    ctx.fit(dX, dy, wl.lr, 5, w_b, b_b, h_b[:5])
+    ctx.fit(dX, dy, wl.lr, 7, w_b, b_b, h_b[5:])
+    assert torch.equal(w_a, w_b) and torch.equal(b_a, b_b) and torch.equal(h_a, h_b)
+    assert ctx.device_status() == 0
+
+
 def test_row_sharded_entry_points_match_oracle(ctx):
     # three row shards on one GPU, one after the other (no kernel waits on another): lr_shard_sums per shard,
     # lr_apply_sums over the stacked sums, for several steps; against the checker's unsharded fit
