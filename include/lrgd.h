@@ -111,7 +111,8 @@ int lr_loss_grad(lr_ctx* ctx, const float* d_X, const float* d_y, int64_t m, int
  * problem whose rows all fit the CTAs' shared memory (up to ~28 MB) is fetched once and kept there for the whole call.
  * The library takes the persistent kernel wherever the shape allows it (it measures at least as fast everywhere).
  * lr_set_persistent(ctx, 0) forces two kernels (also used while lr_profile_enable is on, so that single launches can
- * be timed), any other value restores the default.  The same choice applies to lr_fit_tol and the bfloat16 calls.
+ * be timed), a negative value restores the default, and a positive value asks for this persistent kernel in particular
+ * (the default may take the single-cluster form below instead).  The same choice applies to lr_fit_tol and the bfloat16 calls.
  * If a bounded wait inside the persistent kernel expires, the kernel stops, the status word reports LR_ERR_TIMEOUT and
  * d_w, d_b are left as they were on entry.
  */
@@ -120,18 +121,21 @@ int lr_fit(lr_ctx* ctx, const float* d_X, const float* d_y, int64_t m, int32_t n
 int lr_set_persistent(lr_ctx* ctx, int32_t on);
 /*
  * Third form of lr_fit, for problems whose X fits the shared memory of ONE thread-block cluster of 16 (or 8) CTAs (up to
- * ~3 MB; rows of 16-byte groups as for the persistent kernel; at least one batch of rows for every CTA): X is fetched
- * once, and in every iteration each CTA pushes its partial sums into the shared memory of all CTAs of the cluster with
- * asynchronous remote stores that complete on the receiver's mbarrier, so an iteration never touches global memory.
- * Taken by default where it applies and no SM limit is set.  The result has the bits of the other forms run under
- * lr_set_sm_limit(ctx, C), C the cluster size -- the rows are divided among C CTAs instead of all SMs, which changes
- * the order of the sums.  lr_set_cluster(ctx, 0) switches the form off, any other value restores the default.
+ * ~3 MB; rows of 16-byte groups as for the persistent kernel; at least one batch of rows for every CTA).  Such a
+ * problem is planned on that many CTAs by every entry point (lr_plan_query shows grid = 16 or 8), so all of them divide
+ * the rows the same way and all forms of the fit give the same bits.  lr_fit then runs the whole call as one launch on
+ * one cluster: X is fetched once, and in every iteration each CTA pushes its partial sums into the shared memory of all
+ * CTAs of the cluster with asynchronous remote stores that complete on the receiver's mbarrier, so an iteration never
+ * touches global memory (10,000 x 32: 3 us per iteration where the grid-wide persistent kernel takes 4.3).
+ * Taken by default where it applies, unless lr_set_persistent has asked for a particular form.  lr_set_cluster(ctx, 0)
+ * switches the form off (the persistent kernel then runs on the same plan), any other value restores the default.
  * lr_fit_tol and lr_fit_sharded do not use it.  A wait that expires ends the kernel as it ends the persistent one.
- * lr_cluster_ctas (host only, no CUDA call) returns the cluster size the form would use for a shape, 0 if none;
- * whether a cluster of that size can be resident is known at launch only (if not, the persistent kernel runs).
+ * lr_cluster_ctas (host only, no CUDA call; arguments as lr_plan_query) returns the cluster size the form would use
+ * for a shape, 0 if none; whether a cluster of that size can be resident is known at launch only (if not, the
+ * persistent kernel runs).
  */
 int lr_set_cluster(lr_ctx* ctx, int32_t on);
-int32_t lr_cluster_ctas(int64_t m, int32_t n, int32_t x_aligned16, int32_t bf16);
+int32_t lr_cluster_ctas(int64_t m, int32_t n, int32_t x_aligned16, int32_t sm_count, int32_t bf16);
 
 /*
  * Overlap between the kernels of one call (on by default).  Every iteration of the two-kernel form is a pass followed by

@@ -85,7 +85,7 @@ def lib() -> ctypes.CDLL:
         L.lr_set_l2_keep.argtypes = [P, I64]
         L.lr_set_sm_limit.argtypes = [P, I32]
         L.lr_set_cluster.argtypes = [P, I32]
-        L.lr_cluster_ctas.argtypes = [I64, I32, I32, I32]
+        L.lr_cluster_ctas.argtypes = [I64, I32, I32, I32, I32]
         L.lr_cluster_ctas.restype = I32
         L.lr_exchange_bytes.argtypes = [I32, I32, ctypes.POINTER(I64)]
         L.lr_fit_sharded.argtypes = [P, P, P, I64, I64, I32, F, I32, P, P, P, I32, I32, ctypes.POINTER(P), I64, I32, P]
@@ -125,9 +125,9 @@ def plan_query(m: int, n: int, x_aligned16: bool = True, sm_count: int = 148, bf
     return p.as_dict()
 
 
-def cluster_ctas(m: int, n: int, x_aligned16: bool = True, bf16: bool = False) -> int:
+def cluster_ctas(m: int, n: int, x_aligned16: bool = True, sm_count: int = 148, bf16: bool = False) -> int:
     """Cluster size the single-cluster form of ``fit`` would use for an m-by-n problem, 0 if it has none (host only)."""
-    return int(lib().lr_cluster_ctas(int(m), int(n), int(bool(x_aligned16)), int(bool(bf16))))
+    return int(lib().lr_cluster_ctas(int(m), int(n), int(bool(x_aligned16)), int(sm_count), int(bool(bf16))))
 
 
 def exchange_bytes(world: int, n: int) -> int:
@@ -426,12 +426,12 @@ class Context:
 
     def set_persistent(self, on: bool | None):
         """Form of ``fit`` / ``fit_tol``: True = the single-launch persistent kernel wherever the shape allows, False = two
-        kernels per iteration, None = the library chooses (default).  Results are identical either way."""
+        kernels per iteration, None = the library chooses (default; small problems may then run on one thread-block
+        cluster, see ``set_cluster``).  True and False give identical results."""
         self._check(lib().lr_set_persistent(self._h, -1 if on is None else int(bool(on))), "lr_set_persistent")
 
     def set_cluster(self, on: bool):
-        """Allow (default) or forbid the single-cluster form of ``fit``.  Its results are those of the other forms under
-        ``set_sm_limit(cluster_ctas(m, n))``."""
+        """Allow (default) or forbid the single-cluster form of ``fit`` for small problems; same results either way."""
         self._check(lib().lr_set_cluster(self._h, int(bool(on))), "lr_set_cluster")
 
     def set_overlap(self, on: bool):

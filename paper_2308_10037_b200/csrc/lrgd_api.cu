@@ -75,6 +75,24 @@ bool any_row_shape_for(int n, RowShape* s) {
 }
 
 // bf16: X holds bfloat16 (2-byte) elements instead of fp32; a 16-byte group is then 8 columns instead of 4.
+// Cluster sizes of the single-cluster fit, largest first (sixteen needs the non-portable opt-in).
+constexpr int kClusterSizes[] = {16, 8};
+
+// A narrow-row problem of `slots` CTA-loads of batches (nw batches each) whose rows all fit the shared memory of one
+// thread-block cluster of C <= sms CTAs, every CTA busy, is PLANNED on C CTAs -- for every entry point, so that all of
+// them divide the rows the same way and give the same bits as the single-cluster fit (k_fit_cluster), which is what
+// lr_fit then runs.  Returns C, or 0 if the problem is not of that kind.
+int cluster_size_for(int64_t slots, int nw, int64_t stage_stride, int32_t n, int32_t sms) {
+    for (const int C : kClusterSizes) {
+        if (C > sms || slots < C) continue;
+        const int64_t per_warp = (slots + C - 1) / C;                          // stages per warp: all its batches at once
+        if (per_warp > kMaxDepth) continue;
+        if (kHeaderBytes + nw * per_warp * stage_stride + fit_tail_bytes(n) + 2LL * C * (n + 2) * 8 + 16 > kMaxDynamicSmem) continue;
+        return C;
+    }
+    return 0;
+}
+
 int make_plan(int64_t m, int32_t n, bool aligned16, int32_t sms, lr_plan* P, bool bf16 = false) {
     if (!P) return LR_ERR_NULL;
     if (m < 1 || m > kMaxRows || n < 1 || sms < 1) return LR_ERR_SHAPE;
@@ -89,9 +107,10 @@ int make_plan(int64_t m, int32_t n, bool aligned16, int32_t sms, lr_plan* P, boo
         const int rpb = rs.rb * (32 / rs.lpr);                                  // rows per batch = rows per stage
         const int64_t B = (m + rpb - 1) / rpb;                                  // batches
         const int64_t slots = (B + rs.nw - 1) / rs.nw;                              // CTA-level groups of nw batches
-        const int grid = int(std::min<int64_t>(slots, sms));
-        const int64_t per_warp = (slots + grid - 1) / grid;                     // most batches any warp handles
         const int64_t stage_stride = (int64_t(rpb) * n * eb + (any_len ? 16 : 0) + 127) & ~int64_t(127);   // as the kernel lays it out
+        const int cluster = grouped ? cluster_size_for(slots, rs.nw, stage_stride, n, sms) : 0;
+        const int grid = cluster ? cluster : int(std::min<int64_t>(slots, sms));
+        const int64_t per_warp = (slots + grid - 1) / grid;                     // most batches any warp handles
         int D = int(std::min<int64_t>(kMaxDepth, kStageBudgetBytes / (rs.nw * stage_stride)));
         D = int(std::min<int64_t>(D, per_warp));
         if (D < 1) D = 1;
@@ -555,69 +574,65 @@ FitParams fit_params(lr_ctx* ctx, const lr_plan& P, bool bf16, const void* d_X, 
     return fp;
 }
 
-// Cluster sizes the single-cluster fit tries, largest first (sixteen needs the non-portable opt-in).
-constexpr int kClusterSizes[] = {16, 8};
-
-// The plan of the single-cluster fit on a cluster of C CTAs, if the problem allows one: the narrow-row plan for a grid of C
-// CTAs, all of them busy, in which every warp keeps all its batches in shared memory.  The result has the bits of any
-// other form of the fit run under lr_set_sm_limit(C).
-bool cluster_plan(int64_t m, int32_t n, bool aligned16, bool bf16, int C, lr_plan* P, FitLayout* L, int* smem) {
-    if (make_plan(m, n, aligned16, C, P, bf16) != LR_OK || P->variant != 0 || P->grid != C) return false;
-    *L = fit_layout(*P, bf16, m, n, C);
-    const int64_t stage_stride = (int64_t(P->rows_per_batch) * n * (bf16 ? 2 : 4) + 127) & ~int64_t(127);
-    const int64_t need = cluster_fit_smem(n, P->threads / 32, L->depth, int(stage_stride), C);
-    if (!L->resident || need > kMaxDynamicSmem) return false;
-    *smem = int(need);
-    return true;
+// Whether a plan is one that make_plan put on a cluster's worth of CTAs (see cluster_size_for): returns the cluster size with
+// the layout and the dynamic shared memory of k_fit_cluster, or 0.
+int cluster_plan(const lr_plan& P, bool bf16, int64_t m, int32_t n, FitLayout* L, int* smem) {
+    if (P.variant != 0) return 0;
+    const int nw = P.threads / 32;
+    const int64_t stage_stride = (int64_t(P.rows_per_batch) * n * (bf16 ? 2 : 4) + 127) & ~int64_t(127);
+    const int64_t B = (m + P.rows_per_batch - 1) / P.rows_per_batch;
+    const int C = cluster_size_for((B + nw - 1) / nw, nw, stage_stride, n, P.grid);   // (C <= grid rules out larger clusters than planned)
+    if (C == 0 || C != P.grid) return 0;
+    *L = fit_layout(P, bf16, m, n, C);
+    *smem = cluster_fit_smem(n, nw, L->depth, int(stage_stride), C);
+    return L->resident ? C : 0;
 }
 
 // Problems whose X fits the shared memory of one thread-block cluster: the whole fit without leaving the cluster (see
 // k_fit_cluster).  Returns cudaErrorNotSupported when the problem or the device does not allow it (the caller then takes
-// the grid-wide persistent kernel).
-cudaError_t launch_cluster_fit(lr_ctx* ctx, bool bf16, const void* d_X, const float* d_y, int64_t m, int32_t n,
+// the grid-wide persistent kernel, which gives the same bits on the same plan).
+cudaError_t launch_cluster_fit(lr_ctx* ctx, const lr_plan& P, bool bf16, const void* d_X, const float* d_y, int64_t m, int32_t n,
                                float lr, int32_t iters, float* d_w, float* d_b, float* d_loss_hist, cudaStream_t st) {
-    if (ctx->cluster_mode == 0 || ctx->sm_limit > 0) return cudaErrorNotSupported;
-    for (const int C : kClusterSizes) {
-        lr_plan P;
-        FitLayout L;
-        int smem = 0;
-        if (!cluster_plan(m, n, aligned(d_X, 16), bf16, C, &P, &L, &smem)) continue;
-        const cudaError_t e = for_row_shape(P, bf16, [&](auto shape) {
-            using S = decltype(shape);
-            if constexpr (S::Elem::EPG > 1) {
-                auto kern = k_fit_cluster<typename S::Elem, S::nv, S::lpr, S::rb, S::nw>;
-                cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-                if (e == cudaSuccess && C > 8) e = cudaFuncSetAttribute(kern, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
-                if (e != cudaSuccess) return e;
-                cudaLaunchConfig_t cfg = {};
-                cfg.gridDim = dim3(C);
-                cfg.blockDim = dim3(P.threads);
-                cfg.dynamicSmemBytes = size_t(smem);
-                cfg.stream = st;
-                cudaLaunchAttribute attr[1];
-                attr[0].id = cudaLaunchAttributeClusterDimension;
-                attr[0].val.clusterDim.x = unsigned(C);
-                attr[0].val.clusterDim.y = 1;
-                attr[0].val.clusterDim.z = 1;
-                cfg.attrs = attr;
-                cfg.numAttrs = 1;
-                int clusters = 0;
-                e = cudaOccupancyMaxActiveClusters(&clusters, kern, &cfg);
-                if (e != cudaSuccess) return e;
-                if (clusters < 1) return cudaErrorNotSupported;   // a cluster of this size cannot be resident here
-                ClusterFitParams cp{};
-                cp.X = d_X; cp.y = d_y; cp.m = m; cp.n = n; cp.w = d_w; cp.b = d_b; cp.loss_hist = d_loss_hist;
-                cp.status = ctx->d_status; cp.depth = L.depth;
-                cp.num_batches = (m + P.rows_per_batch - 1) / P.rows_per_batch;
-                cp.iters = iters; cp.lr = double(lr); cp.inv_m = 1.0 / double(m);
-                return cudaLaunchKernelEx(&cfg, kern, cp);
-            } else {
-                return cudaErrorNotSupported;
-            }
-        });
-        if (e == cudaSuccess) { ctx->launches += 1; return cudaSuccess; }
-        cudaGetLastError();
-    }
+    if (ctx->cluster_mode == 0 || ctx->persistent_mode != -1) return cudaErrorNotSupported;
+    FitLayout L;
+    int smem = 0;
+    const int C = cluster_plan(P, bf16, m, n, &L, &smem);
+    if (C == 0) return cudaErrorNotSupported;
+    const cudaError_t e = for_row_shape(P, bf16, [&](auto shape) {
+        using S = decltype(shape);
+        if constexpr (S::Elem::EPG > 1) {
+            auto kern = k_fit_cluster<typename S::Elem, S::nv, S::lpr, S::rb, S::nw>;
+            cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+            if (e == cudaSuccess && C > 8) e = cudaFuncSetAttribute(kern, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+            if (e != cudaSuccess) return e;
+            cudaLaunchConfig_t cfg = {};
+            cfg.gridDim = dim3(C);
+            cfg.blockDim = dim3(P.threads);
+            cfg.dynamicSmemBytes = size_t(smem);
+            cfg.stream = st;
+            cudaLaunchAttribute attr[1];
+            attr[0].id = cudaLaunchAttributeClusterDimension;
+            attr[0].val.clusterDim.x = unsigned(C);
+            attr[0].val.clusterDim.y = 1;
+            attr[0].val.clusterDim.z = 1;
+            cfg.attrs = attr;
+            cfg.numAttrs = 1;
+            int clusters = 0;
+            e = cudaOccupancyMaxActiveClusters(&clusters, kern, &cfg);
+            if (e != cudaSuccess) return e;
+            if (clusters < 1) return cudaErrorNotSupported;   // a cluster of this size cannot be resident here
+            ClusterFitParams cp{};
+            cp.X = d_X; cp.y = d_y; cp.m = m; cp.n = n; cp.w = d_w; cp.b = d_b; cp.loss_hist = d_loss_hist;
+            cp.status = ctx->d_status; cp.depth = L.depth;
+            cp.num_batches = (m + P.rows_per_batch - 1) / P.rows_per_batch;
+            cp.iters = iters; cp.lr = double(lr); cp.inv_m = 1.0 / double(m);
+            return cudaLaunchKernelEx(&cfg, kern, cp);
+        } else {
+            return cudaErrorNotSupported;
+        }
+    });
+    if (e == cudaSuccess) { ctx->launches += 1; return cudaSuccess; }
+    cudaGetLastError();
     return cudaErrorNotSupported;
 }
 
@@ -940,7 +955,7 @@ int fit_impl(lr_ctx* ctx, const void* d_X, bool bf16, const float* d_y, int64_t 
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     // Narrow rows, several iterations: one cooperative launch runs the whole fit (same bits as the loop below).
     if (iters >= 2 && want_persistent(ctx, P, bf16, m, n, iters)) {
-        if (launch_cluster_fit(ctx, bf16, d_X, d_y, m, n, lr, iters, d_w, d_b, d_loss_hist, st) == cudaSuccess) return LR_OK;
+        if (launch_cluster_fit(ctx, P, bf16, d_X, d_y, m, n, lr, iters, d_w, d_b, d_loss_hist, st) == cudaSuccess) return LR_OK;
         const cudaError_t le = launch_persistent_fit(ctx, P, bf16, d_X, d_y, m, n, lr, iters, d_w, d_b, d_loss_hist, nullptr, st);
         if (le == cudaSuccess) return LR_OK;
         if (le != cudaErrorCooperativeLaunchTooLarge) { ctx->last_cuda = int(le); return LR_ERR_CUDA; }
@@ -999,14 +1014,12 @@ int lr_set_persistent(lr_ctx* ctx, int32_t on) {
     return LR_OK;
 }
 
-int32_t lr_cluster_ctas(int64_t m, int32_t n, int32_t x_aligned16, int32_t bf16) {
-    for (const int C : kClusterSizes) {
-        lr_plan P;
-        FitLayout L;
-        int smem = 0;
-        if (cluster_plan(m, n, x_aligned16 != 0, bf16 != 0, C, &P, &L, &smem)) return C;
-    }
-    return 0;
+int32_t lr_cluster_ctas(int64_t m, int32_t n, int32_t x_aligned16, int32_t sm_count, int32_t bf16) {
+    lr_plan P;
+    FitLayout L;
+    int smem = 0;
+    if (make_plan(m, n, x_aligned16 != 0, sm_count, &P, bf16 != 0) != LR_OK) return 0;
+    return cluster_plan(P, bf16 != 0, m, n, &L, &smem);
 }
 
 int lr_set_cluster(lr_ctx* ctx, int32_t on) {
@@ -1595,24 +1608,36 @@ extern "C" int lr_loss_grad_noalloc(int32_t device, const float* d_X, const floa
     NoAllocDevice* dev = nullptr;
     int rc = noalloc_setup(device, &dev);
     if (rc != LR_OK) return rc;
-    // n <= LR_NOALLOC_MAX_N, so the plan is always one of the two narrow-row staged kernels (16-byte groups, or single
-    // elements for odd lengths and 4-byte-aligned matrices), whose grid never exceeds the SM count given here
+    // n <= LR_NOALLOC_MAX_N, so the plan is one of the narrow-row staged kernels (16-byte groups, or single elements for odd
+    // lengths and 4-byte-aligned matrices) or, for such rows of more than 512 columns, the kernel with CTA-wide stages; the
+    // grid never exceeds the SM count given here
     lr_plan P;
     rc = make_plan(m, n, aligned(d_X, 16), std::min(dev->sm_count, kNoAllocMaxGrid), &P);
     if (rc != LR_OK) return rc;
-    if ((P.variant != 0 && P.variant != 3) || P.grid > kNoAllocMaxGrid) return LR_ERR_SHAPE;
+    if ((P.variant != 0 && P.variant != 3 && P.variant != 4) || P.grid > kNoAllocMaxGrid) return LR_ERR_SHAPE;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     double* partial = dev->scratch;
     int* status = d_status ? d_status : reinterpret_cast<int*>(dev->scratch + size_t(kNoAllocMaxGrid) * kNoAllocRowDoubles);
     // the array keeps whatever the previous call left: the status word must start at zero (the partial rows are
     // fully rewritten by the CTAs that the reduction reads)
     if (cudaMemsetAsync(status, 0, sizeof(int), st) != cudaSuccess) return LR_ERR_CUDA;
-    StreamParams sp{};
-    sp.X = d_X; sp.y = d_y; sp.m = m; sp.n = n; sp.w = d_w; sp.b = d_b;
-    sp.partial = partial; sp.labels = nullptr; sp.cut = 0.f; sp.status = status;
-    sp.depth = P.stages;
-    sp.num_batches = (m + P.rows_per_batch - 1) / P.rows_per_batch;
-    const cudaError_t e = launch_rows<false>(P, sp, st);
+    cudaError_t e;
+    if (P.variant == 4) {
+        WideParams wp{};
+        wp.X = d_X; wp.y = d_y; wp.m = m; wp.n = n; wp.w = d_w; wp.b = d_b;
+        wp.partial = partial; wp.labels = nullptr; wp.cut = 0.f; wp.status = status;
+        wp.depth = P.stages;
+        wp.cw = (n + P.threads / 32 - 1) / (P.threads / 32);
+        wp.num_batches = (m + P.rows_per_batch - 1) / P.rows_per_batch;
+        e = launch_wide<false>(P, wp, st, false, false);
+    } else {
+        StreamParams sp{};
+        sp.X = d_X; sp.y = d_y; sp.m = m; sp.n = n; sp.w = d_w; sp.b = d_b;
+        sp.partial = partial; sp.labels = nullptr; sp.cut = 0.f; sp.status = status;
+        sp.depth = P.stages;
+        sp.num_batches = (m + P.rows_per_batch - 1) / P.rows_per_batch;
+        e = launch_rows<false>(P, sp, st);
+    }
     if (e != cudaSuccess) return LR_ERR_CUDA;
     ReduceParams rp{};
     rp.partial = partial; rp.G = P.grid; rp.n = n; rp.inv_m = 1.0 / double(m); rp.lr = 0.0; rp.update = 0;

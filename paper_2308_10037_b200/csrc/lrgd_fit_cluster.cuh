@@ -136,11 +136,24 @@ __global__ void __launch_bounds__(NW * 32, 1) k_fit_cluster(const __grid_constan
     const int myr = ((sub >> SHIFT) & (RB - 1)) * RPW + slot;
     const bool owner = (sub & ((1 << SHIFT) - 1)) == 0;
     const bool full_cols = n4 == NV * LPR;
-    const float y_first = (cnt > 0 && first_row + myr < p.m) ? __ldg(p.y + first_row + myr) : 0.f;
+    float yreg[kMaxDepth];                         // y of this lane's row in each of the warp's batches: the same in every iteration
+#pragma unroll
+    for (int i = 0; i < kMaxDepth; ++i) {
+        const long long r = first_row + i * stride_rows + myr;
+        yreg[i] = (i < cnt && r < p.m) ? __ldg(p.y + r) : 0.f;
+    }
+    // where the pushes of this warp go: the slot of this CTA and the mbarrier in the CTAs warp, warp + NW, ...
+    constexpr int DPW = (kClusterMaxCtas + NW - 1) / NW;
+    uint32_t push_slot[DPW], push_bar[DPW];
+#pragma unroll
+    for (int j = 0; j < DPW; ++j) {
+        const int r = warp + j * NW < C ? warp + j * NW : 0;
+        push_slot[j] = map_to_cta(smem_u32(slots) + static_cast<uint32_t>(cta) * stride * 8u, r);
+        push_bar[j] = map_to_cta(smem_u32(xbar), r);
+    }
 
     cluster.sync();                                // everybody's mbarriers exist before anybody sends
 
-    const uint32_t slots_addr = smem_u32(slots), xbar_addr = smem_u32(xbar);
     bool alive = true;                             // CTA-uniform
     bool staged = false;                           // this warp's stages have landed (they are waited for in the first iteration)
     for (int t = 0; t < p.iters && alive; ++t) {
@@ -160,7 +173,6 @@ __global__ void __launch_bounds__(NW * 32, 1) k_fit_cluster(const __grid_constan
             for (int c = 0; c < EPG; ++c) dacc[k][c] = 0.0;
         int since_flush = 0;
         long long row0 = first_row;
-        float y_next = y_first;
         bool ok = true;                            // warp-uniform until the exchange wait below
 
         for (int i = 0; i < cnt; ++i) {
@@ -174,11 +186,9 @@ __global__ void __launch_bounds__(NW * 32, 1) k_fit_cluster(const __grid_constan
             uint4 x[RB][NV];
             load_row_batch<uint4, NV, LPR, RB>(x, t4, rows, n4, full_cols && rows == RPB, sub, slot);
             const bool myvalid = myr < rows;
-            const float yv = y_next;
-            {
-                const long long rn = row0 + stride_rows + myr;
-                y_next = (i + 1 < cnt && rn < p.m) ? __ldg(p.y + rn) : 0.f;
-            }
+            float yv = yreg[0];
+#pragma unroll
+            for (int j = 1; j < kMaxDepth; ++j) yv = i == j ? yreg[j] : yv;
             const float z = batch_dot<E, NV, LPR, RB>(x, lm, lane) + bval;
             float e, L;
             logistic_terms(z, yv, e, L);
@@ -196,55 +206,82 @@ __global__ void __launch_bounds__(NW * 32, 1) k_fit_cluster(const __grid_constan
 
         // ---- fixed-order combine of the CTA's warps (as k_fit_rows and k_stream_rows do) into my_row ----
 #pragma unroll
-        for (int k2 = 0; k2 < NV; ++k2)
-#pragma unroll
-            for (int c = 0; c < EPG; ++c) {
-                double tsum = 0.0;
-#pragma unroll
-                for (int sidx = 0; sidx < RPW; ++sidx) tsum += __shfl_sync(FULL, dacc[k2][c], sub + sidx * LPR);
-                dacc[k2][c] = tsum;
-            }
-#pragma unroll
         for (int msk = 16; msk >= 1; msk >>= 1) {
             dse += __shfl_xor_sync(FULL, dse, msk);
             dsl += __shfl_xor_sync(FULL, dsl, msk);
         }
         if (lane == 0) { red_e[warp] = dse; red_l[warp] = dsl; }
-        for (int c0 = 0; c0 < n; c0 += kFitCombineCols) {
+        // Several row slots per warp and all of them fit the combine buffer at once (narrow fp32 rows): every lane stores its
+        // sums and the combining thread adds a warp's slots in slot order itself -- the additions of slot_order_sum without
+        // its shuffles (32 per warp, on a unit that issues one per clock for the whole SM).
+        constexpr int NC = NV * LPR * EPG;         // columns a warp's lanes cover
+        constexpr bool kSlotsInSmem = RPW > 1 && RPW * NC <= kFitCombineCols;
+        if constexpr (kSlotsInSmem) {
 #pragma unroll
-            for (int k2 = 0; k2 < NV; ++k2) {
-                const int idx = sub + k2 * LPR;
-                const int col = idx * EPG - c0;
-                if (slot == 0 && idx < n4 && col >= 0 && col < kFitCombineCols) {
+            for (int k2 = 0; k2 < NV; ++k2)
 #pragma unroll
-                    for (int c = 0; c < EPG; ++c) red[warp * kFitCombineCols + col + c] = dacc[k2][c];
+                for (int c = 0; c < EPG; c += 2)
+                    *reinterpret_cast<double2*>(red + (warp * RPW + slot) * NC + (sub + k2 * LPR) * EPG + c) = make_double2(dacc[k2][c], dacc[k2][c + 1]);
+            __syncthreads();
+            if (threadIdx.x < n) {
+                double a[NW];                      // per warp: its slots in slot order from +0.0; then warp_tree_sum's tree
+#pragma unroll
+                for (int wi = 0; wi < NW; ++wi) {
+                    double ws = 0.0;
+#pragma unroll
+                    for (int sidx = 0; sidx < RPW; ++sidx) ws += red[(wi * RPW + sidx) * NC + threadIdx.x];
+                    a[wi] = ws;
                 }
-            }
-            __syncthreads();
-            if (threadIdx.x < kFitCombineCols && c0 + threadIdx.x < n) {
-                double tsum = 0.0;
-                for (int wi = 0; wi < NW; ++wi) tsum += red[wi * kFitCombineCols + threadIdx.x];
-                my_row[c0 + threadIdx.x] = tsum;
-            } else if (c0 + kFitCombineCols >= n && threadIdx.x >= NW * 32 - 2) {   // with the last chunk: the two scalar sums
+#pragma unroll
+                for (int h = NW / 2; h >= 1; h >>= 1)
+#pragma unroll
+                    for (int i = 0; i < h; ++i) a[i] += a[i + h];
+                my_row[threadIdx.x] = a[0] + 0.0;
+            } else if (threadIdx.x >= NW * 32 - 2) {
                 const int which = threadIdx.x - (NW * 32 - 2);
-                const double* src = which == 0 ? red_e : red_l;
-                double tsum = 0.0;
-                for (int wi = 0; wi < NW; ++wi) tsum += src[wi];
-                my_row[n + which] = tsum;
+                my_row[n + which] = warp_tree_sum<NW>(which == 0 ? red_e : red_l, 1);
             }
             __syncthreads();
+        } else {
+#pragma unroll
+            for (int k2 = 0; k2 < NV; ++k2)
+#pragma unroll
+                for (int c = 0; c < EPG; ++c) dacc[k2][c] = slot_order_sum<LPR>(dacc[k2][c], sub);
+            for (int c0 = 0; c0 < n; c0 += kFitCombineCols) {
+#pragma unroll
+                for (int k2 = 0; k2 < NV; ++k2) {
+                    const int idx = sub + k2 * LPR;
+                    const int col = idx * EPG - c0;
+                    if (slot == 0 && idx < n4 && col >= 0 && col < kFitCombineCols) {
+#pragma unroll
+                        for (int c = 0; c < EPG; ++c) red[warp * kFitCombineCols + col + c] = dacc[k2][c];
+                    }
+                }
+                __syncthreads();
+                if (threadIdx.x < kFitCombineCols && c0 + threadIdx.x < n) {
+                    my_row[c0 + threadIdx.x] = warp_tree_sum<NW>(red + threadIdx.x, kFitCombineCols);
+                } else if (c0 + kFitCombineCols >= n && threadIdx.x >= NW * 32 - 2) {   // with the last chunk: the two scalar sums
+                    const int which = threadIdx.x - (NW * 32 - 2);
+                    my_row[n + which] = warp_tree_sum<NW>(which == 0 ? red_e : red_l, 1);
+                }
+                __syncthreads();
+            }
         }
 
         // ---- this CTA's row into slot [set][cta] of every CTA (its own included), 16 bytes per store ----
         if (*abort_flag == 0) {                    // CTA-uniform here: a CTA that gave up on its stages sends nothing more
-            const int total = C * npairs;
-            for (int idx = threadIdx.x; idx < total; idx += NW * 32) {
-                const int r = idx / npairs, q = idx - r * npairs;
-                const double2 v = reinterpret_cast<const double2*>(my_row)[q];
-                const uint32_t dst = slots_addr + static_cast<uint32_t>(((set * C + cta) * stride + 2 * q) * 8);
-                st_async_f64x2(map_to_cta(dst, r), v.x, v.y, map_to_cta(xbar_addr + set * 8u, r));
+            const uint32_t set_off = static_cast<uint32_t>(set) * C * stride * 8u;
+#pragma unroll
+            for (int j = 0; j < DPW; ++j) {
+                if (warp + j * NW < C) {           // warp-uniform
+                    for (int q = lane; q < npairs; q += 32) {
+                        const double2 v = reinterpret_cast<const double2*>(my_row)[q];
+                        st_async_f64x2(push_slot[j] + set_off + static_cast<uint32_t>(q) * 16u, v.x, v.y, push_bar[j] + set * 8u);
+                    }
+                }
             }
-            ok = mbar_wait_bounded(&xbar[set], static_cast<uint32_t>(t >> 1) & 1u, abort_flag);
+            // only the threads that read the rows wait for them; the others go on to the barrier below
+            if (threadIdx.x < stride) ok = mbar_wait_bounded(&xbar[set], static_cast<uint32_t>(t >> 1) & 1u, abort_flag);
         } else {
             ok = false;
         }

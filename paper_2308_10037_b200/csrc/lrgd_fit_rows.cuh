@@ -162,16 +162,23 @@ __device__ __forceinline__ double single_row_slices_sum(int G, F&& row_value) {
     constexpr int K = kRedSlices / NW;
     static_assert(K * NW == kRedSlices && (K & (K - 1)) == 0, "slices must split evenly");
     double a[NW];
+    if (G <= NW) {
+        // slices NW and up are absent: each would add +0.0 to a row entry, which leaves it as it is (an entry is never -0.0:
+        // warp_tree_sum ends with + 0.0)
 #pragma unroll
-    for (int i = 0; i < NW; ++i) {
-        double r[K];
+        for (int i = 0; i < NW; ++i) a[i] = i < G ? row_value(i) : 0.0;
+    } else {
 #pragma unroll
-        for (int k = 0; k < K; ++k) r[k] = i + k * NW < G ? row_value(i + k * NW) : 0.0;
+        for (int i = 0; i < NW; ++i) {
+            double r[K];
 #pragma unroll
-        for (int h = K / 2; h >= 1; h >>= 1)
+            for (int k = 0; k < K; ++k) r[k] = i + k * NW < G ? row_value(i + k * NW) : 0.0;
 #pragma unroll
-            for (int k = 0; k < h; ++k) r[k] += r[k + h];
-        a[i] = r[0];
+            for (int h = K / 2; h >= 1; h >>= 1)
+#pragma unroll
+                for (int k = 0; k < h; ++k) r[k] += r[k + h];
+            a[i] = r[0];
+        }
     }
 #pragma unroll
     for (int h = NW / 2; h >= 1; h >>= 1)
@@ -506,12 +513,7 @@ __device__ __forceinline__ void fit_rows_body(const FitParams& p, const int cta,
 #pragma unroll
         for (int k2 = 0; k2 < NV; ++k2)
 #pragma unroll
-            for (int c = 0; c < EPG; ++c) {
-                double tsum = 0.0;
-#pragma unroll
-                for (int sidx = 0; sidx < RPW; ++sidx) tsum += __shfl_sync(FULL, dacc[k2][c], sub + sidx * LPR);
-                dacc[k2][c] = tsum;
-            }
+            for (int c = 0; c < EPG; ++c) dacc[k2][c] = slot_order_sum<LPR>(dacc[k2][c], sub);
 #pragma unroll
         for (int msk = 16; msk >= 1; msk >>= 1) {
             dse += __shfl_xor_sync(FULL, dse, msk);
@@ -530,19 +532,11 @@ __device__ __forceinline__ void fit_rows_body(const FitParams& p, const int cta,
                 }
             }
             __syncthreads();
-            if (threadIdx.x < kFitCombineCols && c0 + threadIdx.x < n) {
-                double tsum = 0.0;
-                for (int wi = 0; wi < NW; ++wi) tsum += red[wi * kFitCombineCols + threadIdx.x];
-                out[c0 + threadIdx.x] = tsum;
-            }
+            if (threadIdx.x < kFitCombineCols && c0 + threadIdx.x < n)
+                out[c0 + threadIdx.x] = warp_tree_sum<NW>(red + threadIdx.x, kFitCombineCols);
             __syncthreads();
         }
-        if (threadIdx.x < 2) {
-            const double* src = threadIdx.x == 0 ? red_e : red_l;
-            double tsum = 0.0;
-            for (int wi = 0; wi < NW; ++wi) tsum += src[wi];
-            out[n + threadIdx.x] = tsum;
-        }
+        if (threadIdx.x < 2) out[n + threadIdx.x] = warp_tree_sum<NW>(threadIdx.x == 0 ? red_e : red_l, 1);
 
         barrier_no += 1;
         alive = grid_barrier(p.gbar, static_cast<unsigned int>(G) * barrier_no, p.status, abort_flag);

@@ -103,6 +103,38 @@ __device__ __forceinline__ void fold_into_fp64(typename E::template Lane<NV>& lm
     dse += se; dsl += sl; se = 0.f; sl = 0.f;
 }
 
+// Sum of a value over the row slots of a warp that own the same columns (lanes sub, sub + LPR, ...), in slot order, starting
+// from +0.0; every lane gets it.  With one slot per warp the value itself (it may then be -0.0 where the sum would be +0.0:
+// the combine of the CTA's warps starts from +0.0 and wipes that out).
+template <int LPR>
+__device__ __forceinline__ double slot_order_sum(double v, int sub) {
+    constexpr int RPW = 32 / LPR;
+    if constexpr (RPW == 1) {
+        return v;
+    } else {
+        double t = 0.0;
+#pragma unroll
+        for (int sidx = 0; sidx < RPW; ++sidx) t += __shfl_sync(0xffffffffu, v, sub + sidx * LPR);
+        return t;
+    }
+}
+
+// Sum of the per-warp values src[0], src[step], ..., src[(NW-1) step] in a fixed pairwise tree (warp w with w + NW/2, then
+// distance NW/4, ... 1), plus +0.0 so that the result is never -0.0.  The order every narrow-row kernel uses for the combine
+// of a CTA's warps: log2(NW) dependent fp64 additions instead of NW in a row (which is what a thread waits for).
+template <int NW>
+__device__ __forceinline__ double warp_tree_sum(const double* src, size_t step) {
+    static_assert((NW & (NW - 1)) == 0, "a power of two of warps");
+    double a[NW];
+#pragma unroll
+    for (int i = 0; i < NW; ++i) a[i] = src[i * step];
+#pragma unroll
+    for (int h = NW / 2; h >= 1; h >>= 1)
+#pragma unroll
+        for (int i = 0; i < h; ++i) a[i] += a[i + h];
+    return a[0] + 0.0;
+}
+
 // one batch from a narrow-row stage into registers (rows packed at n4 groups; lanes beyond the row or rows beyond the
 // matrix read zeros); `full` = every lane's groups exist and the batch is complete: no bounds logic
 template <class Raw, int NV, int LPR, int RB>
@@ -336,9 +368,7 @@ __global__ void __launch_bounds__(NW * 32, 1) k_stream_rows(const StreamParams p
         for (int k2 = 0; k2 < NV; ++k2) {
 #pragma unroll
             for (int c = 0; c < EPG; ++c) {
-                double t = 0.0;
-#pragma unroll
-                for (int sidx = 0; sidx < RPW; ++sidx) t += __shfl_sync(FULL, dacc[k2][c], sub + sidx * LPR);
+                const double t = slot_order_sum<LPR>(dacc[k2][c], sub);
                 const int idx = sub + k2 * LPR;
                 if (slot == 0 && idx < n4) red[static_cast<size_t>(warp) * n + idx * EPG + c] = t;
             }
@@ -352,14 +382,7 @@ __global__ void __launch_bounds__(NW * 32, 1) k_stream_rows(const StreamParams p
         __syncthreads();
         double* out = p.partial + static_cast<size_t>(blockIdx.x) * (n + 2);
         for (int c = threadIdx.x; c < n + 2; c += blockDim.x) {
-            double t = 0.0;
-            if (c < n) {
-                for (int wi = 0; wi < NW; ++wi) t += red[static_cast<size_t>(wi) * n + c];
-            } else {
-                const double* src = (c == n) ? red_e : red_l;
-                for (int wi = 0; wi < NW; ++wi) t += src[wi];
-            }
-            out[c] = t;
+            out[c] = c < n ? warp_tree_sum<NW>(red + c, static_cast<size_t>(n)) : warp_tree_sum<NW>(c == n ? red_e : red_l, 1);
         }
     }
 }

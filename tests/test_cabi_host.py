@@ -65,7 +65,8 @@ def test_plan_staged_shapes(m, n, lpr, nv, nw):
     assert 1024 + nw * p["stages"] * stage <= p["smem_bytes"]
     # the warps of a CTA take one batch each per round; the grid never exceeds the rounds available
     batches = -(-m // p["rows_per_batch"])
-    assert p["grid"] == min(-(-batches // nw), 148)
+    # (a problem that fits the shared memory of one thread-block cluster is planned on that cluster's CTAs)
+    assert p["grid"] == (api.cluster_ctas(m, n) or min(-(-batches // nw), 148))
     if nw == 8 and nv == 1:
         assert p["rows_per_batch"] == 16                      # 68..128 fp32 columns: sixteen rows per batch, eight warps
 
@@ -162,9 +163,11 @@ def test_cluster_plan(m, n, bf16, aligned, want):
     C = api.cluster_ctas(m, n, x_aligned16=aligned, bf16=bf16)
     assert C == want
     if C:
-        # the plan is the narrow-row plan for C SMs with every CTA busy and all batches of a warp resident at once
-        p = api.plan_query(m, n, sm_count=C, bf16=bf16)
+        # every entry point plans the problem on C CTAs, all of them busy, all batches of a warp resident at once
+        p = api.plan_query(m, n, bf16=bf16)
         assert p["variant"] == 0 and p["grid"] == C
+        assert api.cluster_ctas(m, n, sm_count=C, bf16=bf16) == C and api.cluster_ctas(m, n, sm_count=7, bf16=bf16) == 0
+        assert api.plan_query(m, n, sm_count=7, bf16=bf16)["grid"] == 7
         warps = p["threads"] // 32
         batches = -(-m // p["rows_per_batch"])
         per_warp = -(-(-(-batches // warps)) // C)

@@ -363,8 +363,8 @@ def test_single_launch_fit_equals_two_kernel_fit_all_shapes(ctx, m, n, bf16):
 
 
 # problems that fit the shared memory of one thread-block cluster run lr_fit there (partial sums pushed from CTA to CTA);
-# clusters of 16 and of 8, one to four batches per warp, ragged last batches, idle warps, and bfloat16 storage.  The bits are
-# those of the other forms with the rows divided among as many CTAs as the cluster has.
+# clusters of 16 and of 8, one to four batches per warp, ragged last batches, idle warps, and bfloat16 storage.  Every entry
+# point plans such a problem on as many CTAs as the cluster has, so all forms give the same bits.
 CLUSTER_CASES = [("cfg1", 10_000, False), ("cfg1", 4_100, False), ("cfg1", 7_777, False), ("cfg1", 24_000, False),
                  ("cfg3", 1_500, False), ("cfg3", 600, False), ("cfg5", 2_000, False), ("cfg5", 12_001, False),
                  ("higgs_like", 20_003, False), ("cfg2", 3_000, False),
@@ -382,13 +382,13 @@ def test_cluster_form_equals_the_other_forms(ctx, name, m, bf16):
         dX = dev(X)
     C = api.cluster_ctas(wl.m, wl.n, bf16=bf16)
     assert C in (8, 16), "every case here is meant to have a cluster plan"
+    assert api.plan_query(wl.m, wl.n, bf16=bf16)["grid"] == C
     dy, iters = dev(y), 9
     try:
         n0 = ctx.launch_count()
         w1, b1, h1 = api.lr_fit(dX, dy, wl.lr, iters, return_history=True, ctx=ctx)          # default: the cluster form
         assert ctx.launch_count() == n0 + 1
         ctx.set_cluster(False)
-        ctx.set_sm_limit(C)
         w2, b2, h2 = api.lr_fit(dX, dy, wl.lr, iters, return_history=True, ctx=ctx)          # grid-wide persistent kernel on C CTAs
         assert ctx.launch_count() == n0 + 2
         ctx.set_persistent(False)
@@ -396,7 +396,6 @@ def test_cluster_form_equals_the_other_forms(ctx, name, m, bf16):
         assert ctx.launch_count() == n0 + 2 + 2 * iters
     finally:
         ctx.set_cluster(True)
-        ctx.set_sm_limit(0)
         ctx.set_persistent(None)
     assert torch.equal(w1, w2) and torch.equal(b1, b2) and torch.equal(h1, h2)
     assert torch.equal(w1, w3) and torch.equal(b1, b3) and torch.equal(h1, h3)

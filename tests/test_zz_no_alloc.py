@@ -76,7 +76,8 @@ def test_two_calls_in_a_row_match_the_context_entry_point_and_the_checker():
         _run_pair(ctx, 70_003, 32, seed=903)        # 16-byte groups, 8 lanes per row
         _run_pair(ctx, 20_000, 30, seed=904)        # n % 4 != 0: the element-wise staged kernel
         _run_pair(ctx, 900, 1020, seed=905)         # 16-byte groups, eight warps per CTA
-        _run_pair(ctx, 800, 1022, seed=906)         # the largest n: element-wise staged kernel, eight warps per CTA
+        _run_pair(ctx, 800, 1022, seed=906)         # the largest n, not a whole number of 16-byte groups: CTA-wide stages
+        _run_pair(ctx, 2_001, 777, seed=909, shift=1)    # the same kernel on a matrix that is 4-byte aligned only
         _run_pair(ctx, 40_001, 449, seed=907, shift=1)   # X 4-byte aligned only: element-wise kernel, head and tail by plain loads
         _run_pair(ctx, 5_003, 64, seed=908, shift=3)
         assert ctx.device_status() == 0
