@@ -44,17 +44,17 @@ NOMINAL_HBM_GBS = 8000.0
 # bfloat16 storage.  Remove an entry when its kernel changes.
 KEPT_BYTES = 33_030_144                         # a quarter of the 126 MB L2, as lr_set_l2_keep's default for the persistent kernel
 NCU_TRAFFIC_BYTES_PER_ROW = {
-    "cfg2": {"k_stream_rows": (404.025344e6 + 3.488768e6) / 1_000_000,
-             "k_fit_rows": (1.111132e9 + 4.197632e6 + 2 * KEPT_BYTES) / 3 / 1_000_000},
-    "cfg5": {"k_stream_rows": (520.023552e6 + 3.864576e6) / 2_000_000,
-             "k_fit_rows": (1.446715e9 + 7.011840e6 + 2 * KEPT_BYTES) / 3 / 2_000_000},
-    "higgs_like": {"k_stream_rows": (464.036864e6 + 3.543040e6) / 4_000_000,
-                   "k_fit_rows": (1.269865e9 + 5.956608e6 + 2 * KEPT_BYTES) / 3 / 4_000_000},
-    "cfg3": {"k_stream_rows": (514.040064e6 + 3.598336e6) / 500_000,
-             "k_fit_rows": (1.439553e9 + 3.939840e6 + 2 * KEPT_BYTES) / 3 / 500_000},
+    "cfg2": {"k_stream_rows": (404.038400e6 + 5.690624e6) / 1_000_000,
+             "k_fit_rows": (1.111161e9 + 3.984640e6 + 2 * KEPT_BYTES) / 3 / 1_000_000},
+    "cfg5": {"k_stream_rows": (520.023296e6 + 4.371200e6) / 2_000_000,
+             "k_fit_rows": (1.445884e9 + 3.818496e6 + 2 * KEPT_BYTES) / 3 / 2_000_000},
+    "higgs_like": {"k_stream_rows": (464.071168e6 + 3.365120e6) / 4_000_000,
+                   "k_fit_rows": (1.272406e9 + 3.437568e6 + 2 * KEPT_BYTES) / 3 / 4_000_000},
+    "cfg3": {"k_stream_rows": (514.070528e6 + 3.252736e6) / 500_000,
+             "k_fit_rows": (1.438903e9 + 3.893760e6 + 2 * KEPT_BYTES) / 3 / 500_000},
     "cfg4": {"k_stream_split": (491.682048e6 + 3.577600e6) / 30_000},
-    "cfg3_bf16": {"k_stream_rows": (516.026624e6 + 3.481088e6) / 1_000_000,
-                  "k_fit_rows": (1.441246e9 + 4.163328e6 + 2 * KEPT_BYTES) / 3 / 1_000_000},
+    "cfg3_bf16": {"k_stream_rows": (516.026880e6 + 4.308992e6) / 1_000_000,
+                  "k_fit_rows": (1.441072e9 + 4.183552e6 + 2 * KEPT_BYTES) / 3 / 1_000_000},
     "cfg4_bf16": {"k_stream_split": (491.803904e6 + 5.702400e6) / 60_000},
 }
 
