@@ -129,7 +129,8 @@ int lr_set_persistent(lr_ctx* ctx, int32_t on);
  * touches global memory (10,000 x 32: 3 us per iteration where the grid-wide persistent kernel takes 4.3).
  * Taken by default where it applies, unless lr_set_persistent has asked for a particular form.  lr_set_cluster(ctx, 0)
  * switches the form off (the persistent kernel then runs on the same plan), any other value restores the default.
- * lr_fit_tol and lr_fit_sharded do not use it.  A wait that expires ends the kernel as it ends the persistent one.
+ * lr_fit_tol uses it too (the stopping rule is evaluated by every CTA of the cluster, same bits as the persistent kernel);
+ * lr_fit_sharded does not.  A wait that expires ends the kernel as it ends the persistent one.
  * lr_cluster_ctas (host only, no CUDA call; arguments as lr_plan_query) returns the cluster size the form would use
  * for a shape, 0 if none; whether a cluster of that size can be resident is known at launch only (if not, the
  * persistent kernel runs).

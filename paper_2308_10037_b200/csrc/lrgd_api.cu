@@ -592,12 +592,17 @@ int cluster_plan(const lr_plan& P, bool bf16, int64_t m, int32_t n, FitLayout* L
 // k_fit_cluster).  Returns cudaErrorNotSupported when the problem or the device does not allow it (the caller then takes
 // the grid-wide persistent kernel, which gives the same bits on the same plan).
 cudaError_t launch_cluster_fit(lr_ctx* ctx, const lr_plan& P, bool bf16, const void* d_X, const float* d_y, int64_t m, int32_t n,
-                               float lr, int32_t iters, float* d_w, float* d_b, float* d_loss_hist, cudaStream_t st) {
+                               float lr, int32_t iters, float* d_w, float* d_b, float* d_loss_hist, const PersistentTol* tol,
+                               cudaStream_t st) {
     if (ctx->cluster_mode == 0 || ctx->persistent_mode != -1) return cudaErrorNotSupported;
     FitLayout L;
     int smem = 0;
     const int C = cluster_plan(P, bf16, m, n, &L, &smem);
     if (C == 0) return cudaErrorNotSupported;
+    if (cudaMemsetAsync(ctx->d_gbar, 0, 2 * sizeof(unsigned int), st) != cudaSuccess) {   // [1]: the launch's abort word
+        cudaGetLastError();
+        return cudaErrorNotSupported;
+    }
     const cudaError_t e = for_row_shape(P, bf16, [&](auto shape) {
         using S = decltype(shape);
         if constexpr (S::Elem::EPG > 1) {
@@ -626,6 +631,8 @@ cudaError_t launch_cluster_fit(lr_ctx* ctx, const lr_plan& P, bool bf16, const v
             cp.status = ctx->d_status; cp.depth = L.depth;
             cp.num_batches = (m + P.rows_per_batch - 1) / P.rows_per_batch;
             cp.iters = iters; cp.lr = double(lr); cp.inv_m = 1.0 / double(m);
+            cp.abort_word = ctx->d_gbar + 1;
+            if (tol) { cp.tol = tol->state; cp.eps = tol->eps; cp.gnorm_hist = tol->gnorm_hist; }
             return cudaLaunchKernelEx(&cfg, kern, cp);
         } else {
             return cudaErrorNotSupported;
@@ -955,7 +962,7 @@ int fit_impl(lr_ctx* ctx, const void* d_X, bool bf16, const float* d_y, int64_t 
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     // Narrow rows, several iterations: one cooperative launch runs the whole fit (same bits as the loop below).
     if (iters >= 2 && want_persistent(ctx, P, bf16, m, n, iters)) {
-        if (launch_cluster_fit(ctx, P, bf16, d_X, d_y, m, n, lr, iters, d_w, d_b, d_loss_hist, st) == cudaSuccess) return LR_OK;
+        if (launch_cluster_fit(ctx, P, bf16, d_X, d_y, m, n, lr, iters, d_w, d_b, d_loss_hist, nullptr, st) == cudaSuccess) return LR_OK;
         const cudaError_t le = launch_persistent_fit(ctx, P, bf16, d_X, d_y, m, n, lr, iters, d_w, d_b, d_loss_hist, nullptr, st);
         if (le == cudaSuccess) return LR_OK;
         if (le != cudaErrorCooperativeLaunchTooLarge) { ctx->last_cuda = int(le); return LR_ERR_CUDA; }
@@ -1058,7 +1065,9 @@ int fit_tol_impl(lr_ctx* ctx, const void* d_X, bool bf16, const float* d_y, int6
     // Narrow rows: one persistent launch that leaves its loop on the device as soon as the norm is small enough.
     if (want_persistent(ctx, P, bf16, m, n, max_iters)) {
         const PersistentTol pt{ctx->d_tol, double(eps), d_gnorm_hist};
-        const cudaError_t le = launch_persistent_fit(ctx, P, bf16, d_X, d_y, m, n, lr, max_iters, d_w, d_b, d_loss_hist, &pt, st);
+        // (a problem that fits one thread-block cluster runs there; otherwise, or if the device refuses, the grid-wide kernel)
+        cudaError_t le = launch_cluster_fit(ctx, P, bf16, d_X, d_y, m, n, lr, max_iters, d_w, d_b, d_loss_hist, &pt, st);
+        if (le != cudaSuccess) le = launch_persistent_fit(ctx, P, bf16, d_X, d_y, m, n, lr, max_iters, d_w, d_b, d_loss_hist, &pt, st);
         if (le == cudaSuccess) {
             LR_CK(ctx, cudaMemcpyAsync(ctx->h_tol, ctx->d_tol, sizeof(TolState), cudaMemcpyDeviceToHost, st));
             LR_CK(ctx, cudaMemcpyAsync(&ctx->h_words[2], ctx->d_gbar + 1, sizeof(int), cudaMemcpyDeviceToHost, st));

@@ -18,8 +18,11 @@
 //
 // Every wait is bounded.  A CTA whose wait expires raises the status word and stops sending; the others then run into
 // their own bound.  Nobody leaves before all CTAs have stopped sending (the cluster barrier at the end, which every CTA
-// reaches because nothing before it waits without a bound).  Fixed iteration counts only (the stopping rule and row shards stay
-// with k_fit_rows).
+// reaches because nothing before it waits without a bound).
+//
+// With a tolerance (lr_fit_tol) every CTA also forms ||grad||_2 of the update just applied, in k_fit_rows' order, so all CTAs
+// get the same bits and leave the loop in the same iteration once it is <= eps (Algorithm 7's stopping rule).  Row shards
+// stay with k_fit_rows.
 #pragma once
 #include <cooperative_groups.h>
 
@@ -46,12 +49,18 @@ struct ClusterFitParams {
     int iters;
     double lr;
     double inv_m;
+    unsigned int* abort_word;  // raised (1) if a bounded wait expired anywhere in the cluster; zero at launch
+    // stopping rule (all null / zero for a fixed-count fit): as in k_fit_rows
+    TolState* tol;
+    double eps;
+    float* gnorm_hist;         // nullable [iters]
 };
 
 // shared memory of a CTA: header and stages as k_fit_rows lays them out, its tail (combine buffer, parameters, this CTA's
-// partial row), then the received rows [2][C][n+2] and the two mbarriers they complete
+// partial row), then the received rows [2][C][n+2], the two mbarriers they complete and the gradient entries [n+2] of the
+// stopping rule
 __host__ __device__ constexpr int cluster_fit_smem(int n, int nw, int depth, int stage_stride, int C) {
-    return kHeaderBytes + nw * depth * stage_stride + fit_tail_bytes(n) + 2 * C * (n + 2) * 8 + 16;
+    return kHeaderBytes + nw * depth * stage_stride + fit_tail_bytes(n) + 2 * C * (n + 2) * 8 + 16 + (n + 2) * 8;
 }
 
 // address of the same shared-memory location in CTA `rank` of the cluster
@@ -102,6 +111,7 @@ __global__ void __launch_bounds__(NW * 32, 1) k_fit_cluster(const __grid_constan
     double* my_row = reinterpret_cast<double*>(tail + kFitRedBytes + fit_param_bytes(n));   // [n+2]: this CTA's partial row
     double* slots = reinterpret_cast<double*>(tail + fit_tail_bytes(n));                     // [2][C][n+2]: everybody's rows
     uint64_t* xbar = reinterpret_cast<uint64_t*>(slots + 2 * static_cast<size_t>(C) * stride);   // [2]
+    double* grad_s = reinterpret_cast<double*>(xbar + 2);                                         // [n+2], tolerance mode only
     uint64_t* my_bars = bars + warp * kMaxDepth;
 
     const long long B = p.num_batches;
@@ -292,14 +302,41 @@ __global__ void __launch_bounds__(NW * 32, 1) k_fit_cluster(const __grid_constan
             const double* rows_in = slots + static_cast<size_t>(set) * C * stride;
             for (int c = threadIdx.x; c < stride; c += NW * 32) {
                 const double v = single_row_slices_sum<NW>(C, [&](int g) { return rows_in[static_cast<size_t>(g) * stride + c]; }) * p.inv_m;
-                if (c <= n) w_s[c] = static_cast<float>(static_cast<double>(w_s[c]) - p.lr * v);
-                else if (cta == 0 && p.loss_hist) p.loss_hist[t] = static_cast<float>(v);
+                if (c <= n) {
+                    w_s[c] = static_cast<float>(static_cast<double>(w_s[c]) - p.lr * v);
+                    if (p.tol != nullptr) grad_s[c] = v;               // gradient entry, for the norm below
+                } else if (cta == 0 && p.loss_hist) {
+                    p.loss_hist[t] = static_cast<float>(v);
+                }
             }
         }
         alive = __syncthreads_and(ok) != 0;
+
+        // ---- stopping rule (Algorithm 7): ||(grad_w, grad_b)||_2 of the update just applied, formed by every warp in the
+        // order of k_fit_rows and k_reduce_update (lane-strided squares, xor tree): the same bits in every CTA ----
+        if (p.tol != nullptr && alive) {
+            double q = 0.0;
+            for (int c = lane; c <= n; c += 32) {
+                const double v = grad_s[c];
+                q += v * v;
+            }
+#pragma unroll
+            for (int msk = 16; msk >= 1; msk >>= 1) q += __shfl_xor_sync(FULL, q, msk);
+            const double nrm = sqrt(q);
+            if (cta == 0 && threadIdx.x == 0) {
+                p.tol->grad_norm = nrm;
+                p.tol->iters_done = t + 1;
+                if (p.gnorm_hist) p.gnorm_hist[t] = static_cast<float>(nrm);
+                if (nrm <= p.eps) p.tol->stop = 1;
+            }
+            if (nrm <= p.eps) break;               // uniform over the whole cluster
+        }
     }
 
-    if (!alive && threadIdx.x == 0) atomicExch(p.status, kStatusTimeout);
+    if (!alive && threadIdx.x == 0) {
+        atomicExch(p.status, kStatusTimeout);
+        atomicExch(p.abort_word, 1u);
+    }
     // nobody may leave while another CTA could still send to it; the outcome of every CTA is looked at together
     int* flag_s = reinterpret_cast<int*>(red);
     if (threadIdx.x == 0) *flag_s = alive ? 0 : 1;

@@ -43,7 +43,9 @@ def run_gpu(ctx, dX, dy, n, lr, eps, max_iters, check_every=16):
 # cfg4's own recipe (uncentred features, lr 0.05) makes GD oscillate, so its gradient norm never settles below a
 # threshold; the wide-row kernels are exercised with the cfg3 recipe widened to 2048 and 4096 columns instead
 CASES = [("cfg1", 10_000, 60, None), ("cfg3", 40_003, 40, None), ("cfg5", 120_001, 40, None), ("cfg3", 6_001, 40, 2048),
-         ("cfg3", 5_003, 30, 4096), ("cfg2", 20_000, 40, 30), ("higgs_like", 90_007, 60, None)]
+         ("cfg3", 5_003, 30, 4096), ("cfg2", 20_000, 40, 30), ("higgs_like", 90_007, 60, None),
+         # problems that fit one thread-block cluster (the library's own choice of form then differs from the forced ones)
+         ("cfg5", 12_001, 40, None), ("cfg3", 1_500, 40, None), ("cfg1", 4_100, 60, None)]
 
 
 @pytest.mark.parametrize("name,m,max_iters,n", CASES)
@@ -75,6 +77,15 @@ def test_stops_at_the_same_iteration_as_the_checker(ctx, name, m, max_iters, n):
     assert np.max(np.abs(lh[:k] - lh_ref)) <= LOSS_TOL
     assert np.max(np.abs(gh[:k] - gh_ref) / gh_ref) <= 10 * GRAD_TOL       # free-running iterates: parameters differ by <= W_TOL
     assert np.isnan(lh[k:]).all() and np.isnan(gh[k:]).all()               # nothing is written after the stop
+
+    # the library's own choice of form (one thread-block cluster where the problem fits one): the same bits, one launch
+    n0 = ctx.launch_count()
+    w1, b1, k1, nrm1, lh1, gh1 = run_gpu(ctx, dX, dy, wl.n, wl.lr, eps, max_iters)
+    if api.plan_query(wl.m, wl.n)["variant"] == 0:
+        assert ctx.launch_count() == n0 + 1
+    assert k1 == k and nrm1 == nrm and torch.equal(w1, w) and torch.equal(b1, b)
+    assert np.array_equal(gh1[:k], gh[:k]) and np.isnan(gh1[k:]).all()
+    assert np.array_equal(lh1[:k], lh[:k]) and np.isnan(lh1[k:]).all()
 
     # narrow rows stop inside one persistent launch; the two-kernel form (a device flag turns later launches into no-ops)
     # must give the same bits, however often the host looks at the flag
