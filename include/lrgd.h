@@ -53,7 +53,8 @@ typedef struct lr_plan {
     int32_t variant;       /* 0 = row-per-lane-group staged kernel, 1 = row-split staged kernel, 2 = unstaged generic kernel,
                               3 = row-per-lane-group staged kernel for rows of any length up to 512 in a matrix aligned to its
                               element size only (a lane owns single elements: vec_per_lane counts elements, not 16-byte groups),
-                              4 = row-split kernel with CTA-wide stages for such rows of 513..8192 elements */
+                              4 = row-split kernel with CTA-wide stages for such rows of 513..8192 elements and for every row of
+                              8193..16384 elements */
     int32_t lanes_per_row; /* staged kernels: lanes that share one row (8, 16, 32; all threads of the CTA for the row-split kernel) */
     int32_t vec_per_lane;  /* staged kernels: 16-byte column groups owned by one lane */
     int32_t rows_per_batch;/* rows one warp (or one CTA for the row-split kernel) holds in registers at a time */
@@ -88,9 +89,9 @@ int lr_destroy(lr_ctx* ctx);
  *   d_loss[0] = loss, d_grad_w[0..n) = X^T err / m, d_grad_b[0] = sum err / m.
  * Inputs d_X [m*n], d_y [m], d_w [n], d_b [1] are read only.  Two kernels are enqueued: the fused
  * streaming kernel (reads X once) and the fixed-order cross-CTA reduction.
- * Which streaming kernel runs depends on the shape (lr_plan_query tells): rows of up to 8192 columns always take a staged
- * kernel (at HBM speed with d_X 16-byte aligned and n % 4 == 0, at a half to nine tenths of it for other lengths and for
- * matrices that are only 4-byte aligned); wider rows run on a slower unstaged kernel.
+ * Which streaming kernel runs depends on the shape (lr_plan_query tells): rows of up to 16384 columns always take a staged
+ * kernel (at HBM speed with d_X 16-byte aligned, n % 4 == 0 and n <= 8192; at a half to nine tenths of it for other lengths, for
+ * matrices that are only 4-byte aligned and for rows beyond 8192 columns); wider rows run on a slower unstaged kernel.
  */
 int lr_loss_grad(lr_ctx* ctx, const float* d_X, const float* d_y, int64_t m, int32_t n,
                  const float* d_w, const float* d_b,
@@ -225,7 +226,7 @@ int lr_predict(lr_ctx* ctx, const float* d_X, int64_t m, int32_t n,
  * with leading dimension n, 2-byte aligned.  Only X changes: y, w, b, the gradient and every sum stay as in the fp32
  * calls, each element of X is widened exactly to fp32 when it is used, so the three calls below compute exactly what
  * lr_loss_grad / lr_fit / lr_predict would compute on the fp32 matrix holding the same (bfloat16-representable) values.
- * Rows of up to 8192 columns always take a staged kernel (fastest with n % 8 == 0 and d_Xh 16-byte aligned); wider rows
+ * Rows of up to 16384 columns always take a staged kernel (fastest with n % 8 == 0, d_Xh 16-byte aligned and n <= 8192); wider rows
  * run on the unstaged kernel.  lr_fit_bf16 takes the persistent kernel of lr_fit for rows of up to 512 columns with n % 8 == 0 and
  * d_Xh 16-byte aligned.  Errors as the fp32 calls.
  *

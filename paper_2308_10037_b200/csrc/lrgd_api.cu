@@ -36,7 +36,7 @@ constexpr int kMaxGridPerSm = 8;               // widest launch any variant uses
 constexpr int kMaxProfiled = 4096;
 constexpr int kMaxDynamicSmem = 232448;         // opt-in dynamic shared memory per CTA on sm_100
 constexpr int64_t kMaxRows = int64_t(1) << 40;
-constexpr int kWideAnyMaxCols = 8192;           // widest row of the CTA-wide staged kernel for rows of any length
+constexpr int kWideAnyMaxCols = 16384;          // widest row of the CTA-wide staged kernel for rows of any length
 
 struct RowShape { int nv, lpr, rb; int nw = kNW; };    // nw = warps per CTA
 
@@ -175,9 +175,11 @@ int make_plan(int64_t m, int32_t n, bool aligned16, int32_t sms, lr_plan* P, boo
         // elements per lane and row: the smallest of 2, 3, 4, 6, 8, 12, 16 that covers the slice (a lane's slots beyond the
         // slice are dead work, so the steps are kept fine); rows per batch: as many as the registers hold (32 or 48 elements
         // of a batch per lane), because all warps meet once per batch
-        static const int kNv[7] = {2, 3, 4, 6, 8, 12, 16}, kRb[7] = {16, 16, 8, 8, 4, 4, 2};
+        // (rows beyond 8192 elements: one row per batch, 24 or 32 elements of it per lane; aligned rows of that width
+        // land here too, since the row-split kernel's tensor-map boxes end at 8192 columns)
+        static const int kNv[9] = {2, 3, 4, 6, 8, 12, 16, 24, 32}, kRb[9] = {16, 16, 8, 8, 4, 4, 2, 1, 1};
         int pick = 0;
-        while (pick < 6 && kNv[pick] * 32 < cw) ++pick;
+        while (pick < 8 && kNv[pick] * 32 < cw) ++pick;
         const int nv = kNv[pick], rb = nw == 8 ? 16 : kRb[pick];
         const int64_t B = (m + rb - 1) / rb;
         const int grid = int(std::min<int64_t>(B, sms));
@@ -464,9 +466,11 @@ cudaError_t launch_wide(const lr_plan& P, const WideParams& wp, cudaStream_t st,
     if (bf16) {
         LRGD_WIDE(ElemBF16Any, 2, 16) LRGD_WIDE(ElemBF16Any, 3, 16) LRGD_WIDE(ElemBF16Any, 4, 8) LRGD_WIDE(ElemBF16Any, 6, 8)
         LRGD_WIDE(ElemBF16Any, 8, 4) LRGD_WIDE(ElemBF16Any, 12, 4) LRGD_WIDE(ElemBF16Any, 16, 2)
+        LRGD_WIDE(ElemBF16Any, 24, 1) LRGD_WIDE(ElemBF16Any, 32, 1)
     } else {
         LRGD_WIDE(ElemF32Any, 2, 16) LRGD_WIDE(ElemF32Any, 3, 16) LRGD_WIDE(ElemF32Any, 4, 8) LRGD_WIDE(ElemF32Any, 6, 8)
         LRGD_WIDE(ElemF32Any, 8, 4) LRGD_WIDE(ElemF32Any, 12, 4) LRGD_WIDE(ElemF32Any, 16, 2)
+        LRGD_WIDE(ElemF32Any, 24, 1) LRGD_WIDE(ElemF32Any, 32, 1)
     }
 #undef LRGD_WIDE
     return cudaErrorInvalidValue;

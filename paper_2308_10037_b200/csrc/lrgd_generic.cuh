@@ -1,6 +1,5 @@
-// Unstaged kernel for shapes the staged kernels do not take (a row that is not a whole number of 16-byte
-// groups, X not 16-byte aligned, or rows wider than the staged kernels cover).  E is the storage type of X.  Plain coalesced loads; X is read from HBM
-// once and a second time through the cache hierarchy.
+// Unstaged kernel for the rows the staged kernels do not take: more than 16384 elements.  E is the storage type of X.
+// Plain coalesced loads; X is read from HBM once and a second time through the cache hierarchy.
 //
 // A CTA walks chunks of kGenRows rows (chunk c belongs to CTA c mod grid).  Phase 1: one warp per row
 // forms z = x.w + b (model equation, Section II-A), then err and the loss term (Eq. 1, Algorithm 7,

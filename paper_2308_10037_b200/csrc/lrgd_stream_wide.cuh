@@ -1,5 +1,6 @@
 // Fused single-pass streaming kernel for wide rows of ANY length in a matrix aligned only to its element size
-// (fp32: 513 <= n <= 8192 with n % 4 != 0 or X not 16-byte aligned; bfloat16 likewise with n % 8 / 2-byte alignment).
+// (fp32: 513 <= n <= 8192 with n % 4 != 0 or X not 16-byte aligned; bfloat16 likewise with n % 8 / 2-byte alignment),
+// and for every row of 8193..16384 elements (one row per batch).
 // E is ElemF32Any or ElemBF16Any: the unit a lane owns is a single element.
 //
 // Such rows cannot be cut into aligned 16-byte groups, so neither a tensor map nor per-warp boxes can describe a
@@ -51,9 +52,14 @@ __global__ void __launch_bounds__(NW * 32, 1) k_stream_wide(const WideParams p) 
     constexpr int LOG_RB = Log2<RB>::value;
     constexpr int SHIFT = 5 - LOG_RB;              // log2 of the lanes holding the same row after the reduction
     constexpr int DUP = 1 << SHIFT;
-    constexpr int PER_DUP = NW / DUP;              // partial logits each of those lanes adds up
+    constexpr int PER_DUP = NW >= DUP ? NW / DUP : 1;   // partial logits each of those lanes adds up (with one row per batch
+                                                        // there are more such lanes than warps: the first NW take one each)
     constexpr unsigned FULL = 0xffffffffu;
-    static_assert(NW % DUP == 0, "warps must split evenly over the duplicate lanes");
+    // Slices of more than 16 elements per lane (rows beyond 8192 elements, one row per batch) leave no registers for fp64
+    // copies of the accumulators: the fp32 sums are then added straight into the CTA's own fp64 partial row in global memory
+    // (each column belongs to one lane, so the read-modify-write needs no ordering), once per 64 rows.
+    constexpr bool FLUSH_GLOBAL = NV > 16;
+    static_assert(NW % DUP == 0 || DUP % NW == 0, "warps must split evenly over the duplicate lanes");
     static_assert(kMaxDepth * 8 + 16 <= kSplitZOffset, "header too small");
     static_assert(kSplitZOffset + 2 * NW * RB * 4 <= kSplitHeaderBytes, "header too small");
 
@@ -109,12 +115,23 @@ __global__ void __launch_bounds__(NW * 32, 1) k_stream_wide(const WideParams p) 
     };
 
     typename E::template Lane<NV> lm;              // this lane's elements of w (c0 + lane + 32k) and its fp32 accumulators
-    double dacc[NV][1];
+    double dacc[FLUSH_GLOBAL ? 1 : NV][1];
     float se = 0.f, sl = 0.f;
     double dse = 0.0, dsl = 0.0;
     lm.zero();
 #pragma unroll
-    for (int k = 0; k < NV; ++k) dacc[k][0] = 0.0;
+    for (int k = 0; k < (FLUSH_GLOBAL ? 1 : NV); ++k) dacc[k][0] = 0.0;
+    double* const out_row = PREDICT ? nullptr : p.partial + static_cast<size_t>(blockIdx.x) * (n + 2);
+    // adds this lane's fp32 sums to its columns of the CTA's partial row and clears them
+    auto flush_global = [&]() {
+#pragma unroll
+        for (int k = 0; k < NV; ++k) {
+            const int loc = lane + 32 * k;
+            if (loc < mycw) out_row[c0 + loc] += static_cast<double>(lm.acc[k]);
+            lm.acc[k] = 0.f;
+        }
+        dse += se; dsl += sl; se = 0.f; sl = 0.f;
+    };
     const int myr = (lane >> SHIFT) & (RB - 1);    // the row of a batch whose logit ends up on this lane
     const int dup = lane & (DUP - 1);              // which of the lanes sharing that row this one is
     const bool owner = dup == 0;
@@ -145,6 +162,14 @@ __global__ void __launch_bounds__(NW * 32, 1) k_stream_wide(const WideParams p) 
     }
     lm.template load_w<WSource::GlobalL2>(p.w, c0 + lane, 32, c0 + mycw);    // through L2: the kernel before this one may just have written them
     const float bval = __ldcg(p.b);
+    if constexpr (FLUSH_GLOBAL && !PREDICT) {
+        // the row is accumulated into: start it at zero (only this lane ever touches these columns of it)
+#pragma unroll
+        for (int k = 0; k < NV; ++k) {
+            const int loc = lane + 32 * k;
+            if (loc < mycw) out_row[c0 + loc] = 0.0;
+        }
+    }
 
     for (int i = 0; i < cnt; ++i) {
         const bool myvalid = row0 + myr < p.m;
@@ -204,7 +229,8 @@ __global__ void __launch_bounds__(NW * 32, 1) k_stream_wide(const WideParams p) 
         // the lanes that share a row add PER_DUP partials each (warp order), then a butterfly: one fixed order, same in every warp
         float zs = 0.f;
 #pragma unroll
-        for (int j = 0; j < PER_DUP; ++j) zs += zp[(dup * PER_DUP + j) * RB + myr];
+        for (int j = 0; j < PER_DUP; ++j)
+            if (NW >= DUP || dup < NW) zs += zp[(dup * PER_DUP + j) * RB + myr];
 #pragma unroll
         for (int msk = DUP / 2; msk >= 1; msk >>= 1) zs += __shfl_xor_sync(FULL, zs, msk);
         const float z = zs + bval;
@@ -234,9 +260,16 @@ __global__ void __launch_bounds__(NW * 32, 1) k_stream_wide(const WideParams p) 
             }
             if (!myvalid) e = 0.f;
             batch_accumulate<E, NV, 32, RB>(x, e, lm);
-            if (++since_flush == 2 * kFlushBatches) {
-                since_flush = 0;
-                fold_into_fp64<E, NV>(lm, dacc, se, sl, dse, dsl);
+            if constexpr (FLUSH_GLOBAL) {
+                if (++since_flush == 64 / RB) {
+                    since_flush = 0;
+                    flush_global();
+                }
+            } else {
+                if (++since_flush == 2 * kFlushBatches) {
+                    since_flush = 0;
+                    fold_into_fp64<E, NV>(lm, dacc, se, sl, dse, dsl);
+                }
             }
         }
         row0 += stride_rows;
@@ -252,12 +285,16 @@ __global__ void __launch_bounds__(NW * 32, 1) k_stream_wide(const WideParams p) 
         __syncthreads();
     }
     if constexpr (!PREDICT) {
-        double* out = p.partial + static_cast<size_t>(blockIdx.x) * (n + 2);
-        fold_into_fp64<E, NV>(lm, dacc, se, sl, dse, dsl);
+        double* out = out_row;
+        if constexpr (FLUSH_GLOBAL) {
+            flush_global();
+        } else {
+            fold_into_fp64<E, NV>(lm, dacc, se, sl, dse, dsl);
 #pragma unroll
-        for (int k = 0; k < NV; ++k) {
-            const int loc = lane + 32 * k;
-            if (loc < mycw) out[c0 + loc] = dacc[k][0];
+            for (int k = 0; k < NV; ++k) {
+                const int loc = lane + 32 * k;
+                if (loc < mycw) out[c0 + loc] = dacc[k][0];
+            }
         }
         if (warp == 0) {
 #pragma unroll

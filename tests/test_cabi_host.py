@@ -73,7 +73,7 @@ def test_plan_staged_shapes(m, n, lpr, nv, nw):
 
 def test_plan_for_unaligned_or_odd_shapes():
     # rows of any length in a matrix aligned to its element size: per-warp stages up to 512 columns (variant 3), CTA-wide
-    # stages of whole rows up to 8192 (variant 4); only wider rows run unstaged (variant 2)
+    # stages of whole rows up to 16384 (variant 4); only wider rows run unstaged (variant 2)
     assert api.plan_query(1000, 1027)["variant"] == 4        # n not a multiple of 4 and wider than 1024
     assert api.plan_query(1000, 1028, x_aligned16=False)["variant"] == 4   # the row-split kernel needs a 16-byte aligned matrix
     assert api.plan_query(1000, 515)["variant"] == 4 and api.plan_query(1000, 516, x_aligned16=False)["variant"] == 4
@@ -82,11 +82,17 @@ def test_plan_for_unaligned_or_odd_shapes():
     assert api.plan_query(1000, 30, x_aligned16=False)["variant"] == 3
     assert api.plan_query(1000, 32, x_aligned16=False, bf16=True)["variant"] == 3
     assert api.plan_query(1000, 8191)["variant"] == 4 and api.plan_query(1000, 8192, x_aligned16=False)["variant"] == 4
-    assert api.plan_query(1000, 8196)["variant"] == 2         # wider than any staged kernel
-    assert api.plan_query(1000, 8200, bf16=True)["variant"] == 2
+    # beyond the row-split kernel's 8192 columns every row, aligned or not, takes the CTA-wide stages: one row per batch
+    for n, nv in ((8193, 24), (8196, 24), (12288, 24), (12289, 32), (16384, 32)):
+        for bf16 in (False, True):
+            q = api.plan_query(1000, n, bf16=bf16)
+            assert (q["variant"], q["vec_per_lane"], q["rows_per_batch"], q["threads"]) == (4, nv, 1, 512)
+            assert q["stages"] >= (3 if not bf16 else 4)
+    assert api.plan_query(1000, 16385)["variant"] == 2        # wider than any staged kernel
+    assert api.plan_query(1000, 16392, bf16=True)["variant"] == 2
     assert api.plan_query(1000, 30, bf16=True)["variant"] == 3   # element-wise staged kernel, bfloat16 too
     assert api.plan_query(1000, 1036, bf16=True)["variant"] == 4 # 1036 % 8 != 0 and wider than 1024
-    g = api.plan_query(100, 8197)
+    g = api.plan_query(100, 16389)
     assert g["variant"] == 2 and g["grid"] == 2 and g["threads"] == 256
     w = api.plan_query(100_000, 1027)
     assert w["vec_per_lane"] == 3 and w["rows_per_batch"] == 16 and w["stages"] == 3 and w["threads"] == 512
@@ -207,7 +213,7 @@ def test_any_length_copies_stay_inside_the_matrix():
     import random
     rnd = random.Random(1)
     shapes = [(2758, 449), (1, 1), (7, 3), (300, 1), (640, 30), (1025, 101), (526, 255), (999, 511), (5, 510), (3, 258),
-              (17, 257), (2, 449), (1, 511)]
+              (17, 257), (2, 449), (1, 511), (40, 8193), (33, 12291), (19, 16383), (7, 16384)]
     shapes += [(rnd.randint(1, 3000), rnd.choice([n for n in range(1, 513) if n % 4])) for _ in range(200)]
     shapes += [(3, 513), (1, 1023), (77, 1021), (500, 777), (2, 1022), (9, 8191), (33, 4099), (5, 2049), (64, 1025)]
     shapes += [(rnd.randint(1, 400), rnd.choice([n for n in range(513, 8192) if n % 4])) for _ in range(60)]
@@ -250,12 +256,12 @@ def test_any_length_copies_stay_inside_the_matrix():
 
 
 def test_every_row_length_gets_a_launchable_plan():
-    """Sweeps n = 1 .. 8300 for both storage types and both alignments: the plan always names a kernel shape that exists,
+    """Sweeps n = 1 .. 16500 for both storage types and both alignments: the plan always names a kernel shape that exists,
     fits the shared memory of a CTA, keeps at least one stage, and (staged kernels) sizes its stages as the kernels do."""
     for bf16 in (False, True):
         eb, epg = (2, 8) if bf16 else (4, 4)
         for aligned in (True, False):
-            for n in list(range(1, 1100)) + list(range(1100, 8301, 4)) + [4097, 8191, 8193]:
+            for n in list(range(1, 1100)) + list(range(1100, 8301, 4)) + list(range(8301, 16500, 52)) + [4097, 8191, 8193, 12288, 12289, 16383, 16384, 16385, 16388]:
                 p = api.plan_query(70_001, n, x_aligned16=aligned, bf16=bf16)
                 v = p["variant"]
                 assert p["smem_bytes"] <= 227 * 1024 and p["grid"] >= 1 and p["threads"] in (256, 512)
@@ -277,12 +283,13 @@ def test_every_row_length_gets_a_launchable_plan():
                 elif v == 4:
                     # wide rows of any length: CTA-wide stages of whole rows; eight warps up to 1024 elements, sixteen beyond
                     nw = p["threads"] // 32
-                    assert 512 < n <= 8192 and nw == (8 if n <= 1024 else 16)
+                    assert 512 < n <= 16384 and nw == (8 if n <= 1024 else 16)
                     # rows of any length or alignment, and the aligned fp32 rows of 4100..6144 columns the row-split kernel is weak on
-                    assert not (aligned and n % epg == 0) or (not bf16 and 4096 < n <= 6144)
+                    assert not (aligned and n % epg == 0) or (not bf16 and 4096 < n <= 6144) or n > 8192
                     cw = -(-n // nw)
-                    assert p["vec_per_lane"] in (2, 3, 4, 6, 8, 12, 16) and p["vec_per_lane"] * 32 >= cw
-                    assert p["vec_per_lane"] * p["rows_per_batch"] in (32, 48, 64) and p["rows_per_batch"] in (2, 4, 8, 16)
+                    assert p["vec_per_lane"] in (2, 3, 4, 6, 8, 12, 16, 24, 32) and p["vec_per_lane"] * 32 >= cw
+                    assert p["vec_per_lane"] * p["rows_per_batch"] in (24, 32, 48, 64) and p["rows_per_batch"] in (1, 2, 4, 8, 16)
+                    assert (p["rows_per_batch"] == 1) == (n > 8192)
                     assert 2 * nw * p["rows_per_batch"] * 4 <= 4096 - 1024                   # the logit exchange fits the header
                     stage = -(-(p["rows_per_batch"] * n * eb + 16) // 128) * 128
                     assert 1 <= p["stages"] <= 4 and p["smem_bytes"] == 4096 + p["stages"] * stage
@@ -297,5 +304,4 @@ def test_every_row_length_gets_a_launchable_plan():
                     stage = -(-p["rows_per_batch"] * cw * 16 // 128) * 128
                     assert 1 <= p["stages"] <= 4 and p["smem_bytes"] == 4096 + nw * p["stages"] * stage
                 else:
-                    assert v == 2 and p["threads"] == 256 and n > 8192
-                    assert n > 1024 and (not aligned or n % epg != 0 or n > 8192)
+                    assert v == 2 and p["threads"] == 256 and n > 16384

@@ -21,7 +21,7 @@ from _parity import GRAD_TOL, LABEL_AGREE, LOSS_TOL, W_TOL, assert_grad_close, g
 def ctx():
     from paper_2308_10037_b200 import build
     build.build()
-    c = api.Context(n_max=8200, device=0)
+    c = api.Context(n_max=16400, device=0)
     yield c
     assert c.device_status() == 0
     c.close()
@@ -68,9 +68,9 @@ def check_loss_grad(ctx, Xv, dXh, y, w, b, loss_tol=LOSS_TOL):
 
 
 # every staged instantiation for 8-column groups (n/8 <= 8, 16, 32, 64), partly filled lane groups, the wide-row kernel
-# (n/8 > 64: full and partly idle warp slices), the unstaged kernel (n % 8 != 0, n > 8192), tiny / ragged / many-tile rows
+# (n/8 > 64: full and partly idle warp slices), rows beyond 8192 columns (CTA-wide stages, one row per batch), the unstaged kernel (n > 16384), tiny / ragged / many-tile rows
 SHAPES = [(1, 8), (7, 8), (9, 5), (33, 56), (1000, 64), (4097, 64), (5003, 128), (2500, 72), (3001, 100), (9999, 256),
-          (777, 200), (1500, 512), (2049, 264), (640, 30), (300, 1), (50, 8200), (20011, 16), (1025, 36),
+          (777, 200), (1500, 512), (2049, 264), (640, 30), (300, 1), (50, 8200), (301, 8193), (97, 16384), (20, 16392), (20011, 16), (1025, 36),
           (200_003, 256), (400_001, 64), (200_002, 128), (150_001, 24), (60_001, 512), (90_001, 200), (120_007, 104),
           (5_001, 4096), (20_003, 1024), (2_500, 520), (1_203, 2056), (701, 4088), (9_000, 2048), (3, 8192), (130, 8192),
           (1_001, 6000)]
@@ -84,7 +84,7 @@ def test_loss_grad_matches_oracle(ctx, m, n):
 
 
 # both sides of every boundary between the bfloat16 kernel shapes
-@pytest.mark.parametrize("n", [8, 16, 64, 72, 128, 136, 256, 264, 512, 520, 1024, 1032, 2048, 2056, 4096, 4104, 8192, 8200, 9, 65,
+@pytest.mark.parametrize("n", [8, 16, 64, 72, 128, 136, 256, 264, 512, 520, 1024, 1032, 2048, 2056, 4096, 4104, 8192, 8200, 12288, 12296, 16384, 16392, 9, 65,
                                257, 511, 516])
 def test_shape_boundaries_bf16(ctx, n):
     m = max(40, min(60_001, 24_000_000 // n)) + 3
@@ -247,7 +247,7 @@ def test_argument_checks(ctx):
     assert L.lr_loss_grad_bf16(ctx._h, None, P(y), 16, 8, P(w), P(b), P(out), P(out[1:]), P(out[9:]), None) == api.LR_ERR_NULL
     assert L.lr_loss_grad_bf16(ctx._h, ctypes.c_void_p(Xh.data_ptr() + 1), P(y), 16, 8, P(w), P(b), P(out), P(out[1:]),
                                P(out[9:]), None) == api.LR_ERR_ALIGNMENT
-    assert L.lr_fit_bf16(ctx._h, P(Xh), P(y), 16, 9000, 0.1, 1, P(w), P(b), None, None) == api.LR_ERR_SHAPE
+    assert L.lr_fit_bf16(ctx._h, P(Xh), P(y), 16, 16408, 0.1, 1, P(w), P(b), None, None) == api.LR_ERR_SHAPE
     assert L.lr_predict_bf16(ctx._h, P(Xh), 16, 8, P(w), P(b), 1.5, P(out), None) == api.LR_ERR_VALUE
     assert L.lr_convert_bf16(ctx._h, P(out), -1, P(Xh), None) == api.LR_ERR_SHAPE
 

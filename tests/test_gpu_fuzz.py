@@ -30,6 +30,9 @@ def _shapes():
         m = int(g.integers(1, max(2, min(budget, 60_000))))
         iters = int(g.integers(2, 9))
         out.append((m, n, iters, 7000 + k))
+    for k in range(36, 40):                                     # rows beyond 8192 columns: CTA-wide stages, one row per batch
+        n = int(g.integers(8193, 16385))
+        out.append((int(g.integers(1, 500)), n, int(g.integers(2, 6)), 7000 + k))
     return out
 
 
@@ -37,7 +40,7 @@ def _shapes():
 def ctx():
     from paper_2308_10037_b200 import build
     build.build()
-    c = api.Context(n_max=8192, device=0)
+    c = api.Context(n_max=16384, device=0)
     yield c
     assert c.device_status() == 0
     c.close()

@@ -23,7 +23,7 @@ from _parity import (GRAD_TOL, LABEL_AGREE, LOSS_TOL, W_TOL, allowed_drift, asse
 def ctx():
     from paper_2308_10037_b200 import build
     build.build()
-    c = api.Context(n_max=8200, device=0)
+    c = api.Context(n_max=16400, device=0)
     yield c
     assert c.device_status() == 0
     c.close()
@@ -44,9 +44,9 @@ def check_loss_grad(ctx, X, y, w, b, grad_tol=GRAD_TOL, loss_tol=LOSS_TOL):
 
 
 # shapes: every staged instantiation (n/4 <= 8, 16, 32, 64, 128), partly filled lane groups (28, 100, 200, 36),
-# rows of any length (n % 4 != 0, n <= 512), the unstaged kernel (n % 4 != 0 and n > 512, n > 4096), and row counts that
+# rows of any length (n % 4 != 0, n <= 512), CTA-wide stages (n % 4 != 0 and n > 512, every n > 8192), the unstaged kernel (n > 16384), and row counts that
 # are tiny, ragged, or span many tiles
-SHAPES = [(777, 515), (301, 1001), (301, 1027), (200, 2050), (3_001, 8192), (1_001, 5000), (777, 6148), (20, 8196), (1, 4), (7, 4), (8, 3), (33, 28), (1000, 32), (4097, 32), (5003, 64), (2500, 36), (3001, 100), (9999, 256),
+SHAPES = [(777, 515), (301, 1001), (301, 1027), (200, 2050), (3_001, 8192), (1_001, 5000), (777, 6148), (20, 8196), (301, 8193), (203, 12288), (150, 12291), (97, 16384), (40, 16385), (20, 16388), (1, 4), (7, 4), (8, 3), (33, 28), (1000, 32), (4097, 32), (5003, 64), (2500, 36), (3001, 100), (9999, 256),
           (777, 200), (1500, 512), (2049, 260), (640, 30), (1025, 101), (300, 1), (130, 4096), (50, 8192), (20011, 8),
           # enough rows that every warp refills its shared-memory stages many times, with a ragged last batch
           (200_003, 256), (400_001, 32), (200_002, 64), (120_007, 100), (150_001, 28), (60_001, 512), (90_001, 200),
@@ -63,7 +63,7 @@ def test_loss_grad_matches_oracle(ctx, m, n):
 # both sides of every boundary between kernel shapes (lanes per row, groups per lane, warps per CTA, rows per batch,
 # narrow / split / unstaged), for a row count that gives every warp several batches with a ragged last one
 BOUNDARY_N = [4, 8, 12, 32, 36, 64, 68, 128, 132, 256, 260, 384, 388, 512, 516, 1024, 1028, 1536, 1540, 2048, 2052, 3072, 3076,
-              4096, 4100, 6144, 6148, 8192, 8196, 9, 17, 33, 65, 129, 257, 513, 1025, 8191]
+              4096, 4100, 6144, 6148, 8192, 8196, 12288, 12292, 16384, 16388, 9, 17, 33, 65, 129, 257, 513, 1025, 8191, 8193, 16383, 16385]
 
 
 @pytest.mark.parametrize("n", BOUNDARY_N)
@@ -194,7 +194,7 @@ def test_fit_is_deterministic_and_resumable(ctx):
 
 
 @pytest.mark.parametrize("m,n", [(5003, 64), (9999, 256), (3001, 100), (640, 30), (130, 4096), (33, 28), (4001, 1028),
-                                 (50, 8192)])
+                                 (50, 8192), (301, 8193), (97, 16384), (20, 16388)])
 def test_predict_matches_oracle(ctx, m, n):
     X, y, w, b = datagen.random_problem(m, n, seed=50 + n, wscale=2.0)
     dX, dw, db = dev(X), dev(w), dev(np.array([b], dtype=np.float32))
