@@ -134,9 +134,9 @@ int make_plan(int64_t m, int32_t n, bool aligned16, int32_t sms, lr_plan* P, boo
     const bool split_weak = !bf16 && n / epg > 1024 && n / epg <= 1536;
     if (aligned16 && n % epg == 0 && n / epg <= kNW * (bf16 ? 64 : 128) && !split_weak && m < (int64_t(1) << 31) - 65536) {   // TMA coordinates are int32
         // wide rows: the warps of a CTA split each row by columns
-        // bfloat16 rows of up to 384 groups (1032..3072 columns) are split across eight warps instead of sixteen: wider
+        // bfloat16 rows of up to 512 groups (1032..4096 columns) are split across eight warps instead of sixteen: wider
         // slices, and 255 registers per thread, which batches of 16 (one group per lane) or 8 rows (two groups) need
-        const int nw = (bf16 && n / epg <= 384) ? 8 : kNW;
+        const int nw = (bf16 && n / epg <= 512) ? 8 : kNW;
         const int cw = (n / epg + nw - 1) / nw;                                 // 16-byte column groups per warp slice
         const int nv = cw > 64 ? 4 : (cw > 32 ? 2 : 1);            // fp32 rows of 4100..8192 columns: four groups per lane, two rows
         // Rows per batch.  All warps of a CTA meet once per batch, so a batch must carry enough bytes to cover that

@@ -295,7 +295,7 @@ def test_every_row_length_gets_a_launchable_plan():
                     assert 1 <= p["stages"] <= 4 and p["smem_bytes"] == 4096 + p["stages"] * stage
                 elif v == 1:
                     nw = p["threads"] // 32
-                    assert aligned and n % epg == 0 and nw == (8 if bf16 and n // epg <= 384 else 16)
+                    assert aligned and n % epg == 0 and nw == (8 if bf16 and n // epg <= 512 else 16)
                     assert bf16 or not (4096 < n <= 6144)
                     cw = -(-(n // epg) // nw)
                     assert p["vec_per_lane"] * 32 >= cw and p["vec_per_lane"] in (1, 2, 4)
