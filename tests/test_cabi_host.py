@@ -101,7 +101,7 @@ def test_plan_for_unaligned_or_odd_shapes():
     assert n513["rows_per_batch"] == 16 and n513["threads"] == 256 and n513["vec_per_lane"] == 3
 
 
-@pytest.mark.parametrize("n,lpr,nv,rb", [(1, 8, 1, 8), (7, 8, 1, 8), (13, 16, 1, 8), (30, 32, 1, 16), (33, 32, 2, 16), (101, 32, 4, 8),
+@pytest.mark.parametrize("n,lpr,nv,rb", [(1, 8, 1, 8), (7, 8, 1, 8), (13, 16, 1, 16), (30, 32, 1, 32), (33, 32, 2, 16), (101, 32, 4, 8),
                                          (255, 32, 8, 4), (258, 32, 16, 2), (511, 32, 16, 2)])
 def test_plan_rows_of_any_length(n, lpr, nv, rb):
     # fp32 rows whose length is not a multiple of four still take a staged kernel: a lane owns single elements
