@@ -55,8 +55,12 @@ bool row_shape_for(int ng, bool bf16, RowShape* s) {
     else if (ng <= 32) *s = {1, 32, 8};
     else if (ng <= 64 && !bf16) *s = {2, 32, 4};
     else if (ng <= 64 && bf16) *s = {2, 32, 8, 8};          // 264..512 bfloat16 columns: eight warps, eight rows (no spills)
-    else if (ng <= 128 && !bf16) *s = {4, 32, 4, 8};        // 260..512 fp32 columns: eight warps, four rows (4..8 KB batches)
-    else if (ng <= 128 && bf16) *s = {4, 32, 2, 8};         // 520..1024 bfloat16 columns: eight warps, as below
+    else if (ng <= 96 && !bf16) *s = {3, 32, 4, 8};         // 260..384 fp32 columns: three groups per lane (with four, a quarter
+                                                            // to a half of a lane's slots would be dead work)
+    else if (ng <= 128 && !bf16) *s = {4, 32, 4, 8};        // 388..512 fp32 columns: eight warps, four rows (4..8 KB batches)
+    else if (ng <= 96 && bf16) *s = {3, 32, 2, 8};          // 520..768 bfloat16 columns
+    else if (ng <= 128 && bf16) *s = {4, 32, 2, 8};         // 776..1024 bfloat16 columns: eight warps, as below
+    else if (ng <= 192 && !bf16) *s = {6, 32, 2, 8};        // 516..768 fp32 columns
     else if (ng <= 256 && !bf16) *s = {8, 32, 2, 8};
     else return false;
     return true;
@@ -134,16 +138,16 @@ int make_plan(int64_t m, int32_t n, bool aligned16, int32_t sms, lr_plan* P, boo
     const bool split_weak = !bf16 && n / epg > 1024 && n / epg <= 1536;
     if (aligned16 && n % epg == 0 && n / epg <= kNW * (bf16 ? 64 : 128) && !split_weak && m < (int64_t(1) << 31) - 65536) {   // TMA coordinates are int32
         // wide rows: the warps of a CTA split each row by columns
-        // bfloat16 rows of up to 512 groups (1032..4096 columns) are split across eight warps instead of sixteen: wider
-        // slices, and 255 registers per thread, which batches of 16 (one group per lane) or 8 rows (two groups) need
-        const int nw = (bf16 && n / epg <= 512) ? 8 : kNW;
+        // bfloat16 rows are split across eight warps instead of sixteen: wider slices, and 255 registers per thread, which
+        // batches of 16 (one group per lane), 8 (two groups) or 4 rows (four groups: 4104..8192 columns) need
+        const int nw = bf16 ? 8 : kNW;
         const int cw = (n / epg + nw - 1) / nw;                                 // 16-byte column groups per warp slice
         const int nv = cw > 64 ? 4 : (cw > 32 ? 2 : 1);            // fp32 rows of 4100..8192 columns: four groups per lane, two rows
         // Rows per batch.  All warps of a CTA meet once per batch, so a batch must carry enough bytes to cover that
         // round trip: slices of up to 24 groups per warp take 16 rows at a time and slices of 33..48 groups 8 rows, where 8
         // and 4 left the pass latency-bound (1028 columns: 3.6 TB/s, 2052: 4.2 TB/s); wider slices would leave room for
         // one stage only.
-        const int rb = nv == 4 ? 2 : nv == 2 ? (nw == 8 || (cw <= 48 && !bf16) ? 8 : 4)  // (the 16-warp bfloat16 kernels would spill
+        const int rb = nv == 4 ? (nw == 8 ? 4 : 2) : nv == 2 ? (nw == 8 || (cw <= 48 && !bf16) ? 8 : 4)  // (the 16-warp bfloat16 kernels would spill
                                : (nw == 8 || (cw <= 24 && !bf16) ? 16 : 8);          //  registers with the larger batches)
         const int64_t B = (m + rb - 1) / rb;
         const int grid = int(std::min<int64_t>(B, sms));
@@ -357,12 +361,12 @@ cudaError_t for_row_shape(const lr_plan& P, bool bf16, F&& f) {
         }
     } else if (bf16) {
         LRGD_SHAPE(ElemBF16, 1, 8, 8, 16) LRGD_SHAPE(ElemBF16, 1, 16, 8, 16) LRGD_SHAPE(ElemBF16, 1, 32, 8, 16)
-        LRGD_SHAPE(ElemBF16, 2, 32, 8, 8) LRGD_SHAPE(ElemBF16, 4, 32, 2, 8)
+        LRGD_SHAPE(ElemBF16, 2, 32, 8, 8) LRGD_SHAPE(ElemBF16, 3, 32, 2, 8) LRGD_SHAPE(ElemBF16, 4, 32, 2, 8)
     } else {
         LRGD_SHAPE(ElemF32, 1, 2, 2, 16) LRGD_SHAPE(ElemF32, 1, 4, 4, 16)
         LRGD_SHAPE(ElemF32, 1, 8, 8, 16) LRGD_SHAPE(ElemF32, 1, 16, 8, 16) LRGD_SHAPE(ElemF32, 1, 32, 16, 8)
-        LRGD_SHAPE(ElemF32, 2, 32, 4, 16) LRGD_SHAPE(ElemF32, 4, 32, 4, 8)
-        LRGD_SHAPE(ElemF32, 8, 32, 2, 8)
+        LRGD_SHAPE(ElemF32, 2, 32, 4, 16) LRGD_SHAPE(ElemF32, 3, 32, 4, 8) LRGD_SHAPE(ElemF32, 4, 32, 4, 8)
+        LRGD_SHAPE(ElemF32, 6, 32, 2, 8) LRGD_SHAPE(ElemF32, 8, 32, 2, 8)
     }
 #undef LRGD_SHAPE
     return cudaErrorInvalidValue;
@@ -384,7 +388,7 @@ cudaError_t launch_rows(const lr_plan& P, const StreamParams& sp, cudaStream_t s
 // The copy moves bytes untouched, and a box may span at most 256 elements per dimension, so a bfloat16 matrix is
 // described as 32-bit words (n/2 per row): the widest slice, 64 groups, is then 256 elements for either storage type.
 // The encoder is a driver entry point, resolved at run time so that the library links against the runtime only.
-bool split_words64(bool bf16, int cw) { return !bf16 && cw > 64; }
+bool split_words64(bool /*bf16*/, int cw) { return cw > 64; }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
                                   const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
@@ -434,10 +438,11 @@ cudaError_t launch_split(const lr_plan& P, const void* X, const SplitParams& sp,
     cudaError_t e = make_x_tensor_map(X, bf16, sp.m, sp.n, sp.cw, P.rows_per_batch, &tm);
     if (e != cudaSuccess) return e;
     if (bf16) {
-        if (P.threads == 256 && P.vec_per_lane == 2) return launch_split_t<ElemBF16, 2, 8, PRED, 8>(P, tm, sp, st, dependent);
-        if (P.threads == 256) return launch_split_t<ElemBF16, 1, 16, PRED, 8>(P, tm, sp, st, dependent);    // eight warps per CTA
-        if (P.vec_per_lane == 2) return launch_split_t<ElemBF16, 2, 4, PRED>(P, tm, sp, st, dependent);
-        return launch_split_t<ElemBF16, 1, 8, PRED>(P, tm, sp, st, dependent);
+        // eight warps per CTA for every bfloat16 shape: 16, 8 or 4 rows per batch with one, two or four groups per lane
+        if (P.threads != 256) return cudaErrorInvalidValue;
+        if (P.vec_per_lane == 4) return launch_split_t<ElemBF16, 4, 4, PRED, 8>(P, tm, sp, st, dependent);
+        if (P.vec_per_lane == 2) return launch_split_t<ElemBF16, 2, 8, PRED, 8>(P, tm, sp, st, dependent);
+        return launch_split_t<ElemBF16, 1, 16, PRED, 8>(P, tm, sp, st, dependent);
     }
     if (P.vec_per_lane == 4) return launch_split_t<ElemF32, 4, 2, PRED>(P, tm, sp, st, dependent);
     if (P.vec_per_lane == 2 && P.rows_per_batch == 8) return launch_split_t<ElemF32, 2, 8, PRED>(P, tm, sp, st, dependent);
