@@ -506,8 +506,20 @@ def main():
         pe1.record()
         torch.cuda.synchronize()
         p_ms = pe0.elapsed_time(pe1) / 10
-        f1, tp, fp, fn = f1_score(labels.cpu().numpy(), y_np)
+        # the confusion counts on the device (lr_f1_counts), timed; the host count over the downloaded labels must agree
+        f1, tp, fp, fn = ctx.f1_counts(labels, dy)
+        ce0, ce1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        counts = torch.empty(3, dtype=torch.int64, device="cuda")
+        ce0.record()
+        for _ in range(10):
+            ctx.f1_counts_async(labels, dy, counts)
+        ce1.record()
+        torch.cuda.synchronize()
+        c_ms = ce0.elapsed_time(ce1) / 10
+        if (f1, tp, fp, fn) != f1_score(labels.cpu().numpy(), y_np):
+            raise SystemExit("device confusion counts differ from the host count")
         predict = {"thr": wl.predict_thr, "f1_vs_y": f1, "tp": tp, "fp": fp, "fn": fn, "ms_per_predict": p_ms,
+                   "ms_per_f1_counts": c_ms, "f1_counts_gbs": 5 * wl.m / (c_ms * 1e-3) / 1e9,
                    "gbs": (elem_bytes * wl.m * wl.n + wl.m) / (p_ms * 1e-3) / 1e9, "after_iterations": wl.iters}
 
     # ---- CPU checker on this host's cores (reported baseline, not a target) ----

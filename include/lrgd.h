@@ -221,6 +221,20 @@ int lr_predict(lr_ctx* ctx, const float* d_X, int64_t m, int32_t n,
                const float* d_w, const float* d_b, float thr, uint8_t* d_labels, void* stream);
 
 /*
+ * Confusion counts behind the f1 score that the paper reports beside every timing (Section IV, Tables I and II; it
+ * does not spell the score out, so the usual definition is used).  With "predicted positive" = d_labels[i] != 0 and
+ * "positive" = d_y[i] > 0.5:
+ *   d_counts[0] = tp = predicted positive and positive,  d_counts[1] = fp = predicted positive and not positive,
+ *   d_counts[2] = fn = not predicted positive and positive;   f1 = 2 tp / (2 tp + fp + fn), 0 when tp == 0
+ * (the quotient is left to the caller: three integers are exact, a device-side double would add nothing).
+ * d_labels is a DEVICE array uint8 [m] (lr_predict's output), d_y DEVICE fp32 [m], d_counts DEVICE int64 [3], 8-byte
+ * aligned, overwritten (zeroed on the stream, then added to by one kernel; integer sums, so the result does not depend
+ * on the order).  m == 0 gives three zeros.  Fastest with d_labels and d_y 16-byte aligned.  Errors: LR_ERR_NULL,
+ * LR_ERR_SHAPE (m < 0 or beyond 2^40), LR_ERR_ALIGNMENT (d_y not 4-byte, d_counts not 8-byte aligned), LR_ERR_CUDA.
+ */
+int lr_f1_counts(lr_ctx* ctx, const uint8_t* d_labels, const float* d_y, int64_t m, int64_t* d_counts, void* stream);
+
+/*
  * bfloat16 storage of X (not in the paper, which is silent on storage precision; it halves the bytes the pass has to
  * stream).  d_Xh is a DEVICE array of m*n bfloat16 patterns (uint16: the upper half of a binary32 pattern), row-major
  * with leading dimension n, 2-byte aligned.  Only X changes: y, w, b, the gradient and every sum stay as in the fp32

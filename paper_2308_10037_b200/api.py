@@ -25,7 +25,7 @@ EXPORTS = ["lr_plan_query", "lr_create", "lr_destroy", "lr_loss_grad", "lr_fit",
            "lr_convert_bf16", "lr_loss_grad_bf16", "lr_fit_bf16", "lr_predict_bf16", "lr_plan_query_bf16",
            "lr_fit_tol_bf16", "lr_fit_opt_bf16", "lr_fit_sgd_bf16", "lr_shard_sums_bf16", "lr_set_overlap",
            "lr_fit_host_bf16", "lr_predict_host_bf16", "lr_exchange_bytes", "lr_fit_sharded", "lr_fit_sharded_bf16", "lr_fit_sharded_local", "lr_set_sm_limit",
-           "lr_set_cluster", "lr_cluster_ctas"]
+           "lr_set_cluster", "lr_cluster_ctas", "lr_f1_counts"]
 
 
 class LrPlan(ctypes.Structure):
@@ -65,6 +65,7 @@ def lib() -> ctypes.CDLL:
         L.lr_fit.argtypes = [P, P, P, I64, I32, F, I32, P, P, P, P]
         L.lr_predict.argtypes = [P, P, I64, I32, P, P, F, P, P]
         L.lr_shard_sums.argtypes = [P, P, P, I64, I32, P, P, P, P]
+        L.lr_f1_counts.argtypes = [P, P, P, I64, P, P]
         L.lr_convert_bf16.argtypes = [P, P, I64, P, P]
         L.lr_loss_grad_bf16.argtypes = L.lr_loss_grad.argtypes
         L.lr_fit_bf16.argtypes = L.lr_fit.argtypes
@@ -301,6 +302,25 @@ class Context:
                                                 self._p(labels, torch.uint8, "labels", m), self._stream())
         self._check(rc, "lr_predict" + sfx)
         return labels
+
+    def f1_counts_async(self, labels, y, counts):
+        """Enqueues the confusion counts of uint8 ``labels`` against 0/1 targets ``y`` into ``counts`` (int64 CUDA tensor
+        [3]: tp, fp, fn) without reading them back."""
+        if not isinstance(labels, torch.Tensor) or labels.dim() != 1:
+            raise ValueError("labels: expected a 1-D uint8 CUDA tensor")
+        m = labels.numel()
+        rc = lib().lr_f1_counts(self._h, self._p(labels, torch.uint8, "labels", m) if m else None,
+                                self._p(y, torch.float32, "y", m) if m else None, m,
+                                self._p(counts, torch.int64, "counts", 3), self._stream())
+        self._check(rc, "lr_f1_counts")
+
+    def f1_counts(self, labels, y):
+        """``(f1, tp, fp, fn)`` of uint8 ``labels`` against 0/1 targets ``y``, counted on the device; f1 = 2tp / (2tp + fp
+        + fn), 0 when tp == 0.  Reads the three counters back, so it waits for the stream."""
+        counts = torch.empty(3, dtype=torch.int64, device=labels.device if isinstance(labels, torch.Tensor) else None)
+        self.f1_counts_async(labels, y, counts)
+        tp, fp, fn = (int(v) for v in counts.tolist())
+        return (2.0 * tp / (2.0 * tp + fp + fn) if tp > 0 else 0.0), tp, fp, fn
 
     def shard_sums(self, X, y, w, b, sums):
         """Unnormalised fp64 sums [n+2] of the local rows into ``sums`` (float64 CUDA tensor)."""

@@ -19,6 +19,7 @@
 #include "lrgd_fit_rows.cuh"
 #include "lrgd_generic.cuh"
 #include "lrgd_reduce.cuh"
+#include "lrgd_score.cuh"
 #include "lrgd_stream_rows.cuh"
 #include "lrgd_stream_split.cuh"
 #include "lrgd_stream_wide.cuh"
@@ -913,6 +914,25 @@ int lr_predict(lr_ctx* ctx, const float* d_X, int64_t m, int32_t n, const float*
 int lr_predict_bf16(lr_ctx* ctx, const uint16_t* d_Xh, int64_t m, int32_t n, const float* d_w, const float* d_b, float thr,
                     uint8_t* d_labels, void* stream) {
     return predict_impl(ctx, d_Xh, true, m, n, d_w, d_b, thr, d_labels, stream);
+}
+
+int lr_f1_counts(lr_ctx* ctx, const uint8_t* d_labels, const float* d_y, int64_t m, int64_t* d_counts, void* stream) {
+    if (!ctx) return LR_ERR_NULL;
+    if (m < 0 || m > kMaxRows) return LR_ERR_SHAPE;
+    if (!d_counts || (m > 0 && (!d_labels || !d_y))) return LR_ERR_NULL;
+    if (!aligned(d_counts, 8) || (m > 0 && !aligned(d_y, 4))) return LR_ERR_ALIGNMENT;
+    DeviceGuard g(ctx);
+    if (!g.ok) return LR_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    LR_CK(ctx, cudaMemsetAsync(d_counts, 0, 3 * sizeof(int64_t), st));
+    if (m == 0) return LR_OK;
+    const bool vec = aligned(d_labels, 16) && aligned(d_y, 16);
+    const int64_t units = vec ? (m + 15) / 16 : m;
+    const int grid = int(std::max<int64_t>(1, std::min<int64_t>((units + kScoreThreads - 1) / kScoreThreads, int64_t(ctx->sm_count) * 8)));
+    k_confusion<<<grid, kScoreThreads, 0, st>>>(d_labels, d_y, m, reinterpret_cast<unsigned long long*>(d_counts), vec ? 1 : 0);
+    LR_CK(ctx, cudaGetLastError());
+    ctx->launches += 1;
+    return LR_OK;
 }
 
 int lr_convert_bf16(lr_ctx* ctx, const float* d_X, int64_t count, uint16_t* d_Xh, void* stream) {

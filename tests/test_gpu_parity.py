@@ -207,6 +207,48 @@ def test_predict_matches_oracle(ctx, m, n):
         assert (got == ref).mean() >= LABEL_AGREE or m < 10_000 and (got != ref).sum() <= 1
 
 
+# confusion counts behind the f1 score: integers, so the device must agree with the checker exactly.  Sizes span the
+# vector path (16 rows per thread step), its scalar tail, several CTAs, views that are not 16-byte aligned, and the
+# degenerate cases (no row, nothing predicted, everything predicted, no positive target)
+@pytest.mark.parametrize("m,shift", [(0, 0), (1, 0), (15, 0), (16, 0), (17, 0), (4099, 0), (1_000_003, 0), (70_001, 1), (70_001, 3),
+                                     (5_000_000, 0)])
+def test_f1_counts_match_oracle(ctx, m, shift):
+    g = np.random.Generator(np.random.Philox(key=np.array([77, m + shift], dtype=np.uint64)))
+    y = (g.random(m) < 0.3).astype(np.float32)
+    for kind in ("random", "none", "all", "no_positive_target"):
+        labels = {"random": (g.random(m) < 0.4), "none": np.zeros(m, bool), "all": np.ones(m, bool),
+                  "no_positive_target": (g.random(m) < 0.4)}[kind].astype(np.uint8)
+        if kind == "random" and m > 3:
+            labels[::7] *= 200                           # any non-zero byte counts as a predicted positive
+        yy = np.zeros(m, np.float32) if kind == "no_positive_target" else y
+        lab_buf = torch.zeros(m + 16, dtype=torch.uint8, device="cuda")
+        y_buf = torch.full((m + 16,), float("nan"), dtype=torch.float32, device="cuda")
+        lab_buf[shift:shift + m] = torch.from_numpy(labels).cuda()
+        y_buf[shift:shift + m] = torch.from_numpy(yy).cuda()
+        got = ctx.f1_counts(lab_buf[shift:shift + m], y_buf[shift:shift + m])
+        ref = oracle.f1_score(labels, yy)
+        assert got[1:] == ref[1:], (kind, got, ref)
+        assert got[0] == ref[0]                          # the same quotient of the same integers
+    if m == 0:
+        assert got == (0.0, 0, 0, 0)
+
+
+def test_f1_counts_argument_checks(ctx):
+    import ctypes
+    L = api.lib()
+    P = lambda t: ctypes.c_void_p(t.data_ptr())
+    lab = torch.zeros(32, dtype=torch.uint8, device="cuda"); y = torch.zeros(32, device="cuda")
+    cnt = torch.zeros(4, dtype=torch.int64, device="cuda")
+    assert L.lr_f1_counts(ctx._h, None, P(y), 32, P(cnt), None) == api.LR_ERR_NULL
+    assert L.lr_f1_counts(ctx._h, P(lab), P(y), 32, None, None) == api.LR_ERR_NULL
+    assert L.lr_f1_counts(ctx._h, P(lab), P(y), -1, P(cnt), None) == api.LR_ERR_SHAPE
+    assert L.lr_f1_counts(ctx._h, P(lab), ctypes.c_void_p(y.data_ptr() + 2), 8, P(cnt), None) == api.LR_ERR_ALIGNMENT
+    assert L.lr_f1_counts(ctx._h, P(lab), P(y), 8, ctypes.c_void_p(cnt.data_ptr() + 4), None) == api.LR_ERR_ALIGNMENT
+    assert L.lr_f1_counts(ctx._h, None, None, 0, P(cnt), None) == api.LR_OK     # no rows: the pointers are not looked at
+    torch.cuda.synchronize()
+    assert cnt[:3].tolist() == [0, 0, 0]
+
+
 # fp32 rows whose length is not a multiple of four (a lane owns single elements): every instantiation (n <= 8, 16, 32, 64,
 # 128, 256, 512), batches that do not start on a 16-byte boundary (two-row batches of odd-length rows), ragged tails whose
 # byte count is not a multiple of 16, stage reuse
