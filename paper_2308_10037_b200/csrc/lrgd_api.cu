@@ -70,7 +70,9 @@ bool row_shape_for(int ng, bool bf16, RowShape* s) {
 // Narrow rows whose length is not a whole number of 16-byte groups, or whose matrix is not 16-byte aligned: a lane owns
 // single elements (nv of them per row).
 bool any_row_shape_for(int n, RowShape* s) {
-    if (n <= 8) *s = {1, 8, 8};
+    if (n <= 2) *s = {1, 2, 2};                             // one or two columns: two lanes per row (32 rows per batch either way)
+    else if (n <= 4) *s = {1, 4, 4};
+    else if (n <= 8) *s = {1, 8, 8};
     else if (n <= 16) *s = {1, 16, 16};
     else if (n <= 32) *s = {1, 32, 32};
     else if (n <= 64) *s = {2, 32, 16};
@@ -352,10 +354,12 @@ cudaError_t for_row_shape(const lr_plan& P, bool bf16, F&& f) {
 #define LRGD_SHAPE(E, a, b, c, d) if (is(a, b, c, d)) return f(RowKernelShape<E, a, b, c, d>{});
     if (P.variant == 3) {                          // rows of any length: a lane owns single elements
         if (bf16) {
+            LRGD_SHAPE(ElemBF16Any, 1, 2, 2, 16) LRGD_SHAPE(ElemBF16Any, 1, 4, 4, 16)
             LRGD_SHAPE(ElemBF16Any, 1, 8, 8, 16) LRGD_SHAPE(ElemBF16Any, 1, 16, 16, 16) LRGD_SHAPE(ElemBF16Any, 1, 32, 32, 16)
             LRGD_SHAPE(ElemBF16Any, 2, 32, 16, 16) LRGD_SHAPE(ElemBF16Any, 4, 32, 8, 16) LRGD_SHAPE(ElemBF16Any, 8, 32, 4, 16)
             LRGD_SHAPE(ElemBF16Any, 16, 32, 2, 16)
         } else {
+            LRGD_SHAPE(ElemF32Any, 1, 2, 2, 16) LRGD_SHAPE(ElemF32Any, 1, 4, 4, 16)
             LRGD_SHAPE(ElemF32Any, 1, 8, 8, 16) LRGD_SHAPE(ElemF32Any, 1, 16, 16, 16) LRGD_SHAPE(ElemF32Any, 1, 32, 32, 16)
             LRGD_SHAPE(ElemF32Any, 2, 32, 16, 16) LRGD_SHAPE(ElemF32Any, 4, 32, 8, 16) LRGD_SHAPE(ElemF32Any, 8, 32, 4, 16)
             LRGD_SHAPE(ElemF32Any, 16, 32, 2, 16)

@@ -101,7 +101,7 @@ def test_plan_for_unaligned_or_odd_shapes():
     assert n513["rows_per_batch"] == 16 and n513["threads"] == 256 and n513["vec_per_lane"] == 3
 
 
-@pytest.mark.parametrize("n,lpr,nv,rb", [(1, 8, 1, 8), (7, 8, 1, 8), (13, 16, 1, 16), (30, 32, 1, 32), (33, 32, 2, 16), (101, 32, 4, 8),
+@pytest.mark.parametrize("n,lpr,nv,rb", [(1, 2, 1, 2), (3, 4, 1, 4), (7, 8, 1, 8), (13, 16, 1, 16), (30, 32, 1, 32), (33, 32, 2, 16), (101, 32, 4, 8),
                                          (255, 32, 8, 4), (258, 32, 16, 2), (511, 32, 16, 2)])
 def test_plan_rows_of_any_length(n, lpr, nv, rb):
     # fp32 rows whose length is not a multiple of four still take a staged kernel: a lane owns single elements
@@ -271,7 +271,7 @@ def test_every_row_length_gets_a_launchable_plan():
                     assert nw in (8, 16) and 1 <= p["stages"] <= 4
                     lanes = p["lanes_per_row"]
                     groups = n if v == 3 else n // epg
-                    assert lanes in ((2, 4, 8, 16, 32) if v == 0 and not bf16 else (8, 16, 32))
+                    assert lanes in ((2, 4, 8, 16, 32) if (v == 0 and not bf16) or v == 3 else (8, 16, 32))
                     assert p["vec_per_lane"] * lanes >= groups and (lanes >= 8 or groups <= lanes)
                     assert p["rows_per_batch"] % (32 // lanes) == 0
                     stage = -(-(p["rows_per_batch"] * n * eb + (16 if v == 3 else 0)) // 128) * 128

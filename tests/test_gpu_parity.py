@@ -207,6 +207,19 @@ def test_predict_matches_oracle(ctx, m, n):
         assert (got == ref).mean() >= LABEL_AGREE or m < 10_000 and (got != ref).sum() <= 1
 
 
+def test_every_narrow_row_length(ctx):
+    """Every row length from 1 to 72 columns (grouped and element-wise lane shapes, all their boundaries), on a row count that
+    leaves a ragged last batch: loss, gradient and labels against the checker."""
+    for n in range(1, 73):
+        m = 4001 + 13 * n
+        X, y, w, b = datagen.random_problem(m, n, seed=8800 + n, wscale=1.0)
+        check_loss_grad(ctx, X, y, w, b)
+        ref, z = oracle.predict(X, w, b, 0.5, return_z=True)
+        got = ctx.predict(dev(X), dev(w), dev(np.array([b], dtype=np.float32)), 0.5).cpu().numpy()
+        clear = np.abs(z) > 1e-4 * (1 + np.abs(z))
+        assert np.array_equal(got[clear], ref[clear]), n
+
+
 # confusion counts behind the f1 score: integers, so the device must agree with the checker exactly.  Sizes span the
 # vector path (16 rows per thread step), its scalar tail, several CTAs, views that are not 16-byte aligned, and the
 # degenerate cases (no row, nothing predicted, everything predicted, no positive target)
