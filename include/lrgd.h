@@ -378,6 +378,16 @@ int lr_launch_count(lr_ctx* ctx, int64_t* out);
 int lr_last_device_status(lr_ctx* ctx, int32_t* out);
 
 /*
+ * Bounds check of the library's own device workspaces (no counterpart in the paper).  Every array that the kernels index
+ * by a computed offset -- the per-CTA partial rows, the gradient buffer of the stopping rule, the context's velocity and
+ * the optimiser scratch -- is allocated between two 256-byte guard regions filled with a fixed pattern when the context
+ * is created.  lr_check_guards synchronises the device, reads the guard regions back and returns in *corrupted how many of
+ * them (0..8) no longer hold the pattern: anything but 0 means a kernel wrote outside its array.  It changes nothing, so it
+ * can be called at any point between calls; the tests call it after every batch of shapes.
+ */
+int lr_check_guards(lr_ctx* ctx, int32_t* corrupted);
+
+/*
  * Exercises the give-up path of the bounded device-side waits without harming the device: enqueues a one-warp
  * kernel that waits on an mbarrier which is completed up front (arm != 0) or never (arm == 0), for at most limit_ms
  * (1..1000) milliseconds.  When the wait runs out the kernel sets the device status word, exactly as a streaming kernel

@@ -25,7 +25,7 @@ EXPORTS = ["lr_plan_query", "lr_create", "lr_destroy", "lr_loss_grad", "lr_fit",
            "lr_convert_bf16", "lr_loss_grad_bf16", "lr_fit_bf16", "lr_predict_bf16", "lr_plan_query_bf16",
            "lr_fit_tol_bf16", "lr_fit_opt_bf16", "lr_fit_sgd_bf16", "lr_shard_sums_bf16", "lr_set_overlap",
            "lr_fit_host_bf16", "lr_predict_host_bf16", "lr_exchange_bytes", "lr_fit_sharded", "lr_fit_sharded_bf16", "lr_fit_sharded_local", "lr_set_sm_limit",
-           "lr_set_cluster", "lr_cluster_ctas", "lr_f1_counts"]
+           "lr_set_cluster", "lr_cluster_ctas", "lr_f1_counts", "lr_check_guards"]
 
 
 class LrPlan(ctypes.Structure):
@@ -66,6 +66,7 @@ def lib() -> ctypes.CDLL:
         L.lr_predict.argtypes = [P, P, I64, I32, P, P, F, P, P]
         L.lr_shard_sums.argtypes = [P, P, P, I64, I32, P, P, P, P]
         L.lr_f1_counts.argtypes = [P, P, P, I64, P, P]
+        L.lr_check_guards.argtypes = [P, ctypes.POINTER(I32)]
         L.lr_convert_bf16.argtypes = [P, P, I64, P, P]
         L.lr_loss_grad_bf16.argtypes = L.lr_loss_grad.argtypes
         L.lr_fit_bf16.argtypes = L.lr_fit.argtypes
@@ -434,6 +435,13 @@ class Context:
         n, ms = ctypes.c_int32(), ctypes.c_double()
         self._check(lib().lr_profile_read(self._h, ctypes.byref(n), ctypes.byref(ms)), "lr_profile_read")
         return n.value, ms.value
+
+    def check_guards(self) -> int:
+        """Number of guard regions around the context's device workspaces that no longer hold their pattern (0 = no kernel
+        wrote outside its array).  Waits for the device."""
+        v = ctypes.c_int32()
+        self._check(lib().lr_check_guards(self._h, ctypes.byref(v)), "lr_check_guards")
+        return v.value
 
     def launch_count(self) -> int:
         v = ctypes.c_int64()

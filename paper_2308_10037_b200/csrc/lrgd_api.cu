@@ -258,9 +258,32 @@ struct lr_ctx {
     int prof_used = 0;
     int64_t launches = 0;
     int last_cuda = 0;
+    // guard regions: every device workspace that kernels index by a computed offset sits between two of them
+    std::vector<unsigned char*> guard_bases;        // allocation bases; the user range starts kGuardBytes in
+    std::vector<size_t> guard_sizes;                // user bytes, rounded up to kGuardBytes
 };
 
 namespace {
+
+// Guard regions around the context's device workspaces (per-CTA partial rows, gradient buffer, velocity, optimiser scratch):
+// kGuardBytes of a fixed pattern before and after each, written once at creation.  No kernel of the library has any
+// business there, so a changed byte (lr_check_guards) means an index ran out of its array.
+constexpr size_t kGuardBytes = 256;
+constexpr int kGuardPattern = 0xA5;
+
+template <class T>
+cudaError_t guarded_alloc(lr_ctx* c, T** user, size_t bytes) {
+    const size_t body = (bytes + kGuardBytes - 1) / kGuardBytes * kGuardBytes;
+    unsigned char* base = nullptr;
+    cudaError_t e = cudaMalloc(reinterpret_cast<void**>(&base), body + 2 * kGuardBytes);
+    if (e != cudaSuccess) return e;
+    c->guard_bases.push_back(base);
+    c->guard_sizes.push_back(body);
+    e = cudaMemset(base, kGuardPattern, kGuardBytes);
+    if (e == cudaSuccess) e = cudaMemset(base + kGuardBytes + body, kGuardPattern, kGuardBytes);
+    *user = reinterpret_cast<T*>(base + kGuardBytes);
+    return e;
+}
 
 // A named range around a whole library call, visible on a profiler's timeline (costs nothing when no tool is attached).
 struct NvtxRange {
@@ -815,18 +838,18 @@ int lr_create(lr_ctx** out, int32_t device, int32_t n_max) {
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, device);
     if (e == cudaSuccess) {
         const size_t bytes = size_t(c->sm_count) * kMaxGridPerSm * (size_t(n_max) + 2) * sizeof(double);
-        e = cudaMalloc(reinterpret_cast<void**>(&c->d_partial), bytes);
+        e = guarded_alloc(c, &c->d_partial, bytes);
         if (e == cudaErrorMemoryAllocation) rc = LR_ERR_NOMEM;
     }
     if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&c->d_status), sizeof(int));
     if (e == cudaSuccess) e = cudaMemset(c->d_status, 0, sizeof(int));
     if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&c->d_tol), sizeof(TolState));
     if (e == cudaSuccess) e = cudaMemset(c->d_tol, 0, sizeof(TolState));
-    if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&c->d_gbuf), (size_t(n_max) + 1) * sizeof(double));
+    if (e == cudaSuccess) e = guarded_alloc(c, &c->d_gbuf, (size_t(n_max) + 1) * sizeof(double));
     if (e == cudaSuccess) e = cudaMallocHost(reinterpret_cast<void**>(&c->h_tol), sizeof(TolState));
     if (e == cudaSuccess) e = cudaMallocHost(reinterpret_cast<void**>(&c->h_words), 4 * sizeof(int));
-    if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&c->d_vel), (size_t(n_max) + 1) * sizeof(float));
-    if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&c->d_oscr), (size_t(n_max) + 2) * sizeof(double));
+    if (e == cudaSuccess) e = guarded_alloc(c, &c->d_vel, (size_t(n_max) + 1) * sizeof(float));
+    if (e == cudaSuccess) e = guarded_alloc(c, &c->d_oscr, (size_t(n_max) + 2) * sizeof(double));
     if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&c->d_oticket), sizeof(unsigned int));
     if (e == cudaSuccess) e = cudaMemset(c->d_oticket, 0, sizeof(unsigned int));
     if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&c->d_gbar), 2 * kMaxWorld * sizeof(unsigned int));
@@ -844,14 +867,11 @@ int lr_create(lr_ctx** out, int32_t device, int32_t n_max) {
     if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&c->hstream, cudaStreamNonBlocking);
     if (prev >= 0) cudaSetDevice(prev);
     if (e != cudaSuccess) {
-        if (c->d_partial) cudaFree(c->d_partial);
+        for (unsigned char* base : c->guard_bases) cudaFree(base);     // d_partial, d_gbuf, d_vel, d_oscr
         if (c->d_status) cudaFree(c->d_status);
         if (c->d_tol) cudaFree(c->d_tol);
-        if (c->d_gbuf) cudaFree(c->d_gbuf);
         if (c->h_tol) cudaFreeHost(c->h_tol);
         if (c->h_words) cudaFreeHost(c->h_words);
-        if (c->d_vel) cudaFree(c->d_vel);
-        if (c->d_oscr) cudaFree(c->d_oscr);
         if (c->d_oticket) cudaFree(c->d_oticket);
         if (c->d_gbar) cudaFree(c->d_gbar);
         if (c->d_rank_params) cudaFree(c->d_rank_params);
@@ -869,14 +889,11 @@ int lr_destroy(lr_ctx* ctx) {
         cudaDeviceSynchronize();
         for (cudaEvent_t e : ctx->ev) cudaEventDestroy(e);
         if (ctx->hstream) cudaStreamDestroy(ctx->hstream);
-        cudaFree(ctx->d_partial);
+        for (unsigned char* base : ctx->guard_bases) cudaFree(base);   // d_partial, d_gbuf, d_vel, d_oscr
         cudaFree(ctx->d_status);
         cudaFree(ctx->d_tol);
-        cudaFree(ctx->d_gbuf);
         if (ctx->h_tol) cudaFreeHost(ctx->h_tol);
         if (ctx->h_words) cudaFreeHost(ctx->h_words);
-        cudaFree(ctx->d_vel);
-        cudaFree(ctx->d_oscr);
         cudaFree(ctx->d_oticket);
         cudaFree(ctx->d_gbar);
         cudaFree(ctx->d_rank_params);
@@ -1436,6 +1453,26 @@ int lr_last_device_status(lr_ctx* ctx, int32_t* out) {
     LR_CK(ctx, cudaMemcpy(&v, ctx->d_status, sizeof(int), cudaMemcpyDeviceToHost));
     LR_CK(ctx, cudaMemset(ctx->d_status, 0, sizeof(int)));
     *out = v;
+    return LR_OK;
+}
+
+int lr_check_guards(lr_ctx* ctx, int32_t* corrupted) {
+    if (!ctx || !corrupted) return LR_ERR_NULL;
+    DeviceGuard g(ctx);
+    if (!g.ok) return LR_ERR_CUDA;
+    LR_CK(ctx, cudaDeviceSynchronize());
+    int bad = 0;
+    unsigned char host[kGuardBytes];
+    for (size_t i = 0; i < ctx->guard_bases.size(); ++i) {
+        for (int side = 0; side < 2; ++side) {
+            const unsigned char* src = ctx->guard_bases[i] + (side ? kGuardBytes + ctx->guard_sizes[i] : 0);
+            LR_CK(ctx, cudaMemcpy(host, src, kGuardBytes, cudaMemcpyDeviceToHost));
+            bool clean = true;
+            for (size_t k = 0; k < kGuardBytes; ++k) clean = clean && host[k] == static_cast<unsigned char>(kGuardPattern);
+            if (!clean) ++bad;
+        }
+    }
+    *corrupted = bad;
     return LR_OK;
 }
 

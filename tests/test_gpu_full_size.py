@@ -30,6 +30,7 @@ def ctx():
     c = api.Context(n_max=4096, device=0)
     yield c
     assert c.device_status() == 0
+    assert c.check_guards() == 0                   # no kernel of the module wrote outside a workspace array
     c.close()
 
 

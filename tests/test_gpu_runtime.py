@@ -128,3 +128,27 @@ def test_c_example_program_runs():
         out = subprocess.run([exe], capture_output=True, text=True, timeout=120)
         assert out.returncode == 0, out.stdout + out.stderr
         assert "device status 0" in out.stdout
+
+
+def test_guard_regions_stay_clean_at_the_context_limit(ctx):
+    """Every workspace array sits between two guard regions; runs at the widest row the context allows (n = n_max), in every
+    fit form that uses a workspace (partial rows, gradient buffer, context-owned velocity, optimiser scratch), must leave all
+    eight regions untouched.  A clean context reports 0 to begin with."""
+    fresh = api.Context(n_max=512, device=0)
+    assert fresh.check_guards() == 0
+    fresh.close()
+    for m, n in [(30_011, 512), (2_001, 511), (150_001, 28), (9, 512)]:
+        X, y, w, b = datagen.random_problem(m, n, seed=31 + n)
+        dX, dy = torch.from_numpy(X).cuda(), torch.from_numpy(y).cuda()
+        zeros = lambda: (torch.zeros(n, device="cuda"), torch.zeros(1, device="cuda"))
+        ctx.loss_grad(dX, dy, torch.from_numpy(w).cuda(), torch.tensor([b], device="cuda"))
+        for persistent in (None, True, False):
+            ctx.set_persistent(persistent)
+            ctx.fit(dX, dy, 0.05, 4, *zeros())
+            ctx.fit_tol(dX, dy, 0.05, 1e-9, 5, *zeros(), check_every=2)
+            ctx.fit_opt(dX, dy, 0.05, 4, *zeros(), l2=1e-3, momentum=0.9, nesterov=True)
+        ctx.set_persistent(None)
+        ctx.fit_sgd(dX, dy, 0.05, max(1, m // 3), 5, *zeros())
+        ctx.predict(dX, torch.from_numpy(w).cuda(), torch.tensor([b], device="cuda"), 0.5)
+    assert ctx.device_status() == 0
+    assert ctx.check_guards() == 0
