@@ -48,8 +48,8 @@ struct RowShape { int nv, lpr, rb; int nw = kNW; };    // nw = warps per CTA
 // bfloat16 rows of 33..128 groups (a thread holds its 32 columns of a row slice, their weights and accumulators).  The
 // bytes in flight per SM stay the same.
 bool row_shape_for(int ng, bool bf16, RowShape* s) {
-    if (ng <= 2 && !bf16) *s = {1, 2, 2};                     // 4 or 8 fp32 columns: two lanes per row, no idle lanes
-    else if (ng <= 4 && !bf16) *s = {1, 4, 4};               // 12 or 16
+    if (ng <= 2) *s = {1, 2, 2};                              // 4 or 8 fp32 (8 or 16 bfloat16) columns: two lanes per row
+    else if (ng <= 4) *s = {1, 4, 4};                        // 12 or 16 (24 or 32)
     else if (ng <= 8) *s = {1, 8, 8};
     else if (ng <= 16) *s = {1, 16, 8};
     else if (ng <= 32 && !bf16) *s = {1, 32, 16, 8};        // 68..128 fp32 columns: eight warps, sixteen rows
@@ -388,6 +388,7 @@ cudaError_t for_row_shape(const lr_plan& P, bool bf16, F&& f) {
             LRGD_SHAPE(ElemF32Any, 16, 32, 2, 16)
         }
     } else if (bf16) {
+        LRGD_SHAPE(ElemBF16, 1, 2, 2, 16) LRGD_SHAPE(ElemBF16, 1, 4, 4, 16)
         LRGD_SHAPE(ElemBF16, 1, 8, 8, 16) LRGD_SHAPE(ElemBF16, 1, 16, 8, 16) LRGD_SHAPE(ElemBF16, 1, 32, 8, 16)
         LRGD_SHAPE(ElemBF16, 2, 32, 8, 8) LRGD_SHAPE(ElemBF16, 3, 32, 2, 8) LRGD_SHAPE(ElemBF16, 4, 32, 2, 8)
     } else {

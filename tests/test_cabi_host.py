@@ -271,7 +271,7 @@ def test_every_row_length_gets_a_launchable_plan():
                     assert nw in (8, 16) and 1 <= p["stages"] <= 4
                     lanes = p["lanes_per_row"]
                     groups = n if v == 3 else n // epg
-                    assert lanes in ((2, 4, 8, 16, 32) if (v == 0 and not bf16) or v == 3 else (8, 16, 32))
+                    assert lanes in (2, 4, 8, 16, 32)
                     assert p["vec_per_lane"] * lanes >= groups and (lanes >= 8 or groups <= lanes)
                     assert p["rows_per_batch"] % (32 // lanes) == 0
                     stage = -(-(p["rows_per_batch"] * n * eb + (16 if v == 3 else 0)) // 128) * 128
