@@ -207,12 +207,15 @@ int make_plan(int64_t m, int32_t n, bool aligned16, int32_t sms, lr_plan* P, boo
         if (per_cta >= (int64_t(1) << 31)) return LR_ERR_SHAPE;
         return LR_OK;
     }
-    const int64_t nchunks = (m + kGenRows - 1) / kGenRows;
+    // rows per chunk: 64, halved down to 8 while the chunks would not give every SM a few CTAs
+    int gen_rows = kGenRows;
+    while (gen_rows > 8 && (m + gen_rows - 1) / gen_rows < int64_t(sms) * kMaxGridPerSm) gen_rows /= 2;
+    const int64_t nchunks = (m + gen_rows - 1) / gen_rows;
     P->variant = 2;
     P->lanes_per_row = 32;
     P->vec_per_lane = 0;
     P->rows_per_batch = 1;
-    P->tile_rows = kGenRows;
+    P->tile_rows = gen_rows;
     P->stages = 0;
     P->grid = int(std::min<int64_t>(nchunks, int64_t(sms) * kMaxGridPerSm));
     P->threads = kGenThreads;
@@ -755,7 +758,7 @@ int launch_stream_pass(lr_ctx* ctx, const lr_plan& P, const Pass& a, uint8_t* la
     } else {
         GenericParams gp{};
         gp.X = a.X; gp.y = a.y; gp.m = a.m; gp.n = a.n; gp.w = a.w; gp.b = a.b;
-        gp.partial = ctx->d_partial; gp.labels = labels; gp.cut = cut; gp.stop = a.stop;
+        gp.partial = ctx->d_partial; gp.labels = labels; gp.cut = cut; gp.stop = a.stop; gp.rows = P.tile_rows;
         const dim3 g(P.grid), t(P.threads);
         if (a.bf16) e = predict ? launch_kernel(k_generic<ElemBF16, true>, g, t, 0, st, dep, gp)
                                 : launch_kernel(k_generic<ElemBF16, false>, g, t, 0, st, dep, gp);

@@ -1,7 +1,8 @@
 // Unstaged kernel for the rows the staged kernels do not take: more than 16384 elements.  E is the storage type of X.
 // Plain coalesced loads; X is read from HBM once and a second time through the cache hierarchy.
 //
-// A CTA walks chunks of kGenRows rows (chunk c belongs to CTA c mod grid).  Phase 1: one warp per row
+// A CTA walks chunks of `rows` (8..kGenRows) rows (chunk c belongs to CTA c mod grid; the host picks the chunk so that
+// the grid fills the GPU: with 64-row chunks of 64 KB rows a 512 MB matrix gave 128 CTAs work and ran at 0.5 TB/s).  Phase 1: one warp per row
 // forms z = x.w + b (model equation, Section II-A), then err and the loss term (Eq. 1, Algorithm 7,
 // log-likelihood), and parks err in shared memory.  Phase 2: thread t owns columns t, t+T, ...; it sums
 // x[r][c]*err[r] over the chunk's rows in fp32 and adds the result to the CTA's own fp64 partial row
@@ -26,6 +27,7 @@ struct GenericParams {
     unsigned char* labels;    // predict mode
     float cut;
     const int* stop;          // nullable: non-zero makes the launch a no-op
+    int rows;                 // rows per chunk (a multiple of 8, at most kGenRows)
 };
 
 template <class E, bool PREDICT>
@@ -44,10 +46,11 @@ __global__ void __launch_bounds__(kGenThreads) k_generic(const GenericParams p) 
         for (int c = threadIdx.x; c < n + 2; c += kGenThreads) out[c] = 0.0;
     }
     double dse = 0.0, dsl = 0.0;                   // lane 0 of each warp
-    const long long nchunks = (p.m + kGenRows - 1) / kGenRows;
+    const int R = p.rows;
+    const long long nchunks = (p.m + R - 1) / R;
     for (long long chunk = blockIdx.x; chunk < nchunks; chunk += gridDim.x) {
-        const long long row0 = chunk * kGenRows;
-        const int rows = static_cast<int>(p.m - row0 < kGenRows ? p.m - row0 : kGenRows);
+        const long long row0 = chunk * R;
+        const int rows = static_cast<int>(p.m - row0 < R ? p.m - row0 : R);
         for (int r = warp; r < rows; r += NWARP) {
             const long long xr = (row0 + r) * n;
             float d = 0.f;

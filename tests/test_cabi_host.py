@@ -93,7 +93,9 @@ def test_plan_for_unaligned_or_odd_shapes():
     assert api.plan_query(1000, 30, bf16=True)["variant"] == 3   # element-wise staged kernel, bfloat16 too
     assert api.plan_query(1000, 1036, bf16=True)["variant"] == 4 # 1036 % 8 != 0 and wider than 1024
     g = api.plan_query(100, 16389)
-    assert g["variant"] == 2 and g["grid"] == 2 and g["threads"] == 256
+    assert g["variant"] == 2 and g["tile_rows"] == 8 and g["grid"] == 13 and g["threads"] == 256   # few rows: 8-row chunks
+    g = api.plan_query(200_000, 16389)
+    assert g["tile_rows"] == 64 and g["grid"] == 148 * 8                 # enough rows for 64-row chunks on every SM
     w = api.plan_query(100_000, 1027)
     assert w["vec_per_lane"] == 3 and w["rows_per_batch"] == 16 and w["stages"] == 3 and w["threads"] == 512
     assert api.plan_query(100_000, 8191)["rows_per_batch"] == 2
