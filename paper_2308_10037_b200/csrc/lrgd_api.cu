@@ -61,7 +61,9 @@ bool row_shape_for(int ng, bool bf16, RowShape* s) {
     else if (ng <= 128 && !bf16) *s = {4, 32, 4, 8};        // 388..512 fp32 columns: eight warps, four rows (4..8 KB batches)
     else if (ng <= 96 && bf16) *s = {3, 32, 2, 8};          // 520..768 bfloat16 columns
     else if (ng <= 128 && bf16) *s = {4, 32, 2, 8};         // 776..1024 bfloat16 columns: eight warps, as below
-    else if (ng <= 192 && !bf16) *s = {6, 32, 2, 8};        // 516..768 fp32 columns
+    else if (ng <= 160 && !bf16) *s = {5, 32, 2, 8};        // 516..640 fp32 columns: no more groups per lane than the row needs
+    else if (ng <= 192 && !bf16) *s = {6, 32, 2, 8};        // 644..768
+    else if (ng <= 224 && !bf16) *s = {7, 32, 2, 8};        // 772..896
     else if (ng <= 256 && !bf16) *s = {8, 32, 2, 8};
     else return false;
     return true;
@@ -398,7 +400,7 @@ cudaError_t for_row_shape(const lr_plan& P, bool bf16, F&& f) {
         LRGD_SHAPE(ElemF32, 1, 2, 2, 16) LRGD_SHAPE(ElemF32, 1, 4, 4, 16)
         LRGD_SHAPE(ElemF32, 1, 8, 8, 16) LRGD_SHAPE(ElemF32, 1, 16, 8, 16) LRGD_SHAPE(ElemF32, 1, 32, 16, 8)
         LRGD_SHAPE(ElemF32, 2, 32, 4, 16) LRGD_SHAPE(ElemF32, 3, 32, 4, 8) LRGD_SHAPE(ElemF32, 4, 32, 4, 8)
-        LRGD_SHAPE(ElemF32, 6, 32, 2, 8) LRGD_SHAPE(ElemF32, 8, 32, 2, 8)
+        LRGD_SHAPE(ElemF32, 5, 32, 2, 8) LRGD_SHAPE(ElemF32, 6, 32, 2, 8) LRGD_SHAPE(ElemF32, 7, 32, 2, 8) LRGD_SHAPE(ElemF32, 8, 32, 2, 8)
     }
 #undef LRGD_SHAPE
     return cudaErrorInvalidValue;

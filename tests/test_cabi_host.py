@@ -119,7 +119,7 @@ def test_plan_rows_of_516_to_1024_columns_use_eight_warps():
     for m, n in [(5000, 516), (5000, 1024), (200_000, 1000)]:
         p = api.plan_query(m, n)
         assert p["variant"] == 0 and p["threads"] == 256 and p["rows_per_batch"] == 2
-        assert p["vec_per_lane"] == (6 if n <= 768 else 8)            # 129..192 groups: six per lane, no more than needed
+        assert p["vec_per_lane"] == -(-(n // 4) // 32)                # 129..256 groups: five to eight per lane, no more than needed
         stage = -(-2 * n * 4 // 128) * 128
         assert 1024 + 8 * p["stages"] * stage <= p["smem_bytes"] <= 227 * 1024
         assert p["smem_bytes"] >= 1024 + 8 * n * 8 + 2 * 8 * 8         # room for the end-of-kernel combine of eight warps
