@@ -54,6 +54,7 @@ bool row_shape_for(int ng, bool bf16, RowShape* s) {
     else if (ng <= 16) *s = {1, 16, 8};
     else if (ng <= 32 && !bf16) *s = {1, 32, 16, 8};        // 68..128 fp32 columns: eight warps, sixteen rows
     else if (ng <= 32) *s = {1, 32, 8};
+    else if (ng <= 48 && !bf16) *s = {3, 16, 2};            // 132..192 fp32 columns: sixteen lanes per row, three groups each
     else if (ng <= 64 && !bf16) *s = {2, 32, 4};
     else if (ng <= 64 && bf16) *s = {2, 32, 8, 8};          // 264..512 bfloat16 columns: eight warps, eight rows (no spills)
     else if (ng <= 96 && !bf16) *s = {3, 32, 4, 8};         // 260..384 fp32 columns: three groups per lane (with four, a quarter
@@ -399,7 +400,7 @@ cudaError_t for_row_shape(const lr_plan& P, bool bf16, F&& f) {
     } else {
         LRGD_SHAPE(ElemF32, 1, 2, 2, 16) LRGD_SHAPE(ElemF32, 1, 4, 4, 16)
         LRGD_SHAPE(ElemF32, 1, 8, 8, 16) LRGD_SHAPE(ElemF32, 1, 16, 8, 16) LRGD_SHAPE(ElemF32, 1, 32, 16, 8)
-        LRGD_SHAPE(ElemF32, 2, 32, 4, 16) LRGD_SHAPE(ElemF32, 3, 32, 4, 8) LRGD_SHAPE(ElemF32, 4, 32, 4, 8)
+        LRGD_SHAPE(ElemF32, 3, 16, 2, 16) LRGD_SHAPE(ElemF32, 2, 32, 4, 16) LRGD_SHAPE(ElemF32, 3, 32, 4, 8) LRGD_SHAPE(ElemF32, 4, 32, 4, 8)
         LRGD_SHAPE(ElemF32, 5, 32, 2, 8) LRGD_SHAPE(ElemF32, 6, 32, 2, 8) LRGD_SHAPE(ElemF32, 7, 32, 2, 8) LRGD_SHAPE(ElemF32, 8, 32, 2, 8)
     }
 #undef LRGD_SHAPE
